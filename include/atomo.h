@@ -1,0 +1,172 @@
+/*
+ * atomo.h -- C ABI of the B200 (sm_100a) ATOMO gradient encode / decode library.
+ *
+ * ATOMO ("atomic sparsification") writes a gradient as g = sum_i lambda_i a_i over unit-norm
+ * atoms a_i, keeps atom i with probability p_i and rescales it by 1/p_i, so that the sparse
+ * estimator  g_hat = sum_i (lambda_i t_i / p_i) a_i,  t_i ~ Bernoulli(p_i)  (Eq. 2) is unbiased;
+ * the p_i minimise its variance under the budget  sum_i p_i = s  (Eq. 3, Algorithm 1).
+ * Two decompositions are provided (Section 5): entry-wise (atoms e_i, lambda_i = g_i) and
+ * spectral (atoms u_i v_i^T, lambda_i = sigma_i, from the SVD of the layer gradient seen as a
+ * matrix).
+ *
+ * Conventions
+ *   - Every pointer marked DEVICE is a CUDA device pointer owned by the caller; arrays of
+ *     descriptors (atomo_mat, atomo_vec, pointer lists, shape lists) are HOST memory and are
+ *     consumed before the call returns.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     Encode calls wait on the host for the eigen-solver's convergence flag once per sweep, so
+ *     they are not capturable in a CUDA graph; decode calls never synchronise.
+ *   - Matrices are fp32 row-major with leading dimension `ld` (elements, ld >= cols).
+ *   - Functions return an atomo_status.  Problems visible on the host (NULL, bad sizes,
+ *     s <= 0 or not finite, payload capacity too small) return at once and launch nothing.
+ *     Problems only the device can see (more kept atoms than k_cap, NaN/Inf input, sweep cap
+ *     hit) set the layer's status word in the payload header, leave that layer with k = 0
+ *     (or, for ATOMO_ERR_NOT_CONVERGED, with its best result) and are read back with
+ *     atomo_payload_status().  Nothing is ever silently truncated: dropping kept atoms would
+ *     bias the estimator of Eq. (2).
+ *   - Randomness is counter based (Philox4x32-10): the output is a pure function of the
+ *     inputs, s, seed, step and the position of the layer in the call.  Key = (seed low 32,
+ *     seed high 32); counter = (i>>2 low, i>>2 high, layer, (kind<<31)|(step & 0x7fffffff)),
+ *     atom i takes word i&3; kind 0 = spectral (i = rank in descending sigma), 1 = entry-wise
+ *     (i = flat element index).  Atom i is kept iff p_i >= 1 or word < floor(p_i * 2^32).
+ *
+ * Payload (DEVICE buffer, caller owned, self-describing; all offsets in bytes from its start,
+ * 16-byte aligned):
+ *   atomo_payload_header, then n_layers x atomo_layer_header, then per layer
+ *     entry-wise: idx  u32[k_cap] ascending flat indices, val f32[k_cap] = g_i / p_i
+ *     spectral  : idx  u32[k_cap] ascending ranks, coef f32[k_cap] = sigma_i / p_i,
+ *                 short f32[k_cap][r]  unit vectors of the short side (length r = min(rows,cols)),
+ *                 long  f32[k_cap][L]  unit vectors of the long side  (length L = max(rows,cols));
+ *                 for rows <= cols the short vectors are the u_i and the long ones the v_i,
+ *                 otherwise the other way round.
+ *   Only the first k entries of each array are meaningful (k is in the layer header).
+ */
+#ifndef ATOMO_H_
+#define ATOMO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct atomo_ctx atomo_ctx; /* opaque; owns workspace, events and the status mirror */
+
+typedef enum {
+  ATOMO_OK = 0,
+  ATOMO_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, ld < cols, too many atoms      */
+  ATOMO_ERR_BUDGET = 2,        /* s <= 0, NaN or Inf                                               */
+  ATOMO_ERR_CAPACITY = 3,      /* host: payload buffer too small; device: kept atoms > k_cap       */
+  ATOMO_ERR_NONFINITE = 4,     /* NaN or Inf found in a gradient                                   */
+  ATOMO_ERR_NOT_CONVERGED = 5, /* eigen-solver hit its sweep cap (result still orthogonal, usable) */
+  ATOMO_ERR_TIMEOUT = 6,       /* reserved for bounded device-side waits                           */
+  ATOMO_ERR_CUDA = 7,          /* a CUDA runtime call failed; see atomo_last_cuda_error            */
+  ATOMO_ERR_PAYLOAD = 8        /* decode: header does not match the shapes given                   */
+} atomo_status;
+
+enum { ATOMO_KIND_SPECTRAL = 0, ATOMO_KIND_ENTRYWISE = 1 };
+enum { ATOMO_MAGIC = 0x4F4D5441 /* "ATMO" */, ATOMO_VERSION = 1 };
+
+typedef struct { const float* data; /* DEVICE */ int32_t rows, cols; int64_t ld; } atomo_mat;
+typedef struct { const float* data; /* DEVICE */ int64_t n; } atomo_vec;
+
+/* Payload headers as they sit in DEVICE memory (also what atomo_payload_read_headers copies). */
+typedef struct {
+  uint32_t magic, version, kind, n_layers;
+  uint64_t total_bytes;
+  uint64_t seed, step;
+  double   s;
+  uint64_t reserved[2];
+} atomo_payload_header;                       /* 64 bytes */
+
+typedef struct {
+  int64_t  rows, cols;        /* entry-wise: rows = 1, cols = n                                  */
+  uint32_t k_cap, k;          /* capacity and number of kept atoms                               */
+  uint32_t n_sat;             /* atoms with p = 1                                                */
+  uint32_t status;            /* atomo_status seen by the device for this layer                  */
+  float    c;                 /* common weight |lambda_i|/p_i of the kept atoms with p < 1       */
+  uint32_t sweeps;            /* spectral: Jacobi sweeps used                                    */
+  uint64_t off_idx, off_val;  /* val = entry-wise values / spectral coefficients                 */
+  uint64_t off_short, off_long;
+  double   l1;                /* sum |lambda| over all atoms (||g||_1 or the nuclear norm)       */
+} atomo_layer_header;                         /* 80 bytes */
+
+/* Optional per-atom outputs for parity checks (DEVICE; any pointer may be NULL).
+ * Layer l's atoms start at element offset sum_{j<l} n_atoms_j in sigma/prob (n_atoms = r for
+ * spectral, n for entry-wise) and at word offset sum_{j<l} ceil(n_atoms_j/32) in mask_words
+ * (bit i&31 of word i>>5 = t_i).  sigma is spectral only (descending).  short_vecs is spectral
+ * only: all r short-side singular vectors, rank-major (r x r per layer, offset sum r_j^2).  */
+typedef struct { float* sigma; float* prob; uint32_t* mask_words; float* short_vecs; } atomo_debug;
+
+/* Stage timers (milliseconds of device time, CUDA events on the call's stream) filled while
+ * profiling is on.  `launches[i]` counts the kernels of stage i in the last call.             */
+enum { ATOMO_STAGE_GRAM = 0, ATOMO_STAGE_EIG, ATOMO_STAGE_SAMPLE, ATOMO_STAGE_BACKPROJECT,
+       ATOMO_STAGE_EW_REDUCE, ATOMO_STAGE_EW_PACK, ATOMO_STAGE_DECODE, ATOMO_N_STAGES };
+
+/* --- lifetime ------------------------------------------------------------------------------
+ * atomo_create binds the context to CUDA device `device` (made current for each call).
+ * Workspace is allocated on first use and grown when a larger batch arrives (cudaMalloc, which
+ * synchronises the device); a context serves one call at a time.                               */
+int atomo_create(atomo_ctx** out, int device);
+int atomo_destroy(atomo_ctx* ctx);
+const char* atomo_last_cuda_error(atomo_ctx* ctx);   /* text of the last failing CUDA call       */
+
+/* --- sizes (host only, no CUDA call) --------------------------------------------------------
+ * Bytes a payload needs for these shapes when every layer may keep up to k_cap atoms
+ * (k_cap is clamped to the layer's atom count).  Returns -1 on bad arguments.
+ * Since k = sum of independent Bernoulli(p_i) with sum p_i <= s, a k_cap of about
+ * s + 8 sqrt(s) + 8 is never exceeded in practice; k_cap = #atoms can never overflow.          */
+int64_t atomo_payload_bytes_spectral(const int32_t* rows, const int32_t* cols, int32_t n_layers,
+                                     int32_t k_cap);
+int64_t atomo_payload_bytes_entrywise(const int64_t* n, int32_t n_vecs, int64_t k_cap);
+
+/* --- encode ---------------------------------------------------------------------------------
+ * Spectral ATOMO (Section 5; Eq. 2, Eq. 3 / Algorithm 1) over a batch of layer gradients.
+ * Per layer: thin SVD (Gram matrix of the short side -> Jacobi eigen-solver -> sigma and the
+ * short-side vectors), probabilities from the descending sigma, Bernoulli draws, and for the
+ * kept atoms the long-side vector by back-projection (G^T u_i or G v_i, normalised; its norm
+ * is the sigma_i used in coef = sigma_i / p_i).  Each layer needs min(rows, cols) <= 4096.     */
+int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers /*HOST array*/, int32_t n_layers,
+                          double s, uint64_t seed, uint64_t step, int32_t k_cap,
+                          void* payload /*DEVICE*/, int64_t capacity_bytes,
+                          const atomo_debug* dbg /*HOST struct or NULL*/, void* stream);
+
+/* Entry-wise ATOMO (Section 3; the QSGD / TernGrad family of Section 4) over a batch of flat
+ * gradients, each with n < 2^32 elements and its own budget s (same s for every vector).       */
+int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/, int32_t n_vecs,
+                           double s, uint64_t seed, uint64_t step, int64_t k_cap,
+                           void* payload /*DEVICE*/, int64_t capacity_bytes,
+                           const atomo_debug* dbg, void* stream);
+
+/* --- decode (Eq. 2 summed back to a dense gradient) ----------------------------------------
+ * out[l] (DEVICE, fp32) receives layer l: rows[l] x cols[l] row-major with leading dimension
+ * cols[l] (entry-wise: rows[l] = 1).  `kind` and the shapes must match the payload's header;
+ * a mismatch sets ATOMO_ERR_PAYLOAD in that layer's status word and writes zeros.
+ * Never synchronises; every element of every output is written.                                */
+int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload /*DEVICE*/,
+                 const int64_t* rows, const int64_t* cols, float* const* out /*HOST array of DEVICE ptrs*/,
+                 int32_t n_layers, void* stream);
+
+/* --- status / introspection -----------------------------------------------------------------
+ * Copies the payload header and the n_layers layer headers to HOST memory (synchronises
+ * `stream`).  Either output may be NULL.                                                       */
+int atomo_payload_read_headers(atomo_ctx* ctx, const void* payload /*DEVICE*/, int32_t n_layers,
+                               atomo_payload_header* hdr /*HOST*/, atomo_layer_header* layers /*HOST*/,
+                               void* stream);
+/* Worst device-side status over the layers of a payload and the first layer that has it.       */
+int atomo_payload_status(atomo_ctx* ctx, const void* payload /*DEVICE*/, int32_t n_layers,
+                         int32_t* worst /*HOST*/, int32_t* first_bad_layer /*HOST*/, void* stream);
+
+/* --- profiling ------------------------------------------------------------------------------ */
+int atomo_set_profiling(atomo_ctx* ctx, int enabled);
+/* ms[ATOMO_N_STAGES], launches[ATOMO_N_STAGES] for the last encode/decode call (synchronises). */
+int atomo_get_stage_times(atomo_ctx* ctx, float* ms /*HOST*/, int64_t* launches /*HOST*/);
+
+/* Eigen-solver knobs: max Jacobi sweeps (default 40) and the relative rotation threshold
+ * (default 1e-6: rows p, q are rotated while |<x_p,x_q>| > tol ||x_p|| ||x_q||).               */
+int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATOMO_H_ */

@@ -1,0 +1,357 @@
+"""Thin Python binding of the C ABI in ``include/atomo.h`` (argument marshalling only).
+
+Every step of the encode / decode path runs in the CUDA library; PyTorch is used for device
+memory and streams.  There is no CPU fallback: if the shared library is missing or no CUDA
+device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libatomo_b200.so")
+
+KIND_SPECTRAL = 0
+KIND_ENTRYWISE = 1
+STATUS_NAMES = ["OK", "INVALID_ARG", "BUDGET", "CAPACITY", "NONFINITE", "NOT_CONVERGED", "TIMEOUT", "CUDA",
+                "PAYLOAD"]
+STAGES = ["gram", "eig", "sample", "backproject", "ew_reduce", "ew_pack", "decode"]
+
+# every symbol include/atomo.h declares
+EXPORTS = [
+    "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
+    "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
+    "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
+    "atomo_set_eig_params",
+]
+
+
+class AtomoError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        name = STATUS_NAMES[code] if 0 <= code < len(STATUS_NAMES) else str(code)
+        super().__init__(f"{where}: ATOMO_ERR_{name}" + (f" ({detail})" if detail else ""))
+        self.code = code
+
+
+class _Mat(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("rows", ctypes.c_int32), ("cols", ctypes.c_int32), ("ld", ctypes.c_int64)]
+
+
+class _Vec(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("n", ctypes.c_int64)]
+
+
+class _Debug(ctypes.Structure):
+    _fields_ = [("sigma", ctypes.c_void_p), ("prob", ctypes.c_void_p), ("mask_words", ctypes.c_void_p),
+                ("short_vecs", ctypes.c_void_p)]
+
+
+class PayloadHeader(ctypes.Structure):
+    _fields_ = [("magic", ctypes.c_uint32), ("version", ctypes.c_uint32), ("kind", ctypes.c_uint32),
+                ("n_layers", ctypes.c_uint32), ("total_bytes", ctypes.c_uint64), ("seed", ctypes.c_uint64),
+                ("step", ctypes.c_uint64), ("s", ctypes.c_double), ("reserved", ctypes.c_uint64 * 2)]
+
+
+class LayerHeader(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("k_cap", ctypes.c_uint32), ("k", ctypes.c_uint32),
+                ("n_sat", ctypes.c_uint32), ("status", ctypes.c_uint32), ("c", ctypes.c_float),
+                ("sweeps", ctypes.c_uint32), ("off_idx", ctypes.c_uint64), ("off_val", ctypes.c_uint64),
+                ("off_short", ctypes.c_uint64), ("off_long", ctypes.c_uint64), ("l1", ctypes.c_double)]
+
+
+assert ctypes.sizeof(PayloadHeader) == 64 and ctypes.sizeof(LayerHeader) == 80
+
+_lib = None
+
+
+def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
+    """Load libatomo_b200.so (no CUDA call is made by loading)."""
+    global _lib
+    if _lib is not None and path == LIB_PATH:
+        return _lib
+    if not os.path.exists(path):
+        raise FileNotFoundError(
+            f"{path} not found: build it with `python -m paper_1806_04090_b200.build` (there is no CPU fallback)")
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, u64, dbl = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint64, ctypes.c_double
+    lib.atomo_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int]
+    lib.atomo_destroy.argtypes = [vp]
+    lib.atomo_last_cuda_error.argtypes = [vp]
+    lib.atomo_last_cuda_error.restype = ctypes.c_char_p
+    lib.atomo_payload_bytes_spectral.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(i32), i32, i32]
+    lib.atomo_payload_bytes_spectral.restype = i64
+    lib.atomo_payload_bytes_entrywise.argtypes = [ctypes.POINTER(i64), i32, i64]
+    lib.atomo_payload_bytes_entrywise.restype = i64
+    lib.atomo_encode_spectral.argtypes = [vp, ctypes.POINTER(_Mat), i32, dbl, u64, u64, i32, vp, i64,
+                                          ctypes.POINTER(_Debug), vp]
+    lib.atomo_encode_entrywise.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, u64, u64, i64, vp, i64,
+                                           ctypes.POINTER(_Debug), vp]
+    lib.atomo_decode.argtypes = [vp, i32, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(vp), i32, vp]
+    lib.atomo_payload_read_headers.argtypes = [vp, vp, i32, ctypes.POINTER(PayloadHeader),
+                                               ctypes.POINTER(LayerHeader), vp]
+    lib.atomo_payload_status.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
+    lib.atomo_set_profiling.argtypes = [vp, ctypes.c_int]
+    lib.atomo_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i64)]
+    lib.atomo_set_eig_params.argtypes = [vp, i32, ctypes.c_float]
+    if path == LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def payload_bytes_spectral(shapes: Sequence[Sequence[int]], k_cap: int) -> int:
+    lib = load_library()
+    n = len(shapes)
+    rows = (ctypes.c_int32 * n)(*[int(s[0]) for s in shapes])
+    cols = (ctypes.c_int32 * n)(*[int(s[1]) for s in shapes])
+    return int(lib.atomo_payload_bytes_spectral(rows, cols, n, int(k_cap)))
+
+
+def payload_bytes_entrywise(lengths: Sequence[int], k_cap: int) -> int:
+    lib = load_library()
+    n = len(lengths)
+    arr = (ctypes.c_int64 * n)(*[int(x) for x in lengths])
+    return int(lib.atomo_payload_bytes_entrywise(arr, n, int(k_cap)))
+
+
+def default_k_cap(s: float, n_atoms: int) -> int:
+    """k is a sum of independent Bernoulli draws with mean <= s: s + 8 sqrt(s) + 8 is never reached."""
+    return int(min(n_atoms, np.ceil(s + 8.0 * np.sqrt(s) + 8.0)))
+
+
+@dataclass
+class Debug:
+    """Optional per-atom outputs (device tensors) for parity checks."""
+    sigma: Optional[torch.Tensor] = None
+    prob: Optional[torch.Tensor] = None
+    mask_words: Optional[torch.Tensor] = None
+    short_vecs: Optional[torch.Tensor] = None
+    atom_offsets: List[int] = field(default_factory=list)
+    word_offsets: List[int] = field(default_factory=list)
+    sq_offsets: List[int] = field(default_factory=list)
+
+    def layer_mask(self, l: int, n_atoms: int) -> np.ndarray:
+        w0 = self.word_offsets[l]
+        words = self.mask_words[w0: w0 + (n_atoms + 31) // 32].cpu().numpy().astype(np.uint32)
+        bits = np.unpackbits(words.view(np.uint8), bitorder="little")
+        return bits[:n_atoms].astype(bool)
+
+    def layer_prob(self, l: int, n_atoms: int) -> np.ndarray:
+        a0 = self.atom_offsets[l]
+        return self.prob[a0: a0 + n_atoms].cpu().numpy()
+
+    def layer_sigma(self, l: int, n_atoms: int) -> np.ndarray:
+        a0 = self.atom_offsets[l]
+        return self.sigma[a0: a0 + n_atoms].cpu().numpy()
+
+    def layer_short(self, l: int, r: int) -> np.ndarray:
+        o = self.sq_offsets[l]
+        return self.short_vecs[o: o + r * r].cpu().numpy().reshape(r, r)
+
+
+@dataclass
+class Payload:
+    """A device payload plus the host-side facts needed to decode it."""
+    buf: torch.Tensor            # uint8, device
+    kind: int
+    shapes: List[tuple]          # (rows, cols) per layer; entry-wise: (1, n)
+    k_cap: int
+    ctx: "Atomo"
+
+    @property
+    def n_layers(self) -> int:
+        return len(self.shapes)
+
+    def headers(self):
+        return self.ctx.read_headers(self)
+
+    def layer_arrays(self, l: int, hdrs=None):
+        """Host copies of one layer's kept atoms (test / inspection helper)."""
+        _, lh = hdrs if hdrs is not None else self.headers()
+        h = lh[l]
+        k = int(h.k)
+        raw = self.buf
+
+        def view(off, count, dtype):
+            nbytes = count * 4
+            return raw[off: off + nbytes].cpu().numpy().view(dtype)
+
+        idx = view(h.off_idx, k, np.uint32).copy()
+        val = view(h.off_val, k, np.float32).copy()
+        if self.kind == KIND_ENTRYWISE:
+            return dict(k=k, idx=idx, val=val)
+        rows, cols = self.shapes[l]
+        r, L = min(rows, cols), max(rows, cols)
+        short = view(h.off_short, k * r, np.float32).reshape(k, r).copy()
+        long_ = view(h.off_long, k * L, np.float32).reshape(k, L).copy()
+        U, V = (short, long_) if rows <= cols else (long_, short)
+        return dict(k=k, idx=idx, coef=val, U=U.T.copy(), V=V.T.copy())
+
+
+class Atomo:
+    """One library context bound to a CUDA device."""
+
+    def __init__(self, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("atomo: no CUDA device available (the library has no CPU fallback)")
+        self.lib = load_library()
+        self.device = int(device)
+        torch.cuda.init()
+        h = ctypes.c_void_p()
+        rc = self.lib.atomo_create(ctypes.byref(h), self.device)
+        self._h = h
+        if rc != 0:
+            raise AtomoError(rc, "atomo_create", self._cuda_error())
+
+    def _cuda_error(self) -> str:
+        try:
+            return (self.lib.atomo_last_cuda_error(self._h) or b"").decode()
+        except Exception:  # pragma: no cover
+            return ""
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self.lib.atomo_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, where: str):
+        if rc != 0:
+            raise AtomoError(rc, where, self._cuda_error() if rc == 7 else "")
+
+    @staticmethod
+    def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> ctypes.c_void_p:
+        s = stream if stream is not None else torch.cuda.current_stream()
+        return ctypes.c_void_p(s.cuda_stream)
+
+    def _make_debug(self, n_atoms: Sequence[int], spectral: bool, want_short: bool, dev) -> Debug:
+        a_off = np.concatenate([[0], np.cumsum(n_atoms)]).astype(np.int64)
+        w_off = np.concatenate([[0], np.cumsum([(n + 31) // 32 for n in n_atoms])]).astype(np.int64)
+        sq_off = np.concatenate([[0], np.cumsum([n * n for n in n_atoms])]).astype(np.int64)
+        d = Debug(atom_offsets=a_off.tolist(), word_offsets=w_off.tolist(), sq_offsets=sq_off.tolist())
+        d.prob = torch.zeros(int(a_off[-1]), dtype=torch.float32, device=dev)
+        d.mask_words = torch.zeros(int(w_off[-1]), dtype=torch.int32, device=dev)
+        if spectral:
+            d.sigma = torch.zeros(int(a_off[-1]), dtype=torch.float32, device=dev)
+            if want_short:
+                d.short_vecs = torch.zeros(int(sq_off[-1]), dtype=torch.float32, device=dev)
+        return d
+
+    @staticmethod
+    def _debug_struct(d: Optional[Debug]):
+        if d is None:
+            return None
+        ptr = lambda t: ctypes.c_void_p(t.data_ptr()) if t is not None else None
+        return _Debug(ptr(d.sigma), ptr(d.prob), ptr(d.mask_words), ptr(d.short_vecs))
+
+    # ------------------------------------------------------------------------------------------
+    def atomo_encode_spectral(self, layers: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,
+                              k_cap: Optional[int] = None, payload: Optional[torch.Tensor] = None,
+                              debug: bool = False, debug_short: bool = False,
+                              stream: Optional[torch.cuda.Stream] = None):
+        """Spectral ATOMO over a batch of 2-D fp32 CUDA tensors.  Returns (Payload, Debug | None)."""
+        n = len(layers)
+        mats = (_Mat * n)()
+        shapes = []
+        for i, g in enumerate(layers):
+            if not (g.is_cuda and g.dtype == torch.float32 and g.dim() == 2 and g.stride(1) == 1):
+                raise ValueError("layers must be 2-D fp32 CUDA tensors with unit column stride")
+            mats[i] = _Mat(g.data_ptr(), g.shape[0], g.shape[1], g.stride(0) if g.shape[0] > 1 else g.shape[1])
+            shapes.append((int(g.shape[0]), int(g.shape[1])))
+        if k_cap is None:
+            k_cap = default_k_cap(s, max(min(r, c) for r, c in shapes))
+        nbytes = payload_bytes_spectral(shapes, k_cap)
+        if nbytes < 0:
+            raise AtomoError(1, "atomo_payload_bytes_spectral")
+        dev = layers[0].device
+        if payload is None:
+            payload = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        dbg = self._make_debug([min(r, c) for r, c in shapes], True, debug_short, dev) if (debug or debug_short) else None
+        ds = self._debug_struct(dbg)
+        rc = self.lib.atomo_encode_spectral(self._h, mats, n, float(s), int(seed), int(step), int(k_cap),
+                                            ctypes.c_void_p(payload.data_ptr()), payload.numel(),
+                                            ctypes.byref(ds) if ds is not None else None, self._stream_ptr(stream))
+        self._check(rc, "atomo_encode_spectral")
+        return Payload(payload, KIND_SPECTRAL, shapes, int(k_cap), self), dbg
+
+    def atomo_encode_entrywise(self, vecs: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,
+                               k_cap: Optional[int] = None, payload: Optional[torch.Tensor] = None,
+                               debug: bool = False, stream: Optional[torch.cuda.Stream] = None):
+        """Entry-wise ATOMO over a batch of flat fp32 CUDA tensors.  Returns (Payload, Debug | None)."""
+        n = len(vecs)
+        arr = (_Vec * n)()
+        lengths = []
+        for i, g in enumerate(vecs):
+            if not (g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()):
+                raise ValueError("vectors must be contiguous fp32 CUDA tensors")
+            arr[i] = _Vec(g.data_ptr(), g.numel())
+            lengths.append(int(g.numel()))
+        if k_cap is None:
+            k_cap = default_k_cap(s, max(lengths))
+        nbytes = payload_bytes_entrywise(lengths, k_cap)
+        if nbytes < 0:
+            raise AtomoError(1, "atomo_payload_bytes_entrywise")
+        dev = vecs[0].device
+        if payload is None:
+            payload = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        dbg = self._make_debug(lengths, False, False, dev) if debug else None
+        ds = self._debug_struct(dbg)
+        rc = self.lib.atomo_encode_entrywise(self._h, arr, n, float(s), int(seed), int(step), int(k_cap),
+                                             ctypes.c_void_p(payload.data_ptr()), payload.numel(),
+                                             ctypes.byref(ds) if ds is not None else None, self._stream_ptr(stream))
+        self._check(rc, "atomo_encode_entrywise")
+        return Payload(payload, KIND_ENTRYWISE, [(1, x) for x in lengths], int(k_cap), self), dbg
+
+    def atomo_decode(self, payload: Payload, out: Optional[Sequence[torch.Tensor]] = None,
+                     stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
+        """Dense fp32 gradients from a payload (one tensor per layer)."""
+        n = payload.n_layers
+        dev = payload.buf.device
+        if out is None:
+            out = [torch.empty(r * c, dtype=torch.float32, device=dev).view((c,) if payload.kind == KIND_ENTRYWISE else (r, c))
+                   for r, c in payload.shapes]
+        rows = (ctypes.c_int64 * n)(*[r for r, _ in payload.shapes])
+        cols = (ctypes.c_int64 * n)(*[c for _, c in payload.shapes])
+        ptrs = (ctypes.c_void_p * n)(*[o.data_ptr() for o in out])
+        rc = self.lib.atomo_decode(self._h, payload.kind, ctypes.c_void_p(payload.buf.data_ptr()), rows, cols, ptrs, n,
+                                   self._stream_ptr(stream))
+        self._check(rc, "atomo_decode")
+        return list(out)
+
+    # ------------------------------------------------------------------------------------------
+    def read_headers(self, payload: Payload, stream: Optional[torch.cuda.Stream] = None):
+        gh = PayloadHeader()
+        lh = (LayerHeader * payload.n_layers)()
+        rc = self.lib.atomo_payload_read_headers(self._h, ctypes.c_void_p(payload.buf.data_ptr()), payload.n_layers,
+                                                 ctypes.byref(gh), lh, self._stream_ptr(stream))
+        self._check(rc, "atomo_payload_read_headers")
+        return gh, list(lh)
+
+    def payload_status(self, payload: Payload, stream: Optional[torch.cuda.Stream] = None):
+        worst, first = ctypes.c_int32(0), ctypes.c_int32(-1)
+        rc = self.lib.atomo_payload_status(self._h, ctypes.c_void_p(payload.buf.data_ptr()), payload.n_layers,
+                                           ctypes.byref(worst), ctypes.byref(first), self._stream_ptr(stream))
+        self._check(rc, "atomo_payload_status")
+        return int(worst.value), int(first.value)
+
+    def set_profiling(self, on: bool):
+        self._check(self.lib.atomo_set_profiling(self._h, 1 if on else 0), "atomo_set_profiling")
+
+    def stage_times(self):
+        ms = (ctypes.c_float * len(STAGES))()
+        ln = (ctypes.c_int64 * len(STAGES))()
+        self._check(self.lib.atomo_get_stage_times(self._h, ms, ln), "atomo_get_stage_times")
+        return {k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)}
+
+    def set_eig_params(self, max_sweeps: int, tol: float):
+        self._check(self.lib.atomo_set_eig_params(self._h, int(max_sweeps), float(tol)), "atomo_set_eig_params")

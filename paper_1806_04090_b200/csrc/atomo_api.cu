@@ -1,0 +1,503 @@
+// C ABI of the library (see include/atomo.h): argument checks, payload layout, workspace
+// carving and kernel sequencing.  No arithmetic of the method lives here.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "atomo_kernels.cuh"
+
+using namespace atomo;
+
+struct atomo_ctx {
+  int device = 0;
+  uint8_t* ws = nullptr;
+  size_t ws_bytes = 0;
+  uint32_t* h_flag = nullptr;        // pinned: convergence flag / state mirror
+  EwState* h_state = nullptr;        // pinned
+  cudaEvent_t ev_sync = nullptr;
+  cudaEvent_t ev[ATOMO_N_STAGES][2] = {};
+  bool ev_used[ATOMO_N_STAGES] = {};
+  int64_t launches[ATOMO_N_STAGES] = {};
+  bool profiling = false;
+  bool configured = false;
+  int max_sweeps = 40;
+  float tol = 1e-6f;
+  std::string err;
+};
+
+namespace {
+
+struct Arena {
+  uint8_t* base; size_t off = 0;
+  explicit Arena(uint8_t* b) : base(b) {}
+  template <typename T> T* take(size_t count) {
+    off = (off + 255) & ~size_t(255);
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+int fail_cuda(atomo_ctx* ctx, cudaError_t e, const char* what) {
+  ctx->err = std::string(what) + ": " + cudaGetErrorString(e);
+  return ATOMO_ERR_CUDA;
+}
+#define CK(call)                                                            \
+  do {                                                                      \
+    cudaError_t e__ = (call);                                               \
+    if (e__ != cudaSuccess) return fail_cuda(ctx, e__, #call);              \
+  } while (0)
+
+int ensure_ws(atomo_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->ws_bytes) return ATOMO_OK;
+  if (ctx->ws) { CK(cudaDeviceSynchronize()); CK(cudaFree(ctx->ws)); ctx->ws = nullptr; ctx->ws_bytes = 0; }
+  const size_t want = bytes + bytes / 8 + (1 << 20);
+  CK(cudaMalloc(&ctx->ws, want));
+  ctx->ws_bytes = want;
+  return ATOMO_OK;
+}
+
+void stage_begin(atomo_ctx* ctx, int stage, cudaStream_t st) {
+  if (!ctx->profiling) return;
+  cudaEventRecord(ctx->ev[stage][0], st);
+  ctx->ev_used[stage] = true;
+}
+void stage_end(atomo_ctx* ctx, int stage, cudaStream_t st, int64_t n_launch) {
+  ctx->launches[stage] += n_launch;
+  if (!ctx->profiling) return;
+  cudaEventRecord(ctx->ev[stage][1], st);
+}
+void stage_reset(atomo_ctx* ctx) {
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) { ctx->ev_used[i] = false; ctx->launches[i] = 0; }
+}
+
+int next_pow2_at_least(int x, int lo) { int p = lo; while (p < x) p <<= 1; return p; }
+
+struct SpLayout {                 // payload offsets of one spectral layer
+  uint32_t kc; uint64_t off_idx, off_coef, off_short, off_long;
+};
+
+uint64_t layout_spectral(const int32_t* rows, const int32_t* cols, int n_layers, int32_t k_cap,
+                         std::vector<SpLayout>* out) {
+  uint64_t off = sizeof(atomo_payload_header) + (uint64_t)n_layers * sizeof(atomo_layer_header);
+  for (int l = 0; l < n_layers; ++l) {
+    const int64_t r = std::min(rows[l], cols[l]), L = std::max(rows[l], cols[l]);
+    const uint32_t kc = (uint32_t)std::min<int64_t>(k_cap, r);
+    SpLayout lo;
+    lo.kc = kc;
+    off = align_up(off, 16); lo.off_idx = off; off += (uint64_t)kc * 4;
+    off = align_up(off, 16); lo.off_coef = off; off += (uint64_t)kc * 4;
+    off = align_up(off, 16); lo.off_short = off; off += (uint64_t)kc * r * 4;
+    off = align_up(off, 16); lo.off_long = off; off += (uint64_t)kc * L * 4;
+    if (out) out->push_back(lo);
+  }
+  return align_up(off, 16);
+}
+
+struct EwLayout { uint32_t kc; uint64_t off_idx, off_val; };
+
+uint64_t layout_entrywise(const int64_t* n, int n_vecs, int64_t k_cap, std::vector<EwLayout>* out) {
+  uint64_t off = sizeof(atomo_payload_header) + (uint64_t)n_vecs * sizeof(atomo_layer_header);
+  for (int l = 0; l < n_vecs; ++l) {
+    const uint32_t kc = (uint32_t)std::min<int64_t>(k_cap, n[l]);
+    EwLayout lo;
+    lo.kc = kc;
+    off = align_up(off, 16); lo.off_idx = off; off += (uint64_t)kc * 4;
+    off = align_up(off, 16); lo.off_val = off; off += (uint64_t)kc * 4;
+    if (out) out->push_back(lo);
+  }
+  return align_up(off, 16);
+}
+
+bool bad_budget(double s) { return !(s > 0.0) || !std::isfinite(s); }
+
+}  // namespace
+
+extern "C" {
+
+int atomo_create(atomo_ctx** out, int device) {
+  if (!out || device < 0) return ATOMO_ERR_INVALID_ARG;
+  atomo_ctx* ctx = new atomo_ctx();
+  ctx->device = device;
+  *out = ctx;
+  CK(cudaSetDevice(device));
+  CK(cudaMallocHost(&ctx->h_flag, 256));
+  CK(cudaMallocHost(&ctx->h_state, sizeof(EwState)));
+  CK(cudaEventCreateWithFlags(&ctx->ev_sync, cudaEventDisableTiming));
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) { CK(cudaEventCreate(&ctx->ev[i][0])); CK(cudaEventCreate(&ctx->ev[i][1])); }
+  const int e = sp_configure();
+  if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaFuncSetAttribute(max dynamic shared memory)");
+  ctx->configured = true;
+  return ATOMO_OK;
+}
+
+int atomo_destroy(atomo_ctx* ctx) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaDeviceSynchronize();
+  if (ctx->ws) cudaFree(ctx->ws);
+  if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
+  if (ctx->h_state) cudaFreeHost(ctx->h_state);
+  if (ctx->ev_sync) cudaEventDestroy(ctx->ev_sync);
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) for (int j = 0; j < 2; ++j) if (ctx->ev[i][j]) cudaEventDestroy(ctx->ev[i][j]);
+  delete ctx;
+  return ATOMO_OK;
+}
+
+const char* atomo_last_cuda_error(atomo_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int64_t atomo_payload_bytes_spectral(const int32_t* rows, const int32_t* cols, int32_t n_layers, int32_t k_cap) {
+  if (!rows || !cols || n_layers <= 0 || k_cap <= 0) return -1;
+  for (int l = 0; l < n_layers; ++l) if (rows[l] <= 0 || cols[l] <= 0) return -1;
+  return (int64_t)layout_spectral(rows, cols, n_layers, k_cap, nullptr);
+}
+
+int64_t atomo_payload_bytes_entrywise(const int64_t* n, int32_t n_vecs, int64_t k_cap) {
+  if (!n || n_vecs <= 0 || k_cap <= 0) return -1;
+  for (int l = 0; l < n_vecs; ++l) if (n[l] <= 0 || n[l] >= (int64_t(1) << 32)) return -1;
+  return (int64_t)layout_entrywise(n, n_vecs, k_cap, nullptr);
+}
+
+int atomo_set_profiling(atomo_ctx* ctx, int enabled) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  ctx->profiling = enabled != 0;
+  return ATOMO_OK;
+}
+
+int atomo_get_stage_times(atomo_ctx* ctx, float* ms, int64_t* launches) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) {
+    if (launches) launches[i] = ctx->launches[i];
+    if (!ms) continue;
+    ms[i] = 0.0f;
+    if (ctx->profiling && ctx->ev_used[i]) {
+      CK(cudaEventSynchronize(ctx->ev[i][1]));
+      CK(cudaEventElapsedTime(&ms[i], ctx->ev[i][0], ctx->ev[i][1]));
+    }
+  }
+  return ATOMO_OK;
+}
+
+int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
+  if (!ctx || max_sweeps < 1 || max_sweeps > 1000 || !(tol > 0.0f) || !(tol < 1.0f)) return ATOMO_ERR_INVALID_ARG;
+  ctx->max_sweeps = max_sweeps;
+  ctx->tol = tol;
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
+int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers, double s, uint64_t seed,
+                          uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
+                          const atomo_debug* dbg, void* stream) {
+  if (!ctx || !layers || n_layers <= 0 || k_cap <= 0 || !payload) return ATOMO_ERR_INVALID_ARG;
+  if (bad_budget(s)) return ATOMO_ERR_BUDGET;
+  if ((reinterpret_cast<uintptr_t>(payload) & 15u) != 0) return ATOMO_ERR_INVALID_ARG;
+  std::vector<int32_t> rows(n_layers), cols(n_layers);
+  for (int l = 0; l < n_layers; ++l) {
+    const atomo_mat& m = layers[l];
+    if (!m.data || m.rows <= 0 || m.cols <= 0 || m.ld < m.cols) return ATOMO_ERR_INVALID_ARG;
+    if (std::min(m.rows, m.cols) > kSmemRowsMaxRp) return ATOMO_ERR_INVALID_ARG;
+    rows[l] = m.rows; cols[l] = m.cols;
+  }
+  std::vector<SpLayout> lay;
+  const uint64_t total = layout_spectral(rows.data(), cols.data(), n_layers, k_cap, &lay);
+  if ((int64_t)total > capacity_bytes) return ATOMO_ERR_CAPACITY;
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  stage_reset(ctx);
+  const int max_sweeps = ctx->max_sweeps;
+  uint8_t* pay = static_cast<uint8_t*>(payload);
+  atomo_layer_header* d_hdr = reinterpret_cast<atomo_layer_header*>(pay + sizeof(atomo_payload_header));
+
+  // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
+  std::vector<SpLayer> L(n_layers);
+  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles;
+  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    SpLayer& d = L[l];
+    const atomo_mat& m = layers[l];
+    d.G = m.data; d.rows = m.rows; d.cols = m.cols; d.ld = m.ld;
+    d.tall = m.rows > m.cols;
+    d.r = std::min(m.rows, m.cols); d.L = std::max(m.rows, m.cols);
+    d.rp = next_pow2_at_least(d.r, 32);
+    d.B = d.rp <= 512 ? 16 : 8;
+    d.nb = d.rp / d.B;
+    d.layer = (uint32_t)l; d.k_cap = lay[l].kc;
+    r_max = std::max(r_max, d.r);
+    const int gt = (d.r + 63) / 64;
+    for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
+    for (int p = 0; p < d.nb / 2; ++p) (d.B == 16 ? pairs16 : pairs8).push_back({l, p, 0, 0});
+    if (d.B == 16) { rp16_max = std::max(rp16_max, d.rp); steps16 = std::max(steps16, d.nb - 1); }
+    else steps8 = std::max(steps8, d.nb - 1);
+    d.bp_tiles = d.tall ? (d.L + sp_bp_rows_per_tile() - 1) / sp_bp_rows_per_tile()
+                        : (d.L + sp_bp_cols_per_tile() - 1) / sp_bp_cols_per_tile();
+    for (int t = 0; t < d.bp_tiles; ++t) bp_tiles.push_back({l, t, 0, 0});
+  }
+  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr;
+  uint32_t* d_flag = nullptr;
+  uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
+  size_t need = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    Arena A(pass ? ctx->ws : nullptr);
+    d_layers = A.take<SpLayer>(n_layers);
+    d_gram = A.take<TileRef>(gram_tiles.size());
+    d_p16 = A.take<TileRef>(pairs16.size());
+    d_p8 = A.take<TileRef>(pairs8.size());
+    d_bp = A.take<TileRef>(bp_tiles.size());
+    d_flag = A.take<uint32_t>(4);
+    size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      SpLayer& d = L[l];
+      d.lam = A.take<float>(d.rp);
+      d.perm = A.take<int>(d.r);
+      float* sig_ws = A.take<float>(d.r);
+      float* prob_ws = A.take<float>(d.r);
+      uint32_t* mask_ws = A.take<uint32_t>((d.r + 31) / 32);
+      d.sigma = (dbg && dbg->sigma) ? dbg->sigma + dbg_atoms : sig_ws;
+      d.prob = (dbg && dbg->prob) ? dbg->prob + dbg_atoms : prob_ws;
+      d.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
+      d.dbg_short = (dbg && dbg->short_vecs) ? dbg->short_vecs + dbg_sq : nullptr;
+      dbg_atoms += d.r; dbg_words += (d.r + 31) / 32; dbg_sq += (size_t)d.r * d.r;
+      d.p_sel = A.take<float>(d.k_cap);
+      d.bp_partials = A.take<float>((size_t)d.bp_tiles * d.k_cap);
+      d.scale = A.take<float>(1);
+      d.hdr = d_hdr + l;
+      d.idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_idx);
+      d.coef = reinterpret_cast<float*>(pay + lay[l].off_coef);
+      d.shortv = reinterpret_cast<float*>(pay + lay[l].off_short);
+      d.longv = reinterpret_cast<float*>(pay + lay[l].off_long);
+    }
+    // zero-filled region: rotation counters and the X matrices
+    uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
+    size_t z0 = A.off;
+    for (int l = 0; l < n_layers; ++l) L[l].rot_count = A.take<uint32_t>(max_sweeps);
+    for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * 2 * L[l].rp);
+    zero_beg = zb; zero_bytes = A.off - z0;
+    need = A.off + 256;
+    if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
+  }
+
+  // ---- uploads ----
+  std::vector<uint8_t> hdr_blob(sizeof(atomo_payload_header) + (size_t)n_layers * sizeof(atomo_layer_header), 0);
+  atomo_payload_header gh{};
+  gh.magic = ATOMO_MAGIC; gh.version = ATOMO_VERSION; gh.kind = ATOMO_KIND_SPECTRAL; gh.n_layers = (uint32_t)n_layers;
+  gh.total_bytes = total; gh.seed = seed; gh.step = step; gh.s = s;
+  std::memcpy(hdr_blob.data(), &gh, sizeof(gh));
+  for (int l = 0; l < n_layers; ++l) {
+    atomo_layer_header h{};
+    h.rows = rows[l]; h.cols = cols[l]; h.k_cap = lay[l].kc; h.k = 0; h.status = ATOMO_OK;
+    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_coef; h.off_short = lay[l].off_short; h.off_long = lay[l].off_long;
+    std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
+  }
+  CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(d_layers, L.data(), L.size() * sizeof(SpLayer), cudaMemcpyHostToDevice, st));
+  if (!gram_tiles.empty()) CK(cudaMemcpyAsync(d_gram, gram_tiles.data(), gram_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!pairs16.empty()) CK(cudaMemcpyAsync(d_p16, pairs16.data(), pairs16.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!pairs8.empty()) CK(cudaMemcpyAsync(d_p8, pairs8.data(), pairs8.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
+
+  // ---- S1: Gram matrix, scaling ----
+  stage_begin(ctx, ATOMO_STAGE_GRAM, st);
+  launch_sp_init(d_layers, n_layers, nullptr, 0, st);
+  launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
+  launch_sp_scale(d_layers, n_layers, st);
+  stage_end(ctx, ATOMO_STAGE_GRAM, st, 4);
+  CK(cudaGetLastError());
+
+  // ---- S1: eigen-solver; the host reads a convergence flag once per sweep of the largest layer ----
+  stage_begin(ctx, ATOMO_STAGE_EIG, st);
+  int t16 = 0, t8 = 0;
+  int64_t n_eig_launch = 0;
+  for (int it = 0; it < max_sweeps; ++it) {
+    for (int j = 0; j < steps16; ++j, ++t16, ++n_eig_launch)
+      launch_sp_jacobi_step(d_layers, d_p16, (int)pairs16.size(), 16, rp16_max, t16, max_sweeps, ctx->tol, st);
+    for (int j = 0; j < steps8; ++j, ++t8, ++n_eig_launch)
+      launch_sp_jacobi_step(d_layers, d_p8, (int)pairs8.size(), 8, 1024, t8, max_sweeps, ctx->tol, st);
+    launch_sp_check(d_layers, n_layers, t16, t8, max_sweeps, d_flag, st);
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (*ctx->h_flag) break;
+  }
+  stage_end(ctx, ATOMO_STAGE_EIG, st, n_eig_launch);
+
+  // ---- S2-S4: probabilities, draws, compaction ----
+  stage_begin(ctx, ATOMO_STAGE_SAMPLE, st);
+  const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
+  launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps, st);
+  stage_end(ctx, ATOMO_STAGE_SAMPLE, st, 1);
+
+  // ---- S4: long-side vectors of the kept atoms ----
+  stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);
+  launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), r_max, st);
+  launch_sp_finish_atoms(d_layers, n_layers, st);
+  stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, 2);
+  CK(cudaGetLastError());
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
+int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs, double s, uint64_t seed,
+                           uint64_t step, int64_t k_cap, void* payload, int64_t capacity_bytes,
+                           const atomo_debug* dbg, void* stream) {
+  if (!ctx || !vecs || n_vecs <= 0 || k_cap <= 0 || !payload) return ATOMO_ERR_INVALID_ARG;
+  if (bad_budget(s)) return ATOMO_ERR_BUDGET;
+  if ((reinterpret_cast<uintptr_t>(payload) & 15u) != 0) return ATOMO_ERR_INVALID_ARG;
+  std::vector<int64_t> ns(n_vecs);
+  for (int l = 0; l < n_vecs; ++l) {
+    if (!vecs[l].data || vecs[l].n <= 0 || vecs[l].n >= (int64_t(1) << 32)) return ATOMO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(vecs[l].data) & 3u) != 0) return ATOMO_ERR_INVALID_ARG;
+    ns[l] = vecs[l].n;
+  }
+  std::vector<EwLayout> lay;
+  const uint64_t total = layout_entrywise(ns.data(), n_vecs, k_cap, &lay);
+  if ((int64_t)total > capacity_bytes) return ATOMO_ERR_CAPACITY;
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  stage_reset(ctx);
+  uint8_t* pay = static_cast<uint8_t*>(payload);
+  atomo_layer_header* d_hdr = reinterpret_cast<atomo_layer_header*>(pay + sizeof(atomo_payload_header));
+  const int tile = ew_tile_elems();
+
+  std::vector<EwVec> V(n_vecs);
+  size_t need = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    Arena A(pass ? ctx->ws : nullptr);
+    size_t dbg_atoms = 0, dbg_words = 0;
+    for (int l = 0; l < n_vecs; ++l) {
+      EwVec& v = V[l];
+      v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
+      v.n_tiles = (v.n + tile - 1) / tile;
+      v.n_words = (v.n + 31) / 32;
+      const int64_t want_chunks = std::min<int64_t>(148 * 8, (v.n + 4095) / 4096);
+      v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
+      v.n_chunks = (int)((v.n + v.chunk - 1) / v.chunk);
+      v.hdr = d_hdr + l;
+      v.idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_idx);
+      v.val = reinterpret_cast<float*>(pay + lay[l].off_val);
+      v.partials = A.take<EwPartial>(v.n_chunks);
+      v.state = A.take<EwState>(1);
+      uint32_t* mask_ws = A.take<uint32_t>(v.n_words);
+      v.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
+      v.prob_out = (dbg && dbg->prob) ? dbg->prob + dbg_atoms : nullptr;
+      dbg_atoms += v.n; dbg_words += v.n_words;
+      v.tile_counts = A.take<uint32_t>(v.n_tiles);
+      v.tile_offsets = A.take<uint64_t>(v.n_tiles);
+    }
+    need = A.off + 256;
+    if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
+  }
+
+  std::vector<uint8_t> hdr_blob(sizeof(atomo_payload_header) + (size_t)n_vecs * sizeof(atomo_layer_header), 0);
+  atomo_payload_header gh{};
+  gh.magic = ATOMO_MAGIC; gh.version = ATOMO_VERSION; gh.kind = ATOMO_KIND_ENTRYWISE; gh.n_layers = (uint32_t)n_vecs;
+  gh.total_bytes = total; gh.seed = seed; gh.step = step; gh.s = s;
+  std::memcpy(hdr_blob.data(), &gh, sizeof(gh));
+  for (int l = 0; l < n_vecs; ++l) {
+    atomo_layer_header h{};
+    h.rows = 1; h.cols = ns[l]; h.k_cap = lay[l].kc; h.status = ATOMO_OK;
+    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val;
+    std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
+  }
+  CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
+
+  const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
+  const uint32_t ks = kind_step_word(ATOMO_KIND_ENTRYWISE, step);
+  // pass 1 for every vector, then water-filling rounds where the gradient is not s-balanced
+  stage_begin(ctx, ATOMO_STAGE_EW_REDUCE, st);
+  int64_t n_launch = 0;
+  for (int l = 0; l < n_vecs; ++l) { launch_ew_reduce_all(V[l], s, st); n_launch += 2; }
+  for (int l = 0; l < n_vecs; ++l) {
+    for (int round = 0; round <= kEwMaxRounds; ++round) {
+      CK(cudaMemcpyAsync(ctx->h_state, V[l].state, sizeof(EwState), cudaMemcpyDeviceToHost, st));
+      CK(cudaStreamSynchronize(st));
+      if (ctx->h_state->done) break;
+      launch_ew_round(V[l], s, st); n_launch += 2;
+    }
+  }
+  stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_launch);
+  stage_begin(ctx, ATOMO_STAGE_EW_PACK, st);
+  for (int l = 0; l < n_vecs; ++l) launch_ew_sample_pack(V[l], key, ks, st);
+  stage_end(ctx, ATOMO_STAGE_EW_PACK, st, 3 * (int64_t)n_vecs);
+  CK(cudaGetLastError());
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
+int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload, const int64_t* rows, const int64_t* cols,
+                 float* const* out, int32_t n_layers, void* stream) {
+  if (!ctx || !payload || !rows || !cols || !out || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;
+  if (kind != ATOMO_KIND_SPECTRAL && kind != ATOMO_KIND_ENTRYWISE) return ATOMO_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) if (!out[l] || rows[l] <= 0 || cols[l] <= 0) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  stage_reset(ctx);
+  const uint8_t* pay = static_cast<const uint8_t*>(payload);
+  const atomo_payload_header* d_gh = reinterpret_cast<const atomo_payload_header*>(pay);
+  const atomo_layer_header* d_hdr = reinterpret_cast<const atomo_layer_header*>(pay + sizeof(atomo_payload_header));
+  stage_begin(ctx, ATOMO_STAGE_DECODE, st);
+  if (kind == ATOMO_KIND_ENTRYWISE) {
+    for (int l = 0; l < n_layers; ++l) {
+      if (rows[l] != 1) return ATOMO_ERR_INVALID_ARG;
+      EwDecode d{pay, d_gh, d_hdr + l, out[l], cols[l]};
+      launch_ew_decode(d, st);
+    }
+    stage_end(ctx, ATOMO_STAGE_DECODE, st, n_layers);
+  } else {
+    std::vector<SpDecodeLayer> D(n_layers);
+    std::vector<TileRef> tiles;
+    const int tr = sp_decode_tile_rows(), tc = sp_decode_tile_cols();
+    for (int l = 0; l < n_layers; ++l) {
+      D[l] = SpDecodeLayer{d_hdr + l, out[l], rows[l], cols[l]};
+      const int na = (int)((rows[l] + tr - 1) / tr), nbt = (int)((cols[l] + tc - 1) / tc);
+      for (int a = 0; a < na; ++a) for (int b = 0; b < nbt; ++b) tiles.push_back({l, a, b, 0});
+    }
+    SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
+    for (int pass = 0; pass < 2; ++pass) {
+      Arena A(pass ? ctx->ws : nullptr);
+      d_layers = A.take<SpDecodeLayer>(n_layers);
+      d_tiles = A.take<TileRef>(tiles.size());
+      if (pass == 0) { const int rc = ensure_ws(ctx, A.off + 256); if (rc != ATOMO_OK) return rc; }
+    }
+    CK(cudaMemcpyAsync(d_layers, D.data(), D.size() * sizeof(SpDecodeLayer), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+    launch_sp_decode(pay, d_layers, d_tiles, (int)tiles.size(), st);
+    stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
+  }
+  CK(cudaGetLastError());
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
+int atomo_payload_read_headers(atomo_ctx* ctx, const void* payload, int32_t n_layers, atomo_payload_header* hdr,
+                               atomo_layer_header* layers, void* stream) {
+  if (!ctx || !payload || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const uint8_t* pay = static_cast<const uint8_t*>(payload);
+  if (hdr) CK(cudaMemcpyAsync(hdr, pay, sizeof(*hdr), cudaMemcpyDeviceToHost, st));
+  if (layers)
+    CK(cudaMemcpyAsync(layers, pay + sizeof(atomo_payload_header), (size_t)n_layers * sizeof(atomo_layer_header),
+                       cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return ATOMO_OK;
+}
+
+int atomo_payload_status(atomo_ctx* ctx, const void* payload, int32_t n_layers, int32_t* worst, int32_t* first_bad_layer,
+                         void* stream) {
+  if (!ctx || !payload || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;
+  std::vector<atomo_layer_header> h(n_layers);
+  const int rc = atomo_payload_read_headers(ctx, payload, n_layers, nullptr, h.data(), stream);
+  if (rc != ATOMO_OK) return rc;
+  int32_t w = ATOMO_OK, first = -1;
+  for (int l = 0; l < n_layers; ++l)
+    if (h[l].status != ATOMO_OK && first < 0) { w = (int32_t)h[l].status; first = l; }
+  if (worst) *worst = w;
+  if (first_bad_layer) *first_bad_layer = first;
+  return ATOMO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,98 @@
+// Device-side descriptors and kernel launchers shared by the API translation unit.
+#pragma once
+#include "atomo_common.cuh"
+
+namespace atomo {
+
+// ================================= entry-wise path ===============================================
+constexpr int kEwAll = 0, kEwRound = 1;
+constexpr int kEwMaxRounds = 64;      // water-filling rounds; Algorithm 1 saturates < ceil(s) atoms,
+                                      // a round usually takes many at once
+
+struct EwPartial { double sum; float amax; uint32_t cnt; uint32_t nonfinite; };
+
+struct EwState {
+  double T0;        // ||g||_1
+  double T;         // sum of |g| over unsaturated atoms
+  double s_cur;     // s - n_sat
+  double theta;     // atoms with |g| > theta have p = 1
+  float scale;      // p_i = |g_i| * scale for the rest
+  float c;          // T / s_cur
+  float theta_f, amax;
+  uint32_t n_sat, rounds, done, nonfinite;
+};
+
+struct EwVec {
+  const float* g; int64_t n;
+  uint32_t layer; uint32_t k_cap;
+  int64_t chunk; int n_chunks;            // reduction split (chunk is a multiple of 4)
+  int64_t n_tiles; int64_t n_words;
+  atomo_layer_header* hdr; uint32_t* idx; float* val;          // payload
+  EwPartial* partials; EwState* state;                         // workspace
+  uint32_t* mask_words; uint32_t* tile_counts; uint64_t* tile_offsets;
+  float* prob_out;                                             // debug or nullptr
+};
+
+struct EwDecode {
+  const uint8_t* payload; const atomo_payload_header* ghdr; const atomo_layer_header* hdr;
+  float* out; int64_t n;
+};
+
+void launch_ew_reduce_all(const EwVec& v, double s, cudaStream_t st);
+void launch_ew_round(const EwVec& v, double s, cudaStream_t st);
+void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st);
+void launch_ew_decode(const EwDecode& d, cudaStream_t st);
+int ew_tile_elems();
+
+// ================================= spectral path =================================================
+constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
+constexpr int kSmemRowsMaxRp = 1024;  // largest padded short side the shared-memory Jacobi kernel holds
+
+struct SpLayer {
+  const float* G; int rows, cols; int64_t ld;
+  int r, L, tall;              // short side, long side, rows > cols
+  int rp, B, nb;               // padded short side, Jacobi block rows, number of blocks (even)
+  uint32_t layer, k_cap;
+  float* X;                    // rp x 2rp: row i = [ x_i (rp) | v_i (rp) ],  x_i = v_i^T A
+  atomo_layer_header* hdr;     // payload
+  uint32_t* idx; float* coef; float* shortv; float* longv;
+  float* lam;                  // rp   eigenvalue per row (unsorted, scaled)
+  int* perm;                   // r    rank -> row
+  float* sigma; float* prob;   // r    descending (debug buffers or workspace)
+  uint32_t* mask_words;        // ceil(r/32)
+  float* p_sel;                // k_cap: p of the kept atoms
+  float* bp_partials;          // [bp_tiles][k_cap] partial squared norms of the long vectors
+  int bp_tiles;
+  uint32_t* rot_count;         // [max_sweeps] rotations applied in each sweep
+  float* scale;                // 1 float: power-of-two scaling applied to A
+  float* dbg_short;            // r x r or nullptr
+};
+
+struct SpDecodeLayer {
+  const atomo_layer_header* hdr; float* out; int64_t rows, cols;
+};
+
+struct TileRef { int32_t layer, a, b, c; };
+
+void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
+void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
+void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling
+// one Jacobi step (global step index t) for every layer of one (B, RP) class
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int rp,
+                           int t, int max_sweeps, float tol, cudaStream_t st);
+// convergence bookkeeping after t16 / t8 steps were enqueued for the two kernel classes
+void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
+                     cudaStream_t st);
+void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key,
+                               uint32_t kind_step, int max_sweeps, cudaStream_t st);
+void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st);
+void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, cudaStream_t st);
+void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,
+                      cudaStream_t st);
+int sp_configure();          // opt in to large dynamic shared memory; returns cudaError_t
+int sp_bp_rows_per_tile();
+int sp_bp_cols_per_tile();
+int sp_decode_tile_rows();
+int sp_decode_tile_cols();
+
+}  // namespace atomo

@@ -1,0 +1,687 @@
+// Spectral ATOMO (Section 5 of the paper): atoms are the rank-one terms sigma_i u_i v_i^T of the
+// layer gradient seen as a matrix; only the singular values are sparsified.
+//
+//   sp_gram            A = G G^T (rows <= cols) or G^T G, r x r on the short side, fp32 products
+//                      accumulated in short fp32 runs that are flushed into fp64
+//   sp_scale           power-of-two normalisation of A by its trace (keeps squared row norms of
+//                      small gradients away from the fp32 underflow range)
+//   sp_jacobi_step     one step of a one-sided (Hestenes) Jacobi eigen-solver on the rows of
+//                      X = [A | I]: row i is (x_i | v_i) with x_i = v_i^T A; orthogonal row
+//                      rotations keep that relation and drive the x_i mutually orthogonal, i.e.
+//                      x_i -> lambda_i v_i^T.  Blocks of B rows are paired round-robin; a CTA holds
+//                      one block pair in shared memory, one warp per rotation.
+//   sp_finalize_sample lambda_i = <x_i, v_i>, descending sort, sigma = sqrt(lambda), the
+//                      probabilities of Algorithm 1, Philox Bernoulli draws (Eq. 2), ordered
+//                      compaction of the kept ranks, short-side vectors of the kept atoms
+//   sp_backproject     long-side vector of each kept atom, w_i = G^T u_i (or G v_i)
+//   sp_finish_atoms    sigma_i = ||w_i||, coef_i = sigma_i / p_i, w_i normalised
+//   sp_decode          G_hat = sum_k coef_k u_k v_k^T, one coalesced write pass
+#include "atomo_kernels.cuh"
+
+namespace atomo {
+
+// =================================================================================================
+// init: V-part of X = identity (X was zero-filled by the caller)
+// =================================================================================================
+__global__ void sp_init_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  const int64_t ldx = 2 * (int64_t)L.rp;
+  for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < L.rp; i += gridDim.y * blockDim.x)
+    L.X[(int64_t)i * ldx + L.rp + i] = 1.0f;
+}
+
+void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef*, int, cudaStream_t st) {
+  sp_init_kernel<<<dim3(n_layers, 4), 256, 0, st>>>(d_layers);
+}
+
+// =================================================================================================
+// Gram matrix of the short side.  64 x 64 output tile per CTA, 16 x 16 threads, 4 x 4 per thread.
+// Short-side vector i is row i of G (rows <= cols) or column i of G (rows > cols).
+// =================================================================================================
+constexpr int kGramTile = 64, kGramK = 16;
+
+__global__ void __launch_bounds__(256) sp_gram_kernel(const SpLayer* __restrict__ layers,
+                                                      const TileRef* __restrict__ tiles) {
+  __shared__ __align__(16) float As[kGramK][kGramTile + 4];
+  __shared__ __align__(16) float Bs[kGramK][kGramTile + 4];
+  const TileRef ref = tiles[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int i0 = ref.a * kGramTile, j0 = ref.b * kGramTile;
+  const bool diag = ref.a == ref.b;
+  const float* __restrict__ G = L.G;
+  const int64_t ld = L.ld;
+  const int r = L.r, len = L.L;
+  const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+  float acc[4][4];
+  double acc64[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) { acc[a][b] = 0.0f; acc64[a][b] = 0.0; }
+
+  int flush = 0;
+  for (int c0 = 0; c0 < len; c0 += kGramK) {
+    // stage As[kk][i] = x_{i0+i}[c0+kk], Bs likewise for j0
+    if (!L.tall) {
+      const int row = t / 4, k4 = (t % 4) * 4;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = c0 + k4 + j;
+        const int ia = i0 + row, ib = j0 + row;
+        As[k4 + j][row] = (ia < r && c < len) ? __ldg(G + (int64_t)ia * ld + c) : 0.0f;
+        if (!diag) Bs[k4 + j][row] = (ib < r && c < len) ? __ldg(G + (int64_t)ib * ld + c) : 0.0f;
+      }
+    } else {
+      const int kk = t / 16, i4 = (t % 16) * 4;
+      const int c = c0 + kk;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int ia = i0 + i4 + j, ib = j0 + i4 + j;
+        As[kk][i4 + j] = (ia < r && c < len) ? __ldg(G + (int64_t)c * ld + ia) : 0.0f;
+        if (!diag) Bs[kk][i4 + j] = (ib < r && c < len) ? __ldg(G + (int64_t)c * ld + ib) : 0.0f;
+      }
+    }
+    __syncthreads();
+    const float(*Bp)[kGramTile + 4] = diag ? As : Bs;
+#pragma unroll
+    for (int kk = 0; kk < kGramK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bp[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[p][q] = fmaf(av[p], bv[q], acc[p][q]);
+    }
+    __syncthreads();
+    if (++flush == 2) {   // 32 products per fp32 run, then into fp64
+      flush = 0;
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { acc64[p][q] += (double)acc[p][q]; acc[p][q] = 0.0f; }
+    }
+  }
+  const int64_t ldx = 2 * (int64_t)L.rp;
+#pragma unroll
+  for (int p = 0; p < 4; ++p)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int i = i0 + ty * 4 + p, j = j0 + tx * 4 + q;
+      if (i < r && j < r) {
+        const float v = (float)(acc64[p][q] + (double)acc[p][q]);
+        L.X[(int64_t)i * ldx + j] = v;
+        if (!diag) L.X[(int64_t)j * ldx + i] = v;
+      }
+    }
+}
+
+void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st) {
+  if (n_tiles > 0) sp_gram_kernel<<<n_tiles, 256, 0, st>>>(d_layers, d_tiles);
+}
+
+// =================================================================================================
+// scale A by a power of two so that trace(A) is about 1
+// =================================================================================================
+__global__ void __launch_bounds__(256) sp_trace_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  const int64_t ldx = 2 * (int64_t)L.rp;
+  __shared__ float s_red[256];
+  float tr = 0.0f;
+  for (int i = threadIdx.x; i < L.r; i += 256) tr += L.X[(int64_t)i * ldx + i];
+  s_red[threadIdx.x] = tr;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
+  tr = s_red[0];
+  float sc = 1.0f;
+  if (tr > 0.0f && tr < 3.0e38f) sc = exp2f(-rintf(log2f(tr)));
+  if (!(sc > 0.0f) || !(sc < 3.0e38f)) sc = 1.0f;
+  if (threadIdx.x == 0) *L.scale = sc;
+}
+
+__global__ void __launch_bounds__(256) sp_scale_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  const int64_t ldx = 2 * (int64_t)L.rp;
+  const float sc = *L.scale;
+  if (sc == 1.0f) return;
+  for (int i = blockIdx.y; i < L.r; i += gridDim.y)
+    for (int j = threadIdx.x; j < L.r; j += 256) L.X[(int64_t)i * ldx + j] *= sc;
+}
+
+void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
+  sp_trace_kernel<<<n_layers, 256, 0, st>>>(d_layers);
+  sp_scale_kernel<<<dim3(n_layers, 32), 256, 0, st>>>(d_layers);
+}
+
+// =================================================================================================
+// One-sided Jacobi, block pair resident in shared memory.
+// =================================================================================================
+// round-robin tournament over n (even) players: pair `slot` of round `round`
+__device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int& q) {
+  const int m = n - 1;
+  if (slot == 0) { p = n - 1; q = round % m; }
+  else { p = (round + slot) % m; q = (round - slot + m) % m; }
+}
+
+template <int T4>
+struct RowRegs { float4 v[T4]; };
+
+// rotate rows (xp, xq) so that their first A4 float4 (the x-parts) become orthogonal.
+// Returns true if a rotation was applied.  All lanes take the same branch.
+template <int T4>
+__device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, int lane, int A4, float tol) {
+  float al = 0.f, be = 0.f, ga = 0.f;
+#pragma unroll
+  for (int t = 0; t < T4; ++t) {
+    if (lane + 32 * t < A4) {
+      const float4 a = xp.v[t], b = xq.v[t];
+      al = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, al))));
+      be = fmaf(b.x, b.x, fmaf(b.y, b.y, fmaf(b.z, b.z, fmaf(b.w, b.w, be))));
+      ga = fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, fmaf(a.w, b.w, ga))));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    al += __shfl_xor_sync(0xffffffffu, al, o);
+    be += __shfl_xor_sync(0xffffffffu, be, o);
+    ga += __shfl_xor_sync(0xffffffffu, ga, o);
+  }
+  // skip when the rows are orthogonal to working precision, or one of them is zero (false for NaN)
+  if (!(fabsf(ga) > tol * sqrtf(al) * sqrtf(be))) return false;
+  const float zeta = (be - al) / (2.0f * ga);
+  const float tt = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
+  const float c = 1.0f / sqrtf(fmaf(tt, tt, 1.0f));
+  const float s = c * tt;
+#pragma unroll
+  for (int t = 0; t < T4; ++t) {
+    const float4 a = xp.v[t], b = xq.v[t];
+    xp.v[t] = make_float4(fmaf(c, a.x, -s * b.x), fmaf(c, a.y, -s * b.y), fmaf(c, a.z, -s * b.z), fmaf(c, a.w, -s * b.w));
+    xq.v[t] = make_float4(fmaf(s, a.x, c * b.x), fmaf(s, a.y, c * b.y), fmaf(s, a.z, c * b.z), fmaf(s, a.w, c * b.w));
+  }
+  return true;
+}
+
+template <int T4>
+__device__ __forceinline__ void load_row(RowRegs<T4>& x, const float* row, int lane, int V4) {
+#pragma unroll
+  for (int t = 0; t < T4; ++t)
+    x.v[t] = (lane + 32 * t < V4) ? reinterpret_cast<const float4*>(row)[lane + 32 * t] : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+template <int T4>
+__device__ __forceinline__ void store_row(const RowRegs<T4>& x, float* row, int lane, int V4) {
+#pragma unroll
+  for (int t = 0; t < T4; ++t)
+    if (lane + 32 * t < V4) reinterpret_cast<float4*>(row)[lane + 32 * t] = x.v[t];
+}
+
+// One block pair of one layer.  B rows per block, B warps; RP = padded short side (row = 2 RP floats).
+template <int B, int RP>
+__device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, float tol,
+                                                  float* smem) {
+  constexpr int LD = 2 * RP, V4 = LD / 4, A4 = RP / 4, T4 = (V4 + 31) / 32;
+  constexpr int NT = 32 * B;
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  int bi, bj;
+  rr_pair(L.nb, local, slot, bi, bj);
+  float* X = L.X;
+  // ---- load 2B rows ----
+  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
+    const int row = idx / V4, q = idx % V4;
+    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
+    reinterpret_cast<float4*>(smem + row * LD)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * LD)[q];
+  }
+  __syncthreads();
+  uint32_t nrot = 0;
+  RowRegs<T4> xp, xq;
+  // ---- pairs inside each block: once per sweep ----
+  if (local == 0) {
+    for (int round = 0; round < B - 1; ++round) {
+      if (w < B) {
+        const int blk = w / (B / 2), sl = w % (B / 2);
+        int p, q;
+        rr_pair(B, round, sl, p, q);
+        float* rowp = smem + (blk * B + p) * LD;
+        float* rowq = smem + (blk * B + q) * LD;
+        load_row<T4>(xp, rowp, lane, V4);
+        load_row<T4>(xq, rowq, lane, V4);
+        if (rotate_pair<T4>(xp, xq, lane, A4, tol)) {
+          store_row<T4>(xp, rowp, lane, V4);
+          store_row<T4>(xq, rowq, lane, V4);
+          ++nrot;
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // ---- pairs across the two blocks: warp w keeps row w of block bi in registers ----
+  if (w < B) load_row<T4>(xp, smem + w * LD, lane, V4);
+  for (int round = 0; round < B; ++round) {
+    if (w < B) {
+      float* rowq = smem + (B + (w + round) % B) * LD;
+      load_row<T4>(xq, rowq, lane, V4);
+      if (rotate_pair<T4>(xp, xq, lane, A4, tol)) {
+        store_row<T4>(xq, rowq, lane, V4);
+        ++nrot;
+      }
+    }
+    __syncthreads();
+  }
+  if (w < B) store_row<T4>(xp, smem + w * LD, lane, V4);
+  __syncthreads();
+  // ---- store ----
+  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
+    const int row = idx / V4, q = idx % V4;
+    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
+    reinterpret_cast<float4*>(X + (int64_t)grow * LD)[q] = reinterpret_cast<const float4*>(smem + row * LD)[q];
+  }
+  if (lane == 0 && nrot) atomicAdd(L.rot_count + sweep, nrot);
+}
+
+// All layers whose padded short side is <= 512: B = 16, 512 threads, one launch per step.
+__global__ void __launch_bounds__(512) sp_jacobi_step16_kernel(const SpLayer* __restrict__ layers,
+                                                               const TileRef* __restrict__ pairs, int t,
+                                                               int max_sweeps, float tol) {
+  extern __shared__ __align__(16) float smem[];
+  const TileRef ref = pairs[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int steps = L.nb - 1;
+  const int sweep = t / steps, local = t % steps;
+  if (sweep >= max_sweeps) return;
+  if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
+  switch (L.rp) {
+    case 32: jacobi_block_pair<16, 32>(L, ref.a, sweep, local, tol, smem); break;
+    case 64: jacobi_block_pair<16, 64>(L, ref.a, sweep, local, tol, smem); break;
+    case 128: jacobi_block_pair<16, 128>(L, ref.a, sweep, local, tol, smem); break;
+    case 256: jacobi_block_pair<16, 256>(L, ref.a, sweep, local, tol, smem); break;
+    case 512: jacobi_block_pair<16, 512>(L, ref.a, sweep, local, tol, smem); break;
+    default: break;
+  }
+}
+
+// Layers with padded short side 1024: B = 8, 256 threads.
+__global__ void __launch_bounds__(256) sp_jacobi_step8_kernel(const SpLayer* __restrict__ layers,
+                                                              const TileRef* __restrict__ pairs, int t,
+                                                              int max_sweeps, float tol) {
+  extern __shared__ __align__(16) float smem[];
+  const TileRef ref = pairs[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int steps = L.nb - 1;
+  const int sweep = t / steps, local = t % steps;
+  if (sweep >= max_sweeps) return;
+  if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;
+  jacobi_block_pair<8, 1024>(L, ref.a, sweep, local, tol, smem);
+}
+
+constexpr int kJacobiSmem = 2 * 16 * 2 * 512 * 4;   // 128 KB: 32 rows of 1024 floats (or 16 rows of 2048)
+
+__global__ void sp_backproject_kernel(const SpLayer* __restrict__ layers, const TileRef* __restrict__ tiles);
+
+int sp_configure() {
+  cudaError_t e = cudaFuncSetAttribute(sp_jacobi_step16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  if (e != cudaSuccess) return (int)e;
+  e = cudaFuncSetAttribute(sp_jacobi_step8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  if (e != cudaSuccess) return (int)e;
+  e = cudaFuncSetAttribute(sp_backproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           8 * kMaxShort * (int)sizeof(float));
+  return (int)e;
+}
+
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int rp_max,
+                           int t, int max_sweeps, float tol, cudaStream_t st) {
+  if (n_pairs <= 0) return;
+  if (B == 16) {
+    const int smem = 2 * 16 * 2 * rp_max * 4;
+    sp_jacobi_step16_kernel<<<n_pairs, 512, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
+  } else {
+    sp_jacobi_step8_kernel<<<n_pairs, 256, kJacobiSmem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
+  }
+}
+
+// convergence bookkeeping after `t_done[group]` steps have been enqueued for each group
+__global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers, int t16, int t8, int max_sweeps,
+                                uint32_t* all_done) {
+  __shared__ int s_pending;
+  if (threadIdx.x == 0) s_pending = 0;
+  __syncthreads();
+  for (int l = threadIdx.x; l < n_layers; l += blockDim.x) {
+    const SpLayer& L = layers[l];
+    const int steps = L.nb - 1;
+    const int t_done = (L.B == 16) ? t16 : t8;
+    const int sweeps_done = min(t_done / steps, max_sweeps);
+    int conv = -1;
+    for (int wv = 0; wv < sweeps_done; ++wv) if (L.rot_count[wv] == 0) { conv = wv; break; }
+    if (conv >= 0) L.hdr->sweeps = (uint32_t)(conv + 1);
+    else {
+      L.hdr->sweeps = (uint32_t)sweeps_done;
+      if (sweeps_done < max_sweeps) atomicAdd(&s_pending, 1);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) *all_done = s_pending == 0 ? 1u : 0u;
+}
+
+// =================================================================================================
+// finalize + probabilities + sampling.  One CTA (512 threads) per layer.
+// =================================================================================================
+constexpr int kFinThreads = 512;
+
+__global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const SpLayer* __restrict__ layers, double s,
+                                                                         PhiloxKey key, uint32_t kind_step,
+                                                                         int max_sweeps) {
+  const SpLayer& L = layers[blockIdx.x];
+  __shared__ float s_lam[kMaxShort];        // eigenvalues by row, later sigma by rank
+  __shared__ float s_sig[kMaxShort];
+  __shared__ double s_red[kFinThreads];
+  __shared__ uint32_t s_scan[kFinThreads / 32];
+  __shared__ double s_T, s_scur;
+  __shared__ uint32_t s_nsat, s_bad, s_k;
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const int r = L.r, rp = L.rp;
+  const int64_t ldx = 2 * (int64_t)rp;
+  const float inv_scale = 1.0f / *L.scale;
+  atomo_layer_header* h = L.hdr;
+  if (tid == 0) { s_bad = 0; s_k = 0; }
+  __syncthreads();
+
+  // lambda_i = <x_i, v_i>  (Rayleigh quotient of A at v_i), one warp per row
+  for (int i = w; i < r; i += kFinThreads / 32) {
+    const float* row = L.X + (int64_t)i * ldx;
+    float d = 0.f;
+    for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[rp + j], d);
+    d = warp_sum(d);
+    if (lane == 0) {
+      const float lam = d * inv_scale;
+      if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
+      s_lam[i] = fmaxf(lam, 0.0f);
+    }
+  }
+  __syncthreads();
+  const bool bad = s_bad != 0;
+  // rank by counting (descending, ties: lower row first); sigma = sqrt(lambda)
+  for (int i = tid; i < r; i += kFinThreads) {
+    const float li = s_lam[i];
+    int rank = 0;
+    for (int j = 0; j < r; ++j) { const float lj = s_lam[j]; rank += (lj > li) || (lj == li && j < i); }
+    s_sig[rank] = bad ? 0.0f : sqrtf(li);
+    L.perm[rank] = i;
+  }
+  __syncthreads();
+  // ||sigma||_1 in fp64, fixed tree
+  double part = 0.0;
+  for (int i = tid; i < r; i += kFinThreads) part += (double)s_sig[i];
+  s_red[tid] = part;
+  __syncthreads();
+  for (int o = kFinThreads / 2; o > 0; o >>= 1) { if (tid < o) s_red[tid] += s_red[tid + o]; __syncthreads(); }
+  if (tid == 0) {
+    // Algorithm 1 on the sorted sigma: peel atoms while sigma_i * s > sum_{j >= i} sigma_j
+    double T = s_red[0], sc = s;
+    int i = 0;
+    while (i < r && (double)s_sig[i] * sc > T) { T -= (double)s_sig[i]; sc -= 1.0; ++i; }
+    if (i == r || !(T > 0.0)) T = 0.0;
+    s_T = T; s_scur = sc; s_nsat = (uint32_t)i;
+    h->n_sat = (uint32_t)i;
+    h->c = (T > 0.0 && sc > 0.0) ? (float)(T / sc) : 0.0f;
+    h->l1 = s_red[0];
+  }
+  __syncthreads();
+  const double T = s_T, scur = s_scur;
+  const int n_sat = (int)s_nsat;
+  const double scale = (T > 0.0 && scur > 0.0) ? scur / T : 0.0;
+
+  // probabilities, Bernoulli draws, ordered compaction of the kept ranks
+  uint32_t carry = 0;
+  for (int base = 0; base < r; base += kFinThreads) {
+    const int i = base + tid;
+    float p = 0.0f;
+    bool keep = false;
+    if (i < r) {
+      const float sg = s_sig[i];
+      p = (i < n_sat) ? 1.0f : fminf((float)((double)sg * scale), 1.0f);
+      if (!(sg > 0.0f)) p = 0.0f;
+      const uint4 wd = atom_block_words((uint64_t)(i >> 2), L.layer, kind_step, key);
+      const uint32_t word = (i & 3) == 0 ? wd.x : (i & 3) == 1 ? wd.y : (i & 3) == 2 ? wd.z : wd.w;
+      keep = !bad && bernoulli_keep(p, word);
+      if (L.sigma) L.sigma[i] = sg;
+      if (L.prob) L.prob[i] = p;
+    }
+    const uint32_t ballot = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) {
+      s_scan[w] = __popc(ballot);
+      if (L.mask_words && base + w * 32 < r) L.mask_words[(base >> 5) + w] = ballot;
+    }
+    __syncthreads();
+    uint32_t off = carry;
+    for (int j = 0; j < w; ++j) off += s_scan[j];
+    uint32_t total = 0;
+    for (int j = 0; j < kFinThreads / 32; ++j) total += s_scan[j];
+    if (keep) {
+      const uint32_t pos = off + __popc(ballot & ((1u << lane) - 1u));
+      if (pos < L.k_cap) { L.idx[pos] = (uint32_t)i; L.p_sel[pos] = p; }
+    }
+    carry += total;
+    __syncthreads();
+  }
+  if (tid == 0) {
+    uint32_t status = ATOMO_OK;
+    if (bad) status = ATOMO_ERR_NONFINITE;
+    else if (carry > L.k_cap) status = ATOMO_ERR_CAPACITY;
+    else if (h->sweeps >= (uint32_t)max_sweeps && L.rot_count[max_sweeps - 1] != 0) status = ATOMO_ERR_NOT_CONVERGED;
+    h->status = status;
+    const uint32_t k = (status == ATOMO_OK || status == ATOMO_ERR_NOT_CONVERGED) ? carry : 0u;
+    h->k = k;
+    s_k = k;
+  }
+  __syncthreads();
+  const uint32_t k = s_k;
+  // short-side vectors of the kept atoms, normalised: payload shortv[a][0..r)
+  for (uint32_t a = w; a < k; a += kFinThreads / 32) {
+    const int row = L.perm[L.idx[a]];
+    const float* v = L.X + (int64_t)row * ldx + rp;
+    float n2 = 0.f;
+    for (int j = lane; j < r; j += 32) n2 = fmaf(v[j], v[j], n2);
+    n2 = warp_sum(n2);
+    const float inv = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
+    for (int j = lane; j < r; j += 32) L.shortv[(int64_t)a * r + j] = v[j] * inv;
+  }
+  // optional: every short-side vector, rank-major
+  if (L.dbg_short) {
+    for (int a = w; a < r; a += kFinThreads / 32) {
+      const float* v = L.X + (int64_t)L.perm[a] * ldx + rp;
+      for (int j = lane; j < r; j += 32) L.dbg_short[(int64_t)a * r + j] = v[j];
+    }
+  }
+}
+
+void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
+                     cudaStream_t st) {
+  sp_check_kernel<<<1, 256, 0, st>>>(d_layers, n_layers, t16, t8, max_sweeps, d_all_done);
+}
+
+void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key, uint32_t kind_step,
+                               int max_sweeps, cudaStream_t st) {
+  sp_finalize_sample_kernel<<<n_layers, kFinThreads, 0, st>>>(d_layers, s, key, kind_step, max_sweeps);
+}
+
+// =================================================================================================
+// back-projection: long-side vector of each kept atom.
+//   rows <= cols: w_a[c]   = sum_i G[i][c] u_a[i]      (tile = 256 columns, thread per column)
+//   rows >  cols: w_a[row] = sum_c G[row][c] v_a[c]    (tile = 32 rows, warp per row)
+// Unnormalised w goes to payload longv; the squared norm of each tile goes to bp_partials.
+// =================================================================================================
+constexpr int kBpThreads = 256, kBpAtoms = 8, kBpCols = 256, kBpRows = 32;
+int sp_bp_cols_per_tile() { return kBpCols; }
+int sp_bp_rows_per_tile() { return kBpRows; }
+
+__global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLayer* __restrict__ layers,
+                                                                    const TileRef* __restrict__ tiles) {
+  extern __shared__ __align__(16) float s_u[];          // kBpAtoms x r
+  __shared__ float s_part[kBpThreads / 32][kBpAtoms];
+  const TileRef ref = tiles[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const uint32_t k = L.hdr->k;
+  const int r = L.r, len = L.L;
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const float* __restrict__ G = L.G;
+  const int64_t ld = L.ld;
+  for (uint32_t a0 = 0; a0 < k; a0 += kBpAtoms) {
+    const int na = min((uint32_t)kBpAtoms, k - a0);
+    __syncthreads();
+    for (int idx = tid; idx < na * r; idx += kBpThreads) s_u[idx] = L.shortv[(int64_t)a0 * r + idx];
+    __syncthreads();
+    float nrm[kBpAtoms];
+#pragma unroll
+    for (int a = 0; a < kBpAtoms; ++a) nrm[a] = 0.f;
+    if (!L.tall) {
+      const int c = ref.a * kBpCols + tid;
+      float acc[kBpAtoms];
+#pragma unroll
+      for (int a = 0; a < kBpAtoms; ++a) acc[a] = 0.f;
+      if (c < len) {
+        for (int i = 0; i < r; ++i) {
+          const float g = __ldg(G + (int64_t)i * ld + c);
+#pragma unroll
+          for (int a = 0; a < kBpAtoms; ++a) if (a < na) acc[a] = fmaf(g, s_u[a * r + i], acc[a]);
+        }
+#pragma unroll
+        for (int a = 0; a < kBpAtoms; ++a) if (a < na) { L.longv[(int64_t)(a0 + a) * len + c] = acc[a]; nrm[a] = acc[a] * acc[a]; }
+      }
+    } else {
+      for (int rr = w; rr < kBpRows; rr += kBpThreads / 32) {
+        const int row = ref.a * kBpRows + rr;
+        if (row >= len) break;
+        float acc[kBpAtoms];
+#pragma unroll
+        for (int a = 0; a < kBpAtoms; ++a) acc[a] = 0.f;
+        for (int c = lane; c < r; c += 32) {
+          const float g = __ldg(G + (int64_t)row * ld + c);
+#pragma unroll
+          for (int a = 0; a < kBpAtoms; ++a) if (a < na) acc[a] = fmaf(g, s_u[a * r + c], acc[a]);
+        }
+#pragma unroll
+        for (int a = 0; a < kBpAtoms; ++a) {
+          acc[a] = warp_sum(acc[a]);
+          if (a < na && lane == 0) { L.longv[(int64_t)(a0 + a) * len + row] = acc[a]; nrm[a] += acc[a] * acc[a]; }
+        }
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < kBpAtoms; ++a) { nrm[a] = warp_sum(nrm[a]); if (lane == 0) s_part[w][a] = nrm[a]; }
+    __syncthreads();
+    if (tid < na) {
+      float tot = 0.f;
+      for (int j = 0; j < kBpThreads / 32; ++j) tot += s_part[j][tid];
+      L.bp_partials[(int64_t)ref.a * L.k_cap + a0 + tid] = tot;
+    }
+  }
+}
+
+void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st) {
+  if (n_tiles > 0)
+    sp_backproject_kernel<<<n_tiles, kBpThreads, kBpAtoms * r_max * sizeof(float), st>>>(d_layers, d_tiles);
+}
+
+// sigma_a = ||w_a||, coef_a = sigma_a / p_a, w_a normalised.  One CTA per layer.
+__global__ void __launch_bounds__(256) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  const uint32_t k = L.hdr->k;
+  __shared__ float s_inv;
+  for (uint32_t a = 0; a < k; ++a) {
+    if (threadIdx.x < 32) {
+      double tot = 0.0;
+      for (int t = threadIdx.x; t < L.bp_tiles; t += 32) tot += (double)L.bp_partials[(int64_t)t * L.k_cap + a];
+      tot = warp_sum(tot);
+      if (threadIdx.x == 0) {
+        const float sg = (float)sqrt(tot);
+        L.coef[a] = sg / L.p_sel[a];
+        s_inv = sg > 0.f ? 1.0f / sg : 0.f;
+      }
+    }
+    __syncthreads();
+    const float inv = s_inv;
+    for (int j = threadIdx.x; j < L.L; j += 256) L.longv[(int64_t)a * L.L + j] *= inv;
+    __syncthreads();
+  }
+}
+
+void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
+  sp_finish_atoms_kernel<<<n_layers, 256, 0, st>>>(d_layers);
+}
+
+// =================================================================================================
+// decode: out[i][c] = sum_a coef_a rowvec_a[i] colvec_a[c].  Tile 32 rows x 256 columns,
+// 256 threads: thread = (row group of 8) x (4 consecutive columns... x 2).
+// =================================================================================================
+constexpr int kDecRows = 32, kDecCols = 256, kDecAtoms = 16;
+int sp_decode_tile_rows() { return kDecRows; }
+int sp_decode_tile_cols() { return kDecCols; }
+
+__global__ void __launch_bounds__(256) sp_decode_kernel(const uint8_t* __restrict__ payload,
+                                                        const SpDecodeLayer* __restrict__ layers,
+                                                        const TileRef* __restrict__ tiles) {
+  __shared__ __align__(16) float s_col[kDecAtoms][kDecCols];
+  __shared__ float s_row[kDecAtoms][kDecRows];
+  const atomo_payload_header* gh = reinterpret_cast<const atomo_payload_header*>(payload);
+  const TileRef ref = tiles[blockIdx.x];
+  const SpDecodeLayer D = layers[ref.layer];
+  const atomo_layer_header* h = D.hdr;
+  const int64_t rows = D.rows, cols = D.cols;
+  const bool ok = gh->magic == ATOMO_MAGIC && gh->kind == ATOMO_KIND_SPECTRAL && h->rows == rows && h->cols == cols &&
+                  h->k <= h->k_cap;
+  if (!ok && ref.a == 0 && ref.b == 0 && threadIdx.x == 0) raise_status(const_cast<atomo_layer_header*>(h), ATOMO_ERR_PAYLOAD);
+  const uint32_t k = ok ? h->k : 0u;
+  const bool tall = rows > cols;
+  const int64_t r = tall ? cols : rows, len = tall ? rows : cols;
+  const float* coef = reinterpret_cast<const float*>(payload + h->off_val);
+  const float* shortv = reinterpret_cast<const float*>(payload + h->off_short);
+  const float* longv = reinterpret_cast<const float*>(payload + h->off_long);
+  const float* rowvec = tall ? longv : shortv;   // indexed by output row
+  const float* colvec = tall ? shortv : longv;   // indexed by output column
+  const int64_t rlen = tall ? len : r, clen = tall ? r : len;
+  const int64_t i0 = (int64_t)ref.a * kDecRows, c0 = (int64_t)ref.b * kDecCols;
+  const int tid = threadIdx.x;
+  const int cg = tid % 64, rg = tid / 64;            // 64 column groups of 4, 4 row groups of 8
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+  for (uint32_t a0 = 0; a0 < k; a0 += kDecAtoms) {
+    const int na = min((uint32_t)kDecAtoms, k - a0);
+    __syncthreads();
+    for (int idx = tid; idx < na * kDecCols; idx += 256) {
+      const int a = idx / kDecCols, c = idx % kDecCols;
+      s_col[a][c] = (c0 + c < clen) ? __ldg(colvec + (int64_t)(a0 + a) * clen + c0 + c) : 0.f;
+    }
+    for (int idx = tid; idx < na * kDecRows; idx += 256) {
+      const int a = idx / kDecRows, i = idx % kDecRows;
+      s_row[a][i] = (i0 + i < rlen) ? __ldg(rowvec + (int64_t)(a0 + a) * rlen + i0 + i) * __ldg(coef + a0 + a) : 0.f;
+    }
+    __syncthreads();
+    for (int a = 0; a < na; ++a) {
+      const float4 cv = *reinterpret_cast<const float4*>(&s_col[a][cg * 4]);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const float rv = s_row[a][rg * 8 + i];
+        acc[i][0] = fmaf(rv, cv.x, acc[i][0]); acc[i][1] = fmaf(rv, cv.y, acc[i][1]);
+        acc[i][2] = fmaf(rv, cv.z, acc[i][2]); acc[i][3] = fmaf(rv, cv.w, acc[i][3]);
+      }
+    }
+  }
+  const bool vec_ok = (cols % 4 == 0) && ((reinterpret_cast<uintptr_t>(D.out) & 15u) == 0);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int64_t row = i0 + rg * 8 + i;
+    if (row >= rows) continue;
+    const int64_t c = c0 + cg * 4;
+    float* o = D.out + row * cols + c;
+    if (vec_ok && c + 3 < cols) *reinterpret_cast<float4*>(o) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    else for (int j = 0; j < 4; ++j) if (c + j < cols) o[j] = acc[i][j];
+  }
+}
+
+void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,
+                      cudaStream_t st) {
+  if (n_tiles > 0) sp_decode_kernel<<<n_tiles, 256, 0, st>>>(payload, d_layers, d_tiles);
+}
+
+}  // namespace atomo
