@@ -1,0 +1,319 @@
+#!/usr/bin/env python
+"""Benchmark of the ATOMO encode + decode hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4|c5] [--impl ours|reference]
+
+A step is one pass of the whole path (encode, then decode) over one batch of synthetic
+gradients.  The default workload is the ResNet-18-shaped layer set (spectral ATOMO, s = 2,
+18 layers, 10,992,320 gradient elements, one batched call).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "gradient elements encoded+decoded/sec"
+UNIT = "elements/s"
+L2_BYTES = 126 * 1024 * 1024
+FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # SMs x FP32 lanes x 2 flop x max SM clock
+# dram bytes per Jacobi-step launch from the ncu capture summarised in profiles/ (None until captured)
+JACOBI_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+
+    def start(self):
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        rows = [r.strip().split(",") for r in open(self.f.name) if r.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except Exception:
+                continue
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            for name, v in zip(names, r[5:9]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ---------------------------------------------------------------------------------------------
+def workload_c2(seed):
+    from paper_1806_04090_b200 import synth
+    return synth.c2_resnet18(seed), synth.layer_elements(synth.RESNET18_LAYERS)
+
+
+def oracle_step(mats, s, seed, step):
+    """Encode + decode of a list of layers with the fp64 oracle (single thread)."""
+    from oracle import atomo_oracle as oracle
+    for l, G in enumerate(mats):
+        enc = oracle.encode_spectral(G, s, seed, step=step, layer=l)
+        oracle.decode_spectral(enc["coef"], enc["U_S"], enc["V_S"])
+
+
+def cpu_baseline_c2(seed=0):
+    """The oracle as it stands on the host cores: one layer per distinct shape is timed and the
+    time is scaled by how often the shape occurs (the full set takes about a minute per step)."""
+    from paper_1806_04090_b200 import synth
+    from oracle import atomo_oracle as oracle
+    oracle.build()
+    layers = synth.RESNET18_LAYERS
+    shapes = {}
+    for i, l in enumerate(layers):
+        shapes.setdefault((l.rows, l.cols), []).append(i)
+    total = 0.0
+    t_all = time.perf_counter()
+    for (rows, cols), idxs in shapes.items():
+        G = synth.c2_resnet18(seed, [layers[idxs[0]]])
+        t0 = time.perf_counter()
+        oracle_step(G, 2.0, seed, 0)
+        total += (time.perf_counter() - t0) * len(idxs)
+    elems = synth.layer_elements(layers)
+    return {"value": elems / total, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"one layer per distinct shape ({len(shapes)} of {len(layers)} layers, "
+                      f"{time.perf_counter() - t_all:.1f} s of CPU), time scaled by shape count to the full set "
+                      f"(extrapolated step time {total:.1f} s)"}
+
+
+def reference_sample_layers():
+    from paper_1806_04090_b200 import synth
+    seen, out = set(), []
+    for l in synth.RESNET18_LAYERS:
+        if min(l.rows, l.cols) <= 256 and (l.rows, l.cols) not in seen:
+            seen.add((l.rows, l.cols)); out.append(l)
+    return out
+
+
+def run_reference(args):
+    """--impl reference: the oracle, as it stands, on the host cores (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1806_04090_b200 import synth
+    from oracle import atomo_oracle as oracle
+    oracle.build()
+    layers = reference_sample_layers()
+    mats = synth.c2_resnet18(0, layers)
+    elems = synth.layer_elements(layers)
+    for w in range(args.warmup):
+        oracle_step(mats, 2.0, 0, w)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        oracle_step(mats, 2.0, 0, args.warmup + k)
+    dt = time.perf_counter() - t0
+    value = elems * args.steps / dt
+    sample = (f"per step: one layer of each distinct ResNet-18 shape with short side <= 256 "
+              f"({len(layers)} layers, {elems} elements); the 512-row layers are left out to bound the run")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": "c2: ResNet-18-shaped layer set, spectral ATOMO s=2 (bounded sample)", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------
+def jacobi_flops(shapes, sweeps):
+    """Algorithmic flops of the eigen-solver: per sweep r(r-1)/2 row pairs, each 3 dot products
+    over r terms (6r flop) and a rotation of two rows of 2r entries (12r flop)."""
+    tot = 0.0
+    for (rows, cols), sw in zip(shapes, sweeps):
+        r = min(rows, cols)
+        tot += sw * (r * (r - 1) / 2.0) * 18.0 * r
+    return tot
+
+
+def run_ours(args):
+    import torch
+    from paper_1806_04090_b200 import api, dist
+
+    backend = "nccl"
+    rank, local_rank, world = dist.init(backend) if int(os.environ.get("WORLD_SIZE", "1")) > 1 else (0, 0, 1)
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    a = api.Atomo(local_rank)
+
+    if args.workload != "c2":
+        raise SystemExit("only the c2 workload is a bench line; the other configs are parity-test cases")
+    s, seed = 2.0, 0
+    # several distinct input sets so that each step's gradients were evicted from L2 since last use
+    mats0, elems = workload_c2(seed)
+    in_bytes = sum(m.nbytes for m in mats0)
+    n_sets = int(np.ceil(2.0 * L2_BYTES / in_bytes)) + 1
+    host_sets = [mats0] + [workload_c2(seed + 1 + i)[0] for i in range(n_sets - 1)]
+    shapes = [m.shape for m in mats0]
+    dev_sets = [[torch.from_numpy(m).to(dev) for m in hs] for hs in host_sets]
+    k_cap = api.default_k_cap(s, max(min(sh) for sh in shapes))
+    payload = torch.empty(api.payload_bytes_spectral(shapes, k_cap), dtype=torch.uint8, device=dev)
+    outs = [torch.empty(sh, dtype=torch.float32, device=dev) for sh in shapes]
+
+    def step(i, layers):
+        pay, _ = a.atomo_encode_spectral(layers, s, seed, step=i, k_cap=k_cap, payload=payload)
+        a.atomo_decode(pay, out=outs)
+        return pay
+
+    # ---- warm-up ----
+    for w in range(args.warmup):
+        step(w, dev_sets[w % n_sets])
+    torch.cuda.synchronize()
+
+    # ---- timed region: device-resident inputs ----
+    a.set_profiling(True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    dist.barrier(); torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    eig_ms = eig_launches = 0.0
+    launches = 0
+    sweeps_seen = None
+    ev0.record()
+    for k in range(args.steps):
+        pay, _ = a.atomo_encode_spectral(dev_sets[(args.warmup + k) % n_sets], s, seed, step=args.warmup + k,
+                                         k_cap=k_cap, payload=payload)
+        ms, ln = a.stage_times()                   # encode has finished its host-side waits here
+        eig_ms += ms["eig"]; eig_launches += ln["eig"]
+        launches += sum(ln.values()) + 7           # + header/descriptor copies and the workspace memset
+        a.atomo_decode(pay, out=outs)
+        launches += 3
+        if k == args.steps - 1:
+            sweeps_seen = [h.sweeps for h in pay.headers()[1]]
+    ev1.record()
+    torch.cuda.synchronize(); dist.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = ev0.elapsed_time(ev1)
+    ms_total = dist.max_over_ranks(ms_total, dev)
+    a.set_profiling(False)
+    ms_per_step = ms_total / args.steps
+    value = world * elems * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end: host buffers, copies inside the timed region ----
+    pinned = [[torch.from_numpy(m).pin_memory() for m in hs] for hs in host_sets]
+    stage_in = [torch.empty(sh, dtype=torch.float32, device=dev) for sh in shapes]
+    host_out = [torch.empty(sh, dtype=torch.float32).pin_memory() for sh in shapes]
+
+    def e2e_step(i):
+        src = pinned[i % n_sets]
+        for d, h in zip(stage_in, src):
+            d.copy_(h, non_blocking=True)
+        pay, _ = a.atomo_encode_spectral(stage_in, s, seed, step=i, k_cap=k_cap, payload=payload)
+        a.atomo_decode(pay, out=outs)
+        for h, d in zip(host_out, outs):
+            h.copy_(d, non_blocking=True)
+
+    for w in range(max(3, min(args.warmup, 5))):
+        e2e_step(w)
+    dist.barrier(); torch.cuda.synchronize()
+    e2e_steps = max(3, args.steps // 2)
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for k in range(e2e_steps):
+        e2e_step(100 + k)
+    t1.record()
+    torch.cuda.synchronize(); dist.barrier()
+    e2e_ms = dist.max_over_ranks(t0.elapsed_time(t1), dev)
+    e2e_value = world * elems * e2e_steps / (e2e_ms * 1e-3)
+
+    if rank == 0:
+        peaks = measured_peaks()
+        flops = jacobi_flops(shapes, sweeps_seen)          # of the last step; sweeps vary little between steps
+        eig_s_per_step = eig_ms * 1e-3 / args.steps
+        launches_per_step = eig_launches / args.steps
+        achieved = flops / eig_s_per_step / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "c2: ResNet-18-shaped layer set (18 layers, 10,992,320 elements), spectral ATOMO "
+                                   "s=2, one batched encode + decode per step",
+                       "k_cap": k_cap, "l2": f"inputs rotate over {n_sets} distinct sets ({n_sets * in_bytes / 2**20:.0f} MiB "
+                                             f"> 126 MiB L2) so each step reads gradients from HBM",
+                       "jacobi_sweeps_last_step": sweeps_seen},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes,
+                    "ms_per_step": e2e_ms / e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "alu", "kernel": "sp_jacobi_step16_kernel", "achieved": achieved,
+                         "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_FMA_PEAK_TFLOPS,
+                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH,
+                         "launches_per_step": launches_per_step,
+                         "avg_launch_us": eig_s_per_step / max(launches_per_step, 1) * 1e6,
+                         "share_of_step": eig_ms / ms_total,
+                         "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz (no measured FP32 peak on file)",
+                         "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline_c2(seed)
+        print(json.dumps(line))
+    a.close()
+    dist.finish()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -166,6 +166,8 @@ __device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int&
 template <int T4>
 struct RowRegs { float4 v[T4]; };
 
+constexpr float kRowFloor = 1e-24f;
+
 // rotate rows (xp, xq) so that their first A4 float4 (the x-parts) become orthogonal.
 // Returns true if a rotation was applied.  All lanes take the same branch.
 template <int T4>
@@ -186,12 +188,15 @@ __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, in
     be += __shfl_xor_sync(0xffffffffu, be, o);
     ga += __shfl_xor_sync(0xffffffffu, ga, o);
   }
-  // skip when the rows are orthogonal to working precision, or one of them is zero (false for NaN)
-  if (!(fabsf(ga) > tol * sqrtf(al) * sqrtf(be))) return false;
+  // skip when the rows are orthogonal to working precision (also false for NaN), or when one of
+  // them is numerically zero: A is scaled to trace 1, so a squared row norm below kRowFloor is an
+  // eigenvalue below 1e-12 of the trace -- rounding noise of the fp32 Gram matrix, not signal
+  if (!(fabsf(ga) > tol * sqrtf(al) * sqrtf(be)) || al < kRowFloor || be < kRowFloor) return false;
   const float zeta = (be - al) / (2.0f * ga);
   const float tt = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
   const float c = 1.0f / sqrtf(fmaf(tt, tt, 1.0f));
   const float s = c * tt;
+  if (s == 0.0f) return false;          // the angle underflowed: nothing to do
 #pragma unroll
   for (int t = 0; t < T4; ++t) {
     const float4 a = xp.v[t], b = xq.v[t];

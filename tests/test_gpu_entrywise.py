@@ -1,0 +1,162 @@
+"""GPU parity: entry-wise ATOMO through the C ABI vs the fp64 oracle (bit-exact masks/indices)."""
+import numpy as np
+import pytest
+
+from paper_1806_04090_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def atomo():
+    import torch
+    from paper_1806_04090_b200 import api
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    a = api.Atomo(0)
+    yield a
+    a.close()
+
+
+def _run(atomo, oracle, vecs, s, seed, step=0, k_cap=None, offset=0):
+    import torch
+    dev = torch.device("cuda:0")
+    ts = []
+    for g in vecs:
+        buf = torch.zeros(g.size + offset, dtype=torch.float32, device=dev)
+        buf[offset:] = torch.from_numpy(g).to(dev)
+        ts.append(buf[offset:])
+    if k_cap is None:
+        k_cap = max(g.size for g in vecs)
+    pay, dbg = atomo.atomo_encode_entrywise(ts, s, seed, step=step, k_cap=k_cap, debug=True)
+    hdrs = pay.headers()
+    outs = atomo.atomo_decode(pay)
+    report = []
+    for l, g in enumerate(vecs):
+        arr = pay.layer_arrays(l, hdrs)
+        same, enc = parity.check_entrywise(atomo, oracle, g, ts[l], s, seed, step, arr, hdrs[1][l], dbg, l, report,
+                                           f"vec{l}[n={g.size},s={s:g}]")
+        out = outs[l].cpu().numpy()
+        # decode kernel: exactly the payload's values at the payload's indices, zeros elsewhere
+        want = np.zeros(g.size, dtype=np.float32)
+        want[arr["idx"].astype(np.int64)] = arr["val"]
+        assert np.array_equal(out, want)
+        if same:
+            ref = oracle.decode_entrywise(g.size, enc["idx"], enc["val"])
+            assert parity.rel(out, ref) <= parity.REL_TOL if enc["idx"].size else not out.any()
+    print("\n".join(report))
+    return pay, hdrs
+
+
+def test_config1_entrywise(atomo, oracle):
+    _run(atomo, oracle, [synth.c1_entrywise(0)], 64.0, seed=1, step=3)
+
+
+def test_qsgd_and_terngrad_budgets(atomo, oracle):
+    # Section 4: s = ||g||_1/||g||_2 and ||g||_1/||g||_inf; kept values are +-||g||_q
+    g = synth.c1_entrywise(1)
+    l1 = float(np.abs(g.astype(np.float64)).sum())
+    for nq in (float(np.linalg.norm(g.astype(np.float64))), float(np.abs(g).max())):
+        pay, hdrs = _run(atomo, oracle, [g], l1 / nq, seed=2)
+        arr = pay.layer_arrays(0, hdrs)
+        np.testing.assert_allclose(np.abs(arr["val"]), nq, rtol=2e-6)
+
+
+@pytest.mark.parametrize("s", [2000.0, 4095.5, 5000.0])
+def test_unbalanced_budgets_saturate(atomo, oracle, s):
+    pay, hdrs = _run(atomo, oracle, [synth.c1_entrywise(1)], s, seed=5)
+    assert hdrs[1][0].n_sat > 0
+
+
+@pytest.mark.parametrize("n", [1, 3, 5, 31, 4095, 4096, 4097, 12289, 1_000_003])
+def test_ragged_lengths(atomo, oracle, n):
+    g = synth.c4_entrywise(3, n=n)
+    _run(atomo, oracle, [g], max(0.5, n / 100.0), seed=9, step=17)
+
+
+def test_batch_and_layer_index(atomo, oracle):
+    vecs = [synth.c4_entrywise(1, n=5000), synth.c1_entrywise(2), synth.c4_entrywise(2, n=70001)]
+    _run(atomo, oracle, vecs, 40.0, seed=0xDEADBEEFCAFE, step=2 ** 31 + 5)
+
+
+def test_unaligned_pointer(atomo, oracle):
+    _run(atomo, oracle, [synth.c4_entrywise(4, n=10007)], 55.5, seed=4, offset=1)
+
+
+def test_zeros(atomo, oracle):
+    g = synth.c1_entrywise(3).copy()
+    g[::3] = 0.0
+    _run(atomo, oracle, [g], 3000.0, seed=8)      # s > number of non-zero atoms: all of them kept
+    pay, hdrs = _run(atomo, oracle, [np.zeros(5000, dtype=np.float32)], 10.0, seed=8)
+    assert hdrs[1][0].k == 0
+
+
+def test_deterministic(atomo):
+    import torch
+    g = torch.from_numpy(synth.c4_entrywise(5, n=300_001)).cuda()
+    p1, _ = atomo.atomo_encode_entrywise([g], 3000.0, seed=3, k_cap=5000)
+    p2, _ = atomo.atomo_encode_entrywise([g], 3000.0, seed=3, k_cap=5000)
+    h = p1.headers()[1][0]
+    a1, a2 = p1.layer_arrays(0), p2.layer_arrays(0)
+    assert h.k > 0 and np.array_equal(a1["idx"], a2["idx"]) and np.array_equal(a1["val"], a2["val"])
+    p3, _ = atomo.atomo_encode_entrywise([g], 3000.0, seed=4, k_cap=5000)
+    assert not np.array_equal(p3.layer_arrays(0)["idx"], a1["idx"])
+
+
+def test_device_side_errors(atomo):
+    import torch
+    g = synth.c1_entrywise(0).copy()
+    t = torch.from_numpy(g).cuda()
+    # more kept atoms than k_cap: status, k = 0, decode gives zeros (never a silent truncation)
+    pay, _ = atomo.atomo_encode_entrywise([t], 64.0, seed=1, k_cap=10)
+    assert atomo.payload_status(pay) == (3, 0)
+    assert pay.headers()[1][0].k == 0 and not atomo.atomo_decode(pay)[0].any()
+    g[7] = np.nan
+    pay, _ = atomo.atomo_encode_entrywise([torch.from_numpy(g).cuda()], 64.0, seed=1, k_cap=4096)
+    assert atomo.payload_status(pay) == (4, 0) and pay.headers()[1][0].k == 0
+    g[7] = np.inf
+    pay, _ = atomo.atomo_encode_entrywise([torch.from_numpy(g).cuda()], 64.0, seed=1, k_cap=4096)
+    assert atomo.payload_status(pay)[0] == 4
+
+
+def test_host_side_errors(atomo):
+    import torch
+    from paper_1806_04090_b200 import api
+    t = torch.ones(100, device="cuda")
+    for bad in (0.0, -2.0, float("nan"), float("inf")):
+        with pytest.raises(api.AtomoError) as e:
+            atomo.atomo_encode_entrywise([t], bad, seed=1)
+        assert e.value.code == 2
+    with pytest.raises(api.AtomoError) as e:
+        atomo.atomo_encode_entrywise([t], 5.0, seed=1, k_cap=50, payload=torch.empty(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == 3
+    # decode with the wrong shape: payload status, zeros written
+    pay, _ = atomo.atomo_encode_entrywise([t], 5.0, seed=1, k_cap=100)
+    pay.shapes = [(1, 99)]
+    out = atomo.atomo_decode(pay)[0]
+    assert not out.any() and atomo.payload_status(pay)[0] == 8
+
+
+def test_unbiased_on_gpu(atomo):
+    # Lemma 1 at a size the oracle never sees: the mean of many decodes approaches g
+    import torch
+    g = torch.from_numpy(synth.c4_entrywise(6, n=20000)).cuda()
+    acc = torch.zeros_like(g, dtype=torch.float64)
+    trials = 400
+    s = 2000.0
+    for t in range(trials):
+        pay, _ = atomo.atomo_encode_entrywise([g], s, seed=100 + t, k_cap=4000)
+        acc += atomo.atomo_decode(pay)[0].double()
+    mean = (acc / trials).cpu().numpy()
+    g64 = g.double().cpu().numpy()
+    p = np.minimum(1.0, np.abs(g64) * s / np.abs(g64).sum())       # balanced here
+    sd = np.sqrt(g64 ** 2 * (1 - p) / np.maximum(p, 1e-300) / trials)
+    assert np.all(np.abs(mean - g64) <= 6 * sd + 1e-12)
+    assert abs(np.sum(mean) - np.sum(g64)) <= 6 * np.sqrt(np.sum(sd ** 2))
+
+
+@pytest.mark.parametrize("frac", [0.001, 0.01, 0.1])
+def test_config4_full_size(atomo, oracle, frac):
+    # 25.6M Laplace(0, 1e-3) entries, budgets 0.1 %, 1 %, 10 % of the length, in the bench's launch configuration
+    g = synth.c4_entrywise(0)
+    _run(atomo, oracle, [g], frac * g.size, seed=7, step=1, k_cap=int(frac * g.size * 1.05) + 1000)
