@@ -147,6 +147,28 @@ int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload /*DEVICE*/,
                  const int64_t* rows, const int64_t* cols, float* const* out /*HOST array of DEVICE ptrs*/,
                  int32_t n_layers, void* stream);
 
+/* --- decode without allocation ---------------------------------------------------------------
+ * (The paper has no counterpart: this entry point exists for deployment, not for the method.)
+ * Same result as atomo_decode() for a spectral payload, for callers that must not allocate device
+ * memory: a process whose framework allocator already owns the whole GPU, a latency-critical
+ * section that cannot take cudaMalloc's device-wide synchronisation, a memory-capped job.  It needs
+ * no context and calls no cudaMalloc / cudaFree: the per-call tables (one descriptor per layer, one
+ * entry per 32 x 256 output tile) go into a fixed array inside the library image, about 130 KB that
+ * every GPU loading the library holds until the process exits.
+ *   - Limits: n_layers <= ATOMO_STATIC_MAX_LAYERS and at most ATOMO_STATIC_MAX_TILES output tiles in
+ *     all (sum over layers of ceil(rows/32) * ceil(cols/256)); beyond that ATOMO_ERR_CAPACITY is
+ *     returned and nothing is launched.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device made current); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array: it still holds the previous call's tables, which
+ *     the next call overwrites in stream order.  Two calls whose work overlaps on the GPU (different
+ *     streams, no dependency) race on it; serialise them.
+ * `device` is the CUDA ordinal; payload, rows, cols, out, stream as in atomo_decode().               */
+enum { ATOMO_STATIC_MAX_LAYERS = 64, ATOMO_STATIC_MAX_TILES = 8192 };
+int atomo_decode_spectral_static(int device, const void* payload /*DEVICE*/, const int64_t* rows,
+                                 const int64_t* cols, float* const* out /*HOST array of DEVICE ptrs*/,
+                                 int32_t n_layers, void* stream);
+
 /* --- status / introspection -----------------------------------------------------------------
  * Copies the payload header and the n_layers layer headers to HOST memory (synchronises
  * `stream`).  Either output may be NULL.                                                       */

@@ -28,7 +28,7 @@ EXPORTS = [
     "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
-    "atomo_set_eig_params",
+    "atomo_set_eig_params", "atomo_decode_spectral_static",
 ]
 
 
@@ -99,6 +99,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.atomo_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i64)]
     lib.atomo_set_eig_params.argtypes = [vp, i32, ctypes.c_float]
+    lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                                 ctypes.POINTER(vp), i32, vp]
     if path == LIB_PATH:
         _lib = lib
     return lib
@@ -191,6 +193,32 @@ class Payload:
         long_ = view(h.off_long, k * L, np.float32).reshape(k, L).copy()
         U, V = (short, long_) if rows <= cols else (long_, short)
         return dict(k=k, idx=idx, coef=val, U=U.T.copy(), V=V.T.copy())
+
+
+def atomo_decode_spectral_static(payload: "Payload", out: Sequence[torch.Tensor], device: Optional[int] = None,
+                                 stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
+    """Spectral decode that allocates nothing on the device: for processes whose framework
+    allocator owns the whole GPU, or that cannot take cudaMalloc's device-wide synchronisation
+    where they decode.  The caller supplies the output tensors; the per-call tables live in a fixed
+    array inside the library (limits: 64 layers, 8192 output tiles of 32 x 256).  Calls on one
+    device share that array, so they must not overlap on the GPU."""
+    lib = load_library()
+    if payload.kind != KIND_SPECTRAL:
+        raise ValueError("atomo_decode_spectral_static decodes spectral payloads only")
+    n = payload.n_layers
+    if len(out) != n:
+        raise ValueError("one output tensor per layer is required (this call does not allocate)")
+    dev = payload.buf.device.index if device is None else int(device)
+    rows = (ctypes.c_int64 * n)(*[r for r, _ in payload.shapes])
+    cols = (ctypes.c_int64 * n)(*[c for _, c in payload.shapes])
+    ptrs = (ctypes.c_void_p * n)(*[o.data_ptr() for o in out])
+    s = stream if stream is not None else torch.cuda.current_stream()
+    rc = lib.atomo_decode_spectral_static(dev, ctypes.c_void_p(payload.buf.data_ptr()), rows, cols, ptrs, n,
+                                          ctypes.c_void_p(s.cuda_stream))
+    if rc != 0:
+        raise AtomoError(rc, "atomo_decode_spectral_static",
+                         "batch exceeds the fixed table (64 layers / 8192 tiles)" if rc == 3 else "")
+    return list(out)
 
 
 class Atomo:
