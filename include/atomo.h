@@ -21,7 +21,8 @@
  *     s <= 0 or not finite, payload capacity too small) return at once and launch nothing.
  *     Problems only the device can see (more kept atoms than k_cap, NaN/Inf input, sweep cap
  *     hit) set the layer's status word in the payload header, leave that layer with k = 0
- *     (or, for ATOMO_ERR_NOT_CONVERGED, with its best result) and are read back with
+ *     (except ATOMO_ERR_NOT_CONVERGED on eigen-solver route 0, whose basis is orthonormal at any
+ *     sweep count and is kept) and are read back with
  *     atomo_payload_status().  Nothing is ever silently truncated: dropping kept atoms would
  *     bias the estimator of Eq. (2).
  *   - Randomness is counter based (Philox4x32-10): the output is a pure function of the
@@ -58,7 +59,7 @@ typedef enum {
   ATOMO_ERR_BUDGET = 2,        /* s <= 0, NaN or Inf                                               */
   ATOMO_ERR_CAPACITY = 3,      /* host: payload buffer too small; device: kept atoms > k_cap       */
   ATOMO_ERR_NONFINITE = 4,     /* NaN or Inf found in a gradient                                   */
-  ATOMO_ERR_NOT_CONVERGED = 5, /* eigen-solver hit its sweep cap (result still orthogonal, usable) */
+  ATOMO_ERR_NOT_CONVERGED = 5, /* eigen-solver hit its sweep cap (route 1: k = 0; route 0: result kept) */
   ATOMO_ERR_TIMEOUT = 6,       /* reserved for bounded device-side waits                           */
   ATOMO_ERR_CUDA = 7,          /* a CUDA runtime call failed; see atomo_last_cuda_error            */
   ATOMO_ERR_PAYLOAD = 8        /* decode: header does not match the shapes given                   */
@@ -185,8 +186,12 @@ int atomo_set_profiling(atomo_ctx* ctx, int enabled);
 int atomo_get_stage_times(atomo_ctx* ctx, float* ms /*HOST*/, int64_t* launches /*HOST*/);
 
 /* Eigen-solver knobs: max Jacobi sweeps (default 40) and the relative rotation threshold
- * (default 1e-6: rows p, q are rotated while |<x_p,x_q>| > tol ||x_p|| ||x_q||).               */
+ * (default 3e-7: rows p, q are rotated while |<x_p,x_q>| > tol ||x_p|| ||x_q||).               */
 int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol);
+/* Eigen-solver route.  1 (default): Cholesky factor of the Gram matrix, then one-sided Jacobi on the
+ * rows of its transpose (row i converges to sigma_i times eigenvector i).  0: one-sided Jacobi on the
+ * rows of [A | I] with accumulated eigenvectors -- slower, kept as a cross-check of route 1.        */
+int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode);
 
 #ifdef __cplusplus
 }

@@ -15,7 +15,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libatomo_b200.so")
+LIB_PATH = os.environ.get("ATOMO_B200_LIB", os.path.join(_HERE, "libatomo_b200.so"))
 
 KIND_SPECTRAL = 0
 KIND_ENTRYWISE = 1
@@ -28,7 +28,7 @@ EXPORTS = [
     "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
-    "atomo_set_eig_params", "atomo_decode_spectral_static",
+    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_decode_spectral_static",
 ]
 
 
@@ -99,6 +99,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.atomo_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i64)]
     lib.atomo_set_eig_params.argtypes = [vp, i32, ctypes.c_float]
+    lib.atomo_set_eig_mode.argtypes = [vp, i32]
     lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                  ctypes.POINTER(vp), i32, vp]
     if path == LIB_PATH:
@@ -380,6 +381,9 @@ class Atomo:
         ln = (ctypes.c_int64 * len(STAGES))()
         self._check(self.lib.atomo_get_stage_times(self._h, ms, ln), "atomo_get_stage_times")
         return {k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)}
+
+    def set_eig_mode(self, mode: int):
+        self._check(self.lib.atomo_set_eig_mode(self._h, int(mode)), "atomo_set_eig_mode")
 
     def set_eig_params(self, max_sweeps: int, tol: float):
         self._check(self.lib.atomo_set_eig_params(self._h, int(max_sweeps), float(tol)), "atomo_set_eig_params")

@@ -23,7 +23,8 @@ struct atomo_ctx {
   bool profiling = false;
   bool configured = false;
   int max_sweeps = 40;
-  float tol = 1e-6f;
+  float tol = 3e-7f;
+  int eig_mode = 1;                  // 1: Cholesky factor + Jacobi on its rows; 0: Jacobi on [A | I]
   std::string err;
 };
 
@@ -188,6 +189,12 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
   return ATOMO_OK;
 }
 
+int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode) {
+  if (!ctx || (mode != 0 && mode != 1)) return ATOMO_ERR_INVALID_ARG;
+  ctx->eig_mode = mode;
+  return ATOMO_OK;
+}
+
 // ==================================================================================================
 int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers, double s, uint64_t seed,
                           uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
@@ -215,7 +222,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
   std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles;
-  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0;
+  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
     const atomo_mat& m = layers[l];
@@ -223,14 +230,17 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d.tall = m.rows > m.cols;
     d.r = std::min(m.rows, m.cols); d.L = std::max(m.rows, m.cols);
     d.rp = next_pow2_at_least(d.r, 32);
-    d.B = d.rp <= 512 ? 16 : 8;
+    d.acc = ctx->eig_mode == 0 ? 1 : 0;
+    d.ldx = d.acc ? 2 * d.rp : d.rp;
+    if (d.ldx > 1024) return ATOMO_ERR_INVALID_ARG;   // route 0 holds rows of 2 rp floats: short side <= 512
+    d.B = 16;
     d.nb = d.rp / d.B;
     d.layer = (uint32_t)l; d.k_cap = lay[l].kc;
-    r_max = std::max(r_max, d.r);
+    r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
     for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
     for (int p = 0; p < d.nb / 2; ++p) (d.B == 16 ? pairs16 : pairs8).push_back({l, p, 0, 0});
-    if (d.B == 16) { rp16_max = std::max(rp16_max, d.rp); steps16 = std::max(steps16, d.nb - 1); }
+    if (d.B == 16) { rp16_max = std::max(rp16_max, d.ldx); steps16 = std::max(steps16, d.nb - 1); }
     else steps8 = std::max(steps8, d.nb - 1);
     d.bp_tiles = d.tall ? (d.L + sp_bp_rows_per_tile() - 1) / sp_bp_rows_per_tile()
                         : (d.L + sp_bp_cols_per_tile() - 1) / sp_bp_cols_per_tile();
@@ -274,8 +284,13 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
     size_t z0 = A.off;
     for (int l = 0; l < n_layers; ++l) L[l].rot_count = A.take<uint32_t>(max_sweeps);
-    for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * 2 * L[l].rp);
+    for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * L[l].ldx);
     zero_beg = zb; zero_bytes = A.off - z0;
+    for (int l = 0; l < n_layers; ++l) {
+      SpLayer& d = L[l];
+      if (d.acc) { d.A = d.X; d.lda = d.ldx; }
+      else { d.A = A.take<float>((size_t)d.r * d.r); d.lda = d.r; }
+    }
     need = A.off + 256;
     if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
   }
@@ -305,7 +320,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   launch_sp_init(d_layers, n_layers, nullptr, 0, st);
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
   launch_sp_scale(d_layers, n_layers, st);
-  stage_end(ctx, ATOMO_STAGE_GRAM, st, 4);
+  if (ctx->eig_mode != 0) launch_sp_cholesky(d_layers, n_layers, rp_max, st);
+  stage_end(ctx, ATOMO_STAGE_GRAM, st, 5);
   CK(cudaGetLastError());
 
   // ---- S1: eigen-solver; the host reads a convergence flag once per sweep of the largest layer ----

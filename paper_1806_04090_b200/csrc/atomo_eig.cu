@@ -1,0 +1,381 @@
+// Eigen-solver of the spectral path: eigenvalues and eigenvectors of the short-side Gram matrix
+// A = G G^T (or G^T G), i.e. sigma_i^2 and the short-side singular vectors of Section 5's SVD.
+//
+// Two routes share one Jacobi kernel:
+//   mode 1 (default)  sp_cholesky : A = L L^T (fp32, pivots below a noise floor are set to zero), then
+//                     one-sided (Hestenes) Jacobi on the rows of L^T.  Orthogonal row rotations J keep
+//                     (J L^T)^T (J L^T) = A; at convergence the rows are mutually orthogonal:
+//                     row i = sigma_i w_i^T, so A = sum_i sigma_i^2 w_i w_i^T.  No eigenvector accumulation.
+//   mode 0            one-sided Jacobi on the rows of X = [A | I]: row i is (x_i | v_i), x_i = v_i^T A; at
+//                     convergence x_i = lambda_i v_i^T.  Twice the row length and about twice the sweeps
+//                     (the rows of A start nearly parallel), kept as a cross-check.
+//
+// Blocks of 16 rows are paired round-robin; a CTA holds one block pair in shared memory, one warp per
+// rotation.  Row norms are tracked (alpha' = alpha - t gamma, beta' = beta + t gamma) and refreshed when
+// they cancel; rotations are applied in the scaled ("fast Givens") form, one FMA per element, with the
+// cosines collected in a per-row factor that is folded back when the block pair is stored.
+#include "atomo_kernels.cuh"
+
+namespace atomo {
+
+// round-robin tournament over n (even) players: pair `slot` of round `round`
+__device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int& q) {
+  const int m = n - 1;
+  if (slot == 0) { p = n - 1; q = round % m; }
+  else { p = (round + slot) % m; q = (round - slot + m) % m; }
+}
+
+// A is scaled to trace 1, so a squared row norm below this is an eigenvalue of A below 1e-12 (mode 0)
+// or a singular value of L below 1e-12 (mode 1): rounding noise of the fp32 Gram matrix, not signal.
+constexpr float kRowFloor = 1e-24f;
+constexpr int kJB = 16;                 // rows per block
+
+// One row held by a warp: lane l keeps float4 number l + 32 t (t < T4).
+template <int T4>
+struct RowRegs { float4 v[T4]; };
+
+template <int T4>
+__device__ __forceinline__ void load_row(RowRegs<T4>& x, const float* row, int lane, int V4) {
+#pragma unroll
+  for (int t = 0; t < T4; ++t)
+    x.v[t] = (lane + 32 * t < V4) ? reinterpret_cast<const float4*>(row)[lane + 32 * t] : make_float4(0.f, 0.f, 0.f, 0.f);
+}
+template <int T4>
+__device__ __forceinline__ void store_row(const RowRegs<T4>& x, float* row, int lane, int V4, float scale = 1.0f) {
+#pragma unroll
+  for (int t = 0; t < T4; ++t)
+    if (lane + 32 * t < V4) {
+      const float4 a = x.v[t];
+      reinterpret_cast<float4*>(row)[lane + 32 * t] = make_float4(a.x * scale, a.y * scale, a.z * scale, a.w * scale);
+    }
+}
+template <int T4>
+__device__ __forceinline__ float row_norm2(const RowRegs<T4>& x, int lane, int A4) {
+  float n = 0.f;
+#pragma unroll
+  for (int t = 0; t < T4; ++t)
+    if (lane + 32 * t < A4) {
+      const float4 a = x.v[t];
+      n = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, n))));
+    }
+  return warp_sum(n);
+}
+
+// One plane rotation of the stored rows (xp, xq); true rows are dp * xp and dq * xq, with tracked squared
+// norms np2, nq2 of their first A4 float4 (the part that is orthogonalised).  All lanes take the same branch.
+//   Rotate while the cosine of the angle between the rows exceeds tol.
+//   tan(2 theta) = 2 gamma / (beta - alpha), |theta| <= pi/4, from normalised quantities (no overflow for
+//   norm ratios up to 1e24): with g = gamma / (||x_p|| ||x_q||), tau = (beta - alpha) / (||x_p|| ||x_q||),
+//   h = sqrt(tau^2 + 4 g^2):  t = tan(theta) = 2 g sign(tau) / (h + |tau|).  Approximate rsqrt / reciprocal
+//   (about 2 ulp) are enough for t: an error there leaves a residual cosine of that relative size, far
+//   below tol.  The cosine c is then derived from t itself with a Newton step, so the applied
+//   transformation is orthogonal to 1 ulp.
+//   Scaled ("fast Givens") update, one FMA per element:  x_p' = c (x_p - t x_q),  x_q' = c (x_q + t x_p)
+//   becomes v_p += a v_q, v_q += b v_p(old) with a = -t d_q/d_p, b = t d_p/d_q, and d_p, d_q *= c.
+//   Norms are tracked: alpha' = alpha - t gamma, beta' = beta + t gamma; the shrinking one loses digits by
+//   cancellation and is recomputed from the row when it dropped by 1000x.  (A stale norm can only waste or
+//   postpone a rotation: a sweep that rotates nothing changes no norm, so the convergence test always sees
+//   norms computed from the rows.)
+template <int T4>
+__device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, float& np2, float& nq2, float& dp,
+                                            float& dq, int lane, int A4, float tol) {
+  float g0 = 0.f, g1 = 0.f;
+#pragma unroll
+  for (int t = 0; t < T4; ++t) {
+    if (lane + 32 * t < A4) {
+      const float4 a = xp.v[t], b = xq.v[t];
+      g0 = fmaf(a.x, b.x, fmaf(a.y, b.y, g0));
+      g1 = fmaf(a.z, b.z, fmaf(a.w, b.w, g1));
+    }
+  }
+  const float al = np2, be = nq2;
+  const float m = rsqrtf(al) * rsqrtf(be);                   // independent of the reduction below
+  const float ratio_qp = __fdividef(dq, dp), ratio_pq = __fdividef(dp, dq);
+  const float ga = warp_sum(g0 + g1) * dp * dq;
+  if (al < kRowFloor || be < kRowFloor) return false;
+  const float gn = ga * m;                                   // cosine of the angle between the rows
+  if (!(fabsf(gn) > tol)) return false;                      // also false for NaN
+  const float tau = (be - al) * m;
+  const float q = fmaf(tau, tau, 4.0f * gn * gn);
+  const float h = q * rsqrtf(q);
+  const float tt = copysignf(2.0f * gn, gn * tau) * __fdividef(1.0f, h + fabsf(tau));
+  if (tt == 0.0f) return false;
+  const float a = -tt * ratio_qp, b = tt * ratio_pq;
+#pragma unroll
+  for (int t = 0; t < T4; ++t) {
+    const float4 u = xp.v[t], w = xq.v[t];
+    xp.v[t] = make_float4(fmaf(a, w.x, u.x), fmaf(a, w.y, u.y), fmaf(a, w.z, u.z), fmaf(a, w.w, u.w));
+    xq.v[t] = make_float4(fmaf(b, u.x, w.x), fmaf(b, u.y, w.y), fmaf(b, u.z, w.z), fmaf(b, u.w, w.w));
+  }
+  const float y = fmaf(tt, tt, 1.0f);
+  float c = rsqrtf(y);
+  c = c * fmaf(-0.5f * y * c, c, 1.5f);
+  dp *= c; dq *= c;
+  const float tg = tt * ga;
+  np2 = al - tg; nq2 = be + tg;
+  if (np2 < 1e-3f * al) np2 = row_norm2<T4>(xp, lane, A4) * dp * dp;
+  if (nq2 < 1e-3f * be) nq2 = row_norm2<T4>(xq, lane, A4) * dq * dq;
+  return true;
+}
+
+// One block pair (2 x 16 rows) of one layer, resident in shared memory, 16 warps, one warp per rotation.
+// RP = padded short side; ACC: rows are [x | v] (2 RP floats, mode 0), else x only (RP floats, mode 1).
+template <int RP, bool ACC>
+__device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, float tol,
+                                                  float* smem) {
+  constexpr int B = kJB;
+  constexpr int LD = ACC ? 2 * RP : RP, V4 = LD / 4, A4 = RP / 4, T4 = (V4 + 31) / 32;
+  constexpr int NT = 32 * B;
+  static_assert(T4 <= 8, "row too long for one warp");
+  float* s_n2 = smem + 2 * B * LD;       // squared norms of the true rows
+  float* s_d = s_n2 + 2 * B;             // true row = s_d * stored row
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  int bi, bj;
+  rr_pair(L.nb, local, slot, bi, bj);
+  float* X = L.X;
+#ifdef ATOMO_PHASE_TIMING
+  long long tk[8]; int nk = 0;
+#define ATOMO_TICK() tk[nk++] = clock64()
+#else
+#define ATOMO_TICK()
+#endif
+  ATOMO_TICK();
+  // ---- load 2B rows ----
+  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
+    const int row = idx / V4, q = idx % V4;
+    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
+    reinterpret_cast<float4*>(smem + row * LD)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * LD)[q];
+  }
+  __syncthreads();
+  RowRegs<T4> xp, xq;
+  // warp w: squared norms of rows w and w + B; row w stays in registers for the cross rounds
+  load_row<T4>(xq, smem + (B + w) * LD, lane, V4);
+  const float nj = row_norm2<T4>(xq, lane, A4);
+  load_row<T4>(xp, smem + w * LD, lane, V4);
+  float np2 = row_norm2<T4>(xp, lane, A4), dp = 1.0f;
+  if (lane == 0) { s_n2[w] = np2; s_n2[B + w] = nj; s_d[w] = 1.0f; s_d[B + w] = 1.0f; }
+  __syncthreads();
+  ATOMO_TICK();
+  uint32_t nrot = 0;
+  // ---- pairs inside each block: once per sweep ----
+  if (local == 0) {
+    for (int round = 0; round < B - 1; ++round) {
+      const int blk = w / (B / 2), sl = w % (B / 2);
+      int p, q;
+      rr_pair(B, round, sl, p, q);
+      p += blk * B; q += blk * B;
+      float* rowp = smem + p * LD;
+      float* rowq = smem + q * LD;
+      load_row<T4>(xp, rowp, lane, V4);
+      load_row<T4>(xq, rowq, lane, V4);
+      float a2 = s_n2[p], b2 = s_n2[q], da = s_d[p], db = s_d[q];
+      if (rotate_pair<T4>(xp, xq, a2, b2, da, db, lane, A4, tol)) {
+        store_row<T4>(xp, rowp, lane, V4);
+        store_row<T4>(xq, rowq, lane, V4);
+        if (lane == 0) { s_n2[p] = a2; s_n2[q] = b2; s_d[p] = da; s_d[q] = db; }
+        ++nrot;
+      }
+      __syncthreads();
+    }
+    load_row<T4>(xp, smem + w * LD, lane, V4);
+    np2 = s_n2[w]; dp = s_d[w];
+  }
+  ATOMO_TICK();
+  // ---- pairs across the two blocks: warp w keeps row w of block bi in registers; the rows of block bj
+  //      visit the warps round-robin ----
+  for (int round = 0; round < B; ++round) {
+    const int j = B + (w + round) % B;
+    float* rowq = smem + j * LD;
+    load_row<T4>(xq, rowq, lane, V4);
+    float nq2 = s_n2[j], dq = s_d[j];
+    if (rotate_pair<T4>(xp, xq, np2, nq2, dp, dq, lane, A4, tol)) {
+      store_row<T4>(xq, rowq, lane, V4);
+      if (lane == 0) { s_n2[j] = nq2; s_d[j] = dq; }
+      ++nrot;
+    }
+    __syncthreads();
+  }
+  ATOMO_TICK();
+  store_row<T4>(xp, smem + w * LD, lane, V4, dp);
+  if (lane == 0) s_d[w] = 1.0f;
+  __syncthreads();
+  // ---- store, folding the collected cosines back into the rows ----
+  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
+    const int row = idx / V4, q = idx % V4;
+    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
+    const float d = s_d[row];
+    const float4 a = reinterpret_cast<const float4*>(smem + row * LD)[q];
+    reinterpret_cast<float4*>(X + (int64_t)grow * LD)[q] = make_float4(a.x * d, a.y * d, a.z * d, a.w * d);
+  }
+  if (lane == 0 && nrot) atomicAdd(L.rot_count + sweep, nrot);
+  ATOMO_TICK();
+#ifdef ATOMO_PHASE_TIMING
+  if (tid == 0 && slot == 0 && (sweep == 2 || sweep == 8) && local < 2)
+    printf("rp %d acc %d sweep %d local %d: load+norm %lld intra %lld cross %lld store %lld (clk) nrot(w0) %u\n", RP, (int)ACC,
+           sweep, local, tk[1] - tk[0], tk[2] - tk[1], tk[3] - tk[2], tk[4] - tk[3], nrot);
+#endif
+}
+
+constexpr int kJacobiThreads = 32 * kJB;
+
+// One Jacobi step for every layer: mode 1 layers with padded short side <= 1024, mode 0 layers with <= 512.
+__global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const SpLayer* __restrict__ layers,
+                                                                        const TileRef* __restrict__ pairs, int t,
+                                                                        int max_sweeps, float tol) {
+  extern __shared__ __align__(16) float smem[];
+  const TileRef ref = pairs[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int steps = L.nb - 1;
+  const int sweep = t / steps, local = t % steps;
+  if (sweep >= max_sweeps) return;
+  if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
+  if (L.acc) {
+    switch (L.rp) {
+      case 32: jacobi_block_pair<32, true>(L, ref.a, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, true>(L, ref.a, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, true>(L, ref.a, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, true>(L, ref.a, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, true>(L, ref.a, sweep, local, tol, smem); break;
+      default: break;
+    }
+  } else {
+    switch (L.rp) {
+      case 32: jacobi_block_pair<32, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 1024: jacobi_block_pair<1024, false>(L, ref.a, sweep, local, tol, smem); break;
+      default: break;
+    }
+  }
+}
+
+constexpr int kJacobiSmem = 32 * 1024 * 4 + 512;   // 32 rows of up to 1024 floats + norms and factors
+
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
+                           int t, int max_sweeps, float tol, cudaStream_t st) {
+  if (n_pairs <= 0) return;
+  (void)B;
+  const int smem = 32 * row_floats_max * 4 + 512;
+  sp_jacobi_step_kernel<<<n_pairs, kJacobiThreads, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
+}
+
+// convergence bookkeeping after t16 / t8 steps have been enqueued for the two kernel classes
+__global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers, int t16, int t8, int max_sweeps,
+                                uint32_t* all_done) {
+  __shared__ int s_pending;
+  if (threadIdx.x == 0) s_pending = 0;
+  __syncthreads();
+  for (int l = threadIdx.x; l < n_layers; l += blockDim.x) {
+    const SpLayer& L = layers[l];
+    const int steps = L.nb - 1;
+    const int t_done = (L.B == 16) ? t16 : t8;
+    const int sweeps_done = min(t_done / steps, max_sweeps);
+    int conv = -1;
+    for (int wv = 0; wv < sweeps_done; ++wv) if (L.rot_count[wv] == 0) { conv = wv; break; }
+    if (conv >= 0) L.hdr->sweeps = (uint32_t)(conv + 1);
+    else {
+      L.hdr->sweeps = (uint32_t)sweeps_done;
+      if (sweeps_done < max_sweeps) atomicAdd(&s_pending, 1);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) *all_done = s_pending == 0 ? 1u : 0u;
+}
+
+void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
+                     cudaStream_t st) {
+  sp_check_kernel<<<1, 256, 0, st>>>(d_layers, n_layers, t16, t8, max_sweeps, d_all_done);
+}
+
+// =================================================================================================
+// Cholesky factor of the scaled Gram matrix, written transposed: X[c][i] = L[i][c].
+// One CTA per layer, one thread per row, left-looking over panels of 32 columns; a thread keeps its
+// row of the current panel in registers.  A pivot below kPivotFloor (trace(A) = 1) is rounding noise
+// of the fp32 Gram matrix: that column of L is set to zero (L L^T then differs from A by that noise).
+// =================================================================================================
+constexpr float kPivotFloor = 1e-9f;
+constexpr int kCholPanel = 32;
+
+__global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  if (L.acc) return;
+  __shared__ float s_k[kCholPanel][kCholPanel + 1];     // L[j0 + c][k0 + kk] for the current k chunk
+  __shared__ float s_ldd[kCholPanel][kCholPanel + 1];   // diagonal block of L
+  __shared__ float s_inv[kCholPanel];
+  const int r = L.r, rp = L.rp;
+  const int i = threadIdx.x, lane = i % 32, warp = i / 32;
+  const float* __restrict__ A = L.A;
+  const int64_t lda = L.lda;
+  float* X = L.X;
+  for (int j0 = 0; j0 < r; j0 += kCholPanel) {
+    const bool active = i >= j0 && i < r;
+    float p[kCholPanel];
+#pragma unroll
+    for (int c = 0; c < kCholPanel; ++c) p[c] = (active && j0 + c < r) ? A[(int64_t)(j0 + c) * lda + i] : 0.0f;
+    // p[c] -= sum_{k < j0} L[i][k] L[j0+c][k]
+    for (int k0 = 0; k0 < j0; k0 += kCholPanel) {
+      __syncthreads();
+      for (int idx = i; idx < kCholPanel * kCholPanel; idx += blockDim.x) {
+        const int kk = idx / kCholPanel, c = idx % kCholPanel;
+        s_k[kk][c] = X[(int64_t)(k0 + kk) * rp + j0 + c];
+      }
+      __syncthreads();
+      if (active) {
+#pragma unroll 4
+        for (int kk = 0; kk < kCholPanel; ++kk) {
+          const float xi = X[(int64_t)(k0 + kk) * rp + i];
+#pragma unroll
+          for (int c = 0; c < kCholPanel; ++c) p[c] = fmaf(-xi, s_k[kk][c], p[c]);
+        }
+      }
+    }
+    // diagonal block: the warp whose lanes own rows j0 .. j0+31
+    if (warp == j0 / 32) {
+#pragma unroll
+      for (int c = 0; c < kCholPanel; ++c) {
+        const float d = __shfl_sync(0xffffffffu, p[c], c);
+        const float lcc = d > kPivotFloor ? sqrtf(d) : 0.0f;
+        const float inv = lcc > 0.0f ? 1.0f / lcc : 0.0f;
+        const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
+        p[c] = lic;
+#pragma unroll
+        for (int c2 = c + 1; c2 < kCholPanel; ++c2) {
+          const float l2 = __shfl_sync(0xffffffffu, lic, c2);
+          if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+        }
+        if (lane == c) s_inv[c] = inv;
+      }
+#pragma unroll
+      for (int c = 0; c < kCholPanel; ++c) s_ldd[lane][c] = p[c];
+    }
+    __syncthreads();
+    // rows below the diagonal block: solve y L_dd^T = p
+    if (active && i >= j0 + kCholPanel) {
+#pragma unroll
+      for (int c = 0; c < kCholPanel; ++c) {
+        float acc = p[c];
+#pragma unroll
+        for (int k = 0; k < c; ++k) acc = fmaf(-p[k], s_ldd[c][k], acc);
+        p[c] = acc * s_inv[c];
+      }
+    }
+    if (active) {
+#pragma unroll
+      for (int c = 0; c < kCholPanel; ++c)
+        if (j0 + c < r) X[(int64_t)(j0 + c) * rp + i] = p[c];
+    }
+    __syncthreads();
+  }
+}
+
+void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
+  sp_cholesky_kernel<<<n_layers, rp_max, 0, st>>>(d_layers);
+}
+
+int sp_configure_eig() {
+  return (int)cudaFuncSetAttribute(sp_jacobi_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+}
+
+}  // namespace atomo

@@ -53,7 +53,10 @@ struct SpLayer {
   int r, L, tall;              // short side, long side, rows > cols
   int rp, B, nb;               // padded short side, Jacobi block rows, number of blocks (even)
   uint32_t layer, k_cap;
-  float* X;                    // rp x 2rp: row i = [ x_i (rp) | v_i (rp) ],  x_i = v_i^T A
+  int acc;                     // eigen-solver route: 1 = rows [x | v] of [A | I] (mode 0), 0 = rows of L^T (mode 1)
+  int ldx;                     // floats per row of X: 2 rp (acc) or rp
+  float* A; int64_t lda;       // scaled Gram matrix, r x r valid (mode 0: the left half of X)
+  float* X;                    // rp x ldx working rows of the Jacobi solver
   atomo_layer_header* hdr;     // payload
   uint32_t* idx; float* coef; float* shortv; float* longv;
   float* lam;                  // rp   eigenvalue per row (unsorted, scaled)
@@ -78,8 +81,10 @@ void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling
 // one Jacobi step (global step index t) for every layer of one (B, RP) class
-void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int rp,
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
+void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
+int sp_configure_eig();
 // convergence bookkeeping after t16 / t8 steps were enqueued for the two kernel classes
 void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st);

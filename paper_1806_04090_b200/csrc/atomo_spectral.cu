@@ -25,7 +25,8 @@ namespace atomo {
 // =================================================================================================
 __global__ void sp_init_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
-  const int64_t ldx = 2 * (int64_t)L.rp;
+  if (!L.acc) return;
+  const int64_t ldx = L.ldx;
   for (int i = blockIdx.y * blockDim.x + threadIdx.x; i < L.rp; i += gridDim.y * blockDim.x)
     L.X[(int64_t)i * ldx + L.rp + i] = 1.0f;
 }
@@ -102,7 +103,7 @@ __global__ void __launch_bounds__(256) sp_gram_kernel(const SpLayer* __restrict_
         for (int q = 0; q < 4; ++q) { acc64[p][q] += (double)acc[p][q]; acc[p][q] = 0.0f; }
     }
   }
-  const int64_t ldx = 2 * (int64_t)L.rp;
+  const int64_t lda = L.lda;
 #pragma unroll
   for (int p = 0; p < 4; ++p)
 #pragma unroll
@@ -110,8 +111,8 @@ __global__ void __launch_bounds__(256) sp_gram_kernel(const SpLayer* __restrict_
       const int i = i0 + ty * 4 + p, j = j0 + tx * 4 + q;
       if (i < r && j < r) {
         const float v = (float)(acc64[p][q] + (double)acc[p][q]);
-        L.X[(int64_t)i * ldx + j] = v;
-        if (!diag) L.X[(int64_t)j * ldx + i] = v;
+        L.A[(int64_t)i * lda + j] = v;
+        if (!diag) L.A[(int64_t)j * lda + i] = v;
       }
     }
 }
@@ -125,10 +126,10 @@ void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles
 // =================================================================================================
 __global__ void __launch_bounds__(256) sp_trace_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
-  const int64_t ldx = 2 * (int64_t)L.rp;
+  const int64_t lda = L.lda;
   __shared__ float s_red[256];
   float tr = 0.0f;
-  for (int i = threadIdx.x; i < L.r; i += 256) tr += L.X[(int64_t)i * ldx + i];
+  for (int i = threadIdx.x; i < L.r; i += 256) tr += L.A[(int64_t)i * lda + i];
   s_red[threadIdx.x] = tr;
   __syncthreads();
   for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
@@ -141,228 +142,16 @@ __global__ void __launch_bounds__(256) sp_trace_kernel(const SpLayer* __restrict
 
 __global__ void __launch_bounds__(256) sp_scale_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
-  const int64_t ldx = 2 * (int64_t)L.rp;
+  const int64_t lda = L.lda;
   const float sc = *L.scale;
   if (sc == 1.0f) return;
   for (int i = blockIdx.y; i < L.r; i += gridDim.y)
-    for (int j = threadIdx.x; j < L.r; j += 256) L.X[(int64_t)i * ldx + j] *= sc;
+    for (int j = threadIdx.x; j < L.r; j += 256) L.A[(int64_t)i * lda + j] *= sc;
 }
 
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
   sp_trace_kernel<<<n_layers, 256, 0, st>>>(d_layers);
   sp_scale_kernel<<<dim3(n_layers, 32), 256, 0, st>>>(d_layers);
-}
-
-// =================================================================================================
-// One-sided Jacobi, block pair resident in shared memory.
-// =================================================================================================
-// round-robin tournament over n (even) players: pair `slot` of round `round`
-__device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int& q) {
-  const int m = n - 1;
-  if (slot == 0) { p = n - 1; q = round % m; }
-  else { p = (round + slot) % m; q = (round - slot + m) % m; }
-}
-
-template <int T4>
-struct RowRegs { float4 v[T4]; };
-
-constexpr float kRowFloor = 1e-24f;
-
-// rotate rows (xp, xq) so that their first A4 float4 (the x-parts) become orthogonal.
-// Returns true if a rotation was applied.  All lanes take the same branch.
-template <int T4>
-__device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, int lane, int A4, float tol) {
-  float al = 0.f, be = 0.f, ga = 0.f;
-#pragma unroll
-  for (int t = 0; t < T4; ++t) {
-    if (lane + 32 * t < A4) {
-      const float4 a = xp.v[t], b = xq.v[t];
-      al = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, al))));
-      be = fmaf(b.x, b.x, fmaf(b.y, b.y, fmaf(b.z, b.z, fmaf(b.w, b.w, be))));
-      ga = fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, fmaf(a.w, b.w, ga))));
-    }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    al += __shfl_xor_sync(0xffffffffu, al, o);
-    be += __shfl_xor_sync(0xffffffffu, be, o);
-    ga += __shfl_xor_sync(0xffffffffu, ga, o);
-  }
-  // skip when the rows are orthogonal to working precision (also false for NaN), or when one of
-  // them is numerically zero: A is scaled to trace 1, so a squared row norm below kRowFloor is an
-  // eigenvalue below 1e-12 of the trace -- rounding noise of the fp32 Gram matrix, not signal
-  if (!(fabsf(ga) > tol * sqrtf(al) * sqrtf(be)) || al < kRowFloor || be < kRowFloor) return false;
-  const float zeta = (be - al) / (2.0f * ga);
-  const float tt = copysignf(1.0f, zeta) / (fabsf(zeta) + sqrtf(fmaf(zeta, zeta, 1.0f)));
-  const float c = 1.0f / sqrtf(fmaf(tt, tt, 1.0f));
-  const float s = c * tt;
-  if (s == 0.0f) return false;          // the angle underflowed: nothing to do
-#pragma unroll
-  for (int t = 0; t < T4; ++t) {
-    const float4 a = xp.v[t], b = xq.v[t];
-    xp.v[t] = make_float4(fmaf(c, a.x, -s * b.x), fmaf(c, a.y, -s * b.y), fmaf(c, a.z, -s * b.z), fmaf(c, a.w, -s * b.w));
-    xq.v[t] = make_float4(fmaf(s, a.x, c * b.x), fmaf(s, a.y, c * b.y), fmaf(s, a.z, c * b.z), fmaf(s, a.w, c * b.w));
-  }
-  return true;
-}
-
-template <int T4>
-__device__ __forceinline__ void load_row(RowRegs<T4>& x, const float* row, int lane, int V4) {
-#pragma unroll
-  for (int t = 0; t < T4; ++t)
-    x.v[t] = (lane + 32 * t < V4) ? reinterpret_cast<const float4*>(row)[lane + 32 * t] : make_float4(0.f, 0.f, 0.f, 0.f);
-}
-template <int T4>
-__device__ __forceinline__ void store_row(const RowRegs<T4>& x, float* row, int lane, int V4) {
-#pragma unroll
-  for (int t = 0; t < T4; ++t)
-    if (lane + 32 * t < V4) reinterpret_cast<float4*>(row)[lane + 32 * t] = x.v[t];
-}
-
-// One block pair of one layer.  B rows per block, B warps; RP = padded short side (row = 2 RP floats).
-template <int B, int RP>
-__device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, float tol,
-                                                  float* smem) {
-  constexpr int LD = 2 * RP, V4 = LD / 4, A4 = RP / 4, T4 = (V4 + 31) / 32;
-  constexpr int NT = 32 * B;
-  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
-  int bi, bj;
-  rr_pair(L.nb, local, slot, bi, bj);
-  float* X = L.X;
-  // ---- load 2B rows ----
-  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
-    const int row = idx / V4, q = idx % V4;
-    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
-    reinterpret_cast<float4*>(smem + row * LD)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * LD)[q];
-  }
-  __syncthreads();
-  uint32_t nrot = 0;
-  RowRegs<T4> xp, xq;
-  // ---- pairs inside each block: once per sweep ----
-  if (local == 0) {
-    for (int round = 0; round < B - 1; ++round) {
-      if (w < B) {
-        const int blk = w / (B / 2), sl = w % (B / 2);
-        int p, q;
-        rr_pair(B, round, sl, p, q);
-        float* rowp = smem + (blk * B + p) * LD;
-        float* rowq = smem + (blk * B + q) * LD;
-        load_row<T4>(xp, rowp, lane, V4);
-        load_row<T4>(xq, rowq, lane, V4);
-        if (rotate_pair<T4>(xp, xq, lane, A4, tol)) {
-          store_row<T4>(xp, rowp, lane, V4);
-          store_row<T4>(xq, rowq, lane, V4);
-          ++nrot;
-        }
-      }
-      __syncthreads();
-    }
-  }
-  // ---- pairs across the two blocks: warp w keeps row w of block bi in registers ----
-  if (w < B) load_row<T4>(xp, smem + w * LD, lane, V4);
-  for (int round = 0; round < B; ++round) {
-    if (w < B) {
-      float* rowq = smem + (B + (w + round) % B) * LD;
-      load_row<T4>(xq, rowq, lane, V4);
-      if (rotate_pair<T4>(xp, xq, lane, A4, tol)) {
-        store_row<T4>(xq, rowq, lane, V4);
-        ++nrot;
-      }
-    }
-    __syncthreads();
-  }
-  if (w < B) store_row<T4>(xp, smem + w * LD, lane, V4);
-  __syncthreads();
-  // ---- store ----
-  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
-    const int row = idx / V4, q = idx % V4;
-    const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
-    reinterpret_cast<float4*>(X + (int64_t)grow * LD)[q] = reinterpret_cast<const float4*>(smem + row * LD)[q];
-  }
-  if (lane == 0 && nrot) atomicAdd(L.rot_count + sweep, nrot);
-}
-
-// All layers whose padded short side is <= 512: B = 16, 512 threads, one launch per step.
-__global__ void __launch_bounds__(512) sp_jacobi_step16_kernel(const SpLayer* __restrict__ layers,
-                                                               const TileRef* __restrict__ pairs, int t,
-                                                               int max_sweeps, float tol) {
-  extern __shared__ __align__(16) float smem[];
-  const TileRef ref = pairs[blockIdx.x];
-  const SpLayer& L = layers[ref.layer];
-  const int steps = L.nb - 1;
-  const int sweep = t / steps, local = t % steps;
-  if (sweep >= max_sweeps) return;
-  if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
-  switch (L.rp) {
-    case 32: jacobi_block_pair<16, 32>(L, ref.a, sweep, local, tol, smem); break;
-    case 64: jacobi_block_pair<16, 64>(L, ref.a, sweep, local, tol, smem); break;
-    case 128: jacobi_block_pair<16, 128>(L, ref.a, sweep, local, tol, smem); break;
-    case 256: jacobi_block_pair<16, 256>(L, ref.a, sweep, local, tol, smem); break;
-    case 512: jacobi_block_pair<16, 512>(L, ref.a, sweep, local, tol, smem); break;
-    default: break;
-  }
-}
-
-// Layers with padded short side 1024: B = 8, 256 threads.
-__global__ void __launch_bounds__(256) sp_jacobi_step8_kernel(const SpLayer* __restrict__ layers,
-                                                              const TileRef* __restrict__ pairs, int t,
-                                                              int max_sweeps, float tol) {
-  extern __shared__ __align__(16) float smem[];
-  const TileRef ref = pairs[blockIdx.x];
-  const SpLayer& L = layers[ref.layer];
-  const int steps = L.nb - 1;
-  const int sweep = t / steps, local = t % steps;
-  if (sweep >= max_sweeps) return;
-  if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;
-  jacobi_block_pair<8, 1024>(L, ref.a, sweep, local, tol, smem);
-}
-
-constexpr int kJacobiSmem = 2 * 16 * 2 * 512 * 4;   // 128 KB: 32 rows of 1024 floats (or 16 rows of 2048)
-
-__global__ void sp_backproject_kernel(const SpLayer* __restrict__ layers, const TileRef* __restrict__ tiles);
-
-int sp_configure() {
-  cudaError_t e = cudaFuncSetAttribute(sp_jacobi_step16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
-  if (e != cudaSuccess) return (int)e;
-  e = cudaFuncSetAttribute(sp_jacobi_step8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
-  if (e != cudaSuccess) return (int)e;
-  e = cudaFuncSetAttribute(sp_backproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           8 * kMaxShort * (int)sizeof(float));
-  return (int)e;
-}
-
-void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int rp_max,
-                           int t, int max_sweeps, float tol, cudaStream_t st) {
-  if (n_pairs <= 0) return;
-  if (B == 16) {
-    const int smem = 2 * 16 * 2 * rp_max * 4;
-    sp_jacobi_step16_kernel<<<n_pairs, 512, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
-  } else {
-    sp_jacobi_step8_kernel<<<n_pairs, 256, kJacobiSmem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
-  }
-}
-
-// convergence bookkeeping after `t_done[group]` steps have been enqueued for each group
-__global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers, int t16, int t8, int max_sweeps,
-                                uint32_t* all_done) {
-  __shared__ int s_pending;
-  if (threadIdx.x == 0) s_pending = 0;
-  __syncthreads();
-  for (int l = threadIdx.x; l < n_layers; l += blockDim.x) {
-    const SpLayer& L = layers[l];
-    const int steps = L.nb - 1;
-    const int t_done = (L.B == 16) ? t16 : t8;
-    const int sweeps_done = min(t_done / steps, max_sweeps);
-    int conv = -1;
-    for (int wv = 0; wv < sweeps_done; ++wv) if (L.rot_count[wv] == 0) { conv = wv; break; }
-    if (conv >= 0) L.hdr->sweeps = (uint32_t)(conv + 1);
-    else {
-      L.hdr->sweeps = (uint32_t)sweeps_done;
-      if (sweeps_done < max_sweeps) atomicAdd(&s_pending, 1);
-    }
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) *all_done = s_pending == 0 ? 1u : 0u;
 }
 
 // =================================================================================================
@@ -382,17 +171,19 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   __shared__ uint32_t s_nsat, s_bad, s_k;
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const int r = L.r, rp = L.rp;
-  const int64_t ldx = 2 * (int64_t)rp;
+  const int64_t ldx = L.ldx;
+  const int voff = L.acc ? rp : 0;          // where the eigenvector sits in a row
   const float inv_scale = 1.0f / *L.scale;
   atomo_layer_header* h = L.hdr;
   if (tid == 0) { s_bad = 0; s_k = 0; }
   __syncthreads();
 
-  // lambda_i = <x_i, v_i>  (Rayleigh quotient of A at v_i), one warp per row
+  // eigenvalue of A per row, one warp per row.  mode 0: lambda_i = <x_i, v_i> (Rayleigh quotient at v_i);
+  // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T)
   for (int i = w; i < r; i += kFinThreads / 32) {
     const float* row = L.X + (int64_t)i * ldx;
     float d = 0.f;
-    for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[rp + j], d);
+    for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[voff + j], d);
     d = warp_sum(d);
     if (lane == 0) {
       const float lam = d * inv_scale;
@@ -472,7 +263,9 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
     else if (carry > L.k_cap) status = ATOMO_ERR_CAPACITY;
     else if (h->sweeps >= (uint32_t)max_sweeps && L.rot_count[max_sweeps - 1] != 0) status = ATOMO_ERR_NOT_CONVERGED;
     h->status = status;
-    const uint32_t k = (status == ATOMO_OK || status == ATOMO_ERR_NOT_CONVERGED) ? carry : 0u;
+    // route 0 keeps an orthonormal basis whatever the sweep count, so its unconverged result is still an
+    // unbiased estimator; route 1's rows are orthogonal only at convergence, so it keeps nothing
+    const uint32_t k = (status == ATOMO_OK || (status == ATOMO_ERR_NOT_CONVERGED && L.acc)) ? carry : 0u;
     h->k = k;
     s_k = k;
   }
@@ -481,25 +274,24 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   // short-side vectors of the kept atoms, normalised: payload shortv[a][0..r)
   for (uint32_t a = w; a < k; a += kFinThreads / 32) {
     const int row = L.perm[L.idx[a]];
-    const float* v = L.X + (int64_t)row * ldx + rp;
+    const float* v = L.X + (int64_t)row * ldx + voff;
     float n2 = 0.f;
     for (int j = lane; j < r; j += 32) n2 = fmaf(v[j], v[j], n2);
     n2 = warp_sum(n2);
     const float inv = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
     for (int j = lane; j < r; j += 32) L.shortv[(int64_t)a * r + j] = v[j] * inv;
   }
-  // optional: every short-side vector, rank-major
+  // optional: every short-side vector (normalised), rank-major
   if (L.dbg_short) {
     for (int a = w; a < r; a += kFinThreads / 32) {
-      const float* v = L.X + (int64_t)L.perm[a] * ldx + rp;
-      for (int j = lane; j < r; j += 32) L.dbg_short[(int64_t)a * r + j] = v[j];
+      const float* v = L.X + (int64_t)L.perm[a] * ldx + voff;
+      float n2 = 0.f;
+      for (int j = lane; j < r; j += 32) n2 = fmaf(v[j], v[j], n2);
+      n2 = warp_sum(n2);
+      const float inv = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
+      for (int j = lane; j < r; j += 32) L.dbg_short[(int64_t)a * r + j] = v[j] * inv;
     }
   }
-}
-
-void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
-                     cudaStream_t st) {
-  sp_check_kernel<<<1, 256, 0, st>>>(d_layers, n_layers, t16, t8, max_sweeps, d_all_done);
 }
 
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key, uint32_t kind_step,
@@ -578,6 +370,13 @@ __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLaye
       L.bp_partials[(int64_t)ref.a * L.k_cap + a0 + tid] = tot;
     }
   }
+}
+
+int sp_configure() {
+  const int e = sp_configure_eig();
+  if (e != 0) return e;
+  return (int)cudaFuncSetAttribute(sp_backproject_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   kBpAtoms * kMaxShort * (int)sizeof(float));
 }
 
 void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st) {

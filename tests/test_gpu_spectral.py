@@ -146,19 +146,24 @@ def test_host_side_errors(atomo):
 
 
 def test_sweep_cap_reports_not_converged(atomo):
-    # a bounded eigen-solver: with the cap at one sweep the layer reports NOT_CONVERGED and still
-    # returns an orthonormal, usable result (no trap, no hang)
+    # a bounded eigen-solver: with the cap at one sweep the layer reports NOT_CONVERGED (no trap, no hang).
+    # Route 1 (rows orthogonal only at convergence) then keeps nothing; route 0 keeps its orthonormal basis.
     import torch
     G = synth.c2_resnet18(0, [synth.RESNET18_LAYERS[5]])[0]
-    atomo.set_eig_params(1, 1e-6)
+    t = torch.from_numpy(G).cuda()
+    atomo.set_eig_params(1, 3e-7)
     try:
-        pay, dbg = atomo.atomo_encode_spectral([torch.from_numpy(G).cuda()], 2.0, seed=1, k_cap=128, debug=True,
-                                               debug_short=True)
+        pay, _ = atomo.atomo_encode_spectral([t], 2.0, seed=1, k_cap=128)
+        assert atomo.payload_status(pay) == (5, 0) and pay.headers()[1][0].k == 0
+        assert not atomo.atomo_decode(pay)[0].any()
+        atomo.set_eig_mode(0)
+        pay, dbg = atomo.atomo_encode_spectral([t], 2.0, seed=1, k_cap=128, debug=True, debug_short=True)
         assert atomo.payload_status(pay) == (5, 0)
         Us = dbg.layer_short(0, 128).astype(np.float64)
         assert np.abs(Us @ Us.T - np.eye(128)).max() <= 1e-4
     finally:
-        atomo.set_eig_params(40, 1e-6)
+        atomo.set_eig_params(40, 3e-7)
+        atomo.set_eig_mode(1)
 
 
 def test_unbiased_on_gpu(atomo):
@@ -219,3 +224,21 @@ def test_config5_shape_properties(atomo):
             parity.check_full_basis(G, dbg, l, f"L{l}", orth_tol=2e-3)
         if s == 8.0:
             assert all(h.n_sat >= 1 for h in hdrs[1])          # sum(sigma) ~ 7.5 < 8 sigma_1
+
+
+def test_eigen_routes_agree(atomo, oracle):
+    # route 0 (Jacobi on [A | I] with accumulated vectors) is an independent check of route 1
+    # (Cholesky factor, Jacobi on its rows): same singular values, probabilities and masks
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(2, [L[1], L[6], L[10], L[17]])
+    try:
+        atomo.set_eig_mode(0)
+        pay0, dbg0 = _encode(atomo, mats, 2.0, seed=31, step=2)
+        _run(atomo, oracle, mats, 2.0, seed=31, step=2)
+    finally:
+        atomo.set_eig_mode(1)
+    pay1, dbg1 = _encode(atomo, mats, 2.0, seed=31, step=2)
+    for l, G in enumerate(mats):
+        r = min(G.shape)
+        assert parity.rel(dbg1.layer_sigma(l, r), dbg0.layer_sigma(l, r)) <= 3e-5
+        assert parity.rel(dbg1.layer_prob(l, r), dbg0.layer_prob(l, r)) <= 3e-5
