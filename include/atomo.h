@@ -34,7 +34,9 @@
  * Payload (DEVICE buffer, caller owned, self-describing; all offsets in bytes from its start,
  * 16-byte aligned):
  *   atomo_payload_header, then n_layers x atomo_layer_header, then per layer
- *     entry-wise: idx  u32[k_cap] ascending flat indices, val f32[k_cap] = g_i / p_i
+ *     entry-wise: idx  u32[k_cap] ascending flat indices, val f32[k_cap] = g_i / p_i,
+ *                 tiles u32[ceil(n / ATOMO_EW_TILE) + 1]: number of kept atoms with index below
+ *                 t * ATOMO_EW_TILE (last entry = k), at header field off_short
  *     spectral  : idx  u32[k_cap] ascending ranks, coef f32[k_cap] = sigma_i / p_i,
  *                 short f32[k_cap][r]  unit vectors of the short side (length r = min(rows,cols)),
  *                 long  f32[k_cap][L]  unit vectors of the long side  (length L = max(rows,cols));
@@ -66,7 +68,8 @@ typedef enum {
 } atomo_status;
 
 enum { ATOMO_KIND_SPECTRAL = 0, ATOMO_KIND_ENTRYWISE = 1 };
-enum { ATOMO_MAGIC = 0x4F4D5441 /* "ATMO" */, ATOMO_VERSION = 1 };
+enum { ATOMO_MAGIC = 0x4F4D5441 /* "ATMO" */, ATOMO_VERSION = 2 };
+enum { ATOMO_EW_TILE = 4096 };   /* entry-wise payloads carry one offset per tile of this many elements */
 
 typedef struct { const float* data; /* DEVICE */ int32_t rows, cols; int64_t ld; } atomo_mat;
 typedef struct { const float* data; /* DEVICE */ int64_t n; } atomo_vec;
@@ -88,7 +91,7 @@ typedef struct {
   float    c;                 /* common weight |lambda_i|/p_i of the kept atoms with p < 1       */
   uint32_t sweeps;            /* spectral: Jacobi sweeps used                                    */
   uint64_t off_idx, off_val;  /* val = entry-wise values / spectral coefficients                 */
-  uint64_t off_short, off_long;
+  uint64_t off_short, off_long; /* entry-wise: off_short = the per-tile offset table           */
   double   l1;                /* sum |lambda| over all atoms (||g||_1 or the nuclear norm)       */
 } atomo_layer_header;                         /* 80 bytes */
 

@@ -97,7 +97,7 @@ uint64_t layout_spectral(const int32_t* rows, const int32_t* cols, int n_layers,
   return align_up(off, 16);
 }
 
-struct EwLayout { uint32_t kc; uint64_t off_idx, off_val; };
+struct EwLayout { uint32_t kc; uint64_t off_idx, off_val, off_tiles; };
 
 uint64_t layout_entrywise(const int64_t* n, int n_vecs, int64_t k_cap, std::vector<EwLayout>* out) {
   uint64_t off = sizeof(atomo_payload_header) + (uint64_t)n_vecs * sizeof(atomo_layer_header);
@@ -107,6 +107,7 @@ uint64_t layout_entrywise(const int64_t* n, int n_vecs, int64_t k_cap, std::vect
     lo.kc = kc;
     off = align_up(off, 16); lo.off_idx = off; off += (uint64_t)kc * 4;
     off = align_up(off, 16); lo.off_val = off; off += (uint64_t)kc * 4;
+    off = align_up(off, 16); lo.off_tiles = off; off += ((uint64_t)(n[l] + ATOMO_EW_TILE - 1) / ATOMO_EW_TILE + 1) * 4;
     if (out) out->push_back(lo);
   }
   return align_up(off, 16);
@@ -380,6 +381,8 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
 
   std::vector<EwVec> V(n_vecs);
   size_t need = 0;
+  const int max_blocks = ew_solve_max_blocks();
+  if (max_blocks <= 0) return fail_cuda(ctx, cudaGetLastError(), "occupancy query for the cooperative solve");
   for (int pass = 0; pass < 2; ++pass) {
     Arena A(pass ? ctx->ws : nullptr);
     size_t dbg_atoms = 0, dbg_words = 0;
@@ -388,13 +391,14 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
       v.n_words = (v.n + 31) / 32;
-      const int64_t want_chunks = std::min<int64_t>(148 * 8, (v.n + 4095) / 4096);
+      const int64_t want_chunks = std::min<int64_t>(max_blocks, (v.n + 4095) / 4096);
       v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
       v.n_chunks = (int)((v.n + v.chunk - 1) / v.chunk);
       v.hdr = d_hdr + l;
       v.idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_idx);
       v.val = reinterpret_cast<float*>(pay + lay[l].off_val);
-      v.partials = A.take<EwPartial>(v.n_chunks);
+      v.tile_table = reinterpret_cast<uint32_t*>(pay + lay[l].off_tiles);
+      v.partials = A.take<EwPartial>((size_t)3 * v.n_chunks);
       v.state = A.take<EwState>(1);
       uint32_t* mask_ws = A.take<uint32_t>(v.n_words);
       v.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
@@ -415,26 +419,20 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   for (int l = 0; l < n_vecs; ++l) {
     atomo_layer_header h{};
     h.rows = 1; h.cols = ns[l]; h.k_cap = lay[l].kc; h.status = ATOMO_OK;
-    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val;
+    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val; h.off_short = lay[l].off_tiles;
     std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
   }
   CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
 
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   const uint32_t ks = kind_step_word(ATOMO_KIND_ENTRYWISE, step);
-  // pass 1 for every vector, then water-filling rounds where the gradient is not s-balanced
+  // probabilities: one cooperative launch per vector (pass 1 and the water-filling rounds)
   stage_begin(ctx, ATOMO_STAGE_EW_REDUCE, st);
-  int64_t n_launch = 0;
-  for (int l = 0; l < n_vecs; ++l) { launch_ew_reduce_all(V[l], s, st); n_launch += 2; }
   for (int l = 0; l < n_vecs; ++l) {
-    for (int round = 0; round <= kEwMaxRounds; ++round) {
-      CK(cudaMemcpyAsync(ctx->h_state, V[l].state, sizeof(EwState), cudaMemcpyDeviceToHost, st));
-      CK(cudaStreamSynchronize(st));
-      if (ctx->h_state->done) break;
-      launch_ew_round(V[l], s, st); n_launch += 2;
-    }
+    const int e = launch_ew_solve(V[l], s, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(ew_solve)");
   }
-  stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_launch);
+  stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_vecs);
   stage_begin(ctx, ATOMO_STAGE_EW_PACK, st);
   for (int l = 0; l < n_vecs; ++l) launch_ew_sample_pack(V[l], key, ks, st);
   stage_end(ctx, ATOMO_STAGE_EW_PACK, st, 3 * (int64_t)n_vecs);

@@ -5,7 +5,6 @@
 namespace atomo {
 
 // ================================= entry-wise path ===============================================
-constexpr int kEwAll = 0, kEwRound = 1;
 constexpr int kEwMaxRounds = 64;      // water-filling rounds; Algorithm 1 saturates < ceil(s) atoms,
                                       // a round usually takes many at once
 
@@ -30,6 +29,7 @@ struct EwVec {
   atomo_layer_header* hdr; uint32_t* idx; float* val;          // payload
   EwPartial* partials; EwState* state;                         // workspace
   uint32_t* mask_words; uint32_t* tile_counts; uint64_t* tile_offsets;
+  uint32_t* tile_table;                                        // payload: kept atoms before each tile
   float* prob_out;                                             // debug or nullptr
 };
 
@@ -38,8 +38,8 @@ struct EwDecode {
   float* out; int64_t n;
 };
 
-void launch_ew_reduce_all(const EwVec& v, double s, cudaStream_t st);
-void launch_ew_round(const EwVec& v, double s, cudaStream_t st);
+int ew_solve_max_blocks();                                     // co-resident CTAs of the cooperative solve
+int launch_ew_solve(const EwVec& v, double s, cudaStream_t st); // returns a cudaError_t
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st);
 void launch_ew_decode(const EwDecode& d, cudaStream_t st);
 int ew_tile_elems();

@@ -47,7 +47,7 @@ def test_payload_size_queries(lib):
     b2 = api.payload_bytes_spectral([(64, 64), (10, 512)], 4)
     assert b2 > b and b2 % 16 == 0
     e = api.payload_bytes_entrywise([4096], 100)
-    assert e == 64 + 80 + 400 + 400
+    assert e == 64 + 80 + 400 + 400 + 16       # + per-tile offset table (2 entries, 16-byte aligned)
     assert api.payload_bytes_entrywise([0], 10) == -1
     assert api.payload_bytes_entrywise([2 ** 32], 10) == -1
     assert api.payload_bytes_spectral([(0, 5)], 10) == -1
