@@ -195,6 +195,13 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol);
  * rows of its transpose (row i converges to sigma_i times eigenvector i).  0: one-sided Jacobi on the
  * rows of [A | I] with accumulated eigenvectors -- slower, kept as a cross-check of route 1.        */
 int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode);
+/* Singular-value refinement: layers whose short side is at least `min_short_side` take sigma_i from the
+ * norm of the projection, sigma_i = ||G^T u_i|| (or ||G v_i||), for every atom instead of the square root
+ * of the Gram eigenvalue (default 2048; 0 = every layer, a value above 4096 = never).  The Gram route
+ * resolves eigenvalues only to about 1e-8 of the largest, which a long flat tail of small singular values
+ * turns into a visible error of the nuclear norm and thus of every p_i; the projection norm does not
+ * have that floor.  It costs one more pass over G with twice the Gram matrix's arithmetic.              */
+int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
 
 #ifdef __cplusplus
 }

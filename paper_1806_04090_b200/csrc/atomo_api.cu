@@ -25,6 +25,7 @@ struct atomo_ctx {
   int max_sweeps = 40;
   float tol = 3e-7f;
   int eig_mode = 1;                  // 1: Cholesky factor + Jacobi on its rows; 0: Jacobi on [A | I]
+  int refine_min_short = 2048;       // layers with at least this short side get the sigma refinement pass
   std::string err;
 };
 
@@ -190,6 +191,12 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
   return ATOMO_OK;
 }
 
+int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side) {
+  if (!ctx || min_short_side < 0) return ATOMO_ERR_INVALID_ARG;
+  ctx->refine_min_short = min_short_side;
+  return ATOMO_OK;
+}
+
 int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode) {
   if (!ctx || (mode != 0 && mode != 1)) return ATOMO_ERR_INVALID_ARG;
   ctx->eig_mode = mode;
@@ -222,7 +229,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
-  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles;
+  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles, chol_ctas, refine_tiles;
+  int chol_panels = 0;
   int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
@@ -233,21 +241,29 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d.rp = next_pow2_at_least(d.r, 32);
     d.acc = ctx->eig_mode == 0 ? 1 : 0;
     d.ldx = d.acc ? 2 * d.rp : d.rp;
-    if (d.ldx > 1024) return ATOMO_ERR_INVALID_ARG;   // route 0 holds rows of 2 rp floats: short side <= 512
-    d.B = 16;
+    if (d.acc && d.ldx > 1024) return ATOMO_ERR_INVALID_ARG;   // route 0 holds rows of 2 rp floats: short side <= 512
+    d.B = d.ldx <= 1024 ? 16 : (d.ldx == 2048 ? 8 : 4);          // a rotation is shared by 1, 2 or 4 warps
     d.nb = d.rp / d.B;
     d.layer = (uint32_t)l; d.k_cap = lay[l].kc;
     r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
     for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
-    for (int p = 0; p < d.nb / 2; ++p) (d.B == 16 ? pairs16 : pairs8).push_back({l, p, 0, 0});
-    if (d.B == 16) { rp16_max = std::max(rp16_max, d.ldx); steps16 = std::max(steps16, d.nb - 1); }
-    else steps8 = std::max(steps8, d.nb - 1);
+    for (int p = 0; p < d.nb / 2; ++p) pairs16.push_back({l, p, 0, 0});
+    rp16_max = std::max(rp16_max, d.ldx); steps16 = std::max(steps16, d.nb - 1);
+    if (!d.acc && d.rp > 1024) {
+      const int per = sp_cholesky_big_rows_per_cta();
+      for (int c = 0; c < (d.rp + per - 1) / per; ++c) chol_ctas.push_back({l, c, 0, 0});
+      chol_panels = std::max(chol_panels, (d.r + 31) / 32);
+    }
     d.bp_tiles = d.tall ? (d.L + sp_bp_rows_per_tile() - 1) / sp_bp_rows_per_tile()
                         : (d.L + sp_bp_cols_per_tile() - 1) / sp_bp_cols_per_tile();
     for (int t = 0; t < d.bp_tiles; ++t) bp_tiles.push_back({l, t, 0, 0});
+    d.refine = d.r >= ctx->refine_min_short ? 1 : 0;
+    d.refine_tiles = (d.L + 63) / 64;
+    if (d.refine)
+      for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
-  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr;
+  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr;
   uint32_t* d_flag = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
@@ -258,6 +274,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_p16 = A.take<TileRef>(pairs16.size());
     d_p8 = A.take<TileRef>(pairs8.size());
     d_bp = A.take<TileRef>(bp_tiles.size());
+    d_chol = A.take<TileRef>(chol_ctas.size());
+    d_ref = A.take<TileRef>(refine_tiles.size());
     d_flag = A.take<uint32_t>(4);
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -275,6 +293,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       d.p_sel = A.take<float>(d.k_cap);
       d.bp_partials = A.take<float>((size_t)d.bp_tiles * d.k_cap);
       d.scale = A.take<float>(1);
+      d.chol_dd = A.take<float>(32 * 32 + 32);
+      d.row_inv = A.take<float>(d.rp);
+      d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);
       d.hdr = d_hdr + l;
       d.idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_idx);
       d.coef = reinterpret_cast<float*>(pay + lay[l].off_coef);
@@ -314,6 +335,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   if (!pairs16.empty()) CK(cudaMemcpyAsync(d_p16, pairs16.data(), pairs16.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!pairs8.empty()) CK(cudaMemcpyAsync(d_p8, pairs8.data(), pairs8.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!refine_tiles.empty()) CK(cudaMemcpyAsync(d_ref, refine_tiles.data(), refine_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!chol_ctas.empty()) CK(cudaMemcpyAsync(d_chol, chol_ctas.data(), chol_ctas.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
 
   // ---- S1: Gram matrix, scaling ----
@@ -321,7 +344,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   launch_sp_init(d_layers, n_layers, nullptr, 0, st);
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
   launch_sp_scale(d_layers, n_layers, st);
-  if (ctx->eig_mode != 0) launch_sp_cholesky(d_layers, n_layers, rp_max, st);
+  if (ctx->eig_mode != 0) {
+    launch_sp_cholesky(d_layers, n_layers, rp_max, st);
+    const int e = launch_sp_cholesky_big(d_layers, d_chol, (int)chol_ctas.size(), chol_panels, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(cholesky)");
+  }
   stage_end(ctx, ATOMO_STAGE_GRAM, st, 5);
   CK(cudaGetLastError());
 
@@ -341,8 +368,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   }
   stage_end(ctx, ATOMO_STAGE_EIG, st, n_eig_launch);
 
-  // ---- S2-S4: probabilities, draws, compaction ----
+  // ---- S2-S4: (refined singular values,) probabilities, draws, compaction ----
   stage_begin(ctx, ATOMO_STAGE_SAMPLE, st);
+  launch_sp_refine(d_layers, n_layers, d_ref, (int)refine_tiles.size(), st);
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps, st);
   stage_end(ctx, ATOMO_STAGE_SAMPLE, st, 1);

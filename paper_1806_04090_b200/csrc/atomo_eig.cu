@@ -14,7 +14,13 @@
 // rotation.  Row norms are tracked (alpha' = alpha - t gamma, beta' = beta + t gamma) and refreshed when
 // they cancel; rotations are applied in the scaled ("fast Givens") form, one FMA per element, with the
 // cosines collected in a per-row factor that is folded back when the block pair is stored.
+#include <algorithm>
+
+#include <cooperative_groups.h>
+
 #include "atomo_kernels.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace atomo {
 
@@ -50,7 +56,7 @@ __device__ __forceinline__ void store_row(const RowRegs<T4>& x, float* row, int 
     }
 }
 template <int T4>
-__device__ __forceinline__ float row_norm2(const RowRegs<T4>& x, int lane, int A4) {
+__device__ __forceinline__ float row_norm2_partial(const RowRegs<T4>& x, int lane, int A4) {
   float n = 0.f;
 #pragma unroll
   for (int t = 0; t < T4; ++t)
@@ -58,8 +64,29 @@ __device__ __forceinline__ float row_norm2(const RowRegs<T4>& x, int lane, int A
       const float4 a = x.v[t];
       n = fmaf(a.x, a.x, fmaf(a.y, a.y, fmaf(a.z, a.z, fmaf(a.w, a.w, n))));
     }
-  return warp_sum(n);
+  return n;
 }
+
+// Sum of one value per lane over a whole row.  A row is held by WPR warps (one segment each): the warp
+// sums are exchanged through shared memory under a named barrier of the WPR warps that share the pair,
+// and added in a fixed order, so every warp of the pair gets the same bits and takes the same branches.
+template <int WPR>
+struct RowSum {
+  float* slots;      // [2][WPR] for this pair (double-buffered)
+  int bar_id, seg, lane, phase;
+  __device__ __forceinline__ float operator()(float v) {
+    v = warp_sum(v);
+    if constexpr (WPR == 1) return v;
+    float* slot = slots + (phase & 1) * WPR;
+    if (lane == 0) slot[seg] = v;
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(32 * WPR) : "memory");
+    float t = 0.f;
+#pragma unroll
+    for (int i = 0; i < WPR; ++i) t += slot[i];
+    ++phase;
+    return t;
+  }
+};
 
 // One plane rotation of the stored rows (xp, xq); true rows are dp * xp and dq * xq, with tracked squared
 // norms np2, nq2 of their first A4 float4 (the part that is orthogonalised).  All lanes take the same branch.
@@ -76,9 +103,9 @@ __device__ __forceinline__ float row_norm2(const RowRegs<T4>& x, int lane, int A
 //   cancellation and is recomputed from the row when it dropped by 1000x.  (A stale norm can only waste or
 //   postpone a rotation: a sweep that rotates nothing changes no norm, so the convergence test always sees
 //   norms computed from the rows.)
-template <int T4>
+template <int T4, typename Sum>
 __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, float& np2, float& nq2, float& dp,
-                                            float& dq, int lane, int A4, float tol) {
+                                            float& dq, int lane, int A4, float tol, Sum& row_sum) {
   float g0 = 0.f, g1 = 0.f;
 #pragma unroll
   for (int t = 0; t < T4; ++t) {
@@ -91,7 +118,7 @@ __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, fl
   const float al = np2, be = nq2;
   const float m = rsqrtf(al) * rsqrtf(be);                   // independent of the reduction below
   const float ratio_qp = __fdividef(dq, dp), ratio_pq = __fdividef(dp, dq);
-  const float ga = warp_sum(g0 + g1) * dp * dq;
+  const float ga = row_sum(g0 + g1) * dp * dq;
   if (al < kRowFloor || be < kRowFloor) return false;
   const float gn = ga * m;                                   // cosine of the angle between the rows
   if (!(fabsf(gn) > tol)) return false;                      // also false for NaN
@@ -113,23 +140,31 @@ __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, fl
   dp *= c; dq *= c;
   const float tg = tt * ga;
   np2 = al - tg; nq2 = be + tg;
-  if (np2 < 1e-3f * al) np2 = row_norm2<T4>(xp, lane, A4) * dp * dp;
-  if (nq2 < 1e-3f * be) nq2 = row_norm2<T4>(xq, lane, A4) * dq * dq;
+  if (np2 < 1e-3f * al) np2 = row_sum(row_norm2_partial<T4>(xp, lane, A4)) * dp * dp;
+  if (nq2 < 1e-3f * be) nq2 = row_sum(row_norm2_partial<T4>(xq, lane, A4)) * dq * dq;
   return true;
 }
 
-// One block pair (2 x 16 rows) of one layer, resident in shared memory, 16 warps, one warp per rotation.
+// One block pair (2 B rows, B = 16 / WPR) of one layer, resident in shared memory.  16 warps; a rotation
+// is done by WPR warps, each holding one segment of the two rows (WPR = 1 for rows of up to 1024 floats).
 // RP = padded short side; ACC: rows are [x | v] (2 RP floats, mode 0), else x only (RP floats, mode 1).
-template <int RP, bool ACC>
+template <int RP, bool ACC, int WPR>
 __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, float tol,
                                                   float* smem) {
-  constexpr int B = kJB;
-  constexpr int LD = ACC ? 2 * RP : RP, V4 = LD / 4, A4 = RP / 4, T4 = (V4 + 31) / 32;
-  constexpr int NT = 32 * B;
-  static_assert(T4 <= 8, "row too long for one warp");
+  constexpr int B = kJB / WPR;
+  constexpr int LD = ACC ? 2 * RP : RP;                 // floats per row
+  constexpr int SEG = LD / WPR;                         // floats per warp segment
+  constexpr int V4 = SEG / 4, T4 = (V4 + 31) / 32;      // float4 per segment, per lane
+  constexpr int A4 = ACC ? RP / 4 : V4;                 // float4 of a segment that take part in dot products
+  constexpr int NT = 32 * kJB, R4 = LD / 4;
+  static_assert(T4 <= 8, "segment too long for one warp");
+  static_assert(!ACC || WPR == 1, "route 0 rows are held by one warp");
   float* s_n2 = smem + 2 * B * LD;       // squared norms of the true rows
   float* s_d = s_n2 + 2 * B;             // true row = s_d * stored row
+  float* s_part = s_d + 2 * B;           // [B][2][WPR] warp sums of a pair
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const int pi = w / WPR, seg = w % WPR; // pair slot, segment
+  RowSum<WPR> row_sum{s_part + pi * 2 * WPR, 1 + pi, seg, lane, 0};
   int bi, bj;
   rr_pair(L.nb, local, slot, bi, bj);
   float* X = L.X;
@@ -141,67 +176,71 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 #endif
   ATOMO_TICK();
   // ---- load 2B rows ----
-  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
-    const int row = idx / V4, q = idx % V4;
+  for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+    const int row = idx / R4, q = idx % R4;
     const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
     reinterpret_cast<float4*>(smem + row * LD)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * LD)[q];
   }
   __syncthreads();
   RowRegs<T4> xp, xq;
-  // warp w: squared norms of rows w and w + B; row w stays in registers for the cross rounds
-  load_row<T4>(xq, smem + (B + w) * LD, lane, V4);
-  const float nj = row_norm2<T4>(xq, lane, A4);
-  load_row<T4>(xp, smem + w * LD, lane, V4);
-  float np2 = row_norm2<T4>(xp, lane, A4), dp = 1.0f;
-  if (lane == 0) { s_n2[w] = np2; s_n2[B + w] = nj; s_d[w] = 1.0f; s_d[B + w] = 1.0f; }
+  // pair slot pi: squared norms of rows pi and pi + B; row pi stays in registers for the cross rounds
+  load_row<T4>(xq, smem + (B + pi) * LD + seg * SEG, lane, V4);
+  const float nj = row_sum(row_norm2_partial<T4>(xq, lane, A4));
+  load_row<T4>(xp, smem + pi * LD + seg * SEG, lane, V4);
+  float np2 = row_sum(row_norm2_partial<T4>(xp, lane, A4)), dp = 1.0f;
+  if (lane == 0 && seg == 0) { s_n2[pi] = np2; s_n2[B + pi] = nj; s_d[pi] = 1.0f; s_d[B + pi] = 1.0f; }
   __syncthreads();
   ATOMO_TICK();
   uint32_t nrot = 0;
   // ---- pairs inside each block: once per sweep ----
   if (local == 0) {
     for (int round = 0; round < B - 1; ++round) {
-      const int blk = w / (B / 2), sl = w % (B / 2);
+      const int blk = pi / (B / 2), sl = pi % (B / 2);
       int p, q;
       rr_pair(B, round, sl, p, q);
       p += blk * B; q += blk * B;
-      float* rowp = smem + p * LD;
-      float* rowq = smem + q * LD;
+      float* rowp = smem + p * LD + seg * SEG;
+      float* rowq = smem + q * LD + seg * SEG;
       load_row<T4>(xp, rowp, lane, V4);
       load_row<T4>(xq, rowq, lane, V4);
       float a2 = s_n2[p], b2 = s_n2[q], da = s_d[p], db = s_d[q];
-      if (rotate_pair<T4>(xp, xq, a2, b2, da, db, lane, A4, tol)) {
+      const bool rot = rotate_pair<T4>(xp, xq, a2, b2, da, db, lane, A4, tol, row_sum);
+      if (WPR > 1) __syncthreads();       // every warp of the pair has read the old norms and factors
+      if (rot) {
         store_row<T4>(xp, rowp, lane, V4);
         store_row<T4>(xq, rowq, lane, V4);
-        if (lane == 0) { s_n2[p] = a2; s_n2[q] = b2; s_d[p] = da; s_d[q] = db; }
-        ++nrot;
+        if (lane == 0 && seg == 0) { s_n2[p] = a2; s_n2[q] = b2; s_d[p] = da; s_d[q] = db; }
+        if (seg == 0) ++nrot;
       }
       __syncthreads();
     }
-    load_row<T4>(xp, smem + w * LD, lane, V4);
-    np2 = s_n2[w]; dp = s_d[w];
+    load_row<T4>(xp, smem + pi * LD + seg * SEG, lane, V4);
+    np2 = s_n2[pi]; dp = s_d[pi];
   }
   ATOMO_TICK();
-  // ---- pairs across the two blocks: warp w keeps row w of block bi in registers; the rows of block bj
-  //      visit the warps round-robin ----
+  // ---- pairs across the two blocks: slot pi keeps row pi of block bi in registers; the rows of block bj
+  //      visit the slots round-robin ----
   for (int round = 0; round < B; ++round) {
-    const int j = B + (w + round) % B;
-    float* rowq = smem + j * LD;
+    const int j = B + (pi + round) % B;
+    float* rowq = smem + j * LD + seg * SEG;
     load_row<T4>(xq, rowq, lane, V4);
     float nq2 = s_n2[j], dq = s_d[j];
-    if (rotate_pair<T4>(xp, xq, np2, nq2, dp, dq, lane, A4, tol)) {
+    const bool rot = rotate_pair<T4>(xp, xq, np2, nq2, dp, dq, lane, A4, tol, row_sum);
+    if (WPR > 1) __syncthreads();         // every warp of the pair has read the old norm and factor
+    if (rot) {
       store_row<T4>(xq, rowq, lane, V4);
-      if (lane == 0) { s_n2[j] = nq2; s_d[j] = dq; }
-      ++nrot;
+      if (lane == 0 && seg == 0) { s_n2[j] = nq2; s_d[j] = dq; }
+      if (seg == 0) ++nrot;
     }
     __syncthreads();
   }
   ATOMO_TICK();
-  store_row<T4>(xp, smem + w * LD, lane, V4, dp);
-  if (lane == 0) s_d[w] = 1.0f;
+  store_row<T4>(xp, smem + pi * LD + seg * SEG, lane, V4, dp);
+  if (lane == 0 && seg == 0) s_d[pi] = 1.0f;
   __syncthreads();
   // ---- store, folding the collected cosines back into the rows ----
-  for (int idx = tid; idx < 2 * B * V4; idx += NT) {
-    const int row = idx / V4, q = idx % V4;
+  for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+    const int row = idx / R4, q = idx % R4;
     const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
     const float d = s_d[row];
     const float4 a = reinterpret_cast<const float4*>(smem + row * LD)[q];
@@ -218,7 +257,7 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 
 constexpr int kJacobiThreads = 32 * kJB;
 
-// One Jacobi step for every layer: mode 1 layers with padded short side <= 1024, mode 0 layers with <= 512.
+// One Jacobi step for every layer: mode 1 layers with padded short side <= 4096, mode 0 layers with <= 512.
 __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const SpLayer* __restrict__ layers,
                                                                         const TileRef* __restrict__ pairs, int t,
                                                                         int max_sweeps, float tol) {
@@ -231,33 +270,35 @@ __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const Sp
   if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
   if (L.acc) {
     switch (L.rp) {
-      case 32: jacobi_block_pair<32, true>(L, ref.a, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, true>(L, ref.a, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, true>(L, ref.a, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, true>(L, ref.a, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, true>(L, ref.a, sweep, local, tol, smem); break;
+      case 32: jacobi_block_pair<32, true, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, true, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, true, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, true, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, true, 1>(L, ref.a, sweep, local, tol, smem); break;
       default: break;
     }
   } else {
     switch (L.rp) {
-      case 32: jacobi_block_pair<32, false>(L, ref.a, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, false>(L, ref.a, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, false>(L, ref.a, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, false>(L, ref.a, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, false>(L, ref.a, sweep, local, tol, smem); break;
-      case 1024: jacobi_block_pair<1024, false>(L, ref.a, sweep, local, tol, smem); break;
+      case 32: jacobi_block_pair<32, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 1024: jacobi_block_pair<1024, false, 1>(L, ref.a, sweep, local, tol, smem); break;
+      case 2048: jacobi_block_pair<2048, false, 2>(L, ref.a, sweep, local, tol, smem); break;
+      case 4096: jacobi_block_pair<4096, false, 4>(L, ref.a, sweep, local, tol, smem); break;
       default: break;
     }
   }
 }
 
-constexpr int kJacobiSmem = 32 * 1024 * 4 + 512;   // 32 rows of up to 1024 floats + norms and factors
+constexpr int kJacobiSmem = 32 * 1024 * 4 + 1024;   // 32 rows of up to 1024 floats + norms and factors
 
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st) {
   if (n_pairs <= 0) return;
   (void)B;
-  const int smem = 32 * row_floats_max * 4 + 512;
+  const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
   sp_jacobi_step_kernel<<<n_pairs, kJacobiThreads, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
 }
 
@@ -270,7 +311,7 @@ __global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers
   for (int l = threadIdx.x; l < n_layers; l += blockDim.x) {
     const SpLayer& L = layers[l];
     const int steps = L.nb - 1;
-    const int t_done = (L.B == 16) ? t16 : t8;
+    const int t_done = t16; (void)t8;
     const int sweeps_done = min(t_done / steps, max_sweeps);
     int conv = -1;
     for (int wv = 0; wv < sweeps_done; ++wv) if (L.rot_count[wv] == 0) { conv = wv; break; }
@@ -300,7 +341,7 @@ constexpr int kCholPanel = 32;
 
 __global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
-  if (L.acc) return;
+  if (L.acc || L.rp > 1024) return;                      // larger layers: sp_cholesky_big_kernel
   __shared__ float s_k[kCholPanel][kCholPanel + 1];     // L[j0 + c][k0 + kk] for the current k chunk
   __shared__ float s_ldd[kCholPanel][kCholPanel + 1];   // diagonal block of L
   __shared__ float s_inv[kCholPanel];
@@ -370,9 +411,108 @@ __global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __rest
   }
 }
 
-void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
-  sp_cholesky_kernel<<<n_layers, rp_max, 0, st>>>(d_layers);
+// The same factorisation for layers with more than 1024 rows: kCholBigThreads rows per CTA, several CTAs per
+// layer in one cooperative launch.  Per panel: every CTA updates its rows; the CTA that owns the diagonal block
+// factors it and publishes it; grid barrier; every CTA solves its rows against it and stores them; grid barrier
+// (the next panel reads rows of L written by other CTAs).
+constexpr int kCholBigThreads = 1024;
+
+__global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const SpLayer* __restrict__ layers,
+                                                                          const TileRef* __restrict__ ctas, int max_panels) {
+  cg::grid_group grid = cg::this_grid();
+  const TileRef ref = ctas[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  __shared__ float s_k[kCholPanel][kCholPanel + 1];
+  __shared__ float s_ldd[kCholPanel][kCholPanel + 1];
+  __shared__ float s_inv[kCholPanel];
+  const int r = L.r, rp = L.rp;
+  const int tid = threadIdx.x, lane = tid % 32, warp = tid / 32;
+  const int i = ref.a * kCholBigThreads + tid;            // this thread's row
+  const float* __restrict__ A = L.A;
+  const int64_t lda = L.lda;
+  float* X = L.X;
+  float* dd = L.chol_dd;                                   // published diagonal block: 32 x 32, then 32 inverses
+  for (int panel = 0; panel < max_panels; ++panel) {
+    const int j0 = panel * kCholPanel;
+    const bool live = j0 < r;                              // uniform per CTA
+    const bool active = live && i >= j0 && i < r;
+    float p[kCholPanel];
+#pragma unroll
+    for (int c = 0; c < kCholPanel; ++c) p[c] = (active && j0 + c < r) ? A[(int64_t)(j0 + c) * lda + i] : 0.0f;
+    if (live) {
+      for (int k0 = 0; k0 < j0; k0 += kCholPanel) {
+        __syncthreads();
+        for (int idx = tid; idx < kCholPanel * kCholPanel; idx += kCholBigThreads) {
+          const int kk = idx / kCholPanel, c = idx % kCholPanel;
+          s_k[kk][c] = X[(int64_t)(k0 + kk) * rp + j0 + c];
+        }
+        __syncthreads();
+        if (active) {
+#pragma unroll 4
+          for (int kk = 0; kk < kCholPanel; ++kk) {
+            const float xi = X[(int64_t)(k0 + kk) * rp + i];
+#pragma unroll
+            for (int c = 0; c < kCholPanel; ++c) p[c] = fmaf(-xi, s_k[kk][c], p[c]);
+          }
+        }
+      }
+      if (i >= j0 && i < j0 + kCholPanel) {               // the warp that owns the diagonal block
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) {
+          const float d = __shfl_sync(0xffffffffu, p[c], c);
+          const float lcc = d > kPivotFloor ? sqrtf(d) : 0.0f;
+          const float inv = lcc > 0.0f ? 1.0f / lcc : 0.0f;
+          const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
+          p[c] = lic;
+#pragma unroll
+          for (int c2 = c + 1; c2 < kCholPanel; ++c2) {
+            const float l2 = __shfl_sync(0xffffffffu, lic, c2);
+            if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+          }
+          if (lane == c) dd[kCholPanel * kCholPanel + c] = inv;
+        }
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) dd[lane * kCholPanel + c] = p[c];
+        __threadfence();
+      }
+    }
+    (void)warp;
+    grid.sync();
+    if (live) {
+      for (int idx = tid; idx < kCholPanel * kCholPanel; idx += kCholBigThreads) s_ldd[idx / kCholPanel][idx % kCholPanel] = dd[idx];
+      if (tid < kCholPanel) s_inv[tid] = dd[kCholPanel * kCholPanel + tid];
+      __syncthreads();
+      if (active && i >= j0 + kCholPanel) {
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) {
+          float acc = p[c];
+#pragma unroll
+          for (int k = 0; k < c; ++k) acc = fmaf(-p[k], s_ldd[c][k], acc);
+          p[c] = acc * s_inv[c];
+        }
+      }
+      if (active) {
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c)
+          if (j0 + c < r) X[(int64_t)(j0 + c) * rp + i] = p[c];
+      }
+      __threadfence();
+    }
+    grid.sync();
+  }
 }
+
+void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
+  sp_cholesky_kernel<<<n_layers, std::min(rp_max, 1024), 0, st>>>(d_layers);
+}
+
+int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st) {
+  if (n_ctas <= 0) return 0;
+  void* args[] = {(void*)&d_layers, (void*)&d_ctas, (void*)&max_panels};
+  return (int)cudaLaunchCooperativeKernel((const void*)sp_cholesky_big_kernel, dim3(n_ctas), dim3(kCholBigThreads), args, 0, st);
+}
+
+int sp_cholesky_big_rows_per_cta() { return kCholBigThreads; }
 
 int sp_configure_eig() {
   return (int)cudaFuncSetAttribute(sp_jacobi_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);

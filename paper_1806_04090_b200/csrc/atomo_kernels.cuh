@@ -46,7 +46,7 @@ int ew_tile_elems();
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
-constexpr int kSmemRowsMaxRp = 1024;  // largest padded short side the shared-memory Jacobi kernel holds
+constexpr int kSmemRowsMaxRp = 4096;  // largest padded short side the shared-memory Jacobi kernel holds
 
 struct SpLayer {
   const float* G; int rows, cols; int64_t ld;
@@ -68,7 +68,11 @@ struct SpLayer {
   int bp_tiles;
   uint32_t* rot_count;         // [max_sweeps] rotations applied in each sweep
   float* scale;                // 1 float: power-of-two scaling applied to A
+  float* chol_dd;              // 32 x 32 + 32 floats: diagonal block published by its owner (layers > 1024 rows)
   float* dbg_short;            // r x r or nullptr
+  int refine, refine_tiles;    // singular values from the projection norms; tiles along the long side
+  float* row_inv;              // rp: 1 / norm of each short-side vector as stored in X
+  float* refine_partials;      // [refine_tiles][rp] partial squared norms
 };
 
 struct SpDecodeLayer {
@@ -84,10 +88,14 @@ void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
 void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
+// layers with more than 1024 rows: cooperative launch, returns a cudaError_t
+int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
+int sp_cholesky_big_rows_per_cta();
 int sp_configure_eig();
 // convergence bookkeeping after t16 / t8 steps were enqueued for the two kernel classes
 void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st);
+void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key,
                                uint32_t kind_step, int max_sweeps, cudaStream_t st);
 void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st);

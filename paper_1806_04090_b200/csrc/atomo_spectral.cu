@@ -155,6 +155,111 @@ void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
 }
 
 // =================================================================================================
+// Refinement of the singular values: sigma_i = || G^T u_i || (rows <= cols) or || G v_i || for every
+// short-side vector, not only the kept ones.  The Gram route resolves eigenvalues only down to about
+// eps * lambda_1, which for a long flat noise tail adds up in the nuclear norm; the norm of the projection
+// is second-order accurate in the eigenvector error, so the tail comes out right as long as the
+// vectors are orthonormal.  Tile = 64 vectors x 64 positions of the long side; each tile contributes
+// one partial sum of squares per vector (summed in a fixed order by sp_finalize_sample).
+// =================================================================================================
+__global__ void __launch_bounds__(256) sp_rowinv_kernel(const SpLayer* __restrict__ layers) {
+  const SpLayer& L = layers[blockIdx.x];
+  if (!L.refine) return;
+  const int lane = threadIdx.x % 32, w = threadIdx.x / 32;
+  const int voff = L.acc ? L.rp : 0;
+  for (int i = blockIdx.y * 8 + w; i < L.rp; i += gridDim.y * 8) {
+    float n2 = 0.f;
+    if (i < L.r) {
+      const float* v = L.X + (int64_t)i * L.ldx + voff;
+      for (int j = lane; j < L.r; j += 32) n2 = fmaf(v[j], v[j], n2);
+    }
+    n2 = warp_sum(n2);
+    if (lane == 0) L.row_inv[i] = n2 > 0.f ? 1.0f / sqrtf(n2) : 0.f;
+  }
+}
+
+__global__ void __launch_bounds__(256) sp_refine_kernel(const SpLayer* __restrict__ layers,
+                                                        const TileRef* __restrict__ tiles) {
+  __shared__ __align__(16) float As[kGramK][kGramTile + 4];   // As[k][a] = u_a[k0 + k]
+  __shared__ __align__(16) float Bs[kGramK][kGramTile + 4];   // Bs[k][c] = G(k0 + k, c0 + c) seen from the short side
+  __shared__ float s_sq[16][kGramTile];
+  const TileRef ref = tiles[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int a0 = ref.a * kGramTile, c0 = ref.b * kGramTile;
+  const float* __restrict__ G = L.G;
+  const int64_t ld = L.ld, ldx = L.ldx;
+  const int r = L.r, len = L.L;
+  const int voff = L.acc ? L.rp : 0;
+  const int t = threadIdx.x, ty = t / 16, tx = t % 16;
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+  for (int k0 = 0; k0 < r; k0 += kGramK) {
+    {
+      const int row = t / 4, k4 = (t % 4) * 4;               // vector a0 + row, components k0 + k4 ..
+      const int a = a0 + row;
+      const float inv = a < r ? L.row_inv[a] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int k = k0 + k4 + j;
+        As[k4 + j][row] = (a < r && k < r) ? L.X[(int64_t)a * ldx + voff + k] * inv : 0.0f;
+      }
+    }
+    if (!L.tall) {                                           // G[k][c]: contiguous in c
+      const int kk = t / 16, c4 = (t % 16) * 4;
+      const int k = k0 + kk;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c = c0 + c4 + j;
+        Bs[kk][c4 + j] = (k < r && c < len) ? __ldg(G + (int64_t)k * ld + c) : 0.0f;
+      }
+    } else {                                                 // G[c][k]: contiguous in k
+      const int row = t / 4, k4 = (t % 4) * 4;
+      const int c = c0 + row;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int k = k0 + k4 + j;
+        Bs[k4 + j][row] = (k < r && c < len) ? __ldg(G + (int64_t)c * ld + k) : 0.0f;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kGramK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int p = 0; p < 4; ++p)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) acc[p][q] = fmaf(av[p], bv[q], acc[p][q]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    float sq = 0.f;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) sq = fmaf(acc[p][q], acc[p][q], sq);
+    s_sq[tx][ty * 4 + p] = sq;
+  }
+  __syncthreads();
+  if (t < kGramTile && a0 + t < r) {
+    float tot = 0.f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) tot += s_sq[j][t];            // fixed order
+    L.refine_partials[(int64_t)ref.b * L.rp + a0 + t] = tot;
+  }
+}
+
+void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st) {
+  if (n_tiles <= 0) return;
+  sp_rowinv_kernel<<<dim3(n_layers, 16), 256, 0, st>>>(d_layers);
+  sp_refine_kernel<<<n_tiles, 256, 0, st>>>(d_layers, d_tiles);
+}
+
+// =================================================================================================
 // finalize + probabilities + sampling.  One CTA (512 threads) per layer.
 // =================================================================================================
 constexpr int kFinThreads = 512;
@@ -179,14 +284,21 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   __syncthreads();
 
   // eigenvalue of A per row, one warp per row.  mode 0: lambda_i = <x_i, v_i> (Rayleigh quotient at v_i);
-  // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T)
+  // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T).  With refinement: the sum of the tiles' partial
+  // squared norms of the projection (already in the units of G).
   for (int i = w; i < r; i += kFinThreads / 32) {
-    const float* row = L.X + (int64_t)i * ldx;
-    float d = 0.f;
-    for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[voff + j], d);
-    d = warp_sum(d);
+    float lam;
+    if (L.refine) {
+      double d = 0.0;
+      for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
+      lam = (float)warp_sum(d);
+    } else {
+      const float* row = L.X + (int64_t)i * ldx;
+      float d = 0.f;
+      for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[voff + j], d);
+      lam = warp_sum(d) * inv_scale;
+    }
     if (lane == 0) {
-      const float lam = d * inv_scale;
       if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
       s_lam[i] = fmaxf(lam, 0.0f);
     }

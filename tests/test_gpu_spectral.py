@@ -242,3 +242,59 @@ def test_eigen_routes_agree(atomo, oracle):
         r = min(G.shape)
         assert parity.rel(dbg1.layer_sigma(l, r), dbg0.layer_sigma(l, r)) <= 3e-5
         assert parity.rel(dbg1.layer_prob(l, r), dbg0.layer_prob(l, r)) <= 3e-5
+
+
+def test_config3_vgg11_properties(atomo):
+    # VGG-11-shaped set with two 4096 x 4096 layers, budgets 1, 2, 3.  The oracle SVD would take hours
+    # there, so the checks are the ones that hold at any size, in fp64: singular values against a library
+    # SVD, sum(p) = s, kept atoms as singular triplets, the decode kernel against its definition, and the
+    # small layers against the expected saturation (the 10 x 4096 layer saturates at s = 3)
+    import torch
+    mats = synth.c3_vgg11(0)
+    refs = [np.linalg.svd(G.astype(np.float64), compute_uv=False) for G in mats]
+    ts = [torch.from_numpy(G).cuda() for G in mats]
+    for s in (1.0, 2.0, 3.0):
+        pay, dbg = atomo.atomo_encode_spectral(ts, s, seed=900 + int(s), step=int(s), k_cap=32, debug=True)
+        hdrs = pay.headers()
+        outs = atomo.atomo_decode(pay)
+        assert [h.status for h in hdrs[1]] == [0] * len(mats)
+        for l, G in enumerate(mats):
+            r = min(G.shape)
+            ref = refs[l]
+            sig = dbg.layer_sigma(l, r); p = dbg.layer_prob(l, r)
+            assert parity.rel(sig, ref) <= parity.REL_TOL, f"L{l}: sigma {parity.rel(sig, ref)}"
+            assert abs(p.sum() - min(s, r)) <= 1e-4 * s
+            p_ref = np.minimum(1.0, s * ref / ref.sum()) if s <= ref.sum() / ref[0] else None
+            if p_ref is not None:
+                assert parity.rel(p, p_ref) <= parity.REL_TOL
+            arr = pay.layer_arrays(l, hdrs)
+            G64 = G.astype(np.float64)
+            for j in range(arr["k"]):
+                u = arr["U"][:, j].astype(np.float64); v = arr["V"][:, j].astype(np.float64)
+                sg = float(arr["coef"][j]) * float(p[arr["idx"][j]])
+                r_u = np.linalg.norm(G64.T @ u - sg * v); r_v = np.linalg.norm(G64 @ v - sg * u)
+                lo, hi = (r_u, r_v) if G.shape[0] <= G.shape[1] else (r_v, r_u)
+                assert lo <= 2e-5 * ref[0]
+                assert hi <= max(2e-5 * ref[0], parity.RESID_GRAM * ref[0] ** 2 / sg)
+            own = (arr["U"].astype(np.float64) * arr["coef"].astype(np.float64)) @ arr["V"].astype(np.float64).T
+            out = outs[l].cpu().numpy()
+            assert (parity.rel(out, own) <= 1e-5) if arr["k"] else (not out.any())
+        if s == 3.0:
+            assert hdrs[1][10].n_sat >= 1          # 10 x 4096: sum(sigma) ~ 2.93 sigma_1 < 3 sigma_1
+
+
+def test_sigma_refinement_all_layers(atomo, oracle):
+    # with the projection-norm refinement on for every layer the parity protocol still holds, and the
+    # probabilities land within 2e-6 of the oracle's (the Gram route alone is about 10x further away)
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(1, [L[1], L[6], L[10], L[14], L[17]])
+    atomo.set_sigma_refinement(0)
+    try:
+        pay, hdrs, encs = _run(atomo, oracle, mats, 2.0, seed=77, step=3)
+        pay, dbg = _encode(atomo, mats, 2.0, seed=77, step=3)
+        for l, G in enumerate(mats):
+            r = min(G.shape)
+            assert np.abs(dbg.layer_prob(l, r) - encs[l]["p"]).max() <= 2e-6
+            assert np.abs(dbg.layer_sigma(l, r) - encs[l]["sigma"]).max() <= 1e-6 * encs[l]["sigma"][0]
+    finally:
+        atomo.set_sigma_refinement(2048)
