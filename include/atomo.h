@@ -202,6 +202,9 @@ int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode);
  * turns into a visible error of the nuclear norm and thus of every p_i; the projection norm does not
  * have that floor.  It costs one more pass over G with twice the Gram matrix's arithmetic.              */
 int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
+/* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
+ * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
+int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
 
 #ifdef __cplusplus
 }

@@ -26,6 +26,8 @@ struct atomo_ctx {
   float tol = 3e-7f;
   int eig_mode = 1;                  // 1: Cholesky factor + Jacobi on its rows; 0: Jacobi on [A | I]
   int refine_min_short = 2048;       // layers with at least this short side get the sigma refinement pass
+  bool tc_gram = true;               // Gram matrix on tcgen05 where the layer's layout allows it
+  bool tc_ok = false;                // tensor-map entry point found
   std::string err;
 };
 
@@ -132,6 +134,7 @@ int atomo_create(atomo_ctx** out, int device) {
   for (int i = 0; i < ATOMO_N_STAGES; ++i) { CK(cudaEventCreate(&ctx->ev[i][0])); CK(cudaEventCreate(&ctx->ev[i][1])); }
   const int e = sp_configure();
   if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaFuncSetAttribute(max dynamic shared memory)");
+  ctx->tc_ok = sp_tc_configure() == 0;
   ctx->configured = true;
   return ATOMO_OK;
 }
@@ -191,6 +194,12 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
   return ATOMO_OK;
 }
 
+int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  ctx->tc_gram = tensor_cores != 0;
+  return ATOMO_OK;
+}
+
 int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side) {
   if (!ctx || min_short_side < 0) return ATOMO_ERR_INVALID_ARG;
   ctx->refine_min_short = min_short_side;
@@ -229,7 +238,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
-  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles, chol_ctas, refine_tiles;
+  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
+  const int map_bytes = sp_tc_map_bytes();
+  std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
   int chol_panels = 0;
   int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0;
   for (int l = 0; l < n_layers; ++l) {
@@ -247,7 +258,15 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d.layer = (uint32_t)l; d.k_cap = lay[l].kc;
     r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
-    for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
+    d.tc = 0;
+    if (ctx->tc_gram && ctx->tc_ok && !d.acc && sp_tc_eligible(d.G, d.rows, d.cols, d.ld)) {
+      d.tc = 1;
+      if (sp_tc_make_map(maps_blob.data() + (size_t)l * map_bytes, d.G, d.rows, d.cols, d.ld) != 0) return ATOMO_ERR_INVALID_ARG;
+      const int tt = (d.r + sp_tc_tile() - 1) / sp_tc_tile();
+      for (int a = 0; a < tt; ++a) for (int b = a; b < tt; ++b) tc_tiles.push_back({l, a, b, 0});
+    } else {
+      for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
+    }
     for (int p = 0; p < d.nb / 2; ++p) pairs16.push_back({l, p, 0, 0});
     rp16_max = std::max(rp16_max, d.ldx); steps16 = std::max(steps16, d.nb - 1);
     if (!d.acc && d.rp > 1024) {
@@ -263,7 +282,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
-  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr;
+  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
+  uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
@@ -276,6 +296,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_bp = A.take<TileRef>(bp_tiles.size());
     d_chol = A.take<TileRef>(chol_ctas.size());
     d_ref = A.take<TileRef>(refine_tiles.size());
+    d_tc = A.take<TileRef>(tc_tiles.size());
+    d_maps = A.take<uint8_t>(maps_blob.size());
     d_flag = A.take<uint32_t>(4);
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -335,6 +357,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   if (!pairs16.empty()) CK(cudaMemcpyAsync(d_p16, pairs16.data(), pairs16.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!pairs8.empty()) CK(cudaMemcpyAsync(d_p8, pairs8.data(), pairs8.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!tc_tiles.empty()) {
+    CK(cudaMemcpyAsync(d_tc, tc_tiles.data(), tc_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(d_maps, maps_blob.data(), maps_blob.size(), cudaMemcpyHostToDevice, st));
+  }
+  CK(cudaMemsetAsync(d_flag, 0, 4 * sizeof(uint32_t), st));
   if (!refine_tiles.empty()) CK(cudaMemcpyAsync(d_ref, refine_tiles.data(), refine_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!chol_ctas.empty()) CK(cudaMemcpyAsync(d_chol, chol_ctas.data(), chol_ctas.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
@@ -343,6 +370,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   stage_begin(ctx, ATOMO_STAGE_GRAM, st);
   launch_sp_init(d_layers, n_layers, nullptr, 0, st);
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
+  launch_sp_gram_tc(d_layers, d_maps, d_tc, (int)tc_tiles.size(), d_flag + 1, st);
   launch_sp_scale(d_layers, n_layers, st);
   if (ctx->eig_mode != 0) {
     launch_sp_cholesky(d_layers, n_layers, rp_max, st);
@@ -362,9 +390,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     for (int j = 0; j < steps8; ++j, ++t8, ++n_eig_launch)
       launch_sp_jacobi_step(d_layers, d_p8, (int)pairs8.size(), 8, 1024, t8, max_sweeps, ctx->tol, st);
     launch_sp_check(d_layers, n_layers, t16, t8, max_sweeps, d_flag, st);
-    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
-    if (*ctx->h_flag) break;
+    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+    if (ctx->h_flag[0]) break;
   }
   stage_end(ctx, ATOMO_STAGE_EIG, st, n_eig_launch);
 

@@ -70,6 +70,7 @@ struct SpLayer {
   float* scale;                // 1 float: power-of-two scaling applied to A
   float* chol_dd;              // 32 x 32 + 32 floats: diagonal block published by its owner (layers > 1024 rows)
   float* dbg_short;            // r x r or nullptr
+  int tc;                      // Gram matrix came from the tensor-core kernel (see sp_scale_kernel)
   int refine, refine_tiles;    // singular values from the projection norms; tiles along the long side
   float* row_inv;              // rp: 1 / norm of each short-side vector as stored in X
   float* refine_partials;      // [refine_tiles][rp] partial squared norms
@@ -103,6 +104,14 @@ void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, cudaStream_t 
 void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,
                       cudaStream_t st);
 int sp_configure();          // opt in to large dynamic shared memory; returns cudaError_t
+// tensor-core Gram kernel (atomo_tc.cu)
+int sp_tc_configure();       // driver entry point for tensor maps + shared memory opt-in; returns cudaError_t
+bool sp_tc_eligible(const float* g, int rows, int cols, int64_t ld);
+int sp_tc_make_map(void* out_map, const float* g, int rows, int cols, int64_t ld);   // 0 on success
+int sp_tc_map_bytes();
+int sp_tc_tile();
+void launch_sp_gram_tc(const SpLayer* d_layers, const void* d_maps, const TileRef* d_tiles, int n_tiles, uint32_t* d_err,
+                       cudaStream_t st);
 int sp_bp_rows_per_tile();
 int sp_bp_cols_per_tile();
 int sp_decode_tile_rows();

@@ -284,17 +284,39 @@ def test_config3_vgg11_properties(atomo):
 
 
 def test_sigma_refinement_all_layers(atomo, oracle):
-    # with the projection-norm refinement on for every layer the parity protocol still holds, and the
-    # probabilities land within 2e-6 of the oracle's (the Gram route alone is about 10x further away)
+    # with the projection-norm refinement on for every layer the parity protocol still holds; with the
+    # fp32 FMA Gram kernel the probabilities then land within 2e-6 of the oracle's and sigma within
+    # 1e-6 sigma_1 (the Gram route alone is about 10x further away); with the tensor-core Gram kernel,
+    # whose tail vectors are a little less sharp, within 1e-5
     L = synth.RESNET18_LAYERS
     mats = synth.c2_resnet18(1, [L[1], L[6], L[10], L[14], L[17]])
     atomo.set_sigma_refinement(0)
     try:
-        pay, hdrs, encs = _run(atomo, oracle, mats, 2.0, seed=77, step=3)
-        pay, dbg = _encode(atomo, mats, 2.0, seed=77, step=3)
-        for l, G in enumerate(mats):
-            r = min(G.shape)
-            assert np.abs(dbg.layer_prob(l, r) - encs[l]["p"]).max() <= 2e-6
-            assert np.abs(dbg.layer_sigma(l, r) - encs[l]["sigma"]).max() <= 1e-6 * encs[l]["sigma"][0]
+        for tensor_cores, p_bar, s_bar in ((False, 2e-6, 1e-6), (True, 1e-5, 5e-6)):
+            atomo.set_gram_path(tensor_cores)
+            pay, hdrs, encs = _run(atomo, oracle, mats, 2.0, seed=77, step=3)
+            pay, dbg = _encode(atomo, mats, 2.0, seed=77, step=3)
+            for l, G in enumerate(mats):
+                r = min(G.shape)
+                assert np.abs(dbg.layer_prob(l, r) - encs[l]["p"]).max() <= p_bar
+                assert np.abs(dbg.layer_sigma(l, r) - encs[l]["sigma"]).max() <= s_bar * encs[l]["sigma"][0]
     finally:
         atomo.set_sigma_refinement(2048)
+        atomo.set_gram_path(True)
+
+
+def test_gram_paths_agree(atomo, oracle):
+    # the fp32 FMA Gram kernel is an independent check of the tensor-core one (TF32 hi/lo split)
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(3, [L[0], L[2], L[9], L[13], L[17]])
+    try:
+        atomo.set_gram_path(False)
+        _run(atomo, oracle, mats, 2.0, seed=41, step=6)
+        pay0, dbg0 = _encode(atomo, mats, 2.0, seed=41, step=6)
+    finally:
+        atomo.set_gram_path(True)
+    pay1, dbg1 = _encode(atomo, mats, 2.0, seed=41, step=6)
+    for l, G in enumerate(mats):
+        r = min(G.shape)
+        assert parity.rel(dbg1.layer_sigma(l, r), dbg0.layer_sigma(l, r)) <= 3e-5
+        assert np.array_equal(dbg1.layer_mask(l, r), dbg0.layer_mask(l, r))
