@@ -339,10 +339,13 @@ void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int
 constexpr float kPivotFloor = 1e-9f;
 constexpr int kCholPanel = 32;
 
-__global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __restrict__ layers) {
+// kThreads = 512 serves layers of up to 512 rows with more loads in flight per thread (it may use 128 registers),
+// kThreads = 1024 the layers of 513..1024 rows.
+template <int kThreads, int kUnroll>
+__global__ void __launch_bounds__(kThreads) sp_cholesky_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
-  if (L.acc || L.rp > 1024) return;                      // larger layers: sp_cholesky_big_kernel
-  __shared__ float s_k[kCholPanel][kCholPanel + 1];     // L[j0 + c][k0 + kk] for the current k chunk
+  if (L.acc || L.rp > kThreads || (kThreads == 1024 && L.rp <= 512)) return;   // other classes: the other instantiation / sp_cholesky_big_kernel
+  __shared__ __align__(16) float s_k[kCholPanel][kCholPanel];   // L[j0 + c][k0 + kk] for the current k chunk
   __shared__ float s_ldd[kCholPanel][kCholPanel + 1];   // diagonal block of L
   __shared__ float s_inv[kCholPanel];
   const int r = L.r, rp = L.rp;
@@ -364,11 +367,15 @@ __global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __rest
       }
       __syncthreads();
       if (active) {
-#pragma unroll 4
+#pragma unroll kUnroll
         for (int kk = 0; kk < kCholPanel; ++kk) {
-          const float xi = X[(int64_t)(k0 + kk) * rp + i];
+          const float xi = -X[(int64_t)(k0 + kk) * rp + i];
 #pragma unroll
-          for (int c = 0; c < kCholPanel; ++c) p[c] = fmaf(-xi, s_k[kk][c], p[c]);
+          for (int c = 0; c < kCholPanel; c += 4) {
+            const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
+            p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
+            p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
+          }
         }
       }
     }
@@ -382,9 +389,11 @@ __global__ void __launch_bounds__(1024) sp_cholesky_kernel(const SpLayer* __rest
         const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
         p[c] = lic;
 #pragma unroll
-        for (int c2 = c + 1; c2 < kCholPanel; ++c2) {
-          const float l2 = __shfl_sync(0xffffffffu, lic, c2);
-          if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+        for (int c2 = 0; c2 < kCholPanel; ++c2) {      // full range + predicate: a triangular loop is not unrolled
+          if (c2 > c) {                                //                         and would push p[] to local memory
+            const float l2 = __shfl_sync(0xffffffffu, lic, c2);
+            if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+          }
         }
         if (lane == c) s_inv[c] = inv;
       }
@@ -422,7 +431,7 @@ __global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const 
   cg::grid_group grid = cg::this_grid();
   const TileRef ref = ctas[blockIdx.x];
   const SpLayer& L = layers[ref.layer];
-  __shared__ float s_k[kCholPanel][kCholPanel + 1];
+  __shared__ __align__(16) float s_k[kCholPanel][kCholPanel];
   __shared__ float s_ldd[kCholPanel][kCholPanel + 1];
   __shared__ float s_inv[kCholPanel];
   const int r = L.r, rp = L.rp;
@@ -450,9 +459,13 @@ __global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const 
         if (active) {
 #pragma unroll 4
           for (int kk = 0; kk < kCholPanel; ++kk) {
-            const float xi = X[(int64_t)(k0 + kk) * rp + i];
+            const float xi = -X[(int64_t)(k0 + kk) * rp + i];
 #pragma unroll
-            for (int c = 0; c < kCholPanel; ++c) p[c] = fmaf(-xi, s_k[kk][c], p[c]);
+            for (int c = 0; c < kCholPanel; c += 4) {
+              const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
+              p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
+              p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
+            }
           }
         }
       }
@@ -465,9 +478,11 @@ __global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const 
           const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
           p[c] = lic;
 #pragma unroll
-          for (int c2 = c + 1; c2 < kCholPanel; ++c2) {
-            const float l2 = __shfl_sync(0xffffffffu, lic, c2);
-            if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+          for (int c2 = 0; c2 < kCholPanel; ++c2) {
+            if (c2 > c) {
+              const float l2 = __shfl_sync(0xffffffffu, lic, c2);
+              if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+            }
           }
           if (lane == c) dd[kCholPanel * kCholPanel + c] = inv;
         }
@@ -503,7 +518,8 @@ __global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const 
 }
 
 void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
-  sp_cholesky_kernel<<<n_layers, std::min(rp_max, 1024), 0, st>>>(d_layers);
+  sp_cholesky_kernel<512, 16><<<n_layers, std::min(rp_max, 512), 0, st>>>(d_layers);
+  if (rp_max > 512) sp_cholesky_kernel<1024, 4><<<n_layers, 1024, 0, st>>>(d_layers);
 }
 
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st) {
