@@ -205,6 +205,10 @@ int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
 /* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
  * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
+/* Eigen-solver launch scheme: 1 (default) = when every block pair of the batch fits on the GPU at once (one CTA
+ * per SM), the whole solve is one cooperative launch with grid barriers between Jacobi steps and a single host
+ * wait at its end; larger batches, or 0, use one launch per step and one host wait per sweep.              */
+int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
 
 #ifdef __cplusplus
 }

@@ -28,6 +28,7 @@ struct atomo_ctx {
   int refine_min_short = 2048;       // layers with at least this short side get the sigma refinement pass
   bool tc_gram = true;               // Gram matrix on tcgen05 where the layer's layout allows it
   bool tc_ok = false;                // tensor-map entry point found
+  bool persistent_eig = true;        // whole eigen-solve in one cooperative launch when the batch fits the GPU
   std::string err;
 };
 
@@ -191,6 +192,12 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
   if (!ctx || max_sweeps < 1 || max_sweeps > 1000 || !(tol > 0.0f) || !(tol < 1.0f)) return ATOMO_ERR_INVALID_ARG;
   ctx->max_sweeps = max_sweeps;
   ctx->tol = tol;
+  return ATOMO_OK;
+}
+
+int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  ctx->persistent_eig = enabled != 0;
   return ATOMO_OK;
 }
 
@@ -384,11 +391,24 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   stage_begin(ctx, ATOMO_STAGE_EIG, st);
   int t16 = 0, t8 = 0;
   int64_t n_eig_launch = 0;
+  const bool persistent = ctx->persistent_eig && (int)pairs16.size() <= sp_jacobi_persistent_capacity(rp16_max);
+  if (persistent) {
+    // one cooperative launch: d_flag[3] receives the number of steps executed
+    const uint32_t init[2] = {(uint32_t)n_layers, 0u};
+    CK(cudaMemcpyAsync(d_flag + 2, init, sizeof(init), cudaMemcpyHostToDevice, st));
+    const int t_max = steps16 * max_sweeps;
+    const int e = launch_sp_jacobi_persistent(d_layers, n_layers, d_p16, (int)pairs16.size(), rp16_max, t_max, max_sweeps,
+                                              ctx->tol, d_flag + 2, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
+    launch_sp_check(d_layers, n_layers, t_max, 0, max_sweeps, d_flag, st);
+    n_eig_launch = 2;
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+  } else
   for (int it = 0; it < max_sweeps; ++it) {
     for (int j = 0; j < steps16; ++j, ++t16, ++n_eig_launch)
       launch_sp_jacobi_step(d_layers, d_p16, (int)pairs16.size(), 16, rp16_max, t16, max_sweeps, ctx->tol, st);
-    for (int j = 0; j < steps8; ++j, ++t8, ++n_eig_launch)
-      launch_sp_jacobi_step(d_layers, d_p8, (int)pairs8.size(), 8, 1024, t8, max_sweeps, ctx->tol, st);
     launch_sp_check(d_layers, n_layers, t16, t8, max_sweeps, d_flag, st);
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));

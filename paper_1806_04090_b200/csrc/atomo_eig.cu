@@ -257,6 +257,31 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 
 constexpr int kJacobiThreads = 32 * kJB;
 
+__device__ __forceinline__ void jacobi_dispatch(const SpLayer& L, int slot, int sweep, int local, float tol, float* smem) {
+  if (L.acc) {
+    switch (L.rp) {
+      case 32: jacobi_block_pair<32, true, 1>(L, slot, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, true, 1>(L, slot, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, true, 1>(L, slot, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, true, 1>(L, slot, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, true, 1>(L, slot, sweep, local, tol, smem); break;
+      default: break;
+    }
+  } else {
+    switch (L.rp) {
+      case 32: jacobi_block_pair<32, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 64: jacobi_block_pair<64, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 128: jacobi_block_pair<128, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 256: jacobi_block_pair<256, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 512: jacobi_block_pair<512, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 1024: jacobi_block_pair<1024, false, 1>(L, slot, sweep, local, tol, smem); break;
+      case 2048: jacobi_block_pair<2048, false, 2>(L, slot, sweep, local, tol, smem); break;
+      case 4096: jacobi_block_pair<4096, false, 4>(L, slot, sweep, local, tol, smem); break;
+      default: break;
+    }
+  }
+}
+
 // One Jacobi step for every layer: mode 1 layers with padded short side <= 4096, mode 0 layers with <= 512.
 __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const SpLayer* __restrict__ layers,
                                                                         const TileRef* __restrict__ pairs, int t,
@@ -268,31 +293,65 @@ __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const Sp
   const int sweep = t / steps, local = t % steps;
   if (sweep >= max_sweeps) return;
   if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
-  if (L.acc) {
-    switch (L.rp) {
-      case 32: jacobi_block_pair<32, true, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, true, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, true, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, true, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, true, 1>(L, ref.a, sweep, local, tol, smem); break;
-      default: break;
+  jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
+}
+
+// The whole eigen-solve in one cooperative launch, for batches whose block pairs are all co-resident (one CTA per
+// SM): a grid barrier takes the place of the kernel boundary between steps, and no host round trip is needed
+// to see convergence.  Every CTA must leave the loop in the same iteration, so the exit test reads only
+// values that are final once the barrier has been passed: the rotation counts of sweeps that are complete
+// after t + 1 steps (a completed sweep is never touched again) -- never a counter that a CTA running ahead
+// could change.  `state[1]` receives the number of steps executed.
+__global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_persistent_kernel(const SpLayer* __restrict__ layers,
+                                                                              int n_layers,
+                                                                              const TileRef* __restrict__ pairs,
+                                                                              int t_max, int max_sweeps, float tol,
+                                                                              uint32_t* __restrict__ state) {
+  extern __shared__ __align__(16) float smem[];
+  cg::grid_group grid = cg::this_grid();
+  const TileRef ref = pairs[blockIdx.x];
+  const SpLayer& L = layers[ref.layer];
+  const int steps = L.nb - 1;
+  int t = 0;
+  for (; t < t_max; ++t) {
+    const int sweep = t / steps, local = t % steps;
+    // a layer rests once one of its completed sweeps rotated nothing (later sweeps then stay at zero)
+    if (sweep < max_sweeps && !(sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) == 0))
+      jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
+    __threadfence();
+    grid.sync();
+    int pending = 0;
+    for (int l = threadIdx.x; l < n_layers; l += kJacobiThreads) {
+      const int st_l = layers[l].nb - 1;
+      const int done_sweeps = min((t + 1) / st_l, max_sweeps);
+      const bool done = done_sweeps >= max_sweeps ||
+                        (done_sweeps >= 1 && *(volatile uint32_t*)(layers[l].rot_count + done_sweeps - 1) == 0);
+      pending |= done ? 0 : 1;
     }
-  } else {
-    switch (L.rp) {
-      case 32: jacobi_block_pair<32, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 1024: jacobi_block_pair<1024, false, 1>(L, ref.a, sweep, local, tol, smem); break;
-      case 2048: jacobi_block_pair<2048, false, 2>(L, ref.a, sweep, local, tol, smem); break;
-      case 4096: jacobi_block_pair<4096, false, 4>(L, ref.a, sweep, local, tol, smem); break;
-      default: break;
-    }
+    if (!__syncthreads_or(pending)) break;
   }
+  if (blockIdx.x == 0 && threadIdx.x == 0) state[1] = (uint32_t)min(t + 1, t_max);
 }
 
 constexpr int kJacobiSmem = 32 * 1024 * 4 + 1024;   // 32 rows of up to 1024 floats + norms and factors
+
+int sp_jacobi_persistent_capacity(int row_floats_max) {
+  int dev = 0, sms = 0, per_sm = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sp_jacobi_persistent_kernel, kJacobiThreads, smem) != cudaSuccess) return 0;
+  return sms * per_sm;
+}
+
+int launch_sp_jacobi_persistent(const SpLayer* d_layers, int n_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
+                                int t_max, int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st) {
+  const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
+  void* args[] = {(void*)&d_layers, (void*)&n_layers, (void*)&d_pairs, (void*)&t_max, (void*)&max_sweeps, (void*)&tol,
+                  (void*)&d_state};
+  return (int)cudaLaunchCooperativeKernel((const void*)sp_jacobi_persistent_kernel, dim3(n_pairs), dim3(kJacobiThreads), args,
+                                          smem, st);
+}
 
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st) {
@@ -531,7 +590,9 @@ int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n
 int sp_cholesky_big_rows_per_cta() { return kCholBigThreads; }
 
 int sp_configure_eig() {
-  return (int)cudaFuncSetAttribute(sp_jacobi_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  cudaError_t e = cudaFuncSetAttribute(sp_jacobi_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  if (e != cudaSuccess) return (int)e;
+  return (int)cudaFuncSetAttribute(sp_jacobi_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
 }
 
 }  // namespace atomo

@@ -88,6 +88,10 @@ void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   
 // one Jacobi step (global step index t) for every layer of one (B, RP) class
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
+// whole eigen-solve in one cooperative launch when all block pairs are co-resident; returns a cudaError_t
+int sp_jacobi_persistent_capacity(int row_floats_max);
+int launch_sp_jacobi_persistent(const SpLayer* d_layers, int n_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
+                                int t_max, int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
 void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 // layers with more than 1024 rows: cooperative launch, returns a cudaError_t
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
