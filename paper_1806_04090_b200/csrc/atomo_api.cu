@@ -249,7 +249,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   const int map_bytes = sp_tc_map_bytes();
   std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
   int chol_panels = 0;
-  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0;
+  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0, r_max_tall = 0;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
     const atomo_mat& m = layers[l];
@@ -283,7 +283,17 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     }
     d.bp_tiles = d.tall ? (d.L + sp_bp_rows_per_tile() - 1) / sp_bp_rows_per_tile()
                         : (d.L + sp_bp_cols_per_tile() - 1) / sp_bp_cols_per_tile();
-    for (int t = 0; t < d.bp_tiles; ++t) bp_tiles.push_back({l, t, 0, 0});
+    {   // row chunks of the wide back-projection: 64 rows each, fewer and longer when k_cap makes the partials large
+      const int64_t per_chunk = (int64_t)d.k_cap * d.L * (int64_t)sizeof(float);
+      const int unit = sp_bp_chunk_rows();
+      const int want = (d.r + unit - 1) / unit;
+      const int fit = (int)std::max<int64_t>(1, ((int64_t)32 << 20) / per_chunk);
+      const int chunks = d.tall ? 1 : std::min(want, fit);
+      d.bp_chunk_rows = ((d.r + chunks - 1) / chunks + unit - 1) / unit * unit;
+      d.bp_chunks = d.tall ? 1 : (d.r + d.bp_chunk_rows - 1) / d.bp_chunk_rows;
+    }
+    for (int t = 0; t < d.bp_tiles; ++t) for (int c = 0; c < d.bp_chunks; ++c) bp_tiles.push_back({l, t, c, 0});
+    if (d.tall) r_max_tall = std::max(r_max_tall, d.r);
     d.refine = d.r >= ctx->refine_min_short ? 1 : 0;
     d.refine_tiles = (d.L + 63) / 64;
     if (d.refine)
@@ -320,7 +330,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       d.dbg_short = (dbg && dbg->short_vecs) ? dbg->short_vecs + dbg_sq : nullptr;
       dbg_atoms += d.r; dbg_words += (d.r + 31) / 32; dbg_sq += (size_t)d.r * d.r;
       d.p_sel = A.take<float>(d.k_cap);
-      d.bp_partials = A.take<float>((size_t)d.bp_tiles * d.k_cap);
+      d.bp_part = A.take<float>((size_t)d.bp_chunks * d.k_cap * d.L);
       d.scale = A.take<float>(1);
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
@@ -426,7 +436,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S4: long-side vectors of the kept atoms ----
   stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);
-  launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), r_max, st);
+  launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), std::max(r_max_tall, 1), st);
   launch_sp_finish_atoms(d_layers, n_layers, st);
   stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, 2);
   CK(cudaGetLastError());

@@ -64,8 +64,8 @@ struct SpLayer {
   float* sigma; float* prob;   // r    descending (debug buffers or workspace)
   uint32_t* mask_words;        // ceil(r/32)
   float* p_sel;                // k_cap: p of the kept atoms
-  float* bp_partials;          // [bp_tiles][k_cap] partial squared norms of the long vectors
-  int bp_tiles;
+  float* bp_part;              // [bp_chunks][k_cap][L] row-chunk partial sums of the long vectors
+  int bp_tiles, bp_chunks, bp_chunk_rows;
   uint32_t* rot_count;         // [max_sweeps] rotations applied in each sweep
   float* scale;                // 1 float: power-of-two scaling applied to A
   float* chol_dd;              // 32 x 32 + 32 floats: diagonal block published by its owner (layers > 1024 rows)
@@ -118,6 +118,7 @@ void launch_sp_gram_tc(const SpLayer* d_layers, const void* d_maps, const TileRe
                        cudaStream_t st);
 int sp_bp_rows_per_tile();
 int sp_bp_cols_per_tile();
+int sp_bp_chunk_rows();
 int sp_decode_tile_rows();
 int sp_decode_tile_cols();
 

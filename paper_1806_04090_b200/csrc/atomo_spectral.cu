@@ -413,18 +413,21 @@ void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, 
 
 // =================================================================================================
 // back-projection: long-side vector of each kept atom.
-//   rows <= cols: w_a[c]   = sum_i G[i][c] u_a[i]      (tile = 256 columns, thread per column)
-//   rows >  cols: w_a[row] = sum_c G[row][c] v_a[c]    (tile = 32 rows, warp per row)
-// Unnormalised w goes to payload longv; the squared norm of each tile goes to bp_partials.
+//   rows <= cols: w_a[c]   = sum_i G[i][c] u_a[i]   tile = 256 columns x one chunk of rows (a multiple of 64, set
+//                                                     per layer), thread per column, 8 row loads in flight;
+//                                                     chunk partials go to bp_part and are summed in chunk
+//                                                     order by sp_finish_atoms
+//   rows >  cols: w_a[row] = sum_c G[row][c] v_a[c]   tile = 32 rows, warp per row (one chunk)
 // =================================================================================================
-constexpr int kBpThreads = 256, kBpAtoms = 8, kBpCols = 256, kBpRows = 32;
+constexpr int kBpThreads = 256, kBpAtoms = 8, kBpCols = 256, kBpRows = 32, kBpChunk = 64;
 int sp_bp_cols_per_tile() { return kBpCols; }
 int sp_bp_rows_per_tile() { return kBpRows; }
+int sp_bp_chunk_rows() { return kBpChunk; }
 
 __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLayer* __restrict__ layers,
                                                                     const TileRef* __restrict__ tiles) {
-  extern __shared__ __align__(16) float s_u[];          // kBpAtoms x r
-  __shared__ float s_part[kBpThreads / 32][kBpAtoms];
+  __shared__ float s_u[kBpAtoms][kBpChunk];            // wide: the chunk's components of up to 8 short-side vectors
+  extern __shared__ __align__(16) float s_v[];         // tall: kBpAtoms x r
   const TileRef ref = tiles[blockIdx.x];
   const SpLayer& L = layers[ref.layer];
   const uint32_t k = L.hdr->k;
@@ -435,26 +438,41 @@ __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLaye
   for (uint32_t a0 = 0; a0 < k; a0 += kBpAtoms) {
     const int na = min((uint32_t)kBpAtoms, k - a0);
     __syncthreads();
-    for (int idx = tid; idx < na * r; idx += kBpThreads) s_u[idx] = L.shortv[(int64_t)a0 * r + idx];
-    __syncthreads();
-    float nrm[kBpAtoms];
-#pragma unroll
-    for (int a = 0; a < kBpAtoms; ++a) nrm[a] = 0.f;
     if (!L.tall) {
+      const int row_lo = ref.b * L.bp_chunk_rows, row_hi = min(r, row_lo + L.bp_chunk_rows);
       const int c = ref.a * kBpCols + tid;
       float acc[kBpAtoms];
 #pragma unroll
       for (int a = 0; a < kBpAtoms; ++a) acc[a] = 0.f;
-      if (c < len) {
-        for (int i = 0; i < r; ++i) {
-          const float g = __ldg(G + (int64_t)i * ld + c);
-#pragma unroll
-          for (int a = 0; a < kBpAtoms; ++a) if (a < na) acc[a] = fmaf(g, s_u[a * r + i], acc[a]);
+      for (int i0 = row_lo; i0 < row_hi; i0 += kBpChunk) {
+        const int ni = min(kBpChunk, row_hi - i0);
+        if (i0 > row_lo) __syncthreads();
+        for (int idx = tid; idx < na * kBpChunk; idx += kBpThreads) {
+          const int a = idx / kBpChunk, i = idx % kBpChunk;
+          s_u[a][i] = i < ni ? L.shortv[(int64_t)(a0 + a) * r + i0 + i] : 0.0f;
         }
+        __syncthreads();
+        if (c < len) {
+          const float* gp = G + (int64_t)i0 * ld + c;
+          for (int i = 0; i < ni; i += 8) {
+            float g[8];
 #pragma unroll
-        for (int a = 0; a < kBpAtoms; ++a) if (a < na) { L.longv[(int64_t)(a0 + a) * len + c] = acc[a]; nrm[a] = acc[a] * acc[a]; }
+            for (int u = 0; u < 8; ++u) g[u] = (i + u < ni) ? __ldg(gp + (int64_t)(i + u) * ld) : 0.0f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+#pragma unroll
+              for (int a = 0; a < kBpAtoms; ++a) acc[a] = fmaf(g[u], s_u[a][i + u], acc[a]);   // rows past ni hold zeros
+          }
+        }
+      }
+      if (c < len) {
+#pragma unroll
+        for (int a = 0; a < kBpAtoms; ++a)
+          if (a < na) L.bp_part[((int64_t)ref.b * L.k_cap + a0 + a) * len + c] = acc[a];
       }
     } else {
+      for (int idx = tid; idx < na * r; idx += kBpThreads) s_v[idx] = L.shortv[(int64_t)a0 * r + idx];
+      __syncthreads();
       for (int rr = w; rr < kBpRows; rr += kBpThreads / 32) {
         const int row = ref.a * kBpRows + rr;
         if (row >= len) break;
@@ -464,22 +482,14 @@ __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLaye
         for (int c = lane; c < r; c += 32) {
           const float g = __ldg(G + (int64_t)row * ld + c);
 #pragma unroll
-          for (int a = 0; a < kBpAtoms; ++a) if (a < na) acc[a] = fmaf(g, s_u[a * r + c], acc[a]);
+          for (int a = 0; a < kBpAtoms; ++a) if (a < na) acc[a] = fmaf(g, s_v[a * r + c], acc[a]);
         }
 #pragma unroll
         for (int a = 0; a < kBpAtoms; ++a) {
           acc[a] = warp_sum(acc[a]);
-          if (a < na && lane == 0) { L.longv[(int64_t)(a0 + a) * len + row] = acc[a]; nrm[a] += acc[a] * acc[a]; }
+          if (a < na && lane == 0) L.bp_part[(int64_t)(a0 + a) * len + row] = acc[a];
         }
       }
-    }
-#pragma unroll
-    for (int a = 0; a < kBpAtoms; ++a) { nrm[a] = warp_sum(nrm[a]); if (lane == 0) s_part[w][a] = nrm[a]; }
-    __syncthreads();
-    if (tid < na) {
-      float tot = 0.f;
-      for (int j = 0; j < kBpThreads / 32; ++j) tot += s_part[j][tid];
-      L.bp_partials[(int64_t)ref.a * L.k_cap + a0 + tid] = tot;
     }
   }
 }
@@ -491,30 +501,38 @@ int sp_configure() {
                                    kBpAtoms * kMaxShort * (int)sizeof(float));
 }
 
-void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st) {
+void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max_tall, cudaStream_t st) {
   if (n_tiles > 0)
-    sp_backproject_kernel<<<n_tiles, kBpThreads, kBpAtoms * r_max * sizeof(float), st>>>(d_layers, d_tiles);
+    sp_backproject_kernel<<<n_tiles, kBpThreads, kBpAtoms * r_max_tall * sizeof(float), st>>>(d_layers, d_tiles);
 }
 
-// sigma_a = ||w_a||, coef_a = sigma_a / p_a, w_a normalised.  One CTA per layer.
+// w_a = sum over row chunks (in chunk order), sigma_a = ||w_a||, coef_a = sigma_a / p_a, long vector = w_a / sigma_a.
+// One CTA per layer.
 __global__ void __launch_bounds__(256) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.x];
   const uint32_t k = L.hdr->k;
+  const int len = L.L;
+  __shared__ double s_red[256];
   __shared__ float s_inv;
   for (uint32_t a = 0; a < k; ++a) {
-    if (threadIdx.x < 32) {
-      double tot = 0.0;
-      for (int t = threadIdx.x; t < L.bp_tiles; t += 32) tot += (double)L.bp_partials[(int64_t)t * L.k_cap + a];
-      tot = warp_sum(tot);
-      if (threadIdx.x == 0) {
-        const float sg = (float)sqrt(tot);
-        L.coef[a] = sg / L.p_sel[a];
-        s_inv = sg > 0.f ? 1.0f / sg : 0.f;
-      }
+    double part = 0.0;
+    for (int j = threadIdx.x; j < len; j += 256) {
+      float wv = 0.f;
+      for (int ch = 0; ch < L.bp_chunks; ++ch) wv += L.bp_part[((int64_t)ch * L.k_cap + a) * len + j];
+      L.longv[(int64_t)a * len + j] = wv;
+      part += (double)wv * (double)wv;
+    }
+    s_red[threadIdx.x] = part;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
+    if (threadIdx.x == 0) {
+      const float sg = (float)sqrt(s_red[0]);
+      L.coef[a] = sg / L.p_sel[a];
+      s_inv = sg > 0.f ? 1.0f / sg : 0.f;
     }
     __syncthreads();
     const float inv = s_inv;
-    for (int j = threadIdx.x; j < L.L; j += 256) L.longv[(int64_t)a * L.L + j] *= inv;
+    for (int j = threadIdx.x; j < len; j += 256) L.longv[(int64_t)a * len + j] *= inv;
     __syncthreads();
   }
 }
