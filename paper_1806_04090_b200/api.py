@@ -127,7 +127,7 @@ def payload_bytes_entrywise(lengths: Sequence[int], k_cap: int) -> int:
 
 def default_k_cap(s: float, n_atoms: int) -> int:
     """k is a sum of independent Bernoulli draws with mean <= s: s + 8 sqrt(s) + 8 is never reached."""
-    return int(min(n_atoms, np.ceil(s + 8.0 * np.sqrt(s) + 8.0)))
+    return int(min(n_atoms, np.ceil(s + 8.0 * np.sqrt(max(float(s), 0.0)) + 8.0)))
 
 
 @dataclass
