@@ -344,7 +344,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     // zero-filled region: rotation counters and the X matrices
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
     size_t z0 = A.off;
-    for (int l = 0; l < n_layers; ++l) L[l].rot_count = A.take<uint32_t>(max_sweeps);
+    for (int l = 0; l < n_layers; ++l) { L[l].rot_count = A.take<uint32_t>(max_sweeps); L[l].step_bar = A.take<uint32_t>(1); }
     for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * L[l].ldx);
     zero_beg = zb; zero_bytes = A.off - z0;
     for (int l = 0; l < n_layers; ++l) {
@@ -403,18 +403,17 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   int64_t n_eig_launch = 0;
   const bool persistent = ctx->persistent_eig && (int)pairs16.size() <= sp_jacobi_persistent_capacity(rp16_max);
   if (persistent) {
-    // one cooperative launch: d_flag[3] receives the number of steps executed
-    const uint32_t init[2] = {(uint32_t)n_layers, 0u};
-    CK(cudaMemcpyAsync(d_flag + 2, init, sizeof(init), cudaMemcpyHostToDevice, st));
+    // one cooperative launch: d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
+    CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
     const int t_max = steps16 * max_sweeps;
-    const int e = launch_sp_jacobi_persistent(d_layers, n_layers, d_p16, (int)pairs16.size(), rp16_max, t_max, max_sweeps,
-                                              ctx->tol, d_flag + 2, st);
+    const int e = launch_sp_jacobi_persistent(d_layers, d_p16, (int)pairs16.size(), rp16_max, max_sweeps, ctx->tol, d_flag + 2, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
     launch_sp_check(d_layers, n_layers, t_max, 0, max_sweeps, d_flag, st);
     n_eig_launch = 2;
-    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+    if (ctx->h_flag[2] != 0) { ctx->err = "a step barrier of the persistent eigen-solve ran out of polls"; return ATOMO_ERR_TIMEOUT; }
   } else
   for (int it = 0; it < max_sweeps; ++it) {
     for (int j = 0; j < steps16; ++j, ++t16, ++n_eig_launch)

@@ -319,41 +319,51 @@ __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const Sp
   jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
 }
 
-// The whole eigen-solve in one cooperative launch, for batches whose block pairs are all co-resident (one CTA per
-// SM): a grid barrier takes the place of the kernel boundary between steps, and no host round trip is needed
-// to see convergence.  Every CTA must leave the loop in the same iteration, so the exit test reads only
-// values that are final once the barrier has been passed: the rotation counts of sweeps that are complete
-// after t + 1 steps (a completed sweep is never touched again) -- never a counter that a CTA running ahead
-// could change.  `state[1]` receives the number of steps executed.
+// The whole eigen-solve in one cooperative launch, for batches whose block pairs are all co-resident (one CTA
+// per SM; the cooperative launch is what guarantees that).  The kernel boundary between steps becomes a barrier
+// among the CTAs of ONE layer (layers are independent): a counter in global memory that every CTA of the layer
+// increments after its stores and then polls until all have arrived.  The poll is bounded: a CTA that gives up
+// raises state[0] and leaves, and so will the others of its layer.  A layer stops at the first sweep boundary
+// whose finished sweep rotated nothing; its CTAs all read the same, final count there, because every one of them
+// has passed the barrier that closes that sweep.  state[1] receives the largest number of steps any layer took.
+constexpr uint32_t kStepBarSpinLimit = 1u << 22;
+
 __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_persistent_kernel(const SpLayer* __restrict__ layers,
-                                                                              int n_layers,
                                                                               const TileRef* __restrict__ pairs,
-                                                                              int t_max, int max_sweeps, float tol,
+                                                                              int max_sweeps, float tol,
                                                                               uint32_t* __restrict__ state) {
   extern __shared__ __align__(16) float smem[];
-  cg::grid_group grid = cg::this_grid();
+  __shared__ int s_fail;
   const TileRef ref = pairs[blockIdx.x];
   const SpLayer& L = layers[ref.layer];
-  const int steps = L.nb - 1;
+  const int steps = L.nb - 1, n_ctas = L.nb / 2;
+  const int t_max = steps * max_sweeps;
   int t = 0;
   for (; t < t_max; ++t) {
     const int sweep = t / steps, local = t % steps;
-    // a layer rests once one of its completed sweeps rotated nothing (later sweeps then stay at zero)
-    if (sweep < max_sweeps && !(sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) == 0))
-      jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
-    __threadfence();
-    grid.sync();
-    int pending = 0;
-    for (int l = threadIdx.x; l < n_layers; l += kJacobiThreads) {
-      const int st_l = layers[l].nb - 1;
-      const int done_sweeps = min((t + 1) / st_l, max_sweeps);
-      const bool done = done_sweeps >= max_sweeps ||
-                        (done_sweeps >= 1 && *(volatile uint32_t*)(layers[l].rot_count + done_sweeps - 1) == 0);
-      pending |= done ? 0 : 1;
+    if (local == 0 && sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) == 0) break;
+    jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
+    __syncthreads();
+    if (n_ctas > 1) {
+      if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(L.step_bar, 1u);
+        const uint32_t target = (uint32_t)(t + 1) * (uint32_t)n_ctas;
+        uint32_t spins = 0;
+        int fail = 0;
+        while (*(volatile uint32_t*)L.step_bar < target)
+          if (++spins > kStepBarSpinLimit) { fail = 1; break; }
+        __threadfence();
+        s_fail = fail;
+      }
+      __syncthreads();
+      if (s_fail) {
+        if (threadIdx.x == 0) atomicExch(state, 1u);
+        break;
+      }
     }
-    if (!__syncthreads_or(pending)) break;
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0) state[1] = (uint32_t)min(t + 1, t_max);
+  if (threadIdx.x == 0) atomicMax(state + 1, (uint32_t)t);
 }
 
 constexpr int kJacobiSmem = 32 * 1024 * 4 + 1024;   // 32 rows of up to 1024 floats + norms and factors
@@ -367,11 +377,10 @@ int sp_jacobi_persistent_capacity(int row_floats_max) {
   return sms * per_sm;
 }
 
-int launch_sp_jacobi_persistent(const SpLayer* d_layers, int n_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
-                                int t_max, int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st) {
+int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
+                                int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st) {
   const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
-  void* args[] = {(void*)&d_layers, (void*)&n_layers, (void*)&d_pairs, (void*)&t_max, (void*)&max_sweeps, (void*)&tol,
-                  (void*)&d_state};
+  void* args[] = {(void*)&d_layers, (void*)&d_pairs, (void*)&max_sweeps, (void*)&tol, (void*)&d_state};
   return (int)cudaLaunchCooperativeKernel((const void*)sp_jacobi_persistent_kernel, dim3(n_pairs), dim3(kJacobiThreads), args,
                                           smem, st);
 }

@@ -67,6 +67,7 @@ struct SpLayer {
   float* bp_part;              // [bp_chunks][k_cap][L] row-chunk partial sums of the long vectors
   int bp_tiles, bp_chunks, bp_chunk_rows;
   uint32_t* rot_count;         // [max_sweeps] rotations applied in each sweep
+  uint32_t* step_bar;          // arrivals of the layer's CTAs at the step barrier of the persistent eigen-solve
   float* scale;                // 1 float: power-of-two scaling applied to A
   float* chol_dd;              // 32 x 32 + 32 floats: diagonal block published by its owner (layers > 1024 rows)
   float* dbg_short;            // r x r or nullptr
@@ -90,8 +91,8 @@ void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int 
                            int t, int max_sweeps, float tol, cudaStream_t st);
 // whole eigen-solve in one cooperative launch when all block pairs are co-resident; returns a cudaError_t
 int sp_jacobi_persistent_capacity(int row_floats_max);
-int launch_sp_jacobi_persistent(const SpLayer* d_layers, int n_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
-                                int t_max, int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
+int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
+                                int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
 void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 // layers with more than 1024 rows: cooperative launch, returns a cudaError_t
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
