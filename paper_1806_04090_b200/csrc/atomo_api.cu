@@ -249,7 +249,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   const int map_bytes = sp_tc_map_bytes();
   std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
   int chol_panels = 0;
-  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0, r_max_tall = 0;
+  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0, r_max_tall = 0, k_cap_max = 1;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
     const atomo_mat& m = layers[l];
@@ -263,6 +263,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d.B = d.ldx <= 1024 ? 16 : (d.ldx == 2048 ? 8 : 4);          // a rotation is shared by 1, 2 or 4 warps
     d.nb = d.rp / d.B;
     d.layer = (uint32_t)l; d.k_cap = lay[l].kc;
+    k_cap_max = std::max(k_cap_max, (int)d.k_cap);
     r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
     d.tc = 0;
@@ -390,7 +391,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   launch_sp_gram_tc(d_layers, d_maps, d_tc, (int)tc_tiles.size(), d_flag + 1, st);
   launch_sp_scale(d_layers, n_layers, st);
   if (ctx->eig_mode != 0) {
-    launch_sp_cholesky(d_layers, n_layers, rp_max, st);
+    const int ec = launch_sp_cholesky(d_layers, n_layers, rp_max, st);
+    if (ec != 0) return fail_cuda(ctx, (cudaError_t)ec, "cudaLaunchKernelEx(cholesky)");
     const int e = launch_sp_cholesky_big(d_layers, d_chol, (int)chol_ctas.size(), chol_panels, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(cholesky)");
   }
@@ -436,7 +438,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // ---- S4: long-side vectors of the kept atoms ----
   stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);
   launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), std::max(r_max_tall, 1), st);
-  launch_sp_finish_atoms(d_layers, n_layers, st);
+  launch_sp_finish_atoms(d_layers, n_layers, k_cap_max, st);
   stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, 2);
   CK(cudaGetLastError());
   return ATOMO_OK;

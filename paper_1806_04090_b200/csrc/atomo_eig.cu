@@ -511,6 +511,102 @@ __global__ void __launch_bounds__(kThreads) sp_cholesky_kernel(const SpLayer* __
   }
 }
 
+// The same factorisation spread over a cluster of 8 CTAs per layer (layers of up to 1024 rows): the panel
+// update is FMA-bound on one SM, so each CTA takes max(32, rp / 8) consecutive rows, one thread per row.
+// Per panel: every CTA updates its rows; the warp that owns the diagonal block factors it and publishes it in
+// global memory; cluster barrier; every CTA solves its rows against it and stores them; cluster barrier (the
+// next panel reads rows of L written by other CTAs; those reads bypass L1).
+constexpr int kCholClusterCtas = 8, kCholClusterThreads = 128;
+
+__global__ void __launch_bounds__(kCholClusterThreads) sp_cholesky_cluster_kernel(const SpLayer* __restrict__ layers) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const SpLayer& L = layers[blockIdx.x / kCholClusterCtas];
+  if (L.acc || L.rp > 1024) return;                        // the whole cluster leaves: route 0 / sp_cholesky_big_kernel
+  __shared__ __align__(16) float s_k[kCholPanel][kCholPanel];
+  __shared__ float s_ldd[kCholPanel][kCholPanel + 1];
+  __shared__ float s_inv[kCholPanel];
+  const int r = L.r, rp = L.rp;
+  const int rows_per_cta = max(32, rp / kCholClusterCtas);
+  const int tid = threadIdx.x, lane = tid % 32;
+  const int i = (int)cluster.block_rank() * rows_per_cta + tid;      // this thread's row
+  const bool has_row = tid < rows_per_cta && i < r;
+  const float* __restrict__ A = L.A;
+  const int64_t lda = L.lda;
+  float* X = L.X;
+  float* dd = L.chol_dd;                                   // published diagonal block: 32 x 32, then 32 inverses
+  for (int j0 = 0; j0 < r; j0 += kCholPanel) {
+    const bool active = has_row && i >= j0;
+    float p[kCholPanel];
+#pragma unroll
+    for (int c = 0; c < kCholPanel; ++c) p[c] = (active && j0 + c < r) ? A[(int64_t)(j0 + c) * lda + i] : 0.0f;
+    const bool cta_active = (int)cluster.block_rank() * rows_per_cta + rows_per_cta > j0;   // some row of this CTA is >= j0
+    if (cta_active) {
+      for (int k0 = 0; k0 < j0; k0 += kCholPanel) {
+        __syncthreads();
+        for (int idx = tid; idx < kCholPanel * kCholPanel; idx += kCholClusterThreads) {
+          const int kk = idx / kCholPanel, c = idx % kCholPanel;
+          s_k[kk][c] = __ldcg(X + (int64_t)(k0 + kk) * rp + j0 + c);
+        }
+        __syncthreads();
+        if (active) {
+#pragma unroll 8
+          for (int kk = 0; kk < kCholPanel; ++kk) {
+            const float xi = -X[(int64_t)(k0 + kk) * rp + i];
+#pragma unroll
+            for (int c = 0; c < kCholPanel; c += 4) {
+              const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
+              p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
+              p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
+            }
+          }
+        }
+      }
+      if (tid < rows_per_cta && i >= j0 && i < j0 + kCholPanel) {        // the warp that owns the diagonal block
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) {
+          const float d = __shfl_sync(0xffffffffu, p[c], c);
+          const float lcc = d > kPivotFloor ? sqrtf(d) : 0.0f;
+          const float inv = lcc > 0.0f ? 1.0f / lcc : 0.0f;
+          const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
+          p[c] = lic;
+#pragma unroll
+          for (int c2 = 0; c2 < kCholPanel; ++c2) {
+            if (c2 > c) {
+              const float l2 = __shfl_sync(0xffffffffu, lic, c2);
+              if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
+            }
+          }
+          if (lane == c) dd[kCholPanel * kCholPanel + c] = inv;
+        }
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) dd[lane * kCholPanel + c] = p[c];
+      }
+    }
+    cluster.sync();
+    if (cta_active) {
+      for (int idx = tid; idx < kCholPanel * kCholPanel; idx += kCholClusterThreads)
+        s_ldd[idx / kCholPanel][idx % kCholPanel] = __ldcg(dd + idx);
+      if (tid < kCholPanel) s_inv[tid] = __ldcg(dd + kCholPanel * kCholPanel + tid);
+      __syncthreads();
+      if (active && i >= j0 + kCholPanel) {
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c) {
+          float acc = p[c];
+#pragma unroll
+          for (int k = 0; k < c; ++k) acc = fmaf(-p[k], s_ldd[c][k], acc);
+          p[c] = acc * s_inv[c];
+        }
+      }
+      if (active) {
+#pragma unroll
+        for (int c = 0; c < kCholPanel; ++c)
+          if (j0 + c < r) X[(int64_t)(j0 + c) * rp + i] = p[c];
+      }
+    }
+    cluster.sync();
+  }
+}
+
 // The same factorisation for layers with more than 1024 rows: kCholBigThreads rows per CTA, several CTAs per
 // layer in one cooperative launch.  Per panel: every CTA updates its rows; the CTA that owns the diagonal block
 // factors it and publishes it; grid barrier; every CTA solves its rows against it and stores them; grid barrier
@@ -608,9 +704,17 @@ __global__ void __launch_bounds__(kCholBigThreads) sp_cholesky_big_kernel(const 
   }
 }
 
-void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
-  sp_cholesky_kernel<512, 16><<<n_layers, std::min(rp_max, 512), 0, st>>>(d_layers);
-  if (rp_max > 512) sp_cholesky_kernel<1024, 4><<<n_layers, 1024, 0, st>>>(d_layers);
+int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
+  (void)rp_max;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_layers * kCholClusterCtas);
+  cfg.blockDim = dim3(kCholClusterThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kCholClusterCtas; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, sp_cholesky_cluster_kernel, d_layers);
 }
 
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st) {

@@ -93,7 +93,7 @@ void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int 
 int sp_jacobi_persistent_capacity(int row_floats_max);
 int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                                 int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
-void launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
+int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 // layers with more than 1024 rows: cooperative launch, returns a cudaError_t
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
 int sp_cholesky_big_rows_per_cta();
@@ -105,7 +105,7 @@ void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_ti
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key,
                                uint32_t kind_step, int max_sweeps, cudaStream_t st);
 void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st);
-void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, cudaStream_t st);
+void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, int k_cap_max, cudaStream_t st);
 void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,
                       cudaStream_t st);
 int sp_configure();          // opt in to large dynamic shared memory; returns cudaError_t

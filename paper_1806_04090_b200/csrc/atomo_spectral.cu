@@ -293,10 +293,17 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
       for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
       lam = (float)warp_sum(d);
     } else {
-      const float* row = L.X + (int64_t)i * ldx;
-      float d = 0.f;
-      for (int j = lane; j < r; j += 32) d = fmaf(row[j], row[voff + j], d);
-      lam = warp_sum(d) * inv_scale;
+      // rows are zero-padded to rp floats (a multiple of 32): whole float4, several loads in flight
+      const float4* x4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx);
+      const float4* v4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx + voff);
+      float d0 = 0.f, d1 = 0.f;
+#pragma unroll 4
+      for (int j = lane; j < rp / 4; j += 32) {
+        const float4 a = x4[j], b = v4[j];
+        d0 = fmaf(a.x, b.x, fmaf(a.y, b.y, d0));
+        d1 = fmaf(a.z, b.z, fmaf(a.w, b.w, d1));
+      }
+      lam = warp_sum(d0 + d1) * inv_scale;
     }
     if (lane == 0) {
       if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
@@ -507,38 +514,32 @@ void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int 
 }
 
 // w_a = sum over row chunks (in chunk order), sigma_a = ||w_a||, coef_a = sigma_a / p_a, long vector = w_a / sigma_a.
-// One CTA per layer.
-__global__ void __launch_bounds__(256) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers) {
-  const SpLayer& L = layers[blockIdx.x];
-  const uint32_t k = L.hdr->k;
+// One CTA per (layer, kept-atom slot); slots beyond the layer's k leave at once.
+__global__ void __launch_bounds__(256) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers, int k_cap_max) {
+  const SpLayer& L = layers[blockIdx.x / k_cap_max];
+  const uint32_t a = blockIdx.x % k_cap_max;
+  if (a >= L.hdr->k) return;
   const int len = L.L;
   __shared__ double s_red[256];
-  __shared__ float s_inv;
-  for (uint32_t a = 0; a < k; ++a) {
-    double part = 0.0;
-    for (int j = threadIdx.x; j < len; j += 256) {
-      float wv = 0.f;
-      for (int ch = 0; ch < L.bp_chunks; ++ch) wv += L.bp_part[((int64_t)ch * L.k_cap + a) * len + j];
-      L.longv[(int64_t)a * len + j] = wv;
-      part += (double)wv * (double)wv;
-    }
-    s_red[threadIdx.x] = part;
-    __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
-    if (threadIdx.x == 0) {
-      const float sg = (float)sqrt(s_red[0]);
-      L.coef[a] = sg / L.p_sel[a];
-      s_inv = sg > 0.f ? 1.0f / sg : 0.f;
-    }
-    __syncthreads();
-    const float inv = s_inv;
-    for (int j = threadIdx.x; j < len; j += 256) L.longv[(int64_t)a * len + j] *= inv;
-    __syncthreads();
+  double part = 0.0;
+  float* out = L.longv + (int64_t)a * len;
+  for (int j = threadIdx.x; j < len; j += 256) {
+    float wv = 0.f;
+    for (int ch = 0; ch < L.bp_chunks; ++ch) wv += L.bp_part[((int64_t)ch * L.k_cap + a) * len + j];
+    out[j] = wv;
+    part += (double)wv * (double)wv;
   }
+  s_red[threadIdx.x] = part;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
+  const float sg = (float)sqrt(s_red[0]);
+  if (threadIdx.x == 0) L.coef[a] = sg / L.p_sel[a];
+  const float inv = sg > 0.f ? 1.0f / sg : 0.f;
+  for (int j = threadIdx.x; j < len; j += 256) out[j] *= inv;       // each thread rescales what it wrote itself
 }
 
-void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
-  sp_finish_atoms_kernel<<<n_layers, 256, 0, st>>>(d_layers);
+void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, int k_cap_max, cudaStream_t st) {
+  sp_finish_atoms_kernel<<<n_layers * k_cap_max, 256, 0, st>>>(d_layers, k_cap_max);
 }
 
 // =================================================================================================
