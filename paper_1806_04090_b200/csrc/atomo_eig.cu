@@ -541,32 +541,53 @@ __global__ void __launch_bounds__(kCholClusterThreads) sp_cholesky_cluster_kerne
     for (int c = 0; c < kCholPanel; ++c) p[c] = (active && j0 + c < r) ? A[(int64_t)(j0 + c) * lda + i] : 0.0f;
     const bool cta_active = (int)cluster.block_rank() * rows_per_cta + rows_per_cta > j0;   // some row of this CTA is >= j0
     if (cta_active) {
+      // p[c] -= sum_{k < j0} L[i][k] L[j0+c][k], 32 values of k at a time; the next chunk's operands (this row's
+      // L[i][k], and this thread's 8 elements of the 32 x 32 tile of the panel rows) are fetched while the current
+      // chunk is multiplied
+      constexpr int kTilePer = kCholPanel * kCholPanel / kCholClusterThreads;
+      float xc[kCholPanel], tn[kTilePer];
+      auto fetch = [&](int k0, float (&xv)[kCholPanel]) {
+#pragma unroll
+        for (int kk = 0; kk < kCholPanel; ++kk) xv[kk] = active ? X[(int64_t)(k0 + kk) * rp + i] : 0.0f;
+#pragma unroll
+        for (int u = 0; u < kTilePer; ++u) {
+          const int idx = tid + u * kCholClusterThreads;
+          tn[u] = __ldcg(X + (int64_t)(k0 + idx / kCholPanel) * rp + j0 + idx % kCholPanel);
+        }
+      };
+      if (j0 > 0) fetch(0, xc);
       for (int k0 = 0; k0 < j0; k0 += kCholPanel) {
-        __syncthreads();
-        for (int idx = tid; idx < kCholPanel * kCholPanel; idx += kCholClusterThreads) {
-          const int kk = idx / kCholPanel, c = idx % kCholPanel;
-          s_k[kk][c] = __ldcg(X + (int64_t)(k0 + kk) * rp + j0 + c);
+        __syncthreads();                                   // the previous chunk's tile has been read by everyone
+#pragma unroll
+        for (int u = 0; u < kTilePer; ++u) {
+          const int idx = tid + u * kCholClusterThreads;
+          s_k[idx / kCholPanel][idx % kCholPanel] = tn[u];
         }
         __syncthreads();
-        if (active) {
-#pragma unroll 8
-          for (int kk = 0; kk < kCholPanel; ++kk) {
-            const float xi = -X[(int64_t)(k0 + kk) * rp + i];
+        float xn[kCholPanel];
+        if (k0 + kCholPanel < j0) fetch(k0 + kCholPanel, xn);
 #pragma unroll
-            for (int c = 0; c < kCholPanel; c += 4) {
-              const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
-              p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
-              p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
-            }
+        for (int kk = 0; kk < kCholPanel; ++kk) {
+          const float xi = -xc[kk];
+#pragma unroll
+          for (int c = 0; c < kCholPanel; c += 4) {
+            const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
+            p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
+            p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
           }
         }
+#pragma unroll
+        for (int kk = 0; kk < kCholPanel; ++kk) xc[kk] = xn[kk];
       }
       if (tid < rows_per_cta && i >= j0 && i < j0 + kCholPanel) {        // the warp that owns the diagonal block
 #pragma unroll
         for (int c = 0; c < kCholPanel; ++c) {
           const float d = __shfl_sync(0xffffffffu, p[c], c);
-          const float lcc = d > kPivotFloor ? sqrtf(d) : 0.0f;
-          const float inv = lcc > 0.0f ? 1.0f / lcc : 0.0f;
+          // 1 / sqrt(d) from the approximation and one Newton step (1 ulp), sqrt(d) = d / sqrt(d)
+          float inv = rsqrt_approx(fmaxf(d, kPivotFloor));
+          inv = inv * fmaf(-0.5f * d * inv, inv, 1.5f);
+          inv = d > kPivotFloor ? inv : 0.0f;
+          const float lcc = d * inv;
           const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
           p[c] = lic;
 #pragma unroll
