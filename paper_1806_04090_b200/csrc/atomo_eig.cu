@@ -31,6 +31,20 @@ __device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int&
   else { p = (round + slot) % m; q = (round - slot + m) % m; }
 }
 
+// Which two blocks a CTA pairs at step `local` of a sweep (nb blocks, a power of two; nb / 2 CTAs; nb - 1 steps).
+// Recursive halving: at level l the blocks form groups of g = nb >> l; inside a group, CTA k keeps block k of
+// the first half for the g / 2 steps of the level while the blocks of the second half pass by, one per step
+// ((k + t) mod g/2 at step t); the next level treats each half as a group of its own.  Every pair of blocks
+// meets exactly once in nb/2 + nb/4 + ... + 1 = nb - 1 steps, and only half of the blocks move at a step.
+struct StepPlan { int bi, bj; bool first_in_level, last_in_level; };
+__device__ __forceinline__ StepPlan step_plan(int nb, int local, int slot) {
+  int g = nb, base = 0;
+  while (local - base >= g / 2) { base += g / 2; g >>= 1; }
+  const int m = g / 2, t = local - base;
+  const int grp = slot / m, k = slot % m;
+  return {grp * g + k, grp * g + m + (k + t) % m, t == 0, t == m - 1};
+}
+
 // A is scaled to trace 1, so a squared row norm below this is an eigenvalue of A below 1e-12 (mode 0)
 // or a singular value of L below 1e-12 (mode 1): rounding noise of the fp32 Gram matrix, not signal.
 constexpr float kRowFloor = 1e-24f;
@@ -171,8 +185,8 @@ __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, fl
 // is done by WPR warps, each holding one segment of the two rows (WPR = 1 for rows of up to 1024 floats).
 // RP = padded short side; ACC: rows are [x | v] (2 RP floats, mode 0), else x only (RP floats, mode 1).
 template <int RP, bool ACC, int WPR>
-__device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, float tol,
-                                                  float* smem) {
+__device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, int sweep, int local, bool resident,
+                                                  float tol, float* smem) {
   constexpr int B = kJB / WPR;
   constexpr int LD = ACC ? 2 * RP : RP;                 // floats per row
   constexpr int SEG = LD / WPR;                         // floats per warp segment
@@ -187,8 +201,11 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const int pi = w / WPR, seg = w % WPR; // pair slot, segment
   RowSum<WPR> row_sum{s_part + pi * 2 * WPR, 1 + pi, seg, lane, 0};
-  int bi, bj;
-  rr_pair(L.nb, local, slot, bi, bj);
+  // `resident` (the persistent kernel): the first block stays in shared memory, with its tracked norms, for all
+  // steps of a level; it is loaded at the level's first step and stored at its last.
+  const StepPlan plan = step_plan(L.nb, local, slot);
+  const int bi = plan.bi, bj = plan.bj;
+  const bool load_first = !resident || plan.first_in_level, store_first = !resident || plan.last_in_level;
   float* X = L.X;
 #ifdef ATOMO_PHASE_TIMING
   long long tk[8]; int nk = 0;
@@ -197,20 +214,24 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 #define ATOMO_TICK()
 #endif
   ATOMO_TICK();
-  // ---- load 2B rows ----
-  for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+  // ---- load the rows (the first block only when it is not already here) ----
+  for (int idx = tid + (load_first ? 0 : B * R4); idx < 2 * B * R4; idx += NT) {
     const int row = idx / R4, q = idx % R4;
     const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
     reinterpret_cast<float4*>(smem + row * LD)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * LD)[q];
   }
   __syncthreads();
   RowRegs<T4> xp, xq;
-  // pair slot pi: squared norms of rows pi and pi + B; row pi stays in registers for the cross rounds
+  // pair slot pi: squared norms of rows pi and pi + B, computed from every row that was just loaded (a resident
+  // row keeps its tracked norm); row pi stays in registers for the cross rounds
   load_row<T4>(xq, smem + (B + pi) * LD + seg * SEG, lane, V4);
   const float nj = row_sum(row_norm2_partial<T4>(xq, lane, A4));
   load_row<T4>(xp, smem + pi * LD + seg * SEG, lane, V4);
-  float np2 = row_sum(row_norm2_partial<T4>(xp, lane, A4)), dp = 1.0f;
-  if (lane == 0 && seg == 0) { s_n2[pi] = np2; s_n2[B + pi] = nj; s_d[pi] = 1.0f; s_d[B + pi] = 1.0f; }
+  float np2 = load_first ? row_sum(row_norm2_partial<T4>(xp, lane, A4)) : s_n2[pi], dp = 1.0f;
+  if (lane == 0 && seg == 0) {
+    if (load_first) { s_n2[pi] = np2; s_d[pi] = 1.0f; }
+    s_n2[B + pi] = nj; s_d[B + pi] = 1.0f;
+  }
   __syncthreads();
   ATOMO_TICK();
   uint32_t nrot = 0;
@@ -259,10 +280,10 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
   }
   ATOMO_TICK();
   store_row<T4>(xp, smem + pi * LD + seg * SEG, lane, V4, dp);
-  if (lane == 0 && seg == 0) s_d[pi] = 1.0f;
+  if (lane == 0 && seg == 0) { s_d[pi] = 1.0f; s_n2[pi] = np2; }
   __syncthreads();
-  // ---- store, folding the collected cosines back into the rows ----
-  for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+  // ---- store, folding the collected cosines back into the rows (the first block only when it leaves) ----
+  for (int idx = tid + (store_first ? 0 : B * R4); idx < 2 * B * R4; idx += NT) {
     const int row = idx / R4, q = idx % R4;
     const int grow = (row < B) ? bi * B + row : bj * B + (row - B);
     const float d = s_d[row];
@@ -280,26 +301,27 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 
 constexpr int kJacobiThreads = 32 * kJB;
 
-__device__ __forceinline__ void jacobi_dispatch(const SpLayer& L, int slot, int sweep, int local, float tol, float* smem) {
+__device__ __forceinline__ void jacobi_dispatch(const SpLayer& L, int slot, int sweep, int local, bool resident, float tol,
+                                                float* smem) {
   if (L.acc) {
     switch (L.rp) {
-      case 32: jacobi_block_pair<32, true, 1>(L, slot, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, true, 1>(L, slot, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, true, 1>(L, slot, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, true, 1>(L, slot, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, true, 1>(L, slot, sweep, local, tol, smem); break;
+      case 32: jacobi_block_pair<32, true, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 64: jacobi_block_pair<64, true, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 128: jacobi_block_pair<128, true, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 256: jacobi_block_pair<256, true, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 512: jacobi_block_pair<512, true, 1>(L, slot, sweep, local, resident, tol, smem); break;
       default: break;
     }
   } else {
     switch (L.rp) {
-      case 32: jacobi_block_pair<32, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 64: jacobi_block_pair<64, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 128: jacobi_block_pair<128, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 256: jacobi_block_pair<256, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 512: jacobi_block_pair<512, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 1024: jacobi_block_pair<1024, false, 1>(L, slot, sweep, local, tol, smem); break;
-      case 2048: jacobi_block_pair<2048, false, 2>(L, slot, sweep, local, tol, smem); break;
-      case 4096: jacobi_block_pair<4096, false, 4>(L, slot, sweep, local, tol, smem); break;
+      case 32: jacobi_block_pair<32, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 64: jacobi_block_pair<64, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 128: jacobi_block_pair<128, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 256: jacobi_block_pair<256, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 512: jacobi_block_pair<512, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 1024: jacobi_block_pair<1024, false, 1>(L, slot, sweep, local, resident, tol, smem); break;
+      case 2048: jacobi_block_pair<2048, false, 2>(L, slot, sweep, local, resident, tol, smem); break;
+      case 4096: jacobi_block_pair<4096, false, 4>(L, slot, sweep, local, resident, tol, smem); break;
       default: break;
     }
   }
@@ -316,7 +338,7 @@ __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_step_kernel(const Sp
   const int sweep = t / steps, local = t % steps;
   if (sweep >= max_sweeps) return;
   if (sweep > 0 && L.rot_count[sweep - 1] == 0) return;   // the previous sweep rotated nothing: converged
-  jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
+  jacobi_dispatch(L, ref.a, sweep, local, false, tol, smem);
 }
 
 // The whole eigen-solve in one cooperative launch, for batches whose block pairs are all co-resident (one CTA
@@ -342,7 +364,7 @@ __global__ void __launch_bounds__(kJacobiThreads) sp_jacobi_persistent_kernel(co
   for (; t < t_max; ++t) {
     const int sweep = t / steps, local = t % steps;
     if (local == 0 && sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) == 0) break;
-    jacobi_dispatch(L, ref.a, sweep, local, tol, smem);
+    jacobi_dispatch(L, ref.a, sweep, local, true, tol, smem);
     __syncthreads();
     if (n_ctas > 1) {
       if (threadIdx.x == 0) {
