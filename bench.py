@@ -27,8 +27,9 @@ METRIC = "gradient elements encoded+decoded/sec"
 UNIT = "elements/s"
 L2_BYTES = 126 * 1024 * 1024
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # SMs x FP32 lanes x 2 flop x max SM clock
-# dram bytes per Jacobi-step launch from the ncu capture summarised in profiles/ (None until captured)
-JACOBI_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one sp_jacobi_persistent_kernel launch on this workload, from the
+# ncu capture summarised in profiles/sp_jacobi_persistent_c2.txt (5.70 MB read + 0.33 MB written)
+JACOBI_TRAFFIC_BYTES_PER_LAUNCH = 6032896
 
 
 def measured_peaks():
@@ -54,7 +55,7 @@ class ClockSampler:
     def start(self):
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "20", "-i", str(self.gpu)], stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
 
@@ -351,7 +352,7 @@ def run_ours(args):
                          "kernel": "sp_jacobi_persistent_kernel" if launches_per_step <= 2 else "sp_jacobi_step_kernel",
                          "achieved": achieved,
                          "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_FMA_PEAK_TFLOPS,
-                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH,
+                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH if launches_per_step <= 2 else None,
                          "launches_per_step": 1.0 if launches_per_step <= 2 else launches_per_step,
                          "avg_launch_us": eig_s_per_step / (1.0 if launches_per_step <= 2 else launches_per_step) * 1e6,
                          "share_of_step": eig_ms / ms_total,

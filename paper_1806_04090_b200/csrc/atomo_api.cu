@@ -469,6 +469,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
 
   std::vector<EwVec> V(n_vecs);
   size_t need = 0;
+  uint8_t* ew_zero_beg = nullptr; size_t ew_zero_bytes = 0;
   const int max_blocks = ew_solve_max_blocks();
   if (max_blocks <= 0) return fail_cuda(ctx, cudaGetLastError(), "occupancy query for the cooperative solve");
   for (int pass = 0; pass < 2; ++pass) {
@@ -478,6 +479,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       EwVec& v = V[l];
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
+      v.tiles_per_cta = ew_tiles_per_cta(v.n_tiles);
       v.n_words = (v.n + 31) / 32;
       const int64_t want_chunks = std::min<int64_t>(max_blocks, (v.n + 4095) / 4096);
       v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
@@ -492,9 +494,12 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       v.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
       v.prob_out = (dbg && dbg->prob) ? dbg->prob + dbg_atoms : nullptr;
       dbg_atoms += v.n; dbg_words += v.n_words;
-      v.tile_counts = A.take<uint32_t>(v.n_tiles);
-      v.tile_offsets = A.take<uint64_t>(v.n_tiles);
     }
+    // zero-filled per call: look-back status words and tile tickets of all vectors, one contiguous region
+    uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
+    const size_t z0 = A.off;
+    for (int l = 0; l < n_vecs; ++l) { V[l].tile_status = A.take<uint64_t>(V[l].n_tiles); V[l].ticket = A.take<uint32_t>(1); }
+    ew_zero_beg = zb; ew_zero_bytes = A.off - z0;
     need = A.off + 256;
     if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
   }
@@ -522,8 +527,9 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   }
   stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_vecs);
   stage_begin(ctx, ATOMO_STAGE_EW_PACK, st);
+  CK(cudaMemsetAsync(ew_zero_beg, 0, ew_zero_bytes, st));
   for (int l = 0; l < n_vecs; ++l) launch_ew_sample_pack(V[l], key, ks, st);
-  stage_end(ctx, ATOMO_STAGE_EW_PACK, st, 3 * (int64_t)n_vecs);
+  stage_end(ctx, ATOMO_STAGE_EW_PACK, st, (int64_t)n_vecs);
   CK(cudaGetLastError());
   return ATOMO_OK;
 }

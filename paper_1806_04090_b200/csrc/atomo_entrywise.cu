@@ -6,9 +6,10 @@
 //                                |g_i| (s - n_s) > sum_{unsaturated} |g_j| gets p = 1; repeated
 //                                until no new atom saturates (zero rounds when g is s-balanced,
 //                                Lemma 3); grid barriers instead of host round trips
-//   pass 2   ew_sample         : p_i = |g_i| (s-n_s)/T, Philox word, keep bit -> mask words + tile counts
-//            ew_scan           : exclusive scan of tile counts, k, capacity check, header
-//            ew_pack           : ordered compaction: idx ascending, val = g_i / p_i
+//   pass 2   ew_sample_pack    : per chunk of tiles: p_i = |g_i| (s-n_s)/T, Philox word, keep bit -> mask words
+//                                and counts; the counts of the earlier chunks are added (one bounded wait, no
+//                                chain); ordered compaction from the mask words: idx ascending, val = g_i / p_i;
+//                                the last chunk writes k, the capacity check and the header
 //   decode   ew_decode         : zero-fill with vector stores, then the tile's kept values (per-tile
 //                                offsets travel in the payload)
 #include <algorithm>
@@ -140,143 +141,172 @@ __global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s)
   }
 }
 
-// ---- sampling -----------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kEwThreads) ew_sample_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+// ---- sampling + ordered compaction, one kernel -----------------------------------------------------
+// A CTA takes the next chunk of `tiles_per_cta` consecutive tiles (a ticket, so that every chunk it will wait for
+// is already running).  Phase 1: the keep bit of every atom of the chunk (Eq. 2: p_i = 1 on the saturated set,
+// |g_i| (s - n_s) / T elsewhere; Philox word against floor(p 2^32)); mask words go to shared memory (and to the
+// mask output), kept atoms are counted per tile.  The chunk's count is published; the CTA then waits (bounded)
+// until every earlier chunk has published and adds their counts -- all chunks of a wave finish phase 1 together,
+// so nobody waits on a chain.  Phase 2: ordered compaction of the chunk from the mask words in shared memory;
+// only the kept atoms' values are read again (they are still in L2).  The last chunk writes k, the capacity
+// check and the layer header.  A wait that runs out raises ATOMO_ERR_TIMEOUT in the layer header.
+constexpr uint64_t kFlagReady = 1ull << 63;
+constexpr uint32_t kChunkSpinLimit = 1u << 20;
+constexpr int kEwMaxTilesPerCta = 64;
+constexpr int kEwWordsPerTile = kEwTile / 32;
+
+__global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+  constexpr int kIts = kEwTile / (kEwThreads * 4);
+  constexpr int kWarps = kEwThreads / kWarp;
+  extern __shared__ uint32_t s_mask[];            // [tiles_per_cta][128] mask words of the chunk
+  __shared__ uint32_t s_tcnt[kEwMaxTilesPerCta];  // kept atoms per tile, then their exclusive prefix
+  __shared__ uint32_t s_chunk;
+  __shared__ unsigned long long s_base;           // kept atoms before this chunk
+  __shared__ uint32_t s_wsum[kWarps];
+  __shared__ int s_fail;
   const EwState* st = v.state;
-  const float scale = st->scale;
-  const float theta = st->theta_f;
+  const float scale = st->scale, theta = st->theta_f, c = st->c;
+  const float scale32 = scale * 4294967296.0f;    // exact: a power-of-two factor
   const bool dead = st->nonfinite != 0;
   const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
-  const int64_t tile_base = (int64_t)blockIdx.x * kEwTile;
-  uint32_t kept = 0;
+  const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
+  const int tpc = v.tiles_per_cta;
+  if (tid == 0) { s_chunk = atomicAdd(v.ticket, 1u); s_base = 0ull; s_fail = 0; }
+  if (tid < kEwMaxTilesPerCta) s_tcnt[tid] = 0u;
+  __syncthreads();
+  const uint32_t chunk = s_chunk;
+  const int64_t tile0 = (int64_t)chunk * tpc;
+  const int n_my = (int)min((int64_t)tpc, v.n_tiles - tile0);
+
+  // ---- phase 1 ----
+  for (int tl = 0; tl < n_my; ++tl) {
+    const uint32_t tile = (uint32_t)(tile0 + tl);
+    const int64_t tile_base = (int64_t)tile * kEwTile;
+    const bool full = aligned && tile_base + kEwTile <= v.n;
+    float4 x[kIts];
 #pragma unroll
-  for (int it = 0; it < kEwTile / (kEwThreads * 4); ++it) {
-    const int64_t i = tile_base + ((int64_t)it * kEwThreads + threadIdx.x) * 4;
-    uint32_t nib = 0;
-    float4 pv = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i < v.n && !dead) {
-      const float4 x = load4(v.g, i, v.n, aligned);
-      const uint4 wd = atom_block_words((uint64_t)(i >> 2), v.layer, kind_step, key);
-      const float a[4] = {fabsf(x.x), fabsf(x.y), fabsf(x.z), fabsf(x.w)};
+    for (int it = 0; it < kIts; ++it) {
+      const int64_t i = tile_base + ((int64_t)it * kEwThreads + tid) * 4;
+      x[it] = full ? __ldg(reinterpret_cast<const float4*>(v.g + i))
+                   : (i < v.n ? load4(v.g, i, v.n, aligned) : make_float4(0.f, 0.f, 0.f, 0.f));
+    }
+    uint32_t kept = 0;
+#pragma unroll
+    for (int it = 0; it < kIts; ++it) {
+      const int64_t i = tile_base + ((int64_t)it * kEwThreads + tid) * 4;
+      // block of 4 atoms = i >> 2 < 2^30 (n < 2^32): the high counter word is zero
+      const uint4 wd = philox4x32_10(make_uint4(tile * (uint32_t)(kEwTile / 4) + (uint32_t)(it * kEwThreads + tid), 0u, v.layer, kind_step), key);
+      const float a[4] = {fabsf(x[it].x), fabsf(x[it].y), fabsf(x[it].z), fabsf(x[it].w)};
       const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
-      float p[4];
+      uint32_t nb = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        p[j] = (a[j] > theta) ? 1.0f : fminf(a[j] * scale, 1.0f);
-        if (i + j < v.n && bernoulli_keep(p[j], ww[j])) nib |= 1u << j;
+        // p = 1 if saturated, else min(a scale, 1); keep iff p >= 1 or word < floor(p 2^32).  a scale32 is the
+        // same product times 2^32 (exact), and the truncating conversion gives the floor.
+        const float t = a[j] * scale32;
+        const bool one = a[j] > theta || t >= 4294967296.0f;
+        const bool keep = one || ww[j] < __float2uint_rz(t);
+        if (keep && (full || i + j < v.n)) nb |= 1u << j;
       }
-      pv = make_float4(p[0], p[1], p[2], p[3]);
-    }
-    if (v.prob_out != nullptr && i < v.n) {
-      if (i + 3 < v.n && (reinterpret_cast<uintptr_t>(v.prob_out) & 15u) == 0)
-        *reinterpret_cast<float4*>(v.prob_out + i) = pv;
-      else {
-        const float pp[4] = {pv.x, pv.y, pv.z, pv.w};
-        for (int j = 0; j < 4 && i + j < v.n; ++j) v.prob_out[i + j] = pp[j];
+      if (dead) nb = 0;
+      kept += __popc(nb);
+      if (v.prob_out != nullptr && i < v.n) {
+        float pp[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pp[j] = dead ? 0.0f : ((a[j] > theta) ? 1.0f : fminf(a[j] * scale, 1.0f));
+        if (i + 3 < v.n && (reinterpret_cast<uintptr_t>(v.prob_out) & 15u) == 0)
+          *reinterpret_cast<float4*>(v.prob_out + i) = make_float4(pp[0], pp[1], pp[2], pp[3]);
+        else
+          for (int j = 0; j < 4 && i + j < v.n; ++j) v.prob_out[i + j] = pp[j];
+      }
+      // 8 consecutive lanes hold the 32 bits of one mask word
+      uint32_t word = nb << (4 * (tid & 7));
+      word |= __shfl_xor_sync(0xffffffffu, word, 1);
+      word |= __shfl_xor_sync(0xffffffffu, word, 2);
+      word |= __shfl_xor_sync(0xffffffffu, word, 4);
+      if ((tid & 7) == 0) {
+        const int wl = it * (kEwThreads / 8) + (tid >> 3);
+        s_mask[tl * kEwWordsPerTile + wl] = word;
+        const int64_t widx = (tile_base >> 5) + wl;
+        if (widx < v.n_words) v.mask_words[widx] = word;
       }
     }
-    kept += __popc(nib);
-    // 8 consecutive lanes hold the 32 bits of one mask word
-    uint32_t word = nib << (4 * (threadIdx.x & 7));
-    word |= __shfl_xor_sync(0xffffffffu, word, 1);
-    word |= __shfl_xor_sync(0xffffffffu, word, 2);
-    word |= __shfl_xor_sync(0xffffffffu, word, 4);
-    if ((threadIdx.x & 7) == 0) {
-      const int64_t widx = (tile_base >> 5) + it * (kEwThreads / 8) + (threadIdx.x >> 3);
-      if (widx < v.n_words) v.mask_words[widx] = word;
-    }
+    kept = warp_sum(kept);
+    if (lane == 0 && kept) atomicAdd(&s_tcnt[tl], kept);
   }
-  __shared__ uint32_t s_cnt[kEwThreads / kWarp];
-  kept = warp_sum(kept);
-  if (threadIdx.x % kWarp == 0) s_cnt[threadIdx.x / kWarp] = kept;
   __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t t = 0;
-    for (int i = 0; i < kEwThreads / kWarp; ++i) t += s_cnt[i];
-    v.tile_counts[blockIdx.x] = t;
-  }
-}
 
-// exclusive scan of tile_counts (in place), k, capacity check, layer header
-__global__ void __launch_bounds__(1024) ew_scan_kernel(EwVec v) {
-  __shared__ uint32_t s_warp[32];
-  __shared__ uint64_t s_carry;
-  if (threadIdx.x == 0) s_carry = 0;
+  // ---- chunk count out, counts of the earlier chunks in ----
+  if (w == 0) {
+    uint32_t total = 0;
+    for (int t = lane; t < n_my; t += kWarp) total += s_tcnt[t];
+    total = warp_sum(total);
+    if (lane == 0) {
+      *(volatile unsigned long long*)(v.tile_status + chunk) = kFlagReady | (unsigned long long)total;
+      uint32_t run = 0;                                   // exclusive prefix over the chunk's tiles
+      for (int t = 0; t < n_my; ++t) { const uint32_t cnt = s_tcnt[t]; s_tcnt[t] = run; run += cnt; }
+      s_chunk = total;                                    // reuse: the chunk's count
+    }
+  }
+  unsigned long long before = 0;
+  int fail = 0;
+  for (uint32_t cidx = tid; cidx < chunk; cidx += kEwThreads) {
+    unsigned long long sv;
+    uint32_t spins = 0;
+    do { sv = *(volatile const unsigned long long*)(v.tile_status + cidx); } while (!(sv & kFlagReady) && ++spins <= kChunkSpinLimit);
+    if (!(sv & kFlagReady)) fail = 1;
+    before += sv & ~kFlagReady;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+  if (lane == 0 && before) atomicAdd(&s_base, before);
+  if (fail) s_fail = 1;
   __syncthreads();
-  const int lane = threadIdx.x % kWarp, w = threadIdx.x / kWarp;
-  for (int64_t base = 0; base < v.n_tiles; base += 1024) {
-    const int64_t i = base + threadIdx.x;
-    const uint32_t c = i < v.n_tiles ? v.tile_counts[i] : 0u;
-    uint32_t inc = c;
+  const uint64_t base = s_base;
+  const uint32_t total = s_chunk;
+  if (tid == 0) {
+    if (s_fail) raise_status(v.hdr, ATOMO_ERR_TIMEOUT);
+    for (int t = 0; t < n_my; ++t) v.tile_table[tile0 + t] = (uint32_t)min(base + s_tcnt[t], (uint64_t)0xFFFFFFFFull);
+    if (tile0 + n_my == v.n_tiles) {                      // the last chunk knows k: capacity check, layer header
+      const uint64_t k = base + total;
+      atomo_layer_header* h = v.hdr;
+      h->n_sat = st->n_sat; h->c = st->c; h->l1 = st->T0; h->sweeps = st->rounds;
+      if (st->nonfinite) raise_status(h, ATOMO_ERR_NONFINITE);
+      else if (k > (uint64_t)v.k_cap) raise_status(h, ATOMO_ERR_CAPACITY);
+      const bool ok = *(volatile uint32_t*)&h->status == ATOMO_OK;
+      h->k = ok ? (uint32_t)k : 0u;
+      v.tile_table[v.n_tiles] = ok ? (uint32_t)k : 0u;
+    }
+  }
+  if (total == 0) return;
+
+  // ---- phase 2: ordered compaction, indices ascending, value = g_i / p_i ----
+  for (int tl = 0; tl < n_my; ++tl) {
+    const int64_t tile_base = (tile0 + tl) * (int64_t)kEwTile;
+    const uint32_t word = tid < kEwWordsPerTile ? s_mask[tl * kEwWordsPerTile + tid] : 0u;
+    const uint32_t pc = __popc(word);
+    uint32_t inc = pc;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
-    if (lane == 31) s_warp[w] = inc;
+    __syncthreads();                                      // s_wsum of the previous tile has been read
+    if (lane == 31) s_wsum[w] = inc;
     __syncthreads();
-    if (w == 0) {
-      uint32_t x = s_warp[lane], y = x;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, y, o); if (lane >= o) y += t; }
-      s_warp[lane] = y - x;                          // exclusive over warps
+    uint32_t woff = inc - pc;
+    for (int i = 0; i < w; ++i) woff += s_wsum[i];
+    uint64_t pos = base + s_tcnt[tl] + woff;
+    uint32_t m = word;
+    while (m) {
+      const int bpos = __ffs(m) - 1;
+      m &= m - 1;
+      const int64_t i = tile_base + tid * 32 + bpos;
+      if (pos < (uint64_t)v.k_cap) {
+        const float g = __ldg(v.g + i);
+        // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) T / (s - n_s)
+        v.idx[pos] = (uint32_t)i;
+        v.val[pos] = (fabsf(g) > theta) ? g : copysignf(c, g);
+      }
+      ++pos;
     }
-    __syncthreads();
-    const uint64_t carry = s_carry;
-    const uint64_t excl = carry + s_warp[w] + inc - c;
-    if (i < v.n_tiles) { v.tile_offsets[i] = excl; v.tile_table[i] = (uint32_t)min(excl, (uint64_t)0xFFFFFFFFull); }
-    __syncthreads();
-    if (threadIdx.x == 1023) s_carry = excl + c;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) {
-    const uint64_t k = s_carry;
-    const EwState* st = v.state;
-    atomo_layer_header* h = v.hdr;
-    h->n_sat = st->n_sat; h->c = st->c; h->l1 = st->T0; h->sweeps = st->rounds;
-    uint32_t status = ATOMO_OK;
-    if (st->nonfinite) status = ATOMO_ERR_NONFINITE;
-    else if (k > (uint64_t)v.k_cap) status = ATOMO_ERR_CAPACITY;
-    h->status = status;
-    h->k = status == ATOMO_OK ? (uint32_t)k : 0u;
-    v.tile_table[v.n_tiles] = status == ATOMO_OK ? (uint32_t)k : 0u;
-  }
-}
-
-// ordered compaction of one tile: indices ascending, value = g_i / p_i
-__global__ void __launch_bounds__(kEwThreads) ew_pack_kernel(EwVec v) {
-  if (v.hdr->status != ATOMO_OK) return;
-  __shared__ uint32_t s_idx[kEwTile];
-  __shared__ uint32_t s_woff[kEwTile / 32 + 1];
-  __shared__ uint32_t s_wsum[kEwThreads / kWarp];
-  const int64_t tile_base = (int64_t)blockIdx.x * kEwTile;
-  const int64_t wbase = tile_base >> 5;
-  const int t = threadIdx.x, lane = t % kWarp, w = t / kWarp;
-  uint32_t word = 0;
-  if (t < kEwTile / 32 && wbase + t < v.n_words) word = v.mask_words[wbase + t];
-  const uint32_t pc = __popc(word);
-  uint32_t inc = pc;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) { const uint32_t x = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += x; }
-  if (lane == 31) s_wsum[w] = inc;
-  __syncthreads();
-  uint32_t woff = inc - pc;
-  for (int i = 0; i < w; ++i) woff += s_wsum[i];
-  if (t < kEwTile / 32) {
-    uint32_t m = word, o = woff;
-    while (m) { const int b = __ffs(m) - 1; m &= m - 1; s_idx[o++] = (uint32_t)(t * 32 + b); }
-  }
-  if (t == kEwTile / 32 - 1) s_woff[0] = woff + pc;     // tile count
-  __syncthreads();
-  const uint32_t cnt = s_woff[0];
-  const uint64_t out0 = v.tile_offsets[blockIdx.x];
-  const EwState* st = v.state;
-  const float theta = st->theta_f;
-  const float c = st->c;
-  for (uint32_t j = t; j < cnt; j += kEwThreads) {
-    const int64_t i = tile_base + s_idx[j];
-    const float g = __ldg(v.g + i);
-    // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) * T / (s - n_s)
-    const float val = (fabsf(g) > theta) ? g : copysignf(c, g);
-    v.idx[out0 + j] = (uint32_t)i;
-    v.val[out0 + j] = val;
   }
 }
 
@@ -334,10 +364,19 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st) {
   void* args[] = {&vv, &ss};
   return (int)cudaLaunchCooperativeKernel((const void*)ew_solve_kernel, dim3(v.n_chunks), dim3(kEwThreads), args, 0, st);
 }
+int ew_tiles_per_cta(int64_t n_tiles) {
+  // one wave of chunks when it fits (at most 64 tiles per chunk)
+  int dev = 0, sms = 148, per_sm = 4;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel, kEwThreads,
+                                                    16 * kEwWordsPerTile * sizeof(uint32_t)) != cudaSuccess || per_sm < 1)
+    per_sm = 4;
+  const int64_t wave = (int64_t)sms * per_sm;
+  return (int)std::min<int64_t>(kEwMaxTilesPerCta, std::max<int64_t>(1, (n_tiles + wave - 1) / wave));
+}
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
-  ew_sample_kernel<<<(unsigned)v.n_tiles, kEwThreads, 0, st>>>(v, key, kind_step);
-  ew_scan_kernel<<<1, 1024, 0, st>>>(v);
-  ew_pack_kernel<<<(unsigned)v.n_tiles, kEwThreads, 0, st>>>(v);
+  const unsigned grid = (unsigned)((v.n_tiles + v.tiles_per_cta - 1) / v.tiles_per_cta);
+  ew_sample_pack_kernel<<<grid, kEwThreads, (size_t)v.tiles_per_cta * kEwWordsPerTile * sizeof(uint32_t), st>>>(v, key, kind_step);
 }
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {
   const int64_t tiles = (d.n + kEwTile - 1) / kEwTile;

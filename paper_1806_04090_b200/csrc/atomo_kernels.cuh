@@ -28,7 +28,10 @@ struct EwVec {
   int64_t n_tiles; int64_t n_words;
   atomo_layer_header* hdr; uint32_t* idx; float* val;          // payload
   EwPartial* partials; EwState* state;                         // workspace
-  uint32_t* mask_words; uint32_t* tile_counts; uint64_t* tile_offsets;
+  uint32_t* mask_words;
+  int tiles_per_cta;                                           // tiles per chunk of the sample / pack kernel
+  uint64_t* tile_status;                                       // [chunks] ready flag (bit 63) | kept atoms of the chunk; zeroed per call
+  uint32_t* ticket;                                            // next tile to hand out; zeroed per call
   uint32_t* tile_table;                                        // payload: kept atoms before each tile
   float* prob_out;                                             // debug or nullptr
 };
@@ -43,6 +46,7 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st); // returns a cud
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st);
 void launch_ew_decode(const EwDecode& d, cudaStream_t st);
 int ew_tile_elems();
+int ew_tiles_per_cta(int64_t n_tiles);
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
