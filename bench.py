@@ -230,9 +230,19 @@ def run_ours(args):
     payload = torch.empty(api.payload_bytes_spectral(shapes, k_cap), dtype=torch.uint8, device=dev)
     outs = [torch.empty(sh, dtype=torch.float32, device=dev) for sh in shapes]
 
+    exchange = bool(args.exchange) and world > 1
+
+    def combine(pay):
+        """decode; with --exchange on N > 1 GPUs: all-gather the payloads over NCCL, then the averaging decode"""
+        if not exchange:
+            a.atomo_decode(pay, out=outs)
+            return
+        bufs = dist.all_gather_bytes(pay.buf)
+        a.atomo_decode_average([api.Payload(b, pay.kind, pay.shapes, pay.k_cap, a) for b in bufs], out=outs)
+
     def step(i, layers):
-        pay, _ = a.atomo_encode_spectral(layers, s, seed, step=i, k_cap=k_cap, payload=payload)
-        a.atomo_decode(pay, out=outs)
+        pay, _ = a.atomo_encode_spectral(layers, s, seed + rank, step=i, k_cap=k_cap, payload=payload)
+        combine(pay)
         return pay
 
     # ---- warm-up ----
@@ -252,12 +262,12 @@ def run_ours(args):
     sweeps_seen = None
     ev0.record()
     for k in range(args.steps):
-        pay, _ = a.atomo_encode_spectral(dev_sets[(args.warmup + k) % n_sets], s, seed, step=args.warmup + k,
+        pay, _ = a.atomo_encode_spectral(dev_sets[(args.warmup + k) % n_sets], s, seed + rank, step=args.warmup + k,
                                          k_cap=k_cap, payload=payload)
         ms, ln = a.stage_times()                   # encode has finished its host-side waits here
         eig_ms += ms["eig"]; eig_launches += ln["eig"]
         launches += sum(ln.values()) + 7           # + header/descriptor copies and the workspace memset
-        a.atomo_decode(pay, out=outs)
+        combine(pay)
         launches += 3
         if k == args.steps - 1:
             sweeps_seen = [h.sweeps for h in pay.headers()[1]]
@@ -341,6 +351,8 @@ def run_ours(args):
                                    "s=2, one batched encode + decode per step",
                        "k_cap": k_cap, "l2": f"inputs rotate over {n_sets} distinct sets ({n_sets * in_bytes / 2**20:.0f} MiB "
                                              f"> 126 MiB L2) so each step reads gradients from HBM",
+                       "parallelism": ("data-parallel: payload all-gather + averaging decode" if exchange else
+                                       "independent replicas, no collective") if world > 1 else "single GPU",
                        "jacobi_sweeps_last_step": sweeps_seen,
                        "eig_ms_per_step": eig_ms / args.steps},
             "clocks": clocks,
@@ -376,6 +388,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--exchange", action="store_true",
+                    help="N > 1: all-gather the payloads and decode their average on every rank (the data-parallel "
+                         "combine step) instead of independent replicas")
     ap.add_argument("--no-extras", action="store_true", help="skip the entry-wise (config 4) figures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

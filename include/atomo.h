@@ -151,6 +151,18 @@ int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload /*DEVICE*/,
                  const int64_t* rows, const int64_t* cols, float* const* out /*HOST array of DEVICE ptrs*/,
                  int32_t n_layers, void* stream);
 
+/* --- decode and average (the combine step of data-parallel training, Section 2) ---------------
+ * out[l] = (1 / n_payloads) * sum over p of the decoded layer l of payloads[p]: what the receiver of the
+ * workers' sparsified gradients computes before the model update.  All payloads must be of `kind` and of the
+ * shapes given (they normally come from the same encode call on different workers, with different seeds);
+ * a payload that does not match contributes zeros and gets ATOMO_ERR_PAYLOAD in its layer's status word.
+ * payloads: HOST array of DEVICE pointers (e.g. the slices of an all-gather buffer).  The sum runs over the
+ * payloads in array order and over each payload's atoms in payload order, so the result is reproducible.
+ * One pass over the output; never synchronises; every element of every output is written.             */
+int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloads /*HOST array of DEVICE ptrs*/,
+                         int32_t n_payloads, const int64_t* rows, const int64_t* cols,
+                         float* const* out /*HOST array of DEVICE ptrs*/, int32_t n_layers, void* stream);
+
 /* --- decode without allocation ---------------------------------------------------------------
  * (The paper has no counterpart: this entry point exists for deployment, not for the method.)
  * Same result as atomo_decode() for a spectral payload, for callers that must not allocate device

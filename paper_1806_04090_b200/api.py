@@ -28,7 +28,7 @@ EXPORTS = [
     "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
-    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_decode_spectral_static",
+    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_decode_spectral_static", "atomo_decode_average",
 ]
 
 
@@ -93,6 +93,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_encode_entrywise.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, u64, u64, i64, vp, i64,
                                            ctypes.POINTER(_Debug), vp]
     lib.atomo_decode.argtypes = [vp, i32, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(vp), i32, vp]
+    lib.atomo_decode_average.argtypes = [vp, i32, ctypes.POINTER(vp), i32, ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                         ctypes.POINTER(vp), i32, vp]
     lib.atomo_payload_read_headers.argtypes = [vp, vp, i32, ctypes.POINTER(PayloadHeader),
                                                ctypes.POINTER(LayerHeader), vp]
     lib.atomo_payload_status.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
@@ -361,6 +363,30 @@ class Atomo:
         return list(out)
 
     # ------------------------------------------------------------------------------------------
+    def atomo_decode_average(self, payloads: Sequence[Payload], out: Optional[Sequence[torch.Tensor]] = None,
+                             stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
+        """Mean of the dense gradients of several payloads of the same shapes (the workers' payloads after an
+        all-gather), one tensor per layer, in one pass over the output."""
+        if len(payloads) == 0:
+            raise ValueError("atomo_decode_average needs at least one payload")
+        first = payloads[0]
+        for p in payloads[1:]:
+            if p.kind != first.kind or list(p.shapes) != list(first.shapes):
+                raise ValueError("payloads of one average must share kind and shapes")
+        n = first.n_layers
+        dev = first.buf.device
+        if out is None:
+            out = [torch.empty(r * c, dtype=torch.float32, device=dev).view((c,) if first.kind == KIND_ENTRYWISE else (r, c))
+                   for r, c in first.shapes]
+        rows = (ctypes.c_int64 * n)(*[r for r, _ in first.shapes])
+        cols = (ctypes.c_int64 * n)(*[c for _, c in first.shapes])
+        ptrs = (ctypes.c_void_p * n)(*[o.data_ptr() for o in out])
+        pays = (ctypes.c_void_p * len(payloads))(*[p.buf.data_ptr() for p in payloads])
+        rc = self.lib.atomo_decode_average(self._h, first.kind, pays, len(payloads), rows, cols, ptrs, n,
+                                           self._stream_ptr(stream))
+        self._check(rc, "atomo_decode_average")
+        return list(out)
+
     def read_headers(self, payload: Payload, stream: Optional[torch.cuda.Stream] = None):
         gh = PayloadHeader()
         lh = (LayerHeader * payload.n_layers)()

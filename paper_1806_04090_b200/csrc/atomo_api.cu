@@ -479,7 +479,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       EwVec& v = V[l];
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
-      v.tiles_per_cta = ew_tiles_per_cta(v.n_tiles);
+      v.n_ctas = ew_sample_pack_ctas(v.n_tiles);
       v.n_words = (v.n + 31) / 32;
       const int64_t want_chunks = std::min<int64_t>(max_blocks, (v.n + 4095) / 4096);
       v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
@@ -498,7 +498,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     // zero-filled per call: look-back status words and tile tickets of all vectors, one contiguous region
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
     const size_t z0 = A.off;
-    for (int l = 0; l < n_vecs; ++l) { V[l].tile_status = A.take<uint64_t>(V[l].n_tiles); V[l].ticket = A.take<uint32_t>(1); }
+    for (int l = 0; l < n_vecs; ++l) { V[l].tile_status = A.take<uint64_t>(V[l].n_ctas); V[l].ticket = A.take<uint32_t>(1); }
     ew_zero_beg = zb; ew_zero_bytes = A.off - z0;
     need = A.off + 256;
     if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
@@ -574,6 +574,53 @@ int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload, const int64_
     CK(cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
     launch_sp_decode(pay, d_layers, d_tiles, (int)tiles.size(), st);
     stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
+  }
+  CK(cudaGetLastError());
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
+int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloads, int32_t n_payloads,
+                         const int64_t* rows, const int64_t* cols, float* const* out, int32_t n_layers, void* stream) {
+  if (!ctx || !payloads || n_payloads <= 0 || !rows || !cols || !out || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;
+  if (kind != ATOMO_KIND_SPECTRAL && kind != ATOMO_KIND_ENTRYWISE) return ATOMO_ERR_INVALID_ARG;
+  for (int p = 0; p < n_payloads; ++p) if (!payloads[p]) return ATOMO_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (!out[l] || rows[l] <= 0 || cols[l] <= 0) return ATOMO_ERR_INVALID_ARG;
+    if (kind == ATOMO_KIND_ENTRYWISE && rows[l] != 1) return ATOMO_ERR_INVALID_ARG;
+  }
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  stage_reset(ctx);
+  std::vector<SpDecodeLayer> D;
+  std::vector<TileRef> tiles;
+  if (kind == ATOMO_KIND_SPECTRAL) {
+    D.resize(n_layers);
+    const int tr = sp_decode_tile_rows(), tc = sp_decode_tile_cols();
+    for (int l = 0; l < n_layers; ++l) {
+      D[l] = SpDecodeLayer{nullptr, out[l], rows[l], cols[l]};
+      const int na = (int)((rows[l] + tr - 1) / tr), nbt = (int)((cols[l] + tc - 1) / tc);
+      for (int a = 0; a < na; ++a) for (int b = 0; b < nbt; ++b) tiles.push_back({l, a, b, 0});
+    }
+  }
+  const uint8_t** d_pay = nullptr; SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
+  for (int pass = 0; pass < 2; ++pass) {
+    Arena A(pass ? ctx->ws : nullptr);
+    d_pay = A.take<const uint8_t*>(n_payloads);
+    d_layers = A.take<SpDecodeLayer>(D.size());
+    d_tiles = A.take<TileRef>(tiles.size());
+    if (pass == 0) { const int rc = ensure_ws(ctx, A.off + 256); if (rc != ATOMO_OK) return rc; }
+  }
+  stage_begin(ctx, ATOMO_STAGE_DECODE, st);
+  CK(cudaMemcpyAsync(d_pay, payloads, (size_t)n_payloads * sizeof(void*), cudaMemcpyHostToDevice, st));
+  if (kind == ATOMO_KIND_SPECTRAL) {
+    CK(cudaMemcpyAsync(d_layers, D.data(), D.size() * sizeof(SpDecodeLayer), cudaMemcpyHostToDevice, st));
+    CK(cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+    launch_sp_decode_average(d_pay, n_payloads, d_layers, d_tiles, (int)tiles.size(), st);
+    stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
+  } else {
+    for (int l = 0; l < n_layers; ++l) launch_ew_decode_average(d_pay, n_payloads, l, out[l], cols[l], st);
+    stage_end(ctx, ATOMO_STAGE_DECODE, st, n_layers);
   }
   CK(cudaGetLastError());
   return ATOMO_OK;

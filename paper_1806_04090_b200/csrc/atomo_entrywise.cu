@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s)
 }
 
 // ---- sampling + ordered compaction, one kernel -----------------------------------------------------
-// A CTA takes the next chunk of `tiles_per_cta` consecutive tiles (a ticket, so that every chunk it will wait for
+// A CTA takes the next chunk of consecutive tiles (the tiles are spread evenly over the chunks) (a ticket, so that every chunk it will wait for
 // is already running).  Phase 1: the keep bit of every atom of the chunk (Eq. 2: p_i = 1 on the saturated set,
 // |g_i| (s - n_s) / T elsewhere; Philox word against floor(p 2^32)); mask words go to shared memory (and to the
 // mask output), kept atoms are counted per tile.  The chunk's count is published; the CTA then waits (bounded)
@@ -170,13 +170,13 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
   const bool dead = st->nonfinite != 0;
   const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
   const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
-  const int tpc = v.tiles_per_cta;
+  const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;   // the first `rem` chunks have q + 1 tiles
   if (tid == 0) { s_chunk = atomicAdd(v.ticket, 1u); s_base = 0ull; s_fail = 0; }
   if (tid < kEwMaxTilesPerCta) s_tcnt[tid] = 0u;
   __syncthreads();
   const uint32_t chunk = s_chunk;
-  const int64_t tile0 = (int64_t)chunk * tpc;
-  const int n_my = (int)min((int64_t)tpc, v.n_tiles - tile0);
+  const int64_t tile0 = (int64_t)chunk * q + min((int64_t)chunk, rem);
+  const int n_my = (int)(q + ((int64_t)chunk < rem ? 1 : 0));
 
   // ---- phase 1 ----
   for (int tl = 0; tl < n_my; ++tl) {
@@ -364,19 +364,20 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st) {
   void* args[] = {&vv, &ss};
   return (int)cudaLaunchCooperativeKernel((const void*)ew_solve_kernel, dim3(v.n_chunks), dim3(kEwThreads), args, 0, st);
 }
-int ew_tiles_per_cta(int64_t n_tiles) {
-  // one wave of chunks when it fits (at most 64 tiles per chunk)
+int ew_sample_pack_ctas(int64_t n_tiles) {
+  // one wave of chunks when it fits (at most 64 tiles per chunk): tiles spread evenly, sizes differ by at most one
   int dev = 0, sms = 148, per_sm = 4;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel, kEwThreads,
                                                     16 * kEwWordsPerTile * sizeof(uint32_t)) != cudaSuccess || per_sm < 1)
     per_sm = 4;
   const int64_t wave = (int64_t)sms * per_sm;
-  return (int)std::min<int64_t>(kEwMaxTilesPerCta, std::max<int64_t>(1, (n_tiles + wave - 1) / wave));
+  const int64_t min_ctas = (n_tiles + kEwMaxTilesPerCta - 1) / kEwMaxTilesPerCta;
+  return (int)std::max<int64_t>(1, std::max(min_ctas, std::min(n_tiles, wave)));
 }
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
-  const unsigned grid = (unsigned)((v.n_tiles + v.tiles_per_cta - 1) / v.tiles_per_cta);
-  ew_sample_pack_kernel<<<grid, kEwThreads, (size_t)v.tiles_per_cta * kEwWordsPerTile * sizeof(uint32_t), st>>>(v, key, kind_step);
+  const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
+  ew_sample_pack_kernel<<<(unsigned)v.n_ctas, kEwThreads, (size_t)most * kEwWordsPerTile * sizeof(uint32_t), st>>>(v, key, kind_step);
 }
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {
   const int64_t tiles = (d.n + kEwTile - 1) / kEwTile;

@@ -29,7 +29,7 @@ struct EwVec {
   atomo_layer_header* hdr; uint32_t* idx; float* val;          // payload
   EwPartial* partials; EwState* state;                         // workspace
   uint32_t* mask_words;
-  int tiles_per_cta;                                           // tiles per chunk of the sample / pack kernel
+  int n_ctas;                                                  // chunks (CTAs) of the sample / pack kernel
   uint64_t* tile_status;                                       // [chunks] ready flag (bit 63) | kept atoms of the chunk; zeroed per call
   uint32_t* ticket;                                            // next tile to hand out; zeroed per call
   uint32_t* tile_table;                                        // payload: kept atoms before each tile
@@ -46,7 +46,7 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st); // returns a cud
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st);
 void launch_ew_decode(const EwDecode& d, cudaStream_t st);
 int ew_tile_elems();
-int ew_tiles_per_cta(int64_t n_tiles);
+int ew_sample_pack_ctas(int64_t n_tiles);
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
@@ -86,6 +86,12 @@ struct SpDecodeLayer {
 };
 
 struct TileRef { int32_t layer, a, b, c; };
+
+// averaging decode of several payloads (combine step of data-parallel training)
+void launch_sp_decode_average(const uint8_t* const* d_payloads, int n_payloads, const SpDecodeLayer* d_layers,
+                              const TileRef* d_tiles, int n_tiles, cudaStream_t st);
+void launch_ew_decode_average(const uint8_t* const* d_payloads, int n_payloads, int layer, float* out, int64_t n,
+                              cudaStream_t st);
 
 void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);

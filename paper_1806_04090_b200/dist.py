@@ -1,7 +1,8 @@
 """Process-group plumbing for multi-GPU runs (one process per GPU, launched by torchrun).
 
-The encode/decode path has no data-path collective: layers (or whole gradients) are independent
-units, so ranks work on their own units and only timing and unit counts are reduced.
+Encode and decode have no collective inside them: layers (or whole gradients) are independent units.  The one
+exchange step of data-parallel training is between them: an all-gather of the fixed-capacity payload buffers
+(`all_gather_bytes`), after which every rank averages all payloads with `atomo_decode_average`.
 """
 from __future__ import annotations
 
@@ -58,6 +59,20 @@ def shard_units(costs: Sequence[float], world: int) -> List[List[int]]:
         parts[r].append(i)
         loads[r] += costs[i]
     return [sorted(p) for p in parts]
+
+
+def all_gather_bytes(buf: torch.Tensor) -> List[torch.Tensor]:
+    """The exchange step of data-parallel training: every rank contributes its payload buffer (uint8, the same
+    fixed capacity on every rank) and receives all of them, as views of one gathered buffer in rank order.
+    Without a process group the list holds the caller's own buffer."""
+    if buf.dtype != torch.uint8 or buf.dim() != 1:
+        raise ValueError("payload buffers are flat uint8 tensors")
+    if not dist.is_initialized():
+        return [buf]
+    world = dist.get_world_size()
+    gathered = torch.empty(world * buf.numel(), dtype=torch.uint8, device=buf.device)
+    dist.all_gather_into_tensor(gathered, buf.contiguous())
+    return list(gathered.view(world, buf.numel()).unbind(0))
 
 
 def finish() -> None:

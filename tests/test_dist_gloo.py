@@ -19,9 +19,15 @@ def _worker(rank, world, port, q):
     t_max = d.max_over_ranks(10.0 + 5.0 * rank)        # slowest rank decides the step time
     units = d.sum_over_ranks(100.0 * (rank + 1))       # whole-job units
     parts = d.shard_units([9.0, 1.0, 8.0, 2.0, 7.0], w)
+    # exchange step: every rank's fixed-capacity payload buffer reaches every rank, in rank order
+    import torch
+    mine = (torch.arange(1000, dtype=torch.int64) * (rank + 3) % 251).to(torch.uint8)
+    got = d.all_gather_bytes(mine)
+    gathered_ok = len(got) == world and all(
+        torch.equal(got[k], (torch.arange(1000, dtype=torch.int64) * (k + 3) % 251).to(torch.uint8)) for k in range(world))
     d.barrier()
     d.finish()
-    q.put((r, w, t_max, units, parts))
+    q.put((r, w, t_max, units, parts, gathered_ok))
 
 
 def test_two_rank_reduction_and_sharding():
@@ -39,6 +45,7 @@ def test_two_rank_reduction_and_sharding():
     for r in res:
         assert r[1] == 2 and r[2] == 15.0 and r[3] == 300.0
         assert r[4] == [[0, 3, 4], [1, 2]] or sorted(sum(r[4], [])) == [0, 1, 2, 3, 4]
+        assert r[5]
     assert res[0][4] == res[1][4]                      # same partition on every rank
 
 
@@ -49,3 +56,6 @@ def test_single_process_defaults():
     assert d.env_world() == (0, 0, 1)
     assert d.max_over_ranks(3.5) == 3.5 and d.sum_over_ranks(2.0) == 2.0
     assert d.shard_units([1, 2, 3], 1) == [[0, 1, 2]]
+    import torch
+    buf = torch.arange(16, dtype=torch.uint8)
+    assert len(d.all_gather_bytes(buf)) == 1 and d.all_gather_bytes(buf)[0] is buf
