@@ -19,7 +19,7 @@ from __future__ import annotations
 
 import zlib
 from dataclasses import dataclass
-from typing import List, Sequence, Tuple
+from typing import List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -143,6 +143,27 @@ def c3_vgg11(seed: int = 0, layers: Sequence[LayerSpec] = VGG11_LAYERS) -> List[
 def c4_entrywise(seed: int = 0, n: int = 25_600_000) -> np.ndarray:
     """Config 4: flat gradient, i.i.d. Laplace(0, scale 1e-3)."""
     return _rng("c4", seed).laplace(0.0, 1e-3, size=n).astype(np.float32)
+
+
+def paper_reshape(layer: Sequence[int]) -> tuple:
+    """Section 6's own matricisation of a conv gradient of shape (x, y, k, k): x*y/2 rows by 2*k*k columns
+    (a very tall matrix; an fc gradient stays as it is)."""
+    if len(layer) == 2:
+        return int(layer[0]), int(layer[1])
+    x, y, k, _ = layer
+    return (x * y) // 2, 2 * k * k
+
+
+def c2_paper_reshape(seed: int = 0, convs: Optional[Sequence[Sequence[int]]] = None) -> List[np.ndarray]:
+    """ResNet-18-shaped conv gradients in the paper's tall reshape (short side 2 k^2 = 18): sigma_i = i^-1.5,
+    1 % noise, like config 2."""
+    if convs is None:
+        convs = [(64, 3, 3, 3), (64, 64, 3, 3), (128, 64, 3, 3), (256, 128, 3, 3)]
+    out = []
+    for i, c in enumerate(convs):
+        m, n = paper_reshape(c)
+        out.append(lowrank_plus_noise(_rng("c2r", seed, i), m, n, 1.5, noise_rel=0.01))
+    return out
 
 
 def c5_stress(seed: int = 0, count: int = 96, rows: int = 1024, cols: int = 4096

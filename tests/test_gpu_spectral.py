@@ -103,6 +103,13 @@ def test_batch_mixed_sizes(atomo, oracle):
     _run(atomo, oracle, mats, 2.0, seed=3, step=4)
 
 
+def test_paper_reshape_family(atomo, oracle):
+    # Section 6 matricises a conv gradient (x, y, k, k) as x*y/2 rows by 2 k^2 = 18 columns: very tall layers
+    mats = synth.c2_paper_reshape(0)
+    assert [m.shape for m in mats] == [(96, 18), (2048, 18), (4096, 18), (16384, 18)]
+    _run(atomo, oracle, mats, 2.0, seed=17, step=1)
+
+
 def test_leading_dimension(atomo, oracle):
     rng = np.random.default_rng(7)
     mats = [synth.lowrank_plus_noise(rng, 48, 200, 1.0, noise_rel=0.02),
