@@ -142,6 +142,15 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/,
                            void* payload /*DEVICE*/, int64_t capacity_bytes,
                            const atomo_debug* dbg, void* stream);
 
+/* --- l_q budgets (Section 4) ------------------------------------------------------------------
+ * s_out[l] (HOST) = ||g_l||_1 / ||g_l||_q for every vector: the budget at which entry-wise ATOMO is the
+ * unbiased l_q quantiser of Section 4 -- QSGD for q = 2, TernGrad for q = INFINITY (every g is s-balanced at
+ * this budget, so p_i = |g_i| / ||g||_q).  q >= 1; q = INFINITY is accepted.  fp64 accumulation.  Synchronises
+ * the stream (the norms come back to the host).  A zero vector gives s = 0 and a vector with a NaN or Inf gives
+ * NaN, which atomo_encode_entrywise then rejects as ATOMO_ERR_BUDGET.                                    */
+int atomo_lq_budget(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/, int32_t n_vecs, double q,
+                    double* s_out /*HOST*/, void* stream);
+
 /* --- decode (Eq. 2 summed back to a dense gradient) ----------------------------------------
  * out[l] (DEVICE, fp32) receives layer l: rows[l] x cols[l] row-major with leading dimension
  * cols[l] (entry-wise: rows[l] = 1).  `kind` and the shapes must match the payload's header;

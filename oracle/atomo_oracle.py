@@ -11,6 +11,7 @@ What each function follows:
   The paper fixes only the distribution; generator, key and counter layout are this
   project's definition (Philox4x32-10, Salmon et al., SC'11).  Parity of the *stream*
   is therefore pinned by that publication's known-answer vectors, not by the paper.
+* ``lq_budget`` -- Section 4's budget s = ||g||_1 / ||g||_q (QSGD for q = 2, TernGrad for q = inf).
 * ``jacobi_svd`` -- the SVD  X = sum sigma_i u_i v_i^T  of Section 5 (one-sided Jacobi, C).
 * ``encode_entrywise`` / ``encode_spectral`` -- Eq. (2): keep atom i iff t_i = 1, with
   weight lambda_i / p_i.
@@ -176,6 +177,19 @@ def atomo_probabilities(lam: np.ndarray, s: float) -> Tuple[np.ndarray, int, flo
 # --------------------------------------------------------------------------------------
 # SVD
 # --------------------------------------------------------------------------------------
+def lq_budget(g: np.ndarray, q: float) -> float:
+    """Section 4: the budget s = ||g||_1 / ||g||_q at which entry-wise ATOMO is the l_q quantiser
+    (q = 2: QSGD, q = inf: TernGrad).  Plain definition in fp64; a zero vector gives 0."""
+    a = np.abs(np.asarray(g, dtype=np.float64).reshape(-1))
+    if not (q >= 1.0):
+        raise ValueError("q must be >= 1")
+    l1 = float(a.sum())
+    if l1 == 0.0:
+        return 0.0
+    nq = float(a.max()) if np.isinf(q) else float((a ** q).sum() ** (1.0 / q))
+    return l1 / nq
+
+
 def jacobi_svd(G: np.ndarray, tol: float = 1e-15, max_sweeps: int = 60):
     """Thin SVD of G (m x n) -> (U m x r, sigma r descending, V n x r), r = min(m, n)."""
     G = np.ascontiguousarray(np.asarray(G, dtype=np.float64))

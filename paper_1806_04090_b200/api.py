@@ -28,7 +28,7 @@ EXPORTS = [
     "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
-    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_decode_spectral_static", "atomo_decode_average",
+    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
 ]
 
 
@@ -95,6 +95,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_decode.argtypes = [vp, i32, vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(vp), i32, vp]
     lib.atomo_decode_average.argtypes = [vp, i32, ctypes.POINTER(vp), i32, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                          ctypes.POINTER(vp), i32, vp]
+    lib.atomo_lq_budget.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, ctypes.POINTER(dbl), vp]
     lib.atomo_payload_read_headers.argtypes = [vp, vp, i32, ctypes.POINTER(PayloadHeader),
                                                ctypes.POINTER(LayerHeader), vp]
     lib.atomo_payload_status.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
@@ -386,6 +387,18 @@ class Atomo:
                                            self._stream_ptr(stream))
         self._check(rc, "atomo_decode_average")
         return list(out)
+
+    def atomo_lq_budget(self, vecs: Sequence[torch.Tensor], q: float, stream: Optional[torch.cuda.Stream] = None) -> List[float]:
+        """s = ||g||_1 / ||g||_q per vector (Section 4: q = 2 is QSGD's budget, q = inf TernGrad's)."""
+        n = len(vecs)
+        arr = (_Vec * n)()
+        for i, v in enumerate(vecs):
+            if v.dtype != torch.float32 or not v.is_cuda or not v.is_contiguous():
+                raise ValueError("vectors must be contiguous fp32 CUDA tensors")
+            arr[i].data = v.data_ptr(); arr[i].n = v.numel()
+        out = (ctypes.c_double * n)()
+        self._check(self.lib.atomo_lq_budget(self._h, arr, n, float(q), out, self._stream_ptr(stream)), "atomo_lq_budget")
+        return [float(x) for x in out]
 
     def read_headers(self, payload: Payload, stream: Optional[torch.cuda.Stream] = None):
         gh = PayloadHeader()

@@ -535,6 +535,51 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
 }
 
 // ==================================================================================================
+int atomo_lq_budget(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs, double q, double* s_out, void* stream) {
+  if (!ctx || !vecs || n_vecs <= 0 || !s_out || !(q >= 1.0)) return ATOMO_ERR_INVALID_ARG;
+  for (int l = 0; l < n_vecs; ++l) {
+    if (!vecs[l].data || vecs[l].n <= 0) return ATOMO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(vecs[l].data) & 3u) != 0) return ATOMO_ERR_INVALID_ARG;
+  }
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n_ctas = 148 * 8;
+  double* d_sum = nullptr; float* d_max = nullptr;
+  for (int pass = 0; pass < 2; ++pass) {
+    Arena A(pass ? ctx->ws : nullptr);
+    d_sum = A.take<double>(n_ctas);
+    d_max = A.take<float>(n_ctas);
+    if (pass == 0) { const int rc = ensure_ws(ctx, A.off + 256); if (rc != ATOMO_OK) return rc; }
+  }
+  std::vector<double> h_sum(n_ctas);
+  std::vector<float> h_max(n_ctas);
+  for (int l = 0; l < n_vecs; ++l) {
+    launch_ew_lq(vecs[l].data, vecs[l].n, 0, q, 0.0, d_sum, d_max, n_ctas, st);
+    CK(cudaMemcpyAsync(h_sum.data(), d_sum, n_ctas * sizeof(double), cudaMemcpyDeviceToHost, st));
+    CK(cudaMemcpyAsync(h_max.data(), d_max, n_ctas * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    double l1 = 0.0, amax = 0.0;
+    for (int i = 0; i < n_ctas; ++i) { l1 += h_sum[i]; amax = std::max(amax, (double)h_max[i]); }
+    if (!(amax <= 3.0e38) || !(l1 == l1)) { s_out[l] = std::nan(""); continue; }
+    if (amax == 0.0) { s_out[l] = 0.0; continue; }
+    double norm_q;
+    if (std::isinf(q)) norm_q = amax;
+    else if (q == 1.0) norm_q = l1;
+    else {
+      launch_ew_lq(vecs[l].data, vecs[l].n, 1, q, 1.0 / amax, d_sum, d_max, n_ctas, st);
+      CK(cudaMemcpyAsync(h_sum.data(), d_sum, n_ctas * sizeof(double), cudaMemcpyDeviceToHost, st));
+      CK(cudaStreamSynchronize(st));
+      double t = 0.0;
+      for (int i = 0; i < n_ctas; ++i) t += h_sum[i];
+      norm_q = amax * std::pow(t, 1.0 / q);
+    }
+    s_out[l] = l1 / norm_q;
+  }
+  CK(cudaGetLastError());
+  return ATOMO_OK;
+}
+
+// ==================================================================================================
 int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload, const int64_t* rows, const int64_t* cols,
                  float* const* out, int32_t n_layers, void* stream) {
   if (!ctx || !payload || !rows || !cols || !out || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;

@@ -350,6 +350,38 @@ __global__ void __launch_bounds__(kEwThreads) ew_decode_kernel(EwDecode d) {
   }
 }
 
+// ---- l_q budget (Section 4: the budget s = ||g||_1 / ||g||_q turns entry-wise ATOMO into QSGD for q = 2 and
+//      into TernGrad for q = infinity) --------------------------------------------------------------------
+// pass 0: per-CTA sum |g| and max |g|; pass 1 (finite q > 1 only): per-CTA sum (|g| / amax)^q.  fp64 sums.
+__global__ void __launch_bounds__(kEwThreads) ew_lq_kernel(const float* __restrict__ g, int64_t n, int pass, double q,
+                                                           double inv_amax, double* __restrict__ part_sum,
+                                                           float* __restrict__ part_max) {
+  __shared__ double s_sum[kEwThreads / kWarp];
+  __shared__ float s_max[kEwThreads / kWarp];
+  double sum = 0.0;
+  float amax = 0.0f;
+  for (int64_t i = (int64_t)blockIdx.x * kEwThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kEwThreads) {
+    const float a = fabsf(__ldg(g + i));
+    if (pass == 0) { sum += (double)a; amax = fmaxf(amax, a); if (!(a <= 3.0e38f)) amax = __int_as_float(0x7f800000); }
+    else if (a > 0.0f) sum += (q == 2.0) ? ((double)a * inv_amax) * ((double)a * inv_amax) : pow((double)a * inv_amax, q);
+  }
+  sum = warp_sum(sum); amax = warp_max(amax);
+  const int lane = threadIdx.x % kWarp, w = threadIdx.x / kWarp;
+  if (lane == 0) { s_sum[w] = sum; s_max[w] = amax; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double t = 0.0; float m = 0.0f;
+    for (int i = 0; i < kEwThreads / kWarp; ++i) { t += s_sum[i]; m = fmaxf(m, s_max[i]); }   // fixed order
+    part_sum[blockIdx.x] = t;
+    if (pass == 0) part_max[blockIdx.x] = m;
+  }
+}
+
+void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax, double* part_sum, float* part_max,
+                  int n_ctas, cudaStream_t st) {
+  ew_lq_kernel<<<n_ctas, kEwThreads, 0, st>>>(g, n, pass, q, inv_amax, part_sum, part_max);
+}
+
 // ---- host-side launchers --------------------------------------------------------------------------
 int ew_solve_max_blocks() {
   int dev = 0, sms = 0, per_sm = 0;

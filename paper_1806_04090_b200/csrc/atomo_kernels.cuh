@@ -46,6 +46,8 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st); // returns a cud
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st);
 void launch_ew_decode(const EwDecode& d, cudaStream_t st);
 int ew_tile_elems();
+void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax, double* part_sum, float* part_max,
+                  int n_ctas, cudaStream_t st);
 int ew_sample_pack_ctas(int64_t n_tiles);
 
 // ================================= spectral path =================================================

@@ -160,3 +160,27 @@ def test_config4_full_size(atomo, oracle, frac):
     # 25.6M Laplace(0, 1e-3) entries, budgets 0.1 %, 1 %, 10 % of the length, in the bench's launch configuration
     g = synth.c4_entrywise(0)
     _run(atomo, oracle, [g], frac * g.size, seed=7, step=1, k_cap=int(frac * g.size * 1.05) + 1000)
+
+
+def test_lq_budget_front_end(atomo, oracle):
+    """atomo_lq_budget against the plain definition, and the budgets fed back into the encoder (Section 4)."""
+    import torch
+    rng = np.random.default_rng(31)
+    vecs = [synth.c1_entrywise(2), (rng.laplace(0.0, 1e-3, 1_000_003)).astype(np.float32), np.zeros(100, dtype=np.float32)]
+    ts = [torch.from_numpy(v).cuda() for v in vecs]
+    for q in (1.0, 2.0, 3.5, float("inf")):
+        got = atomo.atomo_lq_budget(ts, q)
+        for v, s_gpu in zip(vecs, got):
+            want = oracle.lq_budget(v, q)
+            assert s_gpu == pytest.approx(want, rel=1e-12, abs=0.0), (q, s_gpu, want)
+    # QSGD budget: kept unsaturated values are +-||g||_2 (already covered with host-computed budgets; here end to end)
+    g = vecs[0]
+    s2 = atomo.atomo_lq_budget(ts[:1], 2.0)[0]
+    pay, _ = atomo.atomo_encode_entrywise(ts[:1], s2, seed=3, k_cap=g.size)
+    arr = pay.layer_arrays(0)
+    assert pay.headers()[1][0].n_sat == 0
+    np.testing.assert_allclose(np.abs(arr["val"]), np.linalg.norm(g.astype(np.float64)), rtol=1e-6)
+    bad = torch.tensor([1.0, float("nan"), 2.0], device="cuda")
+    assert np.isnan(atomo.atomo_lq_budget([bad], 2.0)[0])
+    with pytest.raises(Exception):
+        atomo.atomo_lq_budget(ts[:1], 0.5)

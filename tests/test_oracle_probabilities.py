@@ -156,6 +156,32 @@ def test_qsgd_terngrad_lq_special_cases(oracle):
             assert enc["mask"][np.argmax(np.abs(g))] or p[np.argmax(np.abs(g))] < 1.0
 
 
+def test_lq_budget_pins(oracle):
+    # closed forms: a one-hot vector has every norm equal; n equal entries give n^(1 - 1/q)
+    hot = np.zeros(9); hot[4] = -3.5
+    for q in (1.0, 1.5, 2.0, 7.0, np.inf):
+        assert oracle.lq_budget(hot, q) == pytest.approx(1.0, rel=1e-15)
+        flat = np.full(64, -0.25)
+        want = 64.0 if np.isinf(q) else 64.0 ** (1.0 - 1.0 / q)
+        assert oracle.lq_budget(flat, q) == pytest.approx(want, rel=1e-13)
+    assert oracle.lq_budget(np.zeros(5), 2.0) == 0.0
+    g = np.array([3.0, -4.0, 0.0, 12.0])
+    assert oracle.lq_budget(g, 1.0) == pytest.approx(1.0, rel=1e-15)
+    assert oracle.lq_budget(g, 2.0) == pytest.approx(19.0 / 13.0, rel=1e-15)       # ||g||_2 = 13
+    assert oracle.lq_budget(g, np.inf) == pytest.approx(19.0 / 12.0, rel=1e-15)
+    with pytest.raises(ValueError):
+        oracle.lq_budget(g, 0.5)
+    # Section 4: at this budget every vector is s-balanced and Algorithm 1 returns p_i = |g_i| / ||g||_q
+    rng = np.random.default_rng(12)
+    for q in (2.0, 3.0, np.inf):
+        g = rng.standard_normal(500) * np.exp(rng.standard_normal(500))
+        s = oracle.lq_budget(g, q)
+        nq = np.abs(g).max() if np.isinf(q) else (np.abs(g) ** q).sum() ** (1.0 / q)
+        p, n_s, _ = oracle.atomo_probabilities(g, s)
+        assert n_s == 0
+        np.testing.assert_allclose(p, np.abs(g) / nq, rtol=1e-12, atol=0)
+
+
 def test_budget_errors(oracle):
     for bad in (0.0, -1.0, float("nan"), float("inf")):
         with pytest.raises(ValueError):
