@@ -245,11 +245,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
-  std::vector<TileRef> gram_tiles, pairs16, pairs8, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
+  std::vector<TileRef> gram_tiles, pairs16, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
   const int map_bytes = sp_tc_map_bytes();
   std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
   int chol_panels = 0;
-  int rp16_max = 0, steps16 = 0, steps8 = 0, r_max = 0, rp_max = 0, r_max_tall = 0, k_cap_max = 1;
+  int rp16_max = 0, steps16 = 0, r_max = 0, rp_max = 0, r_max_tall = 0, k_cap_max = 1;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
     const atomo_mat& m = layers[l];
@@ -300,7 +300,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
-  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_p8 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
+  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
   uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
@@ -310,7 +310,6 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_layers = A.take<SpLayer>(n_layers);
     d_gram = A.take<TileRef>(gram_tiles.size());
     d_p16 = A.take<TileRef>(pairs16.size());
-    d_p8 = A.take<TileRef>(pairs8.size());
     d_bp = A.take<TileRef>(bp_tiles.size());
     d_chol = A.take<TileRef>(chol_ctas.size());
     d_ref = A.take<TileRef>(refine_tiles.size());
@@ -373,7 +372,6 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   CK(cudaMemcpyAsync(d_layers, L.data(), L.size() * sizeof(SpLayer), cudaMemcpyHostToDevice, st));
   if (!gram_tiles.empty()) CK(cudaMemcpyAsync(d_gram, gram_tiles.data(), gram_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!pairs16.empty()) CK(cudaMemcpyAsync(d_p16, pairs16.data(), pairs16.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!pairs8.empty()) CK(cudaMemcpyAsync(d_p8, pairs8.data(), pairs8.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!tc_tiles.empty()) {
     CK(cudaMemcpyAsync(d_tc, tc_tiles.data(), tc_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
@@ -401,7 +399,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S1: eigen-solver; the host reads a convergence flag once per sweep of the largest layer ----
   stage_begin(ctx, ATOMO_STAGE_EIG, st);
-  int t16 = 0, t8 = 0;
+  int t16 = 0;
   int64_t n_eig_launch = 0;
   const bool persistent = ctx->persistent_eig && (int)pairs16.size() <= sp_jacobi_persistent_capacity(rp16_max);
   if (persistent) {
@@ -410,7 +408,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     const int t_max = steps16 * max_sweeps;
     const int e = launch_sp_jacobi_persistent(d_layers, d_p16, (int)pairs16.size(), rp16_max, max_sweeps, ctx->tol, d_flag + 2, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
-    launch_sp_check(d_layers, n_layers, t_max, 0, max_sweeps, d_flag, st);
+    launch_sp_check(d_layers, n_layers, t_max, max_sweeps, d_flag, st);
     n_eig_launch = 2;
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
@@ -420,7 +418,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   for (int it = 0; it < max_sweeps; ++it) {
     for (int j = 0; j < steps16; ++j, ++t16, ++n_eig_launch)
       launch_sp_jacobi_step(d_layers, d_p16, (int)pairs16.size(), 16, rp16_max, t16, max_sweeps, ctx->tol, st);
-    launch_sp_check(d_layers, n_layers, t16, t8, max_sweeps, d_flag, st);
+    launch_sp_check(d_layers, n_layers, t16, max_sweeps, d_flag, st);
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }

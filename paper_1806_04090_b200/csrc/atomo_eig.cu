@@ -415,8 +415,8 @@ void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int 
   sp_jacobi_step_kernel<<<n_pairs, kJacobiThreads, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
 }
 
-// convergence bookkeeping after t16 / t8 steps have been enqueued for the two kernel classes
-__global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers, int t16, int t8, int max_sweeps,
+// convergence bookkeeping after t_done steps have been enqueued
+__global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers, int t_done, int max_sweeps,
                                 uint32_t* all_done) {
   __shared__ int s_pending;
   if (threadIdx.x == 0) s_pending = 0;
@@ -424,7 +424,6 @@ __global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers
   for (int l = threadIdx.x; l < n_layers; l += blockDim.x) {
     const SpLayer& L = layers[l];
     const int steps = L.nb - 1;
-    const int t_done = t16; (void)t8;
     const int sweeps_done = min(t_done / steps, max_sweeps);
     int conv = -1;
     for (int wv = 0; wv < sweeps_done; ++wv) if (L.rot_count[wv] == 0) { conv = wv; break; }
@@ -438,103 +437,22 @@ __global__ void sp_check_kernel(const SpLayer* __restrict__ layers, int n_layers
   if (threadIdx.x == 0) *all_done = s_pending == 0 ? 1u : 0u;
 }
 
-void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
+void launch_sp_check(const SpLayer* d_layers, int n_layers, int t_done, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st) {
-  sp_check_kernel<<<1, 256, 0, st>>>(d_layers, n_layers, t16, t8, max_sweeps, d_all_done);
+  sp_check_kernel<<<1, 256, 0, st>>>(d_layers, n_layers, t_done, max_sweeps, d_all_done);
 }
 
 // =================================================================================================
 // Cholesky factor of the scaled Gram matrix, written transposed: X[c][i] = L[i][c].
-// One CTA per layer, one thread per row, left-looking over panels of 32 columns; a thread keeps its
-// row of the current panel in registers.  A pivot below kPivotFloor (trace(A) = 1) is rounding noise
-// of the fp32 Gram matrix: that column of L is set to zero (L L^T then differs from A by that noise).
+// One thread per row, left-looking over panels of 32 columns; a thread keeps its row of the current panel
+// in registers.  A pivot below kPivotFloor (trace(A) = 1) is rounding noise of the fp32 Gram matrix: that
+// column of L is set to zero (L L^T then differs from A by that noise).
 // =================================================================================================
 constexpr float kPivotFloor = 1e-9f;
 constexpr int kCholPanel = 32;
 
-// kThreads = 512 serves layers of up to 512 rows with more loads in flight per thread (it may use 128 registers),
-// kThreads = 1024 the layers of 513..1024 rows.
-template <int kThreads, int kUnroll>
-__global__ void __launch_bounds__(kThreads) sp_cholesky_kernel(const SpLayer* __restrict__ layers) {
-  const SpLayer& L = layers[blockIdx.x];
-  if (L.acc || L.rp > kThreads || (kThreads == 1024 && L.rp <= 512)) return;   // other classes: the other instantiation / sp_cholesky_big_kernel
-  __shared__ __align__(16) float s_k[kCholPanel][kCholPanel];   // L[j0 + c][k0 + kk] for the current k chunk
-  __shared__ float s_ldd[kCholPanel][kCholPanel + 1];   // diagonal block of L
-  __shared__ float s_inv[kCholPanel];
-  const int r = L.r, rp = L.rp;
-  const int i = threadIdx.x, lane = i % 32, warp = i / 32;
-  const float* __restrict__ A = L.A;
-  const int64_t lda = L.lda;
-  float* X = L.X;
-  for (int j0 = 0; j0 < r; j0 += kCholPanel) {
-    const bool active = i >= j0 && i < r;
-    float p[kCholPanel];
-#pragma unroll
-    for (int c = 0; c < kCholPanel; ++c) p[c] = (active && j0 + c < r) ? A[(int64_t)(j0 + c) * lda + i] : 0.0f;
-    // p[c] -= sum_{k < j0} L[i][k] L[j0+c][k]
-    for (int k0 = 0; k0 < j0; k0 += kCholPanel) {
-      __syncthreads();
-      for (int idx = i; idx < kCholPanel * kCholPanel; idx += blockDim.x) {
-        const int kk = idx / kCholPanel, c = idx % kCholPanel;
-        s_k[kk][c] = X[(int64_t)(k0 + kk) * rp + j0 + c];
-      }
-      __syncthreads();
-      if (active) {
-#pragma unroll kUnroll
-        for (int kk = 0; kk < kCholPanel; ++kk) {
-          const float xi = -X[(int64_t)(k0 + kk) * rp + i];
-#pragma unroll
-          for (int c = 0; c < kCholPanel; c += 4) {
-            const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
-            p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
-            p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
-          }
-        }
-      }
-    }
-    // diagonal block: the warp whose lanes own rows j0 .. j0+31
-    if (warp == j0 / 32) {
-#pragma unroll
-      for (int c = 0; c < kCholPanel; ++c) {
-        const float d = __shfl_sync(0xffffffffu, p[c], c);
-        const float lcc = d > kPivotFloor ? sqrtf(d) : 0.0f;
-        const float inv = lcc > 0.0f ? 1.0f / lcc : 0.0f;
-        const float lic = lane > c ? p[c] * inv : (lane == c ? lcc : 0.0f);
-        p[c] = lic;
-#pragma unroll
-        for (int c2 = 0; c2 < kCholPanel; ++c2) {      // full range + predicate: a triangular loop is not unrolled
-          if (c2 > c) {                                //                         and would push p[] to local memory
-            const float l2 = __shfl_sync(0xffffffffu, lic, c2);
-            if (lane > c) p[c2] = fmaf(-lic, l2, p[c2]);
-          }
-        }
-        if (lane == c) s_inv[c] = inv;
-      }
-#pragma unroll
-      for (int c = 0; c < kCholPanel; ++c) s_ldd[lane][c] = p[c];
-    }
-    __syncthreads();
-    // rows below the diagonal block: solve y L_dd^T = p
-    if (active && i >= j0 + kCholPanel) {
-#pragma unroll
-      for (int c = 0; c < kCholPanel; ++c) {
-        float acc = p[c];
-#pragma unroll
-        for (int k = 0; k < c; ++k) acc = fmaf(-p[k], s_ldd[c][k], acc);
-        p[c] = acc * s_inv[c];
-      }
-    }
-    if (active) {
-#pragma unroll
-      for (int c = 0; c < kCholPanel; ++c)
-        if (j0 + c < r) X[(int64_t)(j0 + c) * rp + i] = p[c];
-    }
-    __syncthreads();
-  }
-}
-
-// The same factorisation spread over a cluster of 8 CTAs per layer (layers of up to 1024 rows): the panel
-// update is FMA-bound on one SM, so each CTA takes max(32, rp / 8) consecutive rows, one thread per row.
+// Layers of up to 1024 rows: a cluster of 8 CTAs per layer (the panel update would be FMA-bound on one SM);
+// each CTA takes max(32, rp / 8) consecutive rows.
 // Per panel: every CTA updates its rows; the warp that owns the diagonal block factors it and publishes it in
 // global memory; cluster barrier; every CTA solves its rows against it and stores them; cluster barrier (the
 // next panel reads rows of L written by other CTAs; those reads bypass L1).

@@ -111,7 +111,7 @@ int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n
 int sp_cholesky_big_rows_per_cta();
 int sp_configure_eig();
 // convergence bookkeeping after t16 / t8 steps were enqueued for the two kernel classes
-void launch_sp_check(const SpLayer* d_layers, int n_layers, int t16, int t8, int max_sweeps, uint32_t* d_all_done,
+void launch_sp_check(const SpLayer* d_layers, int n_layers, int t_done, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st);
 void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key,
