@@ -230,15 +230,26 @@ def run_ours(args):
     payload = torch.empty(api.payload_bytes_spectral(shapes, k_cap), dtype=torch.uint8, device=dev)
     outs = [torch.empty(sh, dtype=torch.float32, device=dev) for sh in shapes]
 
-    exchange = bool(args.exchange) and world > 1
+    exchange = args.exchange if world > 1 else "none"
+    peers = None
+    if exchange == "p2p":                               # payload lives where the peers can read it in place
+        peers = dist.PeerPayloads(payload.numel(), dev)
+        payload = peers.buf
 
     def combine(pay):
-        """decode; with --exchange on N > 1 GPUs: all-gather the payloads over NCCL, then the averaging decode"""
-        if not exchange:
+        """decode.  --exchange nccl: all-gather the payloads, then the averaging decode.  --exchange p2p: the
+        averaging decode reads every rank's payload in place over NVLink (one kernel, no collective)."""
+        if exchange == "none":
             a.atomo_decode(pay, out=outs)
             return
-        bufs = dist.all_gather_bytes(pay.buf)
+        if exchange == "p2p":
+            peers.publish()
+            bufs = peers.views()
+        else:
+            bufs = dist.all_gather_bytes(pay.buf)
         a.atomo_decode_average([api.Payload(b, pay.kind, pay.shapes, pay.k_cap, a) for b in bufs], out=outs)
+        if exchange == "p2p":
+            peers.release()
 
     def step(i, layers):
         pay, _ = a.atomo_encode_spectral(layers, s, seed + rank, step=i, k_cap=k_cap, payload=payload)
@@ -351,8 +362,10 @@ def run_ours(args):
                                    "s=2, one batched encode + decode per step",
                        "k_cap": k_cap, "l2": f"inputs rotate over {n_sets} distinct sets ({n_sets * in_bytes / 2**20:.0f} MiB "
                                              f"> 126 MiB L2) so each step reads gradients from HBM",
-                       "parallelism": ("data-parallel: payload all-gather + averaging decode" if exchange else
-                                       "independent replicas, no collective") if world > 1 else "single GPU",
+                       "parallelism": {"none": "independent replicas, no collective",
+                                       "nccl": "data-parallel: payload all-gather + averaging decode",
+                                       "p2p": "data-parallel: averaging decode reads the peers' payloads over NVLink"}[exchange]
+                       if world > 1 else "single GPU",
                        "jacobi_sweeps_last_step": sweeps_seen,
                        "eig_ms_per_step": eig_ms / args.steps},
             "clocks": clocks,
@@ -388,9 +401,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--exchange", action="store_true",
-                    help="N > 1: all-gather the payloads and decode their average on every rank (the data-parallel "
-                         "combine step) instead of independent replicas")
+    ap.add_argument("--exchange", default="none", choices=["none", "nccl", "p2p"],
+                    help="N > 1: the data-parallel combine step instead of independent replicas -- nccl: all-gather "
+                         "the payloads, then decode their average; p2p: the averaging decode reads the peers' payloads "
+                         "in place over NVLink")
     ap.add_argument("--no-extras", action="store_true", help="skip the entry-wise (config 4) figures")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -75,6 +75,50 @@ def all_gather_bytes(buf: torch.Tensor) -> List[torch.Tensor]:
     return list(gathered.view(world, buf.numel()).unbind(0))
 
 
+class PeerPayloads:
+    """Payload buffers that every rank of one node can read in place (CUDA peer access over NVLink through
+    torch's symmetric memory).  Each rank encodes into `self.buf`; after `publish()` the averaging decode is
+    given `self.views()` -- tensors that alias the peers' buffers -- so ONE kernel both fetches every
+    worker's payload over NVLink (plain loads, a few hundred KB) and forms the averaged gradient: there is no
+    separate collective and no staging copy.  `release()` keeps a rank from overwriting its buffer while a
+    peer may still be reading it.  Without a process group (or without symmetric memory) the object holds a
+    plain local buffer and `views()` is just that buffer.
+    Not exercised on more than one GPU in this build (one GPU available): the single-rank path and the gloo
+    fallback are what the tests cover."""
+
+    def __init__(self, nbytes: int, device: torch.device):
+        self.handle = None
+        self.world = dist.get_world_size() if dist.is_initialized() else 1
+        self.nbytes = int(nbytes)
+        if self.world > 1 and device.type == "cuda":
+            import torch.distributed._symmetric_memory as symm_mem
+            self.buf = symm_mem.empty(self.nbytes, dtype=torch.uint8, device=device)
+            self.handle = symm_mem.rendezvous(self.buf, dist.group.WORLD)
+        else:
+            self.buf = torch.empty(self.nbytes, dtype=torch.uint8, device=device)
+
+    def publish(self) -> None:
+        """Call after encode has been enqueued: when it returns, every rank's payload of this step is complete
+        and visible to the kernels enqueued next on the current stream."""
+        if self.handle is not None:
+            self.handle.barrier(channel=0)
+        elif self.world > 1:
+            dist.barrier()
+
+    def views(self) -> List[torch.Tensor]:
+        if self.handle is None:
+            return [self.buf] if self.world == 1 else all_gather_bytes(self.buf)
+        return [self.handle.get_buffer(r, (self.nbytes,), torch.uint8) for r in range(self.world)]
+
+    def release(self) -> None:
+        """Call after the averaging decode has been enqueued: no rank starts the next encode (which rewrites its
+        buffer) before every rank has finished reading."""
+        if self.handle is not None:
+            self.handle.barrier(channel=1)
+        elif self.world > 1:
+            dist.barrier()
+
+
 def finish() -> None:
     if dist.is_initialized():
         dist.destroy_process_group()

@@ -25,6 +25,14 @@ def _worker(rank, world, port, q):
     got = d.all_gather_bytes(mine)
     gathered_ok = len(got) == world and all(
         torch.equal(got[k], (torch.arange(1000, dtype=torch.int64) * (k + 3) % 251).to(torch.uint8)) for k in range(world))
+    # the same exchange through the peer-buffer object (on CPU it falls back to the all-gather)
+    peers = d.PeerPayloads(1000, torch.device("cpu"))
+    peers.buf.copy_(mine)
+    peers.publish()
+    views = peers.views()
+    gathered_ok = gathered_ok and len(views) == world and all(
+        torch.equal(views[k], (torch.arange(1000, dtype=torch.int64) * (k + 3) % 251).to(torch.uint8)) for k in range(world))
+    peers.release()
     d.barrier()
     d.finish()
     q.put((r, w, t_max, units, parts, gathered_ok))
