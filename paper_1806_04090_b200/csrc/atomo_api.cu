@@ -245,11 +245,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
-  std::vector<TileRef> gram_tiles, pairs16, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
+  std::vector<TileRef> gram_tiles, block_pairs, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
   const int map_bytes = sp_tc_map_bytes();
   std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
   int chol_panels = 0;
-  int rp16_max = 0, steps16 = 0, r_max = 0, rp_max = 0, r_max_tall = 0, k_cap_max = 1;
+  int row_floats_max = 0, steps_max = 0, r_max = 0, rp_max = 0, r_max_tall = 0, k_cap_max = 1;
   for (int l = 0; l < n_layers; ++l) {
     SpLayer& d = L[l];
     const atomo_mat& m = layers[l];
@@ -275,8 +275,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     } else {
       for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
     }
-    for (int p = 0; p < d.nb / 2; ++p) pairs16.push_back({l, p, 0, 0});
-    rp16_max = std::max(rp16_max, d.ldx); steps16 = std::max(steps16, d.nb - 1);
+    for (int p = 0; p < d.nb / 2; ++p) block_pairs.push_back({l, p, 0, 0});
+    row_floats_max = std::max(row_floats_max, d.ldx); steps_max = std::max(steps_max, d.nb - 1);
     if (!d.acc && d.rp > 1024) {
       const int per = sp_cholesky_big_rows_per_cta();
       for (int c = 0; c < (d.rp + per - 1) / per; ++c) chol_ctas.push_back({l, c, 0, 0});
@@ -300,7 +300,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
-  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_p16 = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
+  SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_pairs = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
   uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
@@ -309,7 +309,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     Arena A(pass ? ctx->ws : nullptr);
     d_layers = A.take<SpLayer>(n_layers);
     d_gram = A.take<TileRef>(gram_tiles.size());
-    d_p16 = A.take<TileRef>(pairs16.size());
+    d_pairs = A.take<TileRef>(block_pairs.size());
     d_bp = A.take<TileRef>(bp_tiles.size());
     d_chol = A.take<TileRef>(chol_ctas.size());
     d_ref = A.take<TileRef>(refine_tiles.size());
@@ -371,7 +371,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(d_layers, L.data(), L.size() * sizeof(SpLayer), cudaMemcpyHostToDevice, st));
   if (!gram_tiles.empty()) CK(cudaMemcpyAsync(d_gram, gram_tiles.data(), gram_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!pairs16.empty()) CK(cudaMemcpyAsync(d_p16, pairs16.data(), pairs16.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  if (!block_pairs.empty()) CK(cudaMemcpyAsync(d_pairs, block_pairs.data(), block_pairs.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
   if (!tc_tiles.empty()) {
     CK(cudaMemcpyAsync(d_tc, tc_tiles.data(), tc_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
@@ -399,14 +399,14 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S1: eigen-solver; the host reads a convergence flag once per sweep of the largest layer ----
   stage_begin(ctx, ATOMO_STAGE_EIG, st);
-  int t16 = 0;
+  int t_done = 0;
   int64_t n_eig_launch = 0;
-  const bool persistent = ctx->persistent_eig && (int)pairs16.size() <= sp_jacobi_persistent_capacity(rp16_max);
+  const bool persistent = ctx->persistent_eig && (int)block_pairs.size() <= sp_jacobi_persistent_capacity(row_floats_max);
   if (persistent) {
     // one cooperative launch: d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
     CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
-    const int t_max = steps16 * max_sweeps;
-    const int e = launch_sp_jacobi_persistent(d_layers, d_p16, (int)pairs16.size(), rp16_max, max_sweeps, ctx->tol, d_flag + 2, st);
+    const int t_max = steps_max * max_sweeps;
+    const int e = launch_sp_jacobi_persistent(d_layers, d_pairs, (int)block_pairs.size(), row_floats_max, max_sweeps, ctx->tol, d_flag + 2, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
     launch_sp_check(d_layers, n_layers, t_max, max_sweeps, d_flag, st);
     n_eig_launch = 2;
@@ -416,9 +416,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (ctx->h_flag[2] != 0) { ctx->err = "a step barrier of the persistent eigen-solve ran out of polls"; return ATOMO_ERR_TIMEOUT; }
   } else
   for (int it = 0; it < max_sweeps; ++it) {
-    for (int j = 0; j < steps16; ++j, ++t16, ++n_eig_launch)
-      launch_sp_jacobi_step(d_layers, d_p16, (int)pairs16.size(), 16, rp16_max, t16, max_sweeps, ctx->tol, st);
-    launch_sp_check(d_layers, n_layers, t16, max_sweeps, d_flag, st);
+    for (int j = 0; j < steps_max; ++j, ++t_done, ++n_eig_launch)
+      launch_sp_jacobi_step(d_layers, d_pairs, (int)block_pairs.size(), row_floats_max, t_done, max_sweeps, ctx->tol, st);
+    launch_sp_check(d_layers, n_layers, t_done, max_sweeps, d_flag, st);
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }

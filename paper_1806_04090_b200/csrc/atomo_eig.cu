@@ -407,10 +407,9 @@ int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs,
                                           smem, st);
 }
 
-void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st) {
   if (n_pairs <= 0) return;
-  (void)B;
   const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
   sp_jacobi_step_kernel<<<n_pairs, kJacobiThreads, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
 }

@@ -99,7 +99,7 @@ void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling
 // one Jacobi step (global step index t) for every layer of one (B, RP) class
-void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int B, int row_floats_max,
+void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
 // whole eigen-solve in one cooperative launch when all block pairs are co-resident; returns a cudaError_t
 int sp_jacobi_persistent_capacity(int row_floats_max);
