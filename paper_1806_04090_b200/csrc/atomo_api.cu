@@ -401,15 +401,34 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   stage_begin(ctx, ATOMO_STAGE_EIG, st);
   int t_done = 0;
   int64_t n_eig_launch = 0;
-  const bool persistent = ctx->persistent_eig && (int)block_pairs.size() <= sp_jacobi_persistent_capacity(row_floats_max);
+  // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
+  // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
+  // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
+  const int capacity = ctx->persistent_eig ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
+  int max_layer_pairs = 0;
+  for (int l = 0; l < n_layers; ++l) max_layer_pairs = std::max(max_layer_pairs, L[l].nb / 2);
+  const bool persistent = capacity > 0 && max_layer_pairs <= capacity;
   if (persistent) {
-    // one cooperative launch: d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
+    // d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
     CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
     const int t_max = steps_max * max_sweeps;
-    const int e = launch_sp_jacobi_persistent(d_layers, d_pairs, (int)block_pairs.size(), row_floats_max, max_sweeps, ctx->tol, d_flag + 2, st);
-    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
+    size_t first = 0;                                     // block_pairs is ordered by layer
+    while (first < block_pairs.size()) {
+      size_t last = first;
+      while (last < block_pairs.size()) {
+        const int l = block_pairs[last].layer;
+        const size_t layer_pairs = (size_t)L[l].nb / 2;
+        if (last + layer_pairs - first > (size_t)capacity) break;
+        last += layer_pairs;
+      }
+      const int e = launch_sp_jacobi_persistent(d_layers, d_pairs + first, (int)(last - first), row_floats_max, max_sweeps,
+                                                ctx->tol, d_flag + 2, st);
+      if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(jacobi)");
+      ++n_eig_launch;
+      first = last;
+    }
     launch_sp_check(d_layers, n_layers, t_max, max_sweeps, d_flag, st);
-    n_eig_launch = 2;
+    ++n_eig_launch;
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
