@@ -226,9 +226,11 @@ int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
 /* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
  * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
-/* Eigen-solver launch scheme: 1 (default) = when every block pair of the batch fits on the GPU at once (one CTA
- * per SM), the whole solve is one cooperative launch with grid barriers between Jacobi steps and a single host
- * wait at its end; larger batches, or 0, use one launch per step and one host wait per sweep.              */
+/* Eigen-solver launch scheme: 1 (default) = cooperative launches in which the block pairs of a group of whole
+ * layers are co-resident (one CTA per SM) and run all their Jacobi steps, with a barrier among the CTAs of a layer
+ * between steps, and a single host wait at the end; a batch that fits the GPU is one such launch.  A batch with a
+ * layer that alone needs more CTAs than the GPU holds (short side above 2048), or 0, uses one launch per step and
+ * one host wait per sweep.                                                                                   */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
 
 #ifdef __cplusplus
