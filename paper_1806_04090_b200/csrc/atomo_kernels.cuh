@@ -31,7 +31,7 @@ struct EwVec {
   uint32_t* mask_words;
   int n_ctas;                                                  // chunks (CTAs) of the sample / pack kernel
   uint64_t* tile_status;                                       // [chunks] ready flag (bit 63) | kept atoms of the chunk; zeroed per call
-  uint32_t* ticket;                                            // next tile to hand out; zeroed per call
+  uint32_t* ticket;                                            // next chunk to hand out; zeroed per call
   uint32_t* tile_table;                                        // payload: kept atoms before each tile
   float* prob_out;                                             // debug or nullptr
 };
@@ -75,7 +75,7 @@ struct SpLayer {
   uint32_t* rot_count;         // [max_sweeps] rotations applied in each sweep
   uint32_t* step_bar;          // arrivals of the layer's CTAs at the step barrier of the persistent eigen-solve
   float* scale;                // 1 float: power-of-two scaling applied to A
-  float* chol_dd;              // 32 x 32 + 32 floats: diagonal block published by its owner (layers > 1024 rows)
+  float* chol_dd;              // 32 x 32 + 32 floats: diagonal block of the current Cholesky panel, published by its owner
   float* dbg_short;            // r x r or nullptr
   int tc;                      // Gram matrix came from the tensor-core kernel (see sp_scale_kernel)
   int refine, refine_tiles;    // singular values from the projection norms; tiles along the long side
@@ -98,19 +98,19 @@ void launch_ew_decode_average(const uint8_t* const* d_payloads, int n_payloads, 
 void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling
-// one Jacobi step (global step index t) for every layer of one (B, RP) class
+// one Jacobi step (global step index t) for every layer of the batch
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
-// whole eigen-solve in one cooperative launch when all block pairs are co-resident; returns a cudaError_t
+// whole eigen-solve of a group of layers in one cooperative launch (block pairs co-resident); returns a cudaError_t
 int sp_jacobi_persistent_capacity(int row_floats_max);
 int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                                 int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
+// layers of up to 1024 rows: clusters of 8 CTAs; more rows: cooperative launch.  Both return a cudaError_t
 int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
-// layers with more than 1024 rows: cooperative launch, returns a cudaError_t
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
 int sp_cholesky_big_rows_per_cta();
 int sp_configure_eig();
-// convergence bookkeeping after t16 / t8 steps were enqueued for the two kernel classes
+// convergence bookkeeping after t_done steps were enqueued
 void launch_sp_check(const SpLayer* d_layers, int n_layers, int t_done, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st);
 void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
