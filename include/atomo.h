@@ -226,11 +226,17 @@ int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
 /* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
  * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
-/* Eigen-solver launch scheme: 1 (default) = cooperative launches in which the block pairs of a group of whole
- * layers are co-resident (one CTA per SM) and run all their Jacobi steps, with a barrier among the CTAs of a layer
- * between steps, and a single host wait at the end; a batch that fits the GPU is one such launch.  A batch with a
- * layer that alone needs more CTAs than the GPU holds (short side above 2048), or 0, uses one launch per step and
- * one host wait per sweep.                                                                                   */
+/* Eigen-solver launch scheme (`enabled` = 0, 1 or 2):
+ * 2 (default) = thread-block clusters where they apply: when every layer of the batch has at most 16 block
+ *     pairs (padded short side <= 512), each layer's CTAs sit in one 16-CTA cluster for the whole solve and hand
+ *     their blocks to one another through distributed shared memory, with a cluster barrier per Jacobi step;
+ *     other batches, or a GPU that cannot place such clusters, take scheme 1;
+ * 1 = cooperative launches in which the block pairs of a group of whole layers are co-resident (one CTA per SM)
+ *     and run all their Jacobi steps, blocks exchanged through global memory (L2) with a barrier among the CTAs
+ *     of a layer between steps; a batch that fits the GPU is one such launch.  A batch with a layer that alone
+ *     needs more CTAs than the GPU holds (short side above 2048) takes scheme 0;
+ * 0 = one launch per step and one host wait per sweep.
+ * Schemes 1 and 2 wait on the host once, at the end of the solve.                                            */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
 
 #ifdef __cplusplus

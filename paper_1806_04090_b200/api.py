@@ -424,8 +424,9 @@ class Atomo:
         self._check(self.lib.atomo_get_stage_times(self._h, ms, ln), "atomo_get_stage_times")
         return {k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)}
 
-    def set_persistent_eig(self, enabled: bool):
-        self._check(self.lib.atomo_set_persistent_eig(self._h, 1 if enabled else 0), "atomo_set_persistent_eig")
+    def set_persistent_eig(self, enabled):
+        """0 / False: one launch per Jacobi step; 1 / True: persistent cooperative launches; 2: clusters first (default)."""
+        self._check(self.lib.atomo_set_persistent_eig(self._h, int(enabled)), "atomo_set_persistent_eig")
 
     def set_gram_path(self, tensor_cores: bool):
         self._check(self.lib.atomo_set_gram_path(self._h, 1 if tensor_cores else 0), "atomo_set_gram_path")

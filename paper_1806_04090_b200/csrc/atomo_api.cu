@@ -1,5 +1,6 @@
 // C ABI of the library (see include/atomo.h): argument checks, payload layout, workspace
 // carving and kernel sequencing.  No arithmetic of the method lives here.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -28,7 +29,7 @@ struct atomo_ctx {
   int refine_min_short = 2048;       // layers with at least this short side get the sigma refinement pass
   bool tc_gram = true;               // Gram matrix on tcgen05 where the layer's layout allows it
   bool tc_ok = false;                // tensor-map entry point found
-  bool persistent_eig = true;        // whole eigen-solve in one cooperative launch when the batch fits the GPU
+  int eig_scheme = 2;                // eigen-solve launches: 0 = one per step, 1 = persistent (cooperative), 2 = clusters first
   std::string err;
 };
 
@@ -196,8 +197,8 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
 }
 
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
-  if (!ctx) return ATOMO_ERR_INVALID_ARG;
-  ctx->persistent_eig = enabled != 0;
+  if (!ctx || enabled < 0 || enabled > 2) return ATOMO_ERR_INVALID_ARG;
+  ctx->eig_scheme = enabled;
   return ATOMO_OK;
 }
 
@@ -303,6 +304,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_pairs = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
   uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
+  ClusterCta* d_ctas = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
   for (int pass = 0; pass < 2; ++pass) {
@@ -316,6 +318,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_tc = A.take<TileRef>(tc_tiles.size());
     d_maps = A.take<uint8_t>(maps_blob.size());
     d_flag = A.take<uint32_t>(4);
+    d_ctas = A.take<ClusterCta>((size_t)n_layers * sp_jacobi_cluster_ctas());   // at most one cluster per layer
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
@@ -404,11 +407,42 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
-  const int capacity = ctx->persistent_eig ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
+  // Cluster form first: every layer's block pairs inside one 16-CTA cluster, blocks exchanged through
+  // distributed shared memory (layers of up to 16 block pairs, route 1).
+  bool cluster_form = ctx->eig_scheme == 2 && ctx->eig_mode != 0;
+  for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
+  if (cluster_form && sp_jacobi_cluster_capacity(rp_max) < 1) cluster_form = false;
+  if (cluster_form) {
+    const int per = sp_jacobi_cluster_ctas();
+    std::vector<int> order(n_layers);
+    for (int l = 0; l < n_layers; ++l) order[l] = l;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].nb > L[b].nb; });
+    std::vector<int> used;                                 // slots taken in each cluster (first fit, largest first)
+    std::vector<ClusterCta> ctas;
+    for (int l : order) {
+      const int need_slots = L[l].nb / 2;
+      size_t c = 0;
+      while (c < used.size() && used[c] + need_slots > per) ++c;
+      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
+      for (int sl = 0; sl < need_slots; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], 0};
+      used[c] += need_slots;
+    }
+    CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
+    const int e = launch_sp_jacobi_cluster(d_layers, d_ctas, (int)used.size(), rp_max, max_sweeps, ctx->tol, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(jacobi clusters)");
+    launch_sp_check(d_layers, n_layers, steps_max * max_sweeps, max_sweeps, d_flag, st);
+    n_eig_launch = 2;
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+  }
+  const int capacity = (!cluster_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
   int max_layer_pairs = 0;
   for (int l = 0; l < n_layers; ++l) max_layer_pairs = std::max(max_layer_pairs, L[l].nb / 2);
   const bool persistent = capacity > 0 && max_layer_pairs <= capacity;
-  if (persistent) {
+  if (cluster_form) {
+    // done above
+  } else if (persistent) {
     // d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
     CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
     const int t_max = steps_max * max_sweeps;

@@ -37,12 +37,25 @@ __device__ __forceinline__ void rr_pair(int n, int round, int slot, int& p, int&
 // ((k + t) mod g/2 at step t); the next level treats each half as a group of its own.  Every pair of blocks
 // meets exactly once in nb/2 + nb/4 + ... + 1 = nb - 1 steps, and only half of the blocks move at a step.
 struct StepPlan { int bi, bj; bool first_in_level, last_in_level; };
+struct StepLevel { int lg, t; };                       // group size 2^lg, step t inside the level
+__device__ __forceinline__ StepLevel step_level(int nb, int local) {
+  int lg = 31 - __clz(nb), base = 0;
+  while (local - base >= (1 << (lg - 1))) { base += 1 << (lg - 1); --lg; }
+  return {lg, local - base};
+}
 __device__ __forceinline__ StepPlan step_plan(int nb, int local, int slot) {
-  int g = nb, base = 0;
-  while (local - base >= g / 2) { base += g / 2; g >>= 1; }
-  const int m = g / 2, t = local - base;
-  const int grp = slot / m, k = slot % m;
-  return {grp * g + k, grp * g + m + (k + t) % m, t == 0, t == m - 1};
+  const StepLevel lv = step_level(nb, local);
+  const int m = 1 << (lv.lg - 1);
+  const int grp = slot >> (lv.lg - 1), k = slot & (m - 1);
+  return {(grp << lv.lg) + k, (grp << lv.lg) + m + ((k + lv.t) & (m - 1)), lv.t == 0, lv.t == m - 1};
+}
+// the inverse: which CTA pairs block `blk` at step `local`, and as what (0 = resident, 1 = moving)
+__device__ __forceinline__ void find_holder(int nb, int local, int blk, int& slot, int& role) {
+  const StepLevel lv = step_level(nb, local);
+  const int m = 1 << (lv.lg - 1);
+  const int grp = blk >> lv.lg, pos = blk & ((1 << lv.lg) - 1);
+  role = pos >= m;
+  slot = grp * m + (role ? ((pos - m - lv.t) & (m - 1)) : pos);
 }
 
 // A is scaled to trace 1, so a squared row norm below this is an eigenvalue of A below 1e-12 (mode 0)
@@ -300,6 +313,7 @@ __device__ __forceinline__ void jacobi_block_pair(const SpLayer& L, int slot, in
 }
 
 constexpr int kJacobiThreads = 32 * kJB;
+constexpr int kJacobiThreadsC = kJacobiThreads;
 
 __device__ __forceinline__ void jacobi_dispatch(const SpLayer& L, int slot, int sweep, int local, bool resident, float tol,
                                                 float* smem) {
@@ -412,6 +426,225 @@ void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int 
   if (n_pairs <= 0) return;
   const int smem = 32 * std::min(row_floats_max, 1024) * 4 + 1024;
   sp_jacobi_step_kernel<<<n_pairs, kJacobiThreads, smem, st>>>(d_layers, d_pairs, t, max_sweeps, tol);
+}
+
+// =================================================================================================
+// Cluster form of the persistent eigen-solve, for layers of up to 16 block pairs (padded short side <= 512).
+// The CTAs of a layer sit in one thread-block cluster (16 CTAs; smaller layers share a cluster) and the blocks
+// never return to global memory between steps: at the end of a step a CTA writes its moving block (and, when a
+// level of the schedule ends, its resident block) straight into the shared memory of the CTA that pairs it
+// next -- distributed shared memory -- together with the rows' tracked norms, and a cluster barrier takes the
+// place of the global-memory barrier.  Four row regions per CTA: resident block x 2 and moving block x 2, so
+// that an incoming block never lands in a region that is still being rotated.  Norms are recomputed from
+// the rows at the start of every sweep.  A cluster ends when all its layers have converged (or hit the sweep
+// cap): every CTA announces the iteration in which it finished in every CTA's `done` table, and after barrier t
+// all CTAs take the same decision from the announcements made up to iteration t, so they leave together.  Rotation formulas, pairings and thresholds are those of the kernels above.
+// =================================================================================================
+constexpr int kClusterCtas = 16;
+
+template <int RP>
+struct ClusterRegion {
+  static constexpr int kRowFloats = kJB * RP;
+  static constexpr int kFloats = kRowFloats + 2 * kJB;            // rows, squared norms, factors
+  float* base;
+  __device__ __forceinline__ float* row(int i) const { return base + i * RP; }
+  __device__ __forceinline__ float* n2() const { return base + kRowFloats; }
+  __device__ __forceinline__ float* d() const { return base + kRowFloats + kJB; }
+};
+
+template <int RP>
+__device__ __forceinline__ void cluster_step(const SpLayer& L, const ClusterCta& me, int t, int& fpar, int& mpar,
+                                             int max_sweeps, float tol, float* smem, uint32_t* s_mask,
+                                             cg::cluster_group& cluster, bool& done) {
+  constexpr int B = kJB, V4 = RP / 4, T4 = (V4 + 31) / 32, NT = kJacobiThreadsC, R4 = RP / 4;
+  using Region = ClusterRegion<RP>;
+  const int tid = threadIdx.x, lane = tid % 32, pi = tid / 32;
+  const int steps = L.nb - 1;
+  const int sweep = t / steps, local = t % steps;
+  const StepPlan plan = step_plan(L.nb, local, me.slot);
+  Region F{smem + fpar * Region::kFloats}, M{smem + (2 + mpar) * Region::kFloats};
+  float* X = L.X;
+  RowSum<1> row_sum{nullptr, 0, 0, lane, 0};
+  if (t == 0) {                                                  // the only load from global memory
+    for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+      const int row = idx / R4, q = idx % R4;
+      const int grow = (row < B) ? plan.bi * B + row : plan.bj * B + (row - B);
+      float* dst = row < B ? F.row(row) : M.row(row - B);
+      reinterpret_cast<float4*>(dst)[q] = reinterpret_cast<const float4*>(X + (int64_t)grow * RP)[q];
+    }
+    __syncthreads();
+  }
+  const bool converged = local == 0 && sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) == 0;
+  if (converged || sweep >= max_sweeps) {                        // the blocks held now are those of step `local`
+    for (int idx = tid; idx < 2 * B * R4; idx += NT) {
+      const int row = idx / R4, q = idx % R4;
+      const int grow = (row < B) ? plan.bi * B + row : plan.bj * B + (row - B);
+      const float* src = row < B ? F.row(row) : M.row(row - B);
+      reinterpret_cast<float4*>(X + (int64_t)grow * RP)[q] = reinterpret_cast<const float4*>(src)[q];
+    }
+    done = true;
+    return;
+  }
+  RowRegs<T4> xp, xq;
+  if (local == 0) {                                              // sweep start: norms from the rows (factors are 1)
+    load_row<T4>(xq, M.row(pi), lane, V4);
+    const float nj = warp_sum(row_norm2_partial<T4>(xq, lane, V4));
+    load_row<T4>(xp, F.row(pi), lane, V4);
+    const float ni = warp_sum(row_norm2_partial<T4>(xp, lane, V4));
+    if (lane == 0) { F.n2()[pi] = ni; M.n2()[pi] = nj; }
+  }
+  if (lane == 0) { F.d()[pi] = 1.0f; M.d()[pi] = 1.0f; }
+  __syncthreads();
+  auto rowp_of = [&](int p) { return p < B ? F.row(p) : M.row(p - B); };
+  auto n2_of = [&](int p) -> float& { return p < B ? F.n2()[p] : M.n2()[p - B]; };
+  auto d_of = [&](int p) -> float& { return p < B ? F.d()[p] : M.d()[p - B]; };
+  uint32_t nrot = 0;
+  if (local == 0) {                                              // pairs inside each block: once per sweep
+    for (int round = 0; round < B - 1; ++round) {
+      const int blk = pi / (B / 2), sl = pi % (B / 2);
+      int p, q;
+      rr_pair(B, round, sl, p, q);
+      p += blk * B; q += blk * B;
+      float* rowp = rowp_of(p);
+      float* rowq = rowp_of(q);
+      load_row<T4>(xp, rowp, lane, V4);
+      load_row<T4>(xq, rowq, lane, V4);
+      float a2 = n2_of(p), b2 = n2_of(q), da = d_of(p), db = d_of(q);
+      const bool rot = rotate_pair<T4, 1>(xp, xq, a2, b2, da, db, lane, V4, tol, row_sum, [&] {
+        store_row<T4>(xp, rowp, lane, V4);
+        store_row<T4>(xq, rowq, lane, V4);
+      });
+      if (rot) {
+        if (lane == 0) { n2_of(p) = a2; n2_of(q) = b2; d_of(p) = da; d_of(q) = db; }
+        ++nrot;
+      }
+      __syncthreads();
+    }
+  }
+  // Late sweeps rotate little: when the finished sweep averaged fewer than 8 rotations per CTA and step, look at
+  // all 16 x 16 cosines first (each warp: 2 resident rows against 8 moving rows, no barrier, nothing written)
+  // and run only the rounds that hold a pair above tol.  (A rotation changes the other cosines of its two rows
+  // only to second order; whatever that lifts above tol is met again in the next sweep, which then takes place
+  // because this one rotated.)  Factors are 1 here, so the stored rows are the true rows.
+  uint32_t round_mask = 0xffffu;
+  if (local != 0 && sweep > 0 && *(volatile uint32_t*)(L.rot_count + sweep - 1) < (uint32_t)(8 * steps * (L.nb / 2))) {
+    const int a = pi >> 1, half = pi & 1;
+    RowRegs<T4> x0, x1;
+    load_row<T4>(x0, F.row(2 * a), lane, V4);
+    load_row<T4>(x1, F.row(2 * a + 1), lane, V4);
+    const float r0 = rsqrt_approx(F.n2()[2 * a]), r1 = rsqrt_approx(F.n2()[2 * a + 1]);
+    const bool ok0 = F.n2()[2 * a] >= kRowFloor, ok1 = F.n2()[2 * a + 1] >= kRowFloor;
+    uint32_t need = 0;
+#pragma unroll 2
+    for (int jj = 0; jj < B / 2; ++jj) {
+      const int j = half * (B / 2) + jj;
+      load_row<T4>(xq, M.row(j), lane, V4);
+      float g0 = 0.f, g1 = 0.f;
+#pragma unroll
+      for (int u = 0; u < T4; ++u) {
+        if (lane + 32 * u < V4) {
+          const float4 q4 = xq.v[u], p0 = x0.v[u], p1 = x1.v[u];
+          g0 = fmaf(p0.x, q4.x, fmaf(p0.y, q4.y, fmaf(p0.z, q4.z, fmaf(p0.w, q4.w, g0))));
+          g1 = fmaf(p1.x, q4.x, fmaf(p1.y, q4.y, fmaf(p1.z, q4.z, fmaf(p1.w, q4.w, g1))));
+        }
+      }
+      const float nq = M.n2()[j];
+      const float rq = rsqrt_approx(nq) * 536870912.0f;          // 2^29: the same fixed-point cosine as rotate_pair
+      const int c0 = __reduce_add_sync(0xffffffffu, __float2int_rn(g0 * (r0 * rq)));
+      const int c1 = __reduce_add_sync(0xffffffffu, __float2int_rn(g1 * (r1 * rq)));
+      const float lim = tol * 536870912.0f;
+      const bool okq = nq >= kRowFloor;
+      // row i of the resident block meets row j of the moving block in round (j - i) mod 16
+      if (okq && ok0 && !(fabsf((float)c0) <= lim)) need |= 1u << ((j - 2 * a) & (B - 1));
+      if (okq && ok1 && !(fabsf((float)c1) <= lim)) need |= 1u << ((j - 2 * a - 1) & (B - 1));
+    }
+    if (lane == 0 && need) atomicOr(s_mask, need);
+    __syncthreads();
+    round_mask = *s_mask;
+    __syncthreads();
+    if (tid == 0) *s_mask = 0;                                     // for the next step (ordered by the barriers below)
+  }
+  load_row<T4>(xp, F.row(pi), lane, V4);
+  float np2 = F.n2()[pi], dp = F.d()[pi];
+  for (int round = 0; round < B; ++round) {                      // pairs across the two blocks
+    if (!((round_mask >> round) & 1u)) continue;
+    const int j = (pi + round) % B;
+    float* rowq = M.row(j);
+    load_row<T4>(xq, rowq, lane, V4);
+    float nq2 = M.n2()[j], dq = M.d()[j];
+    const bool rot = rotate_pair<T4, 1>(xp, xq, np2, nq2, dp, dq, lane, V4, tol, row_sum,
+                                        [&] { store_row<T4>(xq, rowq, lane, V4); });
+    if (rot) {
+      if (lane == 0) { M.n2()[j] = nq2; M.d()[j] = dq; }
+      ++nrot;
+    }
+    __syncthreads();
+  }
+  store_row<T4>(xp, F.row(pi), lane, V4, dp);
+  if (lane == 0) { F.d()[pi] = 1.0f; F.n2()[pi] = np2; }
+  if (lane == 0 && nrot) atomicAdd(L.rot_count + sweep, nrot);
+  __syncthreads();
+  // ---- hand the blocks to the CTAs that pair them at the next step ----
+  const int next_local = (local + 1) % steps;
+  for (int which = 0; which < 2; ++which) {                      // 0: moving block, 1: resident block (level end only)
+    if (which == 1 && !plan.last_in_level) break;
+    const int blk = which == 0 ? plan.bj : plan.bi;
+    int slot, role;
+    find_holder(L.nb, next_local, blk, slot, role);
+    const Region src = which == 0 ? M : F;
+    const int dst_region = role == 0 ? (fpar ^ 1) : 2 + (mpar ^ 1);
+    float* dst_local = smem + dst_region * Region::kFloats;
+    float* dst = cluster.map_shared_rank(dst_local, me.base_rank + slot);
+    for (int idx = tid; idx < B * R4; idx += NT) {
+      const int row = idx / R4, q = idx % R4;
+      const float dv = src.d()[row];
+      const float4 a = reinterpret_cast<const float4*>(src.row(row))[q];
+      reinterpret_cast<float4*>(dst + row * RP)[q] = make_float4(a.x * dv, a.y * dv, a.z * dv, a.w * dv);
+    }
+    if (tid < B) dst[Region::kRowFloats + tid] = src.n2()[tid];
+  }
+  mpar ^= 1;
+  if (plan.last_in_level) fpar ^= 1;
+}
+
+__global__ void __launch_bounds__(kJacobiThreadsC) sp_jacobi_cluster_kernel(const SpLayer* __restrict__ layers,
+                                                                            const ClusterCta* __restrict__ ctas,
+                                                                            int max_sweeps, float tol) {
+  extern __shared__ __align__(16) float smem[];
+  __shared__ int s_done[kClusterCtas];
+  __shared__ uint32_t s_mask;                            // rounds of the current step that hold a pair to rotate
+  cg::cluster_group cluster = cg::this_cluster();
+  const ClusterCta me = ctas[blockIdx.x];
+  const int my_rank = (int)cluster.block_rank();
+  // s_done[r] = the iteration in which CTA r finished (a CTA may already be writing the next iteration's
+  // announcement while another still reads the table: comparing with the iteration number makes the
+  // decision after barrier t depend only on announcements made before barrier t)
+  if (threadIdx.x < kClusterCtas) s_done[threadIdx.x] = 0x7fffffff;
+  if (threadIdx.x == 0) s_mask = 0;
+  bool done = me.layer < 0, announced = false;
+  int fpar = 0, mpar = 0;
+  cluster.sync();
+  for (int t = 0;; ++t) {
+    if (!done) {
+      const SpLayer& L = layers[me.layer];
+      switch (L.rp) {
+        case 32: cluster_step<32>(L, me, t, fpar, mpar, max_sweeps, tol, smem, &s_mask, cluster, done); break;
+        case 64: cluster_step<64>(L, me, t, fpar, mpar, max_sweeps, tol, smem, &s_mask, cluster, done); break;
+        case 128: cluster_step<128>(L, me, t, fpar, mpar, max_sweeps, tol, smem, &s_mask, cluster, done); break;
+        case 256: cluster_step<256>(L, me, t, fpar, mpar, max_sweeps, tol, smem, &s_mask, cluster, done); break;
+        case 512: cluster_step<512>(L, me, t, fpar, mpar, max_sweeps, tol, smem, &s_mask, cluster, done); break;
+        default: done = true; break;
+      }
+    }
+    if (done && !announced) {
+      if (threadIdx.x < kClusterCtas) cluster.map_shared_rank(s_done, threadIdx.x)[my_rank] = t;
+      announced = true;
+    }
+    cluster.sync();
+    int pending = 0;
+    if (threadIdx.x < kClusterCtas) pending = *(volatile int*)(s_done + threadIdx.x) > t;
+    if (!__syncthreads_or(pending)) break;
+  }
 }
 
 // convergence bookkeeping after t_done steps have been enqueued
@@ -685,10 +918,46 @@ int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n
 
 int sp_cholesky_big_rows_per_cta() { return kCholBigThreads; }
 
+// ---- cluster form: host side ----
+static int cluster_smem_bytes(int rp_max) { return 4 * (kJB * rp_max + 2 * kJB) * (int)sizeof(float); }
+int sp_jacobi_cluster_ctas() { return kClusterCtas; }
+int sp_jacobi_cluster_max_rp() { return 512; }
+
+// how many clusters of 16 such CTAs the GPU can hold at once (0: this form cannot run here)
+int sp_jacobi_cluster_capacity(int rp_max) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kClusterCtas); cfg.blockDim = dim3(kJacobiThreads); cfg.dynamicSmemBytes = cluster_smem_bytes(rp_max);
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kClusterCtas; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, sp_jacobi_cluster_kernel, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n;
+}
+
+int launch_sp_jacobi_cluster(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, int max_sweeps,
+                             float tol, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_clusters * kClusterCtas); cfg.blockDim = dim3(kJacobiThreads);
+  cfg.dynamicSmemBytes = cluster_smem_bytes(rp_max); cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = kClusterCtas; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, sp_jacobi_cluster_kernel, d_layers, d_ctas, max_sweeps, tol);
+}
+
 int sp_configure_eig() {
   cudaError_t e = cudaFuncSetAttribute(sp_jacobi_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
   if (e != cudaSuccess) return (int)e;
-  return (int)cudaFuncSetAttribute(sp_jacobi_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  e = cudaFuncSetAttribute(sp_jacobi_persistent_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kJacobiSmem);
+  if (e != cudaSuccess) return (int)e;
+  // the cluster form is optional: a GPU that refuses 16-CTA clusters simply reports a capacity of 0
+  if (cudaFuncSetAttribute(sp_jacobi_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, cluster_smem_bytes(512)) != cudaSuccess ||
+      cudaFuncSetAttribute(sp_jacobi_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+    cudaGetLastError();
+  return 0;
 }
 
 }  // namespace atomo

@@ -106,6 +106,13 @@ int sp_jacobi_persistent_capacity(int row_floats_max);
 int launch_sp_jacobi_persistent(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                                 int max_sweeps, float tol, uint32_t* d_state, cudaStream_t st);
 // layers of up to 1024 rows: clusters of 8 CTAs; more rows: cooperative launch.  Both return a cudaError_t
+// cluster form of the persistent eigen-solve (layers of up to 16 block pairs); one entry per CTA of a cluster
+struct ClusterCta { int32_t layer, slot, base_rank, pad; };       // layer < 0: this CTA only keeps the barriers
+int sp_jacobi_cluster_ctas();                                     // CTAs per cluster
+int sp_jacobi_cluster_max_rp();                                   // largest padded short side it takes
+int sp_jacobi_cluster_capacity(int rp_max);                       // co-resident clusters (0: not available here)
+int launch_sp_jacobi_cluster(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, int max_sweeps,
+                             float tol, cudaStream_t st);         // returns a cudaError_t
 int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
 int sp_cholesky_big_rows_per_cta();

@@ -110,6 +110,29 @@ def test_paper_reshape_family(atomo, oracle):
     _run(atomo, oracle, mats, 2.0, seed=17, step=1)
 
 
+def test_eigen_launch_schemes_agree(atomo):
+    """One launch per step, persistent cooperative launches and the cluster form run the same rotations in the same
+    order per layer: identical masks and singular values to rounding (the forms fold the row factors at different
+    moments, so the bits may differ)."""
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(1, [L[0], L[1], L[5], L[9], L[13], L[17]])
+    got = []
+    try:
+        for scheme in (0, 1, 2):
+            atomo.set_persistent_eig(scheme)
+            pay, dbg = _encode(atomo, mats, 2.0, seed=23, step=2)
+            hdrs = pay.headers()[1]
+            assert [h.status for h in hdrs] == [0] * len(mats)
+            got.append(([dbg.layer_sigma(l, min(m.shape)) for l, m in enumerate(mats)],
+                        [pay.layer_arrays(l)["idx"].copy() for l in range(len(mats))]))
+    finally:
+        atomo.set_persistent_eig(2)
+    for other in got[1:]:
+        for l in range(len(mats)):
+            assert parity.rel(other[0][l], got[0][0][l]) <= 2e-6
+            assert np.array_equal(other[1][l], got[0][1][l])
+
+
 def test_leading_dimension(atomo, oracle):
     rng = np.random.default_rng(7)
     mats = [synth.lowrank_plus_noise(rng, 48, 200, 1.0, noise_rel=0.02),
