@@ -27,9 +27,9 @@ METRIC = "gradient elements encoded+decoded/sec"
 UNIT = "elements/s"
 L2_BYTES = 126 * 1024 * 1024
 FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # SMs x FP32 lanes x 2 flop x max SM clock
-# dram__bytes_read.sum + dram__bytes_write.sum of one sp_jacobi_persistent_kernel launch on this workload, from the
-# ncu capture summarised in profiles/sp_jacobi_persistent_c2.txt (5.70 MB read + 0.33 MB written)
-JACOBI_TRAFFIC_BYTES_PER_LAUNCH = 6032896
+# dram__bytes_read.sum + dram__bytes_write.sum of one sp_jacobi_cluster_kernel launch on this workload, from the
+# ncu capture summarised in profiles/sp_jacobi_cluster_c2.txt (5.66 MB read, nothing written back to DRAM)
+JACOBI_TRAFFIC_BYTES_PER_LAUNCH = 5660672
 
 
 def measured_peaks():
@@ -271,6 +271,7 @@ def run_ours(args):
     eig_ms = eig_launches = 0.0
     launches = 0
     sweeps_seen = None
+    eig_scheme = -1
     ev0.record()
     for k in range(args.steps):
         pay, _ = a.atomo_encode_spectral(dev_sets[(args.warmup + k) % n_sets], s, seed + rank, step=args.warmup + k,
@@ -282,6 +283,7 @@ def run_ours(args):
         launches += 3
         if k == args.steps - 1:
             sweeps_seen = [h.sweeps for h in pay.headers()[1]]
+            eig_scheme = a.last_eig_scheme()
     ev1.record()
     torch.cuda.synchronize(); dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
@@ -374,10 +376,10 @@ def run_ours(args):
                     "overlap": "copies of step k+1 (in) and k-1 (out) run on two copy streams under step k's kernels"},
             "gpu_launches": int(launches),
             "roofline": {"bound": "alu",
-                         "kernel": "sp_jacobi_persistent_kernel" if launches_per_step <= 2 else "sp_jacobi_step_kernel",
+                         "kernel": {2: "sp_jacobi_cluster_kernel", 1: "sp_jacobi_persistent_kernel"}.get(eig_scheme, "sp_jacobi_step_kernel"),
                          "achieved": achieved,
                          "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_FMA_PEAK_TFLOPS,
-                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH if launches_per_step <= 2 else None,
+                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH if eig_scheme == 2 else None,
                          "launches_per_step": 1.0 if launches_per_step <= 2 else launches_per_step,
                          "avg_launch_us": eig_s_per_step / (1.0 if launches_per_step <= 2 else launches_per_step) * 1e6,
                          "share_of_step": eig_ms / ms_total,

@@ -238,6 +238,9 @@ int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
  * 0 = one launch per step and one host wait per sweep.
  * Schemes 1 and 2 wait on the host once, at the end of the solve.                                            */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
+/* The scheme (0, 1 or 2 as above) that the last atomo_encode_spectral() of this context actually ran; -1 before
+ * the first call.  Host only.                                                                                */
+int atomo_last_eig_scheme(atomo_ctx* ctx);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,7 @@ EXPORTS = [
     "atomo_create", "atomo_destroy", "atomo_last_cuda_error", "atomo_payload_bytes_spectral",
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
-    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
+    "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
 ]
 
 
@@ -106,6 +106,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_sigma_refinement.argtypes = [vp, i32]
     lib.atomo_set_gram_path.argtypes = [vp, i32]
     lib.atomo_set_persistent_eig.argtypes = [vp, i32]
+    lib.atomo_last_eig_scheme.argtypes = [vp]
     lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                  ctypes.POINTER(vp), i32, vp]
     if path == LIB_PATH:
@@ -427,6 +428,9 @@ class Atomo:
     def set_persistent_eig(self, enabled):
         """0 / False: one launch per Jacobi step; 1 / True: persistent cooperative launches; 2: clusters first (default)."""
         self._check(self.lib.atomo_set_persistent_eig(self._h, int(enabled)), "atomo_set_persistent_eig")
+
+    def last_eig_scheme(self) -> int:
+        return int(self.lib.atomo_last_eig_scheme(self._h))
 
     def set_gram_path(self, tensor_cores: bool):
         self._check(self.lib.atomo_set_gram_path(self._h, 1 if tensor_cores else 0), "atomo_set_gram_path")

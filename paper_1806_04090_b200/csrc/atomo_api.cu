@@ -30,6 +30,8 @@ struct atomo_ctx {
   bool tc_gram = true;               // Gram matrix on tcgen05 where the layer's layout allows it
   bool tc_ok = false;                // tensor-map entry point found
   int eig_scheme = 2;                // eigen-solve launches: 0 = one per step, 1 = persistent (cooperative), 2 = clusters first
+  int eig_scheme_used = -1;          // what the last spectral encode actually ran
+  int cluster_capacity[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // by log2(rp_max), -1 = not asked yet
   std::string err;
 };
 
@@ -195,6 +197,8 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
   ctx->tol = tol;
   return ATOMO_OK;
 }
+
+int atomo_last_eig_scheme(atomo_ctx* ctx) { return ctx ? ctx->eig_scheme_used : -1; }
 
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
   if (!ctx || enabled < 0 || enabled > 2) return ATOMO_ERR_INVALID_ARG;
@@ -411,7 +415,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // distributed shared memory (layers of up to 16 block pairs, route 1).
   bool cluster_form = ctx->eig_scheme == 2 && ctx->eig_mode != 0;
   for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
-  if (cluster_form && sp_jacobi_cluster_capacity(rp_max) < 1) cluster_form = false;
+  if (cluster_form) {
+    int lg = 0;
+    while ((1 << lg) < rp_max) ++lg;
+    if (ctx->cluster_capacity[lg] < 0) ctx->cluster_capacity[lg] = sp_jacobi_cluster_capacity(rp_max);
+    if (ctx->cluster_capacity[lg] < 1) cluster_form = false;
+  }
   if (cluster_form) {
     const int per = sp_jacobi_cluster_ctas();
     std::vector<int> order(n_layers);
@@ -440,6 +449,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   int max_layer_pairs = 0;
   for (int l = 0; l < n_layers; ++l) max_layer_pairs = std::max(max_layer_pairs, L[l].nb / 2);
   const bool persistent = capacity > 0 && max_layer_pairs <= capacity;
+  ctx->eig_scheme_used = cluster_form ? 2 : (persistent ? 1 : 0);
   if (cluster_form) {
     // done above
   } else if (persistent) {
