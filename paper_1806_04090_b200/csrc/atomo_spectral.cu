@@ -286,28 +286,50 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   // eigenvalue of A per row, one warp per row.  mode 0: lambda_i = <x_i, v_i> (Rayleigh quotient at v_i);
   // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T).  With refinement: the sum of the tiles' partial
   // squared norms of the projection (already in the units of G).
-  for (int i = w; i < r; i += kFinThreads / 32) {
-    float lam;
+  // (without refinement: four rows of a warp at a time, so that their loads are in flight together)
+  constexpr int kRowsAtOnce = 4, kFinWarps = kFinThreads / 32;
+  for (int i0 = w; i0 < r; i0 += kFinWarps * kRowsAtOnce) {
+    float lam[kRowsAtOnce];
     if (L.refine) {
-      double d = 0.0;
-      for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
-      lam = (float)warp_sum(d);
+#pragma unroll
+      for (int u = 0; u < kRowsAtOnce; ++u) {
+        const int i = i0 + u * kFinWarps;
+        double d = 0.0;
+        if (i < r)
+          for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
+        lam[u] = (float)warp_sum(d);
+      }
     } else {
       // rows are zero-padded to rp floats (a multiple of 32): whole float4, several loads in flight
-      const float4* x4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx);
-      const float4* v4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx + voff);
-      float d0 = 0.f, d1 = 0.f;
-#pragma unroll 4
+      float d0[kRowsAtOnce], d1[kRowsAtOnce];
+#pragma unroll
+      for (int u = 0; u < kRowsAtOnce; ++u) { d0[u] = 0.f; d1[u] = 0.f; }
       for (int j = lane; j < rp / 4; j += 32) {
-        const float4 a = x4[j], b = v4[j];
-        d0 = fmaf(a.x, b.x, fmaf(a.y, b.y, d0));
-        d1 = fmaf(a.z, b.z, fmaf(a.w, b.w, d1));
+        float4 a[kRowsAtOnce], b[kRowsAtOnce];
+#pragma unroll
+        for (int u = 0; u < kRowsAtOnce; ++u) {
+          const int i = min(i0 + u * kFinWarps, r - 1);
+          a[u] = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx)[j];
+          b[u] = voff ? reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx + voff)[j] : a[u];
+        }
+#pragma unroll
+        for (int u = 0; u < kRowsAtOnce; ++u) {
+          d0[u] = fmaf(a[u].x, b[u].x, fmaf(a[u].y, b[u].y, d0[u]));
+          d1[u] = fmaf(a[u].z, b[u].z, fmaf(a[u].w, b[u].w, d1[u]));
+        }
       }
-      lam = warp_sum(d0 + d1) * inv_scale;
+#pragma unroll
+      for (int u = 0; u < kRowsAtOnce; ++u) lam[u] = warp_sum(d0[u] + d1[u]) * inv_scale;
     }
     if (lane == 0) {
-      if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
-      s_lam[i] = fmaxf(lam, 0.0f);
+#pragma unroll
+      for (int u = 0; u < kRowsAtOnce; ++u) {
+        const int i = i0 + u * kFinWarps;
+        if (i < r) {
+          if (!(fabsf(lam[u]) <= 3.0e38f)) atomicOr(&s_bad, 1u);
+          s_lam[i] = fmaxf(lam[u], 0.0f);
+        }
+      }
     }
   }
   __syncthreads();
@@ -515,31 +537,43 @@ void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int 
 
 // w_a = sum over row chunks (in chunk order), sigma_a = ||w_a||, coef_a = sigma_a / p_a, long vector = w_a / sigma_a.
 // One CTA per (layer, kept-atom slot); slots beyond the layer's k leave at once.
-__global__ void __launch_bounds__(256) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers, int k_cap_max) {
+constexpr int kFinishThreads = 1024;
+__global__ void __launch_bounds__(kFinishThreads) sp_finish_atoms_kernel(const SpLayer* __restrict__ layers, int k_cap_max) {
   const SpLayer& L = layers[blockIdx.x / k_cap_max];
   const uint32_t a = blockIdx.x % k_cap_max;
   if (a >= L.hdr->k) return;
-  const int len = L.L;
-  __shared__ double s_red[256];
+  const int len = L.L, chunks = L.bp_chunks;
+  __shared__ double s_red[kFinishThreads / 32];
+  __shared__ float s_sg;
   double part = 0.0;
   float* out = L.longv + (int64_t)a * len;
-  for (int j = threadIdx.x; j < len; j += 256) {
+  const float* in = L.bp_part + (int64_t)a * len;
+  const int64_t chunk_stride = (int64_t)L.k_cap * len;
+  for (int j = threadIdx.x; j < len; j += kFinishThreads) {
     float wv = 0.f;
-    for (int ch = 0; ch < L.bp_chunks; ++ch) wv += L.bp_part[((int64_t)ch * L.k_cap + a) * len + j];
+#pragma unroll 8
+    for (int ch = 0; ch < chunks; ++ch) wv += in[ch * chunk_stride + j];
     out[j] = wv;
     part += (double)wv * (double)wv;
   }
-  s_red[threadIdx.x] = part;
+  part = warp_sum(part);
+  if (threadIdx.x % 32 == 0) s_red[threadIdx.x / 32] = part;
   __syncthreads();
-  for (int o = 128; o > 0; o >>= 1) { if (threadIdx.x < o) s_red[threadIdx.x] += s_red[threadIdx.x + o]; __syncthreads(); }
-  const float sg = (float)sqrt(s_red[0]);
-  if (threadIdx.x == 0) L.coef[a] = sg / L.p_sel[a];
+  if (threadIdx.x == 0) {
+    double t = 0.0;
+    for (int i = 0; i < kFinishThreads / 32; ++i) t += s_red[i];            // fixed order
+    const float sg = (float)sqrt(t);
+    L.coef[a] = sg / L.p_sel[a];
+    s_sg = sg;
+  }
+  __syncthreads();
+  const float sg = s_sg;
   const float inv = sg > 0.f ? 1.0f / sg : 0.f;
-  for (int j = threadIdx.x; j < len; j += 256) out[j] *= inv;       // each thread rescales what it wrote itself
+  for (int j = threadIdx.x; j < len; j += kFinishThreads) out[j] *= inv;   // each thread rescales what it wrote itself
 }
 
 void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, int k_cap_max, cudaStream_t st) {
-  sp_finish_atoms_kernel<<<n_layers * k_cap_max, 256, 0, st>>>(d_layers, k_cap_max);
+  sp_finish_atoms_kernel<<<n_layers * k_cap_max, kFinishThreads, 0, st>>>(d_layers, k_cap_max);
 }
 
 // =================================================================================================
