@@ -256,6 +256,45 @@ def test_config5_shape_properties(atomo):
             assert all(h.n_sat >= 1 for h in hdrs[1])          # sum(sigma) ~ 7.5 < 8 sigma_1
 
 
+def test_config5_full_size(atomo):
+    """Config 5 at its full size (96 layers of 1024 x 4096, 402,653,184 elements): more block pairs than the GPU
+    holds CTAs, so the eigen-solve runs as a sequence of persistent launches over groups of layers.  Six distinct
+    seeded matrices, each used 16 times (generating 96 Haar factors of order 4096 would take minutes on the host);
+    every copy is its own layer with its own Philox stream.  Checked: status, singular values against a library SVD
+    in fp64, sum(p) = s, kept atoms as singular triplets on sampled layers, the decode against its definition."""
+    import torch
+    base = synth.c5_stress(0, count=6)
+    refs = [np.linalg.svd(G.astype(np.float64), compute_uv=False) for G in base]
+    dev = torch.device("cuda:0")
+    ts = [torch.from_numpy(base[i % 6]).to(dev).clone() for i in range(96)]
+    s = 4.0
+    pay, dbg = atomo.atomo_encode_spectral(ts, s, seed=91, step=5, k_cap=48, debug=True)
+    assert atomo.last_eig_scheme() == 1
+    hdrs = pay.headers()
+    assert [h.status for h in hdrs[1]] == [0] * 96
+    outs = atomo.atomo_decode(pay)
+    ks = [h.k for h in hdrs[1]]
+    assert len(set(ks)) > 1                                   # the copies draw from different Philox streams
+    for l in range(96):
+        sig = dbg.layer_sigma(l, 1024)
+        assert parity.rel(sig, refs[l % 6]) <= parity.REL_TOL
+        p = dbg.layer_prob(l, 1024)
+        assert abs(p.sum() - s) <= 1e-4 * s
+    for l in (0, 17, 40, 63, 95):                             # kept atoms of a few layers, in fp64
+        G64 = base[l % 6].astype(np.float64)
+        ref = refs[l % 6]
+        arr = pay.layer_arrays(l, hdrs)
+        p = dbg.layer_prob(l, 1024)
+        for j in range(arr["k"]):
+            u = arr["U"][:, j].astype(np.float64); v = arr["V"][:, j].astype(np.float64)
+            sg = float(arr["coef"][j]) * float(p[arr["idx"][j]])
+            assert np.linalg.norm(G64.T @ u - sg * v) <= 2e-5 * ref[0]
+            assert np.linalg.norm(G64 @ v - sg * u) <= max(2e-5 * ref[0], parity.RESID_GRAM * ref[0] ** 2 / sg)
+        own = (arr["U"].astype(np.float64) * arr["coef"].astype(np.float64)) @ arr["V"].astype(np.float64).T
+        out = outs[l].cpu().numpy()
+        assert (parity.rel(out, own) <= 1e-5) if arr["k"] else (not out.any())
+
+
 def test_eigen_routes_agree(atomo, oracle):
     # route 0 (Jacobi on [A | I] with accumulated vectors) is an independent check of route 1
     # (Cholesky factor, Jacobi on its rows): same singular values, probabilities and masks
