@@ -178,10 +178,10 @@ int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloa
  * memory: a process whose framework allocator already owns the whole GPU, a latency-critical
  * section that cannot take cudaMalloc's device-wide synchronisation, a memory-capped job.  It needs
  * no context and calls no cudaMalloc / cudaFree: the per-call tables (one descriptor per layer, one
- * entry per 32 x 256 output tile) go into a fixed array inside the library image, about 130 KB that
+ * entry per 64 x 1024 output tile) go into a fixed array inside the library image, about 130 KB that
  * every GPU loading the library holds until the process exits.
  *   - Limits: n_layers <= ATOMO_STATIC_MAX_LAYERS and at most ATOMO_STATIC_MAX_TILES output tiles in
- *     all (sum over layers of ceil(rows/32) * ceil(cols/256)); beyond that ATOMO_ERR_CAPACITY is
+ *     all (sum over layers of ceil(rows/64) * ceil(cols/1024)); beyond that ATOMO_ERR_CAPACITY is
  *     returned and nothing is launched.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device made current); make that first call before any stream capture begins.

@@ -15,7 +15,7 @@
 //                      compaction of the kept ranks, short-side vectors of the kept atoms
 //   sp_backproject     long-side vector of each kept atom, w_i = G^T u_i (or G v_i)
 //   sp_finish_atoms    sigma_i = ||w_i||, coef_i = sigma_i / p_i, w_i normalised
-//   sp_decode          G_hat = sum_k coef_k u_k v_k^T, one coalesced write pass
+//   sp_decode          G_hat = sum_k coef_k u_k v_k^T, one streaming write pass (8 atoms per pass)
 #include "atomo_kernels.cuh"
 
 namespace atomo {
@@ -577,80 +577,120 @@ void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, int k_cap_max
 }
 
 // =================================================================================================
-// decode: out[i][c] = sum_a coef_a rowvec_a[i] colvec_a[c].  Tile 32 rows x 256 columns,
-// 256 threads: thread = (row group of 8) x (4 consecutive columns... x 2).
+// decode: out[i][c] = sum_a coef_a rowvec_a[i] colvec_a[c], a streaming write of the output.
+// Tile 64 rows x 1024 columns, 256 threads: a thread owns 4 consecutive columns, keeps the column-vector
+// entries of up to 8 atoms in registers and walks down the 64 rows, one 16-byte store per row; the row-vector
+// entries (times coef) of the tile sit in shared memory and are read as broadcasts.  k is about s, a handful:
+// a layer with more than 8 kept atoms takes further passes that add to what the first one wrote.
 // =================================================================================================
-constexpr int kDecRows = 32, kDecCols = 256, kDecAtoms = 16;
+constexpr int kDecRows = 64, kDecCols = 1024, kDecAtoms = 8, kDecThreads = 256;
 int sp_decode_tile_rows() { return kDecRows; }
 int sp_decode_tile_cols() { return kDecCols; }
 
-__global__ void __launch_bounds__(256) sp_decode_kernel(const uint8_t* __restrict__ payload,
-                                                        const SpDecodeLayer* __restrict__ layers,
-                                                        const TileRef* __restrict__ tiles) {
-  __shared__ __align__(16) float s_col[kDecAtoms][kDecCols];
-  __shared__ float s_row[kDecAtoms][kDecRows];
-  const atomo_payload_header* gh = reinterpret_cast<const atomo_payload_header*>(payload);
+// `single` (one payload) or `list[0 .. n_payloads)`: the kept atoms of all payloads are walked as one sequence,
+// payload after payload, 8 per pass; `scale` multiplies every term (1, or 1 / n_payloads for the average).
+__global__ void __launch_bounds__(kDecThreads) sp_decode_kernel(const uint8_t* __restrict__ single,
+                                                                const uint8_t* const* __restrict__ list, int n_payloads,
+                                                                float scale, const SpDecodeLayer* __restrict__ layers,
+                                                                const TileRef* __restrict__ tiles) {
+  __shared__ __align__(16) float s_rc[kDecRows][kDecAtoms];      // scale * coef_a * rowvec_a[i] of the tile's rows
   const TileRef ref = tiles[blockIdx.x];
   const SpDecodeLayer D = layers[ref.layer];
-  const atomo_layer_header* h = D.hdr;
   const int64_t rows = D.rows, cols = D.cols;
-  const bool ok = gh->magic == ATOMO_MAGIC && gh->kind == ATOMO_KIND_SPECTRAL && h->rows == rows && h->cols == cols &&
-                  h->k <= h->k_cap;
-  if (!ok && ref.a == 0 && ref.b == 0 && threadIdx.x == 0) raise_status(const_cast<atomo_layer_header*>(h), ATOMO_ERR_PAYLOAD);
-  const uint32_t k = ok ? h->k : 0u;
   const bool tall = rows > cols;
   const int64_t r = tall ? cols : rows, len = tall ? rows : cols;
-  const float* coef = reinterpret_cast<const float*>(payload + h->off_val);
-  const float* shortv = reinterpret_cast<const float*>(payload + h->off_short);
-  const float* longv = reinterpret_cast<const float*>(payload + h->off_long);
-  const float* rowvec = tall ? longv : shortv;   // indexed by output row
-  const float* colvec = tall ? shortv : longv;   // indexed by output column
-  const int64_t rlen = tall ? len : r, clen = tall ? r : len;
-  const int64_t i0 = (int64_t)ref.a * kDecRows, c0 = (int64_t)ref.b * kDecCols;
-  const int tid = threadIdx.x;
-  const int cg = tid % 64, rg = tid / 64;            // 64 column groups of 4, 4 row groups of 8
-  float acc[8][4];
-#pragma unroll
-  for (int i = 0; i < 8; ++i)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-  for (uint32_t a0 = 0; a0 < k; a0 += kDecAtoms) {
-    const int na = min((uint32_t)kDecAtoms, k - a0);
-    __syncthreads();
-    for (int idx = tid; idx < na * kDecCols; idx += 256) {
-      const int a = idx / kDecCols, c = idx % kDecCols;
-      s_col[a][c] = (c0 + c < clen) ? __ldg(colvec + (int64_t)(a0 + a) * clen + c0 + c) : 0.f;
+  const int64_t rlen = tall ? len : r, clen = tall ? r : len;     // lengths of the row- and column-indexed vectors
+  const int64_t i0 = (int64_t)ref.a * kDecRows, c = (int64_t)ref.b * kDecCols + 4 * threadIdx.x;
+  const int n_rows = (int)min((int64_t)kDecRows, rows - i0);
+  const bool vec_out = (cols % 4 == 0) && ((reinterpret_cast<uintptr_t>(D.out) & 15u) == 0);
+  float* out = D.out + i0 * cols + c;
+  int p = 0;                                                     // cursor over (payload, atom)
+  uint32_t a_next = 0;
+  bool first_pass = true;
+  for (;;) {
+    // up to 8 atoms for this pass
+    const float* rowv[kDecAtoms]; const float* colv[kDecAtoms]; float cf[kDecAtoms];
+    int na = 0;
+    while (na < kDecAtoms && p < n_payloads) {
+      const uint8_t* payload = list ? list[p] : single;
+      const atomo_payload_header* gh = reinterpret_cast<const atomo_payload_header*>(payload);
+      const atomo_layer_header* h = reinterpret_cast<const atomo_layer_header*>(payload + sizeof(atomo_payload_header)) + ref.layer;
+      const bool ok = gh->magic == ATOMO_MAGIC && gh->kind == ATOMO_KIND_SPECTRAL && h->rows == rows && h->cols == cols &&
+                      h->k <= h->k_cap;
+      if (!ok && a_next == 0 && ref.a == 0 && ref.b == 0 && threadIdx.x == 0)
+        raise_status(const_cast<atomo_layer_header*>(h), ATOMO_ERR_PAYLOAD);
+      const uint32_t k = ok ? h->k : 0u;
+      if (a_next >= k) { ++p; a_next = 0; continue; }
+      const float* shortv = reinterpret_cast<const float*>(payload + h->off_short);
+      const float* longv = reinterpret_cast<const float*>(payload + h->off_long);
+      rowv[na] = (tall ? longv : shortv) + (int64_t)a_next * rlen;     // indexed by output row
+      colv[na] = (tall ? shortv : longv) + (int64_t)a_next * clen;     // indexed by output column
+      cf[na] = __ldg(reinterpret_cast<const float*>(payload + h->off_val) + a_next) * scale;
+      ++na; ++a_next;
     }
-    for (int idx = tid; idx < na * kDecRows; idx += 256) {
-      const int a = idx / kDecRows, i = idx % kDecRows;
-      s_row[a][i] = (i0 + i < rlen) ? __ldg(rowvec + (int64_t)(a0 + a) * rlen + i0 + i) * __ldg(coef + a0 + a) : 0.f;
-    }
+    if (na == 0 && !first_pass) break;
     __syncthreads();
-    for (int a = 0; a < na; ++a) {
-      const float4 cv = *reinterpret_cast<const float4*>(&s_col[a][cg * 4]);
+    for (int idx = threadIdx.x; idx < kDecRows * kDecAtoms; idx += kDecThreads) {
+      const int i = idx / kDecAtoms, a = idx % kDecAtoms;
+      float v = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const float rv = s_row[a][rg * 8 + i];
-        acc[i][0] = fmaf(rv, cv.x, acc[i][0]); acc[i][1] = fmaf(rv, cv.y, acc[i][1]);
-        acc[i][2] = fmaf(rv, cv.z, acc[i][2]); acc[i][3] = fmaf(rv, cv.w, acc[i][3]);
+      for (int u = 0; u < kDecAtoms; ++u) if (u == a && u < na && i < n_rows) v = __ldg(rowv[u] + i0 + i) * cf[u];
+      s_rc[i][a] = v;
+    }
+    float4 cv[kDecAtoms];
+#pragma unroll
+    for (int a = 0; a < kDecAtoms; ++a) {
+      cv[a] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (a < na && c < cols) {
+        const float* src = colv[a] + c;
+        if ((clen % 4 == 0) && ((reinterpret_cast<uintptr_t>(colv[a]) & 15u) == 0) && c + 3 < cols)
+          cv[a] = __ldg(reinterpret_cast<const float4*>(src));
+        else {
+          cv[a].x = __ldg(src);
+          if (c + 1 < cols) cv[a].y = __ldg(src + 1);
+          if (c + 2 < cols) cv[a].z = __ldg(src + 2);
+          if (c + 3 < cols) cv[a].w = __ldg(src + 3);
+        }
       }
     }
-  }
-  const bool vec_ok = (cols % 4 == 0) && ((reinterpret_cast<uintptr_t>(D.out) & 15u) == 0);
+    __syncthreads();
+    if (c < cols) {
+      const bool add = !first_pass;
+#pragma unroll 4
+      for (int i = 0; i < n_rows; ++i) {
+        const float4 r0 = *reinterpret_cast<const float4*>(&s_rc[i][0]);
+        const float4 r1 = *reinterpret_cast<const float4*>(&s_rc[i][4]);
+        const float rc[kDecAtoms] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int64_t row = i0 + rg * 8 + i;
-    if (row >= rows) continue;
-    const int64_t c = c0 + cg * 4;
-    float* o = D.out + row * cols + c;
-    if (vec_ok && c + 3 < cols) *reinterpret_cast<float4*>(o) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-    else for (int j = 0; j < 4; ++j) if (c + j < cols) o[j] = acc[i][j];
+        for (int a = 0; a < kDecAtoms; ++a) {
+          v.x = fmaf(rc[a], cv[a].x, v.x); v.y = fmaf(rc[a], cv[a].y, v.y);
+          v.z = fmaf(rc[a], cv[a].z, v.z); v.w = fmaf(rc[a], cv[a].w, v.w);
+        }
+        float* o = out + (int64_t)i * cols;
+        if (vec_out && c + 3 < cols) {
+          if (add) { const float4 old = *reinterpret_cast<const float4*>(o); v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w; }
+          *reinterpret_cast<float4*>(o) = v;
+        } else {
+          const float vv[4] = {v.x, v.y, v.z, v.w};
+          for (int j = 0; j < 4; ++j) if (c + j < cols) o[j] = add ? o[j] + vv[j] : vv[j];
+        }
+      }
+    }
+    first_pass = false;
+    if (na < kDecAtoms) break;                                    // the sequence is exhausted
   }
 }
 
 void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,
                       cudaStream_t st) {
-  if (n_tiles > 0) sp_decode_kernel<<<n_tiles, 256, 0, st>>>(payload, d_layers, d_tiles);
+  if (n_tiles > 0) sp_decode_kernel<<<n_tiles, kDecThreads, 0, st>>>(payload, nullptr, 1, 1.0f, d_layers, d_tiles);
+}
+
+void launch_sp_decode_average(const uint8_t* const* d_payloads, int n_payloads, const SpDecodeLayer* d_layers,
+                              const TileRef* d_tiles, int n_tiles, cudaStream_t st) {
+  if (n_tiles > 0)
+    sp_decode_kernel<<<n_tiles, kDecThreads, 0, st>>>(nullptr, d_payloads, n_payloads, 1.0f / (float)n_payloads, d_layers, d_tiles);
 }
 
 }  // namespace atomo

@@ -49,8 +49,8 @@ def test_static_decode_rejects_oversized_batches():
     with pytest.raises(api.AtomoError) as e:
         api.atomo_decode_spectral_static(big, [torch.empty(64, 64, device="cuda")] * 65)
     assert e.value.code == 3
-    # more output tiles than the fixed table holds (8192 tiles of 32 x 256 elements)
-    huge = api.Payload(pay.buf, api.KIND_SPECTRAL, [(32 * 8193, 256)], 8, a)
+    # more output tiles than the fixed table holds (8192 tiles of 64 x 1024 elements)
+    huge = api.Payload(pay.buf, api.KIND_SPECTRAL, [(64 * 8193, 256)], 8, a)
     with pytest.raises(api.AtomoError) as e:
         api.atomo_decode_spectral_static(huge, [torch.empty(1, device="cuda")])
     assert e.value.code == 3
