@@ -442,21 +442,21 @@ void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, 
 
 // =================================================================================================
 // back-projection: long-side vector of each kept atom.
-//   rows <= cols: w_a[c]   = sum_i G[i][c] u_a[i]   tile = 256 columns x one chunk of rows (a multiple of 64, set
-//                                                     per layer), thread per column, 8 row loads in flight;
+//   rows <= cols: w_a[c]   = sum_i G[i][c] u_a[i]   tile = 1024 columns x one chunk of rows (a multiple of 64, set
+//                                                     per layer), 4 columns per thread, 8 row loads in flight;
 //                                                     chunk partials go to bp_part and are summed in chunk
 //                                                     order by sp_finish_atoms
 //   rows >  cols: w_a[row] = sum_c G[row][c] v_a[c]   tile = 32 rows, warp per row (one chunk)
 // =================================================================================================
-constexpr int kBpThreads = 256, kBpAtoms = 8, kBpCols = 256, kBpRows = 32, kBpChunk = 64;
+constexpr int kBpThreads = 256, kBpAtoms = 8, kBpCols = 1024, kBpRows = 32, kBpChunk = 64;
 int sp_bp_cols_per_tile() { return kBpCols; }
 int sp_bp_rows_per_tile() { return kBpRows; }
 int sp_bp_chunk_rows() { return kBpChunk; }
 
 __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLayer* __restrict__ layers,
                                                                     const TileRef* __restrict__ tiles) {
-  __shared__ float s_u[kBpAtoms][kBpChunk];            // wide: the chunk's components of up to 8 short-side vectors
-  extern __shared__ __align__(16) float s_v[];         // tall: kBpAtoms x r
+  __shared__ __align__(16) float s_u[kBpChunk][kBpAtoms];   // wide: the chunk's components of up to 8 short-side vectors
+  extern __shared__ __align__(16) float s_v[];              // tall: kBpAtoms x r
   const TileRef ref = tiles[blockIdx.x];
   const SpLayer& L = layers[ref.layer];
   const uint32_t k = L.hdr->k;
@@ -464,40 +464,65 @@ __global__ void __launch_bounds__(kBpThreads) sp_backproject_kernel(const SpLaye
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const float* __restrict__ G = L.G;
   const int64_t ld = L.ld;
+  const bool vec = (ld % 4 == 0) && ((reinterpret_cast<uintptr_t>(G) & 15u) == 0);
   for (uint32_t a0 = 0; a0 < k; a0 += kBpAtoms) {
     const int na = min((uint32_t)kBpAtoms, k - a0);
     __syncthreads();
     if (!L.tall) {
+      // a thread owns 4 consecutive columns: one 16-byte load per row, 8 rows in flight, 32 FMAs per row
       const int row_lo = ref.b * L.bp_chunk_rows, row_hi = min(r, row_lo + L.bp_chunk_rows);
-      const int c = ref.a * kBpCols + tid;
-      float acc[kBpAtoms];
+      const int c = ref.a * kBpCols + 4 * tid;
+      float acc[kBpAtoms][4];
 #pragma unroll
-      for (int a = 0; a < kBpAtoms; ++a) acc[a] = 0.f;
+      for (int a = 0; a < kBpAtoms; ++a) { acc[a][0] = 0.f; acc[a][1] = 0.f; acc[a][2] = 0.f; acc[a][3] = 0.f; }
       for (int i0 = row_lo; i0 < row_hi; i0 += kBpChunk) {
         const int ni = min(kBpChunk, row_hi - i0);
         if (i0 > row_lo) __syncthreads();
-        for (int idx = tid; idx < na * kBpChunk; idx += kBpThreads) {
-          const int a = idx / kBpChunk, i = idx % kBpChunk;
-          s_u[a][i] = i < ni ? L.shortv[(int64_t)(a0 + a) * r + i0 + i] : 0.0f;
+        for (int idx = tid; idx < kBpAtoms * kBpChunk; idx += kBpThreads) {
+          const int i = idx / kBpAtoms, a = idx % kBpAtoms;
+          s_u[i][a] = (a < na && i < ni) ? L.shortv[(int64_t)(a0 + a) * r + i0 + i] : 0.0f;
         }
         __syncthreads();
         if (c < len) {
           const float* gp = G + (int64_t)i0 * ld + c;
+          const bool full4 = vec && c + 3 < len;
           for (int i = 0; i < ni; i += 8) {
-            float g[8];
+            float4 g[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) g[u] = (i + u < ni) ? __ldg(gp + (int64_t)(i + u) * ld) : 0.0f;
+            for (int u = 0; u < 8; ++u) {
+              g[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+              if (i + u < ni) {
+                const float* src = gp + (int64_t)(i + u) * ld;
+                if (full4) g[u] = __ldg(reinterpret_cast<const float4*>(src));
+                else {
+                  g[u].x = __ldg(src);
+                  if (c + 1 < len) g[u].y = __ldg(src + 1);
+                  if (c + 2 < len) g[u].z = __ldg(src + 2);
+                  if (c + 3 < len) g[u].w = __ldg(src + 3);
+                }
+              }
+            }
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
+            for (int u = 0; u < 8; ++u) {
+              const float4 u0 = *reinterpret_cast<const float4*>(&s_u[i + u][0]);     // rows past ni hold zeros
+              const float4 u1 = *reinterpret_cast<const float4*>(&s_u[i + u][4]);
+              const float uu[kBpAtoms] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
 #pragma unroll
-              for (int a = 0; a < kBpAtoms; ++a) acc[a] = fmaf(g[u], s_u[a][i + u], acc[a]);   // rows past ni hold zeros
+              for (int a = 0; a < kBpAtoms; ++a) {
+                acc[a][0] = fmaf(g[u].x, uu[a], acc[a][0]); acc[a][1] = fmaf(g[u].y, uu[a], acc[a][1]);
+                acc[a][2] = fmaf(g[u].z, uu[a], acc[a][2]); acc[a][3] = fmaf(g[u].w, uu[a], acc[a][3]);
+              }
+            }
           }
         }
       }
       if (c < len) {
 #pragma unroll
         for (int a = 0; a < kBpAtoms; ++a)
-          if (a < na) L.bp_part[((int64_t)ref.b * L.k_cap + a0 + a) * len + c] = acc[a];
+          if (a < na) {
+            float* dst = L.bp_part + ((int64_t)ref.b * L.k_cap + a0 + a) * len + c;
+            for (int j = 0; j < 4; ++j) if (c + j < len) dst[j] = acc[a][j];
+          }
       }
     } else {
       for (int idx = tid; idx < na * r; idx += kBpThreads) s_v[idx] = L.shortv[(int64_t)a0 * r + idx];
