@@ -286,50 +286,28 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   // eigenvalue of A per row, one warp per row.  mode 0: lambda_i = <x_i, v_i> (Rayleigh quotient at v_i);
   // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T).  With refinement: the sum of the tiles' partial
   // squared norms of the projection (already in the units of G).
-  // (without refinement: four rows of a warp at a time, so that their loads are in flight together)
-  constexpr int kRowsAtOnce = 4, kFinWarps = kFinThreads / 32;
-  for (int i0 = w; i0 < r; i0 += kFinWarps * kRowsAtOnce) {
-    float lam[kRowsAtOnce];
+  for (int i = w; i < r; i += kFinThreads / 32) {
+    float lam;
     if (L.refine) {
-#pragma unroll
-      for (int u = 0; u < kRowsAtOnce; ++u) {
-        const int i = i0 + u * kFinWarps;
-        double d = 0.0;
-        if (i < r)
-          for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
-        lam[u] = (float)warp_sum(d);
-      }
+      double d = 0.0;
+      for (int tl = lane; tl < L.refine_tiles; tl += 32) d += (double)L.refine_partials[(int64_t)tl * rp + i];
+      lam = (float)warp_sum(d);
     } else {
       // rows are zero-padded to rp floats (a multiple of 32): whole float4, several loads in flight
-      float d0[kRowsAtOnce], d1[kRowsAtOnce];
-#pragma unroll
-      for (int u = 0; u < kRowsAtOnce; ++u) { d0[u] = 0.f; d1[u] = 0.f; }
+      const float4* x4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx);
+      const float4* v4 = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx + voff);
+      float d0 = 0.f, d1 = 0.f;
+#pragma unroll 4
       for (int j = lane; j < rp / 4; j += 32) {
-        float4 a[kRowsAtOnce], b[kRowsAtOnce];
-#pragma unroll
-        for (int u = 0; u < kRowsAtOnce; ++u) {
-          const int i = min(i0 + u * kFinWarps, r - 1);
-          a[u] = reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx)[j];
-          b[u] = voff ? reinterpret_cast<const float4*>(L.X + (int64_t)i * ldx + voff)[j] : a[u];
-        }
-#pragma unroll
-        for (int u = 0; u < kRowsAtOnce; ++u) {
-          d0[u] = fmaf(a[u].x, b[u].x, fmaf(a[u].y, b[u].y, d0[u]));
-          d1[u] = fmaf(a[u].z, b[u].z, fmaf(a[u].w, b[u].w, d1[u]));
-        }
+        const float4 a = x4[j], b = v4[j];
+        d0 = fmaf(a.x, b.x, fmaf(a.y, b.y, d0));
+        d1 = fmaf(a.z, b.z, fmaf(a.w, b.w, d1));
       }
-#pragma unroll
-      for (int u = 0; u < kRowsAtOnce; ++u) lam[u] = warp_sum(d0[u] + d1[u]) * inv_scale;
+      lam = warp_sum(d0 + d1) * inv_scale;
     }
     if (lane == 0) {
-#pragma unroll
-      for (int u = 0; u < kRowsAtOnce; ++u) {
-        const int i = i0 + u * kFinWarps;
-        if (i < r) {
-          if (!(fabsf(lam[u]) <= 3.0e38f)) atomicOr(&s_bad, 1u);
-          s_lam[i] = fmaxf(lam[u], 0.0f);
-        }
-      }
+      if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
+      s_lam[i] = fmaxf(lam, 0.0f);
     }
   }
   __syncthreads();
