@@ -14,8 +14,9 @@
  *     descriptors (atomo_mat, atomo_vec, pointer lists, shape lists) are HOST memory and are
  *     consumed before the call returns.
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
- *     Encode calls wait on the host for the eigen-solver's convergence flag once per sweep, so
- *     they are not capturable in a CUDA graph; decode calls never synchronise.
+ *     atomo_encode_spectral waits on the host once, after it has enqueued all its work (the kernels' bounded
+ *     waits report there), or once per Jacobi sweep in launch scheme 0; atomo_encode_entrywise and the decode
+ *     calls never synchronise.  No claim is made about capture in a CUDA graph.
  *   - Matrices are fp32 row-major with leading dimension `ld` (elements, ld >= cols).
  *   - Functions return an atomo_status.  Problems visible on the host (NULL, bad sizes,
  *     s <= 0 or not finite, payload capacity too small) return at once and launch nothing.

@@ -408,6 +408,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   stage_begin(ctx, ATOMO_STAGE_EIG, st);
   int t_done = 0;
   int64_t n_eig_launch = 0;
+  bool flags_pending = false;
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
@@ -441,9 +442,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(jacobi clusters)");
     launch_sp_check(d_layers, n_layers, steps_max * max_sweeps, max_sweeps, d_flag, st);
     n_eig_launch = 2;
-    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
-    CK(cudaStreamSynchronize(st));
-    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+    CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    flags_pending = true;                                  // read at the end of the call, after everything is enqueued
   }
   const int capacity = (!cluster_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
   int max_layer_pairs = 0;
@@ -474,9 +475,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     launch_sp_check(d_layers, n_layers, t_max, max_sweeps, d_flag, st);
     ++n_eig_launch;
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
-    CK(cudaStreamSynchronize(st));
-    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
-    if (ctx->h_flag[2] != 0) { ctx->err = "a step barrier of the persistent eigen-solve ran out of polls"; return ATOMO_ERR_TIMEOUT; }
+    flags_pending = true;                                  // read at the end of the call, after everything is enqueued
   } else
   for (int it = 0; it < max_sweeps; ++it) {
     for (int j = 0; j < steps_max; ++j, ++t_done, ++n_eig_launch)
@@ -502,6 +501,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   launch_sp_finish_atoms(d_layers, n_layers, k_cap_max, st);
   stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, 2);
   CK(cudaGetLastError());
+  if (flags_pending) {
+    // the one host wait of the persistent forms: the kernels' bounded waits report here
+    CK(cudaStreamSynchronize(st));
+    if (ctx->h_flag[1] != 0) { ctx->err = "a bounded wait in the tensor-core Gram kernel ran out"; return ATOMO_ERR_TIMEOUT; }
+    if (ctx->h_flag[2] != 0) { ctx->err = "a step barrier of the persistent eigen-solve ran out of polls"; return ATOMO_ERR_TIMEOUT; }
+  }
   return ATOMO_OK;
 }
 
