@@ -10,10 +10,19 @@
 //                     convergence x_i = lambda_i v_i^T.  Twice the row length and about twice the sweeps
 //                     (the rows of A start nearly parallel), kept as a cross-check.
 //
-// Blocks of 16 rows are paired round-robin; a CTA holds one block pair in shared memory, one warp per
-// rotation.  Row norms are tracked (alpha' = alpha - t gamma, beta' = beta + t gamma) and refreshed when
-// they cancel; rotations are applied in the scaled ("fast Givens") form, one FMA per element, with the
-// cosines collected in a per-row factor that is folded back when the block pair is stored.
+// Blocks of 16 rows are paired by a recursive-halving schedule (step_plan); a CTA holds one block pair in shared
+// memory, one warp per rotation; inside a block the pairs follow a round-robin tournament, once per sweep.  Row
+// norms are tracked (alpha' = alpha - t gamma, beta' = beta + t gamma) and refreshed when they cancel; rotations
+// are applied in the scaled ("fast Givens") form, one FMA per element, with the cosines collected in a per-row
+// factor that is folded back when a block is stored or handed over.
+//
+// Three launch forms around the same rotation code (rotate_pair):
+//   sp_jacobi_cluster_kernel     layers of up to 16 block pairs: a layer's CTAs in one 16-CTA cluster for the whole
+//                                solve, blocks handed over through distributed shared memory, cluster barrier per step
+//   sp_jacobi_persistent_kernel  cooperative launch over groups of whole layers, blocks through global memory (L2),
+//                                a barrier among the CTAs of a layer per step
+//   sp_jacobi_step_kernel        one launch per step, the host reads a convergence flag once per sweep
+// and, before them, the Cholesky factorisation (clusters of 8 CTAs per layer; a cooperative kernel above 1024 rows).
 #include <algorithm>
 
 #include <cooperative_groups.h>
