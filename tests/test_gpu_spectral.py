@@ -133,6 +133,44 @@ def test_eigen_launch_schemes_agree(atomo):
             assert np.array_equal(other[1][l], got[0][1][l])
 
 
+def test_random_batches(atomo):
+    """Seeded random batches (1 to 39 layers, short sides 1 to 512, wide and tall, several spectra, noise levels and
+    budgets): the packing of layers into clusters, idle CTAs, tiny and ragged layers.  Properties that hold at any
+    size: status, singular values against a library SVD, sum(p) = min(s, rank), decode = its definition."""
+    import torch
+    rng = np.random.default_rng(77)
+    for trial in range(8):
+        n_layers = int(rng.integers(1, 40))
+        mats = []
+        for l in range(n_layers):
+            m = int(rng.choice([1, 3, 10, 17, 33, 64, 100, 129, 200, 256, 300, 512]))
+            n = int(rng.choice([1, 5, 18, 27, 64, 130, 576, 700, 1152]))
+            if rng.random() < 0.3:
+                m, n = n, m
+            mats.append(synth.lowrank_plus_noise(np.random.default_rng([trial, l]), m, n, float(rng.choice([0.5, 1.0, 1.5])),
+                                                 noise_rel=float(rng.choice([0.0, 0.01, 0.1]))))
+        s = float(rng.choice([0.5, 1.0, 2.0, 3.7]))
+        ts = [torch.from_numpy(G).cuda() for G in mats]
+        pay, dbg = atomo.atomo_encode_spectral(ts, s, seed=trial, step=trial, k_cap=64, debug=True)
+        hdrs = pay.headers()
+        assert [h.status for h in hdrs[1]] == [0] * n_layers
+        outs = atomo.atomo_decode(pay)
+        for l, G in enumerate(mats):
+            r = min(G.shape)
+            ref = np.linalg.svd(G.astype(np.float64), compute_uv=False)
+            sig = dbg.layer_sigma(l, r)
+            assert parity.rel(sig, ref) <= parity.REL_TOL, (trial, l, G.shape)
+            p = dbg.layer_prob(l, r)
+            assert abs(p.sum() - min(s, float((sig > 0).sum()))) <= 1e-3 * max(s, 1.0), (trial, l, G.shape)
+            arr = pay.layer_arrays(l, hdrs)
+            out = outs[l].cpu().numpy()
+            if arr["k"]:
+                own = (arr["U"].astype(np.float64) * arr["coef"].astype(np.float64)) @ arr["V"].astype(np.float64).T
+                assert parity.rel(out, own) <= 1e-5, (trial, l, G.shape)
+            else:
+                assert not out.any()
+
+
 def test_leading_dimension(atomo, oracle):
     rng = np.random.default_rng(7)
     mats = [synth.lowrank_plus_noise(rng, 48, 200, 1.0, noise_rel=0.02),
