@@ -250,6 +250,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- host descriptors, tiles, workspace carving (two passes: size, then pointers) ----
   std::vector<SpLayer> L(n_layers);
+  std::vector<int> tc_layers;
   std::vector<TileRef> gram_tiles, block_pairs, bp_tiles, chol_ctas, refine_tiles, tc_tiles;
   const int map_bytes = sp_tc_map_bytes();
   std::vector<uint8_t> maps_blob((size_t)n_layers * map_bytes, 0);
@@ -271,12 +272,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     k_cap_max = std::max(k_cap_max, (int)d.k_cap);
     r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
-    d.tc = 0;
+    d.tc = 0; d.gram_split = 1;
     if (ctx->tc_gram && ctx->tc_ok && !d.acc && sp_tc_eligible(d.G, d.rows, d.cols, d.ld)) {
       d.tc = 1;
       if (sp_tc_make_map(maps_blob.data() + (size_t)l * map_bytes, d.G, d.rows, d.cols, d.ld) != 0) return ATOMO_ERR_INVALID_ARG;
-      const int tt = (d.r + sp_tc_tile() - 1) / sp_tc_tile();
-      for (int a = 0; a < tt; ++a) for (int b = a; b < tt; ++b) tc_tiles.push_back({l, a, b, 0});
+      tc_layers.push_back(l);
     } else {
       for (int a = 0; a < gt; ++a) for (int b = a; b < gt; ++b) gram_tiles.push_back({l, a, b, 0});
     }
@@ -304,6 +304,32 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d.refine_tiles = (d.L + 63) / 64;
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
+  }
+  // tensor-core Gram tiles: while the batch has fewer CTAs than the GPU has SMs, the K range of the layers with the
+  // longest rows is split over 2 or 4 CTAs per tile (at least 16 stages of 32 columns per part)
+  {
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    auto tiles_of = [&](int l) { const int tt = (L[l].r + sp_tc_tile() - 1) / sp_tc_tile(); return tt * (tt + 1) / 2; };
+    int total = 0;
+    for (int l : tc_layers) { L[l].gram_split = 1; total += tiles_of(l); }
+    for (;;) {
+      int best = -1;
+      for (int l : tc_layers) {
+        const int stages = (L[l].L + 31) / 32 / L[l].gram_split;
+        if (L[l].gram_split < 4 && stages >= 32 && total + tiles_of(l) * L[l].gram_split <= sms &&
+            (best < 0 || stages > (L[best].L + 31) / 32 / L[best].gram_split))
+          best = l;
+      }
+      if (best < 0) break;
+      total += tiles_of(best) * L[best].gram_split;
+      L[best].gram_split *= 2;
+    }
+    for (int l : tc_layers) {
+      const int tt = (L[l].r + sp_tc_tile() - 1) / sp_tc_tile();
+      for (int a = 0; a < tt; ++a) for (int b = a; b < tt; ++b)
+        for (int c = 0; c < L[l].gram_split; ++c) tc_tiles.push_back({l, a, b, c});
+    }
   }
   SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_pairs = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
   uint8_t* d_maps = nullptr;
@@ -339,6 +365,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       d.p_sel = A.take<float>(d.k_cap);
       d.bp_part = A.take<float>((size_t)d.bp_chunks * d.k_cap * d.L);
       d.scale = A.take<float>(1);
+      {
+        const int tt = (d.r + sp_tc_tile() - 1) / sp_tc_tile();
+        d.gram_part = A.take<float>(d.tc && d.gram_split > 1
+                                        ? (size_t)tt * (tt + 1) / 2 * d.gram_split * sp_tc_tile() * sp_tc_tile() : 0);
+      }
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
       d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);
@@ -352,6 +383,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
     size_t z0 = A.off;
     for (int l = 0; l < n_layers; ++l) { L[l].rot_count = A.take<uint32_t>(max_sweeps); L[l].step_bar = A.take<uint32_t>(1); }
+    for (int l = 0; l < n_layers; ++l) {
+      const int tt = (L[l].r + sp_tc_tile() - 1) / sp_tc_tile();
+      L[l].gram_ticket = A.take<uint32_t>(L[l].tc && L[l].gram_split > 1 ? (size_t)tt * (tt + 1) / 2 : 0);
+    }
     for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * L[l].ldx);
     zero_beg = zb; zero_bytes = A.off - z0;
     for (int l = 0; l < n_layers; ++l) {

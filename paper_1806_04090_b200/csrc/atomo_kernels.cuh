@@ -78,6 +78,9 @@ struct SpLayer {
   float* chol_dd;              // 32 x 32 + 32 floats: diagonal block of the current Cholesky panel, published by its owner
   float* dbg_short;            // r x r or nullptr
   int tc;                      // Gram matrix came from the tensor-core kernel (see sp_scale_kernel)
+  int gram_split;              // tensor-core Gram: CTAs per output tile (parts of the K range), 1 = no split
+  float* gram_part;            // [tiles][gram_split][128 x 128] partial tiles (column-major) when gram_split > 1
+  uint32_t* gram_ticket;       // [tiles] parts finished; zeroed per call
   int refine, refine_tiles;    // singular values from the projection norms; tiles along the long side
   float* row_inv;              // rp: 1 / norm of each short-side vector as stored in X
   float* refine_partials;      // [refine_tiles][rp] partial squared norms

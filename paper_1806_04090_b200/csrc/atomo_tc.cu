@@ -100,13 +100,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) sp_gram_tc_kernel(const SpLayer
   auto tempty_bar = [&](int b) { return bars + 8u * (3 * kTcStages + 2 + b); };   // accumulator b has been drained
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(base_ptr + kTcStages * kTcStageBytes + 8 * (3 * kTcStages + 4));
   volatile uint32_t* s_abort = s_tmem + 1;
+  volatile uint32_t* s_last = s_tmem + 2;
 
   const TileRef ref = tiles[blockIdx.x];
   const SpLayer& L = layers[ref.layer];
   const CUtensorMap* map = maps + ref.layer;
   const int ti = ref.a, tj = ref.b;
   const bool diag = ti == tj;
-  const int num_kb = (L.L + kTcKBlk - 1) / kTcKBlk;
+  // a tile's K range may be split over L.gram_split CTAs (ref.c = which part); the parts are added by the last
+  // CTA of the tile to finish, in part order
+  const int all_kb = (L.L + kTcKBlk - 1) / kTcKBlk;
+  const int n_split = L.gram_split;
+  const int kb_lo = (int)((int64_t)all_kb * ref.c / n_split), kb_hi = (int)((int64_t)all_kb * (ref.c + 1) / n_split);
+  const int num_kb = kb_hi - kb_lo;                         // stage / phase arithmetic below counts from kb_lo
   const int tid = threadIdx.x, warp = tid / 32, lane = tid % 32;
 
   if (tid == 0) {
@@ -133,8 +139,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) sp_gram_tc_kernel(const SpLayer
         if (!tc_mbar_wait(empty_bar(s), ph ^ 1u, s_abort)) break;
         const uint32_t stage = base + s * kTcStageBytes;
         tc_mbar_expect_tx(full_bar(s), diag ? kTcTileBytes : 2 * kTcTileBytes);
-        tc_tma_load_2d(stage, map, full_bar(s), kb * kTcKBlk, ti * kTcTile);
-        if (!diag) tc_tma_load_2d(stage + 2 * kTcTileBytes, map, full_bar(s), kb * kTcKBlk, tj * kTcTile);
+        tc_tma_load_2d(stage, map, full_bar(s), (kb_lo + kb) * kTcKBlk, ti * kTcTile);
+        if (!diag) tc_tma_load_2d(stage + 2 * kTcTileBytes, map, full_bar(s), (kb_lo + kb) * kTcKBlk, tj * kTcTile);
       }
     }
   } else if (warp == 1) {
@@ -219,18 +225,49 @@ __global__ void __launch_bounds__(kTcThreads, 1) sp_gram_tc_kernel(const SpLayer
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       tc_mbar_arrive(tempty_bar(buf));
     }
-    if (ok) {
-      const int gi = ti * kTcTile + row;
-      const int r = L.r;
-      const int64_t lda = L.lda;
-      float* A = L.A;
+    // Epilogue.  The stage buffers are free now (every load has landed and every MMA has completed): the tile goes
+    // through shared memory (row stride 129 floats, conflict-free both ways) so that both triangles of A are written
+    // with consecutive lanes on consecutive addresses.
+    const int r = L.r;
+    const int64_t lda = L.lda;
+    float* A = L.A;
+    float* s_tile = reinterpret_cast<float*>(base_ptr);
+    constexpr int kPad = kTcTile + 1;
+    const int dt = tid - 6 * 32;                               // 0 .. 127 among the drain warps (= row)
+    bool write_tile = ok;
+    if (n_split > 1) {
+      // this part's tile to the workspace, column-major (consecutive lanes, consecutive addresses)
+      const int tt = (r + kTcTile - 1) / kTcTile;
+      const int tile_id = ti * tt - ti * (ti - 1) / 2 + (tj - ti);
+      float* part = L.gram_part + ((int64_t)tile_id * n_split + ref.c) * (kTcTile * kTcTile);
 #pragma unroll
-      for (int j = 0; j < kTcTile; ++j) {
-        const int gj = tj * kTcTile + j;
-        if (gi < r && gj < r) {
-          A[(int64_t)gi * lda + gj] = acc[j];
-          if (!diag) A[(int64_t)gj * lda + gi] = acc[j];
+      for (int j = 0; j < kTcTile; ++j) part[j * kTcTile + row] = acc[j];
+      __threadfence();
+      asm volatile("bar.sync 2, 128;" ::: "memory");           // the four drain warps
+      if (dt == 0) *s_last = atomicAdd(L.gram_ticket + tile_id, 1u) == (uint32_t)(n_split - 1) ? 1u : 0u;
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+      write_tile = *s_last != 0;                               // the last part to finish adds them all, in part order
+      if (write_tile) {
+        __threadfence();
+        const float* parts = L.gram_part + (int64_t)tile_id * n_split * (kTcTile * kTcTile);
+#pragma unroll
+        for (int j = 0; j < kTcTile; ++j) acc[j] = 0.f;
+        for (int sp = 0; sp < n_split; ++sp) {
+          const float* ps = parts + (int64_t)sp * (kTcTile * kTcTile) + row;
+#pragma unroll
+          for (int j = 0; j < kTcTile; ++j) acc[j] += __ldcg(ps + j * kTcTile);
         }
+      }
+    }
+    if (write_tile) {                                          // uniform over the drain warps
+#pragma unroll
+      for (int j = 0; j < kTcTile; ++j) s_tile[row * kPad + j] = acc[j];
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+      const int gcol = tj * kTcTile + dt, grow_m = ti * kTcTile + dt;
+      for (int rr = 0; rr < kTcTile; ++rr) {
+        const int gi = ti * kTcTile + rr, gj = tj * kTcTile + rr;
+        if (gi < r && gcol < r) A[(int64_t)gi * lda + gcol] = s_tile[rr * kPad + dt];
+        if (!diag && gj < r && grow_m < r) A[(int64_t)gj * lda + grow_m] = s_tile[dt * kPad + rr];
       }
     }
   }
