@@ -747,16 +747,22 @@ __global__ void __launch_bounds__(kCholClusterThreads) sp_cholesky_cluster_kerne
         __syncthreads();
         float xn[kCholPanel];
         if (k0 + kCholPanel < j0) fetch(k0 + kCholPanel, xn);
+        // packed fp32 pairs: one instruction updates two columns
+        uint64_t pk[kCholPanel / 2];
+#pragma unroll
+        for (int c = 0; c < kCholPanel / 2; ++c) pk[c] = pack2(p[2 * c], p[2 * c + 1]);
 #pragma unroll
         for (int kk = 0; kk < kCholPanel; ++kk) {
-          const float xi = -xc[kk];
+          const uint64_t xi2 = pack2(-xc[kk], -xc[kk]);
 #pragma unroll
           for (int c = 0; c < kCholPanel; c += 4) {
-            const float4 lk = *reinterpret_cast<const float4*>(&s_k[kk][c]);   // same address in every lane: broadcast
-            p[c] = fmaf(xi, lk.x, p[c]); p[c + 1] = fmaf(xi, lk.y, p[c + 1]);
-            p[c + 2] = fmaf(xi, lk.z, p[c + 2]); p[c + 3] = fmaf(xi, lk.w, p[c + 3]);
+            const ulonglong2 lk = *reinterpret_cast<const ulonglong2*>(&s_k[kk][c]);   // same address in every lane: broadcast
+            pk[c / 2] = fma2(xi2, lk.x, pk[c / 2]);
+            pk[c / 2 + 1] = fma2(xi2, lk.y, pk[c / 2 + 1]);
           }
         }
+#pragma unroll
+        for (int c = 0; c < kCholPanel / 2; ++c) unpack2(pk[c], p[2 * c], p[2 * c + 1]);
 #pragma unroll
         for (int kk = 0; kk < kCholPanel; ++kk) xc[kk] = xn[kk];
       }
