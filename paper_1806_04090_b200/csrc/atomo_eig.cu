@@ -152,15 +152,19 @@ __device__ __forceinline__ float rsqrt_approx(float v) { float r; asm("rsqrt.app
 template <int T4, int WPR, typename Store>
 __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, float& np2, float& nq2, float& dp,
                                             float& dq, int lane, int A4, float tol, RowSum<WPR>& row_sum, Store&& store) {
-  float g0 = 0.f, g1 = 0.f;
+  // dot product and update in packed fp32 pairs (one instruction per two elements)
+  uint64_t gA = 0ull, gB = 0ull;
 #pragma unroll
   for (int t = 0; t < T4; ++t) {
     if (lane + 32 * t < A4) {
       const float4 a = xp.v[t], b = xq.v[t];
-      g0 = fmaf(a.x, b.x, fmaf(a.y, b.y, g0));
-      g1 = fmaf(a.z, b.z, fmaf(a.w, b.w, g1));
+      gA = fma2(pack2(a.x, a.y), pack2(b.x, b.y), gA);
+      gB = fma2(pack2(a.z, a.w), pack2(b.z, b.w), gB);
     }
   }
+  float g0, g1, g2, g3;
+  unpack2(gA, g0, g2); unpack2(gB, g1, g3);
+  g0 += g2; g1 += g3;
   // everything that does not need the dot product
   const float al = np2, be = nq2;
   const float m = rsqrt_approx(al) * rsqrt_approx(be);
@@ -185,11 +189,15 @@ __device__ __forceinline__ bool rotate_pair(RowRegs<T4>& xp, RowRegs<T4>& xq, fl
   const float tt = copysignf(2.0f * gn, gn * tau) * rcp_approx(h + atau);
   if (tt == 0.0f) return false;
   const float a = -tt * ratio_qp, b = tt * ratio_pq;
+  const uint64_t a2 = pack2(a, a), b2 = pack2(b, b);
 #pragma unroll
   for (int t = 0; t < T4; ++t) {
     const float4 u = xp.v[t], w = xq.v[t];
-    xp.v[t] = make_float4(fmaf(a, w.x, u.x), fmaf(a, w.y, u.y), fmaf(a, w.z, u.z), fmaf(a, w.w, u.w));
-    xq.v[t] = make_float4(fmaf(b, u.x, w.x), fmaf(b, u.y, w.y), fmaf(b, u.z, w.z), fmaf(b, u.w, w.w));
+    const uint64_t u01 = pack2(u.x, u.y), u23 = pack2(u.z, u.w), w01 = pack2(w.x, w.y), w23 = pack2(w.z, w.w);
+    unpack2(fma2(a2, w01, u01), xp.v[t].x, xp.v[t].y);
+    unpack2(fma2(a2, w23, u23), xp.v[t].z, xp.v[t].w);
+    unpack2(fma2(b2, u01, w01), xq.v[t].x, xq.v[t].y);
+    unpack2(fma2(b2, u23, w23), xq.v[t].z, xq.v[t].w);
   }
   store();
   const float y = fmaf(tt, tt, 1.0f);
