@@ -305,6 +305,17 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
+  // Cluster form first: every layer's block pairs inside one 16-CTA cluster, blocks exchanged through
+  // distributed shared memory (layers of up to 16 block pairs, route 1).
+  bool cluster_form = ctx->eig_scheme == 2 && ctx->eig_mode != 0;
+  for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
+  if (cluster_form) {
+    int lg = 0;
+    while ((1 << lg) < rp_max) ++lg;
+    if (ctx->cluster_capacity[lg] < 0) ctx->cluster_capacity[lg] = sp_jacobi_cluster_capacity(rp_max);
+    if (ctx->cluster_capacity[lg] < 1) cluster_form = false;
+  }
+  for (int l = 0; l < n_layers; ++l) L[l].lam_ready = cluster_form ? 1 : 0;
   // tensor-core Gram tiles: while the batch has fewer CTAs than the GPU has SMs, the K range of the layers with the
   // longest rows is split over 2 or 4 CTAs per tile (at least 16 stages of 32 columns per part)
   {
@@ -447,16 +458,6 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
-  // Cluster form first: every layer's block pairs inside one 16-CTA cluster, blocks exchanged through
-  // distributed shared memory (layers of up to 16 block pairs, route 1).
-  bool cluster_form = ctx->eig_scheme == 2 && ctx->eig_mode != 0;
-  for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
-  if (cluster_form) {
-    int lg = 0;
-    while ((1 << lg) < rp_max) ++lg;
-    if (ctx->cluster_capacity[lg] < 0) ctx->cluster_capacity[lg] = sp_jacobi_cluster_capacity(rp_max);
-    if (ctx->cluster_capacity[lg] < 1) cluster_form = false;
-  }
   if (cluster_form) {
     const int per = sp_jacobi_cluster_ctas();
     std::vector<int> order(n_layers);

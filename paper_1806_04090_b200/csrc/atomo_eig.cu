@@ -499,6 +499,12 @@ __device__ __forceinline__ void cluster_step(const SpLayer& L, const ClusterCta&
       const float* src = row < B ? F.row(row) : M.row(row - B);
       reinterpret_cast<float4*>(X + (int64_t)grow * RP)[q] = reinterpret_cast<const float4*>(src)[q];
     }
+    // the rows' squared norms as well: after a sweep that rotated nothing they are the ones computed from the rows
+    // at its start, which is what the singular values are taken from
+    if (tid < 2 * B) {
+      const int grow = (tid < B) ? plan.bi * B + tid : plan.bj * B + (tid - B);
+      L.lam[grow] = tid < B ? F.n2()[tid] : M.n2()[tid - B];
+    }
     done = true;
     return;
   }

@@ -65,7 +65,8 @@ struct SpLayer {
   float* X;                    // rp x ldx working rows of the Jacobi solver
   atomo_layer_header* hdr;     // payload
   uint32_t* idx; float* coef; float* shortv; float* longv;
-  float* lam;                  // rp   eigenvalue per row (unsorted, scaled)
+  float* lam;                  // rp   squared norm per row of X as the cluster eigen-solve left it (scaled units)
+  int lam_ready;               // lam was written by the eigen-solve (cluster form): finalize need not re-read X for it
   int* perm;                   // r    rank -> row
   float* sigma; float* prob;   // r    descending (debug buffers or workspace)
   uint32_t* mask_words;        // ceil(r/32)

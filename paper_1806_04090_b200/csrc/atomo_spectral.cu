@@ -286,6 +286,13 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   // eigenvalue of A per row, one warp per row.  mode 0: lambda_i = <x_i, v_i> (Rayleigh quotient at v_i);
   // mode 1: lambda_i = ||x_i||^2 (row i = sigma_i w_i^T).  With refinement: the sum of the tiles' partial
   // squared norms of the projection (already in the units of G).
+  if (L.lam_ready && !L.refine && !L.acc) {
+    for (int i = tid; i < r; i += kFinThreads) {
+      const float lam = L.lam[i] * inv_scale;
+      if (!(fabsf(lam) <= 3.0e38f)) atomicOr(&s_bad, 1u);
+      s_lam[i] = fmaxf(lam, 0.0f);
+    }
+  } else
   for (int i = w; i < r; i += kFinThreads / 32) {
     float lam;
     if (L.refine) {
