@@ -437,7 +437,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S1: Gram matrix, scaling ----
   stage_begin(ctx, ATOMO_STAGE_GRAM, st);
-  launch_sp_init(d_layers, n_layers, nullptr, 0, st);
+  if (ctx->eig_mode == 0) launch_sp_init(d_layers, n_layers, nullptr, 0, st);   // the identity half of [A | I]
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
   launch_sp_gram_tc(d_layers, d_maps, d_tc, (int)tc_tiles.size(), d_flag + 1, st);
   launch_sp_scale(d_layers, n_layers, st);
