@@ -71,6 +71,18 @@ typedef enum {
 enum { ATOMO_KIND_SPECTRAL = 0, ATOMO_KIND_ENTRYWISE = 1 };
 enum { ATOMO_MAGIC = 0x4F4D5441 /* "ATMO" */, ATOMO_VERSION = 2 };
 enum { ATOMO_EW_TILE = 4096 };   /* entry-wise payloads carry one offset per tile of this many elements */
+/* Entry-wise payload formats.  EXPLICIT: idx u32[k_cap] ascending and val f32[k_cap] = g_i / p_i.
+ * COMPACT (the ternary form of Section 4: a kept atom with p_i < 1 has g_i / p_i = sign(g_i) c with one
+ * scalar c = sum_unsaturated |g| / (s - n_sat) per vector, so its index and one sign bit say everything):
+ *   off_idx   u16[k_cap]  one entry per kept atom with p_i < 1, ascending by index: bits 0..11 = index inside
+ *                         its tile of ATOMO_EW_TILE elements, bit 15 = sign of g_i (the tile follows from the
+ *                         offset table), value sign * c with c from the layer header
+ *   off_short u32[n_tiles + 1]  number of such entries before each tile
+ *   off_long  u32[sat_cap] indices of the atoms with p_i = 1 (all kept), ascending
+ *   off_val   f32[sat_cap] their values g_i
+ * with k = all kept atoms, n_sat = the length of the saturated list, k - n_sat entries in off_idx.
+ * Both formats decode to the same dense gradient, bit for bit.                                         */
+enum { ATOMO_EW_EXPLICIT = 0, ATOMO_EW_COMPACT = 1 };
 
 typedef struct { const float* data; /* DEVICE */ int32_t rows, cols; int64_t ld; } atomo_mat;
 typedef struct { const float* data; /* DEVICE */ int64_t n; } atomo_vec;
@@ -81,7 +93,8 @@ typedef struct {
   uint64_t total_bytes;
   uint64_t seed, step;
   double   s;
-  uint64_t reserved[2];
+  uint64_t ew_format;         /* entry-wise: ATOMO_EW_EXPLICIT or ATOMO_EW_COMPACT; spectral: 0   */
+  uint64_t ew_sat_cap;        /* compact entry-wise: capacity of the saturated list; else 0       */
 } atomo_payload_header;                       /* 64 bytes */
 
 typedef struct {
@@ -124,6 +137,10 @@ const char* atomo_last_cuda_error(atomo_ctx* ctx);   /* text of the last failing
 int64_t atomo_payload_bytes_spectral(const int32_t* rows, const int32_t* cols, int32_t n_layers,
                                      int32_t k_cap);
 int64_t atomo_payload_bytes_entrywise(const int64_t* n, int32_t n_vecs, int64_t k_cap);
+/* Compact format: k_cap bounds the kept atoms with p < 1, sat_cap (>= 0, clamped to n) the atoms with p = 1.
+ * n_sat < s always (every saturated atom uses one unit of the budget), so sat_cap >= s cannot overflow; at the
+ * l_q budgets of Section 4 every vector is s-balanced and sat_cap = 0 is enough.                           */
+int64_t atomo_payload_bytes_entrywise_compact(const int64_t* n, int32_t n_vecs, int64_t k_cap, int64_t sat_cap);
 
 /* --- encode ---------------------------------------------------------------------------------
  * Spectral ATOMO (Section 5; Eq. 2, Eq. 3 / Algorithm 1) over a batch of layer gradients.
@@ -142,6 +159,11 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/,
                            double s, uint64_t seed, uint64_t step, int64_t k_cap,
                            void* payload /*DEVICE*/, int64_t capacity_bytes,
                            const atomo_debug* dbg, void* stream);
+/* Format of the payloads the context's later atomo_encode_entrywise calls write (default ATOMO_EW_EXPLICIT;
+ * sat_cap is read for ATOMO_EW_COMPACT only).  The draws, the kept set and the decoded gradient do not depend
+ * on the format.  A vector whose kept unsaturated atoms exceed k_cap or whose saturated atoms exceed sat_cap
+ * gets ATOMO_ERR_CAPACITY in its status word and k = 0.  Decoders read the format from the payload.       */
+int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap);
 
 /* --- l_q budgets (Section 4) ------------------------------------------------------------------
  * s_out[l] (HOST) = ||g_l||_1 / ||g_l||_q for every vector: the budget at which entry-wise ATOMO is the

@@ -19,6 +19,8 @@ LIB_PATH = os.environ.get("ATOMO_B200_LIB", os.path.join(_HERE, "libatomo_b200.s
 
 KIND_SPECTRAL = 0
 KIND_ENTRYWISE = 1
+EW_EXPLICIT, EW_COMPACT = 0, 1      # entry-wise payload formats
+EW_TILE = 4096                       # elements per tile of the entry-wise offset table
 STATUS_NAMES = ["OK", "INVALID_ARG", "BUDGET", "CAPACITY", "NONFINITE", "NOT_CONVERGED", "TIMEOUT", "CUDA",
                 "PAYLOAD"]
 STAGES = ["gram", "eig", "sample", "backproject", "ew_reduce", "ew_pack", "decode"]
@@ -29,6 +31,7 @@ EXPORTS = [
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
+    "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format",
 ]
 
 
@@ -55,7 +58,7 @@ class _Debug(ctypes.Structure):
 class PayloadHeader(ctypes.Structure):
     _fields_ = [("magic", ctypes.c_uint32), ("version", ctypes.c_uint32), ("kind", ctypes.c_uint32),
                 ("n_layers", ctypes.c_uint32), ("total_bytes", ctypes.c_uint64), ("seed", ctypes.c_uint64),
-                ("step", ctypes.c_uint64), ("s", ctypes.c_double), ("reserved", ctypes.c_uint64 * 2)]
+                ("step", ctypes.c_uint64), ("s", ctypes.c_double), ("ew_format", ctypes.c_uint64), ("ew_sat_cap", ctypes.c_uint64)]
 
 
 class LayerHeader(ctypes.Structure):
@@ -88,6 +91,9 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_payload_bytes_spectral.restype = i64
     lib.atomo_payload_bytes_entrywise.argtypes = [ctypes.POINTER(i64), i32, i64]
     lib.atomo_payload_bytes_entrywise.restype = i64
+    lib.atomo_payload_bytes_entrywise_compact.argtypes = [ctypes.POINTER(i64), i32, i64, i64]
+    lib.atomo_payload_bytes_entrywise_compact.restype = i64
+    lib.atomo_set_entrywise_format.argtypes = [vp, i32, i64]
     lib.atomo_encode_spectral.argtypes = [vp, ctypes.POINTER(_Mat), i32, dbl, u64, u64, i32, vp, i64,
                                           ctypes.POINTER(_Debug), vp]
     lib.atomo_encode_entrywise.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, u64, u64, i64, vp, i64,
@@ -127,6 +133,13 @@ def payload_bytes_entrywise(lengths: Sequence[int], k_cap: int) -> int:
     n = len(lengths)
     arr = (ctypes.c_int64 * n)(*[int(x) for x in lengths])
     return int(lib.atomo_payload_bytes_entrywise(arr, n, int(k_cap)))
+
+
+def payload_bytes_entrywise_compact(lengths: Sequence[int], k_cap: int, sat_cap: int) -> int:
+    lib = load_library()
+    n = len(lengths)
+    arr = (ctypes.c_int64 * n)(*[int(x) for x in lengths])
+    return int(lib.atomo_payload_bytes_entrywise_compact(arr, n, int(k_cap), int(sat_cap)))
 
 
 def default_k_cap(s: float, n_atoms: int) -> int:
@@ -172,6 +185,8 @@ class Payload:
     shapes: List[tuple]          # (rows, cols) per layer; entry-wise: (1, n)
     k_cap: int
     ctx: "Atomo"
+    ew_format: int = 0           # entry-wise: EW_EXPLICIT or EW_COMPACT
+    sat_cap: int = 0             # compact entry-wise: capacity of the saturated list
 
     @property
     def n_layers(self) -> int:
@@ -191,6 +206,25 @@ class Payload:
             nbytes = count * 4
             return raw[off: off + nbytes].cpu().numpy().view(dtype)
 
+        if self.kind == KIND_ENTRYWISE and self.ew_format == EW_COMPACT:
+            # expand the compact form to the explicit (idx, val) pair: entries carry the index inside their tile
+            # and the sign of +-c; the saturated atoms sit in a list of their own
+            n = self.shapes[l][1]
+            n_sat = int(h.n_sat)
+            k_list = k - n_sat
+            n_tiles = (n + EW_TILE - 1) // EW_TILE
+            ent = raw[h.off_idx: h.off_idx + 2 * k_list].cpu().numpy().view(np.uint16).astype(np.int64)
+            table = view(h.off_short, n_tiles + 1, np.uint32).astype(np.int64)
+            tile_of = np.searchsorted(table[1:], np.arange(k_list), side="right")
+            idx_u = tile_of * EW_TILE + (ent & (EW_TILE - 1))
+            val_u = np.where(ent & 0x8000, -np.float32(h.c), np.float32(h.c)).astype(np.float32)
+            idx_s = view(h.off_long, n_sat, np.uint32).astype(np.int64)
+            val_s = view(h.off_val, n_sat, np.float32)
+            idx = np.concatenate([idx_u, idx_s])
+            val = np.concatenate([val_u, val_s])
+            order = np.argsort(idx, kind="stable")
+            return dict(k=k, idx=idx[order].astype(np.uint32), val=val[order].astype(np.float32),
+                        n_sat_kept=n_sat, table=table)
         idx = view(h.off_idx, k, np.uint32).copy()
         val = view(h.off_val, k, np.float32).copy()
         if self.kind == KIND_ENTRYWISE:
@@ -241,6 +275,7 @@ class Atomo:
         h = ctypes.c_void_p()
         rc = self.lib.atomo_create(ctypes.byref(h), self.device)
         self._h = h
+        self._ew_format, self._ew_sat_cap = EW_EXPLICIT, 0
         if rc != 0:
             raise AtomoError(rc, "atomo_create", self._cuda_error())
 
@@ -323,7 +358,8 @@ class Atomo:
     def atomo_encode_entrywise(self, vecs: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,
                                k_cap: Optional[int] = None, payload: Optional[torch.Tensor] = None,
                                debug: bool = False, stream: Optional[torch.cuda.Stream] = None):
-        """Entry-wise ATOMO over a batch of flat fp32 CUDA tensors.  Returns (Payload, Debug | None)."""
+        """Entry-wise ATOMO over a batch of flat fp32 CUDA tensors.  Returns (Payload, Debug | None).
+        The payload format is the one last chosen with set_entrywise_format (explicit by default)."""
         n = len(vecs)
         arr = (_Vec * n)()
         lengths = []
@@ -334,7 +370,10 @@ class Atomo:
             lengths.append(int(g.numel()))
         if k_cap is None:
             k_cap = default_k_cap(s, max(lengths))
-        nbytes = payload_bytes_entrywise(lengths, k_cap)
+        if self._ew_format == EW_COMPACT:
+            nbytes = payload_bytes_entrywise_compact(lengths, k_cap, self._ew_sat_cap)
+        else:
+            nbytes = payload_bytes_entrywise(lengths, k_cap)
         if nbytes < 0:
             raise AtomoError(1, "atomo_payload_bytes_entrywise")
         dev = vecs[0].device
@@ -346,7 +385,8 @@ class Atomo:
                                              ctypes.c_void_p(payload.data_ptr()), payload.numel(),
                                              ctypes.byref(ds) if ds is not None else None, self._stream_ptr(stream))
         self._check(rc, "atomo_encode_entrywise")
-        return Payload(payload, KIND_ENTRYWISE, [(1, x) for x in lengths], int(k_cap), self), dbg
+        return Payload(payload, KIND_ENTRYWISE, [(1, x) for x in lengths], int(k_cap), self,
+                       ew_format=self._ew_format, sat_cap=self._ew_sat_cap), dbg
 
     def atomo_decode(self, payload: Payload, out: Optional[Sequence[torch.Tensor]] = None,
                      stream: Optional[torch.cuda.Stream] = None) -> List[torch.Tensor]:
@@ -428,6 +468,12 @@ class Atomo:
     def set_persistent_eig(self, enabled):
         """0 / False: one launch per Jacobi step; 1 / True: persistent cooperative launches; 2: clusters first (default)."""
         self._check(self.lib.atomo_set_persistent_eig(self._h, int(enabled)), "atomo_set_persistent_eig")
+
+    def set_entrywise_format(self, fmt: int, sat_cap: int = 0):
+        """EW_EXPLICIT (idx, val per kept atom) or EW_COMPACT (16-bit entry per kept atom with p < 1, one scalar c,
+        explicit values only for the atoms with p = 1, of which at most sat_cap per vector)."""
+        self._check(self.lib.atomo_set_entrywise_format(self._h, int(fmt), int(sat_cap)), "atomo_set_entrywise_format")
+        self._ew_format, self._ew_sat_cap = int(fmt), (int(sat_cap) if int(fmt) == EW_COMPACT else 0)
 
     def last_eig_scheme(self) -> int:
         return int(self.lib.atomo_last_eig_scheme(self._h))

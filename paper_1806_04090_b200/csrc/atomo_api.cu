@@ -31,6 +31,8 @@ struct atomo_ctx {
   bool tc_ok = false;                // tensor-map entry point found
   int eig_scheme = 2;                // eigen-solve launches: 0 = one per step, 1 = persistent (cooperative), 2 = clusters first
   int eig_scheme_used = -1;          // what the last spectral encode actually ran
+  int ew_format = ATOMO_EW_EXPLICIT; // payload format of entry-wise encodes
+  int64_t ew_sat_cap = 0;            // compact format: capacity of the saturated list
   int cluster_capacity[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // by log2(rp_max), -1 = not asked yet
   std::string err;
 };
@@ -104,17 +106,22 @@ uint64_t layout_spectral(const int32_t* rows, const int32_t* cols, int n_layers,
   return align_up(off, 16);
 }
 
-struct EwLayout { uint32_t kc; uint64_t off_idx, off_val, off_tiles; };
+struct EwLayout { uint32_t kc, sc; uint64_t off_idx, off_val, off_tiles, off_sat; };
 
-uint64_t layout_entrywise(const int64_t* n, int n_vecs, int64_t k_cap, std::vector<EwLayout>* out) {
+// explicit: idx u32[kc], val f32[kc], tile table.  compact: entries u16[kc], saturated values f32[sc], tile table,
+// saturated indices u32[sc] (sc = the saturated list's capacity, clamped to n).
+uint64_t layout_entrywise(const int64_t* n, int n_vecs, int64_t k_cap, bool compact, int64_t sat_cap,
+                          std::vector<EwLayout>* out) {
   uint64_t off = sizeof(atomo_payload_header) + (uint64_t)n_vecs * sizeof(atomo_layer_header);
   for (int l = 0; l < n_vecs; ++l) {
     const uint32_t kc = (uint32_t)std::min<int64_t>(k_cap, n[l]);
-    EwLayout lo;
+    EwLayout lo{};
     lo.kc = kc;
-    off = align_up(off, 16); lo.off_idx = off; off += (uint64_t)kc * 4;
-    off = align_up(off, 16); lo.off_val = off; off += (uint64_t)kc * 4;
+    lo.sc = compact ? (uint32_t)std::min<int64_t>(sat_cap, n[l]) : 0u;
+    off = align_up(off, 16); lo.off_idx = off; off += (uint64_t)kc * (compact ? 2 : 4);
+    off = align_up(off, 16); lo.off_val = off; off += (uint64_t)(compact ? lo.sc : kc) * 4;
     off = align_up(off, 16); lo.off_tiles = off; off += ((uint64_t)(n[l] + ATOMO_EW_TILE - 1) / ATOMO_EW_TILE + 1) * 4;
+    off = align_up(off, 16); lo.off_sat = off; off += (uint64_t)lo.sc * 4;
     if (out) out->push_back(lo);
   }
   return align_up(off, 16);
@@ -167,7 +174,21 @@ int64_t atomo_payload_bytes_spectral(const int32_t* rows, const int32_t* cols, i
 int64_t atomo_payload_bytes_entrywise(const int64_t* n, int32_t n_vecs, int64_t k_cap) {
   if (!n || n_vecs <= 0 || k_cap <= 0) return -1;
   for (int l = 0; l < n_vecs; ++l) if (n[l] <= 0 || n[l] >= (int64_t(1) << 32)) return -1;
-  return (int64_t)layout_entrywise(n, n_vecs, k_cap, nullptr);
+  return (int64_t)layout_entrywise(n, n_vecs, k_cap, false, 0, nullptr);
+}
+
+int64_t atomo_payload_bytes_entrywise_compact(const int64_t* n, int32_t n_vecs, int64_t k_cap, int64_t sat_cap) {
+  if (!n || n_vecs <= 0 || k_cap <= 0 || sat_cap < 0) return -1;
+  for (int l = 0; l < n_vecs; ++l) if (n[l] <= 0 || n[l] >= (int64_t(1) << 32)) return -1;
+  return (int64_t)layout_entrywise(n, n_vecs, k_cap, true, sat_cap, nullptr);
+}
+
+int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap) {
+  if (!ctx || (format != ATOMO_EW_EXPLICIT && format != ATOMO_EW_COMPACT)) return ATOMO_ERR_INVALID_ARG;
+  if (format == ATOMO_EW_COMPACT && sat_cap < 0) return ATOMO_ERR_INVALID_ARG;
+  ctx->ew_format = format;
+  ctx->ew_sat_cap = format == ATOMO_EW_COMPACT ? sat_cap : 0;
+  return ATOMO_OK;
 }
 
 int atomo_set_profiling(atomo_ctx* ctx, int enabled) {
@@ -560,7 +581,8 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     ns[l] = vecs[l].n;
   }
   std::vector<EwLayout> lay;
-  const uint64_t total = layout_entrywise(ns.data(), n_vecs, k_cap, &lay);
+  const bool compact = ctx->ew_format == ATOMO_EW_COMPACT;
+  const uint64_t total = layout_entrywise(ns.data(), n_vecs, k_cap, compact, ctx->ew_sat_cap, &lay);
   if ((int64_t)total > capacity_bytes) return ATOMO_ERR_CAPACITY;
   CK(cudaSetDevice(ctx->device));
   cudaStream_t st = (cudaStream_t)stream;
@@ -581,7 +603,11 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       EwVec& v = V[l];
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
-      v.n_ctas = ew_sample_pack_ctas(v.n_tiles);
+      v.n_ctas = ew_sample_pack_ctas(v.n_tiles, compact);
+      v.compact = compact ? 1 : 0; v.sat_cap = lay[l].sc;
+      v.ent = reinterpret_cast<uint16_t*>(pay + lay[l].off_idx);
+      v.sat_idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_sat);
+      v.sat_val = reinterpret_cast<float*>(pay + lay[l].off_val);
       v.n_words = (v.n + 31) / 32;
       const int64_t want_chunks = std::min<int64_t>(max_blocks, (v.n + 4095) / 4096);
       v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
@@ -610,11 +636,13 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   atomo_payload_header gh{};
   gh.magic = ATOMO_MAGIC; gh.version = ATOMO_VERSION; gh.kind = ATOMO_KIND_ENTRYWISE; gh.n_layers = (uint32_t)n_vecs;
   gh.total_bytes = total; gh.seed = seed; gh.step = step; gh.s = s;
+  gh.ew_format = (uint64_t)ctx->ew_format; gh.ew_sat_cap = compact ? (uint64_t)ctx->ew_sat_cap : 0;
   std::memcpy(hdr_blob.data(), &gh, sizeof(gh));
   for (int l = 0; l < n_vecs; ++l) {
     atomo_layer_header h{};
     h.rows = 1; h.cols = ns[l]; h.k_cap = lay[l].kc; h.status = ATOMO_OK;
     h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val; h.off_short = lay[l].off_tiles;
+    h.off_long = compact ? lay[l].off_sat : 0;
     std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
   }
   CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));

@@ -9,9 +9,12 @@
 //   pass 2   ew_sample_pack    : per chunk of tiles: p_i = |g_i| (s-n_s)/T, Philox word, keep bit -> mask words
 //                                and counts; the counts of the earlier chunks are added (one bounded wait, no
 //                                chain); ordered compaction from the mask words: idx ascending, val = g_i / p_i;
-//                                the last chunk writes k, the capacity check and the header
+//                                the last chunk writes k, the capacity check and the header.  Compact format
+//                                (the ternary form of Section 4): a kept atom with p < 1 weighs sign(g_i) c, so
+//                                it travels as a 16-bit entry (index inside its tile, sign bit); the atoms with
+//                                p = 1 keep (idx, val) in a list of their own
 //   decode   ew_decode         : zero-fill with vector stores, then the tile's kept values (per-tile
-//                                offsets travel in the payload)
+//                                offsets travel in the payload), either format
 #include <algorithm>
 
 #include <cooperative_groups.h>
@@ -155,30 +158,17 @@ constexpr uint32_t kChunkSpinLimit = 1u << 20;
 constexpr int kEwMaxTilesPerCta = 64;
 constexpr int kEwWordsPerTile = kEwTile / 32;
 
-__global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+// Phase 1 of the sample / pack kernel over the chunk's tiles: keep bits into the mask words, kept atoms counted per
+// tile.  SAT also records which kept atoms are saturated (a second mask and count; the compact format of a vector
+// that is not s-balanced needs them).
+template <bool SAT>
+__device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key, const uint32_t kind_step,
+                                             const int64_t tile0, const int n_my, const float scale, const float theta,
+                                             const bool dead, const bool aligned, uint32_t* s_mask, uint32_t* s_sat,
+                                             uint32_t* s_tcnt, uint32_t* s_tsat) {
   constexpr int kIts = kEwTile / (kEwThreads * 4);
-  constexpr int kWarps = kEwThreads / kWarp;
-  extern __shared__ uint32_t s_mask[];            // [tiles_per_cta][128] mask words of the chunk
-  __shared__ uint32_t s_tcnt[kEwMaxTilesPerCta];  // kept atoms per tile, then their exclusive prefix
-  __shared__ uint32_t s_chunk;
-  __shared__ unsigned long long s_base;           // kept atoms before this chunk
-  __shared__ uint32_t s_wsum[kWarps];
-  __shared__ int s_fail;
-  const EwState* st = v.state;
-  const float scale = st->scale, theta = st->theta_f, c = st->c;
+  const int tid = threadIdx.x, lane = tid % kWarp;
   const float scale32 = scale * 4294967296.0f;    // exact: a power-of-two factor
-  const bool dead = st->nonfinite != 0;
-  const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
-  const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
-  const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;   // the first `rem` chunks have q + 1 tiles
-  if (tid == 0) { s_chunk = atomicAdd(v.ticket, 1u); s_base = 0ull; s_fail = 0; }
-  if (tid < kEwMaxTilesPerCta) s_tcnt[tid] = 0u;
-  __syncthreads();
-  const uint32_t chunk = s_chunk;
-  const int64_t tile0 = (int64_t)chunk * q + min((int64_t)chunk, rem);
-  const int n_my = (int)(q + ((int64_t)chunk < rem ? 1 : 0));
-
-  // ---- phase 1 ----
   for (int tl = 0; tl < n_my; ++tl) {
     const uint32_t tile = (uint32_t)(tile0 + tl);
     const int64_t tile_base = (int64_t)tile * kEwTile;
@@ -190,7 +180,7 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
       x[it] = full ? __ldg(reinterpret_cast<const float4*>(v.g + i))
                    : (i < v.n ? load4(v.g, i, v.n, aligned) : make_float4(0.f, 0.f, 0.f, 0.f));
     }
-    uint32_t kept = 0;
+    uint32_t kept = 0, kept_sat = 0;
 #pragma unroll
     for (int it = 0; it < kIts; ++it) {
       const int64_t i = tile_base + ((int64_t)it * kEwThreads + tid) * 4;
@@ -198,18 +188,20 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
       const uint4 wd = philox4x32_10(make_uint4(tile * (uint32_t)(kEwTile / 4) + (uint32_t)(it * kEwThreads + tid), 0u, v.layer, kind_step), key);
       const float a[4] = {fabsf(x[it].x), fabsf(x[it].y), fabsf(x[it].z), fabsf(x[it].w)};
       const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
-      uint32_t nb = 0;
+      uint32_t nb = 0, sb = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         // p = 1 if saturated, else min(a scale, 1); keep iff p >= 1 or word < floor(p 2^32).  a scale32 is the
         // same product times 2^32 (exact), and the truncating conversion gives the floor.
         const float t = a[j] * scale32;
-        const bool one = a[j] > theta || t >= 4294967296.0f;
+        const bool sat = a[j] > theta;
+        const bool one = sat || t >= 4294967296.0f;
         const bool keep = one || ww[j] < __float2uint_rz(t);
-        if (keep && (full || i + j < v.n)) nb |= 1u << j;
+        if (keep && (full || i + j < v.n)) { nb |= 1u << j; if (SAT && sat) sb |= 1u << j; }
       }
-      if (dead) nb = 0;
+      if (dead) { nb = 0; sb = 0; }
       kept += __popc(nb);
+      if (SAT) kept_sat += __popc(sb);
       if (v.prob_out != nullptr && i < v.n) {
         float pp[4];
 #pragma unroll
@@ -224,28 +216,78 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
       word |= __shfl_xor_sync(0xffffffffu, word, 1);
       word |= __shfl_xor_sync(0xffffffffu, word, 2);
       word |= __shfl_xor_sync(0xffffffffu, word, 4);
+      uint32_t sword = 0;
+      if (SAT) {
+        sword = sb << (4 * (tid & 7));
+        sword |= __shfl_xor_sync(0xffffffffu, sword, 1);
+        sword |= __shfl_xor_sync(0xffffffffu, sword, 2);
+        sword |= __shfl_xor_sync(0xffffffffu, sword, 4);
+      }
       if ((tid & 7) == 0) {
         const int wl = it * (kEwThreads / 8) + (tid >> 3);
         s_mask[tl * kEwWordsPerTile + wl] = word;
+        if (SAT) s_sat[tl * kEwWordsPerTile + wl] = sword;
         const int64_t widx = (tile_base >> 5) + wl;
         if (widx < v.n_words) v.mask_words[widx] = word;
       }
     }
     kept = warp_sum(kept);
     if (lane == 0 && kept) atomicAdd(&s_tcnt[tl], kept);
+    if (SAT) {
+      kept_sat = warp_sum(kept_sat);
+      if (lane == 0 && kept_sat) atomicAdd(&s_tsat[tl], kept_sat);
+    }
   }
+}
+
+// COMPACT: the payload takes, per kept atom with p < 1, a 16-bit entry (index inside the tile, sign bit) and, per
+// atom with p = 1, index and value in a list of its own; both ascending.  The chunk's status word then carries the
+// saturated count in bits 32..62 beside the total, and the kernel keeps a second bit mask (saturated and kept).
+template <bool COMPACT>
+__global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+  constexpr int kWarps = kEwThreads / kWarp;
+  extern __shared__ uint32_t s_mask[];            // [tiles_per_cta][128] mask words of the chunk (COMPACT: then the saturated masks)
+  __shared__ uint32_t s_tcnt[kEwMaxTilesPerCta];  // kept atoms per tile, then their exclusive prefix
+  __shared__ uint32_t s_tsat[kEwMaxTilesPerCta];  // the same for the saturated kept atoms (COMPACT)
+  __shared__ uint32_t s_chunk, s_chunk_sat;
+  __shared__ unsigned long long s_base;           // kept atoms before this chunk (COMPACT: saturated ones in bits 32..62)
+  __shared__ uint32_t s_wsum[kWarps];
+  __shared__ int s_fail;
+  const EwState* st = v.state;
+  const float scale = st->scale, theta = st->theta_f, c = st->c;
+  const bool dead = st->nonfinite != 0;
+  const bool any_sat = COMPACT && st->n_sat != 0;   // an s-balanced vector (Lemma 3) skips the saturated bookkeeping
+  const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
+  const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
+  const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;   // the first `rem` chunks have q + 1 tiles
+  if (tid == 0) { s_chunk = atomicAdd(v.ticket, 1u); s_base = 0ull; s_fail = 0; }
+  if (tid < kEwMaxTilesPerCta) { s_tcnt[tid] = 0u; s_tsat[tid] = 0u; }
+  __syncthreads();
+  const uint32_t chunk = s_chunk;
+  const int64_t tile0 = (int64_t)chunk * q + min((int64_t)chunk, rem);
+  const int n_my = (int)(q + ((int64_t)chunk < rem ? 1 : 0));
+  uint32_t* s_sat = s_mask + (size_t)(q + (rem ? 1 : 0)) * kEwWordsPerTile;   // COMPACT only
+
+  // ---- phase 1 ----
+  if (any_sat) ew_keep_bits<true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
+  else ew_keep_bits<false>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
   __syncthreads();
 
   // ---- chunk count out, counts of the earlier chunks in ----
   if (w == 0) {
-    uint32_t total = 0;
-    for (int t = lane; t < n_my; t += kWarp) total += s_tcnt[t];
-    total = warp_sum(total);
+    uint32_t total = 0, total_sat = 0;
+    for (int t = lane; t < n_my; t += kWarp) { total += s_tcnt[t]; total_sat += s_tsat[t]; }
+    total = warp_sum(total); total_sat = warp_sum(total_sat);
     if (lane == 0) {
-      *(volatile unsigned long long*)(v.tile_status + chunk) = kFlagReady | (unsigned long long)total;
-      uint32_t run = 0;                                   // exclusive prefix over the chunk's tiles
-      for (int t = 0; t < n_my; ++t) { const uint32_t cnt = s_tcnt[t]; s_tcnt[t] = run; run += cnt; }
-      s_chunk = total;                                    // reuse: the chunk's count
+      *(volatile unsigned long long*)(v.tile_status + chunk) =
+          kFlagReady | ((unsigned long long)total_sat << 32) | (unsigned long long)total;
+      uint32_t run = 0, run_sat = 0;                      // exclusive prefixes over the chunk's tiles
+      for (int t = 0; t < n_my; ++t) {
+        const uint32_t cnt = s_tcnt[t]; s_tcnt[t] = run; run += cnt;
+        const uint32_t cs = s_tsat[t]; s_tsat[t] = run_sat; run_sat += cs;
+      }
+      s_chunk = total;                                    // reuse: the chunk's counts
+      s_chunk_sat = total_sat;
     }
   }
   unsigned long long before = 0;
@@ -255,27 +297,33 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
     uint32_t spins = 0;
     do { sv = *(volatile const unsigned long long*)(v.tile_status + cidx); } while (!(sv & kFlagReady) && ++spins <= kChunkSpinLimit);
     if (!(sv & kFlagReady)) fail = 1;
-    before += sv & ~kFlagReady;
+    before += sv & ~kFlagReady;                           // totals < 2^32 in all: the two fields never mix
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
   if (lane == 0 && before) atomicAdd(&s_base, before);
   if (fail) s_fail = 1;
   __syncthreads();
-  const uint64_t base = s_base;
+  const uint64_t base_all = s_base & 0xFFFFFFFFull;       // kept atoms before this chunk
+  const uint64_t base_sat = s_base >> 32;                 // of them saturated (0 unless COMPACT)
+  const uint64_t base = COMPACT ? base_all - base_sat : base_all;   // position of the chunk's first list entry
   const uint32_t total = s_chunk;
   if (tid == 0) {
     if (s_fail) raise_status(v.hdr, ATOMO_ERR_TIMEOUT);
-    for (int t = 0; t < n_my; ++t) v.tile_table[tile0 + t] = (uint32_t)min(base + s_tcnt[t], (uint64_t)0xFFFFFFFFull);
+    for (int t = 0; t < n_my; ++t)
+      v.tile_table[tile0 + t] = (uint32_t)min(base + s_tcnt[t] - (COMPACT ? s_tsat[t] : 0u), (uint64_t)0xFFFFFFFFull);
     if (tile0 + n_my == v.n_tiles) {                      // the last chunk knows k: capacity check, layer header
-      const uint64_t k = base + total;
+      const uint64_t k = base_all + total;
+      const uint64_t k_sat = base_sat + s_chunk_sat;
+      const uint64_t k_list = COMPACT ? k - k_sat : k;    // entries of the idx / entry list
       atomo_layer_header* h = v.hdr;
       h->n_sat = st->n_sat; h->c = st->c; h->l1 = st->T0; h->sweeps = st->rounds;
       if (st->nonfinite) raise_status(h, ATOMO_ERR_NONFINITE);
-      else if (k > (uint64_t)v.k_cap) raise_status(h, ATOMO_ERR_CAPACITY);
+      else if (k_list > (uint64_t)v.k_cap || (COMPACT && k_sat > (uint64_t)v.sat_cap)) raise_status(h, ATOMO_ERR_CAPACITY);
       const bool ok = *(volatile uint32_t*)&h->status == ATOMO_OK;
       h->k = ok ? (uint32_t)k : 0u;
-      v.tile_table[v.n_tiles] = ok ? (uint32_t)k : 0u;
+      if (COMPACT) h->n_sat = ok ? (uint32_t)k_sat : 0u;  // the length of the saturated list
+      v.tile_table[v.n_tiles] = ok ? (uint32_t)k_list : 0u;
     }
   }
   if (total == 0) return;
@@ -284,7 +332,9 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
   for (int tl = 0; tl < n_my; ++tl) {
     const int64_t tile_base = (tile0 + tl) * (int64_t)kEwTile;
     const uint32_t word = tid < kEwWordsPerTile ? s_mask[tl * kEwWordsPerTile + tid] : 0u;
-    const uint32_t pc = __popc(word);
+    const uint32_t sword = (any_sat && tid < kEwWordsPerTile) ? s_sat[tl * kEwWordsPerTile + tid] : 0u;
+    // COMPACT: two counts in one scan, list entries in the low half and saturated atoms in the high half (<= 4096 each)
+    const uint32_t pc = COMPACT ? (__popc(word & ~sword) | (__popc(sword) << 16)) : __popc(word);
     uint32_t inc = pc;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
@@ -293,19 +343,39 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
     __syncthreads();
     uint32_t woff = inc - pc;
     for (int i = 0; i < w; ++i) woff += s_wsum[i];
-    uint64_t pos = base + s_tcnt[tl] + woff;
-    uint32_t m = word;
-    while (m) {
-      const int bpos = __ffs(m) - 1;
-      m &= m - 1;
-      const int64_t i = tile_base + tid * 32 + bpos;
-      if (pos < (uint64_t)v.k_cap) {
-        const float g = __ldg(v.g + i);
-        // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) T / (s - n_s)
-        v.idx[pos] = (uint32_t)i;
-        v.val[pos] = (fabsf(g) > theta) ? g : copysignf(c, g);
+    if (!COMPACT) {
+      uint64_t pos = base + s_tcnt[tl] + woff;
+      uint32_t m = word;
+      while (m) {
+        const int bpos = __ffs(m) - 1;
+        m &= m - 1;
+        const int64_t i = tile_base + tid * 32 + bpos;
+        if (pos < (uint64_t)v.k_cap) {
+          const float g = __ldg(v.g + i);
+          // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) T / (s - n_s)
+          v.idx[pos] = (uint32_t)i;
+          v.val[pos] = (fabsf(g) > theta) ? g : copysignf(c, g);
+        }
+        ++pos;
       }
-      ++pos;
+    } else {
+      uint64_t pos = base + (s_tcnt[tl] - s_tsat[tl]) + (woff & 0xFFFFu);
+      uint64_t pos_sat = base_sat + s_tsat[tl] + (woff >> 16);
+      uint32_t m = word;
+      while (m) {
+        const int bpos = __ffs(m) - 1;
+        m &= m - 1;
+        const uint32_t off = (uint32_t)(tid * 32 + bpos);
+        const float g = __ldg(v.g + tile_base + off);
+        if ((sword >> bpos) & 1u) {
+          if (pos_sat < (uint64_t)v.sat_cap) { v.sat_idx[pos_sat] = (uint32_t)(tile_base + off); v.sat_val[pos_sat] = g; }
+          ++pos_sat;
+        } else {
+          // value sign(g) c: the entry carries g's sign bit (what copysignf reads in the explicit format)
+          if (pos < (uint64_t)v.k_cap) v.ent[pos] = (uint16_t)(off | ((__float_as_uint(g) >> 31) << 15));
+          ++pos;
+        }
+      }
     }
   }
 }
@@ -319,13 +389,21 @@ __device__ __forceinline__ uint32_t lower_bound_u32(const uint32_t* __restrict__
 
 __global__ void __launch_bounds__(kEwThreads) ew_decode_kernel(EwDecode d) {
   const atomo_layer_header* h = d.hdr;
-  const bool ok = d.ghdr->magic == ATOMO_MAGIC && d.ghdr->kind == ATOMO_KIND_ENTRYWISE &&
-                  h->rows == 1 && h->cols == d.n && h->k <= h->k_cap;
+  const bool compact = d.ghdr->ew_format == ATOMO_EW_COMPACT;
+  const uint32_t sat_cap = compact ? (uint32_t)min(d.ghdr->ew_sat_cap, (uint64_t)0xFFFFFFFFull) : 0u;
+  bool ok = d.ghdr->magic == ATOMO_MAGIC && d.ghdr->kind == ATOMO_KIND_ENTRYWISE && d.ghdr->ew_format <= ATOMO_EW_COMPACT &&
+            h->rows == 1 && h->cols == d.n;
+  if (compact) ok = ok && h->n_sat <= h->k && h->n_sat <= sat_cap && h->k - h->n_sat <= h->k_cap;
+  else ok = ok && h->k <= h->k_cap;
   if (!ok && blockIdx.x == 0 && threadIdx.x == 0) raise_status(const_cast<atomo_layer_header*>(h), ATOMO_ERR_PAYLOAD);
-  const uint32_t k = ok ? h->k : 0u;
+  const uint32_t n_sat = (ok && compact) ? h->n_sat : 0u;
+  const uint32_t k = ok ? h->k - n_sat : 0u;               // entries of the idx / entry list
+  const float c = h->c;
   const uint32_t* idx = reinterpret_cast<const uint32_t*>(d.payload + h->off_idx);
+  const uint16_t* ent = reinterpret_cast<const uint16_t*>(d.payload + h->off_idx);
   const float* val = reinterpret_cast<const float*>(d.payload + h->off_val);
-  const uint32_t* table = reinterpret_cast<const uint32_t*>(d.payload + h->off_short);   // kept atoms before each tile
+  const uint32_t* table = reinterpret_cast<const uint32_t*>(d.payload + h->off_short);   // list entries before each tile
+  const uint32_t* sat_idx = reinterpret_cast<const uint32_t*>(d.payload + h->off_long);
   const int64_t n_tiles = (d.n + kEwTile - 1) / kEwTile;
   const bool vec = (reinterpret_cast<uintptr_t>(d.out) & 15u) == 0;
   // a CTA walks over tiles: zero-fill with vector stores, barrier, then the tile's few kept values
@@ -343,9 +421,25 @@ __global__ void __launch_bounds__(kEwThreads) ew_decode_kernel(EwDecode d) {
     uint32_t lo = 0, hi = 0;
     if (k) { lo = min(__ldg(table + tile), k); hi = min(__ldg(table + tile + 1), k); }
     __syncthreads();                                     // zeros are ordered before the values below
-    for (uint32_t j = lo + threadIdx.x; j < hi; j += kEwThreads) {
-      const uint32_t i = __ldg(idx + j);
-      if ((int64_t)i >= tile_base && (int64_t)i < tile_base + kEwTile && (int64_t)i < d.n) d.out[i] = __ldg(val + j);
+    if (!compact) {
+      for (uint32_t j = lo + threadIdx.x; j < hi; j += kEwThreads) {
+        const uint32_t i = __ldg(idx + j);
+        if ((int64_t)i >= tile_base && (int64_t)i < tile_base + kEwTile && (int64_t)i < d.n) d.out[i] = __ldg(val + j);
+      }
+    } else {
+      for (uint32_t j = lo + threadIdx.x; j < hi; j += kEwThreads) {
+        const uint32_t e = __ldg(ent + j);
+        const int64_t off = e & (uint32_t)(kEwTile - 1);
+        if (off < left) out[off] = (e & 0x8000u) ? -c : c;
+      }
+      if (n_sat) {                                       // the saturated atoms of this tile (ascending list)
+        const uint32_t s_lo = lower_bound_u32(sat_idx, n_sat, (uint64_t)tile_base);
+        for (uint32_t j = s_lo + threadIdx.x; j < n_sat; j += kEwThreads) {
+          const int64_t off = (int64_t)__ldg(sat_idx + j) - tile_base;
+          if (off >= kEwTile) break;
+          if (off >= 0 && off < left) out[off] = __ldg(val + j);
+        }
+      }
     }
   }
 }
@@ -396,20 +490,30 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st) {
   void* args[] = {&vv, &ss};
   return (int)cudaLaunchCooperativeKernel((const void*)ew_solve_kernel, dim3(v.n_chunks), dim3(kEwThreads), args, 0, st);
 }
-int ew_sample_pack_ctas(int64_t n_tiles) {
-  // one wave of chunks when it fits (at most 64 tiles per chunk): tiles spread evenly, sizes differ by at most one
+int ew_sample_pack_ctas(int64_t n_tiles, bool compact) {
+  // one wave of chunks when it fits (at most 64 tiles per chunk, 32 for the compact format): tiles spread evenly, sizes differ by at most one
   int dev = 0, sms = 148, per_sm = 4;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel, kEwThreads,
-                                                    16 * kEwWordsPerTile * sizeof(uint32_t)) != cudaSuccess || per_sm < 1)
-    per_sm = 4;
+  const cudaError_t e = compact
+      ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel<true>, kEwThreads,
+                                                      32 * kEwWordsPerTile * sizeof(uint32_t))
+      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel<false>, kEwThreads,
+                                                      16 * kEwWordsPerTile * sizeof(uint32_t));
+  if (e != cudaSuccess || per_sm < 1) per_sm = 4;
   const int64_t wave = (int64_t)sms * per_sm;
-  const int64_t min_ctas = (n_tiles + kEwMaxTilesPerCta - 1) / kEwMaxTilesPerCta;
+  const int max_tiles = compact ? kEwMaxTilesPerCta / 2 : kEwMaxTilesPerCta;   // compact: two masks per tile in shared memory
+  const int64_t min_ctas = (n_tiles + max_tiles - 1) / max_tiles;
   return (int)std::max<int64_t>(1, std::max(min_ctas, std::min(n_tiles, wave)));
 }
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
   const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
-  ew_sample_pack_kernel<<<(unsigned)v.n_ctas, kEwThreads, (size_t)most * kEwWordsPerTile * sizeof(uint32_t), st>>>(v, key, kind_step);
+  const size_t smem = (size_t)most * kEwWordsPerTile * sizeof(uint32_t);
+  if (v.compact) {
+    // two masks per tile; chunks of at most 32 tiles keep them inside the default 48 KB of dynamic shared memory
+    ew_sample_pack_kernel<true><<<(unsigned)v.n_ctas, kEwThreads, 2 * smem, st>>>(v, key, kind_step);
+  } else {
+    ew_sample_pack_kernel<false><<<(unsigned)v.n_ctas, kEwThreads, smem, st>>>(v, key, kind_step);
+  }
 }
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {
   const int64_t tiles = (d.n + kEwTile - 1) / kEwTile;

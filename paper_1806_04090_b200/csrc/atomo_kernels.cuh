@@ -34,6 +34,10 @@ struct EwVec {
   uint32_t* ticket;                                            // next chunk to hand out; zeroed per call
   uint32_t* tile_table;                                        // payload: kept atoms before each tile
   float* prob_out;                                             // debug or nullptr
+  // compact payload format (else compact = 0 and the rest unused)
+  int compact; uint32_t sat_cap;
+  uint16_t* ent;                                               // [k_cap] tile-local index | sign << 15 of kept atoms with p < 1
+  uint32_t* sat_idx; float* sat_val;                           // [sat_cap] atoms with p = 1
 };
 
 struct EwDecode {
@@ -48,7 +52,7 @@ void launch_ew_decode(const EwDecode& d, cudaStream_t st);
 int ew_tile_elems();
 void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax, double* part_sum, float* part_max,
                   int n_ctas, cudaStream_t st);
-int ew_sample_pack_ctas(int64_t n_tiles);
+int ew_sample_pack_ctas(int64_t n_tiles, bool compact);
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)

@@ -48,6 +48,13 @@ def test_payload_size_queries(lib):
     assert b2 > b and b2 % 16 == 0
     e = api.payload_bytes_entrywise([4096], 100)
     assert e == 64 + 80 + 400 + 400 + 16       # + per-tile offset table (2 entries, 16-byte aligned)
+    # compact format: 2 bytes per entry, then values and indices of the saturated list (here 8 of them)
+    assert api.payload_bytes_entrywise_compact([4096], 100, 8) == 64 + 80 + 208 + 32 + 16 + 32
+    assert api.payload_bytes_entrywise_compact([4096], 100, 0) == 64 + 80 + 208 + 16
+    assert api.payload_bytes_entrywise_compact([4096], 100, 10 ** 9) == api.payload_bytes_entrywise_compact([4096], 100, 4096)
+    assert api.payload_bytes_entrywise_compact([100], 10, -1) == -1
+    n, k_cap = 25_600_000, 300_000                       # a quarter of the explicit format's bytes per kept atom
+    assert api.payload_bytes_entrywise_compact([n], k_cap, 0) < 0.3 * api.payload_bytes_entrywise([n], k_cap)
     assert api.payload_bytes_entrywise([0], 10) == -1
     assert api.payload_bytes_entrywise([2 ** 32], 10) == -1
     assert api.payload_bytes_spectral([(0, 5)], 10) == -1
