@@ -466,7 +466,8 @@ class Atomo:
         return {k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)}
 
     def set_persistent_eig(self, enabled):
-        """0 / False: one launch per Jacobi step; 1 / True: persistent cooperative launches; 2: clusters first (default)."""
+        """Eigen-solver scheme.  0 / False: Jacobi, one launch per step; 1 / True: persistent cooperative launches;
+        2: Jacobi in thread-block clusters first; 3 (default): tridiagonal route first (short sides up to 512)."""
         self._check(self.lib.atomo_set_persistent_eig(self._h, int(enabled)), "atomo_set_persistent_eig")
 
     def set_entrywise_format(self, fmt: int, sat_cap: int = 0):

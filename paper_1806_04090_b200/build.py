@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libatomo_b200.so")
-SOURCES = ["atomo_api.cu", "atomo_entrywise.cu", "atomo_spectral.cu", "atomo_eig.cu", "atomo_tc.cu", "atomo_static.cu", "atomo_average.cu"]
+SOURCES = ["atomo_api.cu", "atomo_entrywise.cu", "atomo_spectral.cu", "atomo_eig.cu", "atomo_tc.cu", "atomo_static.cu", "atomo_average.cu", "atomo_tridiag.cu"]
 HEADERS = ["atomo_common.cuh", "atomo_kernels.cuh"]
 
 

@@ -29,7 +29,8 @@ struct atomo_ctx {
   int refine_min_short = 2048;       // layers with at least this short side get the sigma refinement pass
   bool tc_gram = true;               // Gram matrix on tcgen05 where the layer's layout allows it
   bool tc_ok = false;                // tensor-map entry point found
-  int eig_scheme = 2;                // eigen-solve launches: 0 = one per step, 1 = persistent (cooperative), 2 = clusters first
+  int eig_scheme = 3;                // eigen-solve: 0 = Jacobi, one launch per step, 1 = persistent (cooperative), 2 = clusters first, 3 = tridiagonal route first
+  int tri_clusters = -1;             // co-resident clusters of the tridiagonal reduction (-1 = not asked yet, 0 = unavailable)
   int eig_scheme_used = -1;          // what the last spectral encode actually ran
   int ew_format = ATOMO_EW_EXPLICIT; // payload format of entry-wise encodes
   int64_t ew_sat_cap = 0;            // compact format: capacity of the saturated list
@@ -222,7 +223,7 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
 int atomo_last_eig_scheme(atomo_ctx* ctx) { return ctx ? ctx->eig_scheme_used : -1; }
 
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
-  if (!ctx || enabled < 0 || enabled > 2) return ATOMO_ERR_INVALID_ARG;
+  if (!ctx || enabled < 0 || enabled > 3) return ATOMO_ERR_INVALID_ARG;
   ctx->eig_scheme = enabled;
   return ATOMO_OK;
 }
@@ -328,7 +329,16 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   }
   // Cluster form first: every layer's block pairs inside one 16-CTA cluster, blocks exchanged through
   // distributed shared memory (layers of up to 16 block pairs, route 1).
-  bool cluster_form = ctx->eig_scheme == 2 && ctx->eig_mode != 0;
+  // Tridiagonal route first: eigenvalues of every atom from T = Q^T A Q, vectors for the kept atoms only (short side
+  // <= 512, no per-atom refinement, no request for the whole short-side basis).
+  bool tri_form = ctx->eig_scheme == 3 && ctx->eig_mode != 0 && !(dbg && dbg->short_vecs);
+  for (int l = 0; l < n_layers && tri_form; ++l) tri_form = L[l].rp <= sp_tridiag_max_rp() && !L[l].refine;
+  if (tri_form) {
+    if (ctx->tri_clusters < 0) ctx->tri_clusters = sp_configure_tridiag();
+    if (ctx->tri_clusters < 1) tri_form = false;
+  }
+  for (int l = 0; l < n_layers; ++l) L[l].tri = tri_form ? 1 : 0;
+  bool cluster_form = !tri_form && ctx->eig_scheme >= 2 && ctx->eig_mode != 0;
   for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
   if (cluster_form) {
     int lg = 0;
@@ -336,7 +346,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (ctx->cluster_capacity[lg] < 0) ctx->cluster_capacity[lg] = sp_jacobi_cluster_capacity(rp_max);
     if (ctx->cluster_capacity[lg] < 1) cluster_form = false;
   }
-  for (int l = 0; l < n_layers; ++l) L[l].lam_ready = cluster_form ? 1 : 0;
+  for (int l = 0; l < n_layers; ++l) L[l].lam_ready = (cluster_form || tri_form) ? 1 : 0;
   // tensor-core Gram tiles: while the batch has fewer CTAs than the GPU has SMs, the K range of the layers with the
   // longest rows is split over 2 or 4 CTAs per tile (at least 16 stages of 32 columns per part)
   {
@@ -402,6 +412,9 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
         d.gram_part = A.take<float>(d.tc && d.gram_split > 1
                                         ? (size_t)tt * (tt + 1) / 2 * d.gram_split * sp_tc_tile() * sp_tc_tile() : 0);
       }
+      d.td_d = A.take<double>(d.tri ? d.rp : 0); d.td_e = A.take<double>(d.tri ? d.rp : 0);
+      d.td_tau = A.take<double>(d.tri ? d.rp : 0); d.lam64 = A.take<double>(d.tri ? d.rp : 0);
+      d.td_V = A.take<double>(d.tri ? (size_t)d.r * d.r : 0);
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
       d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);
@@ -414,12 +427,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     // zero-filled region: rotation counters and the X matrices
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
     size_t z0 = A.off;
-    for (int l = 0; l < n_layers; ++l) { L[l].rot_count = A.take<uint32_t>(max_sweeps); L[l].step_bar = A.take<uint32_t>(1); }
+    for (int l = 0; l < n_layers; ++l) { L[l].rot_count = A.take<uint32_t>(max_sweeps); L[l].step_bar = A.take<uint32_t>(1); L[l].vec_ticket = A.take<uint32_t>(1); }
     for (int l = 0; l < n_layers; ++l) {
       const int tt = (L[l].r + sp_tc_tile() - 1) / sp_tc_tile();
       L[l].gram_ticket = A.take<uint32_t>(L[l].tc && L[l].gram_split > 1 ? (size_t)tt * (tt + 1) / 2 : 0);
     }
-    for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>((size_t)L[l].rp * L[l].ldx);
+    for (int l = 0; l < n_layers; ++l) L[l].X = A.take<float>(L[l].tri ? 0 : (size_t)L[l].rp * L[l].ldx);
     zero_beg = zb; zero_bytes = A.off - z0;
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
@@ -462,7 +475,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
   launch_sp_gram_tc(d_layers, d_maps, d_tc, (int)tc_tiles.size(), d_flag + 1, st);
   launch_sp_scale(d_layers, n_layers, st);
-  if (ctx->eig_mode != 0) {
+  if (ctx->eig_mode != 0 && !tri_form) {
     const int ec = launch_sp_cholesky(d_layers, n_layers, rp_max, st);
     if (ec != 0) return fail_cuda(ctx, (cudaError_t)ec, "cudaLaunchKernelEx(cholesky)");
     const int e = launch_sp_cholesky_big(d_layers, d_chol, (int)chol_ctas.size(), chol_panels, st);
@@ -479,6 +492,31 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
+  if (tri_form) {
+    // layers packed into 16-CTA clusters, largest first (a layer takes rp / 32 consecutive ranks of one cluster)
+    const int per = sp_tridiag_cluster_ctas();
+    std::vector<int> order(n_layers);
+    for (int l = 0; l < n_layers; ++l) order[l] = l;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].rp > L[b].rp; });
+    std::vector<int> used;
+    std::vector<ClusterCta> ctas;
+    for (int l : order) {
+      const int nc = sp_tridiag_ctas_of(L[l].rp);
+      size_t c = 0;
+      while (c < used.size() && used[c] + nc > per) ++c;
+      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
+      for (int sl = 0; sl < nc; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], nc};
+      used[c] += nc;
+    }
+    CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
+    const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
+    launch_sp_bisect(d_layers, n_layers, r_max, st);
+    n_eig_launch = 2;
+    CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
+    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    flags_pending = true;                                  // the Gram kernel's bounded waits report at the end of the call
+  }
   if (cluster_form) {
     const int per = sp_jacobi_cluster_ctas();
     std::vector<int> order(n_layers);
@@ -503,12 +541,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     flags_pending = true;                                  // read at the end of the call, after everything is enqueued
   }
-  const int capacity = (!cluster_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
+  const int capacity = (!cluster_form && !tri_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
   int max_layer_pairs = 0;
   for (int l = 0; l < n_layers; ++l) max_layer_pairs = std::max(max_layer_pairs, L[l].nb / 2);
   const bool persistent = capacity > 0 && max_layer_pairs <= capacity;
-  ctx->eig_scheme_used = cluster_form ? 2 : (persistent ? 1 : 0);
-  if (cluster_form) {
+  ctx->eig_scheme_used = tri_form ? 3 : cluster_form ? 2 : (persistent ? 1 : 0);
+  if (cluster_form || tri_form) {
     // done above
   } else if (persistent) {
     // d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
@@ -554,9 +592,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S4: long-side vectors of the kept atoms ----
   stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);
+  if (tri_form) launch_sp_eigvec(d_layers, n_layers, rp_max, st);   // short-side vectors of the kept atoms
   launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), std::max(r_max_tall, 1), st);
   launch_sp_finish_atoms(d_layers, n_layers, k_cap_max, st);
-  stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, 2);
+  stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, tri_form ? 3 : 2);
   CK(cudaGetLastError());
   if (flags_pending) {
     // the one host wait of the persistent forms: the kernels' bounded waits report here

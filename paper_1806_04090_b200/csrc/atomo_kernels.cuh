@@ -89,6 +89,13 @@ struct SpLayer {
   int refine, refine_tiles;    // singular values from the projection norms; tiles along the long side
   float* row_inv;              // rp: 1 / norm of each short-side vector as stored in X
   float* refine_partials;      // [refine_tiles][rp] partial squared norms
+  // tridiagonal route (short side <= 512): T = Q^T A Q, eigenvalues by bisection, vectors of the kept atoms only
+  int tri;                     // this layer takes the tridiagonal route
+  double* td_d; double* td_e;  // rp each: diagonal and off-diagonal of T
+  double* td_tau;              // rp: beta_k of the reflectors H_k = I - beta_k v_k v_k^T
+  double* td_V;                // r x r: row k = v_k (zero up to index k)
+  double* lam64;               // rp: eigenvalues of T, ascending (scaled units); lam holds the same in fp32
+  uint32_t* vec_ticket;        // CTAs of the vector kernel that finished this layer; zeroed per call
 };
 
 struct SpDecodeLayer {
@@ -121,6 +128,14 @@ int sp_jacobi_cluster_max_rp();                                   // largest pad
 int sp_jacobi_cluster_capacity(int rp_max);                       // co-resident clusters (0: not available here)
 int launch_sp_jacobi_cluster(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, int max_sweeps,
                              float tol, cudaStream_t st);         // returns a cudaError_t
+// tridiagonal route (atomo_tridiag.cu)
+int sp_tridiag_max_rp();
+int sp_tridiag_cluster_ctas();
+int sp_tridiag_ctas_of(int rp);                                   // CTAs a layer of padded short side rp takes
+int sp_configure_tridiag();                                       // co-resident clusters (0: route not available)
+int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, cudaStream_t st);  // cudaError_t
+void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, cudaStream_t st);
+void launch_sp_eigvec(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
 int sp_cholesky_big_rows_per_cta();

@@ -397,6 +397,7 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   }
   __syncthreads();
   const uint32_t k = s_k;
+  if (L.tri) return;                       // tridiagonal route: the vectors of the kept atoms come from sp_eigvec_kernel
   // short-side vectors of the kept atoms, normalised: payload shortv[a][0..r)
   for (uint32_t a = w; a < k; a += kFinThreads / 32) {
     const int row = L.perm[L.idx[a]];

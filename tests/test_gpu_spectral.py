@@ -126,7 +126,7 @@ def test_eigen_launch_schemes_agree(atomo):
             got.append(([dbg.layer_sigma(l, min(m.shape)) for l, m in enumerate(mats)],
                         [pay.layer_arrays(l)["idx"].copy() for l in range(len(mats))]))
     finally:
-        atomo.set_persistent_eig(2)
+        atomo.set_persistent_eig(3)
     for other in got[1:]:
         for l in range(len(mats)):
             assert parity.rel(other[0][l], got[0][0][l]) <= 2e-6

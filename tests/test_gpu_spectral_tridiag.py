@@ -1,0 +1,190 @@
+"""GPU parity of the tridiagonal route of the spectral encoder (short sides up to 512: Householder reduction of the
+Gram matrix, all eigenvalues by bisection, vectors for the kept atoms only) against the fp64 oracle, and against the
+Jacobi route of the same library."""
+import numpy as np
+import pytest
+
+from paper_1806_04090_b200 import synth
+from tests import parity
+
+pytestmark = pytest.mark.gpu
+
+TRIDIAG, JACOBI_CLUSTERS = 3, 2
+
+
+@pytest.fixture(scope="module")
+def atomo():
+    import torch
+    from paper_1806_04090_b200 import api
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    a = api.Atomo(0)
+    yield a
+    a.close()
+
+
+def _encode(atomo, mats, s, seed, step=0, k_cap=None, pad_ld=0, scheme=TRIDIAG):
+    import torch
+    ts = []
+    for G in mats:
+        if pad_ld:
+            buf = torch.full((G.shape[0], G.shape[1] + pad_ld), 7.0, dtype=torch.float32, device="cuda")
+            buf[:, : G.shape[1]] = torch.from_numpy(G).cuda()
+            ts.append(buf[:, : G.shape[1]])
+        else:
+            ts.append(torch.from_numpy(G).cuda())
+    if k_cap is None:
+        k_cap = max(min(G.shape) for G in mats)
+    atomo.set_persistent_eig(scheme)
+    try:
+        pay, dbg = atomo.atomo_encode_spectral(ts, s, seed, step=step, k_cap=k_cap, debug=True)
+        assert atomo.last_eig_scheme() == scheme
+    finally:
+        atomo.set_persistent_eig(TRIDIAG)
+    return pay, dbg
+
+
+def _run(atomo, oracle, mats, s, seed, step=0, pad_ld=0, check_vectors=True):
+    pay, dbg = _encode(atomo, mats, s, seed, step, pad_ld=pad_ld)
+    hdrs = pay.headers()
+    outs = atomo.atomo_decode(pay)
+    encs = parity.oracle_spectral_batch(oracle, mats, s, seed, step)
+    report = []
+    n_same = 0
+    for l, G in enumerate(mats):
+        arr = pay.layer_arrays(l, hdrs)
+        out = outs[l].cpu().numpy().astype(np.float64)
+        same, _ = parity.check_spectral_layer(oracle, G, encs[l], hdrs[1][l], arr, dbg, l, out, report,
+                                              f"L{l}{G.shape}", check_vectors)
+        # this route computes the kept vectors one by one: they must still be orthonormal among themselves
+        # (the long-side vectors are back-projections: theirs is the orthogonality the fp32 Gram matrix allows for atoms
+        # with small sigma, as on the Jacobi route)
+        if arr["k"] > 1:
+            short, long_ = (arr["U"], arr["V"]) if G.shape[0] <= G.shape[1] else (arr["V"], arr["U"])
+            for M, tol in ((short.astype(np.float64), 2e-5), (long_.astype(np.float64), 2e-3)):
+                err = np.abs(M.T @ M - np.eye(arr["k"])).max()
+                assert err <= tol, f"L{l}{G.shape}: kept vectors not orthonormal ({err:.2e})"
+        n_same += same
+    print("\n".join(report))
+    print(f"layers with identical masks: {n_same}/{len(mats)}")
+    return pay, hdrs, encs
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_config1_spectral(atomo, oracle, seed):
+    _run(atomo, oracle, [synth.c1_spectral(seed)], 2.0, seed=11 + seed, step=1)
+
+
+@pytest.mark.parametrize("shape", [(1, 1), (1, 9), (7, 1), (2, 6), (3, 5), (5, 3), (10, 512), (64, 27), (33, 100),
+                                   (100, 33), (65, 130), (130, 257), (512, 700), (300, 2000)])
+def test_small_and_ragged_shapes(atomo, oracle, shape):
+    rng = np.random.default_rng(sum(shape))
+    G = synth.lowrank_plus_noise(rng, shape[0], shape[1], 1.0, noise_rel=0.05)
+    _run(atomo, oracle, [G], 1.5, seed=21)
+
+
+@pytest.mark.parametrize("s", [8.0, 40.0])
+def test_many_kept_atoms(atomo, oracle, s):
+    # larger budgets: dozens of kept atoms per layer, among them neighbours in the noise bulk
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(2, [L[1], L[6], L[10]])
+    _run(atomo, oracle, mats, s, seed=31, step=3)
+
+
+def test_saturating_budget(atomo, oracle):
+    G = synth.c2_resnet18(0, [synth.RESNET18_LAYERS[17]])[0]
+    pay, hdrs, encs = _run(atomo, oracle, [G], 2.0, seed=5)
+    assert hdrs[1][0].n_sat == 1 == encs[0]["n_s"]
+    # s >= number of atoms: everything kept, decode reproduces G (no sparsification)
+    pay, hdrs, _ = _run(atomo, oracle, [G], 10.0, seed=5)
+    assert hdrs[1][0].k == 10
+    out = atomo.atomo_decode(pay)[0].cpu().numpy()
+    assert parity.rel(out, G) <= 1e-5
+
+
+def test_all_atoms_kept_reproduces_the_matrix(atomo):
+    # s = r on a full-rank 96 x 200 matrix: every vector comes from the per-atom solver and the sum must be G
+    rng = np.random.default_rng(4)
+    G = rng.standard_normal((96, 200)).astype(np.float32)
+    pay, _ = _encode(atomo, [G], 96.0, seed=1)
+    assert pay.headers()[1][0].k == 96
+    out = atomo.atomo_decode(pay)[0].cpu().numpy()
+    assert parity.rel(out, G) <= 2e-5
+
+
+def test_rank_deficient_and_clustered_inputs(atomo, oracle):
+    ones = np.ones((6, 11), dtype=np.float32)          # single singular value sqrt(66)
+    hot = np.zeros((5, 8), dtype=np.float32); hot[0, 0] = 1.0
+    zero = np.zeros((4, 9), dtype=np.float32)
+    eye = np.eye(40, 64, dtype=np.float32)             # forty equal singular values: any orthonormal basis is right
+    pay, dbg = _encode(atomo, [ones, hot, zero, eye], 1.0, seed=3)
+    hdrs = pay.headers()
+    assert [h.status for h in hdrs[1]] == [0, 0, 0, 0]
+    sig = dbg.layer_sigma(0, 6)
+    assert abs(sig[0] - np.sqrt(66.0)) <= 1e-5 * np.sqrt(66.0) and np.all(sig[1:] <= 1e-3)
+    sig = dbg.layer_sigma(1, 5)
+    assert abs(sig[0] - 1.0) <= 1e-6 and np.all(sig[1:] <= 1e-6)
+    outs = atomo.atomo_decode(pay)
+    assert hdrs[1][2].k == 0 and not outs[2].any()
+    assert parity.rel(outs[0].cpu().numpy(), ones) <= 1e-5
+    assert parity.rel(outs[1].cpu().numpy(), hot) <= 1e-5
+    # identity block with every atom kept (s = 40): the kept vectors span the space whatever basis was picked
+    pay, _ = _encode(atomo, [eye], 40.0, seed=3)
+    assert pay.headers()[1][0].k == 40
+    arr = pay.layer_arrays(0)
+    U = arr["U"].astype(np.float64)
+    assert np.abs(U.T @ U - np.eye(40)).max() <= 1e-5
+    assert parity.rel(atomo.atomo_decode(pay)[0].cpu().numpy(), eye) <= 1e-5
+
+
+def test_batch_mixed_sizes_and_leading_dimension(atomo, oracle):
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(0, [L[0], L[1], L[5], L[6], L[9], L[17]])
+    _run(atomo, oracle, mats, 2.0, seed=3, step=4)
+    _run(atomo, oracle, mats[:3], 2.0, seed=13, pad_ld=5)
+
+
+def test_paper_reshape_family(atomo, oracle):
+    mats = synth.c2_paper_reshape(0)
+    _run(atomo, oracle, mats, 2.0, seed=17, step=1)
+
+
+def test_config2_full(atomo, oracle):
+    mats = synth.c2_resnet18(0)
+    _run(atomo, oracle, mats, 2.0, seed=2024, step=1)
+
+
+def test_routes_agree(atomo):
+    """Same singular values (to fp32 rounding of the Gram route), same masks, and the same decoded gradient where the
+    kept atoms are well separated."""
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(1, [L[0], L[1], L[5], L[9], L[13], L[17]])
+    got = []
+    for scheme in (JACOBI_CLUSTERS, TRIDIAG):
+        pay, dbg = _encode(atomo, mats, 2.0, seed=23, step=2, scheme=scheme)
+        assert [h.status for h in pay.headers()[1]] == [0] * len(mats)
+        got.append(([dbg.layer_sigma(l, min(m.shape)) for l, m in enumerate(mats)],
+                    [pay.layer_arrays(l)["idx"].copy() for l in range(len(mats))]))
+    for l in range(len(mats)):
+        assert parity.rel(got[1][0][l], got[0][0][l]) <= 2e-5
+        assert np.array_equal(got[1][1][l], got[0][1][l])
+
+
+def test_deterministic_and_fallback(atomo):
+    import torch
+    G = [synth.c1_spectral(4)]
+    p1, _ = _encode(atomo, G, 6.0, seed=9)
+    p2, _ = _encode(atomo, G, 6.0, seed=9)
+    a1, a2 = p1.layer_arrays(0), p2.layer_arrays(0)
+    assert a1["k"] == a2["k"] > 0
+    for key in ("idx", "coef", "U", "V"):
+        assert np.array_equal(a1[key], a2[key]), key
+    # a layer with a short side above 512 sends the whole batch to the Jacobi routes
+    big = np.random.default_rng(1).standard_normal((600, 700)).astype(np.float32)
+    t = [torch.from_numpy(G[0]).cuda(), torch.from_numpy(big).cuda()]
+    pay, _ = atomo.atomo_encode_spectral(t, 2.0, seed=9)
+    assert atomo.last_eig_scheme() in (1, 2) and atomo.payload_status(pay)[0] == 0
+    # non-finite input: reported, nothing kept
+    bad = G[0].copy(); bad[3, 7] = np.nan
+    pay, _ = atomo.atomo_encode_spectral([torch.from_numpy(bad).cuda()], 2.0, seed=9)
+    assert atomo.last_eig_scheme() == TRIDIAG
+    assert atomo.payload_status(pay) == (4, 0) and pay.headers()[1][0].k == 0
