@@ -7,7 +7,7 @@
 //                               of a 16-CTA cluster and stay in shared memory; per step the pivot column and the
 //                               product A v travel through distributed shared memory (two cluster barriers per
 //                               step).  The reflectors go to global memory for the back-transformation.
-//   sp_bisect_kernel          : all eigenvalues of T, one warp per eigenvalue: 8 rounds of 33-section on Sturm
+//   sp_bisect_kernel          : all eigenvalues of T, eight lanes per eigenvalue: 13 rounds of 9-section on Sturm
 //                               counts (division-free three-term recurrence with power-of-two rescaling).
 //   (sp_finalize_sample_kernel sorts, solves Algorithm 1 and draws, as for the other routes)
 //   sp_eigvec_kernel          : for the kept atoms only: eigenvector of T by a twisted factorisation with one
@@ -16,7 +16,7 @@
 //                               nearly equal eigenvalues are orthogonalised against each other at the end.
 //
 // Work per layer: about 2 r^3 fp64 flops for the reduction (full symmetric storage: matrix-vector product and
-// rank-two update of the trailing block), r^2 * 8 * 33 recurrence steps for the eigenvalues, O(r^2) per kept atom.
+// rank-two update of the trailing block), r^2 * 13 * 8 recurrence steps for the eigenvalues, O(r^2) per kept atom.
 #include <cooperative_groups.h>
 
 #include "atomo_kernels.cuh"
@@ -41,14 +41,60 @@ __device__ __forceinline__ bool finite64(double x) { return fabs(x) <= 1.7e308; 
 // ---- Householder tridiagonalisation ------------------------------------------------------------------------
 // Step k (k = 0 .. r-3) with x = A[k+1.., k]:  alpha = -sign(x_0) ||x||,  v = x - alpha e_1,  beta = 2 / v^T v,
 // H = I - beta v v^T;  p = beta A22 v,  K = beta/2 p^T v,  w = p - K v,  A22 -= v w^T + w v^T;  d_k = A[k][k],
-// e_k = alpha.  Row i of a layer lives in the CTA with group rank i mod nc at local row i / nc.
+// e_k = alpha.
+// Layout: a layer's rows are dealt cyclically to its nc = rp / 32 CTAs (row i: group rank i mod nc, local row i / nc);
+// a warp keeps its two rows in registers for the whole reduction.  Every vector of length rp (and every row of A) is
+// stored in the order q(j) = (j mod nc) * 32 + j / nc, so that the 32 entries a CTA owns are contiguous: one warp
+// sends them to a peer as one 256-byte store into the peer's shared memory.  A lane holds the entries q = lane + 32 m,
+// that is j = lane * nc + m.
+// One cluster barrier per step: with p_i the owners also send c_i = A[i][k+1] as it is after update k-1, from which
+// every CTA forms the next pivot column x_i = c_i - v_i w_{k+1} - w_i v_{k+1} itself, hence v_{k+1}; the update of
+// step k and the product A v_{k+1} then share one pass over the rows.
+__device__ __forceinline__ double tri_block_sum(double x, double* s_red, int lane, int w) {
+  x = warp_sum(x);
+  if (lane == 0) s_red[w] = x;
+  __syncthreads();
+  double t = s_red[lane & (kTriWarps - 1)];
+#pragma unroll
+  for (int o = kTriWarps / 2; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  return t;                                                   // the same bits in every thread of the CTA
+}
+
+// alpha, beta and the first entry of v from ||x||^2 and x_0
+__device__ __forceinline__ void tri_reflector(double nx2, double x0, double& alpha, double& beta, double& v0) {
+  alpha = 0.0; beta = 0.0; v0 = 0.0;
+  if (nx2 > 0.0) {
+    alpha = -copysign(sqrt(nx2), x0);
+    v0 = x0 - alpha;
+    const double den = alpha * (alpha - x0);                  // = v^T v / 2 > 0
+    beta = den > 0.0 ? 1.0 / den : 0.0;
+  }
+}
+
+// one entry of each of the two register rows, slot chosen at run time (uniform over the warp): a jump, not 16 selects
+#define TRI_PICK(slot, out0, out1)                                                                       \
+  switch (slot) {                                                                                        \
+    case 0: out0 = row0[0]; out1 = row1[0]; break;    case 1: out0 = row0[1]; out1 = row1[1]; break;     \
+    case 2: out0 = row0[2]; out1 = row1[2]; break;    case 3: out0 = row0[3]; out1 = row1[3]; break;     \
+    case 4: out0 = row0[4]; out1 = row1[4]; break;    case 5: out0 = row0[5]; out1 = row1[5]; break;     \
+    case 6: out0 = row0[6]; out1 = row1[6]; break;    case 7: out0 = row0[7]; out1 = row1[7]; break;     \
+    case 8: out0 = row0[8]; out1 = row1[8]; break;    case 9: out0 = row0[9]; out1 = row1[9]; break;     \
+    case 10: out0 = row0[10]; out1 = row1[10]; break; case 11: out0 = row0[11]; out1 = row1[11]; break;  \
+    case 12: out0 = row0[12]; out1 = row1[12]; break; case 13: out0 = row0[13]; out1 = row1[13]; break;  \
+    case 14: out0 = row0[14]; out1 = row1[14]; break; default: out0 = row0[15]; out1 = row1[15]; break;  \
+  }
+
 __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(const SpLayer* __restrict__ layers,
                                                                             const ClusterCta* __restrict__ ctas) {
+  static_assert(kTriCols == 16, "TRI_PICK lists 16 slots");
   cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ __align__(16) unsigned char tri_smem[];
-  double* As = reinterpret_cast<double*>(tri_smem);          // [32][rp]
-  __shared__ double s_v[2][kTriMaxRp];                        // pivot column of step k in s_v[k & 1] (written by the row owners)
-  __shared__ double s_p[kTriMaxRp];                           // beta A22 v (written by the row owners)
+  __shared__ double s_p[2][kTriMaxRp];                        // beta A22 v of step k in s_p[k & 1] (written by the row owners)
+  __shared__ double s_c[2][kTriMaxRp];                        // column k+1 after update k-1, likewise
+  __shared__ double s_v[2][kTriMaxRp];                        // v of step k in s_v[k & 1]
+  __shared__ double s_w[kTriMaxRp];
+  __shared__ double s_stage[2][kTriRows];                     // this CTA's 32 entries of p and c on their way out
+  __shared__ double s_red1[kTriWarps], s_red2[kTriWarps];
+  __shared__ double s_x0, s_scal[3];                          // first entry of the next pivot column; alpha, beta, v_0 of the next reflector
   const ClusterCta me = ctas[blockIdx.x];
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   // every CTA of the cluster keeps the same number of barriers: the longest reduction among the cluster's layers
@@ -59,126 +105,176 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   }
   cluster.sync();                                             // every CTA of the cluster runs: remote stores may start
   if (me.layer < 0) {
-    for (int k = 0; k < steps; ++k) { cluster.sync(); cluster.sync(); }
+    for (int k = 0; k <= steps; ++k) cluster.sync();
     cluster.sync();
     return;
   }
   const SpLayer& L = layers[me.layer];
-  const int r = L.r, rp = L.rp, nc = me.pad, g = me.slot, base = me.base_rank;
-  const int ncol = rp / 32;                                   // columns per lane: j = lane + 32 m
-  for (int li = w; li < kTriRows; li += kTriWarps) {
-    const int i = li * nc + g;
-    for (int j = lane; j < rp; j += 32) As[li * rp + j] = (i < r && j < r) ? (double)L.A[(int64_t)i * L.lda + j] : 0.0;
+  const int r = L.r, nc = me.pad, g = me.slot, base = me.base_rank;
+  // the layer's pointers in registers: a field read through `layers` inside a loop would be a global load each time
+  double* const td_d = L.td_d; double* const td_e = L.td_e; double* const td_tau = L.td_tau; double* const td_V = L.td_V;
+  const float* const gA = L.A; const int64_t lda = L.lda;
+  const int my_steps = max(r - 2, 0);
+  const int li0 = w, li1 = w + kTriWarps;                     // this warp's two rows
+  const int i0 = li0 * nc + g, i1 = li1 * nc + g;
+  double row0[kTriCols], row1[kTriCols];
+#pragma unroll
+  for (int m = 0; m < kTriCols; ++m) {
+    const int j = lane * nc + m;
+    const bool in = m < nc && j < r;
+    row0[m] = (in && i0 < r) ? (double)gA[(int64_t)i0 * lda + j] : 0.0;
+    row1[m] = (in && i1 < r) ? (double)gA[(int64_t)i1 * lda + j] : 0.0;
+  }
+  const int sq = w * 32 + lane;                               // this thread's entry of the vectors (warps < nc)
+  const int sj = lane * nc + w;                               // its index
+  const bool slice = w < nc;
+  // ---- the first reflector and A v_0 ----
+  double beta = 0.0, v0 = 0.0;
+  if (my_steps > 0) {
+    const double xq = (slice && sj > 0 && sj < r) ? (double)gA[sj] : 0.0;   // column 0 = row 0 (symmetric)
+    if (slice) s_v[0][sq] = xq;
+    const double nx2 = tri_block_sum(xq * xq, s_red2, lane, w);
+    const int q1 = (1 % nc) * 32 + 1 / nc;
+    if (tid == 0) {
+      double alpha;
+      tri_reflector(nx2, (double)gA[1], alpha, beta, v0);
+      s_scal[0] = alpha; s_scal[1] = beta; s_scal[2] = v0;
+      s_v[0][q1] = v0;
+      if (g == 0) { td_d[0] = (double)gA[0]; td_e[0] = alpha; td_tau[0] = beta; }
+    }
+    __syncthreads();
+    beta = s_scal[1]; v0 = s_scal[2];
+    if (g == 0)
+      for (int j = tid; j < r; j += kTriThreads) td_V[j] = s_v[0][(j % nc) * 32 + j / nc];
+    double a0 = 0.0, a1 = 0.0;
+#pragma unroll
+    for (int m = 0; m < kTriCols; ++m) {
+      if (m < nc) {
+        const double vq = s_v[0][lane + 32 * m];
+        a0 = fma(row0[m], vq, a0); a1 = fma(row1[m], vq, a1);
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, o); a1 += __shfl_xor_sync(0xffffffffu, a1, o); }
+    double c0 = 0.0, c1 = 0.0;
+    TRI_PICK(q1 >> 5, c0, c1);
+    if (lane == (q1 & 31)) { s_stage[1][li0] = c0; s_stage[1][li1] = c1; }
+    if (lane == 0) {
+      s_stage[0][li0] = (i0 > 0 && i0 < r) ? a0 * beta : 0.0;
+      s_stage[0][li1] = (i1 > 0 && i1 < r) ? a1 * beta : 0.0;
+    }
   }
   __syncthreads();
-  const int my_steps = max(r - 2, 0);
+  if (my_steps > 0 && w < nc) {                               // warp w carries this CTA's 32 entries to peer w
+    cluster.map_shared_rank(&s_p[0][0], base + w)[g * 32 + lane] = s_stage[0][lane];
+    cluster.map_shared_rank(&s_c[0][0], base + w)[g * 32 + lane] = s_stage[1][lane];
+  }
+  cluster.sync();
   for (int k = 0; k < steps; ++k) {
     const bool active = k < my_steps;
-    const int par = k & 1;
+    const bool last = k + 1 == my_steps;                      // no reflector follows
+    const int par = k & 1, nxt = par ^ 1;
+    const int q1 = ((k + 1) % nc) * 32 + (k + 1) / nc;       // where entry k+1 sits
+    const int q2 = ((k + 2) % nc) * 32 + (k + 2) / nc;
+    double beta_n = 0.0, v0_n = 0.0;
     if (active) {
-      // pivot column: every owned entry below the diagonal goes to all CTAs of the layer
-      const int li = tid % kTriRows, dest = tid / kTriRows;
-      const int i = li * nc + g;
-      if (dest < nc && i > k && i < r) cluster.map_shared_rank(&s_v[0][0], base + dest)[par * kTriMaxRp + i] = As[li * rp + k];
-      if (tid == 0 && k % nc == g) L.td_d[k] = As[(k / nc) * rp + k];
+      // K = beta/2 p^T v, each thread one entry
+      const double vq = slice ? s_v[par][sq] : 0.0;
+      const double pq = slice ? s_p[par][sq] : 0.0;
+      const double K = 0.5 * beta * tri_block_sum(pq * vq, s_red1, lane, w);
+      const double w1 = fma(-K, v0, s_p[par][q1]);            // w_{k+1}
+      // w, and the next pivot column x_j = c_j - v_j w_{k+1} - w_j v_{k+1} for j > k+1
+      const double wq = fma(-K, vq, pq);
+      double xn = 0.0;
+      if (slice) {
+        s_w[sq] = wq;
+        if (sj > k + 1 && sj < r && !last) xn = s_c[par][sq] - fma(vq, w1, wq * v0);
+        s_v[nxt][sq] = xn;
+        if (sq == q2) s_x0 = xn;
+      }
+      const double nx2 = tri_block_sum(xn * xn, s_red2, lane, w);
+      if (tid == 0) {                                         // one thread forms the reflector; a zero column gives v = 0
+        double alpha_n;
+        tri_reflector(nx2, s_x0, alpha_n, beta_n, v0_n);
+        s_scal[0] = alpha_n; s_scal[1] = beta_n; s_scal[2] = v0_n;
+        if (!last) s_v[nxt][q2] = v0_n;
+      }
+      __syncthreads();
+      beta_n = s_scal[1]; v0_n = s_scal[2];
+      // update of the two rows with (v, w), fused with their products with the next v
+      const double vi0 = s_v[par][g * 32 + li0], vi1 = s_v[par][g * 32 + li1];
+      const double wi0 = s_w[g * 32 + li0], wi1 = s_w[g * 32 + li1];
+      const double* __restrict__ pv = &s_v[par][lane];
+      const double* __restrict__ pn = &s_v[nxt][lane];
+      const double* __restrict__ pw = &s_w[lane];
+      double a0 = 0.0, a1 = 0.0;
+#pragma unroll
+      for (int m = 0; m < kTriCols; ++m) {
+        if (m < nc) {
+          const double vq2 = pv[32 * m], wq2 = pw[32 * m], vn = pn[32 * m];
+          row0[m] = fma(-vi0, wq2, fma(-wi0, vq2, row0[m]));
+          row1[m] = fma(-vi1, wq2, fma(-wi1, vq2, row1[m]));
+          a0 = fma(row0[m], vn, a0); a1 = fma(row1[m], vn, a1);
+        }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) { a0 += __shfl_xor_sync(0xffffffffu, a0, o); a1 += __shfl_xor_sync(0xffffffffu, a1, o); }
+      // column k+2 of the two rows goes out with the products; column k+1 holds the entries of T that are final now
+      double c20 = 0.0, c21 = 0.0;
+      TRI_PICK(q2 >> 5, c20, c21);
+      if (lane == (q2 & 31)) {
+        s_stage[1][li0] = c20; s_stage[1][li1] = c21;
+        if (last) { if (i0 == r - 1) td_d[r - 1] = c20; if (i1 == r - 1) td_d[r - 1] = c21; }
+      }
+      if (i0 == k + 1 || i1 == k + 1 || (last && (i0 == r - 1 || i1 == r - 1))) {
+        double c10 = 0.0, c11 = 0.0;
+        TRI_PICK(q1 >> 5, c10, c11);
+        if (lane == (q1 & 31)) {
+          if (i0 == k + 1) td_d[k + 1] = c10;
+          if (i1 == k + 1) td_d[k + 1] = c11;
+          if (last) { if (i0 == r - 1) td_e[r - 2] = c10; if (i1 == r - 1) td_e[r - 2] = c11; }
+        }
+      }
+      if (lane == 0) {
+        s_stage[0][li0] = (i0 > k + 1 && i0 < r) ? a0 * beta_n : 0.0;
+        s_stage[0][li1] = (i1 > k + 1 && i1 < r) ? a1 * beta_n : 0.0;
+      }
     }
+    __syncthreads();
+    if (active && !last) {
+      if (w < nc) {
+        cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[0][lane];
+        cluster.map_shared_rank(&s_c[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
+      }
+      if ((k + 1) % nc == g) {                                // one CTA of the layer files the reflector
+        if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
+        for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * r + j] = s_v[nxt][(j % nc) * 32 + j / nc];
+      }
+    }
+    beta = beta_n; v0 = v0_n;
     cluster.sync();
-    double v[kTriCols];
-    double beta = 0.0, v0 = 0.0;
-    if (active) {
-      // every warp forms v and beta from the same values in the same order (no broadcast needed)
-      double nx2 = 0.0;
-#pragma unroll
-      for (int m = 0; m < kTriCols; ++m) {
-        const int j = lane + 32 * m;
-        v[m] = (m < ncol && j > k && j < r) ? s_v[par][j] : 0.0;
-        nx2 = fma(v[m], v[m], nx2);
-      }
-      nx2 = warp_sum(nx2);
-      const double x0 = s_v[par][k + 1];
-      double alpha = 0.0;
-      if (nx2 > 0.0) {
-        alpha = -copysign(sqrt(nx2), x0);
-        v0 = x0 - alpha;
-        const double den = alpha * (alpha - x0);              // = v^T v / 2 > 0
-        beta = den > 0.0 ? 1.0 / den : 0.0;
-      }
-      // v = x with its first entry replaced (a zero column leaves H = I)
-#pragma unroll
-      for (int m = 0; m < kTriCols; ++m) {
-        if (!(nx2 > 0.0)) v[m] = 0.0;
-        else if (lane + 32 * m == k + 1) v[m] = v0;
-      }
-      if (k % nc == g) {                                      // one CTA of the layer files the step's results
-        if (tid == 0) { L.td_e[k] = alpha; L.td_tau[k] = beta; }
-        if (w == 1) {
-#pragma unroll
-          for (int m = 0; m < kTriCols; ++m) if (m < ncol && lane + 32 * m < r) L.td_V[(int64_t)k * r + lane + 32 * m] = v[m];
-        }
-      }
-      // p_i = beta sum_j A_ij v_j for the owned rows below the pivot
-      for (int li = w; li < kTriRows; li += kTriWarps) {
-        const int i = li * nc + g;
-        if (i > k && i < r) {
-          const double* row = As + li * rp;
-          double acc = 0.0;
-#pragma unroll
-          for (int m = 0; m < kTriCols; ++m) if (m < ncol) acc = fma(row[lane + 32 * m], v[m], acc);
-          acc = warp_sum(acc) * beta;
-          if (lane < nc) cluster.map_shared_rank(&s_p[0], base + lane)[i] = acc;
-        }
-      }
-    }
-    cluster.sync();
-    if (active) {
-      double wv[kTriCols];
-      double pv = 0.0;
-#pragma unroll
-      for (int m = 0; m < kTriCols; ++m) {
-        const int j = lane + 32 * m;
-        wv[m] = (m < ncol && j > k && j < r) ? s_p[j] : 0.0;
-        pv = fma(wv[m], v[m], pv);
-      }
-      pv = warp_sum(pv);
-      const double K = 0.5 * beta * pv;
-#pragma unroll
-      for (int m = 0; m < kTriCols; ++m) wv[m] = fma(-K, v[m], wv[m]);
-      for (int li = w; li < kTriRows; li += kTriWarps) {
-        const int i = li * nc + g;
-        if (i > k && i < r) {
-          // v_i and w_i of this row, from the same shared arrays every warp read its columns from
-          const double vi = beta == 0.0 ? 0.0 : (i == k + 1 ? v0 : s_v[par][i]);
-          const double wi = fma(-K, vi, s_p[i]);
-          double* row = As + li * rp;
-#pragma unroll
-          for (int m = 0; m < kTriCols; ++m)
-            if (m < ncol) row[lane + 32 * m] -= fma(vi, wv[m], wi * v[m]);
-        }
-      }
-    }
-    __syncthreads();                                          // the next pivot column is read with another thread mapping
   }
-  // the last 2 x 2 block (r >= 2) or the single entry (r = 1)
-  if (tid == 0) {
-    if (r >= 2) {
-      if ((r - 2) % nc == g) L.td_d[r - 2] = As[((r - 2) / nc) * rp + (r - 2)];
-      if ((r - 1) % nc == g) { L.td_d[r - 1] = As[((r - 1) / nc) * rp + (r - 1)]; L.td_e[r - 2] = As[((r - 1) / nc) * rp + (r - 2)]; }
-    } else if (g == 0) {
-      L.td_d[0] = As[0];
-    }
+  // matrices of order 1 and 2 are tridiagonal as they are
+  if (my_steps == 0 && g == 0 && tid == 0) {
+    td_d[0] = (double)gA[0];
+    if (r == 2) { td_d[1] = (double)gA[lda + 1]; td_e[0] = (double)gA[lda]; }
   }
   cluster.sync();                                             // nobody leaves while a peer may still write here
 }
+#undef TRI_PICK
 
 // ---- eigenvalues of T: Sturm counts -------------------------------------------------------------------------
 // count(x) = number of eigenvalues below x = sign changes of p_0 = 1, p_1 = d_0 - x, p_{i+1} = (d_i - x) p_i -
 // e_{i-1}^2 p_{i-1}.  The pair (p_i, p_{i-1}) is rescaled by a power of two every 8 steps (ratios and signs keep).
 __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const double* __restrict__ e2, int r, double x) {
   double pm = 1.0, p = d[0] - x;
-  int cnt = p < 0.0 ? 1 : 0;
+  int neg = __double2hiint(p);                                // sign bit of the previous term
+  int cnt = (uint32_t)neg >> 31;
   for (int i = 1; i < r; ++i) {
     const double pn = fma(d[i] - x, p, -e2[i - 1] * pm);
-    cnt += ((pn < 0.0) != (p < 0.0)) ? 1 : 0;
+    const int hn = __double2hiint(pn);
+    cnt += (uint32_t)(hn ^ neg) >> 31;
+    neg = hn;
     pm = p; p = pn;
     if ((i & 7) == 0) {
       const int ex = ((__double2hiint(fabs(p) + fabs(pm)) >> 20) & 0x7ff) - 1023;
@@ -190,13 +286,15 @@ __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const d
 }
 
 constexpr int kBisThreads = 256;
-constexpr int kBisRounds = 8;         // 33^8 = 1.4e12: interval width below 1e-12 of the spectrum's extent
+constexpr int kBisLanes = 8;          // points per round and eigenvalue: the interval shrinks 9 times per round
+constexpr int kBisRounds = 13;        // 9^13 = 2.5e12: interval width below 1e-12 of the spectrum's extent
+constexpr int kBisPerCta = kBisThreads / kBisLanes;
 
 __global__ void __launch_bounds__(kBisThreads) sp_bisect_kernel(const SpLayer* __restrict__ layers) {
   const SpLayer& L = layers[blockIdx.y];
   const int r = L.r;
-  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
-  if ((int)blockIdx.x * (kBisThreads / 32) >= r) return;
+  const int tid = threadIdx.x, lane = tid % 32;
+  if ((int)blockIdx.x * kBisPerCta >= r) return;
   __shared__ double s_d[kTriMaxRp], s_e2[kTriMaxRp];
   for (int i = tid; i < r; i += kBisThreads) {
     s_d[i] = L.td_d[i];
@@ -215,24 +313,26 @@ __global__ void __launch_bounds__(kBisThreads) sp_bisect_kernel(const SpLayer* _
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) { gl = fmin(gl, __shfl_xor_sync(0xffffffffu, gl, o)); gu = fmax(gu, __shfl_xor_sync(0xffffffffu, gu, o)); }
   bad = __any_sync(0xffffffffu, bad);
-  const int j = blockIdx.x * (kBisThreads / 32) + w;          // this warp's eigenvalue, ascending order
-  if (j >= r) return;
+  const int grp = lane / kBisLanes, t = lane % kBisLanes;     // 4 eigenvalues per warp, 8 lanes each
+  const int j = blockIdx.x * kBisPerCta + (tid / 32) * (32 / kBisLanes) + grp;   // ascending order
+  const int jj = min(j, r - 1);                               // lanes past the end follow the last eigenvalue
   if (bad) {
-    if (lane == 0) { L.lam64[j] = __longlong_as_double(0x7ff8000000000000ll); L.lam[j] = __int_as_float(0x7fc00000); }
+    if (t == 0 && j < r) { L.lam64[j] = __longlong_as_double(0x7ff8000000000000ll); L.lam[j] = __int_as_float(0x7fc00000); }
     return;
   }
   const double pad = 1.0e-14 * fmax(fabs(gl), fabs(gu)) + 1.0e-300;
   double lo = gl - pad, hi = gu + pad;
   for (int it = 0; it < kBisRounds; ++it) {
-    const double h = (hi - lo) * (1.0 / 33.0);
-    const double x = fma((double)(lane + 1), h, lo);
+    const double h = (hi - lo) * (1.0 / (kBisLanes + 1));
+    const double x = fma((double)(t + 1), h, lo);
     const int cnt = sturm_count(s_d, s_e2, r, x);
-    const int nle = __popc(__ballot_sync(0xffffffffu, cnt <= j));   // points not above lambda_j
+    const uint32_t le = __ballot_sync(0xffffffffu, cnt <= jj);              // points not above lambda_j
+    const int nle = __popc((le >> (grp * kBisLanes)) & ((1u << kBisLanes) - 1u));
     const double nlo = fma((double)nle, h, lo);
     hi = fmin(hi, fma((double)(nle + 1), h, lo));
     lo = nlo;
   }
-  if (lane == 0) { const double lam = 0.5 * (lo + hi); L.lam64[j] = lam; L.lam[j] = (float)lam; }
+  if (t == 0 && j < r) { const double lam = 0.5 * (lo + hi); L.lam64[j] = lam; L.lam[j] = (float)lam; }
 }
 
 // ---- vectors of the kept atoms --------------------------------------------------------------------------------
@@ -256,14 +356,18 @@ __device__ double twisted_vector(const double* __restrict__ d, const double* __r
     double piv = d[cur] - lambda;
     if (fabs(piv) < kPivMin) piv = kPivMin;
     D[cur] = piv;
+    // piv_next = (d_next - lambda) - e^2 / piv: the operands of step t+1 are fetched while step t's reciprocal runs
+    double ee = r > 1 ? e[back ? r - 2 : 0] : 0.0;
+    double dn = r > 1 ? d[back ? r - 2 : 1] : 0.0;
     for (int t = 0; t + 1 < r; ++t) {
-      const int ie = back ? r - 2 - t : t;                    // the off-diagonal between cur and next
       const int nxt = back ? cur - 1 : cur + 1;
-      const double ee = e[ie];
-      piv = fma(-(ee / piv), ee, d[nxt] - lambda);
+      const int ie2 = back ? max(r - 3 - t, 0) : min(t + 1, r - 2);      // next step's off-diagonal and diagonal
+      const int in2 = back ? max(nxt - 1, 0) : min(nxt + 1, r - 1);
+      const double ee2 = e[ie2], dn2 = d[in2];
+      piv = fma(-(ee * ee), __drcp_rn(piv), dn - lambda);
       if (fabs(piv) < kPivMin) piv = kPivMin;
       D[nxt] = piv;
-      cur = nxt;
+      cur = nxt; ee = ee2; dn = dn2;
     }
   }
   __syncwarp();
@@ -355,7 +459,11 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       skip = (int)warp_sum((uint32_t)skip);
       double n2 = 1.0;
       const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, z, lane, skip, &n2);
-      if (finite64(corr) && skip == 0) {                      // one Rayleigh-quotient step, then the vector again
+      // the vector's error is about |correction| / gap to the nearest other eigenvalue: well-separated atoms are done
+      double gap = 1.0e300;
+      if (ei > 0) gap = fmin(gap, fabs(lambda - L.lam64[ei - 1]));
+      if (ei + 1 < r) gap = fmin(gap, fabs(L.lam64[ei + 1] - lambda));
+      if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {   // one Rayleigh-quotient step, then the vector again
         lambda += corr;
         __syncwarp();
         twisted_vector(s_d, s_e, r, lambda, wa, wb, z, lane, 0, &n2);
@@ -476,7 +584,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
 }
 
 // ---- host side ---------------------------------------------------------------------------------------------------
-static size_t tri_smem_bytes(int rp_max) { return (size_t)kTriRows * rp_max * sizeof(double); }
+static size_t tri_smem_bytes(int) { return 0; }             // rows in registers, vectors in static shared memory
 static size_t vec_smem_bytes(int rp_max) { return (size_t)(2 + 2 * kVecGroup + 3 * kVecWarps) * rp_max * sizeof(double); }
 
 int sp_tridiag_max_rp() { return kTriMaxRp; }
@@ -514,8 +622,7 @@ int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_c
 }
 
 void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, cudaStream_t st) {
-  const int per = kBisThreads / 32;
-  sp_bisect_kernel<<<dim3((r_max + per - 1) / per, n_layers), kBisThreads, 0, st>>>(d_layers);
+  sp_bisect_kernel<<<dim3((r_max + kBisPerCta - 1) / kBisPerCta, n_layers), kBisThreads, 0, st>>>(d_layers);
 }
 
 void launch_sp_eigvec(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {
