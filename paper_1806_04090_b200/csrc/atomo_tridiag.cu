@@ -12,7 +12,7 @@
 //   (sp_finalize_sample_kernel sorts, solves Algorithm 1 and draws, as for the other routes)
 //   sp_eigvec_kernel          : for the kept atoms only: eigenvector of T by a twisted factorisation with one
 //                               Rayleigh-quotient correction, back-transformation u = Q z with the reflectors
-//                               (four at a time), normalised short-side vector into the payload; kept atoms with
+//                               (four at a time, fp32), normalised short-side vector into the payload; kept atoms with
 //                               nearly equal eigenvalues are orthogonalised against each other at the end.
 //
 // Work per layer: about 2 r^3 fp64 flops for the reduction (full symmetric storage: matrix-vector product and
@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   const SpLayer& L = layers[me.layer];
   const int r = L.r, nc = me.pad, g = me.slot, base = me.base_rank;
   // the layer's pointers in registers: a field read through `layers` inside a loop would be a global load each time
-  double* const td_d = L.td_d; double* const td_e = L.td_e; double* const td_tau = L.td_tau; double* const td_V = L.td_V;
+  double* const td_d = L.td_d; double* const td_e = L.td_e; double* const td_tau = L.td_tau; float* const td_V = L.td_V;
   const float* const gA = L.A; const int64_t lda = L.lda;
   const int my_steps = max(r - 2, 0);
   const int li0 = w, li1 = w + kTriWarps;                     // this warp's two rows
@@ -144,8 +144,11 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     }
     __syncthreads();
     beta = s_scal[1]; v0 = s_scal[2];
-    if (g == 0)
-      for (int j = tid; j < r; j += kTriThreads) td_V[j] = s_v[0][(j % nc) * 32 + j / nc];
+    {
+      // reflectors are filed as unit vectors (H = I - 2 u u^T, u = v sqrt(beta / 2)): no range trouble in fp32
+      const double un = sqrt(0.5 * beta);
+      if (g == 0) for (int j = tid; j < r; j += kTriThreads) td_V[j] = (float)(s_v[0][(j % nc) * 32 + j / nc] * un);
+    }
     double a0 = 0.0, a1 = 0.0;
 #pragma unroll
     for (int m = 0; m < kTriCols; ++m) {
@@ -241,18 +244,18 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       }
     }
     __syncthreads();
-    if (active && !last) {
-      if (w < nc) {
-        cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[0][lane];
-        cluster.map_shared_rank(&s_c[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
-      }
-      if ((k + 1) % nc == g) {                                // one CTA of the layer files the reflector
-        if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
-        for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * r + j] = s_v[nxt][(j % nc) * 32 + j / nc];
-      }
+    if (active && !last && w < nc) {
+      cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[0][lane];
+      cluster.map_shared_rank(&s_c[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
+    }
+    cluster.barrier_arrive();                                 // (release) the entries above are on their way
+    if (active && !last && (k + 1) % nc == g) {               // meanwhile one CTA of the layer files the reflector
+      if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
+      const double un = sqrt(0.5 * beta_n);                   // filed as a unit vector: H = I - 2 u u^T
+      for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * r + j] = (float)(s_v[nxt][(j % nc) * 32 + j / nc] * un);
     }
     beta = beta_n; v0 = v0_n;
-    cluster.sync();
+    cluster.barrier_wait();
   }
   // matrices of order 1 and 2 are tridiagonal as they are
   if (my_steps == 0 && g == 0 && tid == 0) {
@@ -340,6 +343,7 @@ constexpr int kVecThreads = 256;
 constexpr int kVecWarps = kVecThreads / 32;
 constexpr int kVecCtasPerLayer = 4;
 constexpr int kVecGroup = 4;          // reflectors applied together in the back-transformation
+constexpr int kVecStages = 4;         // groups in flight between global and shared memory
 constexpr double kPivMin = 1.0e-280;
 constexpr double kSameEig = 1.0e-9;   // scaled units (largest eigenvalue below 1): eigenvalues this close share a subspace
 
@@ -430,12 +434,15 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
   const int r = L.r, rp = L.rp;
   double* s_d = reinterpret_cast<double*>(vec_smem);          // [rp]
   double* s_e = s_d + rp;                                     // [rp]
-  double* s_ref = s_e + rp;                                   // [2][kVecGroup][rp] reflectors of the current / next group
-  double* s_work = s_ref + 2 * kVecGroup * rp;                // [warps][3][rp]
-  __shared__ double s_beta[2][kVecGroup];
+  double* s_work = s_e + rp;                                  // [warps][3][rp]
+  float* s_ref = reinterpret_cast<float*>(s_work + (size_t)kVecWarps * 3 * rp);   // [kVecStages][kVecGroup][rp] ring of reflector groups
+  __shared__ float s_beta[kVecStages][kVecGroup];
   __shared__ uint32_t s_last;
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const uint32_t k = L.hdr->k;
+  // the layer's pointers in registers (a field read through `layers` inside a loop is a global load each time)
+  const float* const gV = L.td_V; const double* const gLam = L.lam64;
+  const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
   const int nref = max(r - 2, 0);
   const int ngroups = (nref + kVecGroup - 1) / kVecGroup;
   for (int i = tid; i < r; i += kVecThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
@@ -447,22 +454,22 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
   for (uint32_t a0 = blockIdx.y * kVecWarps; a0 < k; a0 += kVecCtasPerLayer * kVecWarps) {
     const uint32_t a = a0 + w;
     const bool have = a < k;
-    double zr[kCols];                                         // z[lane + 32 m]
+    float zr[kCols];                                          // z[lane + 32 m]
 #pragma unroll
-    for (int m = 0; m < kCols; ++m) zr[m] = 0.0;
+    for (int m = 0; m < kCols; ++m) zr[m] = 0.0f;
     if (have) {
-      const int ei = L.perm[L.idx[a]];                        // index of the atom's eigenvalue (ascending order)
-      double lambda = L.lam64[ei];
+      const int ei = gPerm[gIdx[a]];                          // index of the atom's eigenvalue (ascending order)
+      double lambda = gLam[ei];
       // earlier kept atoms with the same eigenvalue (to the accuracy of the bisection): each takes another twist index
       int skip = 0;
-      for (uint32_t b = lane; b < a; b += 32) skip += fabs(L.lam64[L.perm[L.idx[b]]] - lambda) <= kSameEig ? 1 : 0;
+      for (uint32_t b = lane; b < a; b += 32) skip += fabs(gLam[gPerm[gIdx[b]]] - lambda) <= kSameEig ? 1 : 0;
       skip = (int)warp_sum((uint32_t)skip);
       double n2 = 1.0;
       const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, z, lane, skip, &n2);
       // the vector's error is about |correction| / gap to the nearest other eigenvalue: well-separated atoms are done
       double gap = 1.0e300;
-      if (ei > 0) gap = fmin(gap, fabs(lambda - L.lam64[ei - 1]));
-      if (ei + 1 < r) gap = fmin(gap, fabs(L.lam64[ei + 1] - lambda));
+      if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
+      if (ei + 1 < r) gap = fmin(gap, fabs(gLam[ei + 1] - lambda));
       if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {   // one Rayleigh-quotient step, then the vector again
         lambda += corr;
         __syncwarp();
@@ -470,49 +477,50 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       }
       const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
 #pragma unroll
-      for (int m = 0; m < kCols; ++m) { const int i = lane + 32 * m; zr[m] = i < r ? z[i] * inv : 0.0; }
+      for (int m = 0; m < kCols; ++m) { const int i = lane + 32 * m; zr[m] = i < r ? (float)(z[i] * inv) : 0.0f; }
     }
-    // u = H_0 H_1 ... H_{r-3} z: the reflectors from the last to the first, kVecGroup at a time.  For a group applied in
-    // the order 0, 1, 2, 3:  s_0 = beta_0 v_0.z,  s_i = beta_i (v_i.z - sum_{j<i} s_j v_i.v_j),  z -= sum s_i v_i.
+    // u = H_0 H_1 ... H_{r-3} z: the reflectors from the last to the first, kVecGroup at a time, in fp32 (an orthogonal
+    // map of a unit vector whose result is stored in fp32 anyway).  For a group applied in the order 0, 1, 2, 3:
+    // s_0 = beta_0 v_0.z,  s_i = beta_i (v_i.z - sum_{j<i} s_j v_i.v_j),  z -= sum s_i v_i.
     __syncthreads();
-    // group gi holds the reflectors kk = nref-1 - 4 gi - q, q = 0..3 in the order of application; a thread stages
-    // kPre entries of the next group in registers while the current one is applied
-    constexpr int kPre = kVecGroup * kTriMaxRp / kVecThreads;
-    double pre[kPre];
-    auto fetch_group = [&](int gi) {
-#pragma unroll
-      for (int t = 0; t < kPre; ++t) {
-        const int el = tid + kVecThreads * t;
-        const int q = el / rp, i = el - q * rp;
+    // group gi holds the reflectors kk = nref-1 - 4 gi - q, q = 0..3 in the order of application.  The groups stream
+    // through a ring of kVecStages buffers filled by asynchronous copies, kVecStages - 1 groups ahead of use; warp w
+    // copies half of row q = w mod 4.
+    auto issue_group = [&](int gi) {
+      if (gi < ngroups) {
+        const int buf = gi % kVecStages;
+        const int q = w & (kVecGroup - 1);
         const int kk = nref - 1 - kVecGroup * gi - q;
-        pre[t] = (el < kVecGroup * rp && kk >= 0 && i < r) ? L.td_V[(int64_t)kk * r + i] : 0.0;
+        const float* srow = gV + (int64_t)max(kk, 0) * r;
+        float* drow = s_ref + ((size_t)buf * kVecGroup + q) * rp;
+        for (int i = (w / kVecGroup) * 32 + lane; i < rp; i += 32 * (kVecWarps / kVecGroup)) {
+          const bool in = kk >= 0 && i < r;
+          const uint32_t dst = (uint32_t)__cvta_generic_to_shared(drow + i);
+          const int bytes = in ? 4 : 0;                       // 0: the destination is filled with zeros
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(in ? srow + i : gV), "r"(bytes) : "memory");
+        }
+        if (tid < kVecGroup) { const int kq = nref - 1 - kVecGroup * gi - tid; s_beta[buf][tid] = kq >= 0 ? 2.0f : 0.0f; }   // unit reflectors
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");    // one group per call, empty or not: the counting stays uniform
     };
-    auto store_group = [&](int gi, int buf) {
-#pragma unroll
-      for (int t = 0; t < kPre; ++t) {
-        const int el = tid + kVecThreads * t;
-        if (el < kVecGroup * rp) s_ref[(size_t)buf * kVecGroup * rp + el] = pre[t];
-      }
-      if (tid < kVecGroup) { const int kk = nref - 1 - kVecGroup * gi - tid; s_beta[buf][tid] = kk >= 0 ? L.td_tau[kk] : 0.0; }
-    };
-    if (ngroups > 0) { fetch_group(0); store_group(0, 0); }
-    __syncthreads();
+    for (int st = 0; st < kVecStages - 1; ++st) issue_group(st);
     for (int gi = 0; gi < ngroups; ++gi) {
-      const int buf = gi & 1;
-      if (gi + 1 < ngroups) fetch_group(gi + 1);
+      const int buf = gi % kVecStages;
+      asm volatile("cp.async.wait_group %0;" ::"n"(kVecStages - 2) : "memory");
+      __syncthreads();                                        // group gi has landed for everybody; the buffer of gi-1 is free
+      issue_group(gi + kVecStages - 1);
       if (have) {
-        const double* v0 = s_ref + ((size_t)buf * kVecGroup + 0) * rp;
-        const double* v1 = v0 + rp; const double* v2 = v1 + rp; const double* v3 = v2 + rp;
-        double z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
+        const float* v0 = s_ref + ((size_t)buf * kVecGroup + 0) * rp;
+        const float* v1 = v0 + rp; const float* v2 = v1 + rp; const float* v3 = v2 + rp;
+        float z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
 #pragma unroll
         for (int m = 0; m < kCols; ++m) {
           if (32 * m < rp) {
             const int i = lane + 32 * m;
-            const double a0v = v0[i], a1v = v1[i], a2v = v2[i], a3v = v3[i], zz = zr[m];
-            z0 = fma(a0v, zz, z0); z1 = fma(a1v, zz, z1); z2 = fma(a2v, zz, z2); z3 = fma(a3v, zz, z3);
-            g10 = fma(a1v, a0v, g10); g20 = fma(a2v, a0v, g20); g21 = fma(a2v, a1v, g21);
-            g30 = fma(a3v, a0v, g30); g31 = fma(a3v, a1v, g31); g32 = fma(a3v, a2v, g32);
+            const float a0v = v0[i], a1v = v1[i], a2v = v2[i], a3v = v3[i], zz = zr[m];
+            z0 = fmaf(a0v, zz, z0); z1 = fmaf(a1v, zz, z1); z2 = fmaf(a2v, zz, z2); z3 = fmaf(a3v, zz, z3);
+            g10 = fmaf(a1v, a0v, g10); g20 = fmaf(a2v, a0v, g20); g21 = fmaf(a2v, a1v, g21);
+            g30 = fmaf(a3v, a0v, g30); g31 = fmaf(a3v, a1v, g31); g32 = fmaf(a3v, a2v, g32);
           }
         }
 #pragma unroll
@@ -523,29 +531,28 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
           g21 += __shfl_xor_sync(0xffffffffu, g21, o); g30 += __shfl_xor_sync(0xffffffffu, g30, o);
           g31 += __shfl_xor_sync(0xffffffffu, g31, o); g32 += __shfl_xor_sync(0xffffffffu, g32, o);
         }
-        const double c0 = s_beta[buf][0] * z0;
-        const double c1 = s_beta[buf][1] * (z1 - c0 * g10);
-        const double c2 = s_beta[buf][2] * (z2 - c0 * g20 - c1 * g21);
-        const double c3 = s_beta[buf][3] * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
+        const float c0 = s_beta[buf][0] * z0;
+        const float c1 = s_beta[buf][1] * (z1 - c0 * g10);
+        const float c2 = s_beta[buf][2] * (z2 - c0 * g20 - c1 * g21);
+        const float c3 = s_beta[buf][3] * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
 #pragma unroll
         for (int m = 0; m < kCols; ++m) {
           if (32 * m < rp) {
             const int i = lane + 32 * m;
-            zr[m] -= fma(c0, v0[i], fma(c1, v1[i], fma(c2, v2[i], c3 * v3[i])));
+            zr[m] -= fmaf(c0, v0[i], fmaf(c1, v1[i], fmaf(c2, v2[i], c3 * v3[i])));
           }
         }
       }
-      if (gi + 1 < ngroups) store_group(gi + 1, buf ^ 1);
-      __syncthreads();
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (have) {
-      double n2 = 0.0;
+      float n2 = 0.0f;
 #pragma unroll
-      for (int m = 0; m < kCols; ++m) n2 = fma(zr[m], zr[m], n2);
+      for (int m = 0; m < kCols; ++m) n2 = fmaf(zr[m], zr[m], n2);
       n2 = warp_sum(n2);
-      const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
+      const float inv = n2 > 0.0f ? rsqrtf(n2) : 0.0f;
 #pragma unroll
-      for (int m = 0; m < kCols; ++m) { const int i = lane + 32 * m; if (i < r) L.shortv[(int64_t)a * r + i] = (float)(zr[m] * inv); }
+      for (int m = 0; m < kCols; ++m) { const int i = lane + 32 * m; if (i < r) gShort[(int64_t)a * r + i] = zr[m] * inv; }
     }
   }
   // the last CTA of the layer orthogonalises kept atoms whose eigenvalues nearly coincide (their vectors are
@@ -557,13 +564,13 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
   if (!s_last || w != 0 || k < 2) return;
   __threadfence();
   for (uint32_t a = 1; a < k; ++a) {
-    const double la = L.lam64[L.perm[L.idx[a]]];
+    const double la = gLam[gPerm[gIdx[a]]];
     bool changed = false;
     for (uint32_t b = 0; b < a; ++b) {
-      const double lb = L.lam64[L.perm[L.idx[b]]];
+      const double lb = gLam[gPerm[gIdx[b]]];
       if (fabs(la - lb) > kSameEig) continue;
-      volatile float* va = L.shortv + (int64_t)a * r;
-      const volatile float* vb = L.shortv + (int64_t)b * r;
+      volatile float* va = gShort + (int64_t)a * r;
+      const volatile float* vb = gShort + (int64_t)b * r;
       double dot = 0.0;
       for (int i = lane; i < r; i += 32) dot = fma((double)va[i], (double)vb[i], dot);
       dot = warp_sum(dot);
@@ -572,7 +579,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       changed = true;
     }
     if (changed) {
-      volatile float* va = L.shortv + (int64_t)a * r;
+      volatile float* va = gShort + (int64_t)a * r;
       double n2 = 0.0;
       for (int i = lane; i < r; i += 32) n2 = fma((double)va[i], (double)va[i], n2);
       n2 = warp_sum(n2);
@@ -585,7 +592,9 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
 
 // ---- host side ---------------------------------------------------------------------------------------------------
 static size_t tri_smem_bytes(int) { return 0; }             // rows in registers, vectors in static shared memory
-static size_t vec_smem_bytes(int rp_max) { return (size_t)(2 + 2 * kVecGroup + 3 * kVecWarps) * rp_max * sizeof(double); }
+static size_t vec_smem_bytes(int rp_max) {
+  return (size_t)(2 + 3 * kVecWarps) * rp_max * sizeof(double) + (size_t)kVecStages * kVecGroup * rp_max * sizeof(float);
+}
 
 int sp_tridiag_max_rp() { return kTriMaxRp; }
 int sp_tridiag_cluster_ctas() { return kTriCtas; }
