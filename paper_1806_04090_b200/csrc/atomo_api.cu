@@ -414,7 +414,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       }
       d.td_d = A.take<double>(d.tri ? d.rp : 0); d.td_e = A.take<double>(d.tri ? d.rp : 0);
       d.td_tau = A.take<double>(d.tri ? d.rp : 0); d.lam64 = A.take<double>(d.tri ? d.rp : 0);
-      d.td_V = A.take<float>(d.tri ? (size_t)d.r * d.r : 0);
+      d.td_ldv = (d.r + 3) / 4 * 4;
+      d.td_V = A.take<float>(d.tri ? (size_t)d.r * d.td_ldv : 0);
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
       d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);

@@ -93,7 +93,8 @@ struct SpLayer {
   int tri;                     // this layer takes the tridiagonal route
   double* td_d; double* td_e;  // rp each: diagonal and off-diagonal of T
   double* td_tau;              // rp: beta_k of the reflectors H_k = I - beta_k v_k v_k^T
-  float* td_V;                 // r x r: row k = v_k / ||v_k|| (zero up to index k), fp32 for the back-transformation: H_k = I - 2 u u^T
+  int td_ldv;                  // floats per row of td_V: r rounded up to a multiple of 4 (16-byte rows)
+  float* td_V;                 // r x td_ldv: row k = v_k / ||v_k|| (zero up to index k), fp32 for the back-transformation: H_k = I - 2 u u^T
   double* lam64;               // rp: eigenvalues of T, ascending (scaled units); lam holds the same in fp32
   uint32_t* vec_ticket;        // CTAs of the vector kernel that finished this layer; zeroed per call
 };

@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   const int r = L.r, nc = me.pad, g = me.slot, base = me.base_rank;
   // the layer's pointers in registers: a field read through `layers` inside a loop would be a global load each time
   double* const td_d = L.td_d; double* const td_e = L.td_e; double* const td_tau = L.td_tau; float* const td_V = L.td_V;
-  const float* const gA = L.A; const int64_t lda = L.lda;
+  const float* const gA = L.A; const int64_t lda = L.lda; const int ldv = L.td_ldv;
   const int my_steps = max(r - 2, 0);
   const int li0 = w, li1 = w + kTriWarps;                     // this warp's two rows
   const int i0 = li0 * nc + g, i1 = li1 * nc + g;
@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     {
       // reflectors are filed as unit vectors (H = I - 2 u u^T, u = v sqrt(beta / 2)): no range trouble in fp32
       const double un = sqrt(0.5 * beta);
-      if (g == 0) for (int j = tid; j < r; j += kTriThreads) td_V[j] = (float)(s_v[0][(j % nc) * 32 + j / nc] * un);
+      if (g == 0) for (int j = tid; j < r; j += kTriThreads) td_V[j] = (float)(s_v[0][(j % nc) * 32 + j / nc] * un);   // row 0
     }
     double a0 = 0.0, a1 = 0.0;
 #pragma unroll
@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     if (active && !last && (k + 1) % nc == g) {               // meanwhile one CTA of the layer files the reflector
       if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
       const double un = sqrt(0.5 * beta_n);                   // filed as a unit vector: H = I - 2 u u^T
-      for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * r + j] = (float)(s_v[nxt][(j % nc) * 32 + j / nc] * un);
+      for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * ldv + j] = (float)(s_v[nxt][(j % nc) * 32 + j / nc] * un);
     }
     beta = beta_n; v0 = v0_n;
     cluster.barrier_wait();
@@ -344,23 +344,27 @@ constexpr int kVecWarps = kVecThreads / 32;
 constexpr int kVecCtasPerLayer = 4;
 constexpr int kVecGroup = 4;          // reflectors applied together in the back-transformation
 constexpr int kVecStages = 4;         // groups in flight between global and shared memory
+constexpr int kVecWork = 5;           // work vectors of the twisted factorisation per warp
 constexpr double kPivMin = 1.0e-280;
 constexpr double kSameEig = 1.0e-9;   // scaled units (largest eigenvalue below 1): eigenvalues this close share a subspace
 
-// Twisted factorisation of T - lambda I (forward pivots D+ in lane 0, backward pivots D- in lane 1, the same
-// instructions on mirrored indices), twist index at the smallest |gamma_k| = |D+_k + D-_k - (d_k - lambda)|,
+// Twisted factorisation of T - lambda I: forward pivots D+_i = p_i / p_{i-1} from the leading principal minors
+// p_i = (d_i - lambda) p_{i-1} - e_{i-1}^2 p_{i-2} (lane 0), backward pivots D- from the trailing ones (lane 1, the same
+// instructions on mirrored indices).  The recurrences carry no division: numerator and denominator of every pivot
+// are stored as a pair (the running pair is rescaled by a power of two every 8 steps, after it was stored) and the
+// quotients are taken by all lanes afterwards.  Twist index at the smallest |gamma_k| = |D+_k + D-_k - (d_k - lambda)|,
 // z_k = 1, z_i = -(e_i / D+_i) z_{i+1} above and z_{i+1} = -(e_i / D-_{i+1}) z_i below.  Returns gamma_k / z^T z, the
-// Rayleigh-quotient correction of lambda.  wa, wb, z: r doubles each in shared memory.
+// Rayleigh-quotient correction of lambda.  wa, wb, wc, wd, z: r doubles each in shared memory.
 __device__ double twisted_vector(const double* __restrict__ d, const double* __restrict__ e, int r, double lambda,
-                                 double* wa, double* wb, double* z, int lane, int skip, double* znorm2) {
+                                 double* wa, double* wb, double* wc, double* wd, double* z, int lane, int skip,
+                                 double* znorm2) {
   if (lane < 2) {
     const bool back = lane == 1;
-    double* D = back ? wb : wa;
+    double* N = back ? wb : wa;                               // numerators
+    double* Q = back ? wd : wc;                               // denominators
     int cur = back ? r - 1 : 0;
-    double piv = d[cur] - lambda;
-    if (fabs(piv) < kPivMin) piv = kPivMin;
-    D[cur] = piv;
-    // piv_next = (d_next - lambda) - e^2 / piv: the operands of step t+1 are fetched while step t's reciprocal runs
+    double pm = 1.0, p = d[cur] - lambda;
+    N[cur] = p; Q[cur] = pm;
     double ee = r > 1 ? e[back ? r - 2 : 0] : 0.0;
     double dn = r > 1 ? d[back ? r - 2 : 1] : 0.0;
     for (int t = 0; t + 1 < r; ++t) {
@@ -368,11 +372,26 @@ __device__ double twisted_vector(const double* __restrict__ d, const double* __r
       const int ie2 = back ? max(r - 3 - t, 0) : min(t + 1, r - 2);      // next step's off-diagonal and diagonal
       const int in2 = back ? max(nxt - 1, 0) : min(nxt + 1, r - 1);
       const double ee2 = e[ie2], dn2 = d[in2];
-      piv = fma(-(ee * ee), __drcp_rn(piv), dn - lambda);
-      if (fabs(piv) < kPivMin) piv = kPivMin;
-      D[nxt] = piv;
+      const double pn = fma(dn - lambda, p, -(ee * ee) * pm);
+      N[nxt] = pn; Q[nxt] = p;
+      pm = p; p = pn;
+      if ((t & 7) == 7) {
+        const int ex = ((__double2hiint(fabs(p) + fabs(pm)) >> 20) & 0x7ff) - 1023;
+        const double sc = __hiloint2double((1023 - max(min(ex, 1022), -1022)) << 20, 0);
+        p *= sc; pm *= sc;
+      }
       cur = nxt; ee = ee2; dn = dn2;
     }
+  }
+  __syncwarp();
+  // pivots: wa <- D+, wb <- D- (a zero or non-finite quotient is replaced, as a perturbed pivot would be)
+  for (int i = lane; i < r; i += 32) {
+    double dp = wa[i] / wc[i], dm = wb[i] / wd[i];
+    if (!(fabs(dp) >= kPivMin)) dp = kPivMin;
+    if (!(fabs(dm) >= kPivMin)) dm = kPivMin;
+    if (!finite64(dp)) dp = 1.0e300;
+    if (!finite64(dm)) dm = 1.0e300;
+    wa[i] = dp; wb[i] = dm;
   }
   __syncwarp();
   // twist index: the (skip+1)-th smallest |gamma| (lowest index on ties).  skip > 0 for the later members of a group
@@ -434,22 +453,24 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
   const int r = L.r, rp = L.rp;
   double* s_d = reinterpret_cast<double*>(vec_smem);          // [rp]
   double* s_e = s_d + rp;                                     // [rp]
-  double* s_work = s_e + rp;                                  // [warps][3][rp]
-  float* s_ref = reinterpret_cast<float*>(s_work + (size_t)kVecWarps * 3 * rp);   // [kVecStages][kVecGroup][rp] ring of reflector groups
+  double* s_work = s_e + rp;                                  // [warps][kVecWork][rp]
+  float* s_ref = reinterpret_cast<float*>(s_work + (size_t)kVecWarps * kVecWork * rp);   // [kVecStages][kVecGroup][rp] ring of reflector groups
   __shared__ float s_beta[kVecStages][kVecGroup];
   __shared__ uint32_t s_last;
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const uint32_t k = L.hdr->k;
   // the layer's pointers in registers (a field read through `layers` inside a loop is a global load each time)
-  const float* const gV = L.td_V; const double* const gLam = L.lam64;
+  const float* const gV = L.td_V; const int ldv = L.td_ldv; const double* const gLam = L.lam64;
   const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
   const int nref = max(r - 2, 0);
   const int ngroups = (nref + kVecGroup - 1) / kVecGroup;
   for (int i = tid; i < r; i += kVecThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
   __syncthreads();
-  double* wa = s_work + (size_t)w * 3 * rp;
+  double* wa = s_work + (size_t)w * kVecWork * rp;
   double* wb = wa + rp;
-  double* z = wb + rp;
+  double* wc = wb + rp;
+  double* wd = wc + rp;
+  double* z = wd + rp;
   constexpr int kCols = kTriCols;
   for (uint32_t a0 = blockIdx.y * kVecWarps; a0 < k; a0 += kVecCtasPerLayer * kVecWarps) {
     const uint32_t a = a0 + w;
@@ -465,7 +486,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       for (uint32_t b = lane; b < a; b += 32) skip += fabs(gLam[gPerm[gIdx[b]]] - lambda) <= kSameEig ? 1 : 0;
       skip = (int)warp_sum((uint32_t)skip);
       double n2 = 1.0;
-      const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, z, lane, skip, &n2);
+      const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, z, lane, skip, &n2);
       // the vector's error is about |correction| / gap to the nearest other eigenvalue: well-separated atoms are done
       double gap = 1.0e300;
       if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
@@ -473,7 +494,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {   // one Rayleigh-quotient step, then the vector again
         lambda += corr;
         __syncwarp();
-        twisted_vector(s_d, s_e, r, lambda, wa, wb, z, lane, 0, &n2);
+        twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, z, lane, 0, &n2);
       }
       const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
 #pragma unroll
@@ -491,13 +512,12 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
         const int buf = gi % kVecStages;
         const int q = w & (kVecGroup - 1);
         const int kk = nref - 1 - kVecGroup * gi - q;
-        const float* srow = gV + (int64_t)max(kk, 0) * r;
+        const float* srow = gV + (int64_t)max(kk, 0) * ldv;   // rows start on 16-byte boundaries (ldv is a multiple of 4)
         float* drow = s_ref + ((size_t)buf * kVecGroup + q) * rp;
-        for (int i = (w / kVecGroup) * 32 + lane; i < rp; i += 32 * (kVecWarps / kVecGroup)) {
-          const bool in = kk >= 0 && i < r;
+        for (int i = 4 * ((w / kVecGroup) * 32 + lane); i < rp; i += 4 * 32 * (kVecWarps / kVecGroup)) {
+          const int bytes = kk >= 0 ? 4 * max(0, min(4, r - i)) : 0;   // the rest of the 16 bytes is filled with zeros
           const uint32_t dst = (uint32_t)__cvta_generic_to_shared(drow + i);
-          const int bytes = in ? 4 : 0;                       // 0: the destination is filled with zeros
-          asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(in ? srow + i : gV), "r"(bytes) : "memory");
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(bytes ? srow + i : gV), "r"(bytes) : "memory");
         }
         if (tid < kVecGroup) { const int kq = nref - 1 - kVecGroup * gi - tid; s_beta[buf][tid] = kq >= 0 ? 2.0f : 0.0f; }   // unit reflectors
       }
@@ -593,7 +613,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
 // ---- host side ---------------------------------------------------------------------------------------------------
 static size_t tri_smem_bytes(int) { return 0; }             // rows in registers, vectors in static shared memory
 static size_t vec_smem_bytes(int rp_max) {
-  return (size_t)(2 + 3 * kVecWarps) * rp_max * sizeof(double) + (size_t)kVecStages * kVecGroup * rp_max * sizeof(float);
+  return (size_t)(2 + kVecWork * kVecWarps) * rp_max * sizeof(double) + (size_t)kVecStages * kVecGroup * rp_max * sizeof(float);
 }
 
 int sp_tridiag_max_rp() { return kTriMaxRp; }
