@@ -532,16 +532,21 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
       if (have) {
         const float* v0 = s_ref + ((size_t)buf * kVecGroup + 0) * rp;
         const float* v1 = v0 + rp; const float* v2 = v1 + rp; const float* v3 = v2 + rp;
+        // the group's four reflectors into registers first (64 loads in flight), then the arithmetic
+        float r0[kCols], r1[kCols], r2[kCols], r3[kCols];
+#pragma unroll
+        for (int m = 0; m < kCols; ++m) {
+          const int i = lane + 32 * m;
+          const bool in = 32 * m < rp;
+          r0[m] = in ? v0[i] : 0.0f; r1[m] = in ? v1[i] : 0.0f; r2[m] = in ? v2[i] : 0.0f; r3[m] = in ? v3[i] : 0.0f;
+        }
         float z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
 #pragma unroll
         for (int m = 0; m < kCols; ++m) {
-          if (32 * m < rp) {
-            const int i = lane + 32 * m;
-            const float a0v = v0[i], a1v = v1[i], a2v = v2[i], a3v = v3[i], zz = zr[m];
-            z0 = fmaf(a0v, zz, z0); z1 = fmaf(a1v, zz, z1); z2 = fmaf(a2v, zz, z2); z3 = fmaf(a3v, zz, z3);
-            g10 = fmaf(a1v, a0v, g10); g20 = fmaf(a2v, a0v, g20); g21 = fmaf(a2v, a1v, g21);
-            g30 = fmaf(a3v, a0v, g30); g31 = fmaf(a3v, a1v, g31); g32 = fmaf(a3v, a2v, g32);
-          }
+          const float zz = zr[m];
+          z0 = fmaf(r0[m], zz, z0); z1 = fmaf(r1[m], zz, z1); z2 = fmaf(r2[m], zz, z2); z3 = fmaf(r3[m], zz, z3);
+          g10 = fmaf(r1[m], r0[m], g10); g20 = fmaf(r2[m], r0[m], g20); g21 = fmaf(r2[m], r1[m], g21);
+          g30 = fmaf(r3[m], r0[m], g30); g31 = fmaf(r3[m], r1[m], g31); g32 = fmaf(r3[m], r2[m], g32);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -556,12 +561,7 @@ __global__ void __launch_bounds__(kVecThreads, 1) sp_eigvec_kernel(const SpLayer
         const float c2 = s_beta[buf][2] * (z2 - c0 * g20 - c1 * g21);
         const float c3 = s_beta[buf][3] * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
 #pragma unroll
-        for (int m = 0; m < kCols; ++m) {
-          if (32 * m < rp) {
-            const int i = lane + 32 * m;
-            zr[m] -= fmaf(c0, v0[i], fmaf(c1, v1[i], fmaf(c2, v2[i], c3 * v3[i])));
-          }
-        }
+        for (int m = 0; m < kCols; ++m) zr[m] -= fmaf(c0, r0[m], fmaf(c1, r1[m], fmaf(c2, r2[m], c3 * r3[m])));
       }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
