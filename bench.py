@@ -30,6 +30,9 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # SMs x FP32 lanes x
 # dram__bytes_read.sum + dram__bytes_write.sum of one sp_jacobi_cluster_kernel launch on this workload, from the
 # ncu capture summarised in profiles/sp_jacobi_cluster_c2.txt (5.66 MB read, nothing written back to DRAM)
 JACOBI_TRAFFIC_BYTES_PER_LAUNCH = 5660672
+FP64_FMA_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12        # SMs x FP64 lanes x 2 flop x max SM clock
+# the same two counters for one sp_tridiag_cluster_kernel launch (profiles/sp_tridiag_cluster_c2.txt)
+TRIDIAG_TRAFFIC_BYTES_PER_LAUNCH = None
 
 
 def measured_peaks():
@@ -195,6 +198,13 @@ def jacobi_flops(shapes, sweeps):
         r = min(rows, cols)
         tot += sw * (r * (r - 1) / 2.0) * 8.0 * r
     return tot
+
+
+def tridiag_flops(shapes):
+    """Algorithmic flops of the Householder reduction of the r x r Gram matrix to tridiagonal form as the kernel
+    does it (full symmetric storage): step k works on the trailing block of order m = r - k - 1 with one
+    matrix-vector product (2 m^2 flop) and one rank-two update (4 m^2 flop): 2 r^3 in all, in fp64."""
+    return sum(2.0 * min(rows, cols) ** 3 for rows, cols in shapes)
 
 
 def entrywise_extra(a, dev, measured_hbm_gbs, steps=20):
@@ -377,10 +387,13 @@ def run_ours(args):
 
     if rank == 0:
         peaks = measured_peaks()
-        flops = jacobi_flops(shapes, sweeps_seen)          # of the last step; sweeps vary little between steps
+        tri = eig_scheme == 3
+        # dominant kernel: the fp64 tridiagonal reduction (scheme 3) or the fp32 Jacobi eigen-solve (other schemes)
+        flops = tridiag_flops(shapes) if tri else jacobi_flops(shapes, sweeps_seen)   # sweeps of the last step; they vary little
         eig_s_per_step = eig_ms * 1e-3 / args.steps
         launches_per_step = eig_launches / args.steps
         achieved = flops / eig_s_per_step / 1e12
+        alu_peak = FP64_FMA_PEAK_TFLOPS if tri else FP32_FMA_PEAK_TFLOPS
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -393,7 +406,8 @@ def run_ours(args):
                                        "nccl": "data-parallel: payload all-gather + averaging decode",
                                        "p2p": "data-parallel: averaging decode reads the peers' payloads over NVLink"}[exchange]
                        if world > 1 else "single GPU",
-                       "jacobi_sweeps_last_step": sweeps_seen,
+                       "eigen_scheme": eig_scheme,
+                       "jacobi_sweeps_last_step": None if tri else sweeps_seen,
                        "eig_ms_per_step": eig_ms / args.steps},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes,
@@ -401,14 +415,17 @@ def run_ours(args):
                     "overlap": "copies of step k+1 (in) and k-1 (out) run on two copy streams under step k's kernels"},
             "gpu_launches": int(launches),
             "roofline": {"bound": "alu",
-                         "kernel": {2: "sp_jacobi_cluster_kernel", 1: "sp_jacobi_persistent_kernel"}.get(eig_scheme, "sp_jacobi_step_kernel"),
+                         "kernel": {3: "sp_tridiag_cluster_kernel", 2: "sp_jacobi_cluster_kernel",
+                                    1: "sp_jacobi_persistent_kernel"}.get(eig_scheme, "sp_jacobi_step_kernel"),
                          "achieved": achieved,
-                         "peak": FP32_FMA_PEAK_TFLOPS, "unit": "TFLOP/s", "frac": achieved / FP32_FMA_PEAK_TFLOPS,
-                         "traffic": JACOBI_TRAFFIC_BYTES_PER_LAUNCH if eig_scheme == 2 else None,
+                         "peak": alu_peak, "unit": "TFLOP/s", "frac": achieved / alu_peak,
+                         "traffic": TRIDIAG_TRAFFIC_BYTES_PER_LAUNCH if tri else (JACOBI_TRAFFIC_BYTES_PER_LAUNCH if eig_scheme == 2 else None),
                          "launches_per_step": 1.0 if launches_per_step <= 2 else launches_per_step,
                          "avg_launch_us": eig_s_per_step / (1.0 if launches_per_step <= 2 else launches_per_step) * 1e6,
                          "share_of_step": eig_ms / ms_total,
-                         "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz (no measured FP32 peak on file)",
+                         "peak_source": ("derived: 148 SMs x 64 FP64 lanes x 2 flop x 1.965 GHz (no measured FP64 peak on file)" if tri else
+                                         "derived: 148 SMs x 128 FP32 lanes x 2 flop x 1.965 GHz (no measured FP32 peak on file)"),
+                         "arithmetic": "f64" if tri else "f32",
                          "hbm_peak_gbs": peaks["hbm_gbs"], "hbm_peak_source": peaks["source"]},
         }
         if world == 1 and not args.no_extras:

@@ -117,7 +117,9 @@ typedef struct {
 typedef struct { float* sigma; float* prob; uint32_t* mask_words; float* short_vecs; } atomo_debug;
 
 /* Stage timers (milliseconds of device time, CUDA events on the call's stream) filled while
- * profiling is on.  `launches[i]` counts the kernels of stage i in the last call.             */
+ * profiling is on.  `launches[i]` counts the kernels of stage i in the last call.  On the
+ * tridiagonal route EIG is the Householder reduction alone; the bisection for the eigenvalues
+ * is timed with SAMPLE and the vectors of the kept atoms with BACKPROJECT.                    */
 enum { ATOMO_STAGE_GRAM = 0, ATOMO_STAGE_EIG, ATOMO_STAGE_SAMPLE, ATOMO_STAGE_BACKPROJECT,
        ATOMO_STAGE_EW_REDUCE, ATOMO_STAGE_EW_PACK, ATOMO_STAGE_DECODE, ATOMO_N_STAGES };
 
@@ -249,8 +251,15 @@ int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
 /* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
  * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
-/* Eigen-solver launch scheme (`enabled` = 0, 1 or 2):
- * 2 (default) = thread-block clusters where they apply: when every layer of the batch has at most 16 block
+/* Eigen-solver scheme (`enabled` = 0, 1, 2 or 3):
+ * 3 (default) = tridiagonal route where it applies: when every layer of the batch has a short side of at most 512
+ *     (and neither per-atom refinement nor the whole short-side basis is asked for), the scaled Gram matrix is
+ *     reduced to tridiagonal form by Householder reflectors in fp64 (rows spread over the CTAs of a 16-CTA
+ *     cluster, exchanged through distributed shared memory, one cluster barrier per step), all eigenvalues come
+ *     from bisection on Sturm counts, and eigenvectors are computed for the kept atoms only (twisted
+ *     factorisation, back-transformation with the reflectors).  Only the singular values of all atoms enter the
+ *     probabilities; the vectors of atoms that are not kept are never formed.  Other batches take scheme 2;
+ * 2 = one-sided Jacobi in thread-block clusters where they apply: when every layer of the batch has at most 16 block
  *     pairs (padded short side <= 512), each layer's CTAs sit in one 16-CTA cluster for the whole solve and hand
  *     their blocks to one another through distributed shared memory, with a cluster barrier per Jacobi step;
  *     other batches, or a GPU that cannot place such clusters, take scheme 1;
@@ -259,9 +268,9 @@ int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
  *     of a layer between steps; a batch that fits the GPU is one such launch.  A batch with a layer that alone
  *     needs more CTAs than the GPU holds (short side above 2048) takes scheme 0;
  * 0 = one launch per step and one host wait per sweep.
- * Schemes 1 and 2 wait on the host once, at the end of the solve.                                            */
+ * Schemes 1 to 3 wait on the host once, at the end of the call.                                              */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
-/* The scheme (0, 1 or 2 as above) that the last atomo_encode_spectral() of this context actually ran; -1 before
+/* The scheme (0 to 3 as above) that the last atomo_encode_spectral() of this context actually ran; -1 before
  * the first call.  Host only.                                                                                */
 int atomo_last_eig_scheme(atomo_ctx* ctx);
 

@@ -512,8 +512,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
     const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
-    launch_sp_bisect(d_layers, n_layers, r_max, st);
-    n_eig_launch = 2;
+    n_eig_launch = 1;                                      // the eigenvalues (bisection) are timed with the sampling stage
     CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     flags_pending = true;                                  // the Gram kernel's bounded waits report at the end of the call
@@ -586,10 +585,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S2-S4: (refined singular values,) probabilities, draws, compaction ----
   stage_begin(ctx, ATOMO_STAGE_SAMPLE, st);
+  if (tri_form) launch_sp_bisect(d_layers, n_layers, r_max, st);   // all eigenvalues of the tridiagonal matrices
   launch_sp_refine(d_layers, n_layers, d_ref, (int)refine_tiles.size(), st);
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps, st);
-  stage_end(ctx, ATOMO_STAGE_SAMPLE, st, 1);
+  stage_end(ctx, ATOMO_STAGE_SAMPLE, st, tri_form ? 2 : 1);
 
   // ---- S4: long-side vectors of the kept atoms ----
   stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);

@@ -220,6 +220,7 @@ def test_sweep_cap_reports_not_converged(atomo):
     G = synth.c2_resnet18(0, [synth.RESNET18_LAYERS[5]])[0]
     t = torch.from_numpy(G).cuda()
     atomo.set_eig_params(1, 3e-7)
+    atomo.set_persistent_eig(2)                       # the Jacobi routes are the iterative ones (the tridiagonal route has no sweeps)
     try:
         pay, _ = atomo.atomo_encode_spectral([t], 2.0, seed=1, k_cap=128)
         assert atomo.payload_status(pay) == (5, 0) and pay.headers()[1][0].k == 0
@@ -232,6 +233,7 @@ def test_sweep_cap_reports_not_converged(atomo):
     finally:
         atomo.set_eig_params(40, 3e-7)
         atomo.set_eig_mode(1)
+        atomo.set_persistent_eig(3)
 
 
 def test_unbiased_on_gpu(atomo):
