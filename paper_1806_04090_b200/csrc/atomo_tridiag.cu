@@ -93,7 +93,8 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   __shared__ double s_v[2][kTriMaxRp];                        // v of step k in s_v[k & 1]
   __shared__ double s_w[kTriMaxRp];
   __shared__ double s_stage[2][kTriRows];                     // this CTA's 32 entries of p and c on their way out
-  __shared__ double s_red1[kTriWarps], s_red2[kTriWarps];
+  __shared__ double s_pk[2][kTriCtas];                        // the CTAs' parts of p^T v, sent along with p (same parity)
+  __shared__ double s_red2[kTriWarps];
   __shared__ double s_x0, s_scal[3];                          // first entry of the next pivot column; alpha, beta, v_0 of the next reflector
   const ClusterCta me = ctas[blockIdx.x];
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
@@ -169,8 +170,12 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   }
   __syncthreads();
   if (my_steps > 0 && w < nc) {                               // warp w carries this CTA's 32 entries to peer w
-    cluster.map_shared_rank(&s_p[0][0], base + w)[g * 32 + lane] = s_stage[0][lane];
+    const double pl = s_stage[0][lane];
+    cluster.map_shared_rank(&s_p[0][0], base + w)[g * 32 + lane] = pl;
     cluster.map_shared_rank(&s_c[0][0], base + w)[g * 32 + lane] = s_stage[1][lane];
+    // ... and this CTA's part of p^T v (its 32 rows), from which every CTA forms K without a reduction of its own
+    const double part = warp_sum(pl * s_v[0][g * 32 + lane]);
+    if (lane == 0) cluster.map_shared_rank(&s_pk[0][0], base + w)[g] = part;
   }
   cluster.sync();
   for (int k = 0; k < steps; ++k) {
@@ -181,10 +186,13 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     const int q2 = ((k + 2) % nc) * 32 + (k + 2) / nc;
     double beta_n = 0.0, v0_n = 0.0;
     if (active) {
-      // K = beta/2 p^T v, each thread one entry
+      // K = beta/2 p^T v: the CTAs' parts arrived with p; every thread adds them in the same order
       const double vq = slice ? s_v[par][sq] : 0.0;
       const double pq = slice ? s_p[par][sq] : 0.0;
-      const double K = 0.5 * beta * tri_block_sum(pq * vq, s_red1, lane, w);
+      double ksum = (lane & (kTriCtas - 1)) < nc ? s_pk[par][lane & (kTriCtas - 1)] : 0.0;
+#pragma unroll
+      for (int o = kTriCtas / 2; o > 0; o >>= 1) ksum += __shfl_xor_sync(0xffffffffu, ksum, o);
+      const double K = 0.5 * beta * ksum;
       const double w1 = fma(-K, v0, s_p[par][q1]);            // w_{k+1}
       // w, and the next pivot column x_j = c_j - v_j w_{k+1} - w_j v_{k+1} for j > k+1
       const double wq = fma(-K, vq, pq);
@@ -245,8 +253,11 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     }
     __syncthreads();
     if (active && !last && w < nc) {
-      cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[0][lane];
+      const double pl = s_stage[0][lane];
+      cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = pl;
       cluster.map_shared_rank(&s_c[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
+      const double part = warp_sum(pl * s_v[nxt][g * 32 + lane]);
+      if (lane == 0) cluster.map_shared_rank(&s_pk[0][0], base + w)[nxt * kTriCtas + g] = part;
     }
     cluster.barrier_arrive();                                 // (release) the entries above are on their way
     if (active && !last && (k + 1) % nc == g) {               // meanwhile one CTA of the layer files the reflector
