@@ -284,22 +284,33 @@ __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const d
   double pm = 1.0, p = d[0] - x;
   int neg = __double2hiint(p);                                // sign bit of the previous term
   int cnt = (uint32_t)neg >> 31;
-  for (int i = 1; i < r; ++i) {
-    const double pn = fma(d[i] - x, p, -e2[i - 1] * pm);
-    const int hn = __double2hiint(pn);
-    cnt += (uint32_t)(hn ^ neg) >> 31;
-    neg = hn;
-    pm = p; p = pn;
-    if ((i & 7) == 0) {
-      const int ex = ((__double2hiint(fabs(p) + fabs(pm)) >> 20) & 0x7ff) - 1023;
-      const double sc = __hiloint2double((1023 - max(min(ex, 1022), -1022)) << 20, 0);
-      p *= sc; pm *= sc;
+  // eight steps at a time: their operands are fetched together, so that only the multiply-add chain is serial.
+  // Past the end the step is p <- 1 * p - 0 * p_prev: no sign change.
+  for (int i0 = 1; i0 < r; i0 += 8) {
+    double dd[8], ee[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u;
+      const bool in = i < r;
+      dd[u] = in ? d[i] - x : 1.0;
+      ee[u] = in ? e2[i - 1] : 0.0;
     }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const double pn = fma(dd[u], p, -ee[u] * pm);
+      const int hn = __double2hiint(pn);
+      cnt += (uint32_t)(hn ^ neg) >> 31;
+      neg = hn;
+      pm = p; p = pn;
+    }
+    const int ex = ((__double2hiint(fabs(p) + fabs(pm)) >> 20) & 0x7ff) - 1023;
+    const double sc = __hiloint2double((1023 - max(min(ex, 1022), -1022)) << 20, 0);
+    p *= sc; pm *= sc;
   }
   return cnt;
 }
 
-constexpr int kBisThreads = 256;
+constexpr int kBisThreads = 64;           // small CTAs: the warps of a large layer spread over all SMs (the recurrences are latency-bound)
 constexpr int kBisLanes = 8;          // points per round and eigenvalue: the interval shrinks 9 times per round
 constexpr int kBisRounds = 13;        // 9^13 = 2.5e12: interval width below 1e-12 of the spectrum's extent
 constexpr int kBisPerCta = kBisThreads / kBisLanes;
