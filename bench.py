@@ -32,7 +32,7 @@ FP32_FMA_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # SMs x FP32 lanes x
 JACOBI_TRAFFIC_BYTES_PER_LAUNCH = 5660672
 FP64_FMA_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12        # SMs x FP64 lanes x 2 flop x max SM clock
 # the same two counters for one sp_tridiag_cluster_kernel launch (profiles/sp_tridiag_cluster_c2.txt)
-TRIDIAG_TRAFFIC_BYTES_PER_LAUNCH = None
+TRIDIAG_TRAFFIC_BYTES_PER_LAUNCH = 5638912
 
 
 def measured_peaks():
