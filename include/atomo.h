@@ -14,9 +14,12 @@
  *     descriptors (atomo_mat, atomo_vec, pointer lists, shape lists) are HOST memory and are
  *     consumed before the call returns.
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
- *     atomo_encode_spectral waits on the host once, after it has enqueued all its work (the kernels' bounded
- *     waits report there), or once per Jacobi sweep in launch scheme 0; atomo_encode_entrywise and the decode
- *     calls never synchronise.  No claim is made about capture in a CUDA graph.
+ *     atomo_encode_spectral on the tridiagonal route (eigen scheme 3, the default for short sides <= 512) never
+ *     waits on the host: a bounded device-side wait that ran out shows as ATOMO_ERR_TIMEOUT in the layers' status
+ *     words.  On the Jacobi routes it waits once, after it has enqueued all its work (the kernels' bounded waits
+ *     report there), or once per Jacobi sweep in launch scheme 0.  atomo_encode_entrywise and the decode calls
+ *     never synchronise.  A call that grows the workspace (first call, or a larger batch) does synchronise the
+ *     device (cudaMalloc / cudaFree).  No claim is made about capture in a CUDA graph.
  *   - Matrices are fp32 row-major with leading dimension `ld` (elements, ld >= cols).
  *   - Functions return an atomo_status.  Problems visible on the host (NULL, bad sizes,
  *     s <= 0 or not finite, payload capacity too small) return at once and launch nothing.
@@ -233,6 +236,11 @@ int atomo_payload_status(atomo_ctx* ctx, const void* payload /*DEVICE*/, int32_t
 int atomo_set_profiling(atomo_ctx* ctx, int enabled);
 /* ms[ATOMO_N_STAGES], launches[ATOMO_N_STAGES] for the last encode/decode call (synchronises). */
 int atomo_get_stage_times(atomo_ctx* ctx, float* ms /*HOST*/, int64_t* launches /*HOST*/);
+/* Sums over all encode / decode calls since profiling was last switched on: ms[ATOMO_N_STAGES] of device time,
+ * launches[ATOMO_N_STAGES], and the number of calls (any pointer may be NULL).  The calls themselves record events
+ * only and never wait for them; this function waits for the newest ones.  Lets a caller time a run of
+ * asynchronous steps without a host wait inside it.                                                        */
+int atomo_get_stage_totals(atomo_ctx* ctx, double* ms /*HOST*/, int64_t* launches /*HOST*/, int64_t* calls /*HOST*/);
 
 /* Eigen-solver knobs: max Jacobi sweeps (default 40) and the relative rotation threshold
  * (default 3e-7: rows p, q are rotated while |<x_p,x_q>| > tol ||x_p|| ||x_q||).               */

@@ -31,7 +31,7 @@ EXPORTS = [
     "atomo_payload_bytes_entrywise", "atomo_encode_spectral", "atomo_encode_entrywise", "atomo_decode",
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
-    "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format",
+    "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
 ]
 
 
@@ -107,6 +107,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_payload_status.argtypes = [vp, vp, i32, ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
     lib.atomo_set_profiling.argtypes = [vp, ctypes.c_int]
     lib.atomo_get_stage_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i64)]
+    lib.atomo_get_stage_totals.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.atomo_set_eig_params.argtypes = [vp, i32, ctypes.c_float]
     lib.atomo_set_eig_mode.argtypes = [vp, i32]
     lib.atomo_set_sigma_refinement.argtypes = [vp, i32]
@@ -464,6 +465,16 @@ class Atomo:
         ln = (ctypes.c_int64 * len(STAGES))()
         self._check(self.lib.atomo_get_stage_times(self._h, ms, ln), "atomo_get_stage_times")
         return {k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)}
+
+    def stage_totals(self):
+        """(ms per stage, launches per stage, calls) summed over all encode / decode calls since profiling was switched
+        on; the calls themselves do not wait for their events, this does."""
+        ms = (ctypes.c_double * len(STAGES))()
+        ln = (ctypes.c_int64 * len(STAGES))()
+        calls = ctypes.c_int64(0)
+        self._check(self.lib.atomo_get_stage_totals(self._h, ms, ln, ctypes.byref(calls)), "atomo_get_stage_totals")
+        return ({k: float(ms[i]) for i, k in enumerate(STAGES)}, {k: int(ln[i]) for i, k in enumerate(STAGES)},
+                int(calls.value))
 
     def set_persistent_eig(self, enabled):
         """Eigen-solver scheme.  0 / False: Jacobi, one launch per step; 1 / True: persistent cooperative launches;

@@ -18,9 +18,16 @@ struct atomo_ctx {
   uint32_t* h_flag = nullptr;        // pinned: convergence flag / state mirror
   EwState* h_state = nullptr;        // pinned
   cudaEvent_t ev_sync = nullptr;
-  cudaEvent_t ev[ATOMO_N_STAGES][2] = {};
-  bool ev_used[ATOMO_N_STAGES] = {};
+  // stage timers: one set of events per API call, a ring of kEvRing sets (a set is read out -- its call is long
+  // finished by then -- before it is used again), sums since profiling was switched on
+  static constexpr int kEvRing = 32;
+  cudaEvent_t ev[kEvRing][ATOMO_N_STAGES][2] = {};
+  bool ev_used[kEvRing][ATOMO_N_STAGES] = {};
+  int ev_cur = 0;
   int64_t launches[ATOMO_N_STAGES] = {};
+  double acc_ms[ATOMO_N_STAGES] = {};
+  int64_t acc_launches[ATOMO_N_STAGES] = {};
+  int64_t acc_calls = 0;
   bool profiling = false;
   bool configured = false;
   int max_sweeps = 40;
@@ -72,16 +79,34 @@ int ensure_ws(atomo_ctx* ctx, size_t bytes) {
 
 void stage_begin(atomo_ctx* ctx, int stage, cudaStream_t st) {
   if (!ctx->profiling) return;
-  cudaEventRecord(ctx->ev[stage][0], st);
-  ctx->ev_used[stage] = true;
+  cudaEventRecord(ctx->ev[ctx->ev_cur][stage][0], st);
+  ctx->ev_used[ctx->ev_cur][stage] = true;
 }
 void stage_end(atomo_ctx* ctx, int stage, cudaStream_t st, int64_t n_launch) {
   ctx->launches[stage] += n_launch;
+  ctx->acc_launches[stage] += n_launch;
   if (!ctx->profiling) return;
-  cudaEventRecord(ctx->ev[stage][1], st);
+  cudaEventRecord(ctx->ev[ctx->ev_cur][stage][1], st);
 }
+// adds the times of one event set to the sums and frees the set (waits for its events: only the newest sets can
+// still be running)
+void stage_harvest(atomo_ctx* ctx, int slot) {
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) {
+    if (!ctx->ev_used[slot][i]) continue;
+    float ms = 0.0f;
+    if (cudaEventSynchronize(ctx->ev[slot][i][1]) == cudaSuccess &&
+        cudaEventElapsedTime(&ms, ctx->ev[slot][i][0], ctx->ev[slot][i][1]) == cudaSuccess)
+      ctx->acc_ms[i] += (double)ms;
+    ctx->ev_used[slot][i] = false;
+  }
+}
+// a new API call: the next event set of the ring
 void stage_reset(atomo_ctx* ctx) {
-  for (int i = 0; i < ATOMO_N_STAGES; ++i) { ctx->ev_used[i] = false; ctx->launches[i] = 0; }
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) ctx->launches[i] = 0;
+  ++ctx->acc_calls;
+  if (!ctx->profiling) return;
+  ctx->ev_cur = (ctx->ev_cur + 1) % atomo_ctx::kEvRing;
+  stage_harvest(ctx, ctx->ev_cur);
 }
 
 int next_pow2_at_least(int x, int lo) { int p = lo; while (p < x) p <<= 1; return p; }
@@ -143,7 +168,8 @@ int atomo_create(atomo_ctx** out, int device) {
   CK(cudaMallocHost(&ctx->h_flag, 256));
   CK(cudaMallocHost(&ctx->h_state, sizeof(EwState)));
   CK(cudaEventCreateWithFlags(&ctx->ev_sync, cudaEventDisableTiming));
-  for (int i = 0; i < ATOMO_N_STAGES; ++i) { CK(cudaEventCreate(&ctx->ev[i][0])); CK(cudaEventCreate(&ctx->ev[i][1])); }
+  for (int r = 0; r < atomo_ctx::kEvRing; ++r)
+    for (int i = 0; i < ATOMO_N_STAGES; ++i) { CK(cudaEventCreate(&ctx->ev[r][i][0])); CK(cudaEventCreate(&ctx->ev[r][i][1])); }
   const int e = sp_configure();
   if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaFuncSetAttribute(max dynamic shared memory)");
   ctx->tc_ok = sp_tc_configure() == 0;
@@ -159,7 +185,8 @@ int atomo_destroy(atomo_ctx* ctx) {
   if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
   if (ctx->h_state) cudaFreeHost(ctx->h_state);
   if (ctx->ev_sync) cudaEventDestroy(ctx->ev_sync);
-  for (int i = 0; i < ATOMO_N_STAGES; ++i) for (int j = 0; j < 2; ++j) if (ctx->ev[i][j]) cudaEventDestroy(ctx->ev[i][j]);
+  for (int r = 0; r < atomo_ctx::kEvRing; ++r)
+    for (int i = 0; i < ATOMO_N_STAGES; ++i) for (int j = 0; j < 2; ++j) if (ctx->ev[r][i][j]) cudaEventDestroy(ctx->ev[r][i][j]);
   delete ctx;
   return ATOMO_OK;
 }
@@ -194,7 +221,35 @@ int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap) 
 
 int atomo_set_profiling(atomo_ctx* ctx, int enabled) {
   if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  // switching on starts the sums afresh; event sets still in flight are read out first
+  for (int r = 0; r < atomo_ctx::kEvRing; ++r) stage_harvest(ctx, r);
+  if (enabled) {
+    for (int i = 0; i < ATOMO_N_STAGES; ++i) { ctx->acc_ms[i] = 0.0; ctx->acc_launches[i] = 0; }
+    ctx->acc_calls = 0;
+  }
   ctx->profiling = enabled != 0;
+  return ATOMO_OK;
+}
+
+int atomo_get_stage_totals(atomo_ctx* ctx, double* ms, int64_t* launches, int64_t* calls) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  // everything recorded so far is added up (this waits for the newest calls' events); the current set stays in use
+  // for get_stage_times, so its times are read without freeing it
+  for (int r = 0; r < atomo_ctx::kEvRing; ++r) if (r != ctx->ev_cur) stage_harvest(ctx, r);
+  for (int i = 0; i < ATOMO_N_STAGES; ++i) {
+    double cur = 0.0;
+    if (ctx->profiling && ctx->ev_used[ctx->ev_cur][i]) {
+      float t = 0.0f;
+      CK(cudaEventSynchronize(ctx->ev[ctx->ev_cur][i][1]));
+      CK(cudaEventElapsedTime(&t, ctx->ev[ctx->ev_cur][i][0], ctx->ev[ctx->ev_cur][i][1]));
+      cur = (double)t;
+    }
+    if (ms) ms[i] = ctx->acc_ms[i] + cur;
+    if (launches) launches[i] = ctx->acc_launches[i];
+  }
+  if (calls) *calls = ctx->acc_calls;
   return ATOMO_OK;
 }
 
@@ -205,9 +260,9 @@ int atomo_get_stage_times(atomo_ctx* ctx, float* ms, int64_t* launches) {
     if (launches) launches[i] = ctx->launches[i];
     if (!ms) continue;
     ms[i] = 0.0f;
-    if (ctx->profiling && ctx->ev_used[i]) {
-      CK(cudaEventSynchronize(ctx->ev[i][1]));
-      CK(cudaEventElapsedTime(&ms[i], ctx->ev[i][0], ctx->ev[i][1]));
+    if (ctx->profiling && ctx->ev_used[ctx->ev_cur][i]) {
+      CK(cudaEventSynchronize(ctx->ev[ctx->ev_cur][i][1]));
+      CK(cudaEventElapsedTime(&ms[i], ctx->ev[ctx->ev_cur][i][0], ctx->ev[ctx->ev_cur][i][1]));
     }
   }
   return ATOMO_OK;
@@ -513,9 +568,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
     n_eig_launch = 1;                                      // the eigenvalues (bisection) are timed with the sampling stage
-    CK(cudaMemsetAsync(d_flag + 2, 0, 2 * sizeof(uint32_t), st));
-    CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
-    flags_pending = true;                                  // the Gram kernel's bounded waits report at the end of the call
+    // no host wait on this route: a bounded wait of the Gram kernel that ran out is reported by the sampling kernel
+    // in every layer's status word (ATOMO_ERR_TIMEOUT, nothing kept)
   }
   if (cluster_form) {
     const int per = sp_jacobi_cluster_ctas();
@@ -588,7 +642,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   if (tri_form) launch_sp_bisect(d_layers, n_layers, r_max, st);   // all eigenvalues of the tridiagonal matrices
   launch_sp_refine(d_layers, n_layers, d_ref, (int)refine_tiles.size(), st);
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
-  launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps, st);
+  launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps,
+                            tri_form ? d_flag + 1 : nullptr, st);
   stage_end(ctx, ATOMO_STAGE_SAMPLE, st, tri_form ? 2 : 1);
 
   // ---- S4: long-side vectors of the kept atoms ----

@@ -145,8 +145,10 @@ int sp_configure_eig();
 void launch_sp_check(const SpLayer* d_layers, int n_layers, int t_done, int max_sweeps, uint32_t* d_all_done,
                      cudaStream_t st);
 void launch_sp_refine(const SpLayer* d_layers, int n_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
+// timeout_flag (device, may be null): non-zero means a bounded wait of an earlier kernel of the call ran out;
+// every layer then reports ATOMO_ERR_TIMEOUT and keeps nothing
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key,
-                               uint32_t kind_step, int max_sweeps, cudaStream_t st);
+                               uint32_t kind_step, int max_sweeps, const uint32_t* timeout_flag, cudaStream_t st);
 void launch_sp_backproject(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, int r_max, cudaStream_t st);
 void launch_sp_finish_atoms(const SpLayer* d_layers, int n_layers, int k_cap_max, cudaStream_t st);
 void launch_sp_decode(const uint8_t* payload, const SpDecodeLayer* d_layers, const TileRef* d_tiles, int n_tiles,

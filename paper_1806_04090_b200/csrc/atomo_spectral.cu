@@ -266,7 +266,8 @@ constexpr int kFinThreads = 512;
 
 __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const SpLayer* __restrict__ layers, double s,
                                                                          PhiloxKey key, uint32_t kind_step,
-                                                                         int max_sweeps) {
+                                                                         int max_sweeps,
+                                                                         const uint32_t* __restrict__ timeout_flag) {
   const SpLayer& L = layers[blockIdx.x];
   __shared__ float s_lam[kMaxShort];        // eigenvalues by row, later sigma by rank
   __shared__ float s_sig[kMaxShort];
@@ -385,7 +386,8 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
   }
   if (tid == 0) {
     uint32_t status = ATOMO_OK;
-    if (bad) status = ATOMO_ERR_NONFINITE;
+    if (timeout_flag != nullptr && *timeout_flag != 0) status = ATOMO_ERR_TIMEOUT;
+    else if (bad) status = ATOMO_ERR_NONFINITE;
     else if (carry > L.k_cap) status = ATOMO_ERR_CAPACITY;
     else if (h->sweeps >= (uint32_t)max_sweeps && L.rot_count[max_sweeps - 1] != 0) status = ATOMO_ERR_NOT_CONVERGED;
     h->status = status;
@@ -422,8 +424,8 @@ __global__ void __launch_bounds__(kFinThreads) sp_finalize_sample_kernel(const S
 }
 
 void launch_sp_finalize_sample(const SpLayer* d_layers, int n_layers, double s, PhiloxKey key, uint32_t kind_step,
-                               int max_sweeps, cudaStream_t st) {
-  sp_finalize_sample_kernel<<<n_layers, kFinThreads, 0, st>>>(d_layers, s, key, kind_step, max_sweeps);
+                               int max_sweeps, const uint32_t* timeout_flag, cudaStream_t st) {
+  sp_finalize_sample_kernel<<<n_layers, kFinThreads, 0, st>>>(d_layers, s, key, kind_step, max_sweeps, timeout_flag);
 }
 
 // =================================================================================================

@@ -188,3 +188,26 @@ def test_deterministic_and_fallback(atomo):
     pay, _ = atomo.atomo_encode_spectral([torch.from_numpy(bad).cuda()], 2.0, seed=9)
     assert atomo.last_eig_scheme() == TRIDIAG
     assert atomo.payload_status(pay) == (4, 0) and pay.headers()[1][0].k == 0
+
+
+def test_stage_totals_over_asynchronous_calls(atomo):
+    """The encode on this route enqueues and returns; the stage timers of several calls are read afterwards."""
+    import torch
+    G = [torch.from_numpy(m).cuda() for m in synth.c2_resnet18(0, [synth.RESNET18_LAYERS[1], synth.RESNET18_LAYERS[9]])]
+    atomo.set_profiling(True)
+    try:
+        outs = None
+        for it in range(40):                              # more calls than the library keeps event sets
+            pay, _ = atomo.atomo_encode_spectral(G, 2.0, seed=it)
+            outs = atomo.atomo_decode(pay, out=outs)
+        ms, ln, calls = atomo.stage_totals()
+        assert calls == 80
+        assert ln["eig"] == 40 and ln["sample"] == 80 and ln["backproject"] == 120 and ln["decode"] == 40
+        assert ms["eig"] > 0 and ms["gram"] > 0 and ms["decode"] > 0 and ms["ew_pack"] == 0
+        last, _ = atomo.stage_times()
+        assert last["decode"] > 0 and last["eig"] == 0    # the last call was a decode
+        again, _, _ = atomo.stage_totals()
+        assert again == ms                                # reading twice adds nothing
+        assert atomo.payload_status(pay)[0] == 0
+    finally:
+        atomo.set_profiling(False)
