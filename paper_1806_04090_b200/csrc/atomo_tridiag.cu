@@ -42,11 +42,11 @@ __device__ __forceinline__ bool finite64(double x) { return fabs(x) <= 1.7e308; 
 // Step k (k = 0 .. r-3) with x = A[k+1.., k]:  alpha = -sign(x_0) ||x||,  v = x - alpha e_1,  beta = 2 / v^T v,
 // H = I - beta v v^T;  p = beta A22 v,  K = beta/2 p^T v,  w = p - K v,  A22 -= v w^T + w v^T;  d_k = A[k][k],
 // e_k = alpha.
-// Layout: a layer's rows are dealt cyclically to its nc = rp / 32 CTAs (row i: group rank i mod nc, local row i / nc);
-// a warp keeps its two rows in registers for the whole reduction.  Every vector of length rp (and every row of A) is
-// stored in the order q(j) = (j mod nc) * 32 + j / nc, so that the 32 entries a CTA owns are contiguous: one warp
-// sends them to a peer as one 256-byte store into the peer's shared memory.  A lane holds the entries q = lane + 32 m,
-// that is j = lane * nc + m.
+// Layout: CTA g of a layer's nc = rp / 32 CTAs holds the rows 32 g .. 32 g + 31, two per warp, in registers for the
+// whole reduction; a lane holds the columns j = lane + 32 m.  The 32 entries of a vector that a CTA produces are
+// contiguous: one warp sends them to a peer as one 256-byte store into the peer's shared memory.  The trailing
+// block shrinks from the top left: column slots m < (k+1)/32 are dead and skipped, so a step costs in proportion
+// to the columns that are left (the CTAs of the dead rows only keep the barriers).
 // One cluster barrier per step: with p_i the owners also send c_i = A[i][k+1] as it is after update k-1, from which
 // every CTA forms the next pivot column x_i = c_i - v_i w_{k+1} - w_i v_{k+1} itself, hence v_{k+1}; the update of
 // step k and the product A v_{k+1} then share one pass over the rows.
@@ -117,17 +117,17 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   const float* const gA = L.A; const int64_t lda = L.lda; const int ldv = L.td_ldv;
   const int my_steps = max(r - 2, 0);
   const int li0 = w, li1 = w + kTriWarps;                     // this warp's two rows
-  const int i0 = li0 * nc + g, i1 = li1 * nc + g;
+  const int i0 = 32 * g + li0, i1 = 32 * g + li1;
   double row0[kTriCols], row1[kTriCols];
 #pragma unroll
   for (int m = 0; m < kTriCols; ++m) {
-    const int j = lane * nc + m;
+    const int j = lane + 32 * m;
     const bool in = m < nc && j < r;
     row0[m] = (in && i0 < r) ? (double)gA[(int64_t)i0 * lda + j] : 0.0;
     row1[m] = (in && i1 < r) ? (double)gA[(int64_t)i1 * lda + j] : 0.0;
   }
   const int sq = w * 32 + lane;                               // this thread's entry of the vectors (warps < nc)
-  const int sj = lane * nc + w;                               // its index
+  const int sj = sq;                                          // its index
   const bool slice = w < nc;
   // ---- the first reflector and A v_0 ----
   double beta = 0.0, v0 = 0.0;
@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     const double xq = (slice && sj > 0 && sj < r) ? (double)gA[sj] : 0.0;   // column 0 = row 0 (symmetric)
     if (slice) s_v[0][sq] = xq;
     const double nx2 = tri_block_sum(xq * xq, s_red2, lane, w);
-    const int q1 = (1 % nc) * 32 + 1 / nc;
+    const int q1 = 1;
     if (tid == 0) {
       double alpha;
       tri_reflector(nx2, (double)gA[1], alpha, beta, v0);
@@ -148,7 +148,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     {
       // reflectors are filed as unit vectors (H = I - 2 u u^T, u = v sqrt(beta / 2)): no range trouble in fp32
       const double un = sqrt(0.5 * beta);
-      if (g == 0) for (int j = tid; j < r; j += kTriThreads) td_V[j] = (float)(s_v[0][(j % nc) * 32 + j / nc] * un);   // row 0
+      if (g == 0) for (int j = tid; j < r; j += kTriThreads) td_V[j] = (float)(s_v[0][j] * un);   // row 0
     }
     double a0 = 0.0, a1 = 0.0;
 #pragma unroll
@@ -182,8 +182,8 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     const bool active = k < my_steps;
     const bool last = k + 1 == my_steps;                      // no reflector follows
     const int par = k & 1, nxt = par ^ 1;
-    const int q1 = ((k + 1) % nc) * 32 + (k + 1) / nc;       // where entry k+1 sits
-    const int q2 = ((k + 2) % nc) * 32 + (k + 2) / nc;
+    const int q1 = k + 1, q2 = k + 2;
+    const int m_lo = (k + 1) >> 5;                            // first column slot that is still alive
     double beta_n = 0.0, v0_n = 0.0;
     if (active) {
       // K = beta/2 p^T v: the CTAs' parts arrived with p; every thread adds them in the same order
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       double a0 = 0.0, a1 = 0.0;
 #pragma unroll
       for (int m = 0; m < kTriCols; ++m) {
-        if (m < nc) {
+        if (m >= m_lo && m < nc) {
           const double vq2 = pv[32 * m], wq2 = pw[32 * m], vn = pn[32 * m];
           row0[m] = fma(-vi0, wq2, fma(-wi0, vq2, row0[m]));
           row1[m] = fma(-vi1, wq2, fma(-wi1, vq2, row1[m]));
@@ -260,10 +260,10 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       if (lane == 0) cluster.map_shared_rank(&s_pk[0][0], base + w)[nxt * kTriCtas + g] = part;
     }
     cluster.barrier_arrive();                                 // (release) the entries above are on their way
-    if (active && !last && (k + 1) % nc == g) {               // meanwhile one CTA of the layer files the reflector
+    if (active && !last && g == 0) {                          // meanwhile the CTA of the first rows (dead after 31 steps) files the reflector
       if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
       const double un = sqrt(0.5 * beta_n);                   // filed as a unit vector: H = I - 2 u u^T
-      for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * ldv + j] = (float)(s_v[nxt][(j % nc) * 32 + j / nc] * un);
+      for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * ldv + j] = (float)(s_v[nxt][j] * un);
     }
     beta = beta_n; v0 = v0_n;
     cluster.barrier_wait();
