@@ -60,14 +60,17 @@ __device__ __forceinline__ double tri_block_sum(double x, double* s_red, int lan
   return t;                                                   // the same bits in every thread of the CTA
 }
 
-// alpha, beta and the first entry of v from ||x||^2 and x_0
+// alpha, beta and the first entry of v from ||x||^2 and x_0.  The square root comes from the reciprocal square root
+// and beta from a reciprocal: two short dependent sequences instead of a square root and a division (the chain sits
+// on the critical path of every step); v^T v / 2 = alpha (alpha - x_0) = ||x||^2 + |x_0| ||x||.
 __device__ __forceinline__ void tri_reflector(double nx2, double x0, double& alpha, double& beta, double& v0) {
   alpha = 0.0; beta = 0.0; v0 = 0.0;
-  if (nx2 > 0.0) {
-    alpha = -copysign(sqrt(nx2), x0);
+  if (nx2 > 1.0e-290) {                                       // below: treated as a zero column (H = I)
+    const double nx = nx2 * rsqrt(nx2);
+    alpha = -copysign(nx, x0);
     v0 = x0 - alpha;
-    const double den = alpha * (alpha - x0);                  // = v^T v / 2 > 0
-    beta = den > 0.0 ? 1.0 / den : 0.0;
+    const double den = fma(fabs(x0), nx, nx2);
+    beta = __drcp_rn(den);
   }
 }
 
