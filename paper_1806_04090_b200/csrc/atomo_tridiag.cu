@@ -3,10 +3,11 @@
 // Eq. 2 need their vectors).  For layers with a short side of at most 512:
 //
 //   sp_tridiag_cluster_kernel : Householder reduction of the scaled Gram matrix A (r x r) to a symmetric
-//                               tridiagonal T = Q^T A Q, in fp64.  A layer's rows are dealt cyclically to rp/32 CTAs
-//                               of a 16-CTA cluster and stay in shared memory; per step the pivot column and the
-//                               product A v travel through distributed shared memory (two cluster barriers per
-//                               step).  The reflectors go to global memory for the back-transformation.
+//                               tridiagonal T = Q^T A Q, in fp64.  A layer's rows sit in blocks of 32 on rp/32 CTAs
+//                               of a 16-CTA cluster and stay in registers; per step the product A v, the next
+//                               pivot column's ingredients and the parts of p^T v travel through distributed
+//                               shared memory (one cluster barrier per step).  The reflectors go to global memory
+//                               as fp32 unit vectors for the back-transformation.
 //   sp_bisect_kernel          : all eigenvalues of T, eight lanes per eigenvalue: 13 rounds of 9-section on Sturm
 //                               counts (division-free three-term recurrence with power-of-two rescaling).
 //   (sp_finalize_sample_kernel sorts, solves Algorithm 1 and draws, as for the other routes)
