@@ -289,16 +289,12 @@ __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const d
   int neg = __double2hiint(p);                                // sign bit of the previous term
   int cnt = (uint32_t)neg >> 31;
   // eight steps at a time: their operands are fetched together, so that only the multiply-add chain is serial.
-  // Past the end the step is p <- 1 * p - 0 * p_prev: no sign change.
+  // The caller pads d with kSturmPad (far above every eigenvalue) and e2 with 0 up to a multiple of 8 past the end:
+  // there the step is p <- (pad - x) p, which keeps the sign.
   for (int i0 = 1; i0 < r; i0 += 8) {
     double dd[8], ee[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int i = i0 + u;
-      const bool in = i < r;
-      dd[u] = in ? d[i] - x : 1.0;
-      ee[u] = in ? e2[i - 1] : 0.0;
-    }
+    for (int u = 0; u < 8; ++u) { dd[u] = d[i0 + u] - x; ee[u] = e2[i0 + u - 1]; }   // padded arrays: no bounds test
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const double pn = fma(dd[u], p, -ee[u] * pm);
@@ -314,6 +310,7 @@ __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const d
   return cnt;
 }
 
+constexpr double kSturmPad = 1.0e6;    // diagonal entries past the end (the matrices are scaled to trace <= 1)
 constexpr int kBisThreads = 64;           // small CTAs: the warps of a large layer spread over all SMs (the recurrences are latency-bound)
 constexpr int kBisLanes = 8;          // points per round and eigenvalue: the interval shrinks 9 times per round
 constexpr int kBisRounds = 13;        // 9^13 = 2.5e12: interval width below 1e-12 of the spectrum's extent
@@ -324,9 +321,9 @@ __global__ void __launch_bounds__(kBisThreads) sp_bisect_kernel(const SpLayer* _
   const int r = L.r;
   const int tid = threadIdx.x, lane = tid % 32;
   if ((int)blockIdx.x * kBisPerCta >= r) return;
-  __shared__ double s_d[kTriMaxRp], s_e2[kTriMaxRp];
-  for (int i = tid; i < r; i += kBisThreads) {
-    s_d[i] = L.td_d[i];
+  __shared__ double s_d[kTriMaxRp + 8], s_e2[kTriMaxRp + 8];
+  for (int i = tid; i < r + 8; i += kBisThreads) {
+    s_d[i] = i < r ? L.td_d[i] : kSturmPad;
     const double e = i + 1 < r ? L.td_e[i] : 0.0;
     s_e2[i] = e * e;
   }
