@@ -182,6 +182,11 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     if (lane == 0) cluster.map_shared_rank(&s_pk[0][0], base + w)[g] = part;
   }
   cluster.sync();
+  // warp w < nc talks to peer w: that CTA's copies of the three arrays, mapped once
+  const int peer = base + min(w, nc - 1);
+  double* const peer_p = cluster.map_shared_rank(&s_p[0][0], peer);
+  double* const peer_c = cluster.map_shared_rank(&s_c[0][0], peer);
+  double* const peer_pk = cluster.map_shared_rank(&s_pk[0][0], peer);
   for (int k = 0; k < steps; ++k) {
     const bool active = k < my_steps;
     const bool last = k + 1 == my_steps;                      // no reflector follows
@@ -258,10 +263,10 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     __syncthreads();
     if (active && !last && w < nc) {
       const double pl = s_stage[0][lane];
-      cluster.map_shared_rank(&s_p[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = pl;
-      cluster.map_shared_rank(&s_c[0][0], base + w)[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
+      peer_p[nxt * kTriMaxRp + g * 32 + lane] = pl;
+      peer_c[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
       const double part = warp_sum(pl * s_v[nxt][g * 32 + lane]);
-      if (lane == 0) cluster.map_shared_rank(&s_pk[0][0], base + w)[nxt * kTriCtas + g] = part;
+      if (lane == 0) peer_pk[nxt * kTriCtas + g] = part;
     }
     cluster.barrier_arrive();                                 // (release) the entries above are on their way
     if (active && !last && g == 0) {                          // meanwhile the CTA of the first rows (dead after 31 steps) files the reflector
