@@ -18,6 +18,8 @@
 //
 // Work per layer: about 2 r^3 fp64 flops for the reduction (full symmetric storage: matrix-vector product and
 // rank-two update of the trailing block), r^2 * 13 * 8 recurrence steps for the eigenvalues, O(r^2) per kept atom.
+#include <type_traits>
+
 #include <cooperative_groups.h>
 
 #include "atomo_kernels.cuh"
@@ -187,7 +189,13 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   double* const peer_p = cluster.map_shared_rank(&s_p[0][0], peer);
   double* const peer_c = cluster.map_shared_rank(&s_c[0][0], peer);
   double* const peer_pk = cluster.map_shared_rank(&s_pk[0][0], peer);
-  for (int k = 0; k < steps; ++k) {
+  // A layer that fills its cluster finishes alone: once every live row sits in the CTA of the last rows, that CTA runs
+  // the remaining steps (at most 31) by itself, with stores into its own shared memory and __syncthreads in place of
+  // the cluster barrier, and the other CTAs leave the loop.
+  const int g_last = (max(r, 1) - 1) >> 5;
+  const int k_tail = nc == kTriCtas ? 32 * g_last - 1 : 0x7fffffff;
+  auto step = [&](auto solo_tag, const int k) {               // two instances: with the cluster, and alone
+    constexpr bool solo = decltype(solo_tag)::value;
     const bool active = k < my_steps;
     const bool last = k + 1 == my_steps;                      // no reflector follows
     const int par = k & 1, nxt = par ^ 1;
@@ -198,7 +206,8 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       // K = beta/2 p^T v: the CTAs' parts arrived with p; every thread adds them in the same order
       const double vq = slice ? s_v[par][sq] : 0.0;
       const double pq = slice ? s_p[par][sq] : 0.0;
-      double ksum = (lane & (kTriCtas - 1)) < nc ? s_pk[par][lane & (kTriCtas - 1)] : 0.0;
+      const int kc = lane & (kTriCtas - 1);                   // (alone, only this CTA's part is there)
+      double ksum = (solo ? kc == g : kc < nc) ? s_pk[par][kc] : 0.0;
 #pragma unroll
       for (int o = kTriCtas / 2; o > 0; o >>= 1) ksum += __shfl_xor_sync(0xffffffffu, ksum, o);
       const double K = 0.5 * beta * ksum;
@@ -261,22 +270,28 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       }
     }
     __syncthreads();
-    if (active && !last && w < nc) {
+    if (active && !last && (solo ? w == 0 : w < nc)) {        // alone: the same entries into this CTA's own arrays
+      double* const to_p = solo ? &s_p[0][0] : peer_p;
+      double* const to_c = solo ? &s_c[0][0] : peer_c;
+      double* const to_pk = solo ? &s_pk[0][0] : peer_pk;
       const double pl = s_stage[0][lane];
-      peer_p[nxt * kTriMaxRp + g * 32 + lane] = pl;
-      peer_c[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
+      to_p[nxt * kTriMaxRp + g * 32 + lane] = pl;
+      to_c[nxt * kTriMaxRp + g * 32 + lane] = s_stage[1][lane];
       const double part = warp_sum(pl * s_v[nxt][g * 32 + lane]);
-      if (lane == 0) peer_pk[nxt * kTriCtas + g] = part;
+      if (lane == 0) to_pk[nxt * kTriCtas + g] = part;
     }
-    cluster.barrier_arrive();                                 // (release) the entries above are on their way
-    if (active && !last && g == 0) {                          // meanwhile the CTA of the first rows (dead after 31 steps) files the reflector
+    if (!solo) cluster.barrier_arrive();                      // (release) the entries above are on their way
+    if (active && !last && (solo || g == 0)) {                // meanwhile the CTA of the first rows (dead after 31 steps) files the reflector
       if (tid == 0) { td_e[k + 1] = s_scal[0]; td_tau[k + 1] = beta_n; }
       const double un = sqrt(0.5 * beta_n);                   // filed as a unit vector: H = I - 2 u u^T
       for (int j = tid; j < r; j += kTriThreads) td_V[(int64_t)(k + 1) * ldv + j] = (float)(s_v[nxt][j] * un);
     }
     beta = beta_n; v0 = v0_n;
-    cluster.barrier_wait();
-  }
+    if (solo) __syncthreads(); else cluster.barrier_wait();
+  };
+  const int k_mid = min(steps, k_tail);
+  for (int k = 0; k < k_mid; ++k) step(std::false_type{}, k);
+  if (g == g_last) for (int k = k_mid; k < steps; ++k) step(std::true_type{}, k);
   // matrices of order 1 and 2 are tridiagonal as they are
   if (my_steps == 0 && g == 0 && tid == 0) {
     td_d[0] = (double)gA[0];
