@@ -194,8 +194,10 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   // the cluster barrier, and the other CTAs leave the loop.
   const int g_last = (max(r, 1) - 1) >> 5;
   const int k_tail = nc == kTriCtas ? 32 * g_last - 1 : 0x7fffffff;
-  auto step = [&](auto solo_tag, const int k) {               // two instances: with the cluster, and alone
+  auto step = [&](auto solo_tag, auto full_tag, const int k) {   // instances: with the cluster (a layer that fills it, or a smaller one), and alone
     constexpr bool solo = decltype(solo_tag)::value;
+    constexpr bool full = decltype(full_tag)::value;          // the layer has all kTriCtas CTAs: loop bounds known at compile time
+    const int ncc = full ? kTriCtas : nc;
     const bool active = k < my_steps;
     const bool last = k + 1 == my_steps;                      // no reflector follows
     const int par = k & 1, nxt = par ^ 1;
@@ -207,7 +209,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       const double vq = slice ? s_v[par][sq] : 0.0;
       const double pq = slice ? s_p[par][sq] : 0.0;
       const int kc = lane & (kTriCtas - 1);                   // (alone, only this CTA's part is there)
-      double ksum = (solo ? kc == g : kc < nc) ? s_pk[par][kc] : 0.0;
+      double ksum = (solo ? kc == g : kc < ncc) ? s_pk[par][kc] : 0.0;
 #pragma unroll
       for (int o = kTriCtas / 2; o > 0; o >>= 1) ksum += __shfl_xor_sync(0xffffffffu, ksum, o);
       const double K = 0.5 * beta * ksum;
@@ -239,7 +241,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       double a0 = 0.0, a1 = 0.0;
 #pragma unroll
       for (int m = 0; m < kTriCols; ++m) {
-        if (m >= m_lo && m < nc) {
+        if (m >= m_lo && m < ncc) {
           const double vq2 = pv[32 * m], wq2 = pw[32 * m], vn = pn[32 * m];
           row0[m] = fma(-vi0, wq2, fma(-wi0, vq2, row0[m]));
           row1[m] = fma(-vi1, wq2, fma(-wi1, vq2, row1[m]));
@@ -270,7 +272,7 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
       }
     }
     __syncthreads();
-    if (active && !last && (solo ? w == 0 : w < nc)) {        // alone: the same entries into this CTA's own arrays
+    if (active && !last && (solo ? w == 0 : w < ncc)) {        // alone: the same entries into this CTA's own arrays
       double* const to_p = solo ? &s_p[0][0] : peer_p;
       double* const to_c = solo ? &s_c[0][0] : peer_c;
       double* const to_pk = solo ? &s_pk[0][0] : peer_pk;
@@ -290,8 +292,12 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     if (solo) __syncthreads(); else cluster.barrier_wait();
   };
   const int k_mid = min(steps, k_tail);
-  for (int k = 0; k < k_mid; ++k) step(std::false_type{}, k);
-  if (g == g_last) for (int k = k_mid; k < steps; ++k) step(std::true_type{}, k);
+  if (nc == kTriCtas) {
+    for (int k = 0; k < k_mid; ++k) step(std::false_type{}, std::true_type{}, k);
+    if (g == g_last) for (int k = k_mid; k < steps; ++k) step(std::true_type{}, std::true_type{}, k);
+  } else {
+    for (int k = 0; k < steps; ++k) step(std::false_type{}, std::false_type{}, k);
+  }
   // matrices of order 1 and 2 are tridiagonal as they are
   if (my_steps == 0 && g == 0 && tid == 0) {
     td_d[0] = (double)gA[0];
