@@ -194,15 +194,18 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
   // the cluster barrier, and the other CTAs leave the loop.
   const int g_last = (max(r, 1) - 1) >> 5;
   const int k_tail = nc == kTriCtas ? 32 * g_last - 1 : 0x7fffffff;
-  auto step = [&](auto solo_tag, auto full_tag, const int k) {   // instances: with the cluster (a layer that fills it, or a smaller one), and alone
+  // instances: with the cluster (a layer that fills it, or a smaller one) and alone; for the layers that fill the
+  // cluster also one per first live column slot, so that the pass over the rows is straight-line code
+  auto step = [&](auto solo_tag, auto full_tag, auto mlo_tag, const int k) {
     constexpr bool solo = decltype(solo_tag)::value;
+    constexpr int kMlo = decltype(mlo_tag)::value;            // first live column slot, or -1: taken from k at run time
     constexpr bool full = decltype(full_tag)::value;          // the layer has all kTriCtas CTAs: loop bounds known at compile time
     const int ncc = full ? kTriCtas : nc;
     const bool active = k < my_steps;
     const bool last = k + 1 == my_steps;                      // no reflector follows
     const int par = k & 1, nxt = par ^ 1;
     const int q1 = k + 1, q2 = k + 2;
-    const int m_lo = (k + 1) >> 5;                            // first column slot that is still alive
+    const int m_lo = kMlo >= 0 ? kMlo : (k + 1) >> 5;         // first column slot that is still alive
     double beta_n = 0.0, v0_n = 0.0;
     if (active) {
       // K = beta/2 p^T v: the CTAs' parts arrived with p; every thread adds them in the same order
@@ -292,11 +295,20 @@ __global__ void __launch_bounds__(kTriThreads, 1) sp_tridiag_cluster_kernel(cons
     if (solo) __syncthreads(); else cluster.barrier_wait();
   };
   const int k_mid = min(steps, k_tail);
+  using Dyn = std::integral_constant<int, -1>;
   if (nc == kTriCtas) {
-    for (int k = 0; k < k_mid; ++k) step(std::false_type{}, std::true_type{}, k);
-    if (g == g_last) for (int k = k_mid; k < steps; ++k) step(std::true_type{}, std::true_type{}, k);
+#define TRI_SLOT(M) case M: step(std::false_type{}, std::true_type{}, std::integral_constant<int, M>{}, k); break;
+    for (int k = 0; k < k_mid; ++k) {
+      switch ((k + 1) >> 5) {
+        TRI_SLOT(0) TRI_SLOT(1) TRI_SLOT(2) TRI_SLOT(3) TRI_SLOT(4) TRI_SLOT(5) TRI_SLOT(6) TRI_SLOT(7)
+        TRI_SLOT(8) TRI_SLOT(9) TRI_SLOT(10) TRI_SLOT(11) TRI_SLOT(12) TRI_SLOT(13) TRI_SLOT(14)
+        default: step(std::false_type{}, std::true_type{}, std::integral_constant<int, 15>{}, k); break;
+      }
+    }
+#undef TRI_SLOT
+    if (g == g_last) for (int k = k_mid; k < steps; ++k) step(std::true_type{}, std::true_type{}, Dyn{}, k);
   } else {
-    for (int k = 0; k < steps; ++k) step(std::false_type{}, std::false_type{}, k);
+    for (int k = 0; k < steps; ++k) step(std::false_type{}, std::false_type{}, Dyn{}, k);
   }
   // matrices of order 1 and 2 are tridiagonal as they are
   if (my_steps == 0 && g == 0 && tid == 0) {
