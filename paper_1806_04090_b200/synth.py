@@ -26,6 +26,7 @@ import numpy as np
 __all__ = [
     "haar_columns", "lowrank_plus_noise", "LayerSpec", "RESNET18_LAYERS", "VGG11_LAYERS",
     "c1_spectral", "c1_entrywise", "c2_resnet18", "c3_vgg11", "c4_entrywise", "c5_stress",
+    "c3_vgg11_layer", "c5_stress_layer",
     "layer_elements",
 ]
 
@@ -138,6 +139,17 @@ def c2_resnet18(seed: int = 0, layers: Sequence[LayerSpec] = RESNET18_LAYERS) ->
 def c3_vgg11(seed: int = 0, layers: Sequence[LayerSpec] = VGG11_LAYERS) -> List[np.ndarray]:
     """Config 3: VGG-11 layer set, sigma_i = 1/i, 1% (Frobenius) Gaussian noise."""
     return _layer_set("c3", layers, seed, 1.0, 0.01)
+
+
+def c3_vgg11_layer(seed: int, index: int) -> np.ndarray:
+    """One layer of config 3 (the same matrix ``c3_vgg11(seed)[index]`` holds), without generating the others."""
+    l = VGG11_LAYERS[index]
+    return lowrank_plus_noise(_rng("c3", seed, index), l.rows, l.cols, 1.0, noise_rel=0.01)
+
+
+def c5_stress_layer(seed: int, index: int, rows: int = 1024, cols: int = 4096) -> np.ndarray:
+    """One matrix of config 5 (the same matrix ``c5_stress(seed)[index]`` holds)."""
+    return lowrank_plus_noise(_rng("c5", seed, index), rows, cols, 1.0, noise_rel=0.005)
 
 
 def c4_entrywise(seed: int = 0, n: int = 25_600_000) -> np.ndarray:

@@ -1,0 +1,88 @@
+"""GPU parity at short sides of 1024 and 4096 (configs 5 and 3) against the stored results of the fp64 oracle.
+
+The oracle's one-sided Jacobi SVD takes minutes to hours there, so its results for a few seeded layers are stored
+under ``tests/golden/`` (written by ``make_spectral_golden.py``, which calls only the oracle).  Here the CUDA path
+encodes and decodes the same layers, at the same position of the call, with the same Philox seed and step, and
+goes through the same protocol as the small layers: singular values and probabilities within 1e-4 (and the
+largest |p - p_oracle| reported), masks and kept ranks bit-exact outside the 1e-6 carve-out, kept atoms as
+singular triplets, the decode against the oracle's decode."""
+import numpy as np
+import pytest
+
+from paper_1806_04090_b200 import synth
+from tests import golden_io, parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def atomo():
+    import torch
+    from paper_1806_04090_b200 import api
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    a = api.Atomo(0)
+    yield a
+    a.close()
+
+
+def _check(atomo, oracle, ts, mats, which, metas, encs_by_layer, s, report):
+    """Encodes the batch `ts` and checks the layers listed in `which` against their stored oracle results."""
+    meta = metas[which[0]]
+    pay, dbg = atomo.atomo_encode_spectral(ts, s, meta["philox_seed"], step=meta["step"], k_cap=64, debug=True)
+    hdrs = pay.headers()
+    outs = atomo.atomo_decode(pay)
+    worst_p = 0.0
+    certified = 0
+    for l in which:
+        G = mats[l]
+        r = min(G.shape)
+        enc = dict(encs_by_layer[l][s])
+        enc["words"] = oracle.bernoulli_words(meta["philox_seed"], meta["step"], l, oracle.KIND_SPECTRAL, r)
+        arr = pay.layer_arrays(l, hdrs)
+        out = outs[l].cpu().numpy().astype(np.float64)
+        p = dbg.layer_prob(l, r)
+        dp = float(np.abs(p - enc["p"]).max())
+        worst_p = max(worst_p, dp)
+        same, e2e = parity.check_spectral_layer(oracle, G, enc, hdrs[1][l], arr, dbg, l, out, report,
+                                                f"s={s:g} L{l}{G.shape}")
+        report.append(f"s={s:g} L{l}: max |p - p_oracle| = {dp:.2e}, kept {arr['k']}, masks identical: {same}")
+        assert dp <= 1e-5, f"L{l}: probabilities {dp:.2e} away from the oracle's"
+        certified += 1 if same else 0
+    return worst_p, certified
+
+
+@pytest.mark.parametrize("scheme", [3, 1])
+def test_config5_layers_against_stored_oracle(atomo, oracle, scheme):
+    import torch
+    if not (golden_io.have("c5", 0) and golden_io.have("c5", 1)):
+        pytest.skip("stored case not generated")
+    loaded = [golden_io.load("c5", i) for i in (0, 1)]
+    mats = [g for g, _, _ in loaded]
+    metas = {i: loaded[i][1] for i in (0, 1)}
+    encs = {i: loaded[i][2] for i in (0, 1)}
+    ts = [torch.from_numpy(G).cuda() for G in mats]
+    report = []
+    try:
+        atomo.set_persistent_eig(scheme)
+        for s in metas[0]["budgets"]:
+            _check(atomo, oracle, ts, mats, [0, 1], metas, encs, s, report)
+        used = atomo.last_eig_scheme()
+    finally:
+        atomo.set_persistent_eig(3)
+    print("\n".join(report))
+    print(f"eigen scheme asked {scheme}, used {used}")
+
+
+def test_config3_large_layer_against_stored_oracle(atomo, oracle):
+    import torch
+    if not golden_io.have("c3", 8):
+        pytest.skip("stored case not generated")
+    G8, meta, encs8 = golden_io.load("c3", 8)
+    # the whole VGG-11-shaped batch, so that the stored layer sits at its position (8) among the small layers
+    mats = [synth.c3_vgg11_layer(0, i) if i != 8 else G8 for i in range(len(synth.VGG11_LAYERS))]
+    ts = [torch.from_numpy(G).cuda() for G in mats]
+    report = []
+    for s in meta["budgets"]:
+        _check(atomo, oracle, ts, mats, [8], {8: meta}, {8: encs8}, s, report)
+    print("\n".join(report))
+    print(f"eigen scheme used {atomo.last_eig_scheme()}")
