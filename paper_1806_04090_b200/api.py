@@ -32,6 +32,7 @@ EXPORTS = [
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
+    "atomo_set_tridiag_ctas",
 ]
 
 
@@ -114,6 +115,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_gram_path.argtypes = [vp, i32]
     lib.atomo_set_persistent_eig.argtypes = [vp, i32]
     lib.atomo_last_eig_scheme.argtypes = [vp]
+    lib.atomo_set_tridiag_ctas.argtypes = [vp, i32]
     lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                  ctypes.POINTER(vp), i32, vp]
     if path == LIB_PATH:
@@ -478,7 +480,7 @@ class Atomo:
 
     def set_persistent_eig(self, enabled):
         """Eigen-solver scheme.  0 / False: Jacobi, one launch per step; 1 / True: persistent cooperative launches;
-        2: Jacobi in thread-block clusters first; 3 (default): tridiagonal route first (short sides up to 512)."""
+        2: Jacobi in thread-block clusters first; 3 (default): the tridiagonal routes (any short side up to 4096)."""
         self._check(self.lib.atomo_set_persistent_eig(self._h, int(enabled)), "atomo_set_persistent_eig")
 
     def set_entrywise_format(self, fmt: int, sat_cap: int = 0):
@@ -486,6 +488,11 @@ class Atomo:
         explicit values only for the atoms with p = 1, of which at most sat_cap per vector)."""
         self._check(self.lib.atomo_set_entrywise_format(self._h, int(fmt), int(sat_cap)), "atomo_set_entrywise_format")
         self._ew_format, self._ew_sat_cap = int(fmt), (int(sat_cap) if int(fmt) == EW_COMPACT else 0)
+
+    def set_tridiag_ctas(self, ctas_per_layer: int):
+        """CTAs per layer of the blocked tridiagonal reduction (short sides above 512): 0 = chosen per batch, else 1,
+        2, 4, 8 or 16.  The payload does not depend on it."""
+        self._check(self.lib.atomo_set_tridiag_ctas(self._h, int(ctas_per_layer)), "atomo_set_tridiag_ctas")
 
     def last_eig_scheme(self) -> int:
         return int(self.lib.atomo_last_eig_scheme(self._h))

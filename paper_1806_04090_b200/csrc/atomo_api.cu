@@ -38,6 +38,8 @@ struct atomo_ctx {
   bool tc_ok = false;                // tensor-map entry point found
   int eig_scheme = 3;                // eigen-solve: 0 = Jacobi, one launch per step, 1 = persistent (cooperative), 2 = clusters first, 3 = tridiagonal route first
   int tri_clusters = -1;             // co-resident clusters of the tridiagonal reduction (-1 = not asked yet, 0 = unavailable)
+  int tri_big_ok = -1;               // blocked tridiagonal reduction for short sides above 512 (-1 = not asked yet)
+  int tri_big_ctas = 0;              // CTAs per layer of that reduction: 0 = chosen per batch, else 1, 2, 4, 8 or 16
   int eig_scheme_used = -1;          // what the last spectral encode actually ran
   int ew_format = ATOMO_EW_EXPLICIT; // payload format of entry-wise encodes
   int64_t ew_sat_cap = 0;            // compact format: capacity of the saturated list
@@ -283,6 +285,15 @@ int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
   return ATOMO_OK;
 }
 
+int atomo_set_tridiag_ctas(atomo_ctx* ctx, int32_t ctas_per_layer) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  if (ctas_per_layer != 0 && ctas_per_layer != 1 && ctas_per_layer != 2 && ctas_per_layer != 4 && ctas_per_layer != 8 &&
+      ctas_per_layer != 16)
+    return ATOMO_ERR_INVALID_ARG;
+  ctx->tri_big_ctas = ctas_per_layer;
+  return ATOMO_OK;
+}
+
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores) {
   if (!ctx) return ATOMO_ERR_INVALID_ARG;
   ctx->tc_gram = tensor_cores != 0;
@@ -382,17 +393,27 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (d.refine)
       for (int a = 0; a < gt; ++a) for (int b = 0; b < d.refine_tiles; ++b) refine_tiles.push_back({l, a, b, 0});
   }
-  // Cluster form first: every layer's block pairs inside one 16-CTA cluster, blocks exchanged through
-  // distributed shared memory (layers of up to 16 block pairs, route 1).
-  // Tridiagonal route first: eigenvalues of every atom from T = Q^T A Q, vectors for the kept atoms only (short side
-  // <= 512, no per-atom refinement, no request for the whole short-side basis).
+  // Tridiagonal routes first: eigenvalues of every atom from T = Q^T A Q, vectors for the kept atoms only -- in the
+  // registers of a cluster for short sides up to 512, blocked with A in global memory above (no per-atom refinement,
+  // no request for the whole short-side basis).  Otherwise the Jacobi routes, the cluster form first.
   bool tri_form = ctx->eig_scheme == 3 && ctx->eig_mode != 0 && !(dbg && dbg->short_vecs);
-  for (int l = 0; l < n_layers && tri_form; ++l) tri_form = L[l].rp <= sp_tridiag_max_rp() && !L[l].refine;
-  if (tri_form) {
+  bool any_small = false, any_big = false;
+  for (int l = 0; l < n_layers && tri_form; ++l) (L[l].rp <= sp_tridiag_max_rp() ? any_small : any_big) = true;
+  if (tri_form && any_small) {
     if (ctx->tri_clusters < 0) ctx->tri_clusters = sp_configure_tridiag();
     if (ctx->tri_clusters < 1) tri_form = false;
   }
-  for (int l = 0; l < n_layers; ++l) L[l].tri = tri_form ? 1 : 0;
+  if (tri_form && any_big) {
+    if (ctx->tri_big_ok < 0) ctx->tri_big_ok = sp_configure_tridiag_big() == 0 ? 1 : 0;
+    if (ctx->tri_big_ok < 1 || r_max > sp_tridiag_big_max_r()) tri_form = false;
+  }
+  std::vector<int> big_layers;
+  for (int l = 0; l < n_layers; ++l) {
+    L[l].tri = !tri_form ? 0 : (L[l].rp <= sp_tridiag_max_rp() ? 1 : 2);
+    if (L[l].tri) { L[l].refine = 0; }
+    if (L[l].tri == 2) big_layers.push_back(l);
+  }
+  if (tri_form) refine_tiles.clear();
   bool cluster_form = !tri_form && ctx->eig_scheme >= 2 && ctx->eig_mode != 0;
   for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
   if (cluster_form) {
@@ -432,6 +453,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
   ClusterCta* d_ctas = nullptr;
+  int* d_big = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
   for (int pass = 0; pass < 2; ++pass) {
@@ -446,6 +468,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_maps = A.take<uint8_t>(maps_blob.size());
     d_flag = A.take<uint32_t>(4);
     d_ctas = A.take<ClusterCta>((size_t)n_layers * sp_jacobi_cluster_ctas());   // at most one cluster per layer
+    d_big = A.take<int>(big_layers.size());
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
@@ -471,6 +494,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       d.td_tau = A.take<double>(d.tri ? d.rp : 0); d.lam64 = A.take<double>(d.tri ? d.rp : 0);
       d.td_ldv = (d.r + 3) / 4 * 4;
       d.td_V = A.take<float>(d.tri ? (size_t)d.r * d.td_ldv : 0);
+      d.tb_fp64 = 0;
+      d.tb_ldw = (d.r + 3) / 4 * 4;
+      d.tb_W = A.take<float>(d.tri == 2 ? (size_t)sp_tridiag_big_panel() * d.tb_ldw : 0);
+      d.tb_vecwork = A.take<double>(d.tri == 2 ? (size_t)sp_eigvec_big_slots() * 5 * d.rp : 0);
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
       d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);
@@ -493,6 +520,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
       if (d.acc) { d.A = d.X; d.lda = d.ldx; }
+      else if (d.tri == 2) { d.lda = (d.r + 3) / 4 * 4; d.A = A.take<float>((size_t)d.r * d.lda); d.tb_A = d.A; }   // 16-byte rows
       else { d.A = A.take<float>((size_t)d.r * d.r); d.lda = d.r; }
     }
     need = A.off + 256;
@@ -548,11 +576,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
+  int rp_max_small = 32;
   if (tri_form) {
-    // layers packed into 16-CTA clusters, largest first (a layer takes rp / 32 consecutive ranks of one cluster)
+    // small layers packed into 16-CTA clusters, largest first (a layer takes rp / 32 consecutive ranks of one cluster)
     const int per = sp_tridiag_cluster_ctas();
-    std::vector<int> order(n_layers);
-    for (int l = 0; l < n_layers; ++l) order[l] = l;
+    std::vector<int> order;
+    for (int l = 0; l < n_layers; ++l) if (L[l].tri == 1) { order.push_back(l); rp_max_small = std::max(rp_max_small, L[l].rp); }
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].rp > L[b].rp; });
     std::vector<int> used;
     std::vector<ClusterCta> ctas;
@@ -564,12 +593,30 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       for (int sl = 0; sl < nc; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], nc};
       used[c] += nc;
     }
-    CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
-    const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max, st);
-    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
-    n_eig_launch = 1;                                      // the eigenvalues (bisection) are timed with the sampling stage
-    // no host wait on this route: a bounded wait of the Gram kernel that ran out is reported by the sampling kernel
-    // in every layer's status word (ATOMO_ERR_TIMEOUT, nothing kept)
+    if (!order.empty()) {
+      CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
+      const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max_small, st);
+      if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
+      ++n_eig_launch;
+    }
+    if (!big_layers.empty()) {
+      // larger layers: a cluster of C CTAs each.  C is the smallest that holds the rows; it is doubled while the
+      // batch still leaves SMs idle (the result does not depend on C)
+      int sms = 148, dev = 0;
+      if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      int cmin = 1, rb = 0;
+      for (int l : big_layers) { cmin = std::max(cmin, sp_tridiag_big_min_ctas(L[l].r)); rb = std::max(rb, L[l].r); }
+      int cc = cmin;
+      if (ctx->tri_big_ctas > 0) cc = std::max(cmin, ctx->tri_big_ctas);
+      else while (cc < 16 && (int)big_layers.size() * cc * 2 <= sms) cc *= 2;
+      CK(cudaMemcpyAsync(d_big, big_layers.data(), big_layers.size() * sizeof(int), cudaMemcpyHostToDevice, st));
+      const int e = launch_sp_tridiag_big(d_layers, d_big, (int)big_layers.size(), rb, cc, 0, st);
+      if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(blocked tridiagonal reduction)");
+      ++n_eig_launch;
+    }
+    // the eigenvalues (bisection) are timed with the sampling stage.  No host wait on this route: a bounded wait of
+    // the Gram kernel that ran out is reported by the sampling kernel in every layer's status word
+    // (ATOMO_ERR_TIMEOUT, nothing kept)
   }
   if (cluster_form) {
     const int per = sp_jacobi_cluster_ctas();
@@ -648,10 +695,13 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S4: long-side vectors of the kept atoms ----
   stage_begin(ctx, ATOMO_STAGE_BACKPROJECT, st);
-  if (tri_form) launch_sp_eigvec(d_layers, n_layers, rp_max, st);   // short-side vectors of the kept atoms
+  if (tri_form) {                                                   // short-side vectors of the kept atoms
+    if (any_small) launch_sp_eigvec(d_layers, n_layers, rp_max_small, st);
+    launch_sp_eigvec_big(d_layers, d_big, (int)big_layers.size(), rp_max, st);
+  }
   launch_sp_backproject(d_layers, d_bp, (int)bp_tiles.size(), std::max(r_max_tall, 1), st);
   launch_sp_finish_atoms(d_layers, n_layers, k_cap_max, st);
-  stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, tri_form ? 3 : 2);
+  stage_end(ctx, ATOMO_STAGE_BACKPROJECT, st, tri_form ? 2 + (any_small ? 1 : 0) + (any_big ? 1 : 0) : 2);
   CK(cudaGetLastError());
   if (flags_pending) {
     // the one host wait of the persistent forms: the kernels' bounded waits report here

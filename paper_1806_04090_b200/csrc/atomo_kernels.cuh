@@ -90,13 +90,19 @@ struct SpLayer {
   float* row_inv;              // rp: 1 / norm of each short-side vector as stored in X
   float* refine_partials;      // [refine_tiles][rp] partial squared norms
   // tridiagonal route (short side <= 512): T = Q^T A Q, eigenvalues by bisection, vectors of the kept atoms only
-  int tri;                     // this layer takes the tridiagonal route
+  int tri;                     // this layer takes the tridiagonal route: 1 = registers of a cluster (rp <= 512), 2 = blocked, A in global memory
   double* td_d; double* td_e;  // rp each: diagonal and off-diagonal of T
   double* td_tau;              // rp: beta_k of the reflectors H_k = I - beta_k v_k v_k^T
   int td_ldv;                  // floats per row of td_V: r rounded up to a multiple of 4 (16-byte rows)
   float* td_V;                 // r x td_ldv: row k = v_k / ||v_k|| (zero up to index k), fp32 for the back-transformation: H_k = I - 2 u u^T
   double* lam64;               // rp: eigenvalues of T, ascending (scaled units); lam holds the same in fp32
   uint32_t* vec_ticket;        // CTAs of the vector kernel that finished this layer; zeroed per call
+  // tridiagonal route for short sides above 512 (tri = 2): blocked Householder reduction with A in global memory
+  void* tb_A;                  // r x lda matrix the reduction works on: float (= A) or double (tb_fp64)
+  void* tb_W;                  // [panel][tb_ldw] the panel's w vectors, same type as tb_A
+  int64_t tb_ldw;
+  int tb_fp64;                 // matrix and panel vectors in fp64
+  double* tb_vecwork;          // [slots][5][rp] work vectors of the twisted factorisation
 };
 
 struct SpDecodeLayer {
@@ -137,6 +143,14 @@ int sp_configure_tridiag();                                       // co-resident
 int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, cudaStream_t st);  // cudaError_t
 void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, cudaStream_t st);
 void launch_sp_eigvec(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
+// tridiagonal route for short sides above 512 (atomo_tridiag_big.cu)
+int sp_tridiag_big_max_r();
+int sp_tridiag_big_panel();
+int sp_tridiag_big_min_ctas(int r);                               // fewest CTAs per layer that hold r rows
+int sp_eigvec_big_slots();                                        // warps per layer of the vector kernel (work vectors)
+int sp_configure_tridiag_big();                                   // 0 if available
+int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, int ctas, int fp64, cudaStream_t st);  // cudaError_t
+void launch_sp_eigvec_big(const SpLayer* d_layers, const int* d_big, int n_big, int rp_max, cudaStream_t st);
 int launch_sp_cholesky(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 int launch_sp_cholesky_big(const SpLayer* d_layers, const TileRef* d_ctas, int n_ctas, int max_panels, cudaStream_t st);
 int sp_cholesky_big_rows_per_cta();

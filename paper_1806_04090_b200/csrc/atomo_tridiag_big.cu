@@ -1,0 +1,502 @@
+// Tridiagonal route for layers with a short side above 512 (Section 5 of the paper asks for the SVD of every layer
+// gradient; the probabilities of Eq. 3 / Algorithm 1 need the singular values of all atoms, Eq. 2 the vectors of the
+// kept atoms only).  The scaled Gram matrix A (r x r, r up to 4096) no longer fits the registers of a cluster, so it
+// stays in global memory and the reduction is the blocked (panel) form of the Householder tridiagonalisation:
+//
+//   sp_tridiag_big_kernel : T = Q^T A Q.  A cluster of C CTAs (C = 1, 2, 4, 8 or 16) owns a layer; rows are dealt to
+//                           the CTAs in blocks of 32 (block b belongs to CTA b mod C).  Within a panel of 32 columns
+//                           the stored matrix A0 is not touched: step c forms column c as it would be after the
+//                           panel's earlier reflectors (A0[:, c] - U W[c]^T - W U[c]^T), the unit reflector u_c
+//                           (H_c = I - 2 u u^T), the product y = A0 u (the one pass over the trailing block: one
+//                           warp per row, the lanes along the row) with the same correction, and
+//                           w = 2 y - (2 u^T y) u.  After the panel the trailing block takes the rank-64 update
+//                           A0 -= U W^T + W U^T (register-tiled, 4 x 4 outputs per thread).  The reflectors go to
+//                           global memory as fp32 unit vectors for the back-transformation.
+//                           Storage type T = float: the matrix and the panel vectors are kept in fp32 and the long
+//                           sums (row products) run in fp32 over at most r / 128 terms per lane before they are
+//                           added in fp64; column updates, norms and all scalars are fp64.  T = double keeps
+//                           everything in fp64.  Every sum has a fixed order that does not depend on C: a row product
+//                           is one warp's, block-wide sums go over the 32-row blocks in ascending order.
+//   sp_eigvec_big_kernel  : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
+//                           route, its work vectors in global memory), back-transformation u = Q z four reflectors at
+//                           a time (fp32), one warp per kept atom.
+//
+// The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
+// Work per layer: the matrix-vector products read sum_c (r - c)^2 ~ r^3 / 3 matrix entries (the bound of this kernel:
+// bytes from L2 / HBM), the panel updates cost 2 r^3 / 3 multiply-adds.
+#include <cooperative_groups.h>
+
+#include "atomo_kernels.cuh"
+#include "atomo_twisted.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace atomo {
+
+namespace {
+
+constexpr int kTbThreads = 1024;
+constexpr int kTbWarps = kTbThreads / 32;
+constexpr int kTbNB = 32;                    // columns per panel
+constexpr int kTbMaxC = 16;                  // CTAs per cluster
+constexpr int kTbMaxR = 4096;
+constexpr int kTbMaxBlocks = kTbMaxR / 32;   // 32-row blocks of a layer
+
+template <typename T> struct Vec4;           // 16-byte (float) / 32-byte (double) groups of four matrix entries
+template <> struct Vec4<float> { using type = float4; };
+template <> struct Vec4<double> { using type = double4; };
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ double4 ldcg4(const double* p) {
+  const double2 a = __ldcg(reinterpret_cast<const double2*>(p)), b = __ldcg(reinterpret_cast<const double2*>(p) + 1);
+  return make_double4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void st4(double* p, double4 v) {
+  reinterpret_cast<double2*>(p)[0] = make_double2(v.x, v.y);
+  reinterpret_cast<double2*>(p)[1] = make_double2(v.z, v.w);
+}
+
+// the TR consecutive row operands of a thread as one shared-memory load
+template <typename T> __device__ __forceinline__ void load_rows(const T* p, T* out);
+template <> __device__ __forceinline__ void load_rows<float>(const float* p, float* out) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <> __device__ __forceinline__ void load_rows<double>(const double* p, double* out) {
+  const double2 v = *reinterpret_cast<const double2*>(p);
+  out[0] = v.x; out[1] = v.y;
+}
+
+// sum of the per-block partial sums in ascending block order, the same bits in every thread of every CTA
+__device__ __forceinline__ double tb_ordered_sum(const double* part, int nblk, int lane) {
+  double s = 0.0;
+  for (int b = lane; b < nblk; b += 32) s += part[b];
+  return warp_sum(s);
+}
+
+struct alignas(16) TbShared {
+  double part_a[kTbMaxBlocks];     // per 32-row block: ||x||^2 partial of the current column
+  double part_k[kTbMaxBlocks];     // per 32-row block: u^T p partial
+  double dots[2 * kTbNB];          // a_t = w_t^T u, b_t = u_t^T u of the panel's earlier reflectors
+  double pc[2 * kTbNB];            // u_t[c], w_t[c]: the panel's entries in row c
+  double y[kTbThreads];            // A0 u for this CTA's rows (local row order)
+  double x0;                       // first entry of the pivot column
+};
+
+}  // namespace
+
+template <typename T, int C>
+__global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpLayer* __restrict__ layers,
+                                                                       const int* __restrict__ big_layers) {
+  cg::cluster_group cluster = cg::this_cluster();
+  extern __shared__ __align__(16) unsigned char tb_smem[];
+  TbShared& S = *reinterpret_cast<TbShared*>(tb_smem);
+  T* const s_u = reinterpret_cast<T*>(tb_smem + sizeof(TbShared));            // [r4] current reflector, zero up to c
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const int q = C == 1 ? 0 : (int)cluster.block_rank();
+  const SpLayer& L = layers[big_layers[blockIdx.x / C]];
+  const int r = L.r;
+  const int64_t lda = L.lda;
+  T* const A = reinterpret_cast<T*>(L.tb_A);
+  T* const W = reinterpret_cast<T*>(L.tb_W);
+  const int64_t ldw = L.tb_ldw;
+  float* const V = L.td_V;
+  const int64_t ldv = L.td_ldv;
+  double* const td_d = L.td_d;
+  double* const td_e = L.td_e;
+  const int nblk = (r + 31) / 32;
+  const int r4 = (r + 3) & ~3;
+  T* const s_gemm = s_u + r4;                                                  // operand tiles of the panel update
+  // this thread's row: block (tid / 32) of this CTA = global block (tid / 32) * C + q
+  const int gb = w * C + q;
+  const int g = gb * 32 + lane;
+  const bool valid = gb < nblk && g < r;
+  const int n_lblk = (nblk - q + C - 1) / C;                                   // 32-row blocks of this CTA (<= 32)
+
+  auto sync_all = [&]() { if (C == 1) __syncthreads(); else cluster.sync(); };
+  // a value into the same shared-memory slot of every CTA of the cluster
+  auto bcast = [&](double* slot, double v) {
+    if (C == 1) { *slot = v; return; }
+#pragma unroll
+    for (int rk = 0; rk < C; ++rk) *cluster.map_shared_rank(slot, rk) = v;
+  };
+
+  for (int i = tid; i < r4; i += kTbThreads) s_u[i] = (T)0;
+  if (C > 1) cluster.sync();                                                   // every CTA runs: remote stores may start
+
+  const int n_ref = r - 2;                                                     // reflectors: columns 0 .. r-3
+  for (int c = 0; c < r; ++c) {
+    const int p0 = c / kTbNB * kTbNB;
+    const int i = c < n_ref ? c - p0 : 0;                                      // pending reflectors of this panel (the last panel is applied before the last two columns)
+    // ---- the panel's entries in row c ----
+    if (tid < 2 * i) {
+      const int t = tid >> 1;
+      S.pc[tid] = (tid & 1) ? (double)__ldcg(W + (int64_t)t * ldw + c) : (double)__ldcg(V + (int64_t)(p0 + t) * ldv + c);
+    }
+    __syncthreads();
+    // ---- column c as the earlier reflectors of the panel left it ----
+    double a = 0.0;
+    if (valid && g >= c) {
+      a = (double)__ldcg(A + (int64_t)c * lda + g);
+      for (int t = 0; t < i; ++t) {
+        const double ut = (double)__ldcg(V + (int64_t)(p0 + t) * ldv + g);
+        const double wt = (double)__ldcg(W + (int64_t)t * ldw + g);
+        a -= ut * S.pc[2 * t + 1] + wt * S.pc[2 * t];
+      }
+      if (g == c) td_d[c] = a;
+    }
+    if (c >= n_ref) {                                                          // the last two columns: no reflector
+      if (c == r - 2 && valid && g == r - 1) td_e[c] = a;
+      continue;                                                                // uniform over the cluster
+    }
+    const bool live = valid && g > c;
+    {
+      const double sq = warp_sum(live ? a * a : 0.0);
+      if (lane == 0 && gb < nblk) bcast(&S.part_a[gb], sq);
+      if (valid && g == c + 1) bcast(&S.x0, a);
+    }
+    sync_all();
+    const double nx2 = tb_ordered_sum(S.part_a, nblk, lane);
+    const double x0 = S.x0;
+    double alpha = 0.0, inv = 0.0;
+    if (nx2 > 1.0e-290) {                                                      // below: a zero column, H = I
+      const double nx = sqrt(nx2);
+      alpha = -copysign(nx, x0);
+      inv = rsqrt(2.0 * nx * (nx + fabs(x0)));                                 // 1 / ||x - alpha e_1||
+    }
+    double u_own = 0.0;
+    if (valid) {
+      if (live) u_own = (double)(T)((a - (g == c + 1 ? alpha : 0.0)) * inv);   // the stored precision is the one used
+      V[(int64_t)c * ldv + g] = (float)u_own;
+      if (g == c + 1) td_e[c] = alpha;
+      if (C == 1) s_u[g] = (T)u_own;
+      else {
+#pragma unroll
+        for (int rk = 0; rk < C; ++rk) cluster.map_shared_rank(s_u, rk)[g] = (T)u_own;
+      }
+    }
+    sync_all();
+    // ---- y = A0 u over this CTA's live rows (warp w: lane position w of every block) and the panel dots ----
+    {
+      const int c0 = (c + 1) & ~3;
+      for (int lb = 0; lb < n_lblk; ++lb) {
+        const int row = (lb * C + q) * 32 + w;
+        if (row <= c || row >= r) continue;
+        const T* __restrict__ ar = A + (int64_t)row * lda;
+        T acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;
+        int h = c0 + lane * 4;
+        for (; h + 3 + 128 < r; h += 256) {                                    // two groups of four in flight
+          const typename Vec4<T>::type m0 = ldcg4(ar + h), m1 = ldcg4(ar + h + 128);
+          const typename Vec4<T>::type u0 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h);
+          const typename Vec4<T>::type u1 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h + 128);
+          acc0 = fma(m0.x, u0.x, acc0); acc1 = fma(m0.y, u0.y, acc1); acc2 = fma(m0.z, u0.z, acc2); acc3 = fma(m0.w, u0.w, acc3);
+          acc0 = fma(m1.x, u1.x, acc0); acc1 = fma(m1.y, u1.y, acc1); acc2 = fma(m1.z, u1.z, acc2); acc3 = fma(m1.w, u1.w, acc3);
+        }
+        for (; h + 3 < r; h += 128) {
+          const typename Vec4<T>::type m0 = ldcg4(ar + h);
+          const typename Vec4<T>::type u0 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h);
+          acc0 = fma(m0.x, u0.x, acc0); acc1 = fma(m0.y, u0.y, acc1); acc2 = fma(m0.z, u0.z, acc2); acc3 = fma(m0.w, u0.w, acc3);
+        }
+        {
+          const int ht = (r & ~3) + lane;                                      // the last r mod 4 columns
+          if (ht < r && ht >= c0) acc0 = fma(__ldcg(ar + ht), s_u[ht], acc0);
+        }
+        const double s = warp_sum(((double)acc0 + (double)acc1) + ((double)acc2 + (double)acc3));
+        if (lane == 0) S.y[lb * 32 + w] = s;
+      }
+      for (int id = w; id < 2 * i; id += kTbWarps) {
+        const int t = id >> 1;
+        double acc = 0.0;
+        if (id & 1) { const float* v = V + (int64_t)(p0 + t) * ldv; for (int h = c + 1 + lane; h < r; h += 32) acc = fma((double)__ldcg(v + h), (double)s_u[h], acc); }
+        else { const T* wv = W + (int64_t)t * ldw; for (int h = c + 1 + lane; h < r; h += 32) acc = fma((double)__ldcg(wv + h), (double)s_u[h], acc); }
+        acc = warp_sum(acc);
+        if (lane == 0) S.dots[id] = acc;
+      }
+    }
+    __syncthreads();
+    // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
+    double p = 0.0;
+    if (live) {
+      double y = S.y[tid];
+      for (int t = 0; t < i; ++t) {
+        const double ut = (double)__ldcg(V + (int64_t)(p0 + t) * ldv + g);
+        const double wt = (double)__ldcg(W + (int64_t)t * ldw + g);
+        y -= ut * S.dots[2 * t] + wt * S.dots[2 * t + 1];
+      }
+      p = 2.0 * y;
+    }
+    {
+      const double kp = warp_sum(u_own * p);
+      if (lane == 0 && gb < nblk) bcast(&S.part_k[gb], kp);
+    }
+    sync_all();
+    const double K = tb_ordered_sum(S.part_k, nblk, lane);
+    if (valid) W[(int64_t)(c - p0) * ldw + g] = (T)(live ? p - K * u_own : 0.0);
+    const bool flush = (c - p0 == kTbNB - 1) || (c == n_ref - 1);
+    if (!flush) { sync_all(); continue; }
+    // ---- end of the panel: A0 -= U W^T + W U^T on the rows and columns beyond c (this CTA's rows) ----
+    if (C == 1) { __threadfence_block(); __syncthreads(); } else { __threadfence(); cluster.sync(); }
+    {
+      constexpr int TR = sizeof(T) == 4 ? 4 : 2;                               // rows per thread
+      constexpr int MR = 32 * TR;                                              // local rows per tile (whole 32-row blocks)
+      const int nr = c - p0 + 1;                                               // reflectors in the panel
+      const int g0 = c + 1;
+      T* const s_ur = s_gemm;                                                  // [kTbNB][MR]
+      T* const s_wr = s_ur + kTbNB * MR;
+      T* const s_uc = s_wr + kTbNB * MR;                                       // [kTbNB][128]
+      T* const s_wc = s_uc + kTbNB * 128;
+      const int wr = w >> 3, wc = w & 7;                                       // warp: 8 TR rows x 16 columns
+      const int ly = lane >> 2, lx = lane & 3;
+      const int n_lrows = n_lblk * 32;
+      for (int mr0 = 0; mr0 < n_lrows; mr0 += MR) {
+        // last global row of this tile; dead tiles are skipped
+        const int lb_last = min(mr0 / 32 + MR / 32, n_lblk) - 1;
+        if ((lb_last * C + q) * 32 + 31 < g0) continue;
+        __syncthreads();
+        for (int e = tid; e < nr * MR; e += kTbThreads) {
+          const int t = e / MR, lr = mr0 + e % MR;
+          const int gr = ((lr >> 5) * C + q) * 32 + (lr & 31);
+          const bool in = (lr >> 5) < n_lblk && gr < r;
+          s_ur[t * MR + e % MR] = in ? (T)__ldcg(V + (int64_t)(p0 + t) * ldv + gr) : (T)0;
+          s_wr[t * MR + e % MR] = in ? __ldcg(W + (int64_t)t * ldw + gr) : (T)0;
+        }
+        for (int hc0 = g0 & ~127; hc0 < r; hc0 += 128) {
+          __syncthreads();
+          for (int e = tid; e < nr * 128; e += kTbThreads) {
+            const int t = e >> 7, h = hc0 + (e & 127);
+            s_uc[e] = h < r ? (T)__ldcg(V + (int64_t)(p0 + t) * ldv + h) : (T)0;
+            s_wc[e] = h < r ? __ldcg(W + (int64_t)t * ldw + h) : (T)0;
+          }
+          __syncthreads();
+          T acc[TR][4];
+#pragma unroll
+          for (int x = 0; x < TR; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) acc[x][y] = 0;
+          const int lr0 = wr * (8 * TR) + ly * TR;                             // first local row (in the tile) of this thread
+          const int lc0 = wc * 16 + lx * 4;
+          for (int t = 0; t < nr; ++t) {
+            T ru[TR], rw[TR];
+            load_rows<T>(s_ur + t * MR + lr0, ru);
+            load_rows<T>(s_wr + t * MR + lr0, rw);
+            const typename Vec4<T>::type cu = *reinterpret_cast<const typename Vec4<T>::type*>(s_uc + t * 128 + lc0);
+            const typename Vec4<T>::type cw = *reinterpret_cast<const typename Vec4<T>::type*>(s_wc + t * 128 + lc0);
+#pragma unroll
+            for (int x = 0; x < TR; ++x) {
+              acc[x][0] = fma(ru[x], cw.x, acc[x][0]); acc[x][1] = fma(ru[x], cw.y, acc[x][1]);
+              acc[x][2] = fma(ru[x], cw.z, acc[x][2]); acc[x][3] = fma(ru[x], cw.w, acc[x][3]);
+              acc[x][0] = fma(rw[x], cu.x, acc[x][0]); acc[x][1] = fma(rw[x], cu.y, acc[x][1]);
+              acc[x][2] = fma(rw[x], cu.z, acc[x][2]); acc[x][3] = fma(rw[x], cu.w, acc[x][3]);
+            }
+          }
+#pragma unroll
+          for (int x = 0; x < TR; ++x) {
+            const int lr = mr0 + lr0 + x;
+            const int gr = ((lr >> 5) * C + q) * 32 + (lr & 31);
+            const int h = hc0 + lc0;
+            if ((lr >> 5) >= n_lblk || gr >= r || gr < g0 || h >= r) continue;
+            T* dst = A + (int64_t)gr * lda + h;
+            if (h + 3 < r) {
+              typename Vec4<T>::type o = ldcg4(dst);
+              o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
+              st4(dst, o);
+            } else {
+              for (int y = 0; y < 4 && h + y < r; ++y) dst[y] = __ldcg(dst + y) - acc[x][y];
+            }
+          }
+        }
+      }
+    }
+    if (C == 1) { __threadfence_block(); __syncthreads(); } else { __threadfence(); cluster.sync(); }
+  }
+  if (C > 1) cluster.sync();                                                   // nobody leaves while a peer may still write here
+}
+
+// ---- vectors of the kept atoms ------------------------------------------------------------------------------------
+namespace {
+constexpr int kVbThreads = 128;
+constexpr int kVbWarps = kVbThreads / 32;
+constexpr int kVbCtas = 4;                   // CTAs per layer: 16 warps, one kept atom each at a time
+constexpr double kVbSameEig = 1.0e-9;        // as on the small route
+}  // namespace
+
+__global__ void __launch_bounds__(kVbThreads) sp_eigvec_big_kernel(const SpLayer* __restrict__ layers,
+                                                                   const int* __restrict__ big_layers) {
+  const SpLayer& L = layers[big_layers[blockIdx.x]];
+  extern __shared__ __align__(16) unsigned char vb_smem[];
+  const int r = L.r, rp = L.rp;
+  double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
+  double* s_e = s_d + rp;                                      // [rp]
+  float* s_z = reinterpret_cast<float*>(s_e + rp);             // [warps][rp]
+  __shared__ uint32_t s_last;
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const uint32_t k = L.hdr->k;
+  const float* const gV = L.td_V; const int64_t ldv = L.td_ldv; const double* const gLam = L.lam64;
+  const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
+  const int nref = max(r - 2, 0);
+  for (int i = tid; i < r; i += kVbThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
+  __syncthreads();
+  const int slot = blockIdx.y * kVbWarps + w;                  // 0 .. 15
+  double* wa = L.tb_vecwork + (size_t)slot * 5 * rp;
+  double* wb = wa + rp; double* wc = wb + rp; double* wd = wc + rp; double* zz = wd + rp;
+  float* z = s_z + (size_t)w * rp;
+  for (uint32_t a = slot; a < k; a += kVbCtas * kVbWarps) {
+    const int ei = gPerm[gIdx[a]];                             // index of the atom's eigenvalue (ascending order)
+    double lambda = gLam[ei];
+    int skip = 0;                                              // earlier kept atoms with the same eigenvalue: another twist index each
+    for (uint32_t b = lane; b < a; b += 32) skip += fabs(gLam[gPerm[gIdx[b]]] - lambda) <= kVbSameEig ? 1 : 0;
+    skip = (int)warp_sum((uint32_t)skip);
+    double n2 = 1.0;
+    const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, skip, &n2);
+    double gap = 1.0e300;
+    if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
+    if (ei + 1 < r) gap = fmin(gap, fabs(gLam[ei + 1] - lambda));
+    if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {      // one Rayleigh-quotient step, then the vector again
+      lambda += corr;
+      __syncwarp();
+      twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, 0, &n2);
+    }
+    __syncwarp();
+    const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
+    for (int i = lane; i < r; i += 32) z[i] = (float)(zz[i] * inv);
+    __syncwarp();
+    // u = H_0 H_1 ... H_{r-3} z, H = I - 2 v v^T with unit v: from the last reflector to the first, four at a time.
+    // For a group applied in the order 0, 1, 2, 3:  c_0 = 2 v_0.z,  c_i = 2 (v_i.z - sum_{j<i} c_j v_i.v_j),
+    // z -= sum c_i v_i.  Reflector kk is zero up to index kk, so the sums start at the group's lowest kk + 1.
+    for (int top = nref - 1; top >= 0; top -= 4) {
+      const float* v0 = gV + (int64_t)top * ldv;
+      const float* v1 = gV + (int64_t)max(top - 1, 0) * ldv;
+      const float* v2 = gV + (int64_t)max(top - 2, 0) * ldv;
+      const float* v3 = gV + (int64_t)max(top - 3, 0) * ldv;
+      const float m1 = top - 1 >= 0 ? 1.0f : 0.0f, m2 = top - 2 >= 0 ? 1.0f : 0.0f, m3 = top - 3 >= 0 ? 1.0f : 0.0f;
+      const int h0 = max(top - 3, 0) + 1;
+      float z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
+      for (int h = h0 + lane; h < r; h += 32) {
+        const float zh = z[h];
+        const float r0 = v0[h], r1 = m1 * v1[h], r2 = m2 * v2[h], r3 = m3 * v3[h];
+        z0 = fmaf(r0, zh, z0); z1 = fmaf(r1, zh, z1); z2 = fmaf(r2, zh, z2); z3 = fmaf(r3, zh, z3);
+        g10 = fmaf(r1, r0, g10); g20 = fmaf(r2, r0, g20); g21 = fmaf(r2, r1, g21);
+        g30 = fmaf(r3, r0, g30); g31 = fmaf(r3, r1, g31); g32 = fmaf(r3, r2, g32);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        z0 += __shfl_xor_sync(0xffffffffu, z0, o); z1 += __shfl_xor_sync(0xffffffffu, z1, o);
+        z2 += __shfl_xor_sync(0xffffffffu, z2, o); z3 += __shfl_xor_sync(0xffffffffu, z3, o);
+        g10 += __shfl_xor_sync(0xffffffffu, g10, o); g20 += __shfl_xor_sync(0xffffffffu, g20, o);
+        g21 += __shfl_xor_sync(0xffffffffu, g21, o); g30 += __shfl_xor_sync(0xffffffffu, g30, o);
+        g31 += __shfl_xor_sync(0xffffffffu, g31, o); g32 += __shfl_xor_sync(0xffffffffu, g32, o);
+      }
+      const float c0 = 2.0f * z0;
+      const float c1 = 2.0f * (z1 - c0 * g10);
+      const float c2 = 2.0f * (z2 - c0 * g20 - c1 * g21);
+      const float c3 = 2.0f * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
+      for (int h = h0 + lane; h < r; h += 32)
+        z[h] -= fmaf(c0, v0[h], fmaf(c1, m1 * v1[h], fmaf(c2, m2 * v2[h], c3 * m3 * v3[h])));
+      __syncwarp();
+    }
+    float n2f = 0.0f;
+    for (int i = lane; i < r; i += 32) n2f = fmaf(z[i], z[i], n2f);
+    n2f = warp_sum(n2f);
+    const float invf = n2f > 0.0f ? rsqrtf(n2f) : 0.0f;
+    for (int i = lane; i < r; i += 32) gShort[(int64_t)a * r + i] = z[i] * invf;
+    __syncwarp();
+  }
+  // the last CTA of the layer orthogonalises kept atoms whose eigenvalues nearly coincide (their vectors are
+  // determined only as a subspace): modified Gram-Schmidt in payload order, one warp
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(L.vec_ticket, 1u) == (uint32_t)(kVbCtas - 1) ? 1u : 0u;
+  __syncthreads();
+  if (!s_last || w != 0 || k < 2) return;
+  __threadfence();
+  for (uint32_t a = 1; a < k; ++a) {
+    const double la = gLam[gPerm[gIdx[a]]];
+    bool changed = false;
+    for (uint32_t b = 0; b < a; ++b) {
+      const double lb = gLam[gPerm[gIdx[b]]];
+      if (fabs(la - lb) > kVbSameEig) continue;
+      volatile float* va = gShort + (int64_t)a * r;
+      const volatile float* vb = gShort + (int64_t)b * r;
+      double dot = 0.0;
+      for (int i = lane; i < r; i += 32) dot = fma((double)va[i], (double)vb[i], dot);
+      dot = warp_sum(dot);
+      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] - dot * (double)vb[i]);
+      __syncwarp();
+      changed = true;
+    }
+    if (changed) {
+      volatile float* va = gShort + (int64_t)a * r;
+      double n2 = 0.0;
+      for (int i = lane; i < r; i += 32) n2 = fma((double)va[i], (double)va[i], n2);
+      n2 = warp_sum(n2);
+      const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
+      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] * inv);
+      __syncwarp();
+    }
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------------
+namespace {
+
+template <typename T> size_t tb_smem_bytes(int r_max) {
+  constexpr int TR = sizeof(T) == 4 ? 4 : 2;
+  const size_t r4 = (size_t)((r_max + 3) & ~3);
+  return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128) * sizeof(T);
+}
+size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbWarps * sizeof(float)); }
+
+template <typename T, int C> int tb_configure_one() {
+  auto* fn = sp_tridiag_big_kernel<T, C>;
+  if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tb_smem_bytes<T>(kTbMaxR)) != cudaSuccess) return 1;
+  if (C > 8 && cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) return 1;
+  return 0;
+}
+
+template <typename T, int C>
+int tb_launch_one(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, cudaStream_t st) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_big * C); cfg.blockDim = dim3(kTbThreads);
+  cfg.dynamicSmemBytes = tb_smem_bytes<T>(r_max); cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return (int)cudaLaunchKernelEx(&cfg, sp_tridiag_big_kernel<T, C>, d_layers, d_big);
+}
+
+}  // namespace
+
+int sp_tridiag_big_max_r() { return kTbMaxR; }
+int sp_tridiag_big_panel() { return kTbNB; }
+int sp_tridiag_big_min_ctas(int r) { int c = 1; while (c < kTbMaxC && (int64_t)c * kTbThreads < r) c <<= 1; return c; }
+int sp_eigvec_big_slots() { return kVbCtas * kVbWarps; }
+
+// 0 if the route is available on this GPU
+int sp_configure_tridiag_big() {
+  int bad = 0;
+  bad |= tb_configure_one<float, 1>() | tb_configure_one<float, 2>() | tb_configure_one<float, 4>() |
+         tb_configure_one<float, 8>() | tb_configure_one<float, 16>();
+  bad |= tb_configure_one<double, 1>() | tb_configure_one<double, 2>() | tb_configure_one<double, 4>() |
+         tb_configure_one<double, 8>() | tb_configure_one<double, 16>();
+  bad |= cudaFuncSetAttribute(sp_eigvec_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vb_smem_bytes(kTbMaxR)) != cudaSuccess;
+  if (bad) cudaGetLastError();
+  return bad;
+}
+
+// d_big: n_big layer indices, all stored as fp32 (fp64 = 0) or all as fp64; ctas = CTAs per layer (1, 2, 4, 8, 16)
+int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, int ctas, int fp64, cudaStream_t st) {
+  if (n_big <= 0) return 0;
+#define TB_CASE(CC) case CC: return fp64 ? tb_launch_one<double, CC>(d_layers, d_big, n_big, r_max, st) \
+                                         : tb_launch_one<float, CC>(d_layers, d_big, n_big, r_max, st);
+  switch (ctas) { TB_CASE(1) TB_CASE(2) TB_CASE(4) TB_CASE(8) TB_CASE(16) default: return (int)cudaErrorInvalidValue; }
+#undef TB_CASE
+}
+
+void launch_sp_eigvec_big(const SpLayer* d_layers, const int* d_big, int n_big, int rp_max, cudaStream_t st) {
+  if (n_big <= 0) return;
+  sp_eigvec_big_kernel<<<dim3(n_big, kVbCtas), kVbThreads, vb_smem_bytes(rp_max), st>>>(d_layers, d_big);
+}
+
+}  // namespace atomo
