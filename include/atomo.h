@@ -287,6 +287,12 @@ int atomo_set_tridiag_ctas(atomo_ctx* ctx, int32_t ctas_per_layer);
  * the first call.  Host only.                                                                                */
 int atomo_last_eig_scheme(atomo_ctx* ctx);
 
+/* --- measured arithmetic peaks (benchmark helper; the paper has no counterpart) ---------------
+ * Runs a register-only chain of fused multiply-adds on every SM of `device` for a few milliseconds and writes the
+ * rate to *tflops (HOST): fp32 (fp64 = 0) or fp64 (fp64 = 1).  The roofline of the kernels that are bound by plain
+ * ALU arithmetic is quoted against these figures.  Allocates and frees a small device buffer; synchronises.     */
+int atomo_measure_fma_peak(int device, int fp64, double* tflops /*HOST*/);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,7 +32,7 @@ EXPORTS = [
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
-    "atomo_set_tridiag_ctas",
+    "atomo_set_tridiag_ctas", "atomo_measure_fma_peak",
 ]
 
 
@@ -116,6 +116,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_persistent_eig.argtypes = [vp, i32]
     lib.atomo_last_eig_scheme.argtypes = [vp]
     lib.atomo_set_tridiag_ctas.argtypes = [vp, i32]
+    lib.atomo_measure_fma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
     lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                  ctypes.POINTER(vp), i32, vp]
     if path == LIB_PATH:
@@ -143,6 +144,15 @@ def payload_bytes_entrywise_compact(lengths: Sequence[int], k_cap: int, sat_cap:
     n = len(lengths)
     arr = (ctypes.c_int64 * n)(*[int(x) for x in lengths])
     return int(lib.atomo_payload_bytes_entrywise_compact(arr, n, int(k_cap), int(sat_cap)))
+
+
+def measure_fma_peak(device: int = 0, fp64: bool = False) -> float:
+    """Measured FMA rate of the GPU in TFLOP/s (fp32 or fp64), see atomo_measure_fma_peak."""
+    out = ctypes.c_double(0.0)
+    rc = load_library().atomo_measure_fma_peak(int(device), 1 if fp64 else 0, ctypes.byref(out))
+    if rc != 0:
+        raise AtomoError(rc, "atomo_measure_fma_peak")
+    return float(out.value)
 
 
 def default_k_cap(s: float, n_atoms: int) -> int:

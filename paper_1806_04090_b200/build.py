@@ -15,7 +15,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(HERE, "libatomo_b200.so")
 SOURCES = ["atomo_api.cu", "atomo_entrywise.cu", "atomo_spectral.cu", "atomo_eig.cu", "atomo_tc.cu", "atomo_static.cu",
-           "atomo_average.cu", "atomo_tridiag.cu", "atomo_tridiag_big.cu"]
+           "atomo_average.cu", "atomo_tridiag.cu", "atomo_tridiag_big.cu", "atomo_peaks.cu"]
 HEADERS = ["atomo_common.cuh", "atomo_kernels.cuh", "atomo_twisted.cuh"]
 
 

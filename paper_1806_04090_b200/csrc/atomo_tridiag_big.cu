@@ -24,6 +24,8 @@
 // The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
 // Work per layer: the matrix-vector products read sum_c (r - c)^2 ~ r^3 / 3 matrix entries (the bound of this kernel:
 // bytes from L2 / HBM), the panel updates cost 2 r^3 / 3 multiply-adds.
+#include <cstdio>
+
 #include <cooperative_groups.h>
 
 #include "atomo_kernels.cuh"
@@ -73,6 +75,23 @@ __device__ __forceinline__ double tb_ordered_sum(const double* part, int nblk, i
   double s = 0.0;
   for (int b = lane; b < nblk; b += 32) s += part[b];
   return warp_sum(s);
+}
+
+// this lane's part of sum_{h0 <= h < r} x[h] u[h] (x in global memory, written earlier in this launch; u in shared
+// memory), eight loads in flight
+template <typename X, typename T>
+__device__ __forceinline__ double tb_dot(const X* __restrict__ x, const T* __restrict__ u, int h0, int r, int lane) {
+  double acc = 0.0;
+  int h = h0 + lane;
+  for (; h + 7 * 32 < r; h += 8 * 32) {
+    X xb[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) xb[j] = __ldcg(x + h + 32 * j);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc = fma((double)xb[j], (double)u[h + 32 * j], acc);
+  }
+  for (; h < r; h += 32) acc = fma((double)__ldcg(x + h), (double)u[h], acc);
+  return acc;
 }
 
 struct alignas(16) TbShared {
@@ -125,6 +144,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   for (int i = tid; i < r4; i += kTbThreads) s_u[i] = (T)0;
   if (C > 1) cluster.sync();                                                   // every CTA runs: remote stores may start
 
+#ifdef TB_PROFILE
+  long long tp[6] = {0, 0, 0, 0, 0, 0}, tl = clock64();
+#define TB_MARK(k) { const long long now = clock64(); tp[k] += now - tl; tl = now; }
+#else
+#define TB_MARK(k)
+#endif
   const int n_ref = r - 2;                                                     // reflectors: columns 0 .. r-3
   for (int c = 0; c < r; ++c) {
     const int p0 = c / kTbNB * kTbNB;
@@ -139,10 +164,16 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     double a = 0.0;
     if (valid && g >= c) {
       a = (double)__ldcg(A + (int64_t)c * lda + g);
-      for (int t = 0; t < i; ++t) {
-        const double ut = (double)__ldcg(V + (int64_t)(p0 + t) * ldv + g);
-        const double wt = (double)__ldcg(W + (int64_t)t * ldw + g);
-        a -= ut * S.pc[2 * t + 1] + wt * S.pc[2 * t];
+      for (int t0 = 0; t0 < i; t0 += 8) {                                       // eight reflectors' entries in flight
+        float ub[8]; T wb[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = min(t0 + j, i - 1);
+          ub[j] = __ldcg(V + (int64_t)(p0 + t) * ldv + g); wb[j] = __ldcg(W + (int64_t)t * ldw + g);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (t0 + j < i) a -= (double)ub[j] * S.pc[2 * (t0 + j) + 1] + (double)wb[j] * S.pc[2 * (t0 + j)];
       }
       if (g == c) td_d[c] = a;
     }
@@ -150,6 +181,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       if (c == r - 2 && valid && g == r - 1) td_e[c] = a;
       continue;                                                                // uniform over the cluster
     }
+    TB_MARK(0)
     const bool live = valid && g > c;
     {
       const double sq = warp_sum(live ? a * a : 0.0);
@@ -177,52 +209,99 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       }
     }
     sync_all();
+    TB_MARK(1)
     // ---- y = A0 u over this CTA's live rows (warp w: lane position w of every block) and the panel dots ----
     {
       const int c0 = (c + 1) & ~3;
-      for (int lb = 0; lb < n_lblk; ++lb) {
-        const int row = (lb * C + q) * 32 + w;
-        if (row <= c || row >= r) continue;
-        const T* __restrict__ ar = A + (int64_t)row * lda;
-        T acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;
+      using V4 = typename Vec4<T>::type;
+      constexpr int RB = sizeof(T) == 4 ? 2 : 1;                               // rows per pass of a warp
+      for (int lb = 0; lb < n_lblk; lb += RB) {
+        int row[RB]; bool on[RB]; bool any = false;
+#pragma unroll
+        for (int x = 0; x < RB; ++x) {
+          row[x] = ((lb + x) * C + q) * 32 + w;
+          on[x] = lb + x < n_lblk && row[x] > c && row[x] < r;
+          any |= on[x];
+        }
+        if (!any) continue;
+        const int live_row = on[0] ? row[0] : row[RB - 1];                     // a dead row of the pair reads the live one
+        const T* ar[RB];
+#pragma unroll
+        for (int x = 0; x < RB; ++x) ar[x] = A + (int64_t)(on[x] ? row[x] : live_row) * lda;
+        T acc[RB][4];
+#pragma unroll
+        for (int x = 0; x < RB; ++x) { acc[x][0] = 0; acc[x][1] = 0; acc[x][2] = 0; acc[x][3] = 0; }
         int h = c0 + lane * 4;
-        for (; h + 3 + 128 < r; h += 256) {                                    // two groups of four in flight
-          const typename Vec4<T>::type m0 = ldcg4(ar + h), m1 = ldcg4(ar + h + 128);
-          const typename Vec4<T>::type u0 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h);
-          const typename Vec4<T>::type u1 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h + 128);
-          acc0 = fma(m0.x, u0.x, acc0); acc1 = fma(m0.y, u0.y, acc1); acc2 = fma(m0.z, u0.z, acc2); acc3 = fma(m0.w, u0.w, acc3);
-          acc0 = fma(m1.x, u1.x, acc0); acc1 = fma(m1.y, u1.y, acc1); acc2 = fma(m1.z, u1.z, acc2); acc3 = fma(m1.w, u1.w, acc3);
+        for (; h + 3 + 128 < r; h += 256) {                                    // two groups of four per row in flight
+          V4 m0[RB], m1[RB];
+#pragma unroll
+          for (int x = 0; x < RB; ++x) { m0[x] = ldcg4(ar[x] + h); m1[x] = ldcg4(ar[x] + h + 128); }
+          const V4 u0 = *reinterpret_cast<const V4*>(s_u + h), u1 = *reinterpret_cast<const V4*>(s_u + h + 128);
+#pragma unroll
+          for (int x = 0; x < RB; ++x) {
+            acc[x][0] = fma(m0[x].x, u0.x, acc[x][0]); acc[x][1] = fma(m0[x].y, u0.y, acc[x][1]);
+            acc[x][2] = fma(m0[x].z, u0.z, acc[x][2]); acc[x][3] = fma(m0[x].w, u0.w, acc[x][3]);
+            acc[x][0] = fma(m1[x].x, u1.x, acc[x][0]); acc[x][1] = fma(m1[x].y, u1.y, acc[x][1]);
+            acc[x][2] = fma(m1[x].z, u1.z, acc[x][2]); acc[x][3] = fma(m1[x].w, u1.w, acc[x][3]);
+          }
         }
         for (; h + 3 < r; h += 128) {
-          const typename Vec4<T>::type m0 = ldcg4(ar + h);
-          const typename Vec4<T>::type u0 = *reinterpret_cast<const typename Vec4<T>::type*>(s_u + h);
-          acc0 = fma(m0.x, u0.x, acc0); acc1 = fma(m0.y, u0.y, acc1); acc2 = fma(m0.z, u0.z, acc2); acc3 = fma(m0.w, u0.w, acc3);
+          V4 m0[RB];
+#pragma unroll
+          for (int x = 0; x < RB; ++x) m0[x] = ldcg4(ar[x] + h);
+          const V4 u0 = *reinterpret_cast<const V4*>(s_u + h);
+#pragma unroll
+          for (int x = 0; x < RB; ++x) {
+            acc[x][0] = fma(m0[x].x, u0.x, acc[x][0]); acc[x][1] = fma(m0[x].y, u0.y, acc[x][1]);
+            acc[x][2] = fma(m0[x].z, u0.z, acc[x][2]); acc[x][3] = fma(m0[x].w, u0.w, acc[x][3]);
+          }
         }
         {
           const int ht = (r & ~3) + lane;                                      // the last r mod 4 columns
-          if (ht < r && ht >= c0) acc0 = fma(__ldcg(ar + ht), s_u[ht], acc0);
+          if (ht < r) {
+#pragma unroll
+            for (int x = 0; x < RB; ++x) acc[x][0] = fma(__ldcg(ar[x] + ht), s_u[ht], acc[x][0]);
+          }
         }
-        const double s = warp_sum(((double)acc0 + (double)acc1) + ((double)acc2 + (double)acc3));
-        if (lane == 0) S.y[lb * 32 + w] = s;
+        double sum[RB];
+#pragma unroll
+        for (int x = 0; x < RB; ++x) sum[x] = ((double)acc[x][0] + (double)acc[x][1]) + ((double)acc[x][2] + (double)acc[x][3]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int x = 0; x < RB; ++x) sum[x] += __shfl_xor_sync(0xffffffffu, sum[x], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+          for (int x = 0; x < RB; ++x) if (on[x]) S.y[(lb + x) * 32 + w] = sum[x];
+        }
       }
+      TB_MARK(2)
       for (int id = w; id < 2 * i; id += kTbWarps) {
         const int t = id >> 1;
         double acc = 0.0;
-        if (id & 1) { const float* v = V + (int64_t)(p0 + t) * ldv; for (int h = c + 1 + lane; h < r; h += 32) acc = fma((double)__ldcg(v + h), (double)s_u[h], acc); }
-        else { const T* wv = W + (int64_t)t * ldw; for (int h = c + 1 + lane; h < r; h += 32) acc = fma((double)__ldcg(wv + h), (double)s_u[h], acc); }
+        if (id & 1) acc = tb_dot(V + (int64_t)(p0 + t) * ldv, s_u, c + 1, r, lane);
+        else acc = tb_dot(W + (int64_t)t * ldw, s_u, c + 1, r, lane);
         acc = warp_sum(acc);
         if (lane == 0) S.dots[id] = acc;
       }
     }
     __syncthreads();
+    TB_MARK(3)
     // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
     double p = 0.0;
     if (live) {
       double y = S.y[tid];
-      for (int t = 0; t < i; ++t) {
-        const double ut = (double)__ldcg(V + (int64_t)(p0 + t) * ldv + g);
-        const double wt = (double)__ldcg(W + (int64_t)t * ldw + g);
-        y -= ut * S.dots[2 * t] + wt * S.dots[2 * t + 1];
+      for (int t0 = 0; t0 < i; t0 += 8) {
+        float ub[8]; T wb[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int t = min(t0 + j, i - 1);
+          ub[j] = __ldcg(V + (int64_t)(p0 + t) * ldv + g); wb[j] = __ldcg(W + (int64_t)t * ldw + g);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          if (t0 + j < i) y -= (double)ub[j] * S.dots[2 * (t0 + j)] + (double)wb[j] * S.dots[2 * (t0 + j) + 1];
       }
       p = 2.0 * y;
     }
@@ -234,7 +313,8 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     const double K = tb_ordered_sum(S.part_k, nblk, lane);
     if (valid) W[(int64_t)(c - p0) * ldw + g] = (T)(live ? p - K * u_own : 0.0);
     const bool flush = (c - p0 == kTbNB - 1) || (c == n_ref - 1);
-    if (!flush) { sync_all(); continue; }
+    if (!flush) { sync_all(); TB_MARK(4) continue; }
+    TB_MARK(4)
     // ---- end of the panel: A0 -= U W^T + W U^T on the rows and columns beyond c (this CTA's rows) ----
     if (C == 1) { __threadfence_block(); __syncthreads(); } else { __threadfence(); cluster.sync(); }
     {
@@ -309,7 +389,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       }
     }
     if (C == 1) { __threadfence_block(); __syncthreads(); } else { __threadfence(); cluster.sync(); }
+    TB_MARK(5)
   }
+#ifdef TB_PROFILE
+  if (blockIdx.x == 0 && tid == 0)
+    printf("tridiag_big C=%d r=%d cycles: column %lld reflector %lld matvec %lld dots %lld w %lld gemm %lld\n", C, r, tp[0], tp[1], tp[2], tp[3], tp[4], tp[5]);
+#endif
   if (C > 1) cluster.sync();                                                   // nobody leaves while a peer may still write here
 }
 

@@ -178,6 +178,32 @@ def c2_paper_reshape(seed: int = 0, convs: Optional[Sequence[Sequence[int]]] = N
     return out
 
 
+def torch_lowrank_plus_noise(m: int, n: int, decay: float, seed: int, device, noise_rel: float | None = None,
+                             noise_std: float | None = None):
+    """The recipe of ``lowrank_plus_noise`` generated on a CUDA device with torch's generator (fp64, rounded once
+    to fp32): for benchmarks, where 96 Haar factors of order 4096 would take minutes on the host.  Not bit-equal
+    to the numpy version (another generator); same distribution."""
+    import torch
+    gen = torch.Generator(device=device)
+    gen.manual_seed(int(seed))
+    r = min(m, n)
+
+    def haar(rows, cols):
+        q, rr = torch.linalg.qr(torch.randn(rows, cols, dtype=torch.float64, device=device, generator=gen))
+        d = torch.sign(torch.diagonal(rr))
+        d[d == 0] = 1.0
+        return q * d
+
+    sigma = torch.arange(1, r + 1, dtype=torch.float64, device=device) ** (-decay)
+    g0 = (haar(m, r) * sigma) @ haar(n, r).T
+    if noise_rel is not None and noise_rel > 0:
+        e = torch.randn(m, n, dtype=torch.float64, device=device, generator=gen)
+        g0 = g0 + e * (noise_rel * torch.linalg.norm(g0) / torch.linalg.norm(e))
+    elif noise_std is not None and noise_std > 0:
+        g0 = g0 + noise_std * torch.randn(m, n, dtype=torch.float64, device=device, generator=gen)
+    return g0.to(torch.float32).contiguous()
+
+
 def c5_stress(seed: int = 0, count: int = 96, rows: int = 1024, cols: int = 4096
               ) -> List[np.ndarray]:
     """Config 5: ``count`` matrices rows x cols, sigma_i = 1/i, 0.5% noise."""

@@ -296,9 +296,11 @@ def test_config5_shape_properties(atomo):
             assert all(h.n_sat >= 1 for h in hdrs[1])          # sum(sigma) ~ 7.5 < 8 sigma_1
 
 
-def test_config5_full_size(atomo):
-    """Config 5 at its full size (96 layers of 1024 x 4096, 402,653,184 elements): more block pairs than the GPU
-    holds CTAs, so the eigen-solve runs as a sequence of persistent launches over groups of layers.  Six distinct
+@pytest.mark.parametrize("scheme", [3, 1])
+def test_config5_full_size(atomo, scheme):
+    """Config 5 at its full size (96 layers of 1024 x 4096, 402,653,184 elements) on the default route (the blocked
+    tridiagonal reduction, one CTA per layer) and on the Jacobi fallback (more block pairs than the GPU holds CTAs, so
+    that eigen-solve runs as a sequence of persistent launches over groups of layers).  Six distinct
     seeded matrices, each used 16 times (generating 96 Haar factors of order 4096 would take minutes on the host);
     every copy is its own layer with its own Philox stream.  Checked: status, singular values against a library SVD
     in fp64, sum(p) = s, kept atoms as singular triplets on sampled layers, the decode against its definition."""
@@ -308,8 +310,12 @@ def test_config5_full_size(atomo):
     dev = torch.device("cuda:0")
     ts = [torch.from_numpy(base[i % 6]).to(dev).clone() for i in range(96)]
     s = 4.0
-    pay, dbg = atomo.atomo_encode_spectral(ts, s, seed=91, step=5, k_cap=48, debug=True)
-    assert atomo.last_eig_scheme() == 1
+    try:
+        atomo.set_persistent_eig(scheme)
+        pay, dbg = atomo.atomo_encode_spectral(ts, s, seed=91, step=5, k_cap=48, debug=True)
+    finally:
+        atomo.set_persistent_eig(3)
+    assert atomo.last_eig_scheme() == scheme
     hdrs = pay.headers()
     assert [h.status for h in hdrs[1]] == [0] * 96
     outs = atomo.atomo_decode(pay)
