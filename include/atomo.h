@@ -14,7 +14,7 @@
  *     descriptors (atomo_mat, atomo_vec, pointer lists, shape lists) are HOST memory and are
  *     consumed before the call returns.
  *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
- *     atomo_encode_spectral on the tridiagonal route (eigen scheme 3, the default for short sides <= 512) never
+ *     atomo_encode_spectral on the tridiagonal routes (eigen scheme 3, the default) never
  *     waits on the host: a bounded device-side wait that ran out shows as ATOMO_ERR_TIMEOUT in the layers' status
  *     words.  On the Jacobi routes it waits once, after it has enqueued all its work (the kernels' bounded waits
  *     report there), or once per Jacobi sweep in launch scheme 0.  atomo_encode_entrywise and the decode calls
@@ -66,7 +66,7 @@ typedef enum {
   ATOMO_ERR_CAPACITY = 3,      /* host: payload buffer too small; device: kept atoms > k_cap       */
   ATOMO_ERR_NONFINITE = 4,     /* NaN or Inf found in a gradient                                   */
   ATOMO_ERR_NOT_CONVERGED = 5, /* eigen-solver hit its sweep cap (route 1: k = 0; route 0: result kept) */
-  ATOMO_ERR_TIMEOUT = 6,       /* reserved for bounded device-side waits                           */
+  ATOMO_ERR_TIMEOUT = 6,       /* a bounded device-side wait (mbarrier, step barrier) ran out      */
   ATOMO_ERR_CUDA = 7,          /* a CUDA runtime call failed; see atomo_last_cuda_error            */
   ATOMO_ERR_PAYLOAD = 8        /* decode: header does not match the shapes given                   */
 } atomo_status;
@@ -149,14 +149,26 @@ int64_t atomo_payload_bytes_entrywise_compact(const int64_t* n, int32_t n_vecs, 
 
 /* --- encode ---------------------------------------------------------------------------------
  * Spectral ATOMO (Section 5; Eq. 2, Eq. 3 / Algorithm 1) over a batch of layer gradients.
- * Per layer: thin SVD (Gram matrix of the short side -> Jacobi eigen-solver -> sigma and the
- * short-side vectors), probabilities from the descending sigma, Bernoulli draws, and for the
- * kept atoms the long-side vector by back-projection (G^T u_i or G v_i, normalised; its norm
+ * Per layer: thin SVD (Gram matrix of the short side -> eigenvalues of all atoms, hence every sigma ->
+ * short-side vectors of the kept atoms; see atomo_set_persistent_eig), probabilities from the descending
+ * sigma, Bernoulli draws, and for the kept atoms the long-side vector by back-projection (G^T u_i or G v_i, normalised; its norm
  * is the sigma_i used in coef = sigma_i / p_i).  Each layer needs min(rows, cols) <= 4096.     */
 int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers /*HOST array*/, int32_t n_layers,
                           double s, uint64_t seed, uint64_t step, int32_t k_cap,
                           void* payload /*DEVICE*/, int64_t capacity_bytes,
                           const atomo_debug* dbg /*HOST struct or NULL*/, void* stream);
+
+/* Test entry point: everything downstream of the SVD (Algorithm 1, the draws of Eq. 2, the compaction, the
+ * back-projection and the payload) for a decomposition that the caller supplies, so that a test can separate those
+ * steps from the conditioning of the SVD.  sigma[l] (DEVICE, r_l floats, descending) and short_vecs[l] (DEVICE,
+ * r_l x r_l floats, rank-major: row i = the unit short-side vector of atom i: u_i for rows <= cols, else v_i) replace
+ * the Gram matrix and the eigen-solver; both pointer lists are HOST arrays.  Everything else as atomo_encode_spectral
+ * (short sides up to 4096; the weights still use the norm of the back-projection G^T u_i, which equals sigma_i for an
+ * exact decomposition).                                                                                    */
+int atomo_encode_spectral_from_svd(atomo_ctx* ctx, const atomo_mat* layers /*HOST array*/, int32_t n_layers,
+                                   const float* const* sigma, const float* const* short_vecs, double s, uint64_t seed,
+                                   uint64_t step, int32_t k_cap, void* payload /*DEVICE*/, int64_t capacity_bytes,
+                                   const atomo_debug* dbg /*HOST struct or NULL*/, void* stream);
 
 /* Entry-wise ATOMO (Section 3; the QSGD / TernGrad family of Section 4) over a batch of flat
  * gradients, each with n < 2^32 elements and its own budget s (same s for every vector).       */
@@ -216,6 +228,10 @@ int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloa
  *   - All calls on a device share the one array: it still holds the previous call's tables, which
  *     the next call overwrites in stream order.  Two calls whose work overlaps on the GPU (different
  *     streams, no dependency) race on it; serialise them.
+ *   - The tables are staged in pageable host memory (up to 128 KB per calling thread): the copy may make
+ *     the host wait until earlier work on `stream` has drained, and the staging buffer is reused by the
+ *     thread's next call.
+ *   - out[l] must hold rows[l] * cols[l] floats: every element is written through the raw pointer.
  * `device` is the CUDA ordinal; payload, rows, cols, out, stream as in atomo_decode().               */
 enum { ATOMO_STATIC_MAX_LAYERS = 64, ATOMO_STATIC_MAX_TILES = 8192 };
 int atomo_decode_spectral_static(int device, const void* payload /*DEVICE*/, const int64_t* rows,
@@ -256,17 +272,23 @@ int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode);
  * turns into a visible error of the nuclear norm and thus of every p_i; the projection norm does not
  * have that floor.  It costs one more pass over G with twice the Gram matrix's arithmetic.              */
 int atomo_set_sigma_refinement(atomo_ctx* ctx, int32_t min_short_side);
-/* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols,
- * a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA kernel always.  */
+/* Gram matrix path: 1 (default) = tcgen05 tensor cores with the TF32 hi/lo split for layers with rows <= cols, a short
+ * side of at most 1024, a 16-byte aligned base and ld % 4 == 0 (other layers take the fp32 FMA kernel); 0 = fp32 FMA
+ * kernel always.  The tensor core accumulates in fp32 with truncation: at a short side of 1024 the probabilities then
+ * sit within about 3e-6 of those of an exact decomposition (the few largest p_i; measured), with the FMA kernel within
+ * about 5e-7.  A caller that needs every draw to agree with an fp64 computation outside a 1e-6 margin takes 0.    */
 int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
 /* Eigen-solver scheme (`enabled` = 0, 1, 2 or 3):
- * 3 (default) = tridiagonal route where it applies: when every layer of the batch has a short side of at most 512
- *     (and neither per-atom refinement nor the whole short-side basis is asked for), the scaled Gram matrix is
- *     reduced to tridiagonal form by Householder reflectors in fp64 (rows spread over the CTAs of a 16-CTA
- *     cluster, exchanged through distributed shared memory, one cluster barrier per step), all eigenvalues come
- *     from bisection on Sturm counts, and eigenvectors are computed for the kept atoms only (twisted
- *     factorisation, back-transformation with the reflectors).  Only the singular values of all atoms enter the
- *     probabilities; the vectors of atoms that are not kept are never formed.  Other batches take scheme 2;
+ * 3 (default) = the tridiagonal routes: the scaled Gram matrix of every layer is reduced to tridiagonal form by
+ *     Householder reflectors, all eigenvalues come from bisection on Sturm counts, and eigenvectors are computed for the
+ *     kept atoms only (twisted factorisation, back-transformation with the reflectors): only the singular values of
+ *     all atoms enter the probabilities, the vectors of atoms that are not kept are never formed.  Short sides up to
+ *     512: the rows sit in the registers of the CTAs of a 16-CTA cluster and are exchanged through distributed shared
+ *     memory, fp64 arithmetic, one cluster barrier per step.  Short sides above 512 (up to 4096): the matrix stays in
+ *     global memory (fp32) and the reduction is blocked in panels of 32 columns, a cluster of 1 to 16 CTAs per layer
+ *     (atomo_set_tridiag_ctas); sums and scalars in fp64.  Both kinds of layer can share one call.  A batch takes
+ *     scheme 2 instead when eigen-solver route 0 or the whole short-side basis (atomo_debug.short_vecs) is asked
+ *     for, or when the GPU cannot place the clusters;
  * 2 = one-sided Jacobi in thread-block clusters where they apply: when every layer of the batch has at most 16 block
  *     pairs (padded short side <= 512), each layer's CTAs sit in one 16-CTA cluster for the whole solve and hand
  *     their blocks to one another through distributed shared memory, with a cluster barrier per Jacobi step;
@@ -276,7 +298,9 @@ int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
  *     of a layer between steps; a batch that fits the GPU is one such launch.  A batch with a layer that alone
  *     needs more CTAs than the GPU holds (short side above 2048) takes scheme 0;
  * 0 = one launch per step and one host wait per sweep.
- * Schemes 1 to 3 wait on the host once, at the end of the call.                                              */
+ * Scheme 3 never waits on the host; schemes 1 and 2 wait once, at the end of the call.  The Jacobi schemes work in
+ * fp32 throughout and resolve the probabilities of layers with a short side of 1024 only to a few 1e-5; they are
+ * kept as a fallback and as an independent cross-check of scheme 3.                                              */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
 /* CTAs per layer of the blocked tridiagonal reduction that scheme 3 runs for short sides above 512: 0 (default) =
  * chosen per batch (the fewest that hold the layer's rows, doubled while SMs would stay idle), else 1, 2, 4, 8 or 16

@@ -32,7 +32,7 @@ EXPORTS = [
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
-    "atomo_set_tridiag_ctas", "atomo_measure_fma_peak",
+    "atomo_set_tridiag_ctas", "atomo_measure_fma_peak", "atomo_encode_spectral_from_svd",
 ]
 
 
@@ -116,6 +116,8 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_persistent_eig.argtypes = [vp, i32]
     lib.atomo_last_eig_scheme.argtypes = [vp]
     lib.atomo_set_tridiag_ctas.argtypes = [vp, i32]
+    lib.atomo_encode_spectral_from_svd.argtypes = [vp, ctypes.POINTER(_Mat), i32, ctypes.POINTER(vp), ctypes.POINTER(vp),
+                                                   ctypes.c_double, u64, u64, i32, vp, i64, ctypes.POINTER(_Debug), vp]
     lib.atomo_measure_fma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
     lib.atomo_decode_spectral_static.argtypes = [ctypes.c_int, vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                  ctypes.POINTER(vp), i32, vp]
@@ -255,8 +257,10 @@ def atomo_decode_spectral_static(payload: "Payload", out: Sequence[torch.Tensor]
     """Spectral decode that allocates nothing on the device: for processes whose framework
     allocator owns the whole GPU, or that cannot take cudaMalloc's device-wide synchronisation
     where they decode.  The caller supplies the output tensors; the per-call tables live in a fixed
-    array inside the library (limits: 64 layers, 8192 output tiles of 32 x 256).  Calls on one
-    device share that array, so they must not overlap on the GPU."""
+    array inside the library (limits: 64 layers, 8192 output tiles of 64 x 1024).  Calls on one
+    device share that array, so they must not overlap on the GPU.  Every output must be a contiguous
+    fp32 CUDA tensor on the payload's device with exactly rows * cols elements: the kernel writes all
+    of them through the raw pointer, so anything else is refused here, before the C call."""
     lib = load_library()
     if payload.kind != KIND_SPECTRAL:
         raise ValueError("atomo_decode_spectral_static decodes spectral payloads only")
@@ -264,6 +268,10 @@ def atomo_decode_spectral_static(payload: "Payload", out: Sequence[torch.Tensor]
     if len(out) != n:
         raise ValueError("one output tensor per layer is required (this call does not allocate)")
     dev = payload.buf.device.index if device is None else int(device)
+    for l, (o, (r_, c_)) in enumerate(zip(out, payload.shapes)):
+        if not (isinstance(o, torch.Tensor) and o.is_cuda and o.device.index == dev and o.dtype == torch.float32
+                and o.is_contiguous() and o.numel() == int(r_) * int(c_)):
+            raise ValueError(f"output {l}: a contiguous fp32 CUDA tensor on device {dev} with {int(r_) * int(c_)} elements is required")
     rows = (ctypes.c_int64 * n)(*[r for r, _ in payload.shapes])
     cols = (ctypes.c_int64 * n)(*[c for _, c in payload.shapes])
     ptrs = (ctypes.c_void_p * n)(*[o.data_ptr() for o in out])
@@ -366,6 +374,37 @@ class Atomo:
                                             ctypes.c_void_p(payload.data_ptr()), payload.numel(),
                                             ctypes.byref(ds) if ds is not None else None, self._stream_ptr(stream))
         self._check(rc, "atomo_encode_spectral")
+        return Payload(payload, KIND_SPECTRAL, shapes, int(k_cap), self), dbg
+
+    def atomo_encode_spectral_from_svd(self, layers: Sequence[torch.Tensor], sigma: Sequence[torch.Tensor],
+                                       short_vecs: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,
+                                       k_cap: Optional[int] = None, debug: bool = True,
+                                       stream: Optional[torch.cuda.Stream] = None):
+        """Test entry point: the path downstream of the SVD for a decomposition given by the caller.  sigma[l]: r
+        fp32 values, descending; short_vecs[l]: r x r fp32, row i = the unit short-side vector of atom i."""
+        n = len(layers)
+        mats = (_Mat * n)()
+        shapes = []
+        for i, g in enumerate(layers):
+            if not (g.is_cuda and g.dtype == torch.float32 and g.dim() == 2 and g.is_contiguous()):
+                raise ValueError("layers must be contiguous 2-D fp32 CUDA tensors")
+            r = min(g.shape)
+            for t, want in ((sigma[i], r), (short_vecs[i], r * r)):
+                if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.numel() == want):
+                    raise ValueError("sigma / short_vecs must be contiguous fp32 CUDA tensors of r and r * r elements")
+            mats[i] = _Mat(g.data_ptr(), g.shape[0], g.shape[1], g.shape[1])
+            shapes.append((int(g.shape[0]), int(g.shape[1])))
+        if k_cap is None:
+            k_cap = default_k_cap(s, max(min(r, c) for r, c in shapes))
+        payload = torch.empty(payload_bytes_spectral(shapes, k_cap), dtype=torch.uint8, device=layers[0].device)
+        dbg = self._make_debug([min(r, c) for r, c in shapes], True, False, layers[0].device) if debug else None
+        ds = self._debug_struct(dbg)
+        sp = (ctypes.c_void_p * n)(*[t.data_ptr() for t in sigma])
+        vp_ = (ctypes.c_void_p * n)(*[t.data_ptr() for t in short_vecs])
+        rc = self.lib.atomo_encode_spectral_from_svd(self._h, mats, n, sp, vp_, float(s), int(seed), int(step), int(k_cap),
+                                                     ctypes.c_void_p(payload.data_ptr()), payload.numel(),
+                                                     ctypes.byref(ds) if ds is not None else None, self._stream_ptr(stream))
+        self._check(rc, "atomo_encode_spectral_from_svd")
         return Payload(payload, KIND_SPECTRAL, shapes, int(k_cap), self), dbg
 
     def atomo_encode_entrywise(self, vecs: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,

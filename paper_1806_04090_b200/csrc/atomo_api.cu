@@ -313,9 +313,11 @@ int atomo_set_eig_mode(atomo_ctx* ctx, int32_t mode) {
 }
 
 // ==================================================================================================
-int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers, double s, uint64_t seed,
-                          uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
-                          const atomo_debug* dbg, void* stream) {
+static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers, double s, uint64_t seed,
+                                uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
+                                const atomo_debug* dbg, void* stream, const float* const* given_sigma,
+                                const float* const* given_short) {
+  const bool given = given_sigma != nullptr;                   // the decomposition comes from the caller: S1 is skipped
   if (!ctx || !layers || n_layers <= 0 || k_cap <= 0 || !payload) return ATOMO_ERR_INVALID_ARG;
   if (bad_budget(s)) return ATOMO_ERR_BUDGET;
   if ((reinterpret_cast<uintptr_t>(payload) & 15u) != 0) return ATOMO_ERR_INVALID_ARG;
@@ -361,7 +363,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     r_max = std::max(r_max, d.r); rp_max = std::max(rp_max, d.rp);
     const int gt = (d.r + 63) / 64;
     d.tc = 0; d.gram_split = 1;
-    if (ctx->tc_gram && ctx->tc_ok && !d.acc && sp_tc_eligible(d.G, d.rows, d.cols, d.ld)) {
+    // The tensor core's fp32 accumulation truncates, which perturbs sum(sigma) -- and with it the largest p_i -- by a few
+    // 1e-6 at a short side of 1024 and more above (measured 6e-6 at 4096): layers with a short side above 1024 take the
+    // fp32 FMA kernel, whose sums round to nearest (their Gram matrix is a small part of their cost)
+    if (ctx->tc_gram && ctx->tc_ok && !d.acc && d.r <= 1024 && sp_tc_eligible(d.G, d.rows, d.cols, d.ld)) {
       d.tc = 1;
       if (sp_tc_make_map(maps_blob.data() + (size_t)l * map_bytes, d.G, d.rows, d.cols, d.ld) != 0) return ATOMO_ERR_INVALID_ARG;
       tc_layers.push_back(l);
@@ -396,7 +401,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   // Tridiagonal routes first: eigenvalues of every atom from T = Q^T A Q, vectors for the kept atoms only -- in the
   // registers of a cluster for short sides up to 512, blocked with A in global memory above (no per-atom refinement,
   // no request for the whole short-side basis).  Otherwise the Jacobi routes, the cluster form first.
-  bool tri_form = ctx->eig_scheme == 3 && ctx->eig_mode != 0 && !(dbg && dbg->short_vecs);
+  bool tri_form = !given && ctx->eig_scheme == 3 && ctx->eig_mode != 0 && !(dbg && dbg->short_vecs);
   bool any_small = false, any_big = false;
   for (int l = 0; l < n_layers && tri_form; ++l) (L[l].rp <= sp_tridiag_max_rp() ? any_small : any_big) = true;
   if (tri_form && any_small) {
@@ -414,7 +419,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (L[l].tri == 2) big_layers.push_back(l);
   }
   if (tri_form) refine_tiles.clear();
-  bool cluster_form = !tri_form && ctx->eig_scheme >= 2 && ctx->eig_mode != 0;
+  bool cluster_form = !given && !tri_form && ctx->eig_scheme >= 2 && ctx->eig_mode != 0;
   for (int l = 0; l < n_layers && cluster_form; ++l) cluster_form = L[l].nb / 2 <= sp_jacobi_cluster_ctas() && L[l].rp <= sp_jacobi_cluster_max_rp();
   if (cluster_form) {
     int lg = 0;
@@ -422,7 +427,8 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (ctx->cluster_capacity[lg] < 0) ctx->cluster_capacity[lg] = sp_jacobi_cluster_capacity(rp_max);
     if (ctx->cluster_capacity[lg] < 1) cluster_form = false;
   }
-  for (int l = 0; l < n_layers; ++l) L[l].lam_ready = (cluster_form || tri_form) ? 1 : 0;
+  for (int l = 0; l < n_layers; ++l) L[l].lam_ready = (cluster_form || tri_form || given) ? 1 : 0;
+  if (given) { for (int l = 0; l < n_layers; ++l) L[l].refine = 0; refine_tiles.clear(); }
   // tensor-core Gram tiles: while the batch has fewer CTAs than the GPU has SMs, the K range of the layers with the
   // longest rows is split over 2 or 4 CTAs per tile (at least 16 stages of 32 columns per part)
   {
@@ -454,6 +460,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
   uint32_t* d_flag = nullptr;
   ClusterCta* d_ctas = nullptr;
   int* d_big = nullptr;
+  const float** d_given = nullptr;
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
   for (int pass = 0; pass < 2; ++pass) {
@@ -469,6 +476,7 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     d_flag = A.take<uint32_t>(4);
     d_ctas = A.take<ClusterCta>((size_t)n_layers * sp_jacobi_cluster_ctas());   // at most one cluster per layer
     d_big = A.take<int>(big_layers.size());
+    d_given = A.take<const float*>(given ? (size_t)2 * n_layers : 0);
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
@@ -498,6 +506,10 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
       d.tb_ldw = (d.r + 3) / 4 * 4;
       d.tb_W = A.take<float>(d.tri == 2 ? (size_t)sp_tridiag_big_panel() * d.tb_ldw : 0);
       d.tb_vecwork = A.take<double>(d.tri == 2 ? (size_t)sp_eigvec_big_slots() * 5 * d.rp : 0);
+      {
+        const size_t nb = (size_t)(d.r + 31) / 32;
+        d.tb_At = A.take<float>(d.tri == 2 && d.r <= 1024 ? nb * (nb + 1) / 2 * 1024 : 0);
+      }
       d.chol_dd = A.take<float>(32 * 32 + 32);
       d.row_inv = A.take<float>(d.rp);
       d.refine_partials = A.take<float>(d.refine ? (size_t)d.refine_tiles * d.rp : 0);
@@ -555,11 +567,19 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S1: Gram matrix, scaling ----
   stage_begin(ctx, ATOMO_STAGE_GRAM, st);
+  if (given) {
+    // singular values and short-side vectors as given: squared into the eigenvalue slots, vectors into the rows of X
+    std::vector<const float*> ptrs(2 * (size_t)n_layers);
+    for (int l = 0; l < n_layers; ++l) { ptrs[l] = given_sigma[l]; ptrs[n_layers + l] = given_short[l]; }
+    CK(cudaMemcpyAsync(d_given, ptrs.data(), ptrs.size() * sizeof(const float*), cudaMemcpyHostToDevice, st));
+    launch_sp_load_svd(d_layers, n_layers, d_given, d_given + n_layers, st);
+  } else {
   if (ctx->eig_mode == 0) launch_sp_init(d_layers, n_layers, nullptr, 0, st);   // the identity half of [A | I]
   launch_sp_gram(d_layers, d_gram, (int)gram_tiles.size(), st);
   launch_sp_gram_tc(d_layers, d_maps, d_tc, (int)tc_tiles.size(), d_flag + 1, st);
   launch_sp_scale(d_layers, n_layers, st);
-  if (ctx->eig_mode != 0 && !tri_form) {
+  }
+  if (!given && ctx->eig_mode != 0 && !tri_form) {
     const int ec = launch_sp_cholesky(d_layers, n_layers, rp_max, st);
     if (ec != 0) return fail_cuda(ctx, (cudaError_t)ec, "cudaLaunchKernelEx(cholesky)");
     const int e = launch_sp_cholesky_big(d_layers, d_chol, (int)chol_ctas.size(), chol_panels, st);
@@ -642,12 +662,12 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     CK(cudaMemcpyAsync(ctx->h_flag, d_flag, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
     flags_pending = true;                                  // read at the end of the call, after everything is enqueued
   }
-  const int capacity = (!cluster_form && !tri_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
+  const int capacity = (!given && !cluster_form && !tri_form && ctx->eig_scheme >= 1) ? sp_jacobi_persistent_capacity(row_floats_max) : 0;
   int max_layer_pairs = 0;
   for (int l = 0; l < n_layers; ++l) max_layer_pairs = std::max(max_layer_pairs, L[l].nb / 2);
   const bool persistent = capacity > 0 && max_layer_pairs <= capacity;
-  ctx->eig_scheme_used = tri_form ? 3 : cluster_form ? 2 : (persistent ? 1 : 0);
-  if (cluster_form || tri_form) {
+  if (!given) ctx->eig_scheme_used = tri_form ? 3 : cluster_form ? 2 : (persistent ? 1 : 0);
+  if (cluster_form || tri_form || given) {
     // done above
   } else if (persistent) {
     // d_flag[2] is raised if a step barrier gave up, d_flag[3] receives the steps executed
@@ -686,7 +706,11 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
 
   // ---- S2-S4: (refined singular values,) probabilities, draws, compaction ----
   stage_begin(ctx, ATOMO_STAGE_SAMPLE, st);
-  if (tri_form) launch_sp_bisect(d_layers, n_layers, r_max, st);   // all eigenvalues of the tridiagonal matrices
+  if (tri_form) {                                                   // all eigenvalues of the tridiagonal matrices
+    int64_t n_eig = 0;
+    for (int l = 0; l < n_layers; ++l) n_eig += L[l].r;
+    launch_sp_bisect(d_layers, n_layers, r_max, n_eig, st);
+  }
   launch_sp_refine(d_layers, n_layers, d_ref, (int)refine_tiles.size(), st);
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   launch_sp_finalize_sample(d_layers, n_layers, s, key, kind_step_word(ATOMO_KIND_SPECTRAL, step), max_sweeps,
@@ -710,6 +734,21 @@ int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_lay
     if (ctx->h_flag[2] != 0) { ctx->err = "a step barrier of the persistent eigen-solve ran out of polls"; return ATOMO_ERR_TIMEOUT; }
   }
   return ATOMO_OK;
+}
+
+int atomo_encode_spectral(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers, double s, uint64_t seed,
+                          uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
+                          const atomo_debug* dbg, void* stream) {
+  return encode_spectral_impl(ctx, layers, n_layers, s, seed, step, k_cap, payload, capacity_bytes, dbg, stream, nullptr, nullptr);
+}
+
+int atomo_encode_spectral_from_svd(atomo_ctx* ctx, const atomo_mat* layers, int32_t n_layers,
+                                   const float* const* sigma, const float* const* short_vecs, double s, uint64_t seed,
+                                   uint64_t step, int32_t k_cap, void* payload, int64_t capacity_bytes,
+                                   const atomo_debug* dbg, void* stream) {
+  if (!sigma || !short_vecs || n_layers <= 0) return ATOMO_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) if (!sigma[l] || !short_vecs[l]) return ATOMO_ERR_INVALID_ARG;
+  return encode_spectral_impl(ctx, layers, n_layers, s, seed, step, k_cap, payload, capacity_bytes, dbg, stream, sigma, short_vecs);
 }
 
 // ==================================================================================================

@@ -103,6 +103,8 @@ struct SpLayer {
   int64_t tb_ldw;
   int tb_fp64;                 // matrix and panel vectors in fp64
   double* tb_vecwork;          // [slots][5][rp] work vectors of the twisted factorisation
+  float* tb_At;                // short side <= 1024: the lower triangle in tile-major order (32 x 32 sub-tiles of 4 KB), the
+                               // working copy of the one-CTA-per-layer kernel
 };
 
 struct SpDecodeLayer {
@@ -120,6 +122,8 @@ void launch_ew_decode_average(const uint8_t* const* d_payloads, int n_payloads, 
 void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling
+void launch_sp_load_svd(const SpLayer* d_layers, int n_layers, const float* const* d_sigma, const float* const* d_vecs,
+                        cudaStream_t st);                                       // a decomposition given by the caller
 // one Jacobi step (global step index t) for every layer of the batch
 void launch_sp_jacobi_step(const SpLayer* d_layers, const TileRef* d_pairs, int n_pairs, int row_floats_max,
                            int t, int max_sweeps, float tol, cudaStream_t st);
@@ -141,7 +145,7 @@ int sp_tridiag_cluster_ctas();
 int sp_tridiag_ctas_of(int rp);                                   // CTAs a layer of padded short side rp takes
 int sp_configure_tridiag();                                       // co-resident clusters (0: route not available)
 int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_clusters, int rp_max, cudaStream_t st);  // cudaError_t
-void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, cudaStream_t st);
+void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, int64_t n_eigenvalues, cudaStream_t st);
 void launch_sp_eigvec(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st);
 // tridiagonal route for short sides above 512 (atomo_tridiag_big.cu)
 int sp_tridiag_big_max_r();

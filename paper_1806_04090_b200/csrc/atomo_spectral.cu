@@ -149,6 +149,27 @@ __global__ void __launch_bounds__(256) sp_scale_kernel(const SpLayer* __restrict
     for (int j = threadIdx.x; j < L.r; j += 256) L.A[(int64_t)i * lda + j] *= sc;
 }
 
+// A decomposition supplied by the caller (test entry point): lambda_i = sigma_i^2 in the eigenvalue slots (scale 1),
+// short-side vector i (rank-major input) in row i of X, which the caller zero-filled.
+__global__ void __launch_bounds__(256) sp_load_svd_kernel(const SpLayer* __restrict__ layers, const float* const* __restrict__ sigma,
+                                                          const float* const* __restrict__ vecs) {
+  const SpLayer& L = layers[blockIdx.x];
+  const float* sg = sigma[blockIdx.x];
+  const float* vv = vecs[blockIdx.x];
+  const int r = L.r;
+  if (blockIdx.y == 0) {
+    for (int i = threadIdx.x; i < r; i += 256) { const float x = sg[i]; L.lam[i] = x * x; }
+    if (threadIdx.x == 0) *L.scale = 1.0f;
+  }
+  for (int i = blockIdx.y; i < r; i += gridDim.y)
+    for (int j = threadIdx.x; j < r; j += 256) L.X[(int64_t)i * L.ldx + j] = vv[(int64_t)i * r + j];
+}
+
+void launch_sp_load_svd(const SpLayer* d_layers, int n_layers, const float* const* d_sigma, const float* const* d_vecs,
+                        cudaStream_t st) {
+  sp_load_svd_kernel<<<dim3(n_layers, 32), 256, 0, st>>>(d_layers, d_sigma, d_vecs);
+}
+
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st) {
   sp_trace_kernel<<<n_layers, 256, 0, st>>>(d_layers);
   sp_scale_kernel<<<dim3(n_layers, 32), 256, 0, st>>>(d_layers);
@@ -627,10 +648,21 @@ __global__ void __launch_bounds__(kDecThreads) sp_decode_kernel(const uint8_t* _
     while (na < kDecAtoms && p < n_payloads) {
       const uint8_t* payload = list ? list[p] : single;
       const atomo_payload_header* gh = reinterpret_cast<const atomo_payload_header*>(payload);
-      const atomo_layer_header* h = reinterpret_cast<const atomo_layer_header*>(payload + sizeof(atomo_payload_header)) + ref.layer;
-      const bool ok = gh->magic == ATOMO_MAGIC && gh->kind == ATOMO_KIND_SPECTRAL && h->rows == rows && h->cols == cols &&
-                      h->k <= h->k_cap;
-      if (!ok && a_next == 0 && ref.a == 0 && ref.b == 0 && threadIdx.x == 0)
+      // a payload normally comes from another rank: its header is checked before anything it points to is read.  The
+      // layer headers must exist (layer index below n_layers) and every array must lie inside total_bytes; a header
+      // that fails contributes zeros, and the status word is written only where it is known to be a status word
+      const bool has_hdr = gh->magic == ATOMO_MAGIC && (uint32_t)ref.layer < gh->n_layers &&
+                           sizeof(atomo_payload_header) + (uint64_t)gh->n_layers * sizeof(atomo_layer_header) <= gh->total_bytes;
+      const atomo_layer_header* h = reinterpret_cast<const atomo_layer_header*>(payload + sizeof(atomo_payload_header)) +
+                                    (has_hdr ? ref.layer : 0);
+      bool ok = has_hdr && gh->kind == ATOMO_KIND_SPECTRAL && h->rows == rows && h->cols == cols && h->k <= h->k_cap;
+      if (ok) {
+        const uint64_t kc = h->k_cap, tb = gh->total_bytes;
+        ok = h->off_idx <= tb && kc * 4 <= tb - h->off_idx && h->off_val <= tb && kc * 4 <= tb - h->off_val &&
+             h->off_short <= tb && kc * (uint64_t)r * 4 <= tb - h->off_short &&
+             h->off_long <= tb && kc * (uint64_t)len * 4 <= tb - h->off_long;
+      }
+      if (!ok && has_hdr && a_next == 0 && ref.a == 0 && ref.b == 0 && threadIdx.x == 0)
         raise_status(const_cast<atomo_layer_header*>(h), ATOMO_ERR_PAYLOAD);
       const uint32_t k = ok ? h->k : 0u;
       if (a_next >= k) { ++p; a_next = 0; continue; }

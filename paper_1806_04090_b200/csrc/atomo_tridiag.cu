@@ -349,11 +349,13 @@ __device__ __forceinline__ int sturm_count(const double* __restrict__ d, const d
 
 constexpr double kSturmPad = 1.0e6;    // diagonal entries past the end (the matrices are scaled to trace <= 1)
 constexpr int kBisThreads = 64;           // small CTAs: the warps of a large layer spread over all SMs (the recurrences are latency-bound)
-constexpr int kBisLanes = 8;          // points per round and eigenvalue: the interval shrinks 9 times per round
-constexpr int kBisRounds = 13;        // 9^13 = 2.5e12: interval width below 1e-12 of the spectrum's extent
-constexpr int kBisPerCta = kBisThreads / kBisLanes;
-
+// Points per round and eigenvalue (kBisLanes lanes work on one eigenvalue: the interval shrinks kBisLanes + 1 times per
+// round) and rounds, chosen so that the final interval is below 1e-12 of the spectrum's extent: 8 lanes and 13 rounds
+// (9^13 = 2.5e12) where the batch has few eigenvalues and the chain of rounds is what takes the time; 2 lanes and 26
+// rounds (3^26 = 2.5e12) where it has many: half the Sturm counts per eigenvalue, and enough eigenvalues to fill the GPU.
+template <int kBisLanes, int kBisRounds>
 __global__ void __launch_bounds__(kBisThreads) sp_bisect_kernel(const SpLayer* __restrict__ layers, int bis_stride) {
+  constexpr int kBisPerCta = kBisThreads / kBisLanes;
   const SpLayer& L = layers[blockIdx.y];
   if (!L.tri) return;
   const int r = L.r;
@@ -589,7 +591,8 @@ int sp_configure_tridiag() {
   if (cudaFuncSetAttribute(sp_tridiag_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri_smem_bytes(kTriMaxRp)) != cudaSuccess ||
       cudaFuncSetAttribute(sp_tridiag_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
       cudaFuncSetAttribute(sp_eigvec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vec_smem_bytes(kTriMaxRp)) != cudaSuccess ||
-      cudaFuncSetAttribute(sp_bisect_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (kMaxShort + 10) * sizeof(double))) != cudaSuccess) {
+      cudaFuncSetAttribute(sp_bisect_kernel<8, 13>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (kMaxShort + 10) * sizeof(double))) != cudaSuccess ||
+      cudaFuncSetAttribute(sp_bisect_kernel<2, 26>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (kMaxShort + 10) * sizeof(double))) != cudaSuccess) {
     cudaGetLastError();
     return 0;
   }
@@ -615,9 +618,16 @@ int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_c
   return (int)cudaLaunchKernelEx(&cfg, sp_tridiag_cluster_kernel, d_layers, d_ctas);
 }
 
-void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, cudaStream_t st) {
+void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, int64_t n_eigenvalues, cudaStream_t st) {
   const int stride = (r_max + 8 + 1) & ~1;
-  sp_bisect_kernel<<<dim3((r_max + kBisPerCta - 1) / kBisPerCta, n_layers), kBisThreads, 2 * (size_t)stride * sizeof(double), st>>>(d_layers, stride);
+  const size_t smem = 2 * (size_t)stride * sizeof(double);
+  if (n_eigenvalues >= 16384) {
+    constexpr int per = kBisThreads / 2;
+    sp_bisect_kernel<2, 26><<<dim3((r_max + per - 1) / per, n_layers), kBisThreads, smem, st>>>(d_layers, stride);
+  } else {
+    constexpr int per = kBisThreads / 8;
+    sp_bisect_kernel<8, 13><<<dim3((r_max + per - 1) / per, n_layers), kBisThreads, smem, st>>>(d_layers, stride);
+  }
 }
 
 void launch_sp_eigvec(const SpLayer* d_layers, int n_layers, int rp_max, cudaStream_t st) {

@@ -33,6 +33,15 @@
 
 namespace cg = cooperative_groups;
 
+// development builds (-DTB_PROFILE) stamp the phases of the reduction kernels with clock64 and print the sums
+#ifdef TB_PROFILE
+#define TB_PROF_DECL long long tp[6] = {0, 0, 0, 0, 0, 0}, tl = clock64();
+#define TB_MARK(k) { const long long now = clock64(); tp[k] += now - tl; tl = now; }
+#else
+#define TB_PROF_DECL
+#define TB_MARK(k)
+#endif
+
 namespace atomo {
 
 namespace {
@@ -144,12 +153,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   for (int i = tid; i < r4; i += kTbThreads) s_u[i] = (T)0;
   if (C > 1) cluster.sync();                                                   // every CTA runs: remote stores may start
 
-#ifdef TB_PROFILE
-  long long tp[6] = {0, 0, 0, 0, 0, 0}, tl = clock64();
-#define TB_MARK(k) { const long long now = clock64(); tp[k] += now - tl; tl = now; }
-#else
-#define TB_MARK(k)
-#endif
+  TB_PROF_DECL
   const int n_ref = r - 2;                                                     // reflectors: columns 0 .. r-3
   for (int c = 0; c < r; ++c) {
     const int p0 = c / kTbNB * kTbNB;
@@ -398,6 +402,345 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   if (C > 1) cluster.sync();                                                   // nobody leaves while a peer may still write here
 }
 
+// ---- one CTA per layer (short side up to 1024) -------------------------------------------------------------------
+// The form a large batch takes (config 5: 96 layers of 1024 rows, one SM each).  Differences from the cluster
+// kernel above, all of them about bytes:
+//   * only the lower triangle of A0 is read and updated.  The product y = A0 u goes over 64 x 64 tiles of the
+//     triangle, one warp per tile: a tile contributes its rows' sums to block I of y and, transposed, its columns'
+//     sums to block J, both into a table of partial vectors in shared memory (slot J of block I, slot I of block J:
+//     every slot has one writer), which the row owners add up in ascending slot order.  Per 32 x 32 sub-tile a lane
+//     holds 8 x 4 entries; the sums over the 8 lanes of a row and the 4 lanes of a column are reduce-scatters (7 + 3
+//     shuffles).  Half the bytes per step of the row-wise product.
+//   * the panel (16 columns: u_t and w_t of all rows) lives in shared memory, so the column update, the correction
+//     of y and the panel dots never leave the SM, and the rank-32 update at the end of a panel takes its operands
+//     from there (4 x 4 outputs per thread on 128 x 128 tiles of the lower triangle).
+//   * thread g owns row g for the whole reduction.
+namespace {
+
+constexpr int kT1NB = 16;                    // columns per panel
+constexpr int kT1MaxR = 1024;
+constexpr int kT1Blk = 64;                   // tile edge of the matrix-vector product
+constexpr int kT1MaxB = kT1MaxR / kT1Blk;    // 16 blocks
+
+struct alignas(16) T1Shared {
+  double part_a[32];
+  double part_k[32];
+  double dots[2 * kT1NB];
+  double x0;
+  double pad;
+};
+
+// The kernel works on a copy of the lower triangle in tile-major order: 32 x 32 sub-tile (I, J), J <= I, is the
+// contiguous 4 KB block number I (I + 1) / 2 + J, row-major inside.  A warp then reads a sub-tile as one contiguous
+// piece of memory (with rows of the row-major matrix it would be 32 pieces of 128 bytes, 4 KB apart, which DRAM
+// serves at little more than half its streaming rate).  Rows and columns from r on are zero.
+__device__ __forceinline__ float* t1_sub(float* At, int I, int J) { return At + ((size_t)(I * (I + 1) / 2 + J) << 10); }
+
+// sum over the 8 lanes lx = lane % 8 of v[k]: lane lx ends with the total of k = lx
+__device__ __forceinline__ float rs8(float (&v)[8], int lane) {
+  const bool b4 = lane & 4, b2 = lane & 2, b1 = lane & 1;
+  float a[4];
+#pragma unroll
+  for (int m = 0; m < 4; ++m) {
+    const float send = b4 ? v[m] : v[m + 4], keep = b4 ? v[m + 4] : v[m];
+    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  float b[2];
+#pragma unroll
+  for (int m = 0; m < 2; ++m) {
+    const float send = b2 ? a[m] : a[m + 2], keep = b2 ? a[m + 2] : a[m];
+    b[m] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+  }
+  const float send = b1 ? b[0] : b[1], keep = b1 ? b[1] : b[0];
+  return keep + __shfl_xor_sync(0xffffffffu, send, 1);
+}
+// sum over the 4 lanes ly = lane / 8 of v[j]: lane ly ends with the total of j = ly
+__device__ __forceinline__ float rs4(float (&v)[4], int lane) {
+  const bool b2 = lane & 16, b1 = lane & 8;
+  float a[2];
+#pragma unroll
+  for (int m = 0; m < 2; ++m) {
+    const float send = b2 ? v[m] : v[m + 2], keep = b2 ? v[m + 2] : v[m];
+    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+  }
+  const float send = b1 ? a[0] : a[1], keep = b1 ? a[1] : a[0];
+  return keep + __shfl_xor_sync(0xffffffffu, send, 8);
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const SpLayer* __restrict__ layers,
+                                                                        const int* __restrict__ big_layers) {
+  extern __shared__ __align__(16) unsigned char tb_smem[];
+  T1Shared& S = *reinterpret_cast<T1Shared*>(tb_smem);
+  float* const s_u = reinterpret_cast<float*>(tb_smem + sizeof(T1Shared));     // [1024] current reflector (zero up to c and from r on)
+  float* const pan_u = s_u + kT1MaxR;                                          // [16][1024]
+  float* const pan_w = pan_u + kT1NB * kT1MaxR;                                // [16][1024]
+  float* const y_part = pan_w + kT1NB * kT1MaxR;                               // [16 blocks][16 slots][64]
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const SpLayer& L = layers[big_layers[blockIdx.x]];
+  const int r = L.r;
+  const int64_t lda = L.lda;
+  float* const A = reinterpret_cast<float*>(L.tb_A);
+  float* const V = L.td_V;
+  const int64_t ldv = L.td_ldv;
+  double* const td_d = L.td_d;
+  double* const td_e = L.td_e;
+  const int nblk = (r + 31) / 32;
+  const int nb64 = (r + kT1Blk - 1) / kT1Blk;
+  const int r4 = (r + 3) & ~3;
+  const int g = tid;
+  const bool valid = g < r;
+  const int ly = lane >> 3, lx = lane & 7;                                     // sub-tile layout: rows 4 k + ly, columns 4 lx .. 4 lx + 3
+  const int idx = 4 * lx + ly;                                                 // the row / column a lane ends up with after the reduce-scatters
+
+  float* const At = L.tb_At;
+  s_u[tid] = 0.0f;
+  // the lower triangle of A into tile-major order (one warp per sub-tile: 32 rows of 128 bytes in, 4 KB out)
+  for (int k = w; k < nblk * (nblk + 1) / 2; k += kTbWarps) {
+    int I = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);
+    while ((I + 1) * (I + 2) / 2 <= k) ++I;
+    while (I * (I + 1) / 2 > k) --I;
+    const int J = k - I * (I + 1) / 2;
+    float* dst = At + ((size_t)k << 10);
+    const int col = 32 * J + lane;
+#pragma unroll 8
+    for (int rr = 0; rr < 32; ++rr) {
+      const int row = 32 * I + rr;
+      dst[rr * 32 + lane] = (row < r && col < r) ? __ldcg(A + (int64_t)row * lda + col) : 0.0f;
+    }
+  }
+  __threadfence_block();
+  __syncthreads();
+  const int n_ref = r - 2;
+  TB_PROF_DECL
+  // element (row, col) of the working copy, col <= row
+  auto at = [&](int row, int col) -> float* { return t1_sub(At, row >> 5, col >> 5) + ((row & 31) << 5) + (col & 31); };
+  float a_pref = valid ? __ldcg(at(g, 0)) : 0.0f;                              // column 0 of row g (lower triangle: g >= 0)
+  for (int c = 0; c < r; ++c) {
+    const int p0 = c / kT1NB * kT1NB;
+    const int i = c < n_ref ? c - p0 : 0;
+    // ---- column c as the earlier reflectors of the panel left it ----
+    double a = 0.0;
+    if (valid && g >= c) {
+      a = (double)a_pref;
+      for (int t = 0; t < i; ++t)
+        a -= (double)pan_u[t * kT1MaxR + g] * (double)pan_w[t * kT1MaxR + c] + (double)pan_w[t * kT1MaxR + g] * (double)pan_u[t * kT1MaxR + c];
+      if (g == c) td_d[c] = a;
+    }
+    if (c >= n_ref) {
+      if (c == r - 2 && valid && g == r - 1) td_e[c] = a;
+      if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;
+      continue;
+    }
+    const bool live = valid && g > c;
+    {
+      const double sq = warp_sum(live ? a * a : 0.0);
+      if (lane == 0) S.part_a[w] = sq;
+      if (g == c + 1) S.x0 = a;
+    }
+    __syncthreads();
+    const double nx2 = tb_ordered_sum(S.part_a, nblk, lane);
+    const double x0 = S.x0;
+    double alpha = 0.0, inv = 0.0;
+    if (nx2 > 1.0e-290) {
+      const double nx = sqrt(nx2);
+      alpha = -copysign(nx, x0);
+      inv = rsqrt(2.0 * nx * (nx + fabs(x0)));
+    }
+    float u_f = 0.0f;
+    if (valid) {
+      if (live) u_f = (float)((a - (g == c + 1 ? alpha : 0.0)) * inv);
+      V[(int64_t)c * ldv + g] = u_f;
+      if (g == c + 1) td_e[c] = alpha;
+      s_u[g] = u_f;
+      pan_u[i * kT1MaxR + g] = u_f;
+    }
+    const double u_own = (double)u_f;
+    __syncthreads();
+    TB_MARK(1)
+    // ---- panel dots (one warp each), then y = A0 u over the tiles of the lower triangle ----
+    if (w < 2 * i) {
+      const int t = w >> 1;
+      const float* x = (w & 1) ? pan_u + t * kT1MaxR : pan_w + t * kT1MaxR;   // odd: b_t = u_t^T u, even: a_t = w_t^T u
+      double acc = 0.0;
+      for (int h = lane; h < r; h += 32) acc = fma((double)x[h], (double)s_u[h], acc);
+      acc = warp_sum(acc);
+      if (lane == 0) S.dots[w] = acc;
+    }
+    {
+      // One warp per 64 x 64 tile (I, J), J <= I, of the live part of the lower triangle, as up to four 32 x 32
+      // sub-tiles.  In a sub-tile a lane holds rows 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3.  Row sums
+      // are accumulated over the two sub-tiles of a row half before the eight lanes of a row are added up
+      // (reduce-scatter: lane 8 ly + lx ends with row 8 ly + lx), column sums over the two sub-tiles of a column half
+      // before the four lanes of a column are (lane ends with column 4 lx + ly).  The tile's sums go to slot J of
+      // block I (rows) and slot I of block J (columns): every slot has exactly one writer per step.
+      // (Tried and dropped: refilling each register group from the warp's next sub-tile as soon as it has been
+      // multiplied -- the extra live state spilled and the product took 2.7 times as long; 32 x 32 work units with
+      // order-free shared-memory adds -- no faster.)
+      const int j0 = (c + 1) / kT1Blk;                                         // first live block
+      const int nbl = nb64 - j0;
+      const int n_tiles = nbl * (nbl + 1) / 2;
+      for (int k = w; k < n_tiles; k += kTbWarps) {
+        int ii = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);
+        while ((ii + 1) * (ii + 2) / 2 <= k) ++ii;
+        while (ii * (ii + 1) / 2 > k) --ii;
+        const int I = j0 + ii, J = j0 + (k - ii * (ii + 1) / 2);
+        float racc[2] = {0.f, 0.f};
+        uint64_t cp[2][2] = {{pack2(0.f, 0.f), pack2(0.f, 0.f)}, {pack2(0.f, 0.f), pack2(0.f, 0.f)}};   // [column half][pair of columns]
+#pragma unroll
+        for (int sa = 0; sa < 2; ++sa) {
+          const int row0 = kT1Blk * I + 32 * sa;
+          if (row0 >= r) continue;
+          float rp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+          const float4 ui0 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly);
+          const float4 ui1 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly + 4);
+          const float uiv[8] = {ui0.x, ui0.y, ui0.z, ui0.w, ui1.x, ui1.y, ui1.z, ui1.w};
+#pragma unroll
+          for (int sb = 0; sb < 2; ++sb) {
+            if (I == J && sb > sa) continue;                                   // above the diagonal
+            const int col0 = kT1Blk * J + 32 * sb;
+            const bool diag = row0 == col0;
+            float4 t[8];
+            {
+              const float* src = t1_sub(At, row0 >> 5, col0 >> 5) + (8 * ly) * 32 + 4 * lx;
+#pragma unroll
+              for (int kk = 0; kk < 8; ++kk) t[kk] = ldcg4(src + kk * 32);
+            }
+            const float4 uj = *reinterpret_cast<const float4*>(s_u + col0 + 4 * lx);
+            const uint64_t uj01 = pack2(uj.x, uj.y), uj23 = pack2(uj.z, uj.w);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+              float4 v = t[kk];
+              const int rr = 8 * ly + kk, cc = 4 * lx;                         // position inside the sub-tile
+              if (diag) {                                                      // lower triangle only
+                if (cc + 0 > rr) v.x = 0.f;
+                if (cc + 1 > rr) v.y = 0.f;
+                if (cc + 2 > rr) v.z = 0.f;
+                if (cc + 3 > rr) v.w = 0.f;
+              }
+              float s0, s1;
+              unpack2(fma2(pack2(v.z, v.w), uj23, fma2(pack2(v.x, v.y), uj01, pack2(0.f, 0.f))), s0, s1);
+              rp[kk] += s0 + s1;
+              if (diag) {                                                      // the diagonal entry counts once (with the rows)
+                if (cc + 0 == rr) v.x = 0.f;
+                if (cc + 1 == rr) v.y = 0.f;
+                if (cc + 2 == rr) v.z = 0.f;
+                if (cc + 3 == rr) v.w = 0.f;
+              }
+              const uint64_t ui2 = pack2(uiv[kk], uiv[kk]);
+              cp[sb][0] = fma2(pack2(v.x, v.y), ui2, cp[sb][0]);
+              cp[sb][1] = fma2(pack2(v.z, v.w), ui2, cp[sb][1]);
+            }
+          }
+          racc[sa] = rs8(rp, lane);
+        }
+        float cacc[2];
+#pragma unroll
+        for (int sb = 0; sb < 2; ++sb) {
+          float cv[4];
+          unpack2(cp[sb][0], cv[0], cv[1]); unpack2(cp[sb][1], cv[2], cv[3]);
+          cacc[sb] = rs4(cv, lane);
+        }
+        float* yi = y_part + ((size_t)I * kT1MaxB + J) * kT1Blk;
+        if (I == J) {
+          // rows and columns of the same block: a column's sum moves to the lane that holds the row of the same index
+          const int from = ((lane & 3) << 3) | (lane >> 2);
+          yi[lane] = racc[0] + __shfl_sync(0xffffffffu, cacc[0], from);
+          yi[32 + lane] = racc[1] + __shfl_sync(0xffffffffu, cacc[1], from);
+        } else {
+          yi[lane] = racc[0]; yi[32 + lane] = racc[1];
+          float* yj = y_part + ((size_t)J * kT1MaxB + I) * kT1Blk;
+          yj[idx] = cacc[0]; yj[32 + idx] = cacc[1];
+        }
+      }
+    }
+    __syncthreads();
+    TB_MARK(2)
+    // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
+    double p = 0.0;
+    double ysum = 0.0;
+    if (live) {                                                                // this row's partial sums in ascending slot order
+      const int j0 = (c + 1) / kT1Blk;
+      const float* yp = y_part + (size_t)(g / kT1Blk) * kT1MaxB * kT1Blk + (g % kT1Blk);
+      for (int sl = j0; sl < nb64; ++sl) ysum += (double)yp[sl * kT1Blk];
+    }
+    if (live) {
+      double y = ysum;
+      for (int t = 0; t < i; ++t)
+        y -= (double)pan_u[t * kT1MaxR + g] * S.dots[2 * t] + (double)pan_w[t * kT1MaxR + g] * S.dots[2 * t + 1];
+      p = 2.0 * y;
+    }
+    {
+      const double kp = warp_sum(u_own * p);
+      if (lane == 0) S.part_k[w] = kp;
+    }
+    if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;   // next column, in flight over the barrier
+    __syncthreads();
+    const double K = tb_ordered_sum(S.part_k, nblk, lane);
+    if (valid) pan_w[i * kT1MaxR + g] = (float)(live ? p - K * u_own : 0.0);
+    const bool flush = (i == kT1NB - 1) || (c == n_ref - 1);
+    __syncthreads();
+    TB_MARK(4)
+    if (!flush) continue;
+    // ---- end of the panel: the lower triangle of A0 -= U W^T + W U^T on rows and columns beyond c ----
+    {
+      const int nr = i + 1, g0 = c + 1;
+      const int wr = w >> 3, wc = w & 7;
+      const int qy = lane >> 2, qx = lane & 3;
+      const int b0 = g0 / 128, nb128 = (r + 127) / 128;
+      for (int RI = b0; RI < nb128; ++RI) {
+        for (int CJ = b0; CJ <= RI; ++CJ) {
+          const int row0 = 128 * RI + 32 * wr + 4 * qy, col0 = 128 * CJ + 16 * wc + 4 * qx;
+          if (col0 > row0 + 3 || row0 >= r) continue;                          // this thread's 4 x 4 lies above the diagonal or below the matrix
+          float acc[4][4];
+#pragma unroll
+          for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+          for (int t = 0; t < nr; ++t) {
+            const float4 ru = *reinterpret_cast<const float4*>(pan_u + t * kT1MaxR + row0);
+            const float4 rw = *reinterpret_cast<const float4*>(pan_w + t * kT1MaxR + row0);
+            const float4 cu = *reinterpret_cast<const float4*>(pan_u + t * kT1MaxR + col0);
+            const float4 cw = *reinterpret_cast<const float4*>(pan_w + t * kT1MaxR + col0);
+            const float rux[4] = {ru.x, ru.y, ru.z, ru.w}, rwx[4] = {rw.x, rw.y, rw.z, rw.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              acc[x][0] = fmaf(rux[x], cw.x, acc[x][0]); acc[x][1] = fmaf(rux[x], cw.y, acc[x][1]);
+              acc[x][2] = fmaf(rux[x], cw.z, acc[x][2]); acc[x][3] = fmaf(rux[x], cw.w, acc[x][3]);
+              acc[x][0] = fmaf(rwx[x], cu.x, acc[x][0]); acc[x][1] = fmaf(rwx[x], cu.y, acc[x][1]);
+              acc[x][2] = fmaf(rwx[x], cu.z, acc[x][2]); acc[x][3] = fmaf(rwx[x], cu.w, acc[x][3]);
+            }
+          }
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            const int gr = row0 + x;
+            if (gr >= r || gr < g0) continue;
+            if (col0 > gr) continue;
+            float* dst = at(gr, col0);                                         // four columns of one sub-tile row
+            if (col0 >= g0 && col0 + 3 <= gr) {                                // four live entries of the lower triangle
+              float4 o = ldcg4(dst);
+              o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
+              st4(dst, o);
+            } else {
+#pragma unroll
+              for (int y = 0; y < 4; ++y) if (col0 + y >= g0 && col0 + y <= gr) dst[y] = __ldcg(dst + y) - acc[x][y];
+            }
+          }
+        }
+      }
+    }
+    __threadfence_block();
+    __syncthreads();
+    if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;   // the update changed it
+    TB_MARK(5)
+  }
+#ifdef TB_PROFILE
+  if (blockIdx.x == 0 && tid == 0)
+    printf("tridiag_big1 r=%d cycles: column+reflector %lld matvec+dots %lld w %lld gemm %lld\n", r, tp[1], tp[2], tp[4], tp[5]);
+#endif
+}
+
 // ---- vectors of the kept atoms ------------------------------------------------------------------------------------
 namespace {
 constexpr int kVbThreads = 128;
@@ -530,6 +873,9 @@ template <typename T> size_t tb_smem_bytes(int r_max) {
   const size_t r4 = (size_t)((r_max + 3) & ~3);
   return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128) * sizeof(T);
 }
+size_t t1_smem_bytes() {
+  return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + (size_t)kT1MaxB * kT1MaxB * kT1Blk);
+}
 size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbWarps * sizeof(float)); }
 
 template <typename T, int C> int tb_configure_one() {
@@ -565,6 +911,7 @@ int sp_configure_tridiag_big() {
          tb_configure_one<float, 8>() | tb_configure_one<float, 16>();
   bad |= tb_configure_one<double, 1>() | tb_configure_one<double, 2>() | tb_configure_one<double, 4>() |
          tb_configure_one<double, 8>() | tb_configure_one<double, 16>();
+  bad |= cudaFuncSetAttribute(sp_tridiag_big1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t1_smem_bytes()) != cudaSuccess;
   bad |= cudaFuncSetAttribute(sp_eigvec_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vb_smem_bytes(kTbMaxR)) != cudaSuccess;
   if (bad) cudaGetLastError();
   return bad;
@@ -573,6 +920,10 @@ int sp_configure_tridiag_big() {
 // d_big: n_big layer indices, all stored as fp32 (fp64 = 0) or all as fp64; ctas = CTAs per layer (1, 2, 4, 8, 16)
 int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, int ctas, int fp64, cudaStream_t st) {
   if (n_big <= 0) return 0;
+  if (ctas == 1 && !fp64 && r_max <= kT1MaxR) {               // one CTA per layer: the triangle-only kernel
+    sp_tridiag_big1_kernel<<<n_big, kTbThreads, t1_smem_bytes(), st>>>(d_layers, d_big);
+    return (int)cudaGetLastError();
+  }
 #define TB_CASE(CC) case CC: return fp64 ? tb_launch_one<double, CC>(d_layers, d_big, n_big, r_max, st) \
                                          : tb_launch_one<float, CC>(d_layers, d_big, n_big, r_max, st);
   switch (ctas) { TB_CASE(1) TB_CASE(2) TB_CASE(4) TB_CASE(8) TB_CASE(16) default: return (int)cudaErrorInvalidValue; }

@@ -1,6 +1,6 @@
 """Shared checks for the GPU parity tests: CUDA path (through the C ABI) vs the fp64 oracle.
 
-Bars (from the benchmark spec of this build): masks and packed indices bit-exact except for
+Bars: masks and packed indices bit-exact except for
 draws within 1e-6 of their probability (counted and reported); singular values, probabilities
 and decoded gradients within 1e-4 relative l2 / Frobenius error.
 """
@@ -15,7 +15,14 @@ CARVE = 1e-6            # |u_i - p_i| below this: the draw is excluded from bit-
 RESID_GRAM = 6e-7       # eigen-residual bar of the fp32 Gram route, in units of lambda_1 = sigma_1^2:
                         # twice the Jacobi rotation threshold (3e-7), i.e. about 10 ulp of fp32
 GAP_MIN = 1e-3          # an atom's rank-one term is comparable across two SVDs only if
-                        # min_j |sigma_i^2 - sigma_j^2| >= GAP_MIN * sigma_1^2 (well-conditioned)
+                        # min_j |sigma_i^2 - sigma_j^2| >= GAP_MIN * sigma_1^2 (well-conditioned).  The bound is the
+                        # Gram matrix's, not the eigen-solver's: A = G G^T is stored in fp32, a perturbation E of
+                        # about 1e-7 lambda_1, and an eigenvector moves by ||E|| / gap; 1e-7 / 1e-3 = 1e-4 is the
+                        # bar for the decoded gradient.  Every test prints the largest (term error x gap) it saw.
+
+# what the spectral checks of this session have compared so far (printed and asserted by the tests)
+TALLY = {"layers": 0, "masks_identical": 0, "kept_atoms": 0, "certified_atoms": 0, "terms_compared": 0,
+         "decodes_compared": 0, "worst_err_times_gap": 0.0}
 
 
 def rel(a, b):
@@ -51,7 +58,10 @@ def check_entrywise(A, oracle, g_np, g_dev, s, seed, step, layer_arrays, hdr, db
     same = check_masks(m, enc, report, tag)
     assert hdr.k == int(m.sum())
     assert np.array_equal(layer_arrays["idx"], np.flatnonzero(m).astype(np.uint32)), f"{tag}: packed indices"
-    assert hdr.n_sat == enc["n_s"] or abs(int(hdr.n_sat) - enc["n_s"]) <= np.count_nonzero(enc["p"] == 1.0)
+    # saturated atoms: the same count, except that atoms sitting exactly on the boundary |lambda_i| (s - n_s) = tail
+    # (p_i = 1 on either branch of Algorithm 1) may be counted on either side
+    ties = int(np.count_nonzero(enc["p"] == 1.0)) - enc["n_s"]
+    assert enc["n_s"] <= int(hdr.n_sat) <= enc["n_s"] + max(ties, 0), f"{tag}: n_sat {hdr.n_sat} vs {enc['n_s']} (+{ties} ties)"
     assert abs(hdr.l1 - np.abs(g_np.astype(np.float64)).sum()) <= 1e-7 * max(hdr.l1, 1e-300)
     # values: g_i / p_i with the oracle's p
     idx = layer_arrays["idx"].astype(np.int64)
@@ -106,19 +116,34 @@ def check_spectral_layer(oracle, G, enc, hdr, arr, dbg, l, out_gpu, report, tag,
         assert rel(out_gpu, own) <= 1e-5, f"{tag}: decode kernel {rel(out_gpu, own)}"
     else:
         assert not out_gpu.any()
-    # P7 end to end vs the oracle's own encode + decode, where the kept atoms are well conditioned
+    # P7 end to end vs the oracle's own encode + decode.  Per kept atom: its rank-one term against the oracle's
+    # where the atom is well conditioned (certified); the whole decoded gradient where every kept atom is.
     e2e = None
+    TALLY["layers"] += 1
     if same:
+        TALLY["masks_identical"] += 1
         ref = oracle.decode_spectral(enc["coef"], enc["U_S"], enc["V_S"])
+        ref_norm = max(np.linalg.norm(ref), 1e-300)
         e2e = rel(out_gpu, ref) if k else 0.0
         lam = enc["sigma"] ** 2
-        ok = True
-        for i in arr["idx"]:
+        all_ok = True
+        for j, i in enumerate(arr["idx"]):
             others = np.delete(lam, i)
             gap = np.min(np.abs(others - lam[i])) / lam[0] if others.size else 1.0
-            ok &= gap >= GAP_MIN
-        report.append(f"{tag}: k={k} end-to-end rel Frobenius {e2e:.2e} ({'certified' if ok else 'ill-conditioned atoms'})")
-        if ok and check_vectors:
+            ok = gap >= GAP_MIN
+            all_ok &= ok
+            TALLY["kept_atoms"] += 1
+            term = float(arr["coef"][j]) * np.outer(arr["U"][:, j].astype(np.float64), arr["V"][:, j].astype(np.float64))
+            term_ref = float(enc["coef"][j]) * np.outer(enc["U_S"][:, j], enc["V_S"][:, j])
+            err = np.linalg.norm(term - term_ref) / ref_norm
+            TALLY["worst_err_times_gap"] = max(TALLY["worst_err_times_gap"], float(err * gap))
+            if ok and check_vectors:
+                TALLY["certified_atoms"] += 1
+                TALLY["terms_compared"] += 1
+                assert err <= REL_TOL, f"{tag}: kept atom {j} (rank {i}, gap {gap:.1e}): term error {err:.2e}"
+        report.append(f"{tag}: k={k} end-to-end rel Frobenius {e2e:.2e} ({'certified' if all_ok else 'ill-conditioned atoms'})")
+        if all_ok and check_vectors:
+            TALLY["decodes_compared"] += 1
             assert e2e <= REL_TOL, f"{tag}: end-to-end {e2e}"
     return same, e2e
 

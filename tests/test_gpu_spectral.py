@@ -260,7 +260,12 @@ def test_unbiased_on_gpu(atomo):
 def test_config2_full(atomo, oracle):
     # the benchmark workload: all 18 ResNet-18-shaped layers in one batched call, s = 2
     mats = synth.c2_resnet18(0)
+    before = dict(parity.TALLY)
     _run(atomo, oracle, mats, 2.0, seed=2024, step=1)
+    t = parity.TALLY
+    print({k: (t[k] - before[k] if k != "worst_err_times_gap" else t[k]) for k in t})
+    assert t["masks_identical"] - before["masks_identical"] == len(mats)
+    assert t["terms_compared"] - before["terms_compared"] >= len(mats) // 2
 
 
 def test_config5_shape_properties(atomo):

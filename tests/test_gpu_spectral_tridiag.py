@@ -150,7 +150,13 @@ def test_paper_reshape_family(atomo, oracle):
 
 def test_config2_full(atomo, oracle):
     mats = synth.c2_resnet18(0)
+    before = dict(parity.TALLY)
     _run(atomo, oracle, mats, 2.0, seed=2024, step=1)
+    # the end-to-end bar was really applied: some kept atoms were certified and compared term by term
+    t = parity.TALLY
+    print({k: (t[k] - before[k] if k != "worst_err_times_gap" else t[k]) for k in t})
+    assert t["masks_identical"] - before["masks_identical"] == len(mats)
+    assert t["terms_compared"] - before["terms_compared"] >= len(mats) // 2
 
 
 def test_routes_agree(atomo):
@@ -178,10 +184,13 @@ def test_deterministic_and_fallback(atomo):
     assert a1["k"] == a2["k"] > 0
     for key in ("idx", "coef", "U", "V"):
         assert np.array_equal(a1[key], a2[key]), key
-    # a layer with a short side above 512 sends the whole batch to the Jacobi routes
+    # a request for the whole short-side basis sends the batch to the Jacobi routes (a layer with a short side above
+    # 512 no longer does: it takes the blocked reduction inside the same call)
     big = np.random.default_rng(1).standard_normal((600, 700)).astype(np.float32)
     t = [torch.from_numpy(G[0]).cuda(), torch.from_numpy(big).cuda()]
     pay, _ = atomo.atomo_encode_spectral(t, 2.0, seed=9)
+    assert atomo.last_eig_scheme() == TRIDIAG and atomo.payload_status(pay)[0] == 0
+    pay, _ = atomo.atomo_encode_spectral(t, 2.0, seed=9, debug=True, debug_short=True)
     assert atomo.last_eig_scheme() in (1, 2) and atomo.payload_status(pay)[0] == 0
     # non-finite input: reported, nothing kept
     bad = G[0].copy(); bad[3, 7] = np.nan

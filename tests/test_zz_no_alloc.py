@@ -44,14 +44,20 @@ def test_static_decode_rejects_oversized_batches():
     a = api.Atomo(0)
     G = torch.from_numpy(synth.c1_spectral(0)).cuda()
     pay, _ = a.atomo_encode_spectral([G], 2.0, seed=1, k_cap=8)
-    # more layers than the fixed table holds
+    # more layers than the fixed table holds (every output is a real 64 x 64 buffer: nothing depends on the refusal)
     big = api.Payload(pay.buf, api.KIND_SPECTRAL, [(64, 64)] * 65, 8, a)
     with pytest.raises(api.AtomoError) as e:
-        api.atomo_decode_spectral_static(big, [torch.empty(64, 64, device="cuda")] * 65)
+        api.atomo_decode_spectral_static(big, [torch.empty(64, 64, device="cuda") for _ in range(65)])
     assert e.value.code == 3
-    # more output tiles than the fixed table holds (8192 tiles of 64 x 1024 elements)
-    huge = api.Payload(pay.buf, api.KIND_SPECTRAL, [(64 * 8193, 256)], 8, a)
+    # more output tiles than the fixed table holds: 8193 row tiles of 64 x 1024, in a buffer of the full size (2 MB)
+    huge = api.Payload(pay.buf, api.KIND_SPECTRAL, [(64 * 8193, 1)], 8, a)
     with pytest.raises(api.AtomoError) as e:
-        api.atomo_decode_spectral_static(huge, [torch.empty(1, device="cuda")])
+        api.atomo_decode_spectral_static(huge, [torch.empty(64 * 8193, 1, device="cuda")])
     assert e.value.code == 3
+    # the binding refuses outputs that are too short, strided, of another type or on the host before the C call
+    ok = api.Payload(pay.buf, api.KIND_SPECTRAL, [(64, 64)], 8, a)
+    for bad in (torch.empty(1, device="cuda"), torch.empty(64, 128, device="cuda")[:, ::2],
+                torch.empty(64, 64, device="cuda", dtype=torch.float64), torch.empty(64, 64)):
+        with pytest.raises(ValueError):
+            api.atomo_decode_spectral_static(ok, [bad])
     a.close()
