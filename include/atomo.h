@@ -248,6 +248,13 @@ int atomo_payload_read_headers(atomo_ctx* ctx, const void* payload /*DEVICE*/, i
 int atomo_payload_status(atomo_ctx* ctx, const void* payload /*DEVICE*/, int32_t n_layers,
                          int32_t* worst /*HOST*/, int32_t* first_bad_layer /*HOST*/, void* stream);
 
+/* Descriptor tables (layer descriptors, tile lists, tensor maps, header templates) are kept in device buffers owned by
+ * the context and uploaded only when they differ from the previous call's: a loop that calls with the same pointers
+ * and shapes every step issues no host-to-device copy in steady state (the payload header travels as a kernel
+ * argument).  Counts since atomo_create: calls that had to upload their tables, and calls that found them in place.
+ * Host only; either pointer may be NULL.                                                              */
+int atomo_get_table_uploads(atomo_ctx* ctx, int64_t* uploads /*HOST*/, int64_t* reuses /*HOST*/);
+
 /* --- profiling ------------------------------------------------------------------------------ */
 int atomo_set_profiling(atomo_ctx* ctx, int enabled);
 /* ms[ATOMO_N_STAGES], launches[ATOMO_N_STAGES] for the last encode/decode call (synchronises). */

@@ -32,7 +32,7 @@ EXPORTS = [
     "atomo_payload_read_headers", "atomo_payload_status", "atomo_set_profiling", "atomo_get_stage_times",
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
-    "atomo_set_tridiag_ctas", "atomo_measure_fma_peak", "atomo_encode_spectral_from_svd",
+    "atomo_set_tridiag_ctas", "atomo_measure_fma_peak", "atomo_encode_spectral_from_svd", "atomo_get_table_uploads",
 ]
 
 
@@ -116,6 +116,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_set_persistent_eig.argtypes = [vp, i32]
     lib.atomo_last_eig_scheme.argtypes = [vp]
     lib.atomo_set_tridiag_ctas.argtypes = [vp, i32]
+    lib.atomo_get_table_uploads.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.atomo_encode_spectral_from_svd.argtypes = [vp, ctypes.POINTER(_Mat), i32, ctypes.POINTER(vp), ctypes.POINTER(vp),
                                                    ctypes.c_double, u64, u64, i32, vp, i64, ctypes.POINTER(_Debug), vp]
     lib.atomo_measure_fma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.POINTER(ctypes.c_double)]
@@ -537,6 +538,12 @@ class Atomo:
         explicit values only for the atoms with p = 1, of which at most sat_cap per vector)."""
         self._check(self.lib.atomo_set_entrywise_format(self._h, int(fmt), int(sat_cap)), "atomo_set_entrywise_format")
         self._ew_format, self._ew_sat_cap = int(fmt), (int(sat_cap) if int(fmt) == EW_COMPACT else 0)
+
+    def table_uploads(self):
+        """(calls that uploaded their descriptor tables, calls that found them on the device) since the context was made."""
+        up, re = ctypes.c_int64(0), ctypes.c_int64(0)
+        self._check(self.lib.atomo_get_table_uploads(self._h, ctypes.byref(up), ctypes.byref(re)), "atomo_get_table_uploads")
+        return int(up.value), int(re.value)
 
     def set_tridiag_ctas(self, ctas_per_layer: int):
         """CTAs per layer of the blocked tridiagonal reduction (short sides above 512): 0 = chosen per batch, else 1,

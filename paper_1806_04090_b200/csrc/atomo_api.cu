@@ -11,8 +11,23 @@
 
 using namespace atomo;
 
+// Descriptor tables of a call (layer descriptors, tile lists, tensor maps, header templates) live in a device buffer
+// of their own and are uploaded only when they differ from what that buffer already holds: a training loop calls
+// with the same pointers and shapes every step, so in steady state a call issues no host-to-device copy at all (a
+// copy of a few KB would otherwise queue behind whatever the application has on the copy engine, e.g. the next
+// step's inputs).
+struct TableCache {
+  uint8_t* d = nullptr; size_t cap = 0;        // device buffer
+  uint8_t* h = nullptr; size_t hcap = 0;       // pinned staging buffer of the last upload
+  std::vector<uint8_t> last;                   // what the device buffer holds
+  cudaEvent_t ev = nullptr; bool ev_pending = false;
+  cudaStream_t last_stream = nullptr;
+};
+
 struct atomo_ctx {
   int device = 0;
+  TableCache tab_sp, tab_dec, tab_avg, tab_ew;
+  int64_t table_uploads = 0, table_reuses = 0;
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
   uint32_t* h_flag = nullptr;        // pinned: convergence flag / state mirror
@@ -69,6 +84,51 @@ int fail_cuda(atomo_ctx* ctx, cudaError_t e, const char* what) {
     cudaError_t e__ = (call);                                               \
     if (e__ != cudaSuccess) return fail_cuda(ctx, e__, #call);              \
   } while (0)
+
+// device buffer of at least `bytes` for a table cache (growing it forgets the cached contents)
+int table_reserve(atomo_ctx* ctx, TableCache& tc, size_t bytes) {
+  if (bytes <= tc.cap) return ATOMO_OK;
+  CK(cudaDeviceSynchronize());
+  if (tc.d) CK(cudaFree(tc.d));
+  tc.d = nullptr; tc.cap = 0; tc.last.clear();
+  const size_t want = bytes + bytes / 4 + 4096;
+  CK(cudaMalloc(&tc.d, want));
+  tc.cap = want;
+  return ATOMO_OK;
+}
+
+// makes the device buffer hold host[0 .. bytes): nothing to do if it already does
+int table_commit(atomo_ctx* ctx, TableCache& tc, const uint8_t* host, size_t bytes, cudaStream_t st) {
+  if (tc.ev == nullptr) CK(cudaEventCreateWithFlags(&tc.ev, cudaEventDisableTiming));
+  if (tc.last.size() == bytes && std::memcmp(tc.last.data(), host, bytes) == 0) {
+    if (st != tc.last_stream && tc.ev_pending) CK(cudaStreamWaitEvent(st, tc.ev, 0));   // the upload ran on another stream
+    ++ctx->table_reuses;
+    return ATOMO_OK;
+  }
+  if (tc.ev_pending) { CK(cudaEventSynchronize(tc.ev)); tc.ev_pending = false; }          // the staging buffer is free again
+  if (tc.last_stream != st && tc.last_stream != nullptr) CK(cudaStreamSynchronize(tc.last_stream));   // readers of the old tables
+  if (bytes > tc.hcap) {
+    if (tc.h) CK(cudaFreeHost(tc.h));
+    tc.h = nullptr; tc.hcap = 0;
+    CK(cudaMallocHost(&tc.h, bytes + bytes / 4 + 4096));
+    tc.hcap = bytes + bytes / 4 + 4096;
+  }
+  std::memcpy(tc.h, host, bytes);
+  CK(cudaMemcpyAsync(tc.d, tc.h, bytes, cudaMemcpyHostToDevice, st));
+  CK(cudaEventRecord(tc.ev, st));
+  tc.ev_pending = true;
+  tc.last.assign(host, host + bytes);
+  tc.last_stream = st;
+  ++ctx->table_uploads;
+  return ATOMO_OK;
+}
+
+void table_free(TableCache& tc) {
+  if (tc.d) cudaFree(tc.d);
+  if (tc.h) cudaFreeHost(tc.h);
+  if (tc.ev) cudaEventDestroy(tc.ev);
+  tc = TableCache();
+}
 
 int ensure_ws(atomo_ctx* ctx, size_t bytes) {
   if (bytes <= ctx->ws_bytes) return ATOMO_OK;
@@ -184,6 +244,7 @@ int atomo_destroy(atomo_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaDeviceSynchronize();
   if (ctx->ws) cudaFree(ctx->ws);
+  table_free(ctx->tab_sp); table_free(ctx->tab_dec); table_free(ctx->tab_avg); table_free(ctx->tab_ew);
   if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
   if (ctx->h_state) cudaFreeHost(ctx->h_state);
   if (ctx->ev_sync) cudaEventDestroy(ctx->ev_sync);
@@ -278,6 +339,13 @@ int atomo_set_eig_params(atomo_ctx* ctx, int32_t max_sweeps, float tol) {
 }
 
 int atomo_last_eig_scheme(atomo_ctx* ctx) { return ctx ? ctx->eig_scheme_used : -1; }
+
+int atomo_get_table_uploads(atomo_ctx* ctx, int64_t* uploads, int64_t* reuses) {
+  if (!ctx) return ATOMO_ERR_INVALID_ARG;
+  if (uploads) *uploads = ctx->table_uploads;
+  if (reuses) *reuses = ctx->table_reuses;
+  return ATOMO_OK;
+}
 
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled) {
   if (!ctx || enabled < 0 || enabled > 3) return ATOMO_ERR_INVALID_ARG;
@@ -455,28 +523,78 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
         for (int c = 0; c < L[l].gram_split; ++c) tc_tiles.push_back({l, a, b, c});
     }
   }
+  // cluster tables of the eigen stage: small tridiagonal layers packed into 16-CTA clusters, largest first (a layer
+  // takes rp / 32 consecutive ranks of one cluster); or, on the Jacobi cluster route, the block pairs of every layer
+  std::vector<ClusterCta> ctas;
+  int n_clusters = 0, rp_max_small = 32;
+  if (tri_form) {
+    const int per = sp_tridiag_cluster_ctas();
+    std::vector<int> order;
+    for (int l = 0; l < n_layers; ++l) if (L[l].tri == 1) { order.push_back(l); rp_max_small = std::max(rp_max_small, L[l].rp); }
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].rp > L[b].rp; });
+    std::vector<int> used;
+    for (int l : order) {
+      const int nc = sp_tridiag_ctas_of(L[l].rp);
+      size_t c = 0;
+      while (c < used.size() && used[c] + nc > per) ++c;
+      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
+      for (int sl = 0; sl < nc; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], nc};
+      used[c] += nc;
+    }
+    n_clusters = (int)used.size();
+  } else if (cluster_form) {
+    const int per = sp_jacobi_cluster_ctas();
+    std::vector<int> order(n_layers);
+    for (int l = 0; l < n_layers; ++l) order[l] = l;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].nb > L[b].nb; });
+    std::vector<int> used;                                 // slots taken in each cluster (first fit, largest first)
+    for (int l : order) {
+      const int need_slots = L[l].nb / 2;
+      size_t c = 0;
+      while (c < used.size() && used[c] + need_slots > per) ++c;
+      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
+      for (int sl = 0; sl < need_slots; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], 0};
+      used[c] += need_slots;
+    }
+    n_clusters = (int)used.size();
+  }
+  // the tables go to the table cache (device buffer tab_sp, host mirror `tables` with the same offsets), everything
+  // the kernels write to the workspace
   SpLayer* d_layers = nullptr; TileRef *d_gram = nullptr, *d_pairs = nullptr, *d_bp = nullptr, *d_chol = nullptr, *d_ref = nullptr, *d_tc = nullptr;
   uint8_t* d_maps = nullptr;
   uint32_t* d_flag = nullptr;
   ClusterCta* d_ctas = nullptr;
   int* d_big = nullptr;
   const float** d_given = nullptr;
+  atomo_layer_header* d_hdr_tmpl = nullptr;
+  std::vector<uint8_t> tables;
+  size_t table_bytes = 0;
+  for (int pass = 0; pass < 2; ++pass) {
+    Arena T(pass ? ctx->tab_sp.d : nullptr);
+    d_layers = T.take<SpLayer>(n_layers);
+    d_gram = T.take<TileRef>(gram_tiles.size());
+    d_pairs = T.take<TileRef>(block_pairs.size());
+    d_bp = T.take<TileRef>(bp_tiles.size());
+    d_chol = T.take<TileRef>(chol_ctas.size());
+    d_ref = T.take<TileRef>(refine_tiles.size());
+    d_tc = T.take<TileRef>(tc_tiles.size());
+    d_maps = T.take<uint8_t>(maps_blob.size());
+    d_ctas = T.take<ClusterCta>(ctas.size());
+    d_big = T.take<int>(big_layers.size());
+    d_given = T.take<const float*>(given ? (size_t)2 * n_layers : 0);
+    d_hdr_tmpl = T.take<atomo_layer_header>(n_layers);
+    table_bytes = T.off + 256;
+    if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_sp, table_bytes); if (rc != ATOMO_OK) return rc; }
+  }
+  tables.assign(table_bytes, 0);
+  auto put = [&](const void* dev_ptr, const void* src, size_t bytes) {
+    if (bytes) std::memcpy(tables.data() + (reinterpret_cast<const uint8_t*>(dev_ptr) - ctx->tab_sp.d), src, bytes);
+  };
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
   for (int pass = 0; pass < 2; ++pass) {
     Arena A(pass ? ctx->ws : nullptr);
-    d_layers = A.take<SpLayer>(n_layers);
-    d_gram = A.take<TileRef>(gram_tiles.size());
-    d_pairs = A.take<TileRef>(block_pairs.size());
-    d_bp = A.take<TileRef>(bp_tiles.size());
-    d_chol = A.take<TileRef>(chol_ctas.size());
-    d_ref = A.take<TileRef>(refine_tiles.size());
-    d_tc = A.take<TileRef>(tc_tiles.size());
-    d_maps = A.take<uint8_t>(maps_blob.size());
     d_flag = A.take<uint32_t>(4);
-    d_ctas = A.take<ClusterCta>((size_t)n_layers * sp_jacobi_cluster_ctas());   // at most one cluster per layer
-    d_big = A.take<int>(big_layers.size());
-    d_given = A.take<const float*>(given ? (size_t)2 * n_layers : 0);
     size_t dbg_atoms = 0, dbg_words = 0, dbg_sq = 0;
     for (int l = 0; l < n_layers; ++l) {
       SpLayer& d = L[l];
@@ -539,39 +657,43 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
   }
 
-  // ---- uploads ----
-  std::vector<uint8_t> hdr_blob(sizeof(atomo_payload_header) + (size_t)n_layers * sizeof(atomo_layer_header), 0);
+  // ---- tables (uploaded only if they changed since the last call), headers, zero-filled regions ----
   atomo_payload_header gh{};
   gh.magic = ATOMO_MAGIC; gh.version = ATOMO_VERSION; gh.kind = ATOMO_KIND_SPECTRAL; gh.n_layers = (uint32_t)n_layers;
   gh.total_bytes = total; gh.seed = seed; gh.step = step; gh.s = s;
-  std::memcpy(hdr_blob.data(), &gh, sizeof(gh));
-  for (int l = 0; l < n_layers; ++l) {
-    atomo_layer_header h{};
-    h.rows = rows[l]; h.cols = cols[l]; h.k_cap = lay[l].kc; h.k = 0; h.status = ATOMO_OK;
-    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_coef; h.off_short = lay[l].off_short; h.off_long = lay[l].off_long;
-    std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
+  {
+    std::vector<atomo_layer_header> tmpl(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+      atomo_layer_header h{};
+      h.rows = rows[l]; h.cols = cols[l]; h.k_cap = lay[l].kc; h.k = 0; h.status = ATOMO_OK;
+      h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_coef; h.off_short = lay[l].off_short; h.off_long = lay[l].off_long;
+      tmpl[l] = h;
+    }
+    put(d_hdr_tmpl, tmpl.data(), tmpl.size() * sizeof(atomo_layer_header));
   }
-  CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
-  CK(cudaMemcpyAsync(d_layers, L.data(), L.size() * sizeof(SpLayer), cudaMemcpyHostToDevice, st));
-  if (!gram_tiles.empty()) CK(cudaMemcpyAsync(d_gram, gram_tiles.data(), gram_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!block_pairs.empty()) CK(cudaMemcpyAsync(d_pairs, block_pairs.data(), block_pairs.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!bp_tiles.empty()) CK(cudaMemcpyAsync(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!tc_tiles.empty()) {
-    CK(cudaMemcpyAsync(d_tc, tc_tiles.data(), tc_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(d_maps, maps_blob.data(), maps_blob.size(), cudaMemcpyHostToDevice, st));
+  put(d_layers, L.data(), L.size() * sizeof(SpLayer));
+  put(d_gram, gram_tiles.data(), gram_tiles.size() * sizeof(TileRef));
+  put(d_pairs, block_pairs.data(), block_pairs.size() * sizeof(TileRef));
+  put(d_bp, bp_tiles.data(), bp_tiles.size() * sizeof(TileRef));
+  put(d_chol, chol_ctas.data(), chol_ctas.size() * sizeof(TileRef));
+  put(d_ref, refine_tiles.data(), refine_tiles.size() * sizeof(TileRef));
+  put(d_tc, tc_tiles.data(), tc_tiles.size() * sizeof(TileRef));
+  put(d_maps, maps_blob.data(), maps_blob.size());
+  put(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta));
+  put(d_big, big_layers.data(), big_layers.size() * sizeof(int));
+  if (given) {
+    std::vector<const float*> ptrs(2 * (size_t)n_layers);
+    for (int l = 0; l < n_layers; ++l) { ptrs[l] = given_sigma[l]; ptrs[n_layers + l] = given_short[l]; }
+    put(d_given, ptrs.data(), ptrs.size() * sizeof(const float*));
   }
-  CK(cudaMemsetAsync(d_flag, 0, 4 * sizeof(uint32_t), st));
-  if (!refine_tiles.empty()) CK(cudaMemcpyAsync(d_ref, refine_tiles.data(), refine_tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
-  if (!chol_ctas.empty()) CK(cudaMemcpyAsync(d_chol, chol_ctas.data(), chol_ctas.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+  { const int rc = table_commit(ctx, ctx->tab_sp, tables.data(), table_bytes, st); if (rc != ATOMO_OK) return rc; }
+  launch_sp_begin(pay, gh, d_hdr_tmpl, n_layers, d_flag, st);          // payload header, layer headers, flags
   CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
 
   // ---- S1: Gram matrix, scaling ----
   stage_begin(ctx, ATOMO_STAGE_GRAM, st);
   if (given) {
     // singular values and short-side vectors as given: squared into the eigenvalue slots, vectors into the rows of X
-    std::vector<const float*> ptrs(2 * (size_t)n_layers);
-    for (int l = 0; l < n_layers; ++l) { ptrs[l] = given_sigma[l]; ptrs[n_layers + l] = given_short[l]; }
-    CK(cudaMemcpyAsync(d_given, ptrs.data(), ptrs.size() * sizeof(const float*), cudaMemcpyHostToDevice, st));
     launch_sp_load_svd(d_layers, n_layers, d_given, d_given + n_layers, st);
   } else {
   if (ctx->eig_mode == 0) launch_sp_init(d_layers, n_layers, nullptr, 0, st);   // the identity half of [A | I]
@@ -596,26 +718,9 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
   // Persistent form: the block pairs of a group of whole layers are co-resident (one CTA per SM) and solve their
   // layers in one cooperative launch.  A batch larger than the GPU is cut into such groups, launched one after
   // the other; a single layer with more block pairs than the GPU holds CTAs falls back to one launch per step.
-  int rp_max_small = 32;
   if (tri_form) {
-    // small layers packed into 16-CTA clusters, largest first (a layer takes rp / 32 consecutive ranks of one cluster)
-    const int per = sp_tridiag_cluster_ctas();
-    std::vector<int> order;
-    for (int l = 0; l < n_layers; ++l) if (L[l].tri == 1) { order.push_back(l); rp_max_small = std::max(rp_max_small, L[l].rp); }
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].rp > L[b].rp; });
-    std::vector<int> used;
-    std::vector<ClusterCta> ctas;
-    for (int l : order) {
-      const int nc = sp_tridiag_ctas_of(L[l].rp);
-      size_t c = 0;
-      while (c < used.size() && used[c] + nc > per) ++c;
-      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
-      for (int sl = 0; sl < nc; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], nc};
-      used[c] += nc;
-    }
-    if (!order.empty()) {
-      CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
-      const int e = launch_sp_tridiag(d_layers, d_ctas, (int)used.size(), rp_max_small, st);
+    if (n_clusters > 0) {
+      const int e = launch_sp_tridiag(d_layers, d_ctas, n_clusters, rp_max_small, st);
       if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(tridiagonal reduction)");
       ++n_eig_launch;
     }
@@ -629,7 +734,6 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
       int cc = cmin;
       if (ctx->tri_big_ctas > 0) cc = std::max(cmin, ctx->tri_big_ctas);
       else while (cc < 16 && (int)big_layers.size() * cc * 2 <= sms) cc *= 2;
-      CK(cudaMemcpyAsync(d_big, big_layers.data(), big_layers.size() * sizeof(int), cudaMemcpyHostToDevice, st));
       const int e = launch_sp_tridiag_big(d_layers, d_big, (int)big_layers.size(), rb, cc, 0, st);
       if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(blocked tridiagonal reduction)");
       ++n_eig_launch;
@@ -639,22 +743,7 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     // (ATOMO_ERR_TIMEOUT, nothing kept)
   }
   if (cluster_form) {
-    const int per = sp_jacobi_cluster_ctas();
-    std::vector<int> order(n_layers);
-    for (int l = 0; l < n_layers; ++l) order[l] = l;
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return L[a].nb > L[b].nb; });
-    std::vector<int> used;                                 // slots taken in each cluster (first fit, largest first)
-    std::vector<ClusterCta> ctas;
-    for (int l : order) {
-      const int need_slots = L[l].nb / 2;
-      size_t c = 0;
-      while (c < used.size() && used[c] + need_slots > per) ++c;
-      if (c == used.size()) { used.push_back(0); ctas.resize(ctas.size() + per, ClusterCta{-1, 0, 0, 0}); }
-      for (int sl = 0; sl < need_slots; ++sl) ctas[c * per + used[c] + sl] = ClusterCta{l, sl, used[c], 0};
-      used[c] += need_slots;
-    }
-    CK(cudaMemcpyAsync(d_ctas, ctas.data(), ctas.size() * sizeof(ClusterCta), cudaMemcpyHostToDevice, st));
-    const int e = launch_sp_jacobi_cluster(d_layers, d_ctas, (int)used.size(), rp_max, max_sweeps, ctx->tol, st);
+    const int e = launch_sp_jacobi_cluster(d_layers, d_ctas, n_clusters, rp_max, max_sweeps, ctx->tol, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(jacobi clusters)");
     launch_sp_check(d_layers, n_layers, steps_max * max_sweeps, max_sweeps, d_flag, st);
     n_eig_launch = 2;
@@ -816,20 +905,25 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     if (pass == 0) { const int rc = ensure_ws(ctx, need); if (rc != ATOMO_OK) return rc; }
   }
 
-  std::vector<uint8_t> hdr_blob(sizeof(atomo_payload_header) + (size_t)n_vecs * sizeof(atomo_layer_header), 0);
   atomo_payload_header gh{};
   gh.magic = ATOMO_MAGIC; gh.version = ATOMO_VERSION; gh.kind = ATOMO_KIND_ENTRYWISE; gh.n_layers = (uint32_t)n_vecs;
   gh.total_bytes = total; gh.seed = seed; gh.step = step; gh.s = s;
   gh.ew_format = (uint64_t)ctx->ew_format; gh.ew_sat_cap = compact ? (uint64_t)ctx->ew_sat_cap : 0;
-  std::memcpy(hdr_blob.data(), &gh, sizeof(gh));
-  for (int l = 0; l < n_vecs; ++l) {
-    atomo_layer_header h{};
-    h.rows = 1; h.cols = ns[l]; h.k_cap = lay[l].kc; h.status = ATOMO_OK;
-    h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val; h.off_short = lay[l].off_tiles;
-    h.off_long = compact ? lay[l].off_sat : 0;
-    std::memcpy(hdr_blob.data() + sizeof(gh) + (size_t)l * sizeof(h), &h, sizeof(h));
+  {
+    // layer header templates through the table cache; the headers themselves are written by a kernel
+    std::vector<atomo_layer_header> tmpl(n_vecs);
+    for (int l = 0; l < n_vecs; ++l) {
+      atomo_layer_header h{};
+      h.rows = 1; h.cols = ns[l]; h.k_cap = lay[l].kc; h.status = ATOMO_OK;
+      h.off_idx = lay[l].off_idx; h.off_val = lay[l].off_val; h.off_short = lay[l].off_tiles;
+      h.off_long = compact ? lay[l].off_sat : 0;
+      tmpl[l] = h;
+    }
+    const size_t tb = tmpl.size() * sizeof(atomo_layer_header);
+    { const int rc = table_reserve(ctx, ctx->tab_ew, tb); if (rc != ATOMO_OK) return rc; }
+    { const int rc = table_commit(ctx, ctx->tab_ew, reinterpret_cast<const uint8_t*>(tmpl.data()), tb, st); if (rc != ATOMO_OK) return rc; }
+    launch_sp_begin(pay, gh, reinterpret_cast<const atomo_layer_header*>(ctx->tab_ew.d), n_vecs, nullptr, st);
   }
-  CK(cudaMemcpyAsync(pay, hdr_blob.data(), hdr_blob.size(), cudaMemcpyHostToDevice, st));
 
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   const uint32_t ks = kind_step_word(ATOMO_KIND_ENTRYWISE, step);
@@ -923,14 +1017,18 @@ int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload, const int64_
       for (int a = 0; a < na; ++a) for (int b = 0; b < nbt; ++b) tiles.push_back({l, a, b, 0});
     }
     SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
+    size_t tb = 0;
     for (int pass = 0; pass < 2; ++pass) {
-      Arena A(pass ? ctx->ws : nullptr);
-      d_layers = A.take<SpDecodeLayer>(n_layers);
-      d_tiles = A.take<TileRef>(tiles.size());
-      if (pass == 0) { const int rc = ensure_ws(ctx, A.off + 256); if (rc != ATOMO_OK) return rc; }
+      Arena T(pass ? ctx->tab_dec.d : nullptr);
+      d_layers = T.take<SpDecodeLayer>(n_layers);
+      d_tiles = T.take<TileRef>(tiles.size());
+      tb = T.off + 256;
+      if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_dec, tb); if (rc != ATOMO_OK) return rc; }
     }
-    CK(cudaMemcpyAsync(d_layers, D.data(), D.size() * sizeof(SpDecodeLayer), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
+    std::vector<uint8_t> tables(tb, 0);
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - ctx->tab_dec.d), D.data(), D.size() * sizeof(SpDecodeLayer));
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - ctx->tab_dec.d), tiles.data(), tiles.size() * sizeof(TileRef));
+    { const int rc = table_commit(ctx, ctx->tab_dec, tables.data(), tb, st); if (rc != ATOMO_OK) return rc; }
     launch_sp_decode(pay, d_layers, d_tiles, (int)tiles.size(), st);
     stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
   }
@@ -963,18 +1061,25 @@ int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloa
     }
   }
   const uint8_t** d_pay = nullptr; SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
+  size_t tb = 0;
   for (int pass = 0; pass < 2; ++pass) {
-    Arena A(pass ? ctx->ws : nullptr);
-    d_pay = A.take<const uint8_t*>(n_payloads);
-    d_layers = A.take<SpDecodeLayer>(D.size());
-    d_tiles = A.take<TileRef>(tiles.size());
-    if (pass == 0) { const int rc = ensure_ws(ctx, A.off + 256); if (rc != ATOMO_OK) return rc; }
+    Arena T(pass ? ctx->tab_avg.d : nullptr);
+    d_pay = T.take<const uint8_t*>(n_payloads);
+    d_layers = T.take<SpDecodeLayer>(D.size());
+    d_tiles = T.take<TileRef>(tiles.size());
+    tb = T.off + 256;
+    if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_avg, tb); if (rc != ATOMO_OK) return rc; }
+  }
+  {
+    std::vector<uint8_t> tables(tb, 0);
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_pay) - ctx->tab_avg.d), payloads, (size_t)n_payloads * sizeof(void*));
+    if (!D.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - ctx->tab_avg.d), D.data(), D.size() * sizeof(SpDecodeLayer));
+    if (!tiles.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - ctx->tab_avg.d), tiles.data(), tiles.size() * sizeof(TileRef));
+    const int rc = table_commit(ctx, ctx->tab_avg, tables.data(), tb, st);
+    if (rc != ATOMO_OK) return rc;
   }
   stage_begin(ctx, ATOMO_STAGE_DECODE, st);
-  CK(cudaMemcpyAsync(d_pay, payloads, (size_t)n_payloads * sizeof(void*), cudaMemcpyHostToDevice, st));
   if (kind == ATOMO_KIND_SPECTRAL) {
-    CK(cudaMemcpyAsync(d_layers, D.data(), D.size() * sizeof(SpDecodeLayer), cudaMemcpyHostToDevice, st));
-    CK(cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(TileRef), cudaMemcpyHostToDevice, st));
     launch_sp_decode_average(d_pay, n_payloads, d_layers, d_tiles, (int)tiles.size(), st);
     stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
   } else {

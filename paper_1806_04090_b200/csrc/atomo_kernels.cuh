@@ -119,6 +119,9 @@ void launch_sp_decode_average(const uint8_t* const* d_payloads, int n_payloads, 
 void launch_ew_decode_average(const uint8_t* const* d_payloads, int n_payloads, int layer, float* out, int64_t n,
                               cudaStream_t st);
 
+// payload header (by value), layer headers from a device template, the call's four flag words (may be null)
+void launch_sp_begin(uint8_t* pay, const atomo_payload_header& gh, const atomo_layer_header* d_tmpl, int n_layers,
+                     uint32_t* d_flags, cudaStream_t st);
 void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling

@@ -16,6 +16,8 @@
 //   sp_backproject     long-side vector of each kept atom, w_i = G^T u_i (or G v_i)
 //   sp_finish_atoms    sigma_i = ||w_i||, coef_i = sigma_i / p_i, w_i normalised
 //   sp_decode          G_hat = sum_k coef_k u_k v_k^T, one streaming write pass (8 atoms per pass)
+#include <algorithm>
+
 #include "atomo_kernels.cuh"
 
 namespace atomo {
@@ -147,6 +149,27 @@ __global__ void __launch_bounds__(256) sp_scale_kernel(const SpLayer* __restrict
   if (sc == 1.0f) return;
   for (int i = blockIdx.y; i < L.r; i += gridDim.y)
     for (int j = threadIdx.x; j < L.r; j += 256) L.A[(int64_t)i * lda + j] *= sc;
+}
+
+// Start of an encode call: the payload header (passed by value), the layer headers from their template in the table
+// cache, and the call's flag words -- a kernel instead of host-to-device copies, which would queue behind whatever the
+// application has on the copy engine.
+__global__ void __launch_bounds__(256) begin_kernel(uint8_t* __restrict__ pay, atomo_payload_header gh,
+                                                    const atomo_layer_header* __restrict__ tmpl, int n_layers,
+                                                    uint32_t* __restrict__ flags) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<atomo_payload_header*>(pay) = gh;
+  if (blockIdx.x == 0 && threadIdx.x < 4 && flags != nullptr) flags[threadIdx.x] = 0u;
+  static_assert(sizeof(atomo_layer_header) % 16 == 0 && sizeof(atomo_payload_header) % 16 == 0, "headers are copied as 16-byte words");
+  uint4* dst = reinterpret_cast<uint4*>(pay + sizeof(atomo_payload_header));
+  const uint4* src = reinterpret_cast<const uint4*>(tmpl);
+  const int n16 = n_layers * (int)(sizeof(atomo_layer_header) / 16);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += gridDim.x * blockDim.x) dst[i] = src[i];
+}
+
+void launch_sp_begin(uint8_t* pay, const atomo_payload_header& gh, const atomo_layer_header* d_tmpl, int n_layers,
+                     uint32_t* d_flags, cudaStream_t st) {
+  const int n16 = n_layers * (int)(sizeof(atomo_layer_header) / 16);
+  begin_kernel<<<std::max(1, std::min(32, (n16 + 255) / 256)), 256, 0, st>>>(pay, gh, d_tmpl, n_layers, d_flags);
 }
 
 // A decomposition supplied by the caller (test entry point): lambda_i = sigma_i^2 in the eigenvalue slots (scale 1),

@@ -414,9 +414,11 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
 //   * the panel (16 columns: u_t and w_t of all rows) lives in shared memory, so the column update, the correction
 //     of y and the panel dots never leave the SM, and the rank-32 update at the end of a panel takes its operands
 //     from there (4 x 4 outputs per thread on 128 x 128 tiles of the lower triangle).
-//   * thread g owns row g for the whole reduction.
+//   * 512 threads; thread t owns rows t and t + 512 for the whole reduction.
 namespace {
 
+constexpr int kT1Threads = 512;              // 128 registers per thread: two sub-tiles of the product in flight per warp
+constexpr int kT1Warps = kT1Threads / 32;
 constexpr int kT1NB = 16;                    // columns per panel
 constexpr int kT1MaxR = 1024;
 constexpr int kT1Blk = 64;                   // tile edge of the matrix-vector product
@@ -469,7 +471,7 @@ __device__ __forceinline__ float rs4(float (&v)[4], int lane) {
 
 }  // namespace
 
-__global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const SpLayer* __restrict__ layers,
+__global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const SpLayer* __restrict__ layers,
                                                                         const int* __restrict__ big_layers) {
   extern __shared__ __align__(16) unsigned char tb_smem[];
   T1Shared& S = *reinterpret_cast<T1Shared*>(tb_smem);
@@ -481,23 +483,22 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
   const SpLayer& L = layers[big_layers[blockIdx.x]];
   const int r = L.r;
   const int64_t lda = L.lda;
-  float* const A = reinterpret_cast<float*>(L.tb_A);
+  const float* const A = reinterpret_cast<const float*>(L.tb_A);
+  float* const At = L.tb_At;
   float* const V = L.td_V;
   const int64_t ldv = L.td_ldv;
   double* const td_d = L.td_d;
   double* const td_e = L.td_e;
   const int nblk = (r + 31) / 32;
   const int nb64 = (r + kT1Blk - 1) / kT1Blk;
-  const int r4 = (r + 3) & ~3;
-  const int g = tid;
-  const bool valid = g < r;
-  const int ly = lane >> 3, lx = lane & 7;                                     // sub-tile layout: rows 4 k + ly, columns 4 lx .. 4 lx + 3
-  const int idx = 4 * lx + ly;                                                 // the row / column a lane ends up with after the reduce-scatters
+  const int g[2] = {tid, tid + kT1Threads};                                    // this thread's two rows (32-row blocks w and w + 16)
+  const bool valid[2] = {g[0] < r, g[1] < r};
+  const int ly = lane >> 3, lx = lane & 7;                                     // sub-tile layout: rows 8 ly + kk, columns 4 lx .. 4 lx + 3
+  const int idx = 4 * lx + ly;                                                 // the column a lane ends up with after the reduce-scatter
 
-  float* const At = L.tb_At;
-  s_u[tid] = 0.0f;
+  s_u[g[0]] = 0.0f; s_u[g[1]] = 0.0f;
   // the lower triangle of A into tile-major order (one warp per sub-tile: 32 rows of 128 bytes in, 4 KB out)
-  for (int k = w; k < nblk * (nblk + 1) / 2; k += kTbWarps) {
+  for (int k = w; k < nblk * (nblk + 1) / 2; k += kT1Warps) {
     int I = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);
     while ((I + 1) * (I + 2) / 2 <= k) ++I;
     while (I * (I + 1) / 2 > k) --I;
@@ -516,28 +517,37 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
   TB_PROF_DECL
   // element (row, col) of the working copy, col <= row
   auto at = [&](int row, int col) -> float* { return t1_sub(At, row >> 5, col >> 5) + ((row & 31) << 5) + (col & 31); };
-  float a_pref = valid ? __ldcg(at(g, 0)) : 0.0f;                              // column 0 of row g (lower triangle: g >= 0)
+  float a_pref[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) a_pref[x] = valid[x] ? __ldcg(at(g[x], 0)) : 0.0f;   // column 0 (lower triangle: every row)
   for (int c = 0; c < r; ++c) {
     const int p0 = c / kT1NB * kT1NB;
     const int i = c < n_ref ? c - p0 : 0;
     // ---- column c as the earlier reflectors of the panel left it ----
-    double a = 0.0;
-    if (valid && g >= c) {
-      a = (double)a_pref;
-      for (int t = 0; t < i; ++t)
-        a -= (double)pan_u[t * kT1MaxR + g] * (double)pan_w[t * kT1MaxR + c] + (double)pan_w[t * kT1MaxR + g] * (double)pan_u[t * kT1MaxR + c];
-      if (g == c) td_d[c] = a;
+    double a[2] = {0.0, 0.0};
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      if (valid[x] && g[x] >= c) {
+        a[x] = (double)a_pref[x];
+        for (int t = 0; t < i; ++t)
+          a[x] -= (double)pan_u[t * kT1MaxR + g[x]] * (double)pan_w[t * kT1MaxR + c] + (double)pan_w[t * kT1MaxR + g[x]] * (double)pan_u[t * kT1MaxR + c];
+        if (g[x] == c) td_d[c] = a[x];
+      }
     }
     if (c >= n_ref) {
-      if (c == r - 2 && valid && g == r - 1) td_e[c] = a;
-      if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;
+#pragma unroll
+      for (int x = 0; x < 2; ++x) {
+        if (c == r - 2 && valid[x] && g[x] == r - 1) td_e[c] = a[x];
+        if (c + 1 < r) a_pref[x] = (valid[x] && g[x] >= c + 1) ? __ldcg(at(g[x], c + 1)) : 0.0f;
+      }
       continue;
     }
-    const bool live = valid && g > c;
-    {
-      const double sq = warp_sum(live ? a * a : 0.0);
-      if (lane == 0) S.part_a[w] = sq;
-      if (g == c + 1) S.x0 = a;
+    const bool live[2] = {valid[0] && g[0] > c, valid[1] && g[1] > c};
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      const double sq = warp_sum(live[x] ? a[x] * a[x] : 0.0);
+      if (lane == 0) S.part_a[w + kT1Warps * x] = sq;
+      if (g[x] == c + 1) S.x0 = a[x];
     }
     __syncthreads();
     const double nx2 = tb_ordered_sum(S.part_a, nblk, lane);
@@ -548,137 +558,180 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
       alpha = -copysign(nx, x0);
       inv = rsqrt(2.0 * nx * (nx + fabs(x0)));
     }
-    float u_f = 0.0f;
-    if (valid) {
-      if (live) u_f = (float)((a - (g == c + 1 ? alpha : 0.0)) * inv);
-      V[(int64_t)c * ldv + g] = u_f;
-      if (g == c + 1) td_e[c] = alpha;
-      s_u[g] = u_f;
-      pan_u[i * kT1MaxR + g] = u_f;
+    float u_f[2] = {0.0f, 0.0f};
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      if (valid[x]) {
+        if (live[x]) u_f[x] = (float)((a[x] - (g[x] == c + 1 ? alpha : 0.0)) * inv);
+        V[(int64_t)c * ldv + g[x]] = u_f[x];
+        if (g[x] == c + 1) td_e[c] = alpha;
+        s_u[g[x]] = u_f[x];
+        pan_u[i * kT1MaxR + g[x]] = u_f[x];
+      }
     }
-    const double u_own = (double)u_f;
     __syncthreads();
     TB_MARK(1)
     // ---- panel dots (one warp each), then y = A0 u over the tiles of the lower triangle ----
-    if (w < 2 * i) {
-      const int t = w >> 1;
-      const float* x = (w & 1) ? pan_u + t * kT1MaxR : pan_w + t * kT1MaxR;   // odd: b_t = u_t^T u, even: a_t = w_t^T u
+    for (int id = w; id < 2 * i; id += kT1Warps) {
+      const int t = id >> 1;
+      const float* xv = (id & 1) ? pan_u + t * kT1MaxR : pan_w + t * kT1MaxR;  // odd: b_t = u_t^T u, even: a_t = w_t^T u
       double acc = 0.0;
-      for (int h = lane; h < r; h += 32) acc = fma((double)x[h], (double)s_u[h], acc);
+      for (int h = lane; h < r; h += 32) acc = fma((double)xv[h], (double)s_u[h], acc);
       acc = warp_sum(acc);
-      if (lane == 0) S.dots[w] = acc;
+      if (lane == 0) S.dots[id] = acc;
     }
     {
       // One warp per 64 x 64 tile (I, J), J <= I, of the live part of the lower triangle, as up to four 32 x 32
-      // sub-tiles.  In a sub-tile a lane holds rows 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3.  Row sums
-      // are accumulated over the two sub-tiles of a row half before the eight lanes of a row are added up
-      // (reduce-scatter: lane 8 ly + lx ends with row 8 ly + lx), column sums over the two sub-tiles of a column half
-      // before the four lanes of a column are (lane ends with column 4 lx + ly).  The tile's sums go to slot J of
-      // block I (rows) and slot I of block J (columns): every slot has exactly one writer per step.
-      // (Tried and dropped: refilling each register group from the warp's next sub-tile as soon as it has been
-      // multiplied -- the extra live state spilled and the product took 2.7 times as long; 32 x 32 work units with
-      // order-free shared-memory adds -- no faster.)
+      // sub-tiles in the order (row half, column half) = (0,0) (0,1) (1,0) (1,1).  In a sub-tile a lane holds rows
+      // 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3.  Row sums are accumulated over the sub-tiles of a row half
+      // before the eight lanes of a row are added up (reduce-scatter: lane 8 ly + lx ends with row 8 ly + lx), column
+      // sums over the sub-tiles of a column half before the four lanes of a column are (lane ends with column
+      // 4 lx + ly).  The tile's sums go to slot J of block I (rows) and slot I of block J (columns): every slot has
+      // exactly one writer per step.  Two sub-tiles are in flight per warp: while one is multiplied the next 4 KB
+      // are on their way (with a single one in flight the SM's loads stop during the arithmetic and the kernel
+      // reaches little more than half of the memory's rate).
       const int j0 = (c + 1) / kT1Blk;                                         // first live block
       const int nbl = nb64 - j0;
       const int n_tiles = nbl * (nbl + 1) / 2;
-      for (int k = w; k < n_tiles; k += kTbWarps) {
-        int ii = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);
-        while ((ii + 1) * (ii + 2) / 2 <= k) ++ii;
-        while (ii * (ii + 1) / 2 > k) --ii;
-        const int I = j0 + ii, J = j0 + (k - ii * (ii + 1) / 2);
-        float racc[2] = {0.f, 0.f};
-        uint64_t cp[2][2] = {{pack2(0.f, 0.f), pack2(0.f, 0.f)}, {pack2(0.f, 0.f), pack2(0.f, 0.f)}};   // [column half][pair of columns]
+      struct Sub { int k, q, I, J; };
+      auto tile_of = [&](Sub& sbt) {
+        int ii = (int)((sqrtf(8.0f * (float)sbt.k + 1.0f) - 1.0f) * 0.5f);
+        while ((ii + 1) * (ii + 2) / 2 <= sbt.k) ++ii;
+        while (ii * (ii + 1) / 2 > sbt.k) --ii;
+        sbt.I = j0 + ii; sbt.J = j0 + (sbt.k - ii * (ii + 1) / 2);
+      };
+      // first sub-tile at or after (k, q) that exists: inside the matrix and not above the diagonal
+      auto settle = [&](Sub& sbt) {
+        while (sbt.k < n_tiles) {
+          if (sbt.q > 3) { sbt.k += kT1Warps; sbt.q = 0; if (sbt.k < n_tiles) tile_of(sbt); continue; }
+          if (2 * sbt.I + (sbt.q >> 1) >= nblk || (sbt.I == sbt.J && (sbt.q & 1) > (sbt.q >> 1))) { ++sbt.q; continue; }
+          return;
+        }
+      };
+      auto next_of = [&](const Sub& sbt) { Sub n = sbt; ++n.q; settle(n); return n; };
+      auto load = [&](float4 (&t)[8], const Sub& sbt) {
+        const float* src = t1_sub(At, 2 * sbt.I + (sbt.q >> 1), 2 * sbt.J + (sbt.q & 1)) + (8 * ly) * 32 + 4 * lx;
 #pragma unroll
-        for (int sa = 0; sa < 2; ++sa) {
-          const int row0 = kT1Blk * I + 32 * sa;
-          if (row0 >= r) continue;
-          float rp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-          const float4 ui0 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly);
-          const float4 ui1 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly + 4);
-          const float uiv[8] = {ui0.x, ui0.y, ui0.z, ui0.w, ui1.x, ui1.y, ui1.z, ui1.w};
+        for (int kk = 0; kk < 8; ++kk) t[kk] = ldcg4(src + kk * 32);
+      };
+      float rp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      float racc[2] = {0.f, 0.f};
+      uint64_t cp[2][2] = {{pack2(0.f, 0.f), pack2(0.f, 0.f)}, {pack2(0.f, 0.f), pack2(0.f, 0.f)}};   // [column half][pair of columns]
+      auto process = [&](const float4 (&t)[8], const Sub& cur, const Sub& nxt) {
+        const int sa = cur.q >> 1, sb = cur.q & 1;
+        const int row0 = kT1Blk * cur.I + 32 * sa, col0 = kT1Blk * cur.J + 32 * sb;
+        const bool diag = row0 == col0;
+        const float4 uj = *reinterpret_cast<const float4*>(s_u + col0 + 4 * lx);
+        const uint64_t uj01 = pack2(uj.x, uj.y), uj23 = pack2(uj.z, uj.w);
+        const float4 ui0 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly);
+        const float4 ui1 = *reinterpret_cast<const float4*>(s_u + row0 + 8 * ly + 4);
+        const float uiv[8] = {ui0.x, ui0.y, ui0.z, ui0.w, ui1.x, ui1.y, ui1.z, ui1.w};
+        uint64_t c01 = pack2(0.f, 0.f), c23 = pack2(0.f, 0.f);
 #pragma unroll
-          for (int sb = 0; sb < 2; ++sb) {
-            if (I == J && sb > sa) continue;                                   // above the diagonal
-            const int col0 = kT1Blk * J + 32 * sb;
-            const bool diag = row0 == col0;
-            float4 t[8];
-            {
-              const float* src = t1_sub(At, row0 >> 5, col0 >> 5) + (8 * ly) * 32 + 4 * lx;
-#pragma unroll
-              for (int kk = 0; kk < 8; ++kk) t[kk] = ldcg4(src + kk * 32);
-            }
-            const float4 uj = *reinterpret_cast<const float4*>(s_u + col0 + 4 * lx);
-            const uint64_t uj01 = pack2(uj.x, uj.y), uj23 = pack2(uj.z, uj.w);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk) {
-              float4 v = t[kk];
-              const int rr = 8 * ly + kk, cc = 4 * lx;                         // position inside the sub-tile
-              if (diag) {                                                      // lower triangle only
-                if (cc + 0 > rr) v.x = 0.f;
-                if (cc + 1 > rr) v.y = 0.f;
-                if (cc + 2 > rr) v.z = 0.f;
-                if (cc + 3 > rr) v.w = 0.f;
-              }
-              float s0, s1;
-              unpack2(fma2(pack2(v.z, v.w), uj23, fma2(pack2(v.x, v.y), uj01, pack2(0.f, 0.f))), s0, s1);
-              rp[kk] += s0 + s1;
-              if (diag) {                                                      // the diagonal entry counts once (with the rows)
-                if (cc + 0 == rr) v.x = 0.f;
-                if (cc + 1 == rr) v.y = 0.f;
-                if (cc + 2 == rr) v.z = 0.f;
-                if (cc + 3 == rr) v.w = 0.f;
-              }
-              const uint64_t ui2 = pack2(uiv[kk], uiv[kk]);
-              cp[sb][0] = fma2(pack2(v.x, v.y), ui2, cp[sb][0]);
-              cp[sb][1] = fma2(pack2(v.z, v.w), ui2, cp[sb][1]);
-            }
+        for (int kk = 0; kk < 8; ++kk) {
+          float4 v = t[kk];
+          const int rr = 8 * ly + kk, cc = 4 * lx;                             // position inside the sub-tile
+          if (diag) {                                                          // lower triangle only
+            if (cc + 0 > rr) v.x = 0.f;
+            if (cc + 1 > rr) v.y = 0.f;
+            if (cc + 2 > rr) v.z = 0.f;
+            if (cc + 3 > rr) v.w = 0.f;
           }
-          racc[sa] = rs8(rp, lane);
+          float s0, s1;
+          unpack2(fma2(pack2(v.z, v.w), uj23, fma2(pack2(v.x, v.y), uj01, pack2(0.f, 0.f))), s0, s1);
+          rp[kk] += s0 + s1;
+          if (diag) {                                                          // the diagonal entry counts once (with the rows)
+            if (cc + 0 == rr) v.x = 0.f;
+            if (cc + 1 == rr) v.y = 0.f;
+            if (cc + 2 == rr) v.z = 0.f;
+            if (cc + 3 == rr) v.w = 0.f;
+          }
+          const uint64_t ui2 = pack2(uiv[kk], uiv[kk]);
+          c01 = fma2(pack2(v.x, v.y), ui2, c01);
+          c23 = fma2(pack2(v.z, v.w), ui2, c23);
         }
-        float cacc[2];
+        {                                                                      // into the column half's accumulators (added in a fixed order)
+          float a0, a1, b0, b1;
+          unpack2(c01, a0, a1); unpack2(cp[sb][0], b0, b1); cp[sb][0] = pack2(a0 + b0, a1 + b1);
+          unpack2(c23, a0, a1); unpack2(cp[sb][1], b0, b1); cp[sb][1] = pack2(a0 + b0, a1 + b1);
+        }
+        const bool tile_ends = nxt.k >= n_tiles || nxt.k != cur.k;
+        if (tile_ends || (nxt.q >> 1) != sa) {                                 // the row half is complete
+          const float rs = rs8(rp, lane);
+          if (sa == 0) racc[0] = rs; else racc[1] = rs;
 #pragma unroll
-        for (int sb = 0; sb < 2; ++sb) {
-          float cv[4];
-          unpack2(cp[sb][0], cv[0], cv[1]); unpack2(cp[sb][1], cv[2], cv[3]);
-          cacc[sb] = rs4(cv, lane);
+          for (int kk = 0; kk < 8; ++kk) rp[kk] = 0.f;
         }
-        float* yi = y_part + ((size_t)I * kT1MaxB + J) * kT1Blk;
-        if (I == J) {
-          // rows and columns of the same block: a column's sum moves to the lane that holds the row of the same index
-          const int from = ((lane & 3) << 3) | (lane >> 2);
-          yi[lane] = racc[0] + __shfl_sync(0xffffffffu, cacc[0], from);
-          yi[32 + lane] = racc[1] + __shfl_sync(0xffffffffu, cacc[1], from);
-        } else {
-          yi[lane] = racc[0]; yi[32 + lane] = racc[1];
-          float* yj = y_part + ((size_t)J * kT1MaxB + I) * kT1Blk;
-          yj[idx] = cacc[0]; yj[32 + idx] = cacc[1];
+        if (tile_ends) {
+          float cacc[2];
+#pragma unroll
+          for (int hb = 0; hb < 2; ++hb) {
+            float cv[4];
+            unpack2(cp[hb][0], cv[0], cv[1]); unpack2(cp[hb][1], cv[2], cv[3]);
+            cacc[hb] = rs4(cv, lane);
+            cp[hb][0] = pack2(0.f, 0.f); cp[hb][1] = pack2(0.f, 0.f);
+          }
+          float* yi = y_part + ((size_t)cur.I * kT1MaxB + cur.J) * kT1Blk;
+          if (cur.I == cur.J) {
+            // rows and columns of the same block: a column's sum moves to the lane that holds the row of the same index
+            const int from = ((lane & 3) << 3) | (lane >> 2);
+            yi[lane] = racc[0] + __shfl_sync(0xffffffffu, cacc[0], from);
+            yi[32 + lane] = racc[1] + __shfl_sync(0xffffffffu, cacc[1], from);
+          } else {
+            yi[lane] = racc[0]; yi[32 + lane] = racc[1];
+            float* yj = y_part + ((size_t)cur.J * kT1MaxB + cur.I) * kT1Blk;
+            yj[idx] = cacc[0]; yj[32 + idx] = cacc[1];
+          }
+          racc[0] = 0.f; racc[1] = 0.f;
+        }
+      };
+      Sub s0{w, 0, 0, 0};
+      if (s0.k < n_tiles) tile_of(s0);
+      settle(s0);
+      if (s0.k < n_tiles) {
+        float4 ta[8], tb[8];
+        Sub s1 = next_of(s0);
+        load(ta, s0);
+        if (s1.k < n_tiles) load(tb, s1);
+        for (;;) {
+          Sub s2 = s1;
+          if (s1.k < n_tiles) s2 = next_of(s1);
+          process(ta, s0, s1);
+          if (s1.k >= n_tiles) break;
+          if (s2.k < n_tiles) load(ta, s2);
+          Sub s3 = s2;
+          if (s2.k < n_tiles) s3 = next_of(s2);
+          process(tb, s1, s2);
+          if (s2.k >= n_tiles) break;
+          if (s3.k < n_tiles) load(tb, s3);
+          s0 = s2; s1 = s3;
         }
       }
     }
     __syncthreads();
     TB_MARK(2)
     // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
-    double p = 0.0;
-    double ysum = 0.0;
-    if (live) {                                                                // this row's partial sums in ascending slot order
-      const int j0 = (c + 1) / kT1Blk;
-      const float* yp = y_part + (size_t)(g / kT1Blk) * kT1MaxB * kT1Blk + (g % kT1Blk);
-      for (int sl = j0; sl < nb64; ++sl) ysum += (double)yp[sl * kT1Blk];
+    double p[2] = {0.0, 0.0};
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      if (live[x]) {                                                           // this row's partial sums in ascending slot order
+        const int j0 = (c + 1) / kT1Blk;
+        const float* yp = y_part + (size_t)(g[x] / kT1Blk) * kT1MaxB * kT1Blk + (g[x] % kT1Blk);
+        double y = 0.0;
+        for (int sl = j0; sl < nb64; ++sl) y += (double)yp[sl * kT1Blk];
+        for (int t = 0; t < i; ++t)
+          y -= (double)pan_u[t * kT1MaxR + g[x]] * S.dots[2 * t] + (double)pan_w[t * kT1MaxR + g[x]] * S.dots[2 * t + 1];
+        p[x] = 2.0 * y;
+      }
+      const double kp = warp_sum((double)u_f[x] * p[x]);
+      if (lane == 0) S.part_k[w + kT1Warps * x] = kp;
+      if (c + 1 < r) a_pref[x] = (valid[x] && g[x] >= c + 1) ? __ldcg(at(g[x], c + 1)) : 0.0f;   // next column, in flight over the barrier
     }
-    if (live) {
-      double y = ysum;
-      for (int t = 0; t < i; ++t)
-        y -= (double)pan_u[t * kT1MaxR + g] * S.dots[2 * t] + (double)pan_w[t * kT1MaxR + g] * S.dots[2 * t + 1];
-      p = 2.0 * y;
-    }
-    {
-      const double kp = warp_sum(u_own * p);
-      if (lane == 0) S.part_k[w] = kp;
-    }
-    if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;   // next column, in flight over the barrier
     __syncthreads();
     const double K = tb_ordered_sum(S.part_k, nblk, lane);
-    if (valid) pan_w[i * kT1MaxR + g] = (float)(live ? p - K * u_own : 0.0);
+#pragma unroll
+    for (int x = 0; x < 2; ++x)
+      if (valid[x]) pan_w[i * kT1MaxR + g[x]] = (float)(live[x] ? p[x] - K * (double)u_f[x] : 0.0);
     const bool flush = (i == kT1NB - 1) || (c == n_ref - 1);
     __syncthreads();
     TB_MARK(4)
@@ -686,12 +739,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
     // ---- end of the panel: the lower triangle of A0 -= U W^T + W U^T on rows and columns beyond c ----
     {
       const int nr = i + 1, g0 = c + 1;
-      const int wr = w >> 3, wc = w & 7;
+      const int wr = w >> 3, wc = w & 7;                                       // 2 x 8 warps: 64 rows x 128 columns per pass
       const int qy = lane >> 2, qx = lane & 3;
-      const int b0 = g0 / 128, nb128 = (r + 127) / 128;
-      for (int RI = b0; RI < nb128; ++RI) {
-        for (int CJ = b0; CJ <= RI; ++CJ) {
-          const int row0 = 128 * RI + 32 * wr + 4 * qy, col0 = 128 * CJ + 16 * wc + 4 * qx;
+      const int nb128 = (r + 127) / 128;
+      for (int RI = g0 / 64; RI < nb64; ++RI) {
+        for (int CJ = g0 / 128; CJ < nb128 && 128 * CJ <= 64 * RI + 63; ++CJ) {
+          const int row0 = 64 * RI + 32 * wr + 4 * qy, col0 = 128 * CJ + 16 * wc + 4 * qx;
           if (col0 > row0 + 3 || row0 >= r) continue;                          // this thread's 4 x 4 lies above the diagonal or below the matrix
           float acc[4][4];
 #pragma unroll
@@ -715,8 +768,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
             const int gr = row0 + x;
-            if (gr >= r || gr < g0) continue;
-            if (col0 > gr) continue;
+            if (gr >= r || gr < g0 || col0 > gr) continue;
             float* dst = at(gr, col0);                                         // four columns of one sub-tile row
             if (col0 >= g0 && col0 + 3 <= gr) {                                // four live entries of the lower triangle
               float4 o = ldcg4(dst);
@@ -732,7 +784,9 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big1_kernel(const Sp
     }
     __threadfence_block();
     __syncthreads();
-    if (c + 1 < r) a_pref = (valid && g >= c + 1) ? __ldcg(at(g, c + 1)) : 0.0f;   // the update changed it
+#pragma unroll
+    for (int x = 0; x < 2; ++x)
+      if (c + 1 < r) a_pref[x] = (valid[x] && g[x] >= c + 1) ? __ldcg(at(g[x], c + 1)) : 0.0f;   // the update changed it
     TB_MARK(5)
   }
 #ifdef TB_PROFILE
@@ -921,7 +975,7 @@ int sp_configure_tridiag_big() {
 int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, int ctas, int fp64, cudaStream_t st) {
   if (n_big <= 0) return 0;
   if (ctas == 1 && !fp64 && r_max <= kT1MaxR) {               // one CTA per layer: the triangle-only kernel
-    sp_tridiag_big1_kernel<<<n_big, kTbThreads, t1_smem_bytes(), st>>>(d_layers, d_big);
+    sp_tridiag_big1_kernel<<<n_big, kT1Threads, t1_smem_bytes(), st>>>(d_layers, d_big);
     return (int)cudaGetLastError();
   }
 #define TB_CASE(CC) case CC: return fp64 ? tb_launch_one<double, CC>(d_layers, d_big, n_big, r_max, st) \
