@@ -6,7 +6,8 @@ may import it; the product never does, and this file imports nothing from the pr
 
 What each function follows:
 
-* ``atomo_probabilities``  -- Algorithm 1 ("ATOMO probabilities"), with the readings below.
+* ``atomo_probabilities``  -- the solution of Eq. (3) in the closed form of Appendix B (what Algorithm 1 computes),
+  with the readings below.
 * ``bernoulli_words`` / ``sample_mask`` -- the independent Bernoulli(p_i) draws of Eq. (2).
   The paper fixes only the distribution; generator, key and counter layout are this
   project's definition (Philox4x32-10, Salmon et al., SC'11).  Parity of the *stream*
@@ -137,11 +138,14 @@ def sample_mask(p: np.ndarray, words: np.ndarray) -> np.ndarray:
 # Algorithm 1
 # --------------------------------------------------------------------------------------
 def atomo_probabilities(lam: np.ndarray, s: float) -> Tuple[np.ndarray, int, float]:
-    """Algorithm 1: the p solving  min sum lambda_i^2 / p_i,  0 < p_i <= 1,  sum p_i = s.
+    """The p solving  min sum lambda_i^2 / p_i,  0 < p_i <= 1,  sum p_i = s  (Eq. 3), from the closed form of
+    Appendix B: with |lambda_1| >= ... >= |lambda_n| and tail_i = sum_{j >= i} |lambda_j|, n_s is the first count of
+    leading atoms for which the rest is (s - n_s)-balanced, |lambda_{n_s+1}| (s - n_s) <= tail_{n_s+1}; those n_s atoms
+    get p = 1 and the rest p_i = |lambda_i| (s - n_s) / tail_{n_s+1}.  (Algorithm 1 reaches the same n_s one atom at a
+    time.)
 
-    Returns (p in the caller's order, n_s = number of atoms the loop set to 1,
-    c = (sum of |lambda| over the rest) / (s - n_s), the common weight |lambda_i|/p_i of the
-    atoms that were not set to 1; c = 0 when that tail is empty or all zero).
+    Returns (p in the caller's order, n_s, c = tail_{n_s+1} / (s - n_s), the common weight |lambda_i| / p_i of the atoms
+    with p < 1; c = 0 when that tail is empty or all zero).
     """
     if not (s > 0.0) or not np.isfinite(s):
         raise ValueError("sparsity budget s must be a positive finite number")
@@ -149,29 +153,21 @@ def atomo_probabilities(lam: np.ndarray, s: float) -> Tuple[np.ndarray, int, flo
     n = a.size
     order = np.argsort(-a, kind="stable")          # |lambda_1| >= ... >= |lambda_n|
     a_sorted = a[order]
-    # tail[i] = sum_{j >= i} |lambda_j|, accumulated from the small end
-    tail = np.cumsum(a_sorted[::-1])[::-1] if n else a_sorted
+    tail = np.cumsum(a_sorted[::-1])[::-1] if n else a_sorted      # tail[i] = sum_{j >= i} |lambda_j|, from the small end
+    budget = float(s) - np.arange(n, dtype=np.float64)             # what is left after i atoms were given p = 1
+    balanced = a_sorted * budget <= tail                           # the remaining atoms are budget-balanced from i on
+    # an atom with lambda = 0 is never given p = 1: where it comes first its tail is 0 and the test holds (0 <= 0), so a
+    # budget s >= n ends with p = 1 exactly on the non-zero atoms
+    n_s = int(np.argmax(balanced)) if balanced.any() else n
     p_sorted = np.zeros(n, dtype=np.float64)
-    s_cur = float(s)
-    i = 0
+    p_sorted[:n_s] = 1.0
     c = 0.0
-    while i < n:
-        t_i = float(tail[i])
-        if a_sorted[i] * s_cur <= t_i:
-            if t_i > 0.0:
-                p_sorted[i:] = a_sorted[i:] * s_cur / t_i
-                c = t_i / s_cur
-            # t_i == 0: every remaining atom has lambda = 0 and keeps p = 0
-            break
-        p_sorted[i] = 1.0
-        s_cur -= 1.0
-        i += 1
-    n_s = i if i < n else n
-    # an atom with lambda = 0 is never set to 1: if the loop reaches it, its tail is 0 and the
-    # first branch fires (0 <= 0); budgets s >= n therefore end with p = 1 exactly on non-zeros
+    if n_s < n and tail[n_s] > 0.0:
+        p_sorted[n_s:] = a_sorted[n_s:] * budget[n_s] / tail[n_s]
+        c = float(tail[n_s] / budget[n_s])
     p = np.empty(n, dtype=np.float64)
     p[order] = p_sorted
-    return p, int(n_s), float(c)
+    return p, n_s, float(c)
 
 
 # --------------------------------------------------------------------------------------
