@@ -30,7 +30,9 @@ UNIT = "elements/s"
 L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (None: no capture on file for that kernel and workload)
-NCU_TRAFFIC = {("sp_tridiag_cluster_kernel", "c2"): 5638912}
+NCU_TRAFFIC = {("sp_tridiag_cluster_kernel", "c2"): 5638912,
+               # profiles/sp_tridiag_big1_c5.txt: 1.661 TB/s of DRAM traffic over the 31.55 ms of the captured launch
+               ("sp_tridiag_big_kernel", "c5"): 52_400_000_000}
 
 
 def measured_peaks():
@@ -126,14 +128,30 @@ ENTRYWISE = {
 }
 
 
+FAST_INPUTS = False      # --fast-inputs: one generated matrix per distinct shape, the others by row / column permutations
+
+
 def make_spectral_inputs(name, seed, dev):
-    """One input set of a spectral workload on the device (torch generator: the recipe of synth.lowrank_plus_noise)."""
+    """One input set of a spectral workload on the device (torch generator: the recipe of synth.lowrank_plus_noise).
+    With --fast-inputs (for profiler captures, where every launch costs) only the first matrix of each shape is
+    generated; the others are that matrix with its rows and columns permuted and random signs (the same spectrum,
+    factors again Haar distributed)."""
+    import torch
     from paper_1806_04090_b200 import synth
     cfg = SPECTRAL[name]
-    out = []
+    out, base = [], {}
     for i, (m, n) in enumerate(spectral_shapes(name)):
-        out.append(synth.torch_lowrank_plus_noise(m, n, cfg["decay"], seed * 1000 + i, dev, noise_rel=cfg.get("noise_rel"),
-                                                  noise_std=cfg.get("noise_std")))
+        if FAST_INPUTS and (m, n) in base:
+            gen = torch.Generator(device=dev); gen.manual_seed(seed * 1000 + i)
+            g0 = base[(m, n)]
+            pr, pc = torch.randperm(m, device=dev, generator=gen), torch.randperm(n, device=dev, generator=gen)
+            sr = (torch.randint(0, 2, (m, 1), device=dev, generator=gen) * 2 - 1).to(torch.float32)
+            out.append((g0[pr][:, pc] * sr).contiguous())
+            continue
+        g = synth.torch_lowrank_plus_noise(m, n, cfg["decay"], seed * 1000 + i, dev, noise_rel=cfg.get("noise_rel"),
+                                           noise_std=cfg.get("noise_std"))
+        base[(m, n)] = g
+        out.append(g)
     return out
 
 
@@ -287,7 +305,7 @@ def roofline_for(run, eig_ms_per_step, eig_launches_per_step, scheme, peaks, fma
         # the blocked reduction dominates whenever it runs (config 3: also one launch of the small-layer kernel in the stage)
         b = tridiag_big_bytes(shapes)
         ach = b / (eig_ms_per_step * 1e-3) / 1e9
-        out.update(bound="hbm", kernel="sp_tridiag_big_kernel", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+        out.update(bound="hbm", kernel="sp_tridiag_big1_kernel (one CTA per layer)" if max(min(sh) for sh in shapes) <= 1024 and len(shapes) >= 75 else "sp_tridiag_big_kernel (clusters)", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
                    frac=ach / peaks["hbm_gbs"], traffic=NCU_TRAFFIC.get(("sp_tridiag_big_kernel", run.name)),
                    peak_source=f"{peaks['source']} copy bandwidth (MEASURED_PEAKS.json)",
                    algorithmic="one triangle of the trailing block per Householder step, 4-byte entries: (2/3) r^3 bytes per layer",
@@ -455,10 +473,12 @@ def run_ours(args):
         run.step(w)
     torch.cuda.synchronize()
     a.set_profiling(True)
+    uploads0 = a.table_uploads()
     dist.barrier(); torch.cuda.synchronize()
     if rank == 0:
         sampler.mark()
     reps_ms = timed_reps(run, args.steps, 0, args.reps, first=args.warmup)
+    uploads1 = a.table_uploads()
     torch.cuda.synchronize(); dist.barrier()
     clocks = sampler.stop() if rank == 0 else None
     reps_ms = [dist.max_over_ranks(m, dev) for m in reps_ms]
@@ -468,7 +488,7 @@ def run_ours(args):
     ms_per_step = float(np.median(reps_ms))
     value = world * elems / (ms_per_step * 1e-3)
     scheme = a.last_eig_scheme() if run.spectral else None
-    launches = (sum(tot_ln.values()) + n_steps * (9 + 3)) / args.reps   # + table / header copies and memsets per step, per run of K steps
+    launches = (sum(tot_ln.values()) + n_steps * 3) / args.reps   # + the header kernel and the workspace memsets per step; per run of K steps
 
     # ---- end to end: host buffers, copies inside the timed region ----
     # Every step's inputs come from pinned host memory and its decoded gradients go back to pinned host memory.
@@ -547,6 +567,8 @@ def run_ours(args):
                     "ms_per_step": e2e_ms / e2e_steps, "steps": e2e_steps,
                     "overlap": "copies of step k+1 (in) and k-1 (out) run on two copy streams under step k's kernels"},
             "gpu_launches": int(launches),
+            "table_uploads_in_timed_region": {"uploads": uploads1[0] - uploads0[0], "calls_served_from_device": uploads1[1] - uploads0[1],
+                                              "note": "host-to-device copies of descriptor tables inside the timed region (0 in steady state)"},
             "measured_fma_peaks_tflops": fma_peaks,
         }
         if run.spectral:
@@ -595,8 +617,13 @@ def main():
                          "the payloads, then decode their average; p2p: the averaging decode reads the peers' payloads "
                          "in place over NVLink")
     ap.add_argument("--no-extras", action="store_true", help="skip the `also` entries (the other configurations)")
+    ap.add_argument("--fast-inputs", action="store_true",
+                    help="generate one matrix per distinct shape and derive the others by permutations and signs "
+                         "(profiler captures: thousands of generator launches less)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    global FAST_INPUTS
+    FAST_INPUTS = bool(args.fast_inputs)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -103,10 +103,29 @@ __device__ __forceinline__ double tb_dot(const X* __restrict__ x, const T* __res
   return acc;
 }
 
+// the same for one of `nsub` warps that share a dot: 32-element blocks of [h0, r) are dealt to the warps in turn
+template <typename X, typename T>
+__device__ __forceinline__ double tb_dot_part(const X* __restrict__ x, const T* __restrict__ u, int h0, int r, int lane,
+                                              int sub, int nsub) {
+  double acc = 0.0;
+  int h = h0 + 32 * sub + lane;
+  const int stride = 32 * nsub;
+  for (; h + 3 * stride < r; h += 4 * stride) {
+    X xb[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) xb[j] = __ldcg(x + h + stride * j);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc = fma((double)xb[j], (double)u[h + stride * j], acc);
+  }
+  for (; h < r; h += stride) acc = fma((double)__ldcg(x + h), (double)u[h], acc);
+  return acc;
+}
+
 struct alignas(16) TbShared {
   double part_a[kTbMaxBlocks];     // per 32-row block: ||x||^2 partial of the current column
   double part_k[kTbMaxBlocks];     // per 32-row block: u^T p partial
   double dots[2 * kTbNB];          // a_t = w_t^T u, b_t = u_t^T u of the panel's earlier reflectors
+  double dot_part[4][8];           // a dot's eight warp partials (four dots in progress per CTA)
   double pc[2 * kTbNB];            // u_t[c], w_t[c]: the panel's entries in row c
   double y[kTbThreads];            // A0 u for this CTA's rows (local row order)
   double x0;                       // first entry of the pivot column
@@ -281,16 +300,32 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
         }
       }
       TB_MARK(2)
-      for (int id = w; id < 2 * i; id += kTbWarps) {
-        const int t = id >> 1;
-        double acc = 0.0;
-        if (id & 1) acc = tb_dot(V + (int64_t)(p0 + t) * ldv, s_u, c + 1, r, lane);
-        else acc = tb_dot(W + (int64_t)t * ldw, s_u, c + 1, r, lane);
-        acc = warp_sum(acc);
-        if (lane == 0) S.dots[id] = acc;
+      // Panel dots.  Dot number id belongs to CTA id mod C; eight warps share a dot (32-element blocks dealt in turn)
+      // and their partial sums are added in warp order -- the same order whatever C is.  The owner sends the result to
+      // every CTA of the cluster.
+      for (int k0 = 0; q + C * k0 < 2 * i; k0 += 4) {
+        const int id = q + C * (k0 + (w >> 3));
+        if (id < 2 * i) {
+          const int t = id >> 1;
+          double acc = (id & 1) ? tb_dot_part(V + (int64_t)(p0 + t) * ldv, s_u, c + 1, r, lane, w & 7, 8)
+                                : tb_dot_part(W + (int64_t)t * ldw, s_u, c + 1, r, lane, w & 7, 8);
+          acc = warp_sum(acc);
+          if (lane == 0) S.dot_part[w >> 3][w & 7] = acc;
+        }
+        __syncthreads();
+        if (tid < 4) {
+          const int id2 = q + C * (k0 + tid);
+          if (id2 < 2 * i) {
+            double tot = 0.0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) tot += S.dot_part[tid][j];
+            bcast(&S.dots[id2], tot);
+          }
+        }
+        __syncthreads();
       }
     }
-    __syncthreads();
+    sync_all();                                                              // the other CTAs' dots have arrived
     TB_MARK(3)
     // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
     double p = 0.0;
@@ -854,7 +889,21 @@ __global__ void __launch_bounds__(kVbThreads) sp_eigvec_big_kernel(const SpLayer
       const float m1 = top - 1 >= 0 ? 1.0f : 0.0f, m2 = top - 2 >= 0 ? 1.0f : 0.0f, m3 = top - 3 >= 0 ? 1.0f : 0.0f;
       const int h0 = max(top - 3, 0) + 1;
       float z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
-      for (int h = h0 + lane; h < r; h += 32) {
+      int h = h0 + lane;
+      for (; h + 96 < r; h += 128) {                                           // sixteen loads in flight
+        float q0[4], q1[4], q2[4], q3[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { q0[j] = v0[h + 32 * j]; q1[j] = v1[h + 32 * j]; q2[j] = v2[h + 32 * j]; q3[j] = v3[h + 32 * j]; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float zh = z[h + 32 * j];
+          const float r0 = q0[j], r1 = m1 * q1[j], r2 = m2 * q2[j], r3 = m3 * q3[j];
+          z0 = fmaf(r0, zh, z0); z1 = fmaf(r1, zh, z1); z2 = fmaf(r2, zh, z2); z3 = fmaf(r3, zh, z3);
+          g10 = fmaf(r1, r0, g10); g20 = fmaf(r2, r0, g20); g21 = fmaf(r2, r1, g21);
+          g30 = fmaf(r3, r0, g30); g31 = fmaf(r3, r1, g31); g32 = fmaf(r3, r2, g32);
+        }
+      }
+      for (; h < r; h += 32) {
         const float zh = z[h];
         const float r0 = v0[h], r1 = m1 * v1[h], r2 = m2 * v2[h], r3 = m3 * v3[h];
         z0 = fmaf(r0, zh, z0); z1 = fmaf(r1, zh, z1); z2 = fmaf(r2, zh, z2); z3 = fmaf(r3, zh, z3);
@@ -873,7 +922,15 @@ __global__ void __launch_bounds__(kVbThreads) sp_eigvec_big_kernel(const SpLayer
       const float c1 = 2.0f * (z1 - c0 * g10);
       const float c2 = 2.0f * (z2 - c0 * g20 - c1 * g21);
       const float c3 = 2.0f * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
-      for (int h = h0 + lane; h < r; h += 32)
+      h = h0 + lane;
+      for (; h + 96 < r; h += 128) {
+        float q0[4], q1[4], q2[4], q3[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { q0[j] = v0[h + 32 * j]; q1[j] = v1[h + 32 * j]; q2[j] = v2[h + 32 * j]; q3[j] = v3[h + 32 * j]; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) z[h + 32 * j] -= fmaf(c0, q0[j], fmaf(c1, m1 * q1[j], fmaf(c2, m2 * q2[j], c3 * m3 * q3[j])));
+      }
+      for (; h < r; h += 32)
         z[h] -= fmaf(c0, v0[h], fmaf(c1, m1 * v1[h], fmaf(c2, m2 * v2[h], c3 * m3 * v3[h])));
       __syncwarp();
     }

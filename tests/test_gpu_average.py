@@ -47,6 +47,29 @@ def test_spectral_average_matches_mean_of_decodes(atomo):
         assert torch.equal(one[l], singles[0][l])
 
 
+def test_spectral_average_against_oracle(atomo, oracle):
+    """The averaging decode against the oracle's definition of the combine step: the mean over the workers of the
+    oracle's decode (Eq. 2) of each worker's own kept atoms."""
+    import torch
+    from paper_1806_04090_b200 import api
+    mats = _spectral_layers()
+    ts = [torch.from_numpy(m).cuda() for m in mats]
+    pays = []
+    for worker in range(4):
+        buf = torch.empty(api.payload_bytes_spectral([m.shape for m in mats], 16), dtype=torch.uint8, device="cuda")
+        pay, _ = atomo.atomo_encode_spectral(ts, 2.5, seed=300 + worker, step=2, k_cap=16, payload=buf)
+        assert max(h.status for h in pay.headers()[1]) == 0
+        pays.append(pay)
+    avg = atomo.atomo_decode_average(pays)
+    for l, G in enumerate(mats):
+        want = np.zeros(G.shape)
+        for pay in pays:
+            arr = pay.layer_arrays(l)
+            want += oracle.decode_spectral(arr["coef"], arr["U"], arr["V"])
+        want /= len(pays)
+        assert parity.rel(avg[l].cpu().numpy(), want) <= 1e-5
+
+
 def test_entrywise_average_against_oracle(atomo, oracle):
     import torch
     from paper_1806_04090_b200 import api

@@ -110,6 +110,20 @@ def test_paper_reshape_family(atomo, oracle):
     _run(atomo, oracle, mats, 2.0, seed=17, step=1)
 
 
+@pytest.mark.parametrize("scheme", [0, 1, 2])
+def test_jacobi_launch_schemes_against_oracle(atomo, oracle, scheme):
+    """Each launch form of the Jacobi fallback (one launch per step, persistent cooperative launches, clusters)
+    directly against the oracle, full protocol."""
+    L = synth.RESNET18_LAYERS
+    mats = synth.c2_resnet18(3, [L[0], L[1], L[5], L[9], L[17]])
+    try:
+        atomo.set_persistent_eig(scheme)
+        _run(atomo, oracle, mats, 2.0, seed=77, step=3)
+        assert atomo.last_eig_scheme() == scheme
+    finally:
+        atomo.set_persistent_eig(3)
+
+
 def test_eigen_launch_schemes_agree(atomo):
     """One launch per step, persistent cooperative launches and the cluster form run the same rotations in the same
     order per layer: identical masks and singular values to rounding (the forms fold the row factors at different
