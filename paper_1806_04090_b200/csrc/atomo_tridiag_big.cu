@@ -52,6 +52,7 @@ constexpr int kTbNB = 32;                    // columns per panel
 constexpr int kTbMaxC = 16;                  // CTAs per cluster
 constexpr int kTbMaxR = 4096;
 constexpr int kTbMaxBlocks = kTbMaxR / 32;   // 32-row blocks of a layer
+constexpr int kTbPanRows = 256;              // rows per CTA up to which the panel entries of the CTA's rows live in shared memory
 
 template <typename T> struct Vec4;           // 16-byte (float) / 32-byte (double) groups of four matrix entries
 template <> struct Vec4<float> { using type = float4; };
@@ -135,7 +136,7 @@ struct alignas(16) TbShared {
 
 template <typename T, int C>
 __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpLayer* __restrict__ layers,
-                                                                       const int* __restrict__ big_layers) {
+                                                                       const int* __restrict__ big_layers, int use_pan) {
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) unsigned char tb_smem[];
   TbShared& S = *reinterpret_cast<TbShared*>(tb_smem);
@@ -155,6 +156,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   const int nblk = (r + 31) / 32;
   const int r4 = (r + 3) & ~3;
   T* const s_gemm = s_u + r4;                                                  // operand tiles of the panel update
+  // use_pan: this CTA holds at most kTbPanRows rows, and the panel entries of its own rows (u_t[g], w_t[g]) are kept in
+  // shared memory beside their copies in global memory: the column update and the correction of y then read them there
+  // instead of from L2 (two dependent round trips per step less)
+  constexpr int TRg = sizeof(T) == 4 ? 4 : 2;
+  T* const pan_u = s_gemm + 2 * kTbNB * 32 * TRg + 2 * kTbNB * 128;            // [kTbNB][kTbPanRows]
+  T* const pan_w = pan_u + kTbNB * kTbPanRows;
   // this thread's row: block (tid / 32) of this CTA = global block (tid / 32) * C + q
   const int gb = w * C + q;
   const int g = gb * 32 + lane;
@@ -187,6 +194,10 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     double a = 0.0;
     if (valid && g >= c) {
       a = (double)__ldcg(A + (int64_t)c * lda + g);
+      if (use_pan) {
+        for (int t = 0; t < i; ++t)
+          a -= (double)pan_u[t * kTbPanRows + tid] * S.pc[2 * t + 1] + (double)pan_w[t * kTbPanRows + tid] * S.pc[2 * t];
+      } else
       for (int t0 = 0; t0 < i; t0 += 8) {                                       // eight reflectors' entries in flight
         float ub[8]; T wb[8];
 #pragma unroll
@@ -224,6 +235,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     if (valid) {
       if (live) u_own = (double)(T)((a - (g == c + 1 ? alpha : 0.0)) * inv);   // the stored precision is the one used
       V[(int64_t)c * ldv + g] = (float)u_own;
+      if (use_pan) pan_u[(c - p0) * kTbPanRows + tid] = (T)u_own;
       if (g == c + 1) td_e[c] = alpha;
       if (C == 1) s_u[g] = (T)u_own;
       else {
@@ -331,6 +343,10 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     double p = 0.0;
     if (live) {
       double y = S.y[tid];
+      if (use_pan) {
+        for (int t = 0; t < i; ++t)
+          y -= (double)pan_u[t * kTbPanRows + tid] * S.dots[2 * t] + (double)pan_w[t * kTbPanRows + tid] * S.dots[2 * t + 1];
+      } else
       for (int t0 = 0; t0 < i; t0 += 8) {
         float ub[8]; T wb[8];
 #pragma unroll
@@ -350,7 +366,11 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     }
     sync_all();
     const double K = tb_ordered_sum(S.part_k, nblk, lane);
-    if (valid) W[(int64_t)(c - p0) * ldw + g] = (T)(live ? p - K * u_own : 0.0);
+    if (valid) {
+      const T wv = (T)(live ? p - K * u_own : 0.0);
+      W[(int64_t)(c - p0) * ldw + g] = wv;
+      if (use_pan) pan_w[(c - p0) * kTbPanRows + tid] = wv;
+    }
     const bool flush = (c - p0 == kTbNB - 1) || (c == n_ref - 1);
     if (!flush) { sync_all(); TB_MARK(4) continue; }
     TB_MARK(4)
@@ -380,7 +400,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
           s_ur[t * MR + e % MR] = in ? (T)__ldcg(V + (int64_t)(p0 + t) * ldv + gr) : (T)0;
           s_wr[t * MR + e % MR] = in ? __ldcg(W + (int64_t)t * ldw + gr) : (T)0;
         }
+        // fp32: a warp's piece of a tile is one 32-row block by 16 columns.  A piece strictly above the diagonal is not
+        // computed: its mirror image, a piece strictly below the diagonal in another block's rows, writes both (the
+        // update is symmetric and so is A0).  Pieces that meet the diagonal are computed and written as they are.
+        const int tile_row_end = (lb_last * C + q) * 32 + 31;
         for (int hc0 = g0 & ~127; hc0 < r; hc0 += 128) {
+          if (sizeof(T) == 4 && hc0 > tile_row_end) break;                      // every piece of this and the later chunks lies above the diagonal
           __syncthreads();
           for (int e = tid; e < nr * 128; e += kTbThreads) {
             const int t = e >> 7, h = hc0 + (e & 127);
@@ -388,13 +413,20 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
             s_wc[e] = h < r ? __ldcg(W + (int64_t)t * ldw + h) : (T)0;
           }
           __syncthreads();
+          const int lr0 = wr * (8 * TR) + ly * TR;                             // first local row (in the tile) of this thread
+          const int lc0 = wc * 16 + lx * 4;
+          bool mirror = false;
+          if (sizeof(T) == 4) {
+            const int blk_start = (((mr0 >> 5) + wr) * C + q) * 32;            // this warp's 32-row block
+            const int pc_start = hc0 + 16 * wc;
+            if (pc_start > blk_start + 31) continue;                           // above the diagonal: written by its mirror image
+            mirror = pc_start + 15 < blk_start;
+          }
           T acc[TR][4];
 #pragma unroll
           for (int x = 0; x < TR; ++x)
 #pragma unroll
             for (int y = 0; y < 4; ++y) acc[x][y] = 0;
-          const int lr0 = wr * (8 * TR) + ly * TR;                             // first local row (in the tile) of this thread
-          const int lc0 = wc * 16 + lx * 4;
           for (int t = 0; t < nr; ++t) {
             T ru[TR], rw[TR];
             load_rows<T>(s_ur + t * MR + lr0, ru);
@@ -409,19 +441,40 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
               acc[x][2] = fma(rw[x], cu.z, acc[x][2]); acc[x][3] = fma(rw[x], cu.w, acc[x][3]);
             }
           }
+          const int h = hc0 + lc0;
+          const int lrf = mr0 + lr0;
+          const int grf = ((lrf >> 5) * C + q) * 32 + (lrf & 31);              // first global row of this thread (its TR rows are consecutive)
 #pragma unroll
           for (int x = 0; x < TR; ++x) {
-            const int lr = mr0 + lr0 + x;
-            const int gr = ((lr >> 5) * C + q) * 32 + (lr & 31);
-            const int h = hc0 + lc0;
-            if ((lr >> 5) >= n_lblk || gr >= r || gr < g0 || h >= r) continue;
-            T* dst = A + (int64_t)gr * lda + h;
-            if (h + 3 < r) {
-              typename Vec4<T>::type o = ldcg4(dst);
-              o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
-              st4(dst, o);
-            } else {
-              for (int y = 0; y < 4 && h + y < r; ++y) dst[y] = __ldcg(dst + y) - acc[x][y];
+            const int gr = grf + x;
+            const bool on = (lrf >> 5) < n_lblk && gr < r && gr >= g0 && h < r;
+            if (on) {
+              T* dst = A + (int64_t)gr * lda + h;
+              if (h + 3 < r) {
+                typename Vec4<T>::type o = ldcg4(dst);
+                o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
+                st4(dst, o);
+                acc[x][0] = o.x; acc[x][1] = o.y; acc[x][2] = o.z; acc[x][3] = o.w;   // the new entries, for the mirror image
+              } else {
+                for (int y = 0; y < 4 && h + y < r; ++y) { const T o = __ldcg(dst + y) - acc[x][y]; dst[y] = o; acc[x][y] = o; }
+              }
+            }
+          }
+          if (mirror && (lrf >> 5) < n_lblk) {
+            // A0[h + y][grf .. grf + TR - 1] = the new A0[grf .. ][h + y]: rows h + y >= g0 only (the others are dead)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) {
+              const int hr = h + y;
+              if (hr < g0 || hr >= r) continue;
+              T* dst = A + (int64_t)hr * lda + grf;
+              if (TR == 4 && grf >= g0 && grf + 3 < r) {
+                typename Vec4<T>::type o;
+                o.x = acc[0][y]; o.y = acc[1][y]; o.z = acc[TR > 2 ? 2 : 0][y]; o.w = acc[TR > 2 ? 3 : 0][y];
+                st4(dst, o);
+              } else {
+#pragma unroll
+                for (int x = 0; x < TR; ++x) if (grf + x >= g0 && grf + x < r) dst[x] = acc[x][y];
+              }
             }
           }
         }
@@ -982,7 +1035,7 @@ namespace {
 template <typename T> size_t tb_smem_bytes(int r_max) {
   constexpr int TR = sizeof(T) == 4 ? 4 : 2;
   const size_t r4 = (size_t)((r_max + 3) & ~3);
-  return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128) * sizeof(T);
+  return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128 + (sizeof(T) == 4 ? 2 * (size_t)kTbNB * kTbPanRows : 0)) * sizeof(T);
 }
 size_t t1_smem_bytes() {
   return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + (size_t)kT1MaxB * kT1MaxB * kT1Blk);
@@ -1005,7 +1058,10 @@ int tb_launch_one(const SpLayer* d_layers, const int* d_big, int n_big, int r_ma
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
   cfg.attrs = at; cfg.numAttrs = 1;
-  return (int)cudaLaunchKernelEx(&cfg, sp_tridiag_big_kernel<T, C>, d_layers, d_big);
+  // rows per CTA: the 32-row blocks of the largest layer dealt to C CTAs
+  const int rows_per_cta = ((r_max + 31) / 32 + C - 1) / C * 32;
+  const int use_pan = (sizeof(T) == 4 && rows_per_cta <= kTbPanRows) ? 1 : 0;   // fp32 only: the fp64 tiles leave no room
+  return (int)cudaLaunchKernelEx(&cfg, sp_tridiag_big_kernel<T, C>, d_layers, d_big, use_pan);
 }
 
 }  // namespace
