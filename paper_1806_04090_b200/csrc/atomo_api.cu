@@ -24,9 +24,21 @@ struct TableCache {
   cudaStream_t last_stream = nullptr;
 };
 
+// A few caches side by side, found by a key over the caller's pointers and shapes: an application that alternates
+// between a few sets of buffers (double-buffered gradients, several payloads in flight) still uploads nothing in
+// steady state.  The key only picks the way; whether an upload is needed is decided on the table bytes themselves.
+struct TableWays {
+  static constexpr int kWays = 8;
+  TableCache way[kWays];
+  uint64_t key[kWays] = {};
+  uint64_t used[kWays] = {};                   // 0 = never used, else the tick of the last use
+  uint64_t tick = 0;
+};
+
 struct atomo_ctx {
   int device = 0;
-  TableCache tab_sp, tab_dec, tab_avg, tab_ew;
+  TableWays tab_sp, tab_dec, tab_avg;
+  TableCache tab_ew;
   int64_t table_uploads = 0, table_reuses = 0;
   uint8_t* ws = nullptr;
   size_t ws_bytes = 0;
@@ -84,6 +96,28 @@ int fail_cuda(atomo_ctx* ctx, cudaError_t e, const char* what) {
     cudaError_t e__ = (call);                                               \
     if (e__ != cudaSuccess) return fail_cuda(ctx, e__, #call);              \
   } while (0)
+
+// FNV-1a over a block of bytes, chained through h
+uint64_t table_key(uint64_t h, const void* data, size_t bytes) {
+  const uint8_t* b = static_cast<const uint8_t*>(data);
+  for (size_t i = 0; i < bytes; ++i) { h ^= b[i]; h *= 1099511628211ull; }
+  return h;
+}
+constexpr uint64_t kKeySeed = 1469598103934665603ull;
+
+// the way that served this key last, else a way never used, else the one unused for longest
+TableCache& table_pick(TableWays& tw, uint64_t key) {
+  int pick = -1;
+  for (int i = 0; i < TableWays::kWays; ++i) if (tw.used[i] && tw.key[i] == key) { pick = i; break; }
+  if (pick < 0) {
+    pick = 0;
+    for (int i = 1; i < TableWays::kWays; ++i) if (tw.used[i] < tw.used[pick]) pick = i;
+  }
+  tw.key[pick] = key; tw.used[pick] = ++tw.tick;
+  return tw.way[pick];
+}
+void table_free(TableCache& tc);
+void table_free(TableWays& tw) { for (auto& w : tw.way) table_free(w); }
 
 // device buffer of at least `bytes` for a table cache (growing it forgets the cached contents)
 int table_reserve(atomo_ctx* ctx, TableCache& tc, size_t bytes) {
@@ -569,8 +603,13 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
   atomo_layer_header* d_hdr_tmpl = nullptr;
   std::vector<uint8_t> tables;
   size_t table_bytes = 0;
+  uint64_t tkey = table_key(kKeySeed, layers, (size_t)n_layers * sizeof(atomo_mat));
+  tkey = table_key(tkey, &payload, sizeof(payload));
+  tkey = table_key(tkey, &k_cap, sizeof(k_cap));
+  if (given) { tkey = table_key(tkey, given_sigma, (size_t)n_layers * sizeof(float*)); tkey = table_key(tkey, given_short, (size_t)n_layers * sizeof(float*)); }
+  TableCache& tab = table_pick(ctx->tab_sp, tkey);
   for (int pass = 0; pass < 2; ++pass) {
-    Arena T(pass ? ctx->tab_sp.d : nullptr);
+    Arena T(pass ? tab.d : nullptr);
     d_layers = T.take<SpLayer>(n_layers);
     d_gram = T.take<TileRef>(gram_tiles.size());
     d_pairs = T.take<TileRef>(block_pairs.size());
@@ -584,11 +623,11 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     d_given = T.take<const float*>(given ? (size_t)2 * n_layers : 0);
     d_hdr_tmpl = T.take<atomo_layer_header>(n_layers);
     table_bytes = T.off + 256;
-    if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_sp, table_bytes); if (rc != ATOMO_OK) return rc; }
+    if (pass == 0) { const int rc = table_reserve(ctx, tab, table_bytes); if (rc != ATOMO_OK) return rc; }
   }
   tables.assign(table_bytes, 0);
   auto put = [&](const void* dev_ptr, const void* src, size_t bytes) {
-    if (bytes) std::memcpy(tables.data() + (reinterpret_cast<const uint8_t*>(dev_ptr) - ctx->tab_sp.d), src, bytes);
+    if (bytes) std::memcpy(tables.data() + (reinterpret_cast<const uint8_t*>(dev_ptr) - tab.d), src, bytes);
   };
   uint8_t* zero_beg = nullptr; size_t zero_bytes = 0;
   size_t need = 0;
@@ -686,7 +725,7 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     for (int l = 0; l < n_layers; ++l) { ptrs[l] = given_sigma[l]; ptrs[n_layers + l] = given_short[l]; }
     put(d_given, ptrs.data(), ptrs.size() * sizeof(const float*));
   }
-  { const int rc = table_commit(ctx, ctx->tab_sp, tables.data(), table_bytes, st); if (rc != ATOMO_OK) return rc; }
+  { const int rc = table_commit(ctx, tab, tables.data(), table_bytes, st); if (rc != ATOMO_OK) return rc; }
   launch_sp_begin(pay, gh, d_hdr_tmpl, n_layers, d_flag, st);          // payload header, layer headers, flags
   CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
 
@@ -1018,17 +1057,20 @@ int atomo_decode(atomo_ctx* ctx, int32_t kind, const void* payload, const int64_
     }
     SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
     size_t tb = 0;
+    uint64_t key = table_key(kKeySeed, &payload, sizeof(payload));
+    key = table_key(key, out, (size_t)n_layers * sizeof(float*));
+    TableCache& tab = table_pick(ctx->tab_dec, key);
     for (int pass = 0; pass < 2; ++pass) {
-      Arena T(pass ? ctx->tab_dec.d : nullptr);
+      Arena T(pass ? tab.d : nullptr);
       d_layers = T.take<SpDecodeLayer>(n_layers);
       d_tiles = T.take<TileRef>(tiles.size());
       tb = T.off + 256;
-      if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_dec, tb); if (rc != ATOMO_OK) return rc; }
+      if (pass == 0) { const int rc = table_reserve(ctx, tab, tb); if (rc != ATOMO_OK) return rc; }
     }
     std::vector<uint8_t> tables(tb, 0);
-    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - ctx->tab_dec.d), D.data(), D.size() * sizeof(SpDecodeLayer));
-    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - ctx->tab_dec.d), tiles.data(), tiles.size() * sizeof(TileRef));
-    { const int rc = table_commit(ctx, ctx->tab_dec, tables.data(), tb, st); if (rc != ATOMO_OK) return rc; }
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - tab.d), D.data(), D.size() * sizeof(SpDecodeLayer));
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - tab.d), tiles.data(), tiles.size() * sizeof(TileRef));
+    { const int rc = table_commit(ctx, tab, tables.data(), tb, st); if (rc != ATOMO_OK) return rc; }
     launch_sp_decode(pay, d_layers, d_tiles, (int)tiles.size(), st);
     stage_end(ctx, ATOMO_STAGE_DECODE, st, 1);
   }
@@ -1062,20 +1104,23 @@ int atomo_decode_average(atomo_ctx* ctx, int32_t kind, const void* const* payloa
   }
   const uint8_t** d_pay = nullptr; SpDecodeLayer* d_layers = nullptr; TileRef* d_tiles = nullptr;
   size_t tb = 0;
+  uint64_t key = table_key(kKeySeed, payloads, (size_t)n_payloads * sizeof(void*));
+  key = table_key(key, out, (size_t)n_layers * sizeof(float*));
+  TableCache& tab = table_pick(ctx->tab_avg, key);
   for (int pass = 0; pass < 2; ++pass) {
-    Arena T(pass ? ctx->tab_avg.d : nullptr);
+    Arena T(pass ? tab.d : nullptr);
     d_pay = T.take<const uint8_t*>(n_payloads);
     d_layers = T.take<SpDecodeLayer>(D.size());
     d_tiles = T.take<TileRef>(tiles.size());
     tb = T.off + 256;
-    if (pass == 0) { const int rc = table_reserve(ctx, ctx->tab_avg, tb); if (rc != ATOMO_OK) return rc; }
+    if (pass == 0) { const int rc = table_reserve(ctx, tab, tb); if (rc != ATOMO_OK) return rc; }
   }
   {
     std::vector<uint8_t> tables(tb, 0);
-    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_pay) - ctx->tab_avg.d), payloads, (size_t)n_payloads * sizeof(void*));
-    if (!D.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - ctx->tab_avg.d), D.data(), D.size() * sizeof(SpDecodeLayer));
-    if (!tiles.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - ctx->tab_avg.d), tiles.data(), tiles.size() * sizeof(TileRef));
-    const int rc = table_commit(ctx, ctx->tab_avg, tables.data(), tb, st);
+    std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_pay) - tab.d), payloads, (size_t)n_payloads * sizeof(void*));
+    if (!D.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_layers) - tab.d), D.data(), D.size() * sizeof(SpDecodeLayer));
+    if (!tiles.empty()) std::memcpy(tables.data() + (reinterpret_cast<uint8_t*>(d_tiles) - tab.d), tiles.data(), tiles.size() * sizeof(TileRef));
+    const int rc = table_commit(ctx, tab, tables.data(), tb, st);
     if (rc != ATOMO_OK) return rc;
   }
   stage_begin(ctx, ATOMO_STAGE_DECODE, st);

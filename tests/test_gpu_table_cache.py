@@ -40,6 +40,19 @@ def test_tables_are_reused_and_refreshed():
     assert up2 == up1 + 1                                   # the encode's tables; the decode's did not change
     for o, r in zip(outs, ref):
         assert torch.equal(o, r)
+    # alternating between a few sets of buffers (double or triple buffering): each set keeps its own tables, so after
+    # one round over the sets nothing is uploaded any more
+    sets = [ts, ts2, [t.clone() for t in ts]]
+    for j, layers in enumerate(sets):
+        step(layers, 5)
+    up_a, _ = a.table_uploads()
+    for rnd in range(3):
+        for layers in sets:
+            step(layers, 5)
+            for o, r in zip(outs, ref):
+                assert torch.equal(o, r)
+    up_b, _ = a.table_uploads()
+    assert up_b == up_a, "alternating between three sets of buffers uploaded tables again"
     # entry-wise: the header template travels through the same mechanism
     g = torch.from_numpy(synth.c1_entrywise(0)).cuda()
     pe, _ = a.atomo_encode_entrywise([g], 64.0, seed=1, step=0, k_cap=4096)
