@@ -181,6 +181,13 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/,
  * on the format.  A vector whose kept unsaturated atoms exceed k_cap or whose saturated atoms exceed sat_cap
  * gets ATOMO_ERR_CAPACITY in its status word and k = 0.  Decoders read the format from the payload.       */
 int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap);
+/* Launch form of the context's later atomo_encode_entrywise calls.  two_kernels = 0 (default): a vector whose tiles
+ * fit one wave of resident CTAs (up to about 48 million elements on a B200) is encoded by ONE cooperative kernel -- a CTA
+ * computes its part of sum |g| and max |g| (Algorithm 1's inputs), all CTAs meet at a grid barrier, and the same CTA
+ * then samples and packs the part it has just read, which is still in the L2 cache on its side of the chip; longer
+ * vectors take the two-kernel form.  two_kernels = 1: always a solve kernel followed by a sample / pack kernel whose
+ * chunks are handed out by ticket.  Payloads, masks and decoded gradients are bit-identical in both forms.     */
+int atomo_set_entrywise_launch(atomo_ctx* ctx, int32_t two_kernels);
 
 /* --- l_q budgets (Section 4) ------------------------------------------------------------------
  * s_out[l] (HOST) = ||g_l||_1 / ||g_l||_q for every vector: the budget at which entry-wise ATOMO is the

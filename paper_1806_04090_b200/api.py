@@ -33,6 +33,7 @@ EXPORTS = [
     "atomo_set_eig_params", "atomo_set_eig_mode", "atomo_set_sigma_refinement", "atomo_set_gram_path", "atomo_set_persistent_eig", "atomo_last_eig_scheme", "atomo_decode_spectral_static", "atomo_decode_average", "atomo_lq_budget",
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
     "atomo_set_tridiag_ctas", "atomo_measure_fma_peak", "atomo_encode_spectral_from_svd", "atomo_get_table_uploads",
+    "atomo_set_entrywise_launch",
 ]
 
 
@@ -95,6 +96,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_payload_bytes_entrywise_compact.argtypes = [ctypes.POINTER(i64), i32, i64, i64]
     lib.atomo_payload_bytes_entrywise_compact.restype = i64
     lib.atomo_set_entrywise_format.argtypes = [vp, i32, i64]
+    lib.atomo_set_entrywise_launch.argtypes = [vp, i32]
     lib.atomo_encode_spectral.argtypes = [vp, ctypes.POINTER(_Mat), i32, dbl, u64, u64, i32, vp, i64,
                                           ctypes.POINTER(_Debug), vp]
     lib.atomo_encode_entrywise.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, u64, u64, i64, vp, i64,
@@ -538,6 +540,11 @@ class Atomo:
         explicit values only for the atoms with p = 1, of which at most sat_cap per vector)."""
         self._check(self.lib.atomo_set_entrywise_format(self._h, int(fmt), int(sat_cap)), "atomo_set_entrywise_format")
         self._ew_format, self._ew_sat_cap = int(fmt), (int(sat_cap) if int(fmt) == EW_COMPACT else 0)
+
+    def set_entrywise_launch(self, two_kernels: bool):
+        """False (default): one cooperative kernel per vector that fits one wave of resident CTAs; True: always the
+        solve kernel followed by the sample / pack kernel.  Same payloads either way."""
+        self._check(self.lib.atomo_set_entrywise_launch(self._h, 1 if two_kernels else 0), "atomo_set_entrywise_launch")
 
     def table_uploads(self):
         """(calls that uploaded their descriptor tables, calls that found them on the device) since the context was made."""

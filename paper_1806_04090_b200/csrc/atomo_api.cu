@@ -69,6 +69,7 @@ struct atomo_ctx {
   int tri_big_ctas = 0;              // CTAs per layer of that reduction: 0 = chosen per batch, else 1, 2, 4, 8 or 16
   int eig_scheme_used = -1;          // what the last spectral encode actually ran
   int ew_format = ATOMO_EW_EXPLICIT; // payload format of entry-wise encodes
+  int ew_launch = 0;                 // 0: one cooperative kernel per vector where it fits one wave; 1: always solve + sample/pack kernels
   int64_t ew_sat_cap = 0;            // compact format: capacity of the saturated list
   int cluster_capacity[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // by log2(rp_max), -1 = not asked yet
   std::string err;
@@ -726,7 +727,7 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     put(d_given, ptrs.data(), ptrs.size() * sizeof(const float*));
   }
   { const int rc = table_commit(ctx, tab, tables.data(), table_bytes, st); if (rc != ATOMO_OK) return rc; }
-  launch_sp_begin(pay, gh, d_hdr_tmpl, n_layers, d_flag, st);          // payload header, layer headers, flags
+  launch_sp_begin(pay, gh, d_hdr_tmpl, n_layers, d_flag, nullptr, 0, st);          // payload header, layer headers, flags
   CK(cudaMemsetAsync(zero_beg, 0, zero_bytes, st));
 
   // ---- S1: Gram matrix, scaling ----
@@ -904,6 +905,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   const int tile = ew_tile_elems();
 
   std::vector<EwVec> V(n_vecs);
+  std::vector<char> fused(n_vecs, 0);
   size_t need = 0;
   uint8_t* ew_zero_beg = nullptr; size_t ew_zero_bytes = 0;
   const int max_blocks = ew_solve_max_blocks();
@@ -915,7 +917,9 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       EwVec& v = V[l];
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
-      v.n_ctas = ew_sample_pack_ctas(v.n_tiles, compact);
+      const int fused_ctas = ctx->ew_launch == 0 ? ew_encode_ctas(v.n_tiles, compact) : 0;
+      fused[l] = fused_ctas > 0;
+      v.n_ctas = fused[l] ? fused_ctas : ew_sample_pack_ctas(v.n_tiles, compact);
       v.compact = compact ? 1 : 0; v.sat_cap = lay[l].sc;
       v.ent = reinterpret_cast<uint16_t*>(pay + lay[l].off_idx);
       v.sat_idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_sat);
@@ -928,7 +932,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       v.idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_idx);
       v.val = reinterpret_cast<float*>(pay + lay[l].off_val);
       v.tile_table = reinterpret_cast<uint32_t*>(pay + lay[l].off_tiles);
-      v.partials = A.take<EwPartial>((size_t)3 * v.n_chunks);
+      v.partials = A.take<EwPartial>((size_t)3 * std::max(v.n_chunks, v.n_ctas));
       v.state = A.take<EwState>(1);
       uint32_t* mask_ws = A.take<uint32_t>(v.n_words);
       v.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
@@ -961,27 +965,43 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     const size_t tb = tmpl.size() * sizeof(atomo_layer_header);
     { const int rc = table_reserve(ctx, ctx->tab_ew, tb); if (rc != ATOMO_OK) return rc; }
     { const int rc = table_commit(ctx, ctx->tab_ew, reinterpret_cast<const uint8_t*>(tmpl.data()), tb, st); if (rc != ATOMO_OK) return rc; }
-    launch_sp_begin(pay, gh, reinterpret_cast<const atomo_layer_header*>(ctx->tab_ew.d), n_vecs, nullptr, st);
+    // ... and the look-back status words and tickets of the sample / pack kernels start at zero
+    launch_sp_begin(pay, gh, reinterpret_cast<const atomo_layer_header*>(ctx->tab_ew.d), n_vecs, nullptr,
+                    reinterpret_cast<uint32_t*>(ew_zero_beg), (int64_t)((ew_zero_bytes + 3) / 4), st);
   }
 
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   const uint32_t ks = kind_step_word(ATOMO_KIND_ENTRYWISE, step);
-  // probabilities: one cooperative launch per vector (pass 1 and the water-filling rounds)
+  // probabilities: one cooperative launch per vector (pass 1 and the water-filling rounds); a vector that fits one
+  // wave of resident chunks goes on to sampling and packing inside the same launch (timed with the pack stage)
+  int n_two = 0, n_one = 0;
   stage_begin(ctx, ATOMO_STAGE_EW_REDUCE, st);
   for (int l = 0; l < n_vecs; ++l) {
+    if (fused[l]) continue;
     const int e = launch_ew_solve(V[l], s, st);
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(ew_solve)");
+    ++n_two;
   }
-  stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_vecs);
+  stage_end(ctx, ATOMO_STAGE_EW_REDUCE, st, n_two);
   stage_begin(ctx, ATOMO_STAGE_EW_PACK, st);
-  CK(cudaMemsetAsync(ew_zero_beg, 0, ew_zero_bytes, st));
-  for (int l = 0; l < n_vecs; ++l) launch_ew_sample_pack(V[l], key, ks, st);
-  stage_end(ctx, ATOMO_STAGE_EW_PACK, st, (int64_t)n_vecs);
+  for (int l = 0; l < n_vecs; ++l) {
+    if (!fused[l]) { launch_ew_sample_pack(V[l], key, ks, st); continue; }
+    const int e = launch_ew_encode(V[l], s, key, ks, st);
+    if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(ew_encode)");
+    ++n_one;
+  }
+  stage_end(ctx, ATOMO_STAGE_EW_PACK, st, (int64_t)(n_two + n_one));
   CK(cudaGetLastError());
   return ATOMO_OK;
 }
 
 // ==================================================================================================
+int atomo_set_entrywise_launch(atomo_ctx* ctx, int32_t two_kernels) {
+  if (!ctx || (two_kernels != 0 && two_kernels != 1)) return ATOMO_ERR_INVALID_ARG;
+  ctx->ew_launch = two_kernels;
+  return ATOMO_OK;
+}
+
 int atomo_lq_budget(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs, double q, double* s_out, void* stream) {
   if (!ctx || !vecs || n_vecs <= 0 || !s_out || !(q >= 1.0)) return ATOMO_ERR_INVALID_ARG;
   for (int l = 0; l < n_vecs; ++l) {

@@ -23,10 +23,23 @@
 
 namespace cg = cooperative_groups;
 
+// development builds (-DEW_PROFILE) print the phase times of a few CTAs of the one-kernel form
+#ifdef EW_PROFILE
+#include <cstdio>
+__device__ __forceinline__ unsigned long long ew_now() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define EW_STAMP(k) if (threadIdx.x == 0) ew_t[k] = ew_now();
+#else
+#define EW_STAMP(k)
+#endif
+
 namespace atomo {
 
 constexpr int kEwThreads = 256;
 constexpr int kEwTile = 4096;                 // elements per tile of the sample / pack / decode passes
+#ifndef EW_MIN_BLOCKS
+#define EW_MIN_BLOCKS 5
+#endif
+constexpr int kEwMinBlocks = EW_MIN_BLOCKS;   // resident CTAs per SM the sample / pack kernels are compiled for
 
 __device__ __forceinline__ float4 load4(const float* __restrict__ g, int64_t i, int64_t n, bool aligned) {
   if (aligned && i + 3 < n) return __ldg(reinterpret_cast<const float4*>(g + i));
@@ -45,10 +58,8 @@ __device__ __forceinline__ float4 load4(const float* __restrict__ g, int64_t i, 
 struct EwAcc { double sum; float amax; uint32_t cnt; uint32_t bad; };
 
 template <bool kRound>
-__device__ __forceinline__ EwAcc ew_chunk_pass(const EwVec& v, float theta) {
+__device__ __forceinline__ EwAcc ew_chunk_pass(const EwVec& v, float theta, const int64_t beg, const int64_t end) {
   const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
-  const int64_t beg = (int64_t)blockIdx.x * v.chunk;
-  const int64_t end = min(v.n, beg + v.chunk);
   EwAcc acc{0.0, 0.0f, 0u, 0u};
   constexpr int kU = 4;
   for (int64_t base = beg + (int64_t)threadIdx.x * 4; base < end; base += (int64_t)kEwThreads * 4 * kU) {
@@ -91,14 +102,19 @@ __device__ __forceinline__ EwAcc ew_block_reduce(EwAcc a, double* s_sum, float* 
   return r;
 }
 
-__global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s) {
+// what the probability solve leaves for the sampling pass (every CTA computes the same values)
+struct EwSolved { double T0; float scale, theta, c; uint32_t n_sat, rounds; bool nonfinite; };
+
+// The solve over this CTA's elements [beg, end) (a multiple of 4 from the start of the vector); all CTAs of the grid
+// call it together (cooperative launch).
+__device__ __forceinline__ EwSolved ew_solve_body(const EwVec& v, const double s, const int64_t beg, const int64_t end) {
   cg::grid_group grid = cg::this_grid();
   __shared__ double s_sum[kEwThreads / kWarp];
   __shared__ float s_max[kEwThreads / kWarp];
   __shared__ uint32_t s_cnt[kEwThreads / kWarp], s_bad[kEwThreads / kWarp];
   const int nb = gridDim.x;
   // ---- pass 1: ||g||_1, ||g||_inf, non-finite scan ----
-  EwAcc mine = ew_block_reduce(ew_chunk_pass<false>(v, 0.0f), s_sum, s_max, s_cnt, s_bad);
+  EwAcc mine = ew_block_reduce(ew_chunk_pass<false>(v, 0.0f, beg, end), s_sum, s_max, s_cnt, s_bad);
   if (threadIdx.x == 0) v.partials[blockIdx.x] = EwPartial{mine.sum, mine.amax, mine.cnt, mine.bad};
   grid.sync();
   EwAcc tot{0.0, 0.0f, 0u, 0u};
@@ -120,7 +136,7 @@ __global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s)
   // ---- water-filling rounds ----
   while (!done && rounds < kEwMaxRounds) {
     EwPartial* buf = v.partials + (size_t)((rounds & 1) + 1) * nb;
-    mine = ew_block_reduce(ew_chunk_pass<true>(v, theta), s_sum, s_max, s_cnt, s_bad);
+    mine = ew_block_reduce(ew_chunk_pass<true>(v, theta, beg, end), s_sum, s_max, s_cnt, s_bad);
     if (threadIdx.x == 0) buf[blockIdx.x] = EwPartial{mine.sum, 0.0f, mine.cnt, 0u};
     grid.sync();
     tot = EwAcc{0.0, 0.0f, 0u, 0u};
@@ -134,14 +150,23 @@ __global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s)
       theta = fminf(theta, th);
     }
   }
+  const bool live = T > 0.0 && s_cur > 0.0 && !nonfinite;
+  EwSolved r;
+  r.T0 = T0; r.theta = theta; r.n_sat = n_sat; r.rounds = rounds; r.nonfinite = nonfinite;
+  r.scale = live ? (float)(s_cur / T) : 0.0f;            // p_i = |g_i| * scale
+  r.c = live ? (float)(T / s_cur) : 0.0f;                // weight of kept unsaturated atoms
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     EwState* st = v.state;
-    const bool live = T > 0.0 && s_cur > 0.0 && !nonfinite;
     st->T0 = T0; st->T = T; st->s_cur = s_cur; st->theta = (double)theta; st->theta_f = theta; st->amax = amax;
     st->n_sat = n_sat; st->rounds = rounds; st->done = 1; st->nonfinite = nonfinite ? 1u : 0u;
-    st->scale = live ? (float)(s_cur / T) : 0.0f;         // p_i = |g_i| * scale
-    st->c = live ? (float)(T / s_cur) : 0.0f;             // weight of kept unsaturated atoms
+    st->scale = r.scale; st->c = r.c;
   }
+  return r;
+}
+
+__global__ void __launch_bounds__(kEwThreads) ew_solve_kernel(EwVec v, double s) {
+  const int64_t beg = (int64_t)blockIdx.x * v.chunk;
+  ew_solve_body(v, s, beg, min(v.n, beg + v.chunk));
 }
 
 // ---- sampling + ordered compaction, one kernel -----------------------------------------------------
@@ -159,50 +184,45 @@ constexpr int kEwMaxTilesPerCta = 64;
 constexpr int kEwWordsPerTile = kEwTile / 32;
 
 // Phase 1 of the sample / pack kernel over the chunk's tiles: keep bits into the mask words, kept atoms counted per
-// tile.  SAT also records which kept atoms are saturated (a second mask and count; the compact format of a vector
-// that is not s-balanced needs them).
-template <bool SAT>
-__device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key, const uint32_t kind_step,
-                                             const int64_t tile0, const int n_my, const float scale, const float theta,
-                                             const bool dead, const bool aligned, uint32_t* s_mask, uint32_t* s_sat,
-                                             uint32_t* s_tcnt, uint32_t* s_tsat) {
-  constexpr int kIts = kEwTile / (kEwThreads * 4);
-  const int tid = threadIdx.x, lane = tid % kWarp;
-  const float scale32 = scale * 4294967296.0f;    // exact: a power-of-two factor
-  for (int tl = 0; tl < n_my; ++tl) {
-    const uint32_t tile = (uint32_t)(tile0 + tl);
-    const int64_t tile_base = (int64_t)tile * kEwTile;
-    const bool full = aligned && tile_base + kEwTile <= v.n;
-    float4 x[kIts];
+// tile.  A thread takes 16 consecutive atoms of a tile (four Philox blocks), so two neighbouring lanes hold a mask
+// word between them.  SAT also records which kept atoms are saturated (a second mask and count; the compact format
+// of a vector that is not s-balanced needs them); UNBAL: the vector is not s-balanced, so some atoms have p = 1 (an
+// s-balanced vector, Lemma 3, skips that test); FULL: the tile lies inside the vector and is 16-byte aligned;
+// PROB: the probabilities are wanted too (debug output).  The tiles are taken from the chunk's last to its first:
+// the reduction kernel read them in ascending order just before, so the end of the chunk is what the L2 still holds.
+template <bool SAT, bool UNBAL, bool FULL, bool PROB>
+__device__ __forceinline__ void ew_tile_bits(const EwVec& v, const PhiloxKey key, const uint32_t kind_step, const uint32_t tile,
+                                             const float scale, const float scale32, const float theta, const bool dead,
+                                             const bool aligned, uint32_t& nb_out, uint32_t& sb_out) {
+  const int tid = threadIdx.x;
+  const int64_t i0 = (int64_t)tile * kEwTile + 16 * tid;
+  float4 x[4];
 #pragma unroll
-    for (int it = 0; it < kIts; ++it) {
-      const int64_t i = tile_base + ((int64_t)it * kEwThreads + tid) * 4;
-      x[it] = full ? __ldg(reinterpret_cast<const float4*>(v.g + i))
-                   : (i < v.n ? load4(v.g, i, v.n, aligned) : make_float4(0.f, 0.f, 0.f, 0.f));
+  for (int it = 0; it < 4; ++it) {
+    const int64_t i = i0 + 4 * it;
+    x[it] = FULL ? __ldg(reinterpret_cast<const float4*>(v.g + i))
+                 : (i < v.n ? load4(v.g, i, v.n, aligned) : make_float4(0.f, 0.f, 0.f, 0.f));
+  }
+  uint32_t nb = 0, sb = 0;
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    // block of 4 atoms = atom >> 2 < 2^30 (n < 2^32): the high counter word is zero
+    const uint4 wd = philox4x32_10(make_uint4(tile * (uint32_t)(kEwTile / 4) + (uint32_t)(4 * tid + it), 0u, v.layer, kind_step), key);
+    const float a[4] = {fabsf(x[it].x), fabsf(x[it].y), fabsf(x[it].z), fabsf(x[it].w)};
+    const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      // p = 1 if saturated, else min(a scale, 1); keep iff p >= 1 or word < floor(p 2^32).  a scale32 is the
+      // same product times 2^32 (exact), and the truncating conversion gives the floor.
+      const float t = a[j] * scale32;
+      const bool sat = UNBAL && a[j] > theta;
+      bool keep = sat || t >= 4294967296.0f || ww[j] < __float2uint_rz(t);
+      if (!FULL) keep = keep && i0 + 4 * it + j < v.n;
+      if (keep) { nb |= 1u << (4 * it + j); if (SAT && sat) sb |= 1u << (4 * it + j); }
     }
-    uint32_t kept = 0, kept_sat = 0;
-#pragma unroll
-    for (int it = 0; it < kIts; ++it) {
-      const int64_t i = tile_base + ((int64_t)it * kEwThreads + tid) * 4;
-      // block of 4 atoms = i >> 2 < 2^30 (n < 2^32): the high counter word is zero
-      const uint4 wd = philox4x32_10(make_uint4(tile * (uint32_t)(kEwTile / 4) + (uint32_t)(it * kEwThreads + tid), 0u, v.layer, kind_step), key);
-      const float a[4] = {fabsf(x[it].x), fabsf(x[it].y), fabsf(x[it].z), fabsf(x[it].w)};
-      const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
-      uint32_t nb = 0, sb = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        // p = 1 if saturated, else min(a scale, 1); keep iff p >= 1 or word < floor(p 2^32).  a scale32 is the
-        // same product times 2^32 (exact), and the truncating conversion gives the floor.
-        const float t = a[j] * scale32;
-        const bool sat = a[j] > theta;
-        const bool one = sat || t >= 4294967296.0f;
-        const bool keep = one || ww[j] < __float2uint_rz(t);
-        if (keep && (full || i + j < v.n)) { nb |= 1u << j; if (SAT && sat) sb |= 1u << j; }
-      }
-      if (dead) { nb = 0; sb = 0; }
-      kept += __popc(nb);
-      if (SAT) kept_sat += __popc(sb);
-      if (v.prob_out != nullptr && i < v.n) {
+    if (PROB) {
+      const int64_t i = i0 + 4 * it;
+      if (i < v.n) {
         float pp[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) pp[j] = dead ? 0.0f : ((a[j] > theta) ? 1.0f : fminf(a[j] * scale, 1.0f));
@@ -211,25 +231,41 @@ __device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key
         else
           for (int j = 0; j < 4 && i + j < v.n; ++j) v.prob_out[i + j] = pp[j];
       }
-      // 8 consecutive lanes hold the 32 bits of one mask word
-      uint32_t word = nb << (4 * (tid & 7));
-      word |= __shfl_xor_sync(0xffffffffu, word, 1);
-      word |= __shfl_xor_sync(0xffffffffu, word, 2);
-      word |= __shfl_xor_sync(0xffffffffu, word, 4);
-      uint32_t sword = 0;
-      if (SAT) {
-        sword = sb << (4 * (tid & 7));
-        sword |= __shfl_xor_sync(0xffffffffu, sword, 1);
-        sword |= __shfl_xor_sync(0xffffffffu, sword, 2);
-        sword |= __shfl_xor_sync(0xffffffffu, sword, 4);
-      }
-      if ((tid & 7) == 0) {
-        const int wl = it * (kEwThreads / 8) + (tid >> 3);
-        s_mask[tl * kEwWordsPerTile + wl] = word;
-        if (SAT) s_sat[tl * kEwWordsPerTile + wl] = sword;
-        const int64_t widx = (tile_base >> 5) + wl;
-        if (widx < v.n_words) v.mask_words[widx] = word;
-      }
+    }
+  }
+  if (dead) { nb = 0; sb = 0; }
+  nb_out = nb; sb_out = sb;
+}
+
+template <bool SAT, bool UNBAL>
+__device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key, const uint32_t kind_step,
+                                             const int64_t tile0, const int n_my, const float scale, const float theta,
+                                             const bool dead, const bool aligned, uint32_t* s_mask, uint32_t* s_sat,
+                                             uint32_t* s_tcnt, uint32_t* s_tsat) {
+  const int tid = threadIdx.x, lane = tid % kWarp;
+  const float scale32 = scale * 4294967296.0f;    // exact: a power-of-two factor
+  for (int tl = n_my - 1; tl >= 0; --tl) {
+    const uint32_t tile = (uint32_t)(tile0 + tl);
+    const int64_t tile_base = (int64_t)tile * kEwTile;
+    const bool full = aligned && tile_base + kEwTile <= v.n;
+    uint32_t nb, sb;
+    if (v.prob_out != nullptr) ew_tile_bits<SAT, UNBAL, false, true>(v, key, kind_step, tile, scale, scale32, theta, dead, aligned, nb, sb);
+    else if (full) ew_tile_bits<SAT, UNBAL, true, false>(v, key, kind_step, tile, scale, scale32, theta, dead, aligned, nb, sb);
+    else ew_tile_bits<SAT, UNBAL, false, false>(v, key, kind_step, tile, scale, scale32, theta, dead, aligned, nb, sb);
+    // two neighbouring lanes hold the 32 bits of one mask word; the even lane stores it
+    const uint32_t other = __shfl_xor_sync(0xffffffffu, nb, 1);
+    const uint32_t word = nb | (other << 16);
+    uint32_t sword = 0;
+    if (SAT) sword = sb | (__shfl_xor_sync(0xffffffffu, sb, 1) << 16);
+    uint32_t kept = 0, kept_sat = 0;
+    if ((lane & 1) == 0) {
+      const int wl = tid >> 1;
+      s_mask[tl * kEwWordsPerTile + wl] = word;
+      if (SAT) s_sat[tl * kEwWordsPerTile + wl] = sword;
+      const int64_t widx = (tile_base >> 5) + wl;
+      if (widx < v.n_words) v.mask_words[widx] = word;
+      kept = __popc(word);
+      if (SAT) kept_sat = __popc(sword);
     }
     kept = warp_sum(kept);
     if (lane == 0 && kept) atomicAdd(&s_tcnt[tl], kept);
@@ -244,34 +280,39 @@ __device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key
 // atom with p = 1, index and value in a list of its own; both ascending.  The chunk's status word then carries the
 // saturated count in bits 32..62 beside the total, and the kernel keeps a second bit mask (saturated and kept).
 template <bool COMPACT>
-__global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+__device__ __forceinline__ void ew_sample_pack_chunk(const EwVec& v, const PhiloxKey key, const uint32_t kind_step,
+                                                     const uint32_t chunk, const EwSolved& S, uint32_t* s_mask
+#ifdef EW_PROFILE
+                                                     , unsigned long long* ew_t = nullptr
+#endif
+                                                     ) {
   constexpr int kWarps = kEwThreads / kWarp;
-  extern __shared__ uint32_t s_mask[];            // [tiles_per_cta][128] mask words of the chunk (COMPACT: then the saturated masks)
   __shared__ uint32_t s_tcnt[kEwMaxTilesPerCta];  // kept atoms per tile, then their exclusive prefix
   __shared__ uint32_t s_tsat[kEwMaxTilesPerCta];  // the same for the saturated kept atoms (COMPACT)
   __shared__ uint32_t s_chunk, s_chunk_sat;
   __shared__ unsigned long long s_base;           // kept atoms before this chunk (COMPACT: saturated ones in bits 32..62)
-  __shared__ uint32_t s_wsum[kWarps];
   __shared__ int s_fail;
-  const EwState* st = v.state;
-  const float scale = st->scale, theta = st->theta_f, c = st->c;
-  const bool dead = st->nonfinite != 0;
-  const bool any_sat = COMPACT && st->n_sat != 0;   // an s-balanced vector (Lemma 3) skips the saturated bookkeeping
+  const float scale = S.scale, theta = S.theta, c = S.c;
+  const bool dead = S.nonfinite;
+  const bool any_sat = COMPACT && S.n_sat != 0;     // an s-balanced vector (Lemma 3) skips the saturated bookkeeping
   const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
   const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
   const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;   // the first `rem` chunks have q + 1 tiles
-  if (tid == 0) { s_chunk = atomicAdd(v.ticket, 1u); s_base = 0ull; s_fail = 0; }
+  if (tid == 0) { s_base = 0ull; s_fail = 0; }
   if (tid < kEwMaxTilesPerCta) { s_tcnt[tid] = 0u; s_tsat[tid] = 0u; }
   __syncthreads();
-  const uint32_t chunk = s_chunk;
   const int64_t tile0 = (int64_t)chunk * q + min((int64_t)chunk, rem);
   const int n_my = (int)(q + ((int64_t)chunk < rem ? 1 : 0));
   uint32_t* s_sat = s_mask + (size_t)(q + (rem ? 1 : 0)) * kEwWordsPerTile;   // COMPACT only
 
   // ---- phase 1 ----
-  if (any_sat) ew_keep_bits<true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
-  else ew_keep_bits<false>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
+  if (any_sat) ew_keep_bits<true, true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
+  else if (S.n_sat != 0) ew_keep_bits<false, true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
+  else ew_keep_bits<false, false>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
   __syncthreads();
+#ifdef EW_PROFILE
+  if (ew_t != nullptr) { EW_STAMP(2) }
+#endif
 
   // ---- chunk count out, counts of the earlier chunks in ----
   if (w == 0) {
@@ -295,7 +336,11 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
   for (uint32_t cidx = tid; cidx < chunk; cidx += kEwThreads) {
     unsigned long long sv;
     uint32_t spins = 0;
-    do { sv = *(volatile const unsigned long long*)(v.tile_status + cidx); } while (!(sv & kFlagReady) && ++spins <= kChunkSpinLimit);
+    for (;;) {
+      sv = *(volatile const unsigned long long*)(v.tile_status + cidx);
+      if ((sv & kFlagReady) || ++spins > kChunkSpinLimit) break;
+      __nanosleep(200);                                   // leave the issue slots to the CTAs that are still sampling
+    }
     if (!(sv & kFlagReady)) fail = 1;
     before += sv & ~kFlagReady;                           // totals < 2^32 in all: the two fields never mix
   }
@@ -304,6 +349,9 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
   if (lane == 0 && before) atomicAdd(&s_base, before);
   if (fail) s_fail = 1;
   __syncthreads();
+#ifdef EW_PROFILE
+  if (ew_t != nullptr) { EW_STAMP(3) }
+#endif
   const uint64_t base_all = s_base & 0xFFFFFFFFull;       // kept atoms before this chunk
   const uint64_t base_sat = s_base >> 32;                 // of them saturated (0 unless COMPACT)
   const uint64_t base = COMPACT ? base_all - base_sat : base_all;   // position of the chunk's first list entry
@@ -317,8 +365,8 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
       const uint64_t k_sat = base_sat + s_chunk_sat;
       const uint64_t k_list = COMPACT ? k - k_sat : k;    // entries of the idx / entry list
       atomo_layer_header* h = v.hdr;
-      h->n_sat = st->n_sat; h->c = st->c; h->l1 = st->T0; h->sweeps = st->rounds;
-      if (st->nonfinite) raise_status(h, ATOMO_ERR_NONFINITE);
+      h->n_sat = S.n_sat; h->c = S.c; h->l1 = S.T0; h->sweeps = S.rounds;
+      if (S.nonfinite) raise_status(h, ATOMO_ERR_NONFINITE);
       else if (k_list > (uint64_t)v.k_cap || (COMPACT && k_sat > (uint64_t)v.sat_cap)) raise_status(h, ATOMO_ERR_CAPACITY);
       const bool ok = *(volatile uint32_t*)&h->status == ATOMO_OK;
       h->k = ok ? (uint32_t)k : 0u;
@@ -329,55 +377,97 @@ __global__ void __launch_bounds__(kEwThreads, 5) ew_sample_pack_kernel(EwVec v, 
   if (total == 0) return;
 
   // ---- phase 2: ordered compaction, indices ascending, value = g_i / p_i ----
-  for (int tl = 0; tl < n_my; ++tl) {
-    const int64_t tile_base = (tile0 + tl) * (int64_t)kEwTile;
-    const uint32_t word = tid < kEwWordsPerTile ? s_mask[tl * kEwWordsPerTile + tid] : 0u;
-    const uint32_t sword = (any_sat && tid < kEwWordsPerTile) ? s_sat[tl * kEwWordsPerTile + tid] : 0u;
-    // COMPACT: two counts in one scan, list entries in the low half and saturated atoms in the high half (<= 4096 each)
-    const uint32_t pc = COMPACT ? (__popc(word & ~sword) | (__popc(sword) << 16)) : __popc(word);
-    uint32_t inc = pc;
+  // A thread takes a run of consecutive mask words of the chunk; one scan over the threads' counts gives every run
+  // its place in the lists.  COMPACT scans two counts at once (list entries in the low half of a 64-bit word,
+  // saturated atoms in the high half).
+  const int n_w = n_my * kEwWordsPerTile;
+  const int wpt = (n_w + kEwThreads - 1) / kEwThreads;                       // words per thread
+  const int w_beg = min(tid * wpt, n_w), w_end = min(w_beg + wpt, n_w);
+  unsigned long long cnt = 0;
+  for (int wi = w_beg; wi < w_end; ++wi) {
+    const uint32_t word = s_mask[wi];
+    const uint32_t sword = any_sat ? s_sat[wi] : 0u;
+    cnt += COMPACT ? ((unsigned long long)__popc(word & ~sword) | ((unsigned long long)__popc(sword) << 32)) : (unsigned long long)__popc(word);
+  }
+  unsigned long long inc = cnt;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
-    __syncthreads();                                      // s_wsum of the previous tile has been read
-    if (lane == 31) s_wsum[w] = inc;
-    __syncthreads();
-    uint32_t woff = inc - pc;
-    for (int i = 0; i < w; ++i) woff += s_wsum[i];
-    if (!COMPACT) {
-      uint64_t pos = base + s_tcnt[tl] + woff;
-      uint32_t m = word;
-      while (m) {
-        const int bpos = __ffs(m) - 1;
-        m &= m - 1;
-        const int64_t i = tile_base + tid * 32 + bpos;
+  for (int o = 1; o < 32; o <<= 1) { const unsigned long long t = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += t; }
+  __shared__ unsigned long long s_wsum2[kWarps];
+  if (lane == 31) s_wsum2[w] = inc;
+  __syncthreads();
+  unsigned long long off = inc - cnt;
+  for (int i = 0; i < w; ++i) off += s_wsum2[i];
+  uint64_t pos = base + (off & 0xFFFFFFFFull);
+  uint64_t pos_sat = base_sat + (off >> 32);
+  for (int wi = w_beg; wi < w_end; ++wi) {
+    uint32_t m = s_mask[wi];
+    const uint32_t sword = any_sat ? s_sat[wi] : 0u;
+    const int tl = wi / kEwWordsPerTile;
+    const uint32_t off0 = (uint32_t)(wi % kEwWordsPerTile) * 32u;            // first atom of the word inside its tile
+    const int64_t tile_base = (tile0 + tl) * (int64_t)kEwTile;
+    while (m) {
+      const int bpos = __ffs(m) - 1;
+      m &= m - 1;
+      const uint32_t o = off0 + (uint32_t)bpos;
+      const float g = __ldg(v.g + tile_base + o);
+      if (!COMPACT) {
         if (pos < (uint64_t)v.k_cap) {
-          const float g = __ldg(v.g + i);
           // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) T / (s - n_s)
-          v.idx[pos] = (uint32_t)i;
+          v.idx[pos] = (uint32_t)(tile_base + o);
           v.val[pos] = (fabsf(g) > theta) ? g : copysignf(c, g);
         }
         ++pos;
-      }
-    } else {
-      uint64_t pos = base + (s_tcnt[tl] - s_tsat[tl]) + (woff & 0xFFFFu);
-      uint64_t pos_sat = base_sat + s_tsat[tl] + (woff >> 16);
-      uint32_t m = word;
-      while (m) {
-        const int bpos = __ffs(m) - 1;
-        m &= m - 1;
-        const uint32_t off = (uint32_t)(tid * 32 + bpos);
-        const float g = __ldg(v.g + tile_base + off);
-        if ((sword >> bpos) & 1u) {
-          if (pos_sat < (uint64_t)v.sat_cap) { v.sat_idx[pos_sat] = (uint32_t)(tile_base + off); v.sat_val[pos_sat] = g; }
-          ++pos_sat;
-        } else {
-          // value sign(g) c: the entry carries g's sign bit (what copysignf reads in the explicit format)
-          if (pos < (uint64_t)v.k_cap) v.ent[pos] = (uint16_t)(off | ((__float_as_uint(g) >> 31) << 15));
-          ++pos;
-        }
+      } else if ((sword >> bpos) & 1u) {
+        if (pos_sat < (uint64_t)v.sat_cap) { v.sat_idx[pos_sat] = (uint32_t)(tile_base + o); v.sat_val[pos_sat] = g; }
+        ++pos_sat;
+      } else {
+        // value sign(g) c: the entry carries g's sign bit (what copysignf reads in the explicit format)
+        if (pos < (uint64_t)v.k_cap) v.ent[pos] = (uint16_t)(o | ((__float_as_uint(g) >> 31) << 15));
+        ++pos;
       }
     }
   }
+}
+
+// The two-kernel form: the solve has left its result in the state record; a CTA takes the next chunk of consecutive
+// tiles by ticket, so that every chunk it will wait for is already running, however many waves the grid takes.
+template <bool COMPACT>
+__global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_sample_pack_kernel(EwVec v, PhiloxKey key, uint32_t kind_step) {
+  extern __shared__ uint32_t s_mask[];            // [tiles_per_cta][128] mask words of the chunk (COMPACT: then the saturated masks)
+  __shared__ uint32_t s_ticket;
+  const EwState* st = v.state;
+  EwSolved S;
+  S.T0 = st->T0; S.scale = st->scale; S.theta = st->theta_f; S.c = st->c; S.n_sat = st->n_sat; S.rounds = st->rounds;
+  S.nonfinite = st->nonfinite != 0;
+  if (threadIdx.x == 0) s_ticket = atomicAdd(v.ticket, 1u);
+  __syncthreads();
+  ew_sample_pack_chunk<COMPACT>(v, key, kind_step, s_ticket, S, s_mask);
+}
+
+// The one-kernel form (cooperative launch, every chunk resident): a CTA solves over its own chunk of tiles and then
+// samples and packs the same chunk, which it finds in the L2 on its own side of the chip.
+template <bool COMPACT>
+__global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step) {
+  extern __shared__ uint32_t s_mask[];
+  const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;
+  const int64_t chunk = blockIdx.x;
+  const int64_t tile0 = chunk * q + min(chunk, rem);
+  const int64_t n_my = q + (chunk < rem ? 1 : 0);
+#ifdef EW_PROFILE
+  unsigned long long ew_t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
+  EW_STAMP(0)
+  const EwSolved S = ew_solve_body(v, s, tile0 * kEwTile, min(v.n, (tile0 + n_my) * kEwTile));
+  EW_STAMP(1)
+#ifdef EW_PROFILE
+  ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask, ew_t);
+  EW_STAMP(5)
+  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
+    printf("cta %d tiles %d: solve %llu ns, keep bits %llu, publish+wait %llu, scan+pack %llu, total %llu\n", (int)blockIdx.x, (int)n_my,
+           ew_t[1] - ew_t[0], ew_t[2] - ew_t[1], ew_t[3] - ew_t[2], ew_t[5] - ew_t[3], ew_t[5] - ew_t[0]);
+#else
+  ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask);
+#endif
 }
 
 // ---- decode -------------------------------------------------------------------------------------
@@ -490,20 +580,35 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st) {
   void* args[] = {&vv, &ss};
   return (int)cudaLaunchCooperativeKernel((const void*)ew_solve_kernel, dim3(v.n_chunks), dim3(kEwThreads), args, 0, st);
 }
-int ew_sample_pack_ctas(int64_t n_tiles, bool compact) {
-  // one wave of chunks when it fits (at most 64 tiles per chunk, 32 for the compact format): tiles spread evenly, sizes differ by at most one
+namespace {
+// co-resident CTAs of a sample / pack style kernel with its largest chunk in shared memory
+template <typename K> int64_t ew_wave(K kernel, bool compact) {
   int dev = 0, sms = 148, per_sm = 4;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const cudaError_t e = compact
-      ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel<true>, kEwThreads,
-                                                      32 * kEwWordsPerTile * sizeof(uint32_t))
-      : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_sample_pack_kernel<false>, kEwThreads,
-                                                      16 * kEwWordsPerTile * sizeof(uint32_t));
-  if (e != cudaSuccess || per_sm < 1) per_sm = 4;
-  const int64_t wave = (int64_t)sms * per_sm;
+  const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kEwThreads,
+                                                                      (compact ? 32 : 16) * kEwWordsPerTile * sizeof(uint32_t));
+  if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 4; }
+  return (int64_t)sms * per_sm;
+}
+}  // namespace
+
+int ew_sample_pack_ctas(int64_t n_tiles, bool compact) {
+  // one wave of chunks when it fits (at most 64 tiles per chunk, 32 for the compact format): tiles spread evenly, sizes differ by at most one
+  const int64_t wave = compact ? ew_wave(ew_sample_pack_kernel<true>, true) : ew_wave(ew_sample_pack_kernel<false>, false);
   const int max_tiles = compact ? kEwMaxTilesPerCta / 2 : kEwMaxTilesPerCta;   // compact: two masks per tile in shared memory
   const int64_t min_ctas = (n_tiles + max_tiles - 1) / max_tiles;
   return (int)std::max<int64_t>(1, std::max(min_ctas, std::min(n_tiles, wave)));
+}
+// CTAs of the one-kernel form, or 0 if the vector does not fit one wave of resident chunks
+int ew_encode_ctas(int64_t n_tiles, bool compact) {
+  static int64_t waves[2] = {0, 0};
+  if (waves[compact] == 0) waves[compact] = compact ? ew_wave(ew_encode_kernel<true>, true) : ew_wave(ew_encode_kernel<false>, false);
+  const int max_tiles = compact ? kEwMaxTilesPerCta / 2 : kEwMaxTilesPerCta;
+  // chunks of at most 16 tiles keep the shared memory the occupancy figure was asked for
+  const int64_t fit_tiles = 16;
+  const int64_t ctas = std::min(n_tiles, waves[compact]);
+  if (ctas < 1 || (n_tiles + ctas - 1) / ctas > std::min<int64_t>(max_tiles, fit_tiles)) return 0;
+  return (int)ctas;
 }
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
   const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
@@ -515,9 +620,17 @@ void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cu
     ew_sample_pack_kernel<false><<<(unsigned)v.n_ctas, kEwThreads, smem, st>>>(v, key, kind_step);
   }
 }
+int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
+  const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
+  const size_t smem = (size_t)most * kEwWordsPerTile * sizeof(uint32_t) * (v.compact ? 2 : 1);
+  EwVec vv = v; double ss = s; PhiloxKey kk = key; uint32_t ks = kind_step;
+  void* args[] = {&vv, &ss, &kk, &ks};
+  const void* fn = v.compact ? (const void*)ew_encode_kernel<true> : (const void*)ew_encode_kernel<false>;
+  return (int)cudaLaunchCooperativeKernel(fn, dim3((unsigned)v.n_ctas), dim3(kEwThreads), args, smem, st);
+}
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {
   const int64_t tiles = (d.n + kEwTile - 1) / kEwTile;
-  ew_decode_kernel<<<(unsigned)std::min<int64_t>(tiles, 148 * 16), kEwThreads, 0, st>>>(d);
+  ew_decode_kernel<<<(unsigned)std::min<int64_t>(tiles, 1 << 20), kEwThreads, 0, st>>>(d);   // a tile per CTA: the CTAs of a wave hide one another's barriers
 }
 int ew_tile_elems() { return kEwTile; }
 

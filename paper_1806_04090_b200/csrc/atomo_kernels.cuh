@@ -53,6 +53,8 @@ int ew_tile_elems();
 void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax, double* part_sum, float* part_max,
                   int n_ctas, cudaStream_t st);
 int ew_sample_pack_ctas(int64_t n_tiles, bool compact);
+int ew_encode_ctas(int64_t n_tiles, bool compact);             // CTAs of the one-kernel form; 0 = the vector needs the two-kernel form
+int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st);   // cudaError_t
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
@@ -121,7 +123,7 @@ void launch_ew_decode_average(const uint8_t* const* d_payloads, int n_payloads, 
 
 // payload header (by value), layer headers from a device template, the call's four flag words (may be null)
 void launch_sp_begin(uint8_t* pay, const atomo_payload_header& gh, const atomo_layer_header* d_tmpl, int n_layers,
-                     uint32_t* d_flags, cudaStream_t st);
+                     uint32_t* d_flags, uint32_t* d_zero, int64_t n_zero, cudaStream_t st);
 void launch_sp_init(const SpLayer* d_layers, int n_layers, const TileRef* d_diag_tiles, int n_diag_tiles, cudaStream_t st);
 void launch_sp_gram(const SpLayer* d_layers, const TileRef* d_tiles, int n_tiles, cudaStream_t st);
 void launch_sp_scale(const SpLayer* d_layers, int n_layers, cudaStream_t st);   // trace, then scaling

@@ -152,13 +152,15 @@ __global__ void __launch_bounds__(256) sp_scale_kernel(const SpLayer* __restrict
 }
 
 // Start of an encode call: the payload header (passed by value), the layer headers from their template in the table
-// cache, and the call's flag words -- a kernel instead of host-to-device copies, which would queue behind whatever the
+// cache, the call's flag words and a region of the workspace that starts at zero (n_zero 32-bit words; small: status
+// words and tickets) -- a kernel instead of host-to-device copies and memsets, which would queue behind whatever the
 // application has on the copy engine.
 __global__ void __launch_bounds__(256) begin_kernel(uint8_t* __restrict__ pay, atomo_payload_header gh,
                                                     const atomo_layer_header* __restrict__ tmpl, int n_layers,
-                                                    uint32_t* __restrict__ flags) {
+                                                    uint32_t* __restrict__ flags, uint32_t* __restrict__ zero, int64_t n_zero) {
   if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<atomo_payload_header*>(pay) = gh;
   if (blockIdx.x == 0 && threadIdx.x < 4 && flags != nullptr) flags[threadIdx.x] = 0u;
+  for (int64_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n_zero; i += gridDim.x * blockDim.x) zero[i] = 0u;
   static_assert(sizeof(atomo_layer_header) % 16 == 0 && sizeof(atomo_payload_header) % 16 == 0, "headers are copied as 16-byte words");
   uint4* dst = reinterpret_cast<uint4*>(pay + sizeof(atomo_payload_header));
   const uint4* src = reinterpret_cast<const uint4*>(tmpl);
@@ -167,9 +169,9 @@ __global__ void __launch_bounds__(256) begin_kernel(uint8_t* __restrict__ pay, a
 }
 
 void launch_sp_begin(uint8_t* pay, const atomo_payload_header& gh, const atomo_layer_header* d_tmpl, int n_layers,
-                     uint32_t* d_flags, cudaStream_t st) {
-  const int n16 = n_layers * (int)(sizeof(atomo_layer_header) / 16);
-  begin_kernel<<<std::max(1, std::min(32, (n16 + 255) / 256)), 256, 0, st>>>(pay, gh, d_tmpl, n_layers, d_flags);
+                     uint32_t* d_flags, uint32_t* d_zero, int64_t n_zero, cudaStream_t st) {
+  const int64_t n16 = std::max<int64_t>(n_layers * (int64_t)(sizeof(atomo_layer_header) / 16), n_zero);
+  begin_kernel<<<(int)std::max<int64_t>(1, std::min<int64_t>(32, (n16 + 255) / 256)), 256, 0, st>>>(pay, gh, d_tmpl, n_layers, d_flags, d_zero, n_zero);
 }
 
 // A decomposition supplied by the caller (test entry point): lambda_i = sigma_i^2 in the eigenvalue slots (scale 1),

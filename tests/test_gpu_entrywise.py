@@ -184,3 +184,49 @@ def test_lq_budget_front_end(atomo, oracle):
     assert np.isnan(atomo.atomo_lq_budget([bad], 2.0)[0])
     with pytest.raises(Exception):
         atomo.atomo_lq_budget(ts[:1], 0.5)
+
+
+@pytest.mark.parametrize("compact", [False, True])
+def test_launch_forms_agree(atomo, compact):
+    """The one-kernel form (solve, grid barrier, sample and pack in one cooperative launch) and the two-kernel form
+    (solve kernel, then sample / pack with chunks handed out by ticket) cut the vector into different chunks on a
+    different number of CTAs: mask words, kept indices, values and decoded gradients have to be identical all the
+    same.  (sum |g| is added up in short fp32 runs and then chunk by chunk in fp64, so it depends on the cut at the
+    1e-8 level: it is compared to 1e-7.  The weight c = T / (s - n_s) and the scale of the probabilities are its
+    fp32 roundings; where they come out equal -- they do for these inputs -- everything else has to be identical.)"""
+    import torch
+    from paper_1806_04090_b200 import api
+    rng = np.random.default_rng(77)
+    big = rng.laplace(0.0, 1e-3, 3_000_017).astype(np.float32)
+    spiky = rng.laplace(0.0, 1e-3, 700_001).astype(np.float32)
+    spiky[rng.choice(spiky.size, 300, replace=False)] *= 1.0e4          # not s-balanced: saturated atoms
+    cases = [([big], 0.01 * big.size), ([spiky], 5000.0), ([big[:4097], spiky[:123], big[:40960]], 64.0)]
+    try:
+        for vecs, s in cases:
+            ts = [torch.from_numpy(g).cuda() for g in vecs]
+            k_cap = int(1.2 * s) + 2000
+            got = []
+            for two in (False, True):
+                atomo.set_entrywise_launch(two)
+                atomo.set_entrywise_format(api.EW_COMPACT if compact else api.EW_EXPLICIT, 1000 if compact else 0)
+                pay, dbg = atomo.atomo_encode_entrywise(ts, s, seed=5, step=3, k_cap=k_cap, debug=True)
+                outs = atomo.atomo_decode(pay)
+                torch.cuda.synchronize()
+                hdrs = pay.headers()
+                assert max(h.status for h in hdrs[1]) == 0
+                got.append((hdrs[1], [pay.layer_arrays(l, hdrs) for l in range(len(vecs))], dbg.mask_words.clone(),
+                            [o.clone() for o in outs]))
+            for l in range(len(vecs)):
+                h0, h1 = got[0][0][l], got[1][0][l]
+                assert abs(h0.l1 - h1.l1) <= 1e-7 * abs(h0.l1)
+                assert h0.c == h1.c, "the fp32 weight differs between the launch forms: choose other test inputs"
+            assert torch.equal(got[0][2], got[1][2]), "mask words differ between the launch forms"
+            for l in range(len(vecs)):
+                h0, h1 = got[0][0][l], got[1][0][l]
+                assert (h0.k, h0.n_sat, h0.sweeps) == (h1.k, h1.n_sat, h1.sweeps)
+                a0, a1 = got[0][1][l], got[1][1][l]
+                assert np.array_equal(a0["idx"], a1["idx"]) and np.array_equal(a0["val"], a1["val"])
+                assert torch.equal(got[0][3][l], got[1][3][l])
+    finally:
+        atomo.set_entrywise_launch(False)
+        atomo.set_entrywise_format(api.EW_EXPLICIT, 0)
