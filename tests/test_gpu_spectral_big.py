@@ -41,7 +41,8 @@ def _against_oracle(atomo, oracle, mats, s, seed, step):
         r = min(G.shape)
         arr = pay.layer_arrays(l, hdrs)
         out = outs[l].cpu().numpy().astype(np.float64)
-        parity.check_spectral_layer(oracle, G, encs[l], hdrs[1][l], arr, dbg, l, out, report, f"L{l}{G.shape}")
+        parity.check_spectral_layer(oracle, G, encs[l], hdrs[1][l], arr, dbg, l, out, report, f"L{l}{G.shape}",
+                                    gap_min=parity.gap_min_for(r, atomo.last_eig_scheme()))
         dp = float(np.abs(dbg.layer_prob(l, r) - encs[l]["p"]).max())
         report.append(f"L{l}{G.shape}: max |p - p_oracle| = {dp:.2e}")
         assert dp <= 2e-6

@@ -54,7 +54,7 @@ def _run(atomo, oracle, mats, s, seed, step=0, pad_ld=0, check_vectors=True):
         arr = pay.layer_arrays(l, hdrs)
         out = outs[l].cpu().numpy().astype(np.float64)
         same, _ = parity.check_spectral_layer(oracle, G, encs[l], hdrs[1][l], arr, dbg, l, out, report,
-                                              f"L{l}{G.shape}", check_vectors)
+                                              f"L{l}{G.shape}", check_vectors, gap_min=parity.gap_min_for(min(G.shape), TRIDIAG))
         # this route computes the kept vectors one by one: they must still be orthonormal among themselves
         # (the long-side vectors are back-projections: theirs is the orthogonality the fp32 Gram matrix allows for atoms
         # with small sigma, as on the Jacobi route)
