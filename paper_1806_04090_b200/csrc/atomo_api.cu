@@ -512,7 +512,7 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
     if (ctx->tri_clusters < 1) tri_form = false;
   }
   if (tri_form && any_big) {
-    if (ctx->tri_big_ok < 0) ctx->tri_big_ok = sp_configure_tridiag_big() == 0 ? 1 : 0;
+    if (ctx->tri_big_ok < 0) ctx->tri_big_ok = (sp_configure_tridiag_big() == 0 && sp_configure_bisect() == 0) ? 1 : 0;
     if (ctx->tri_big_ok < 1 || r_max > sp_tridiag_big_max_r()) tri_form = false;
   }
   std::vector<int> big_layers;

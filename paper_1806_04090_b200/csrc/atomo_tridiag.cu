@@ -586,13 +586,24 @@ int sp_tridiag_max_rp() { return kTriMaxRp; }
 int sp_tridiag_cluster_ctas() { return kTriCtas; }
 int sp_tridiag_ctas_of(int rp) { return rp / kTriRows < 1 ? 1 : rp / kTriRows; }
 
+// the eigenvalue kernel keeps d and e^2 of a layer in shared memory: more than the default 48 KB above a short side of
+// about 3000.  Both tridiagonal routes need this (a batch may hold large layers only).  0 if it went through.
+int sp_configure_bisect() {
+  const int bytes = (int)(2 * (kMaxShort + 10) * sizeof(double));
+  if (cudaFuncSetAttribute(sp_bisect_kernel<8, 13>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sp_bisect_kernel<2, 26>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return 1;
+  }
+  return 0;
+}
+
 int sp_configure_tridiag() {
   // optional route: a GPU that refuses the cluster size or the shared memory simply reports it as unavailable
   if (cudaFuncSetAttribute(sp_tridiag_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tri_smem_bytes(kTriMaxRp)) != cudaSuccess ||
       cudaFuncSetAttribute(sp_tridiag_cluster_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
       cudaFuncSetAttribute(sp_eigvec_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vec_smem_bytes(kTriMaxRp)) != cudaSuccess ||
-      cudaFuncSetAttribute(sp_bisect_kernel<8, 13>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (kMaxShort + 10) * sizeof(double))) != cudaSuccess ||
-      cudaFuncSetAttribute(sp_bisect_kernel<2, 26>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (kMaxShort + 10) * sizeof(double))) != cudaSuccess) {
+      sp_configure_bisect() != 0) {
     cudaGetLastError();
     return 0;
   }

@@ -17,9 +17,11 @@
 //                           added in fp64; column updates, norms and all scalars are fp64.  T = double keeps
 //                           everything in fp64.  Every sum has a fixed order that does not depend on C: a row product
 //                           is one warp's, block-wide sums go over the 32-row blocks in ascending order.
-//   sp_eigvec_big_kernel  : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
+//   sp_eigvec_big_warp_kernel / sp_eigvec_big_kernel (short sides up to 1024 / above)
+//                         : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
 //                           route, its work vectors in global memory), back-transformation u = Q z four reflectors at
-//                           a time (fp32), one warp per kept atom.
+//                           a time (fp32): one warp per kept atom up to a short side of 1024, above it the whole CTA
+//                           on up to eight atoms at once (the reflectors are then read once per eight atoms).
 //
 // The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
 // Work per layer: the matrix-vector products read sum_c (r - c)^2 ~ r^3 / 3 matrix entries (the bound of this kernel:
@@ -884,34 +886,100 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
 }
 
 // ---- vectors of the kept atoms ------------------------------------------------------------------------------------
+// Two phases per CTA.  (A) one warp per kept atom: the eigenvector of T by the twisted factorisation of the small
+// route (work vectors in global memory), normalised, filed in the payload's slot of the atom.  (B) the whole CTA
+// applies the reflectors to up to eight of its atoms at once, u = H_0 H_1 ... H_{r-3} z with H = I - 2 v v^T, from the
+// last reflector to the first, four at a time: a thread owns the columns tid, tid + 512, ... of the four reflector rows
+// (read once per group, kept in registers between the dot products and the update) and of every z (in shared memory;
+// no other thread touches them), so the only exchange per group is the block-wide sum of the products: v_i.z for
+// every atom and the six v_i.v_j.  For a group applied in the order 0, 1, 2, 3:  c_0 = 2 v_0.z,
+// c_i = 2 (v_i.z - sum_{j<i} c_j v_i.v_j),  z -= sum c_i v_i.  The matrix of reflectors is read once per eight atoms
+// instead of once per atom, by 512 threads instead of 32.
 namespace {
-constexpr int kVbThreads = 128;
+constexpr int kVbThreads = 512;
 constexpr int kVbWarps = kVbThreads / 32;
-constexpr int kVbCtas = 4;                   // CTAs per layer: 16 warps, one kept atom each at a time
+constexpr int kVbSlots = 16;                 // work-vector sets per layer (phase A: 16 atoms at a time over the layer's CTAs)
+constexpr int kVbMaxCtas = 4;                // CTAs per layer (the kept atoms are dealt to them)
+constexpr int kVbBatch = 8;                  // atoms per pass over the reflectors
+constexpr int kVbCols = kTbMaxR / kVbThreads;   // columns per thread and reflector row (8)
+constexpr int kVbSums = 4 * kVbBatch + 6;    // products summed per group
 constexpr double kVbSameEig = 1.0e-9;        // as on the small route
 }  // namespace
 
-__global__ void __launch_bounds__(kVbThreads) sp_eigvec_big_kernel(const SpLayer* __restrict__ layers,
+namespace {
+// The last CTA of a layer to finish orthogonalises kept atoms whose eigenvalues nearly coincide (their vectors are
+// determined only as a subspace): modified Gram-Schmidt in payload order, one warp.  Called by every thread of the CTA.
+__device__ __forceinline__ void vb_orthogonalise_equal(const SpLayer& L, uint32_t k, int n_ctas) {
+  __shared__ uint32_t s_last;
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const int r = L.r;
+  const double* const gLam = L.lam64; const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(L.vec_ticket, 1u) == (uint32_t)(n_ctas - 1) ? 1u : 0u;
+  __syncthreads();
+  if (!s_last || w != 0 || k < 2) return;
+  __threadfence();
+  for (uint32_t a = 1; a < k; ++a) {
+    const double la = gLam[gPerm[gIdx[a]]];
+    bool changed = false;
+    for (uint32_t b = 0; b < a; ++b) {
+      const double lb = gLam[gPerm[gIdx[b]]];
+      if (fabs(la - lb) > kVbSameEig) continue;
+      volatile float* va = gShort + (int64_t)a * r;
+      const volatile float* vb = gShort + (int64_t)b * r;
+      double dot = 0.0;
+      for (int i = lane; i < r; i += 32) dot = fma((double)va[i], (double)vb[i], dot);
+      dot = warp_sum(dot);
+      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] - dot * (double)vb[i]);
+      __syncwarp();
+      changed = true;
+    }
+    if (changed) {
+      volatile float* va = gShort + (int64_t)a * r;
+      double n2 = 0.0;
+      for (int i = lane; i < r; i += 32) n2 = fma((double)va[i], (double)va[i], n2);
+      n2 = warp_sum(n2);
+      const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
+      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] * inv);
+      __syncwarp();
+    }
+  }
+}
+}  // namespace
+
+
+namespace {
+constexpr int kVwThreads = 128;              // the warp-per-atom form: short sides up to 1024, many layers
+constexpr int kVwWarps = kVwThreads / 32;
+constexpr int kVwCtas = 4;                   // CTAs per layer: 16 warps, one kept atom each at a time
+constexpr int kVwMaxRp = 1024;
+}  // namespace
+
+// Short sides up to 1024: one warp per kept atom, 16 warps per layer on four small CTAs.  A batch of many such layers
+// (config 5: 96) fills the GPU with independent warps, which hides the latency of the reflector rows better than a
+// CTA-wide exchange per group of reflectors would.
+__global__ void __launch_bounds__(kVwThreads) sp_eigvec_big_warp_kernel(const SpLayer* __restrict__ layers,
                                                                    const int* __restrict__ big_layers) {
   const SpLayer& L = layers[big_layers[blockIdx.x]];
+  if (L.rp > kVwMaxRp) return;                                // larger layers: the cooperative kernel
   extern __shared__ __align__(16) unsigned char vb_smem[];
   const int r = L.r, rp = L.rp;
   double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
   double* s_e = s_d + rp;                                      // [rp]
   float* s_z = reinterpret_cast<float*>(s_e + rp);             // [warps][rp]
-  __shared__ uint32_t s_last;
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const uint32_t k = L.hdr->k;
   const float* const gV = L.td_V; const int64_t ldv = L.td_ldv; const double* const gLam = L.lam64;
   const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
   const int nref = max(r - 2, 0);
-  for (int i = tid; i < r; i += kVbThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
+  for (int i = tid; i < r; i += kVwThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
   __syncthreads();
-  const int slot = blockIdx.y * kVbWarps + w;                  // 0 .. 15
+  const int slot = blockIdx.y * kVwWarps + w;                  // 0 .. 15
   double* wa = L.tb_vecwork + (size_t)slot * 5 * rp;
   double* wb = wa + rp; double* wc = wb + rp; double* wd = wc + rp; double* zz = wd + rp;
   float* z = s_z + (size_t)w * rp;
-  for (uint32_t a = slot; a < k; a += kVbCtas * kVbWarps) {
+  for (uint32_t a = slot; a < k; a += kVwCtas * kVwWarps) {
     const int ei = gPerm[gIdx[a]];                             // index of the atom's eigenvalue (ascending order)
     double lambda = gLam[ei];
     int skip = 0;                                              // earlier kept atoms with the same eigenvalue: another twist index each
@@ -994,39 +1062,180 @@ __global__ void __launch_bounds__(kVbThreads) sp_eigvec_big_kernel(const SpLayer
     for (int i = lane; i < r; i += 32) gShort[(int64_t)a * r + i] = z[i] * invf;
     __syncwarp();
   }
-  // the last CTA of the layer orthogonalises kept atoms whose eigenvalues nearly coincide (their vectors are
-  // determined only as a subspace): modified Gram-Schmidt in payload order, one warp
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = atomicAdd(L.vec_ticket, 1u) == (uint32_t)(kVbCtas - 1) ? 1u : 0u;
-  __syncthreads();
-  if (!s_last || w != 0 || k < 2) return;
-  __threadfence();
-  for (uint32_t a = 1; a < k; ++a) {
-    const double la = gLam[gPerm[gIdx[a]]];
-    bool changed = false;
-    for (uint32_t b = 0; b < a; ++b) {
-      const double lb = gLam[gPerm[gIdx[b]]];
-      if (fabs(la - lb) > kVbSameEig) continue;
-      volatile float* va = gShort + (int64_t)a * r;
-      const volatile float* vb = gShort + (int64_t)b * r;
-      double dot = 0.0;
-      for (int i = lane; i < r; i += 32) dot = fma((double)va[i], (double)vb[i], dot);
-      dot = warp_sum(dot);
-      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] - dot * (double)vb[i]);
-      __syncwarp();
-      changed = true;
+  vb_orthogonalise_equal(L, k, kVwCtas);
+}
+
+namespace {
+// the columns tid, tid + 512, ... of the four reflector rows top, top - 1, top - 2, top - 3 (rows below 0: zeros)
+template <int COLS>
+__device__ __forceinline__ void vb_load_rows(const float* __restrict__ gV, int64_t ldv, int r, int top, float (&q)[4][COLS]) {
+  const int tid = threadIdx.x;
+  const float* v0 = gV + (int64_t)top * ldv;
+  const float* v1 = gV + (int64_t)max(top - 1, 0) * ldv;
+  const float* v2 = gV + (int64_t)max(top - 2, 0) * ldv;
+  const float* v3 = gV + (int64_t)max(top - 3, 0) * ldv;
+  const bool e1 = top - 1 >= 0, e2 = top - 2 >= 0, e3 = top - 3 >= 0;
+  const int h0 = max(top - 3, 0) + 1;                          // reflector kk is zero up to index kk
+#pragma unroll
+  for (int m = 0; m < COLS; ++m) {
+    const int h = tid + m * kVbThreads;
+    const bool in = h >= h0 && h < r;
+    q[0][m] = in ? __ldcg(v0 + h) : 0.0f;
+    q[1][m] = in && e1 ? __ldcg(v1 + h) : 0.0f;
+    q[2][m] = in && e2 ? __ldcg(v2 + h) : 0.0f;
+    q[3][m] = in && e3 ? __ldcg(v3 + h) : 0.0f;
+  }
+}
+
+// z_b <- H_0 ... H_{nref-1} z_b for the nb vectors in s_z, the whole CTA.  PREFETCH: the next group's rows are on their
+// way while this group's sums are added up (needs twice the registers for the rows: short sides up to 2048).
+template <int COLS, bool PREFETCH>
+__device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV, int64_t ldv, int r, int rp, int nref, int nb,
+                                                    float* s_z, float (*s_part)[kVbSums], float* s_tot) {
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  float q[4][COLS], qn[4][PREFETCH ? COLS : 1];
+  if (PREFETCH && nref > 0) vb_load_rows<COLS>(gV, ldv, r, nref - 1, q);
+  for (int top = nref - 1; top >= 0; top -= 4) {
+    if (!PREFETCH) vb_load_rows<COLS>(gV, ldv, r, top, q);
+    float acc[kVbSums];
+#pragma unroll
+    for (int x = 0; x < kVbSums; ++x) acc[x] = 0.0f;
+#pragma unroll
+    for (int m = 0; m < COLS; ++m) {
+      const int h = tid + m * kVbThreads;
+      if (h < r) {
+        acc[0] = fmaf(q[1][m], q[0][m], acc[0]); acc[1] = fmaf(q[2][m], q[0][m], acc[1]); acc[2] = fmaf(q[2][m], q[1][m], acc[2]);
+        acc[3] = fmaf(q[3][m], q[0][m], acc[3]); acc[4] = fmaf(q[3][m], q[1][m], acc[4]); acc[5] = fmaf(q[3][m], q[2][m], acc[5]);
+#pragma unroll
+        for (int b = 0; b < kVbBatch; ++b) {
+          if (b < nb) {
+            const float zh = s_z[(size_t)b * rp + h];
+            acc[6 + 4 * b + 0] = fmaf(q[0][m], zh, acc[6 + 4 * b + 0]); acc[6 + 4 * b + 1] = fmaf(q[1][m], zh, acc[6 + 4 * b + 1]);
+            acc[6 + 4 * b + 2] = fmaf(q[2][m], zh, acc[6 + 4 * b + 2]); acc[6 + 4 * b + 3] = fmaf(q[3][m], zh, acc[6 + 4 * b + 3]);
+          }
+        }
+      }
     }
-    if (changed) {
-      volatile float* va = gShort + (int64_t)a * r;
-      double n2 = 0.0;
-      for (int i = lane; i < r; i += 32) n2 = fma((double)va[i], (double)va[i], n2);
-      n2 = warp_sum(n2);
+    if (PREFETCH && top - 4 >= 0) vb_load_rows<COLS>(gV, ldv, r, top - 4, reinterpret_cast<float (&)[4][COLS]>(qn));
+    const int n_sums = 6 + 4 * nb;
+#pragma unroll
+    for (int x = 0; x < kVbSums; ++x) {
+      if (x < n_sums) {
+        const float t = warp_sum(acc[x]);
+        if (lane == 0) s_part[w][x] = t;
+      }
+    }
+    __syncthreads();
+    if (tid < n_sums) {
+      float t = 0.0f;
+#pragma unroll
+      for (int ww = 0; ww < kVbWarps; ++ww) t += s_part[ww][tid];
+      s_tot[tid] = t;
+    }
+    __syncthreads();
+    const float g10 = s_tot[0], g20 = s_tot[1], g21 = s_tot[2], g30 = s_tot[3], g31 = s_tot[4], g32 = s_tot[5];
+#pragma unroll
+    for (int b = 0; b < kVbBatch; ++b) {
+      if (b < nb) {
+        const float c0 = 2.0f * s_tot[6 + 4 * b];
+        const float c1 = 2.0f * (s_tot[6 + 4 * b + 1] - c0 * g10);
+        const float c2 = 2.0f * (s_tot[6 + 4 * b + 2] - c0 * g20 - c1 * g21);
+        const float c3 = 2.0f * (s_tot[6 + 4 * b + 3] - c0 * g30 - c1 * g31 - c2 * g32);
+#pragma unroll
+        for (int m = 0; m < COLS; ++m) {
+          const int h = tid + m * kVbThreads;
+          if (h < r) s_z[(size_t)b * rp + h] -= fmaf(c0, q[0][m], fmaf(c1, q[1][m], fmaf(c2, q[2][m], c3 * q[3][m])));
+        }
+      }
+    }
+    // (the next group's partial sums go to s_part only after the barrier that follows them in program order for the
+    // slowest reader of s_tot: two barriers separate a write from the reads of the group before)
+    if (PREFETCH) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int m = 0; m < COLS; ++m) q[x][m] = qn[x][PREFETCH ? m : 0];
+    }
+  }
+}
+}  // namespace
+
+__global__ void __launch_bounds__(kVbThreads, 1) sp_eigvec_big_kernel(const SpLayer* __restrict__ layers,
+                                                                      const int* __restrict__ big_layers) {
+  const SpLayer& L = layers[big_layers[blockIdx.x]];
+  if (L.rp <= kVwMaxRp) return;                                // smaller layers: the warp-per-atom kernel
+  extern __shared__ __align__(16) unsigned char vb_smem[];
+  const int r = L.r, rp = L.rp;
+  double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
+  double* s_e = s_d + rp;                                      // [rp]
+  float* s_z = reinterpret_cast<float*>(s_e + rp);             // [kVbBatch][rp]
+  __shared__ float s_part[kVbWarps][kVbSums];
+  __shared__ float s_tot[kVbSums];
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const int n_ctas = gridDim.y, cy = blockIdx.y;
+  const uint32_t k = L.hdr->k;
+  const float* const gV = L.td_V; const int64_t ldv = L.td_ldv; const double* const gLam = L.lam64;
+  const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
+  const int nref = max(r - 2, 0);
+  for (int i = tid; i < r; i += kVbThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
+  __syncthreads();
+  // ---- (A) this CTA's atoms are a = cy, cy + n_ctas, ...; warp w < slots-per-CTA takes every (slots-per-CTA)-th of them ----
+  const int spc = kVbSlots / n_ctas;                           // work-vector sets of this CTA
+  if (w < spc) {
+    double* wa = L.tb_vecwork + (size_t)(cy * spc + w) * 5 * rp;
+    double* wb = wa + rp; double* wc = wb + rp; double* wd = wc + rp; double* zz = wd + rp;
+    for (uint32_t a = cy + (uint32_t)n_ctas * w; a < k; a += (uint32_t)(n_ctas * spc)) {
+      const int ei = gPerm[gIdx[a]];                           // index of the atom's eigenvalue (ascending order)
+      double lambda = gLam[ei];
+      int skip = 0;                                            // earlier kept atoms with the same eigenvalue: another twist index each
+      for (uint32_t b2 = lane; b2 < a; b2 += 32) skip += fabs(gLam[gPerm[gIdx[b2]]] - lambda) <= kVbSameEig ? 1 : 0;
+      skip = (int)warp_sum((uint32_t)skip);
+      double n2 = 1.0;
+      const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, skip, &n2);
+      double gap = 1.0e300;
+      if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
+      if (ei + 1 < r) gap = fmin(gap, fabs(gLam[ei + 1] - lambda));
+      if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {    // one Rayleigh-quotient step, then the vector again
+        lambda += corr;
+        __syncwarp();
+        twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, 0, &n2);
+      }
+      __syncwarp();
       const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
-      for (int i = lane; i < r; i += 32) va[i] = (float)((double)va[i] * inv);
+      for (int i = lane; i < r; i += 32) gShort[(int64_t)a * r + i] = (float)(zz[i] * inv);
       __syncwarp();
     }
   }
+  __syncthreads();
+  // ---- (B) back-transformation, kVbBatch of this CTA's atoms per pass over the reflectors ----
+  const uint32_t n_mine = k > (uint32_t)cy ? (k - (uint32_t)cy + (uint32_t)n_ctas - 1u) / (uint32_t)n_ctas : 0u;
+  for (uint32_t b0 = 0; b0 < n_mine; b0 += kVbBatch) {
+    const int nb = (int)min((uint32_t)kVbBatch, n_mine - b0);
+    for (int b = 0; b < nb; ++b) {
+      const float* src = gShort + (int64_t)(cy + (b0 + b) * n_ctas) * r;
+      for (int i = tid; i < r; i += kVbThreads) s_z[(size_t)b * rp + i] = src[i];
+    }
+    __syncthreads();
+    if (rp <= 4 * kVbThreads) vb_apply_reflectors<4, true>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
+    else vb_apply_reflectors<8, false>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
+    // normalise and file
+    for (int b = 0; b < nb; ++b) {
+      float n2f = 0.0f;
+      for (int i = tid; i < r; i += kVbThreads) n2f = fmaf(s_z[(size_t)b * rp + i], s_z[(size_t)b * rp + i], n2f);
+      n2f = warp_sum(n2f);
+      __syncthreads();
+      if (lane == 0) s_part[w][0] = n2f;
+      __syncthreads();
+      float tot = 0.0f;
+#pragma unroll
+      for (int ww = 0; ww < kVbWarps; ++ww) tot += s_part[ww][0];
+      const float invf = tot > 0.0f ? rsqrtf(tot) : 0.0f;
+      float* dst = gShort + (int64_t)(cy + (b0 + b) * n_ctas) * r;
+      for (int i = tid; i < r; i += kVbThreads) dst[i] = s_z[(size_t)b * rp + i] * invf;
+    }
+    __syncthreads();
+  }
+  vb_orthogonalise_equal(L, k, n_ctas);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------------------
@@ -1040,7 +1249,8 @@ template <typename T> size_t tb_smem_bytes(int r_max) {
 size_t t1_smem_bytes() {
   return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + (size_t)kT1MaxB * kT1MaxB * kT1Blk);
 }
-size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbWarps * sizeof(float)); }
+size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbBatch * sizeof(float)); }
+size_t vw_smem_bytes(int rp_max) { return (size_t)std::min(rp_max, kVwMaxRp) * (2 * sizeof(double) + kVwWarps * sizeof(float)); }
 
 template <typename T, int C> int tb_configure_one() {
   auto* fn = sp_tridiag_big_kernel<T, C>;
@@ -1069,7 +1279,7 @@ int tb_launch_one(const SpLayer* d_layers, const int* d_big, int n_big, int r_ma
 int sp_tridiag_big_max_r() { return kTbMaxR; }
 int sp_tridiag_big_panel() { return kTbNB; }
 int sp_tridiag_big_min_ctas(int r) { int c = 1; while (c < kTbMaxC && (int64_t)c * kTbThreads < r) c <<= 1; return c; }
-int sp_eigvec_big_slots() { return kVbCtas * kVbWarps; }
+int sp_eigvec_big_slots() { return kVbSlots; }
 
 // 0 if the route is available on this GPU
 int sp_configure_tridiag_big() {
@@ -1080,6 +1290,7 @@ int sp_configure_tridiag_big() {
          tb_configure_one<double, 8>() | tb_configure_one<double, 16>();
   bad |= cudaFuncSetAttribute(sp_tridiag_big1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t1_smem_bytes()) != cudaSuccess;
   bad |= cudaFuncSetAttribute(sp_eigvec_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vb_smem_bytes(kTbMaxR)) != cudaSuccess;
+  bad |= cudaFuncSetAttribute(sp_eigvec_big_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)kTbMaxR * (2 * sizeof(double) + kVwWarps * sizeof(float)))) != cudaSuccess;
   if (bad) cudaGetLastError();
   return bad;
 }
@@ -1099,7 +1310,16 @@ int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, 
 
 void launch_sp_eigvec_big(const SpLayer* d_layers, const int* d_big, int n_big, int rp_max, cudaStream_t st) {
   if (n_big <= 0) return;
-  sp_eigvec_big_kernel<<<dim3(n_big, kVbCtas), kVbThreads, vb_smem_bytes(rp_max), st>>>(d_layers, d_big);
+  // layers up to a short side of 1024: one warp per kept atom (the other kernel's CTAs leave such layers at once, and
+  // the other way round)
+  sp_eigvec_big_warp_kernel<<<dim3(n_big, kVwCtas), kVwThreads, vw_smem_bytes(rp_max), st>>>(d_layers, d_big);
+  if (rp_max <= kVwMaxRp) return;
+  // larger layers: CTAs per layer (1, 2 or 4; the kept atoms are dealt to them), as many as keep the launch within one wave
+  static int sms = 0;
+  if (sms == 0) { int dev = 0; if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 1; }
+  int per = 1;
+  while (per < kVbMaxCtas && n_big * per * 2 <= sms) per *= 2;
+  sp_eigvec_big_kernel<<<dim3(n_big, per), kVbThreads, vb_smem_bytes(rp_max), st>>>(d_layers, d_big);
 }
 
 }  // namespace atomo

@@ -15,7 +15,7 @@ constexpr double kPivMin = 1.0e-280;
 // quotients are taken by all lanes afterwards.  Twist index at the smallest |gamma_k| = |D+_k + D-_k - (d_k - lambda)|,
 // z_k = 1, z_i = -(e_i / D+_i) z_{i+1} above and z_{i+1} = -(e_i / D-_{i+1}) z_i below.  Returns gamma_k / z^T z, the
 // Rayleigh-quotient correction of lambda.  wa, wb, wc, wd, z: r doubles each, in shared or global memory.
-static __device__ double twisted_vector(const double* __restrict__ d, const double* __restrict__ e, int r, double lambda,
+static __device__ __noinline__ double twisted_vector(const double* __restrict__ d, const double* __restrict__ e, int r, double lambda,
                                  double* wa, double* wb, double* wc, double* wd, double* z, int lane, int skip,
                                  double* znorm2) {
   if (lane < 2) {

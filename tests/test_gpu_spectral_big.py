@@ -136,3 +136,27 @@ def test_saturated_and_rank_deficient_large_layers(atomo, oracle):
     assert hdrs[1][1].status == 4 and hdrs[1][1].k == 0
     outs = atomo.atomo_decode(pay)
     assert not outs[0].any() and not outs[1].any()
+
+
+def test_large_layers_alone_in_a_fresh_process():
+    """A batch that holds nothing but layers above a short side of 3000 (the eigenvalue kernel then needs more than
+    the default 48 KB of shared memory) in a process that has encoded nothing else before: the shared-memory opt-ins
+    of every kernel on the way must not depend on another route having been configured first."""
+    import subprocess
+    import sys
+    code = (
+        "import numpy as np, torch\n"
+        "from paper_1806_04090_b200 import api, synth\n"
+        "a = api.Atomo(0)\n"
+        "G = synth.torch_lowrank_plus_noise(3100, 3200, 1.0, 5, torch.device('cuda:0'), noise_rel=0.01)\n"
+        "pay, dbg = a.atomo_encode_spectral([G], 2.0, seed=3, step=1, k_cap=16, debug=True)\n"
+        "h = pay.headers()[1][0]\n"
+        "assert h.status == 0 and a.last_eig_scheme() == 3, (h.status, a.last_eig_scheme())\n"
+        "sig = dbg.layer_sigma(0, 3100)\n"
+        "ref = torch.linalg.svdvals(G.double()).cpu().numpy()\n"
+        "assert np.linalg.norm(sig - ref) <= 1e-4 * np.linalg.norm(ref)\n"
+        "out = a.atomo_decode(pay)[0]\n"
+        "assert torch.isfinite(out).all()\n"
+        "print('ok', int(h.k))\n")
+    res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=600)
+    assert res.returncode == 0 and res.stdout.strip().startswith("ok"), res.stdout + res.stderr
