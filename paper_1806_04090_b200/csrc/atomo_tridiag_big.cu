@@ -497,22 +497,22 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
 // kernel above, all of them about bytes:
 //   * only the lower triangle of A0 is read and updated.  The product y = A0 u goes over 64 x 64 tiles of the
 //     triangle, one warp per tile: a tile contributes its rows' sums to block I of y and, transposed, its columns'
-//     sums to block J, both into a table of partial vectors in shared memory (slot J of block I, slot I of block J:
-//     every slot has one writer), which the row owners add up in ascending slot order.  Per 32 x 32 sub-tile a lane
-//     holds 8 x 4 entries; the sums over the 8 lanes of a row and the 4 lanes of a column are reduce-scatters (7 + 3
-//     shuffles).  Half the bytes per step of the row-wise product.
+//     sums to block J, both added to y in fixed point with integer shared-memory atomics (integer addition commutes:
+//     the result does not depend on which warp finishes first).  Per 32 x 32 sub-tile a lane holds 8 x 4 entries; the
+//     sums over the 8 lanes of a row and the 4 lanes of a column are reduce-scatters (7 + 3 shuffles).  Half the bytes
+//     per step of the row-wise product.  A warp has three sub-tiles in work or on their way: two in registers, one in
+//     a 4 KB buffer of its own in shared memory filled by cp.async.
 //   * the panel (16 columns: u_t and w_t of all rows) lives in shared memory, so the column update, the correction
 //     of y and the panel dots never leave the SM, and the rank-32 update at the end of a panel takes its operands
 //     from there (4 x 4 outputs per thread on 128 x 128 tiles of the lower triangle).
 //   * 512 threads; thread t owns rows t and t + 512 for the whole reduction.
 namespace {
 
-constexpr int kT1Threads = 512;              // 128 registers per thread: two sub-tiles of the product in flight per warp
+constexpr int kT1Threads = 512;              // 128 registers per thread: two sub-tiles of the product in registers per warp
 constexpr int kT1Warps = kT1Threads / 32;
 constexpr int kT1NB = 16;                    // columns per panel
 constexpr int kT1MaxR = 1024;
 constexpr int kT1Blk = 64;                   // tile edge of the matrix-vector product
-constexpr int kT1MaxB = kT1MaxR / kT1Blk;    // 16 blocks
 
 struct alignas(16) T1Shared {
   double part_a[32];
@@ -546,6 +546,19 @@ __device__ __forceinline__ float rs8(float (&v)[8], int lane) {
   const float send = b1 ? b[0] : b[1], keep = b1 ? b[1] : b[0];
   return keep + __shfl_xor_sync(0xffffffffu, send, 1);
 }
+// y[row] += v in fixed point: v 2^48 as a 64-bit integer, its upper 40 and lower 24 bits added to two 32-bit words.
+// Integer addition commutes, so the sums of y do not depend on the order in which the warps finish their tiles.  (At
+// most 64 additions per row and step: the lower word cannot overflow; |v| < 2^7, and the matrix has trace 1.)
+__device__ __forceinline__ void t1_add_fix(int32_t* yhi, uint32_t* ylo, int row, float v) {
+  const long long q = __float2ll_rn(v * 281474976710656.0f);
+  atomicAdd(yhi + row, (int32_t)(q >> 24));
+  atomicAdd(ylo + row, (uint32_t)(q & 0xffffffll));
+}
+// 16 bytes from global (L2) to shared memory without passing through registers; waited for with cp.async.wait_group
+__device__ __forceinline__ void t1_cp16(float* dst_smem, const float* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
+}
+
 // sum over the 4 lanes ly = lane / 8 of v[j]: lane ly ends with the total of j = ly
 __device__ __forceinline__ float rs4(float (&v)[4], int lane) {
   const bool b2 = lane & 16, b1 = lane & 8;
@@ -568,7 +581,9 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
   float* const s_u = reinterpret_cast<float*>(tb_smem + sizeof(T1Shared));     // [1024] current reflector (zero up to c and from r on)
   float* const pan_u = s_u + kT1MaxR;                                          // [16][1024]
   float* const pan_w = pan_u + kT1NB * kT1MaxR;                                // [16][1024]
-  float* const y_part = pan_w + kT1NB * kT1MaxR;                               // [16 blocks][16 slots][64]
+  int32_t* const yhi = reinterpret_cast<int32_t*>(pan_w + kT1NB * kT1MaxR);    // [1024] y in fixed point, upper word
+  uint32_t* const ylo = reinterpret_cast<uint32_t*>(yhi + kT1MaxR);            // [1024] lower word
+  float* const stage = reinterpret_cast<float*>(ylo + kT1MaxR) + (threadIdx.x / 32) * 1024;   // this warp's third sub-tile buffer (4 KB)
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   const SpLayer& L = layers[big_layers[blockIdx.x]];
   const int r = L.r;
@@ -587,6 +602,7 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
   const int idx = 4 * lx + ly;                                                 // the column a lane ends up with after the reduce-scatter
 
   s_u[g[0]] = 0.0f; s_u[g[1]] = 0.0f;
+  yhi[g[0]] = 0; yhi[g[1]] = 0; ylo[g[0]] = 0u; ylo[g[1]] = 0u;
   // the lower triangle of A into tile-major order (one warp per sub-tile: 32 rows of 128 bytes in, 4 KB out)
   for (int k = w; k < nblk * (nblk + 1) / 2; k += kT1Warps) {
     int I = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);
@@ -676,10 +692,7 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
       // 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3.  Row sums are accumulated over the sub-tiles of a row half
       // before the eight lanes of a row are added up (reduce-scatter: lane 8 ly + lx ends with row 8 ly + lx), column
       // sums over the sub-tiles of a column half before the four lanes of a column are (lane ends with column
-      // 4 lx + ly).  The tile's sums go to slot J of block I (rows) and slot I of block J (columns): every slot has
-      // exactly one writer per step.  Two sub-tiles are in flight per warp: while one is multiplied the next 4 KB
-      // are on their way (with a single one in flight the SM's loads stop during the arithmetic and the kernel
-      // reaches little more than half of the memory's rate).
+      // 4 lx + ly).  The tile's sums are added to the fixed-point words of y (rows of block I, columns of block J).
       const int j0 = (c + 1) / kT1Blk;                                         // first live block
       const int nbl = nb64 - j0;
       const int n_tiles = nbl * (nbl + 1) / 2;
@@ -707,7 +720,16 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
       float rp[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
       float racc[2] = {0.f, 0.f};
       uint64_t cp[2][2] = {{pack2(0.f, 0.f), pack2(0.f, 0.f)}, {pack2(0.f, 0.f), pack2(0.f, 0.f)}};   // [column half][pair of columns]
-      auto process = [&](const float4 (&t)[8], const Sub& cur, const Sub& nxt) {
+      // the same sub-tile fetched into this warp's buffer in shared memory (each lane copies the sixteen-byte pieces it
+      // will read itself)
+      auto load_stage = [&](const Sub& sbt) {
+        const float* src = t1_sub(At, 2 * sbt.I + (sbt.q >> 1), 2 * sbt.J + (sbt.q & 1)) + (8 * ly) * 32 + 4 * lx;
+        float* dst = stage + (8 * ly) * 32 + 4 * lx;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) t1_cp16(dst + kk * 32, src + kk * 32);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      };
+      auto process = [&](auto get, const Sub& cur, const Sub& nxt) {
         const int sa = cur.q >> 1, sb = cur.q & 1;
         const int row0 = kT1Blk * cur.I + 32 * sa, col0 = kT1Blk * cur.J + 32 * sb;
         const bool diag = row0 == col0;
@@ -719,7 +741,7 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
         uint64_t c01 = pack2(0.f, 0.f), c23 = pack2(0.f, 0.f);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          float4 v = t[kk];
+          float4 v = get(kk);
           const int rr = 8 * ly + kk, cc = 4 * lx;                             // position inside the sub-tile
           if (diag) {                                                          // lower triangle only
             if (cc + 0 > rr) v.x = 0.f;
@@ -761,40 +783,46 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
             cacc[hb] = rs4(cv, lane);
             cp[hb][0] = pack2(0.f, 0.f); cp[hb][1] = pack2(0.f, 0.f);
           }
-          float* yi = y_part + ((size_t)cur.I * kT1MaxB + cur.J) * kT1Blk;
-          if (cur.I == cur.J) {
-            // rows and columns of the same block: a column's sum moves to the lane that holds the row of the same index
-            const int from = ((lane & 3) << 3) | (lane >> 2);
-            yi[lane] = racc[0] + __shfl_sync(0xffffffffu, cacc[0], from);
-            yi[32 + lane] = racc[1] + __shfl_sync(0xffffffffu, cacc[1], from);
-          } else {
-            yi[lane] = racc[0]; yi[32 + lane] = racc[1];
-            float* yj = y_part + ((size_t)cur.J * kT1MaxB + cur.I) * kT1Blk;
-            yj[idx] = cacc[0]; yj[32 + idx] = cacc[1];
-          }
+          // lane 8 ly + lx holds row 8 ly + lx of each row half and column 4 lx + ly of each column half
+          t1_add_fix(yhi, ylo, kT1Blk * cur.I + lane, racc[0]);
+          t1_add_fix(yhi, ylo, kT1Blk * cur.I + 32 + lane, racc[1]);
+          t1_add_fix(yhi, ylo, kT1Blk * cur.J + idx, cacc[0]);
+          t1_add_fix(yhi, ylo, kT1Blk * cur.J + 32 + idx, cacc[1]);
           racc[0] = 0.f; racc[1] = 0.f;
         }
       };
-      Sub s0{w, 0, 0, 0};
-      if (s0.k < n_tiles) tile_of(s0);
-      settle(s0);
-      if (s0.k < n_tiles) {
+      // Three sub-tiles per warp on their way or in work: two in registers (ta, tb), one in the warp's buffer in shared
+      // memory (filled by cp.async, which holds no registers while it flies).  While one is multiplied the other two
+      // are in flight: with a single one in flight the SM's loads stop during the arithmetic, and the latency of DRAM
+      // (two to three thousand cycles under load) is more than one sub-tile's arithmetic covers.
+      Sub e0{w, 0, 0, 0};
+      if (e0.k < n_tiles) tile_of(e0);
+      settle(e0);
+      if (e0.k < n_tiles) {
+        auto ok = [&](const Sub& e) { return e.k < n_tiles; };
+        auto after = [&](const Sub& e) { return ok(e) ? next_of(e) : e; };
         float4 ta[8], tb[8];
-        Sub s1 = next_of(s0);
-        load(ta, s0);
-        if (s1.k < n_tiles) load(tb, s1);
+        Sub e1 = after(e0), e2 = after(e1);
+        load(ta, e0);
+        if (ok(e1)) load(tb, e1);
+        if (ok(e2)) load_stage(e2);
         for (;;) {
-          Sub s2 = s1;
-          if (s1.k < n_tiles) s2 = next_of(s1);
-          process(ta, s0, s1);
-          if (s1.k >= n_tiles) break;
-          if (s2.k < n_tiles) load(ta, s2);
-          Sub s3 = s2;
-          if (s2.k < n_tiles) s3 = next_of(s2);
-          process(tb, s1, s2);
-          if (s2.k >= n_tiles) break;
-          if (s3.k < n_tiles) load(tb, s3);
-          s0 = s2; s1 = s3;
+          const Sub e3 = after(e2);
+          process([&](int kk) { return ta[kk]; }, e0, e1);
+          if (!ok(e1)) break;
+          if (ok(e3)) load(ta, e3);
+          const Sub e4 = after(e3);
+          process([&](int kk) { return tb[kk]; }, e1, e2);
+          if (!ok(e2)) break;
+          if (ok(e4)) load(tb, e4);
+          const Sub e5 = after(e4);
+          asm volatile("cp.async.wait_group 0;" ::: "memory");
+          __syncwarp();
+          process([&](int kk) { return *reinterpret_cast<const float4*>(stage + (8 * ly + kk) * 32 + 4 * lx); }, e2, e3);
+          if (!ok(e3)) break;
+          __syncwarp();                                                        // every lane has read the buffer
+          if (ok(e5)) load_stage(e5);
+          e0 = e3; e1 = e4; e2 = e5;
         }
       }
     }
@@ -802,13 +830,16 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
     TB_MARK(2)
     // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
     double p[2] = {0.0, 0.0};
+    long long yq[2];                                                           // this thread's two rows of y, in fixed point; the words start the next step at zero
 #pragma unroll
     for (int x = 0; x < 2; ++x) {
-      if (live[x]) {                                                           // this row's partial sums in ascending slot order
-        const int j0 = (c + 1) / kT1Blk;
-        const float* yp = y_part + (size_t)(g[x] / kT1Blk) * kT1MaxB * kT1Blk + (g[x] % kT1Blk);
-        double y = 0.0;
-        for (int sl = j0; sl < nb64; ++sl) y += (double)yp[sl * kT1Blk];
+      yq[x] = (long long)yhi[g[x]] * 16777216ll + (long long)ylo[g[x]];
+      yhi[g[x]] = 0; ylo[g[x]] = 0u;
+    }
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      if (live[x]) {
+        double y = (double)yq[x] * 3.552713678800501e-15;                      // 2^-48
         for (int t = 0; t < i; ++t)
           y -= (double)pan_u[t * kT1MaxR + g[x]] * S.dots[2 * t] + (double)pan_w[t * kT1MaxR + g[x]] * S.dots[2 * t + 1];
         p[x] = 2.0 * y;
@@ -1247,7 +1278,7 @@ template <typename T> size_t tb_smem_bytes(int r_max) {
   return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128 + (sizeof(T) == 4 ? 2 * (size_t)kTbNB * kTbPanRows : 0)) * sizeof(T);
 }
 size_t t1_smem_bytes() {
-  return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + (size_t)kT1MaxB * kT1MaxB * kT1Blk);
+  return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + 2 * (size_t)kT1MaxR + (size_t)kT1Warps * 1024);
 }
 size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbBatch * sizeof(float)); }
 size_t vw_smem_bytes(int rp_max) { return (size_t)std::min(rp_max, kVwMaxRp) * (2 * sizeof(double) + kVwWarps * sizeof(float)); }
