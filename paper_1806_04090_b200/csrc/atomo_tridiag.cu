@@ -590,7 +590,8 @@ int sp_tridiag_ctas_of(int rp) { return rp / kTriRows < 1 ? 1 : rp / kTriRows; }
 // about 3000.  Both tridiagonal routes need this (a batch may hold large layers only).  0 if it went through.
 int sp_configure_bisect() {
   const int bytes = (int)(2 * (kMaxShort + 10) * sizeof(double));
-  if (cudaFuncSetAttribute(sp_bisect_kernel<8, 13>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
+  if (cudaFuncSetAttribute(sp_bisect_kernel<1, 41>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sp_bisect_kernel<8, 13>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess ||
       cudaFuncSetAttribute(sp_bisect_kernel<2, 26>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) {
     cudaGetLastError();
     return 1;
@@ -632,7 +633,12 @@ int launch_sp_tridiag(const SpLayer* d_layers, const ClusterCta* d_ctas, int n_c
 void launch_sp_bisect(const SpLayer* d_layers, int n_layers, int r_max, int64_t n_eigenvalues, cudaStream_t st) {
   const int stride = (r_max + 8 + 1) & ~1;
   const size_t smem = 2 * (size_t)stride * sizeof(double);
-  if (n_eigenvalues >= 16384) {
+  if (n_eigenvalues >= 65536) {
+    // enough eigenvalues to fill the fp64 pipes with one lane each: plain bisection gets one bit per Sturm count
+    // (3-section 0.79, 9-section 0.40), 41 rounds for the same final width as the other forms
+    constexpr int per = kBisThreads;
+    sp_bisect_kernel<1, 41><<<dim3((r_max + per - 1) / per, n_layers), kBisThreads, smem, st>>>(d_layers, stride);
+  } else if (n_eigenvalues >= 16384) {
     constexpr int per = kBisThreads / 2;
     sp_bisect_kernel<2, 26><<<dim3((r_max + per - 1) / per, n_layers), kBisThreads, smem, st>>>(d_layers, stride);
   } else {
