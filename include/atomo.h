@@ -317,10 +317,10 @@ int atomo_set_gram_path(atomo_ctx* ctx, int32_t tensor_cores);
  * kept as a fallback and as an independent cross-check of scheme 3.                                              */
 int atomo_set_persistent_eig(atomo_ctx* ctx, int32_t enabled);
 /* CTAs per layer of the blocked tridiagonal reduction that scheme 3 runs for short sides above 512: 0 (default) =
- * chosen per batch (the fewest that hold the layer's rows, doubled while SMs would stay idle), else 1, 2, 4, 8 or 16
- * (raised to the fewest that hold the rows).  With 2 to 16 CTAs a layer runs the cluster kernel, every sum of which has
+ * chosen per batch (the fewest that hold the layer's rows, doubled while SMs would stay idle; never 2 up to a short side
+ * of 1024, where one CTA per layer is faster than a pair), else 1, 2, 4, 8 or 16 (raised to the fewest that hold the rows).  With 2 to 16 CTAs a layer runs the cluster kernel, every sum of which has
  * an order that does not depend on this number: the payload is bit-identical for 2, 4, 8 and 16 (the knob exists for
- * tuning and for checking exactly that).  With 1 CTA per layer (short sides up to 1024; what a batch of 75 layers or
+ * tuning and for checking exactly that).  With 1 CTA per layer (short sides up to 1024; what a batch of 38 layers or
  * more gets) another kernel runs (triangle-only products, panels of 16 columns): same kept atoms, values equal to
  * rounding.                                                                                                    */
 int atomo_set_tridiag_ctas(atomo_ctx* ctx, int32_t ctas_per_layer);

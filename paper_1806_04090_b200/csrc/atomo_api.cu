@@ -773,7 +773,17 @@ static int encode_spectral_impl(atomo_ctx* ctx, const atomo_mat* layers, int32_t
       for (int l : big_layers) { cmin = std::max(cmin, sp_tridiag_big_min_ctas(L[l].r)); rb = std::max(rb, L[l].r); }
       int cc = cmin;
       if (ctx->tri_big_ctas > 0) cc = std::max(cmin, ctx->tri_big_ctas);
-      else while (cc < 16 && (int)big_layers.size() * cc * 2 <= sms) cc *= 2;
+      else {
+        // (clusters sit inside one GPC each: the GPU holds fewer of them than SMs / CTAs, so ask)
+        auto fits = [&](int c2) {
+          const int mc = sp_tridiag_big_max_clusters(c2, rb);
+          return mc > 0 ? (int)big_layers.size() <= mc : (int)big_layers.size() * c2 <= sms;
+        };
+        while (cc < 16 && fits(cc * 2)) cc *= 2;
+        // up to a short side of 1024 one CTA per layer runs the triangle-only kernel, which beats a pair of CTAs on full
+        // rows (40 layers: 25 ms against 36 ms); clusters pay from four CTAs per layer on
+        if (cc == 2 && rb <= 1024) cc = 1;
+      }
       const int e = launch_sp_tridiag_big(d_layers, d_big, (int)big_layers.size(), rb, cc, 0, st);
       if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchKernelEx(blocked tridiagonal reduction)");
       ++n_eig_launch;

@@ -158,6 +158,7 @@ int sp_tridiag_big_panel();
 int sp_tridiag_big_min_ctas(int r);                               // fewest CTAs per layer that hold r rows
 int sp_eigvec_big_slots();                                        // warps per layer of the vector kernel (work vectors)
 int sp_configure_tridiag_big();                                   // 0 if available
+int sp_tridiag_big_max_clusters(int ctas, int r_max);              // co-resident clusters of that many CTAs (0: unknown)
 int sp_configure_bisect();                                        // 0 if the eigenvalue kernel got its shared memory
 int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, int r_max, int ctas, int fp64, cudaStream_t st);  // cudaError_t
 void launch_sp_eigvec_big(const SpLayer* d_layers, const int* d_big, int n_big, int rp_max, cudaStream_t st);

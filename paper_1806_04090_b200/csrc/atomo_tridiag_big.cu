@@ -1307,6 +1307,32 @@ int tb_launch_one(const SpLayer* d_layers, const int* d_big, int n_big, int r_ma
 
 }  // namespace
 
+namespace {
+template <typename T, int C> int tb_max_clusters(int r_max) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(C); cfg.blockDim = dim3(kTbThreads); cfg.dynamicSmemBytes = tb_smem_bytes<T>(r_max);
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = C; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, sp_tridiag_big_kernel<T, C>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n;
+}
+}  // namespace
+
+// clusters of `ctas` CTAs of the fp32 cluster kernel that the GPU runs at the same time (they have to sit inside one
+// GPC each, so this is less than SMs / ctas); 0 if unknown
+int sp_tridiag_big_max_clusters(int ctas, int r_max) {
+  switch (ctas) {
+    case 2: return tb_max_clusters<float, 2>(r_max);
+    case 4: return tb_max_clusters<float, 4>(r_max);
+    case 8: return tb_max_clusters<float, 8>(r_max);
+    case 16: return tb_max_clusters<float, 16>(r_max);
+    default: return 0;
+  }
+}
+
 int sp_tridiag_big_max_r() { return kTbMaxR; }
 int sp_tridiag_big_panel() { return kTbNB; }
 int sp_tridiag_big_min_ctas(int r) { int c = 1; while (c < kTbMaxC && (int64_t)c * kTbThreads < r) c <<= 1; return c; }
