@@ -351,7 +351,7 @@ def roofline_for(run, eig_ms_per_step, eig_launches_per_step, scheme, peaks, fma
         # the blocked reduction dominates whenever it runs (config 3: also one launch of the small-layer kernel in the stage)
         b = tridiag_big_bytes(shapes)
         ach = b / (eig_ms_per_step * 1e-3) / 1e9
-        out.update(bound="hbm", kernel="sp_tridiag_big1_kernel (one CTA per layer)" if max(min(sh) for sh in shapes) <= 1024 and len(shapes) >= 75 else "sp_tridiag_big_kernel (clusters)", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+        out.update(bound="hbm", kernel="sp_tridiag_big1_kernel (one CTA per layer)" if max(min(sh) for sh in shapes) <= 1024 and sum(1 for sh in shapes if min(sh) > 512) >= 38 else "sp_tridiag_big_kernel (clusters)", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
                    frac=ach / peaks["hbm_gbs"], traffic=NCU_TRAFFIC.get(("sp_tridiag_big_kernel", run.name)),
                    peak_source=f"{peaks['source']} copy bandwidth (MEASURED_PEAKS.json)",
                    algorithmic="one triangle of the trailing block per Householder step, 4-byte entries: (2/3) r^3 bytes per layer",
