@@ -31,8 +31,8 @@ L2_BYTES = 126 * 1024 * 1024
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu captures
 # summarised under profiles/ (None: no capture on file for that kernel and workload)
 NCU_TRAFFIC = {("sp_tridiag_cluster_kernel", "c2"): 5638912,
-               # profiles/sp_tridiag_big1_c5.txt: 1.661 TB/s of DRAM traffic over the 31.55 ms of the captured launch
-               ("sp_tridiag_big_kernel", "c5"): 52_400_000_000,
+               # profiles/sp_tridiag_big1_c5.txt: 1.706 TB/s of DRAM traffic over the 29.52 ms of the captured launch
+               ("sp_tridiag_big_kernel", "c5"): 50_400_000_000,
                # profiles/entrywise_c4.txt: the encode kernel (1.92 TB/s over 67.7 us) plus the decode kernel (3.74 TB/s over
                # 24.0 us) of one step at s = 1 %
                ("entrywise", "c4"): 220_000_000}
