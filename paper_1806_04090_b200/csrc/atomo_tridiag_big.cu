@@ -17,11 +17,12 @@
 //                           added in fp64; column updates, norms and all scalars are fp64.  T = double keeps
 //                           everything in fp64.  Every sum has a fixed order that does not depend on C: a row product
 //                           is one warp's, block-wide sums go over the 32-row blocks in ascending order.
-//   sp_eigvec_big_warp_kernel / sp_eigvec_big_kernel (short sides up to 1024 / above)
+//   sp_eigvec_big_cta_kernel / sp_eigvec_big_kernel (short sides up to 1024 / above)
 //                         : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
 //                           route, its work vectors in global memory), back-transformation u = Q z four reflectors at
-//                           a time (fp32): one warp per kept atom up to a short side of 1024, above it the whole CTA
-//                           on up to eight atoms at once (the reflectors are then read once per eight atoms).
+//                           a time (fp32) by a whole CTA: four warps per kept atom up to a short side of 1024, above it
+//                           sixteen warps on up to eight atoms at once (the reflectors are then read once per eight
+//                           atoms).
 //
 // The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
 // Work per layer: the matrix-vector products read sum_c (r - c)^2 ~ r^3 / 3 matrix entries (the bound of this kernel:
@@ -981,124 +982,8 @@ __device__ __forceinline__ void vb_orthogonalise_equal(const SpLayer& L, uint32_
 
 
 namespace {
-constexpr int kVwThreads = 128;              // the warp-per-atom form: short sides up to 1024, many layers
-constexpr int kVwWarps = kVwThreads / 32;
-constexpr int kVwCtas = 4;                   // CTAs per layer: 16 warps, one kept atom each at a time
-constexpr int kVwMaxRp = 1024;
-}  // namespace
-
-// Short sides up to 1024: one warp per kept atom, 16 warps per layer on four small CTAs.  A batch of many such layers
-// (config 5: 96) fills the GPU with independent warps, which hides the latency of the reflector rows better than a
-// CTA-wide exchange per group of reflectors would.
-__global__ void __launch_bounds__(kVwThreads) sp_eigvec_big_warp_kernel(const SpLayer* __restrict__ layers,
-                                                                   const int* __restrict__ big_layers) {
-  const SpLayer& L = layers[big_layers[blockIdx.x]];
-  if (L.rp > kVwMaxRp) return;                                // larger layers: the cooperative kernel
-  extern __shared__ __align__(16) unsigned char vb_smem[];
-  const int r = L.r, rp = L.rp;
-  double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
-  double* s_e = s_d + rp;                                      // [rp]
-  float* s_z = reinterpret_cast<float*>(s_e + rp);             // [warps][rp]
-  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
-  const uint32_t k = L.hdr->k;
-  const float* const gV = L.td_V; const int64_t ldv = L.td_ldv; const double* const gLam = L.lam64;
-  const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
-  const int nref = max(r - 2, 0);
-  for (int i = tid; i < r; i += kVwThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
-  __syncthreads();
-  const int slot = blockIdx.y * kVwWarps + w;                  // 0 .. 15
-  double* wa = L.tb_vecwork + (size_t)slot * 5 * rp;
-  double* wb = wa + rp; double* wc = wb + rp; double* wd = wc + rp; double* zz = wd + rp;
-  float* z = s_z + (size_t)w * rp;
-  for (uint32_t a = slot; a < k; a += kVwCtas * kVwWarps) {
-    const int ei = gPerm[gIdx[a]];                             // index of the atom's eigenvalue (ascending order)
-    double lambda = gLam[ei];
-    int skip = 0;                                              // earlier kept atoms with the same eigenvalue: another twist index each
-    for (uint32_t b = lane; b < a; b += 32) skip += fabs(gLam[gPerm[gIdx[b]]] - lambda) <= kVbSameEig ? 1 : 0;
-    skip = (int)warp_sum((uint32_t)skip);
-    double n2 = 1.0;
-    const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, skip, &n2);
-    double gap = 1.0e300;
-    if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
-    if (ei + 1 < r) gap = fmin(gap, fabs(gLam[ei + 1] - lambda));
-    if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {      // one Rayleigh-quotient step, then the vector again
-      lambda += corr;
-      __syncwarp();
-      twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, 0, &n2);
-    }
-    __syncwarp();
-    const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
-    for (int i = lane; i < r; i += 32) z[i] = (float)(zz[i] * inv);
-    __syncwarp();
-    // u = H_0 H_1 ... H_{r-3} z, H = I - 2 v v^T with unit v: from the last reflector to the first, four at a time.
-    // For a group applied in the order 0, 1, 2, 3:  c_0 = 2 v_0.z,  c_i = 2 (v_i.z - sum_{j<i} c_j v_i.v_j),
-    // z -= sum c_i v_i.  Reflector kk is zero up to index kk, so the sums start at the group's lowest kk + 1.
-    for (int top = nref - 1; top >= 0; top -= 4) {
-      const float* v0 = gV + (int64_t)top * ldv;
-      const float* v1 = gV + (int64_t)max(top - 1, 0) * ldv;
-      const float* v2 = gV + (int64_t)max(top - 2, 0) * ldv;
-      const float* v3 = gV + (int64_t)max(top - 3, 0) * ldv;
-      const float m1 = top - 1 >= 0 ? 1.0f : 0.0f, m2 = top - 2 >= 0 ? 1.0f : 0.0f, m3 = top - 3 >= 0 ? 1.0f : 0.0f;
-      const int h0 = max(top - 3, 0) + 1;
-      float z0 = 0, z1 = 0, z2 = 0, z3 = 0, g10 = 0, g20 = 0, g21 = 0, g30 = 0, g31 = 0, g32 = 0;
-      int h = h0 + lane;
-      for (; h + 96 < r; h += 128) {                                           // sixteen loads in flight
-        float q0[4], q1[4], q2[4], q3[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { q0[j] = v0[h + 32 * j]; q1[j] = v1[h + 32 * j]; q2[j] = v2[h + 32 * j]; q3[j] = v3[h + 32 * j]; }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float zh = z[h + 32 * j];
-          const float r0 = q0[j], r1 = m1 * q1[j], r2 = m2 * q2[j], r3 = m3 * q3[j];
-          z0 = fmaf(r0, zh, z0); z1 = fmaf(r1, zh, z1); z2 = fmaf(r2, zh, z2); z3 = fmaf(r3, zh, z3);
-          g10 = fmaf(r1, r0, g10); g20 = fmaf(r2, r0, g20); g21 = fmaf(r2, r1, g21);
-          g30 = fmaf(r3, r0, g30); g31 = fmaf(r3, r1, g31); g32 = fmaf(r3, r2, g32);
-        }
-      }
-      for (; h < r; h += 32) {
-        const float zh = z[h];
-        const float r0 = v0[h], r1 = m1 * v1[h], r2 = m2 * v2[h], r3 = m3 * v3[h];
-        z0 = fmaf(r0, zh, z0); z1 = fmaf(r1, zh, z1); z2 = fmaf(r2, zh, z2); z3 = fmaf(r3, zh, z3);
-        g10 = fmaf(r1, r0, g10); g20 = fmaf(r2, r0, g20); g21 = fmaf(r2, r1, g21);
-        g30 = fmaf(r3, r0, g30); g31 = fmaf(r3, r1, g31); g32 = fmaf(r3, r2, g32);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        z0 += __shfl_xor_sync(0xffffffffu, z0, o); z1 += __shfl_xor_sync(0xffffffffu, z1, o);
-        z2 += __shfl_xor_sync(0xffffffffu, z2, o); z3 += __shfl_xor_sync(0xffffffffu, z3, o);
-        g10 += __shfl_xor_sync(0xffffffffu, g10, o); g20 += __shfl_xor_sync(0xffffffffu, g20, o);
-        g21 += __shfl_xor_sync(0xffffffffu, g21, o); g30 += __shfl_xor_sync(0xffffffffu, g30, o);
-        g31 += __shfl_xor_sync(0xffffffffu, g31, o); g32 += __shfl_xor_sync(0xffffffffu, g32, o);
-      }
-      const float c0 = 2.0f * z0;
-      const float c1 = 2.0f * (z1 - c0 * g10);
-      const float c2 = 2.0f * (z2 - c0 * g20 - c1 * g21);
-      const float c3 = 2.0f * (z3 - c0 * g30 - c1 * g31 - c2 * g32);
-      h = h0 + lane;
-      for (; h + 96 < r; h += 128) {
-        float q0[4], q1[4], q2[4], q3[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { q0[j] = v0[h + 32 * j]; q1[j] = v1[h + 32 * j]; q2[j] = v2[h + 32 * j]; q3[j] = v3[h + 32 * j]; }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) z[h + 32 * j] -= fmaf(c0, q0[j], fmaf(c1, m1 * q1[j], fmaf(c2, m2 * q2[j], c3 * m3 * q3[j])));
-      }
-      for (; h < r; h += 32)
-        z[h] -= fmaf(c0, v0[h], fmaf(c1, m1 * v1[h], fmaf(c2, m2 * v2[h], c3 * m3 * v3[h])));
-      __syncwarp();
-    }
-    float n2f = 0.0f;
-    for (int i = lane; i < r; i += 32) n2f = fmaf(z[i], z[i], n2f);
-    n2f = warp_sum(n2f);
-    const float invf = n2f > 0.0f ? rsqrtf(n2f) : 0.0f;
-    for (int i = lane; i < r; i += 32) gShort[(int64_t)a * r + i] = z[i] * invf;
-    __syncwarp();
-  }
-  vb_orthogonalise_equal(L, k, kVwCtas);
-}
-
-namespace {
-// the columns tid, tid + 512, ... of the four reflector rows top, top - 1, top - 2, top - 3 (rows below 0: zeros)
-template <int COLS>
+// the columns tid, tid + THREADS, ... of the four reflector rows top, top - 1, top - 2, top - 3 (rows below 0: zeros)
+template <int THREADS, int COLS>
 __device__ __forceinline__ void vb_load_rows(const float* __restrict__ gV, int64_t ldv, int r, int top, float (&q)[4][COLS]) {
   const int tid = threadIdx.x;
   const float* v0 = gV + (int64_t)top * ldv;
@@ -1109,7 +994,7 @@ __device__ __forceinline__ void vb_load_rows(const float* __restrict__ gV, int64
   const int h0 = max(top - 3, 0) + 1;                          // reflector kk is zero up to index kk
 #pragma unroll
   for (int m = 0; m < COLS; ++m) {
-    const int h = tid + m * kVbThreads;
+    const int h = tid + m * THREADS;
     const bool in = h >= h0 && h < r;
     q[0][m] = in ? __ldcg(v0 + h) : 0.0f;
     q[1][m] = in && e1 ? __ldcg(v1 + h) : 0.0f;
@@ -1120,25 +1005,26 @@ __device__ __forceinline__ void vb_load_rows(const float* __restrict__ gV, int64
 
 // z_b <- H_0 ... H_{nref-1} z_b for the nb vectors in s_z, the whole CTA.  PREFETCH: the next group's rows are on their
 // way while this group's sums are added up (needs twice the registers for the rows: short sides up to 2048).
-template <int COLS, bool PREFETCH>
+template <int THREADS, int BATCH, int COLS, bool PREFETCH>
 __device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV, int64_t ldv, int r, int rp, int nref, int nb,
-                                                    float* s_z, float (*s_part)[kVbSums], float* s_tot) {
+                                                    float* s_z, float (*s_part)[4 * BATCH + 6], float* s_tot) {
+  constexpr int kSums = 4 * BATCH + 6, kWarps = THREADS / 32;
   const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
   float q[4][COLS], qn[4][PREFETCH ? COLS : 1];
-  if (PREFETCH && nref > 0) vb_load_rows<COLS>(gV, ldv, r, nref - 1, q);
+  if (PREFETCH && nref > 0) vb_load_rows<THREADS, COLS>(gV, ldv, r, nref - 1, q);
   for (int top = nref - 1; top >= 0; top -= 4) {
-    if (!PREFETCH) vb_load_rows<COLS>(gV, ldv, r, top, q);
-    float acc[kVbSums];
+    if (!PREFETCH) vb_load_rows<THREADS, COLS>(gV, ldv, r, top, q);
+    float acc[kSums];
 #pragma unroll
-    for (int x = 0; x < kVbSums; ++x) acc[x] = 0.0f;
+    for (int x = 0; x < kSums; ++x) acc[x] = 0.0f;
 #pragma unroll
     for (int m = 0; m < COLS; ++m) {
-      const int h = tid + m * kVbThreads;
+      const int h = tid + m * THREADS;
       if (h < r) {
         acc[0] = fmaf(q[1][m], q[0][m], acc[0]); acc[1] = fmaf(q[2][m], q[0][m], acc[1]); acc[2] = fmaf(q[2][m], q[1][m], acc[2]);
         acc[3] = fmaf(q[3][m], q[0][m], acc[3]); acc[4] = fmaf(q[3][m], q[1][m], acc[4]); acc[5] = fmaf(q[3][m], q[2][m], acc[5]);
 #pragma unroll
-        for (int b = 0; b < kVbBatch; ++b) {
+        for (int b = 0; b < BATCH; ++b) {
           if (b < nb) {
             const float zh = s_z[(size_t)b * rp + h];
             acc[6 + 4 * b + 0] = fmaf(q[0][m], zh, acc[6 + 4 * b + 0]); acc[6 + 4 * b + 1] = fmaf(q[1][m], zh, acc[6 + 4 * b + 1]);
@@ -1147,10 +1033,10 @@ __device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV
         }
       }
     }
-    if (PREFETCH && top - 4 >= 0) vb_load_rows<COLS>(gV, ldv, r, top - 4, reinterpret_cast<float (&)[4][COLS]>(qn));
+    if (PREFETCH && top - 4 >= 0) vb_load_rows<THREADS, COLS>(gV, ldv, r, top - 4, reinterpret_cast<float (&)[4][COLS]>(qn));
     const int n_sums = 6 + 4 * nb;
 #pragma unroll
-    for (int x = 0; x < kVbSums; ++x) {
+    for (int x = 0; x < kSums; ++x) {
       if (x < n_sums) {
         const float t = warp_sum(acc[x]);
         if (lane == 0) s_part[w][x] = t;
@@ -1160,13 +1046,13 @@ __device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV
     if (tid < n_sums) {
       float t = 0.0f;
 #pragma unroll
-      for (int ww = 0; ww < kVbWarps; ++ww) t += s_part[ww][tid];
+      for (int ww = 0; ww < kWarps; ++ww) t += s_part[ww][tid];
       s_tot[tid] = t;
     }
     __syncthreads();
     const float g10 = s_tot[0], g20 = s_tot[1], g21 = s_tot[2], g30 = s_tot[3], g31 = s_tot[4], g32 = s_tot[5];
 #pragma unroll
-    for (int b = 0; b < kVbBatch; ++b) {
+    for (int b = 0; b < BATCH; ++b) {
       if (b < nb) {
         const float c0 = 2.0f * s_tot[6 + 4 * b];
         const float c1 = 2.0f * (s_tot[6 + 4 * b + 1] - c0 * g10);
@@ -1174,7 +1060,7 @@ __device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV
         const float c3 = 2.0f * (s_tot[6 + 4 * b + 3] - c0 * g30 - c1 * g31 - c2 * g32);
 #pragma unroll
         for (int m = 0; m < COLS; ++m) {
-          const int h = tid + m * kVbThreads;
+          const int h = tid + m * THREADS;
           if (h < r) s_z[(size_t)b * rp + h] -= fmaf(c0, q[0][m], fmaf(c1, q[1][m], fmaf(c2, q[2][m], c3 * q[3][m])));
         }
       }
@@ -1191,10 +1077,83 @@ __device__ __forceinline__ void vb_apply_reflectors(const float* __restrict__ gV
 }
 }  // namespace
 
+// Short sides up to 1024, any number of layers: a small CTA (four warps) per kept atom at a time, sixteen CTAs per
+// layer.  One warp forms the atom's eigenvector of T; the four warps then apply the reflectors together (a thread owns
+// eight columns of every reflector row: the 16 loads of a group are in flight at once, the next group's are issued
+// before this group's sums are exchanged).  With one warp per atom the same rows took four dependent batches of loads.
+namespace {
+constexpr int kVcThreads = 128;
+constexpr int kVcWarps = kVcThreads / 32;
+constexpr int kVcCtas = 16;                  // CTAs per layer = work-vector sets per layer
+constexpr int kVcMaxRp = 1024;
+}  // namespace
+
+__global__ void __launch_bounds__(kVcThreads) sp_eigvec_big_cta_kernel(const SpLayer* __restrict__ layers,
+                                                                       const int* __restrict__ big_layers) {
+  const SpLayer& L = layers[big_layers[blockIdx.x]];
+  if (L.rp > kVcMaxRp) return;                                 // larger layers: sp_eigvec_big_kernel
+  extern __shared__ __align__(16) unsigned char vb_smem[];
+  const int r = L.r, rp = L.rp;
+  double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
+  double* s_e = s_d + rp;                                      // [rp]
+  float* s_z = reinterpret_cast<float*>(s_e + rp);             // [rp]
+  __shared__ float s_part[kVcWarps][10];
+  __shared__ float s_tot[10];
+  const int tid = threadIdx.x, lane = tid % 32, w = tid / 32;
+  const uint32_t k = L.hdr->k;
+  const float* const gV = L.td_V; const int64_t ldv = L.td_ldv; const double* const gLam = L.lam64;
+  const int* const gPerm = L.perm; const uint32_t* const gIdx = L.idx; float* const gShort = L.shortv;
+  const int nref = max(r - 2, 0);
+  const int slot = blockIdx.y;                                 // 0 .. 15
+  if ((uint32_t)slot < k) {
+    for (int i = tid; i < r; i += kVcThreads) { s_d[i] = L.td_d[i]; s_e[i] = i + 1 < r ? L.td_e[i] : 0.0; }
+    __syncthreads();
+    double* wa = L.tb_vecwork + (size_t)slot * 5 * rp;
+    double* wb = wa + rp; double* wc = wb + rp; double* wd = wc + rp; double* zz = wd + rp;
+    for (uint32_t a = slot; a < k; a += kVcCtas) {
+      if (w == 0) {
+        const int ei = gPerm[gIdx[a]];                         // index of the atom's eigenvalue (ascending order)
+        double lambda = gLam[ei];
+        int skip = 0;                                          // earlier kept atoms with the same eigenvalue: another twist index each
+        for (uint32_t b2 = lane; b2 < a; b2 += 32) skip += fabs(gLam[gPerm[gIdx[b2]]] - lambda) <= kVbSameEig ? 1 : 0;
+        skip = (int)warp_sum((uint32_t)skip);
+        double n2 = 1.0;
+        const double corr = twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, skip, &n2);
+        double gap = 1.0e300;
+        if (ei > 0) gap = fmin(gap, fabs(lambda - gLam[ei - 1]));
+        if (ei + 1 < r) gap = fmin(gap, fabs(gLam[ei + 1] - lambda));
+        if (finite64(corr) && skip == 0 && !(fabs(corr) <= 1.0e-9 * gap)) {  // one Rayleigh-quotient step, then the vector again
+          lambda += corr;
+          __syncwarp();
+          twisted_vector(s_d, s_e, r, lambda, wa, wb, wc, wd, zz, lane, 0, &n2);
+        }
+        __syncwarp();
+        const double inv = n2 > 0.0 ? rsqrt(n2) : 0.0;
+        for (int i = lane; i < r; i += 32) s_z[i] = (float)(zz[i] * inv);
+      }
+      __syncthreads();
+      vb_apply_reflectors<kVcThreads, 1, kVcMaxRp / kVcThreads, true>(gV, ldv, r, rp, nref, 1, s_z, s_part, s_tot);
+      float n2f = 0.0f;
+      for (int i = tid; i < r; i += kVcThreads) n2f = fmaf(s_z[i], s_z[i], n2f);
+      n2f = warp_sum(n2f);
+      __syncthreads();
+      if (lane == 0) s_part[w][0] = n2f;
+      __syncthreads();
+      float tot = 0.0f;
+#pragma unroll
+      for (int ww = 0; ww < kVcWarps; ++ww) tot += s_part[ww][0];
+      const float invf = tot > 0.0f ? rsqrtf(tot) : 0.0f;
+      for (int i = tid; i < r; i += kVcThreads) gShort[(int64_t)a * r + i] = s_z[i] * invf;
+      __syncthreads();
+    }
+  }
+  vb_orthogonalise_equal(L, k, kVcCtas);
+}
+
 __global__ void __launch_bounds__(kVbThreads, 1) sp_eigvec_big_kernel(const SpLayer* __restrict__ layers,
                                                                       const int* __restrict__ big_layers) {
   const SpLayer& L = layers[big_layers[blockIdx.x]];
-  if (L.rp <= kVwMaxRp) return;                                // smaller layers: the warp-per-atom kernel
+  if (L.rp <= 1024) return;                                    // smaller layers: sp_eigvec_big_cta_kernel
   extern __shared__ __align__(16) unsigned char vb_smem[];
   const int r = L.r, rp = L.rp;
   double* s_d = reinterpret_cast<double*>(vb_smem);            // [rp]
@@ -1247,8 +1206,8 @@ __global__ void __launch_bounds__(kVbThreads, 1) sp_eigvec_big_kernel(const SpLa
       for (int i = tid; i < r; i += kVbThreads) s_z[(size_t)b * rp + i] = src[i];
     }
     __syncthreads();
-    if (rp <= 4 * kVbThreads) vb_apply_reflectors<4, true>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
-    else vb_apply_reflectors<8, false>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
+    if (rp <= 4 * kVbThreads) vb_apply_reflectors<kVbThreads, kVbBatch, 4, true>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
+    else vb_apply_reflectors<kVbThreads, kVbBatch, 8, false>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
     // normalise and file
     for (int b = 0; b < nb; ++b) {
       float n2f = 0.0f;
@@ -1281,7 +1240,7 @@ size_t t1_smem_bytes() {
   return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + 2 * (size_t)kT1MaxR + (size_t)kT1Warps * 1024);
 }
 size_t vb_smem_bytes(int rp_max) { return (size_t)rp_max * (2 * sizeof(double) + kVbBatch * sizeof(float)); }
-size_t vw_smem_bytes(int rp_max) { return (size_t)std::min(rp_max, kVwMaxRp) * (2 * sizeof(double) + kVwWarps * sizeof(float)); }
+size_t vc_smem_bytes(int rp_max) { return (size_t)std::min(rp_max, kVcMaxRp) * (2 * sizeof(double) + sizeof(float)); }
 
 template <typename T, int C> int tb_configure_one() {
   auto* fn = sp_tridiag_big_kernel<T, C>;
@@ -1347,7 +1306,6 @@ int sp_configure_tridiag_big() {
          tb_configure_one<double, 8>() | tb_configure_one<double, 16>();
   bad |= cudaFuncSetAttribute(sp_tridiag_big1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)t1_smem_bytes()) != cudaSuccess;
   bad |= cudaFuncSetAttribute(sp_eigvec_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)vb_smem_bytes(kTbMaxR)) != cudaSuccess;
-  bad |= cudaFuncSetAttribute(sp_eigvec_big_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)kTbMaxR * (2 * sizeof(double) + kVwWarps * sizeof(float)))) != cudaSuccess;
   if (bad) cudaGetLastError();
   return bad;
 }
@@ -1367,10 +1325,10 @@ int launch_sp_tridiag_big(const SpLayer* d_layers, const int* d_big, int n_big, 
 
 void launch_sp_eigvec_big(const SpLayer* d_layers, const int* d_big, int n_big, int rp_max, cudaStream_t st) {
   if (n_big <= 0) return;
-  // layers up to a short side of 1024: one warp per kept atom (the other kernel's CTAs leave such layers at once, and
-  // the other way round)
-  sp_eigvec_big_warp_kernel<<<dim3(n_big, kVwCtas), kVwThreads, vw_smem_bytes(rp_max), st>>>(d_layers, d_big);
-  if (rp_max <= kVwMaxRp) return;
+  // layers up to a short side of 1024: a four-warp CTA per kept atom (the other kernel's CTAs leave such layers at once,
+  // and the other way round)
+  sp_eigvec_big_cta_kernel<<<dim3(n_big, kVcCtas), kVcThreads, vc_smem_bytes(rp_max), st>>>(d_layers, d_big);
+  if (rp_max <= kVcMaxRp) return;
   // larger layers: CTAs per layer (1, 2 or 4; the kept atoms are dealt to them), as many as keep the launch within one wave
   static int sms = 0;
   if (sms == 0) { int dev = 0; if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) sms = 1; }
