@@ -21,7 +21,7 @@
 //                         : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
 //                           route, its work vectors in global memory), back-transformation u = Q z four reflectors at
 //                           a time (fp32) by a whole CTA: four warps per kept atom up to a short side of 1024, above it
-//                           sixteen warps on up to eight atoms at once (the reflectors are then read once per eight
+//                           sixteen warps on up to four atoms at once (the reflectors are then read once per four
 //                           atoms).
 //
 // The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
@@ -920,19 +920,19 @@ __global__ void __launch_bounds__(kT1Threads, 1) sp_tridiag_big1_kernel(const Sp
 // ---- vectors of the kept atoms ------------------------------------------------------------------------------------
 // Two phases per CTA.  (A) one warp per kept atom: the eigenvector of T by the twisted factorisation of the small
 // route (work vectors in global memory), normalised, filed in the payload's slot of the atom.  (B) the whole CTA
-// applies the reflectors to up to eight of its atoms at once, u = H_0 H_1 ... H_{r-3} z with H = I - 2 v v^T, from the
+// applies the reflectors to up to four of its atoms at once, u = H_0 H_1 ... H_{r-3} z with H = I - 2 v v^T, from the
 // last reflector to the first, four at a time: a thread owns the columns tid, tid + 512, ... of the four reflector rows
 // (read once per group, kept in registers between the dot products and the update) and of every z (in shared memory;
 // no other thread touches them), so the only exchange per group is the block-wide sum of the products: v_i.z for
 // every atom and the six v_i.v_j.  For a group applied in the order 0, 1, 2, 3:  c_0 = 2 v_0.z,
-// c_i = 2 (v_i.z - sum_{j<i} c_j v_i.v_j),  z -= sum c_i v_i.  The matrix of reflectors is read once per eight atoms
+// c_i = 2 (v_i.z - sum_{j<i} c_j v_i.v_j),  z -= sum c_i v_i.  The matrix of reflectors is read once per four atoms
 // instead of once per atom, by 512 threads instead of 32.
 namespace {
 constexpr int kVbThreads = 512;
 constexpr int kVbWarps = kVbThreads / 32;
 constexpr int kVbSlots = 16;                 // work-vector sets per layer (phase A: 16 atoms at a time over the layer's CTAs)
 constexpr int kVbMaxCtas = 4;                // CTAs per layer (the kept atoms are dealt to them)
-constexpr int kVbBatch = 8;                  // atoms per pass over the reflectors
+constexpr int kVbBatch = 4;                  // atoms per pass over the reflectors
 constexpr int kVbCols = kTbMaxR / kVbThreads;   // columns per thread and reflector row (8)
 constexpr int kVbSums = 4 * kVbBatch + 6;    // products summed per group
 constexpr double kVbSameEig = 1.0e-9;        // as on the small route
@@ -1207,7 +1207,7 @@ __global__ void __launch_bounds__(kVbThreads, 1) sp_eigvec_big_kernel(const SpLa
     }
     __syncthreads();
     if (rp <= 4 * kVbThreads) vb_apply_reflectors<kVbThreads, kVbBatch, 4, true>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
-    else vb_apply_reflectors<kVbThreads, kVbBatch, 8, false>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
+    else vb_apply_reflectors<kVbThreads, kVbBatch, 8, true>(gV, ldv, r, rp, nref, nb, s_z, s_part, s_tot);
     // normalise and file
     for (int b = 0; b < nb; ++b) {
       float n2f = 0.0f;
