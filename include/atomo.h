@@ -184,9 +184,14 @@ int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap);
 /* Launch form of the context's later atomo_encode_entrywise calls.  two_kernels = 0 (default): a vector whose tiles
  * fit one wave of resident CTAs (up to about 48 million elements on a B200) is encoded by ONE cooperative kernel -- a CTA
  * computes its part of sum |g| and max |g| (Algorithm 1's inputs), all CTAs meet at a grid barrier, and the same CTA
- * then samples and packs the part it has just read, which is still in the L2 cache on its side of the chip; longer
- * vectors take the two-kernel form.  two_kernels = 1: always a solve kernel followed by a sample / pack kernel whose
- * chunks are handed out by ticket.  Payloads, masks and decoded gradients are bit-identical in both forms.     */
+ * then samples and packs its part.  The Philox word of an atom depends on its index alone, so the first pass already
+ * draws the words and lists the atoms that an estimate of sum |g| (with a factor of two to spare) cannot rule out; where
+ * the true sum confirms the estimate and no atom has p = 1, the exact keep decision (the same integer comparison) is
+ * taken on the list and the vector is read once.  Otherwise a CTA reads its part a second time (from the L2 cache).
+ * Longer vectors take the two-kernel form.  two_kernels = 1: always a solve kernel followed by a sample / pack kernel
+ * whose chunks are handed out by ticket.  two_kernels = 2: the one-kernel form without the list (every part read
+ * twice).  Payloads, masks and decoded gradients are bit-identical in all forms.  Other values:
+ * ATOMO_ERR_INVALID_ARG.     */
 int atomo_set_entrywise_launch(atomo_ctx* ctx, int32_t two_kernels);
 
 /* --- l_q budgets (Section 4) ------------------------------------------------------------------

@@ -329,12 +329,13 @@ class Atomo:
         s = stream if stream is not None else torch.cuda.current_stream()
         return ctypes.c_void_p(s.cuda_stream)
 
-    def _make_debug(self, n_atoms: Sequence[int], spectral: bool, want_short: bool, dev) -> Debug:
+    def _make_debug(self, n_atoms: Sequence[int], spectral: bool, want_short: bool, dev, want_prob: bool = True) -> Debug:
         a_off = np.concatenate([[0], np.cumsum(n_atoms)]).astype(np.int64)
         w_off = np.concatenate([[0], np.cumsum([(n + 31) // 32 for n in n_atoms])]).astype(np.int64)
         sq_off = np.concatenate([[0], np.cumsum([n * n for n in n_atoms])]).astype(np.int64)
         d = Debug(atom_offsets=a_off.tolist(), word_offsets=w_off.tolist(), sq_offsets=sq_off.tolist())
-        d.prob = torch.zeros(int(a_off[-1]), dtype=torch.float32, device=dev)
+        if want_prob:
+            d.prob = torch.zeros(int(a_off[-1]), dtype=torch.float32, device=dev)
         d.mask_words = torch.zeros(int(w_off[-1]), dtype=torch.int32, device=dev)
         if spectral:
             d.sigma = torch.zeros(int(a_off[-1]), dtype=torch.float32, device=dev)
@@ -412,9 +413,11 @@ class Atomo:
 
     def atomo_encode_entrywise(self, vecs: Sequence[torch.Tensor], s: float, seed: int, step: int = 0,
                                k_cap: Optional[int] = None, payload: Optional[torch.Tensor] = None,
-                               debug: bool = False, stream: Optional[torch.cuda.Stream] = None):
+                               debug=False, stream: Optional[torch.cuda.Stream] = None):
         """Entry-wise ATOMO over a batch of flat fp32 CUDA tensors.  Returns (Payload, Debug | None).
-        The payload format is the one last chosen with set_entrywise_format (explicit by default)."""
+        The payload format is the one last chosen with set_entrywise_format (explicit by default).
+        debug: True = probabilities and mask words, "mask" = the mask words alone (asking for the probabilities makes
+        the one-kernel form read every vector twice)."""
         n = len(vecs)
         arr = (_Vec * n)()
         lengths = []
@@ -434,7 +437,7 @@ class Atomo:
         dev = vecs[0].device
         if payload is None:
             payload = torch.empty(nbytes, dtype=torch.uint8, device=dev)
-        dbg = self._make_debug(lengths, False, False, dev) if debug else None
+        dbg = self._make_debug(lengths, False, False, dev, want_prob=(debug != "mask")) if debug else None
         ds = self._debug_struct(dbg)
         rc = self.lib.atomo_encode_entrywise(self._h, arr, n, float(s), int(seed), int(step), int(k_cap),
                                              ctypes.c_void_p(payload.data_ptr()), payload.numel(),
@@ -541,10 +544,11 @@ class Atomo:
         self._check(self.lib.atomo_set_entrywise_format(self._h, int(fmt), int(sat_cap)), "atomo_set_entrywise_format")
         self._ew_format, self._ew_sat_cap = int(fmt), (int(sat_cap) if int(fmt) == EW_COMPACT else 0)
 
-    def set_entrywise_launch(self, two_kernels: bool):
-        """False (default): one cooperative kernel per vector that fits one wave of resident CTAs; True: always the
-        solve kernel followed by the sample / pack kernel.  Same payloads either way."""
-        self._check(self.lib.atomo_set_entrywise_launch(self._h, 1 if two_kernels else 0), "atomo_set_entrywise_launch")
+    def set_entrywise_launch(self, two_kernels):
+        """0 / False (default): one cooperative kernel per vector that fits one wave of resident CTAs, the keep decisions
+        taken on the candidate list of its first pass where that holds every kept atom; 1 / True: always the solve kernel
+        followed by the sample / pack kernel; 2: the one-kernel form without the list.  Same payloads in every form."""
+        self._check(self.lib.atomo_set_entrywise_launch(self._h, int(two_kernels)), "atomo_set_entrywise_launch")
 
     def table_uploads(self):
         """(calls that uploaded their descriptor tables, calls that found them on the device) since the context was made."""

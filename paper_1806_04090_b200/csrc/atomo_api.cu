@@ -927,14 +927,25 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       EwVec& v = V[l];
       v.g = vecs[l].data; v.n = vecs[l].n; v.layer = (uint32_t)l; v.k_cap = lay[l].kc;
       v.n_tiles = (v.n + tile - 1) / tile;
-      const int fused_ctas = ctx->ew_launch == 0 ? ew_encode_ctas(v.n_tiles, compact) : 0;
+      int fused_ctas = 0;
+      v.candidates = 0;
+      if (ctx->ew_launch != 1) {
+        // the one-kernel form, with the candidate list where the caller does not ask for the probabilities and the
+        // budget is small enough for the list to pay
+        const bool want_list = ctx->ew_launch == 0 && !(dbg && dbg->prob);
+        const int with_list = want_list ? ew_encode_ctas(v.n_tiles, compact, true) : 0;
+        if (with_list > 0 && ew_list_pays(v.n, v.n_tiles, with_list, s)) { fused_ctas = with_list; v.candidates = 1; }
+        else fused_ctas = ew_encode_ctas(v.n_tiles, compact, false);
+      }
       fused[l] = fused_ctas > 0;
       v.n_ctas = fused[l] ? fused_ctas : ew_sample_pack_ctas(v.n_tiles, compact);
       v.compact = compact ? 1 : 0; v.sat_cap = lay[l].sc;
       v.ent = reinterpret_cast<uint16_t*>(pay + lay[l].off_idx);
       v.sat_idx = reinterpret_cast<uint32_t*>(pay + lay[l].off_sat);
       v.sat_val = reinterpret_cast<float*>(pay + lay[l].off_val);
-      v.n_words = (v.n + 31) / 32;
+      const int64_t n_words = (v.n + 31) / 32;
+      const bool want_mask = dbg && dbg->mask_words;           // the mask words leave the kernel only when asked for
+      v.n_words = want_mask ? n_words : 0;
       const int64_t want_chunks = std::min<int64_t>(max_blocks, (v.n + 4095) / 4096);
       v.chunk = (int64_t)align_up((uint64_t)((v.n + want_chunks - 1) / want_chunks), 4);
       v.n_chunks = (int)((v.n + v.chunk - 1) / v.chunk);
@@ -944,10 +955,9 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
       v.tile_table = reinterpret_cast<uint32_t*>(pay + lay[l].off_tiles);
       v.partials = A.take<EwPartial>((size_t)3 * std::max(v.n_chunks, v.n_ctas));
       v.state = A.take<EwState>(1);
-      uint32_t* mask_ws = A.take<uint32_t>(v.n_words);
-      v.mask_words = (dbg && dbg->mask_words) ? dbg->mask_words + dbg_words : mask_ws;
+      v.mask_words = want_mask ? dbg->mask_words + dbg_words : nullptr;
       v.prob_out = (dbg && dbg->prob) ? dbg->prob + dbg_atoms : nullptr;
-      dbg_atoms += v.n; dbg_words += v.n_words;
+      dbg_atoms += v.n; dbg_words += n_words;
     }
     // zero-filled per call: look-back status words and tile tickets of all vectors, one contiguous region
     uint8_t* zb = reinterpret_cast<uint8_t*>(A.take<uint32_t>(0));
@@ -997,6 +1007,15 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   for (int l = 0; l < n_vecs; ++l) {
     if (!fused[l]) { launch_ew_sample_pack(V[l], key, ks, st); continue; }
     const int e = launch_ew_encode(V[l], s, key, ks, st);
+    if (e == (int)cudaErrorCooperativeLaunchTooLarge) {
+      // fewer CTAs fit the GPU at once than the occupancy query promised: the two-kernel form takes the same chunks
+      cudaGetLastError();
+      const int e2 = launch_ew_solve(V[l], s, st);
+      if (e2 != 0) return fail_cuda(ctx, (cudaError_t)e2, "cudaLaunchCooperativeKernel(ew_solve)");
+      launch_ew_sample_pack(V[l], key, ks, st);
+      n_one += 2;
+      continue;
+    }
     if (e != 0) return fail_cuda(ctx, (cudaError_t)e, "cudaLaunchCooperativeKernel(ew_encode)");
     ++n_one;
   }
@@ -1007,7 +1026,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
 
 // ==================================================================================================
 int atomo_set_entrywise_launch(atomo_ctx* ctx, int32_t two_kernels) {
-  if (!ctx || (two_kernels != 0 && two_kernels != 1)) return ATOMO_ERR_INVALID_ARG;
+  if (!ctx || two_kernels < 0 || two_kernels > 2) return ATOMO_ERR_INVALID_ARG;
   ctx->ew_launch = two_kernels;
   return ATOMO_OK;
 }

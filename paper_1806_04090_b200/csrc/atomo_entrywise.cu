@@ -39,7 +39,11 @@ constexpr int kEwTile = 4096;                 // elements per tile of the sample
 #ifndef EW_MIN_BLOCKS
 #define EW_MIN_BLOCKS 5
 #endif
-constexpr int kEwMinBlocks = EW_MIN_BLOCKS;   // resident CTAs per SM the sample / pack kernels are compiled for
+constexpr int kEwMinBlocks = EW_MIN_BLOCKS;   // resident CTAs per SM the sample / pack kernel is compiled for
+#ifndef EW_ENCODE_BLOCKS
+#define EW_ENCODE_BLOCKS 4
+#endif
+constexpr int kEwEncodeBlocks = EW_ENCODE_BLOCKS;   // ... and the one-kernel form (64 registers: two tiles' loads per thread)
 
 __device__ __forceinline__ float4 load4(const float* __restrict__ g, int64_t i, int64_t n, bool aligned) {
   if (aligned && i + 3 < n) return __ldg(reinterpret_cast<const float4*>(g + i));
@@ -102,19 +106,160 @@ __device__ __forceinline__ EwAcc ew_block_reduce(EwAcc a, double* s_sum, float* 
   return r;
 }
 
+// ---- the first pass of the one-kernel form, with a list of candidates --------------------------------------------
+// The keep decision of an atom needs ||g||_1, which only the end of the first pass knows; but the Philox word of an
+// atom depends on its index alone.  So the first pass already draws the words and keeps a list of the few atoms that
+// can still be kept: an atom is kept (Eq. 2 with p < 1) iff word < floor(|g| scale 2^32), and the pass tests
+// word <= |g| M with M = 1.25 scale_est 2^32, where scale_est comes from the sum over the chunk's first tile, scaled to
+// the vector's length.  A thread keeps its candidates (index, value) in slots of its own, so the list needs neither
+// atomics nor votes.  After the grid barrier the true scale is known.  If M >= scale 2^32 (1 + 2^-22) (the slack
+// covers the roundings of both products), the vector is s-balanced (no atom with p = 1) and no thread ran out of
+// slots, the list holds every kept atom of the chunk and the exact decision is taken on its entries alone (their
+// words are drawn again): the chunk is read once.  Otherwise the CTA reads its chunk a second time as the two-kernel form does.  Either way
+// the decision is the same integer comparison on the same operands, so the payload does not depend on which way a
+// chunk went.  The sums are formed exactly as in ew_chunk_pass (same terms per thread, same order).
+constexpr int kEwCandPerThread = 16;             // list entries per thread; 1.25 s (atoms per thread) / n are expected
+constexpr int kEwCandSlots = (kEwCandPerThread + 1) * kEwThreads;   // one more row takes what does not fit (never read)
+struct EwCands {
+  uint32_t* idx;      // [kEwCandPerThread + 1][kEwThreads] atom index inside the chunk, then (same layout) its gradient entry
+  uint32_t* stop;     // set by the first thread that runs out of slots: the CTA stops listing
+  float m32;          // the multiplier M the list was made with (0: no list)
+  uint32_t addr;      // shared-memory address of this thread's next slot: rows of kEwThreads 4-byte entries
+  uint32_t addr0;     // ... of its first slot
+};
+__device__ __forceinline__ uint32_t ew_cand_count(const EwCands& C) { return (C.addr - C.addr0) / (4u * kEwThreads); }
+
+// One tile of the pass: 16 atoms per thread (float4 number tid + 256 u of the tile, u = 0 .. 3).  local0: index of
+// x[0].x inside the chunk; blk0: its Philox block (atom index / 4); left: elements of the chunk from x[0].x on
+// (FULL: the whole tile lies inside the chunk).  amax ignores NaN (and the sum keeps it), so "some entry is NaN" is
+// "the sum is NaN" and "some entry is infinite" is "amax is infinite": no test per entry.
+template <bool FULL>
+__device__ __forceinline__ void ew_cand_tile(const float4 (&x)[4], const uint32_t local0, const uint32_t blk0, const int64_t left,
+                                             const uint32_t layer, const PhiloxKey key, const uint32_t kind_step,
+                                             const bool listing, float& fsum, float& amax, EwCands& C) {
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const float a[4] = {fabsf(x[u].x), fabsf(x[u].y), fabsf(x[u].z), fabsf(x[u].w)};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      fsum += a[j];
+      amax = fmaxf(amax, a[j]);
+    }
+  }
+  if (!listing) return;
+  const float m32 = C.m32;
+  const uint32_t spill = C.addr0 + (uint32_t)(kEwCandPerThread * kEwThreads * 4);   // this thread's slot in the extra row
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    if (!FULL && (int64_t)u * kEwThreads * 4 >= left) continue;
+    const uint4 wd = philox4x32_10(make_uint4(blk0 + (uint32_t)(u * kEwThreads), 0u, layer, kind_step), key);
+    const float gg[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+    const uint32_t ww[4] = {wd.x, wd.y, wd.z, wd.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      // candidate: two predicated stores (index, value) to the thread's next slot and the slot moves on; no branch
+      const uint32_t o = min(C.addr, spill);
+      const uint32_t li = local0 + (uint32_t)(u * kEwThreads * 4 + j);
+      asm volatile(
+          "{\n\t.reg .pred p;\n\t.reg .f32 t, wf;\n\t"
+          "cvt.rz.f32.u32 wf, %3;\n\t"
+          "abs.f32 t, %2;\n\t"
+          "mul.f32 t, t, %4;\n\t"
+          "setp.ge.f32 p, t, wf;\n\t"
+          "@p st.shared.u32 [%1], %5;\n\t"
+          "@p st.shared.f32 [%1 + %6], %2;\n\t"
+          "@p add.u32 %0, %0, %7;\n\t}"
+          : "+r"(C.addr)
+          : "r"(o), "f"(gg[j]), "r"(ww[j]), "f"(m32), "r"(li), "n"(kEwCandSlots * 4), "n"(kEwThreads * 4)
+          : "memory");
+    }
+  }
+  if (C.addr > spill) *(volatile uint32_t*)C.stop = 1u;    // more candidates than slots: this chunk will be read twice
+}
+
+__device__ __forceinline__ EwAcc ew_chunk_pass_cand(const EwVec& v, const PhiloxKey key, const uint32_t kind_step, const double s,
+                                                    const int64_t beg, const int64_t end, const int n_my, EwCands& C,
+                                                    float* s_red) {
+  const bool aligned = (reinterpret_cast<uintptr_t>(v.g) & 15u) == 0;
+  const int tid = threadIdx.x, lane = tid % kWarp, w = tid / kWarp;
+  constexpr int kU = 4;
+  double sum = 0.0;
+  float amax = 0.0f;
+  C.m32 = 0.0f; C.addr = C.addr0;
+  // tiles that lie inside the chunk and can be read with 16-byte loads; the next tile's loads are issued before this
+  // tile's words are drawn, so a warp always has requests in flight
+  const int n_full = aligned ? (int)((end - beg) / kEwTile) : 0;
+  auto load_tile = [&](int tl, float4 (&x)[kU]) {
+    const int64_t base = beg + (int64_t)tl * kEwTile + (int64_t)tid * 4;
+    if (tl < n_full) {
+#pragma unroll
+      for (int u = 0; u < kU; ++u) x[u] = __ldg(reinterpret_cast<const float4*>(v.g + base) + u * kEwThreads);
+    } else {
+#pragma unroll
+      for (int u = 0; u < kU; ++u) {
+        const int64_t i = base + (int64_t)u * kEwThreads * 4;
+        x[u] = i < end ? load4(v.g, i, end, aligned) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+  };
+  // one tile: its sums, and its candidates while the CTA is still listing
+  auto do_tile = [&](int tl, const float4 (&x)[kU]) {
+    const uint32_t local0 = (uint32_t)(tl * kEwTile + tid * 4);
+    const uint32_t blk0 = (uint32_t)(beg >> 2) + (uint32_t)(tl * (kEwTile / 4) + tid);
+    float fsum = 0.0f;                                     // short fp32 run (16 terms), then into fp64: as in ew_chunk_pass
+    if (tl == 0) {                                         // the estimate: this tile's sum, scaled to the vector
+      ew_cand_tile<false>(x, local0, blk0, 0, v.layer, key, kind_step, false, fsum, amax, C);
+      const float ws = warp_sum(fsum);
+      if (lane == 0) s_red[w] = ws;
+      __syncthreads();
+      float ts = 0.0f;
+      for (int i2 = 0; i2 < kEwThreads / kWarp; ++i2) ts += s_red[i2];
+      const double in_tile = (double)min((int64_t)kEwTile, end - beg);
+      // M = 1.25 (s / l1_est) 2^32 with l1_est = ts n / in_tile.  A zero or non-finite ts gives inf or NaN: the threads'
+      // lists overflow or stay empty and the check after the barrier sends the chunk the other way.  No list either
+      // where a thread would expect more than a quarter of its slots to fill (budgets above about 1.5 % of the length:
+      // the list would cost more than the second read)
+      float m32 = (float)(1.25 * s * in_tile * 4294967296.0 / ((double)ts * (double)v.n));
+      const double expect = 1.25 * s * (double)(end - beg) / ((double)v.n * kEwThreads);
+      if (!(m32 > 0.0f) || expect > 0.25 * kEwCandPerThread) m32 = 0.0f;
+      C.m32 = m32;
+      float f2 = 0.0f, u2 = 0.0f;                          // the tile again, for its candidates (sums discarded)
+      if (m32 != 0.0f) ew_cand_tile<false>(x, local0, blk0, end - beg - (int64_t)local0, v.layer, key, kind_step, true, f2, u2, C);
+    } else {
+      const bool listing = C.m32 != 0.0f && *(volatile uint32_t*)C.stop == 0u;
+      if (tl < n_full) ew_cand_tile<true>(x, local0, blk0, 0, v.layer, key, kind_step, listing, fsum, amax, C);
+      else ew_cand_tile<false>(x, local0, blk0, end - beg - (int64_t)local0, v.layer, key, kind_step, listing, fsum, amax, C);
+    }
+    sum += (double)fsum;
+  };
+  float4 x[kU], xn[kU];
+  load_tile(0, x);
+  for (int tl = 0; tl < n_my; ++tl) {
+    if (tl + 1 < n_my) load_tile(tl + 1, xn);
+    do_tile(tl, x);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) x[u] = xn[u];
+  }
+  EwAcc acc;
+  acc.sum = sum; acc.cnt = 0u; acc.amax = amax;
+  acc.bad = (!(sum == sum) || !(amax <= 3.402823466e38f)) ? 1u : 0u;   // an entry is NaN or infinite
+  return acc;
+}
+
 // what the probability solve leaves for the sampling pass (every CTA computes the same values)
 struct EwSolved { double T0; float scale, theta, c; uint32_t n_sat, rounds; bool nonfinite; };
 
 // The solve over this CTA's elements [beg, end) (a multiple of 4 from the start of the vector); all CTAs of the grid
-// call it together (cooperative launch).
-__device__ __forceinline__ EwSolved ew_solve_body(const EwVec& v, const double s, const int64_t beg, const int64_t end) {
+// call it together (cooperative launch).  `first`: the sums of the first pass, if the caller has made it already.
+__device__ __forceinline__ EwSolved ew_solve_body(const EwVec& v, const double s, const int64_t beg, const int64_t end,
+                                                  const EwAcc* first = nullptr) {
   cg::grid_group grid = cg::this_grid();
   __shared__ double s_sum[kEwThreads / kWarp];
   __shared__ float s_max[kEwThreads / kWarp];
   __shared__ uint32_t s_cnt[kEwThreads / kWarp], s_bad[kEwThreads / kWarp];
   const int nb = gridDim.x;
   // ---- pass 1: ||g||_1, ||g||_inf, non-finite scan ----
-  EwAcc mine = ew_block_reduce(ew_chunk_pass<false>(v, 0.0f, beg, end), s_sum, s_max, s_cnt, s_bad);
+  EwAcc mine = ew_block_reduce(first != nullptr ? *first : ew_chunk_pass<false>(v, 0.0f, beg, end), s_sum, s_max, s_cnt, s_bad);
   if (threadIdx.x == 0) v.partials[blockIdx.x] = EwPartial{mine.sum, mine.amax, mine.cnt, mine.bad};
   grid.sync();
   EwAcc tot{0.0, 0.0f, 0u, 0u};
@@ -281,7 +426,8 @@ __device__ __forceinline__ void ew_keep_bits(const EwVec& v, const PhiloxKey key
 // saturated count in bits 32..62 beside the total, and the kernel keeps a second bit mask (saturated and kept).
 template <bool COMPACT>
 __device__ __forceinline__ void ew_sample_pack_chunk(const EwVec& v, const PhiloxKey key, const uint32_t kind_step,
-                                                     const uint32_t chunk, const EwSolved& S, uint32_t* s_mask
+                                                     const uint32_t chunk, const EwSolved& S, uint32_t* s_mask,
+                                                     const EwCands* cands = nullptr
 #ifdef EW_PROFILE
                                                      , unsigned long long* ew_t = nullptr
 #endif
@@ -303,9 +449,42 @@ __device__ __forceinline__ void ew_sample_pack_chunk(const EwVec& v, const Philo
   __syncthreads();
   const int64_t tile0 = (int64_t)chunk * q + min((int64_t)chunk, rem);
   const int n_my = (int)(q + ((int64_t)chunk < rem ? 1 : 0));
-  uint32_t* s_sat = s_mask + (size_t)(q + (rem ? 1 : 0)) * kEwWordsPerTile;   // COMPACT only
+  uint32_t* s_sat = s_mask + (size_t)(q + (rem ? 1 : 0)) * kEwWordsPerTile;   // COMPACT: saturated masks; one-kernel form deciding on its list: the kept atoms' sign bits
 
   // ---- phase 1 ----
+  // the candidate list of the first pass holds every kept atom of the chunk if it was made with a multiplier that
+  // covers the true scale, did not overflow and no atom has p = 1
+  bool from_list = cands != nullptr && cands->m32 > 0.0f && S.n_sat == 0 && !dead && scale > 0.0f &&
+                   cands->m32 >= scale * 4294967296.0f * (1.0f + 2.384185791015625e-07f);
+  if (cands != nullptr) from_list = __syncthreads_or(ew_cand_count(*cands) > (uint32_t)kEwCandPerThread ? 1 : 0) == 0 && from_list;
+  if (from_list) {
+    const float scale32 = scale * 4294967296.0f;
+    const int n_w = n_my * kEwWordsPerTile;
+    for (int wi = tid; wi < n_w; wi += kEwThreads) { s_mask[wi] = 0u; s_sat[wi] = 0u; }
+    __syncthreads();
+    const uint32_t n_c = ew_cand_count(*cands);
+    const uint32_t blk_beg = (uint32_t)(tile0 * (kEwTile / 4));
+    for (uint32_t e = 0; e < n_c; ++e) {                   // this thread's own entries; their words are drawn again
+      const uint32_t li = cands->idx[e * kEwThreads + tid];
+      const uint4 wd = philox4x32_10(make_uint4(blk_beg + (li >> 2), 0u, v.layer, kind_step), key);
+      const uint32_t j = li & 3u;
+      const uint32_t word = j == 0 ? wd.x : j == 1 ? wd.y : j == 2 ? wd.z : wd.w;
+      const uint32_t gbits = cands->idx[kEwCandSlots + e * kEwThreads + tid];
+      const float t = fabsf(__uint_as_float(gbits)) * scale32;           // the same product and comparison as ew_tile_bits
+      if (t >= 4294967296.0f || word < __float2uint_rz(t)) {
+        atomicOr(&s_mask[li >> 5], 1u << (li & 31u));
+        if (gbits >> 31) atomicOr(&s_sat[li >> 5], 1u << (li & 31u));    // the value of a kept atom is sign(g) c: its sign is all that phase 2 needs
+        atomicAdd(&s_tcnt[li / kEwTile], 1u);
+      }
+    }
+    if (v.n_words > 0) {
+      __syncthreads();
+      for (int wi = tid; wi < n_w; wi += kEwThreads) {
+        const int64_t widx = tile0 * kEwWordsPerTile + wi;
+        if (widx < v.n_words) v.mask_words[widx] = s_mask[wi];
+      }
+    }
+  } else
   if (any_sat) ew_keep_bits<true, true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
   else if (S.n_sat != 0) ew_keep_bits<false, true>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
   else ew_keep_bits<false, false>(v, key, kind_step, tile0, n_my, scale, theta, dead, aligned, s_mask, s_sat, s_tcnt, s_tsat);
@@ -409,12 +588,13 @@ __device__ __forceinline__ void ew_sample_pack_chunk(const EwVec& v, const Philo
       const int bpos = __ffs(m) - 1;
       m &= m - 1;
       const uint32_t o = off0 + (uint32_t)bpos;
-      const float g = __ldg(v.g + tile_base + o);
+      // from the list: no atom has p = 1, so only the sign is needed, and the list left it in the second mask
+      const float g = from_list ? (((s_sat[wi] >> bpos) & 1u) ? -1.0f : 1.0f) : __ldg(v.g + tile_base + o);
       if (!COMPACT) {
         if (pos < (uint64_t)v.k_cap) {
           // kept atom: saturated (p = 1) keeps g; otherwise g / p = sign(g) T / (s - n_s)
           v.idx[pos] = (uint32_t)(tile_base + o);
-          v.val[pos] = (fabsf(g) > theta) ? g : copysignf(c, g);
+          v.val[pos] = (!from_list && fabsf(g) > theta) ? g : copysignf(c, g);
         }
         ++pos;
       } else if ((sword >> bpos) & 1u) {
@@ -445,9 +625,12 @@ __global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_sample_pack_kerne
 }
 
 // The one-kernel form (cooperative launch, every chunk resident): a CTA solves over its own chunk of tiles and then
-// samples and packs the same chunk, which it finds in the L2 on its own side of the chip.
-template <bool COMPACT>
-__global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step) {
+// samples and packs the same chunk: from the candidate list of its first pass where that holds every kept atom,
+// else from a second read of the chunk, which it finds in the L2 on its own side of the chip.
+// LIST: the form with the candidate list (64 registers, four CTAs per SM); without it the kernel is compiled for five.
+template <bool COMPACT, bool LIST>
+__global__ void __launch_bounds__(kEwThreads, LIST ? kEwEncodeBlocks : kEwMinBlocks)
+ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step) {
   extern __shared__ uint32_t s_mask[];
   const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;
   const int64_t chunk = blockIdx.x;
@@ -457,17 +640,35 @@ __global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_encode_kernel(EwV
   unsigned long long ew_t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
 #endif
   EW_STAMP(0)
-  const EwSolved S = ew_solve_body(v, s, tile0 * kEwTile, min(v.n, (tile0 + n_my) * kEwTile));
-  EW_STAMP(1)
+  const int64_t beg = tile0 * kEwTile, end = min(v.n, (tile0 + n_my) * kEwTile);
+  if constexpr (LIST) {
+    __shared__ uint32_t s_cand[2 * kEwCandSlots], s_cstop;   // indices, then values
+    __shared__ float s_red[kEwThreads / kWarp];
+    const uint32_t cand0 = (uint32_t)__cvta_generic_to_shared(s_cand) + 4u * threadIdx.x;
+    EwCands cands{s_cand, &s_cstop, 0.0f, cand0, cand0};
+    const bool with_list = v.prob_out == nullptr;
+    EwAcc first;
+    if (with_list) {
+      if (threadIdx.x == 0) s_cstop = 0u;                    // ordered before its first use by the barrier inside the first tile
+      first = ew_chunk_pass_cand(v, key, kind_step, s, beg, end, (int)n_my, cands, s_red);
+      EW_STAMP(6)
+    }
+    const EwSolved S = ew_solve_body(v, s, beg, end, with_list ? &first : nullptr);
+    EW_STAMP(1)
 #ifdef EW_PROFILE
-  ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask, ew_t);
-  EW_STAMP(5)
-  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
-    printf("cta %d tiles %d: solve %llu ns, keep bits %llu, publish+wait %llu, scan+pack %llu, total %llu\n", (int)blockIdx.x, (int)n_my,
-           ew_t[1] - ew_t[0], ew_t[2] - ew_t[1], ew_t[3] - ew_t[2], ew_t[5] - ew_t[3], ew_t[5] - ew_t[0]);
+    ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask, &cands, ew_t);
+    EW_STAMP(5)
+    if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x / 2 || blockIdx.x == gridDim.x - 1))
+      printf("cta %d tiles %d: first pass with list %llu ns (%u candidates in thread 0), solve %llu, keep bits %llu, publish+wait %llu, scan+pack %llu, total %llu\n",
+             (int)blockIdx.x, (int)n_my, ew_t[6] ? ew_t[6] - ew_t[0] : 0ull, ew_cand_count(cands), ew_t[1] - ew_t[0], ew_t[2] - ew_t[1], ew_t[3] - ew_t[2],
+             ew_t[5] - ew_t[3], ew_t[5] - ew_t[0]);
 #else
-  ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask);
+    ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask, &cands);
 #endif
+  } else {
+    const EwSolved S = ew_solve_body(v, s, beg, end);
+    ew_sample_pack_chunk<COMPACT>(v, key, kind_step, (uint32_t)chunk, S, s_mask);
+  }
 }
 
 // ---- decode -------------------------------------------------------------------------------------
@@ -582,11 +783,10 @@ int launch_ew_solve(const EwVec& v, double s, cudaStream_t st) {
 }
 namespace {
 // co-resident CTAs of a sample / pack style kernel with its largest chunk in shared memory
-template <typename K> int64_t ew_wave(K kernel, bool compact) {
+template <typename K> int64_t ew_wave(K kernel, int dyn_tiles) {
   int dev = 0, sms = 148, per_sm = 4;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kEwThreads,
-                                                                      (compact ? 32 : 16) * kEwWordsPerTile * sizeof(uint32_t));
+  const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kEwThreads, (size_t)dyn_tiles * kEwWordsPerTile * sizeof(uint32_t));
   if (e != cudaSuccess || per_sm < 1) { cudaGetLastError(); per_sm = 4; }
   return (int64_t)sms * per_sm;
 }
@@ -594,21 +794,45 @@ template <typename K> int64_t ew_wave(K kernel, bool compact) {
 
 int ew_sample_pack_ctas(int64_t n_tiles, bool compact) {
   // one wave of chunks when it fits (at most 64 tiles per chunk, 32 for the compact format): tiles spread evenly, sizes differ by at most one
-  const int64_t wave = compact ? ew_wave(ew_sample_pack_kernel<true>, true) : ew_wave(ew_sample_pack_kernel<false>, false);
+  const int64_t wave = compact ? ew_wave(ew_sample_pack_kernel<true>, 32) : ew_wave(ew_sample_pack_kernel<false>, 16);
   const int max_tiles = compact ? kEwMaxTilesPerCta / 2 : kEwMaxTilesPerCta;   // compact: two masks per tile in shared memory
   const int64_t min_ctas = (n_tiles + max_tiles - 1) / max_tiles;
   return (int)std::max<int64_t>(1, std::max(min_ctas, std::min(n_tiles, wave)));
 }
-// CTAs of the one-kernel form, or 0 if the vector does not fit one wave of resident chunks
-int ew_encode_ctas(int64_t n_tiles, bool compact) {
-  static int64_t waves[2] = {0, 0};
-  if (waves[compact] == 0) waves[compact] = compact ? ew_wave(ew_encode_kernel<true>, true) : ew_wave(ew_encode_kernel<false>, false);
+namespace {
+const void* ew_encode_fn(bool compact, bool list) {
+  if (list) return compact ? (const void*)ew_encode_kernel<true, true> : (const void*)ew_encode_kernel<false, true>;
+  return compact ? (const void*)ew_encode_kernel<true, false> : (const void*)ew_encode_kernel<false, false>;
+}
+}  // namespace
+// CTAs of the one-kernel form, or 0 if the vector does not fit one wave of resident chunks.  `list`: the form that
+// keeps a candidate list during its first pass.
+int ew_encode_ctas(int64_t n_tiles, bool compact, bool list) {
+  static int64_t waves[2][2] = {{0, 0}, {0, 0}};
+  // chunks of at most 12 tiles with the list: with the two masks (12 KB) and the list a CTA stays below 48 KB, so that
+  // four CTAs per SM fit the 196 KB carve-out a cooperative launch is checked against; 16 without (8 or 16 KB of masks)
+  const int64_t fit_tiles = list ? 12 : 16;
+  if (waves[compact][list] == 0) {
+    int dev = 0, sms = 148, per_sm = 4;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const size_t dyn = (size_t)fit_tiles * kEwWordsPerTile * sizeof(uint32_t) * ((compact || list) ? 2 : 1);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ew_encode_fn(compact, list), kEwThreads, dyn) != cudaSuccess || per_sm < 1) {
+      cudaGetLastError(); per_sm = 4;
+    }
+    waves[compact][list] = (int64_t)sms * per_sm;
+  }
   const int max_tiles = compact ? kEwMaxTilesPerCta / 2 : kEwMaxTilesPerCta;
-  // chunks of at most 16 tiles keep the shared memory the occupancy figure was asked for
-  const int64_t fit_tiles = 16;
-  const int64_t ctas = std::min(n_tiles, waves[compact]);
+  const int64_t ctas = std::min(n_tiles, waves[compact][list]);
   if (ctas < 1 || (n_tiles + ctas - 1) / ctas > std::min<int64_t>(max_tiles, fit_tiles)) return 0;
   return (int)ctas;
+}
+// Whether the list pays for a vector of n elements in `ctas` chunks at budget s: a thread expects 1.25 s (its atoms) / n
+// candidates and has kEwCandPerThread slots; beyond a quarter of them (budgets above about 1.5 % of the length) the
+// appends cost more than the second read saves and overflows become likely.
+bool ew_list_pays(int64_t n, int64_t n_tiles, int ctas, double s) {
+  if (ctas < 1) return false;
+  const double chunk = (double)((n_tiles + ctas - 1) / ctas) * kEwTile;
+  return 1.25 * s * chunk / ((double)n * kEwThreads) <= 0.25 * kEwCandPerThread;
 }
 void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
   const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
@@ -622,11 +846,11 @@ void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cu
 }
 int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
   const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
-  const size_t smem = (size_t)most * kEwWordsPerTile * sizeof(uint32_t) * (v.compact ? 2 : 1);
+  // mask words; a second mask for the saturated atoms (compact format) or the sign bits (list)
+  const size_t smem = (size_t)most * kEwWordsPerTile * sizeof(uint32_t) * ((v.compact || v.candidates) ? 2 : 1);
   EwVec vv = v; double ss = s; PhiloxKey kk = key; uint32_t ks = kind_step;
   void* args[] = {&vv, &ss, &kk, &ks};
-  const void* fn = v.compact ? (const void*)ew_encode_kernel<true> : (const void*)ew_encode_kernel<false>;
-  return (int)cudaLaunchCooperativeKernel(fn, dim3((unsigned)v.n_ctas), dim3(kEwThreads), args, smem, st);
+  return (int)cudaLaunchCooperativeKernel(ew_encode_fn(v.compact != 0, v.candidates != 0), dim3((unsigned)v.n_ctas), dim3(kEwThreads), args, smem, st);
 }
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {
   const int64_t tiles = (d.n + kEwTile - 1) / kEwTile;

@@ -36,6 +36,7 @@ struct EwVec {
   float* prob_out;                                             // debug or nullptr
   // compact payload format (else compact = 0 and the rest unused)
   int compact; uint32_t sat_cap;
+  int candidates;                                              // one-kernel form: keep a candidate list during the first pass (else read the chunk twice)
   uint16_t* ent;                                               // [k_cap] tile-local index | sign << 15 of kept atoms with p < 1
   uint32_t* sat_idx; float* sat_val;                           // [sat_cap] atoms with p = 1
 };
@@ -53,7 +54,8 @@ int ew_tile_elems();
 void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax, double* part_sum, float* part_max,
                   int n_ctas, cudaStream_t st);
 int ew_sample_pack_ctas(int64_t n_tiles, bool compact);
-int ew_encode_ctas(int64_t n_tiles, bool compact);             // CTAs of the one-kernel form; 0 = the vector needs the two-kernel form
+int ew_encode_ctas(int64_t n_tiles, bool compact, bool list);  // CTAs of the one-kernel form (with or without the candidate list); 0 = the vector needs the two-kernel form
+bool ew_list_pays(int64_t n, int64_t n_tiles, int ctas, double s);   // whether the candidate list is worth keeping at this budget
 int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st);   // cudaError_t
 
 // ================================= spectral path =================================================

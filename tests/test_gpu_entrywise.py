@@ -45,6 +45,16 @@ def _run(atomo, oracle, vecs, s, seed, step=0, k_cap=None, offset=0):
             ref = oracle.decode_entrywise(g.size, enc["idx"], enc["val"])
             assert parity.rel(out, ref) <= parity.REL_TOL if enc["idx"].size else not out.any()
     print("\n".join(report))
+    # Without the probabilities asked for, the one-kernel form takes the keep decisions on the candidate list of its
+    # first pass wherever that list is complete: the same masks and payload arrays have to come out.
+    pay2, dbg2 = atomo.atomo_encode_entrywise(ts, s, seed, step=step, k_cap=k_cap, debug="mask")
+    hdrs2 = pay2.headers()
+    assert torch.equal(dbg2.mask_words, dbg.mask_words), "mask words differ when the probabilities are not asked for"
+    for l in range(len(vecs)):
+        h, h2 = hdrs[1][l], hdrs2[1][l]
+        assert (h.status, h.k, h.n_sat, h.c, h.l1) == (h2.status, h2.k, h2.n_sat, h2.c, h2.l1)
+        a, a2 = pay.layer_arrays(l, hdrs), pay2.layer_arrays(l, hdrs2)
+        assert np.array_equal(a["idx"], a2["idx"]) and np.array_equal(a["val"], a2["val"])
     return pay, hdrs
 
 
@@ -193,40 +203,52 @@ def test_launch_forms_agree(atomo, compact):
     different number of CTAs: mask words, kept indices, values and decoded gradients have to be identical all the
     same.  (sum |g| is added up in short fp32 runs and then chunk by chunk in fp64, so it depends on the cut at the
     1e-8 level: it is compared to 1e-7.  The weight c = T / (s - n_s) and the scale of the probabilities are its
-    fp32 roundings; where they come out equal -- they do for these inputs -- everything else has to be identical.)"""
+    fp32 roundings; where they come out equal -- they do for these inputs -- everything else has to be identical.)
+    The one-kernel form is run three ways: deciding on the candidate list of its first pass (the default), without the
+    list (launch form 2), and with the probabilities asked for, which switches the list off as well."""
     import torch
     from paper_1806_04090_b200 import api
     rng = np.random.default_rng(77)
     big = rng.laplace(0.0, 1e-3, 3_000_017).astype(np.float32)
     spiky = rng.laplace(0.0, 1e-3, 700_001).astype(np.float32)
     spiky[rng.choice(spiky.size, 300, replace=False)] *= 1.0e4          # not s-balanced: saturated atoms
-    cases = [([big], 0.01 * big.size), ([spiky], 5000.0), ([big[:4097], spiky[:123], big[:40960]], 64.0)]
+    # inputs on which a chunk's own estimate of sum |g| is wrong in either direction, so that some chunks of the
+    # one-kernel form decide on their candidate list and others read their part a second time: half the vector zero,
+    # a scale that grows a hundredfold along the vector, and zero first tiles followed by data
+    half = big.copy(); half[: half.size // 2] = 0.0
+    ramp = (big * np.linspace(0.05, 5.0, big.size, dtype=np.float32)).astype(np.float32)
+    holes = big.copy(); holes.reshape(-1)[: (holes.size // 8192) * 8192].reshape(-1, 8192)[:, :4096] = 0.0
+    cases = [([big], 0.01 * big.size), ([spiky], 5000.0), ([big[:4097], spiky[:123], big[:40960]], 64.0),
+             ([half], 0.01 * big.size), ([ramp], 0.01 * big.size), ([holes], 0.002 * big.size), ([big], 0.04 * big.size)]
     try:
         for vecs, s in cases:
             ts = [torch.from_numpy(g).cuda() for g in vecs]
             k_cap = int(1.2 * s) + 2000
             got = []
-            for two in (False, True):
-                atomo.set_entrywise_launch(two)
+            # (launch form, debug outputs): the one-kernel form with the candidate list first (asking for the
+            # probabilities switches the list off), then the two-kernel form and the one-kernel form without the list
+            for form, debug in ((0, "mask"), (1, True), (2, True), (0, True)):
+                atomo.set_entrywise_launch(form)
                 atomo.set_entrywise_format(api.EW_COMPACT if compact else api.EW_EXPLICIT, 1000 if compact else 0)
-                pay, dbg = atomo.atomo_encode_entrywise(ts, s, seed=5, step=3, k_cap=k_cap, debug=True)
+                pay, dbg = atomo.atomo_encode_entrywise(ts, s, seed=5, step=3, k_cap=k_cap, debug=debug)
                 outs = atomo.atomo_decode(pay)
                 torch.cuda.synchronize()
                 hdrs = pay.headers()
                 assert max(h.status for h in hdrs[1]) == 0
                 got.append((hdrs[1], [pay.layer_arrays(l, hdrs) for l in range(len(vecs))], dbg.mask_words.clone(),
                             [o.clone() for o in outs]))
-            for l in range(len(vecs)):
-                h0, h1 = got[0][0][l], got[1][0][l]
-                assert abs(h0.l1 - h1.l1) <= 1e-7 * abs(h0.l1)
-                assert h0.c == h1.c, "the fp32 weight differs between the launch forms: choose other test inputs"
-            assert torch.equal(got[0][2], got[1][2]), "mask words differ between the launch forms"
-            for l in range(len(vecs)):
-                h0, h1 = got[0][0][l], got[1][0][l]
-                assert (h0.k, h0.n_sat, h0.sweeps) == (h1.k, h1.n_sat, h1.sweeps)
-                a0, a1 = got[0][1][l], got[1][1][l]
-                assert np.array_equal(a0["idx"], a1["idx"]) and np.array_equal(a0["val"], a1["val"])
-                assert torch.equal(got[0][3][l], got[1][3][l])
+            for other in got[1:]:
+                for l in range(len(vecs)):
+                    h0, h1 = got[0][0][l], other[0][l]
+                    assert abs(h0.l1 - h1.l1) <= 1e-7 * abs(h0.l1)
+                    assert h0.c == h1.c, "the fp32 weight differs between the launch forms: choose other test inputs"
+                assert torch.equal(got[0][2], other[2]), "mask words differ between the launch forms"
+                for l in range(len(vecs)):
+                    h0, h1 = got[0][0][l], other[0][l]
+                    assert (h0.k, h0.n_sat, h0.sweeps) == (h1.k, h1.n_sat, h1.sweeps)
+                    a0, a1 = got[0][1][l], other[1][l]
+                    assert np.array_equal(a0["idx"], a1["idx"]) and np.array_equal(a0["val"], a1["val"])
+                    assert torch.equal(got[0][3][l], other[3][l])
     finally:
         atomo.set_entrywise_launch(False)
         atomo.set_entrywise_format(api.EW_EXPLICIT, 0)
