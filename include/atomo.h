@@ -182,7 +182,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs /*HOST array*/,
  * gets ATOMO_ERR_CAPACITY in its status word and k = 0.  Decoders read the format from the payload.       */
 int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap);
 /* Launch form of the context's later atomo_encode_entrywise calls.  two_kernels = 0 (default): a vector whose tiles
- * fit one wave of resident CTAs (up to about 48 million elements on a B200) is encoded by ONE cooperative kernel -- a CTA
+ * fit one wave of resident CTAs (up to about 48 million elements on a B200, 29 million with the list below) is encoded by ONE cooperative kernel -- a CTA
  * computes its part of sum |g| and max |g| (Algorithm 1's inputs), all CTAs meet at a grid barrier, and the same CTA
  * then samples and packs its part.  The Philox word of an atom depends on its index alone, so the first pass already
  * draws the words and lists the atoms that an estimate of sum |g| (with a factor of two to spare) cannot rule out; where
