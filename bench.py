@@ -528,7 +528,9 @@ def run_ours(args):
     ms_per_step = float(np.median(reps_ms))
     value = world * elems / (ms_per_step * 1e-3)
     scheme = a.last_eig_scheme() if run.spectral else None
-    launches = (sum(tot_ln.values()) / stage_steps + 1) * args.steps   # the stages' kernels + the header kernel, per run of K steps
+    # the stages' kernels + the header kernel, per run of K steps (an entry-wise call with one vector writes its headers
+    # inside the encode kernel: no header kernel)
+    launches = (sum(tot_ln.values()) / stage_steps + (1 if run.spectral else 0)) * args.steps
 
     # ---- end to end: host buffers, copies inside the timed region ----
     # Every step's inputs come from pinned host memory and its decoded gradients go back to pinned host memory.

@@ -985,10 +985,17 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     const size_t tb = tmpl.size() * sizeof(atomo_layer_header);
     { const int rc = table_reserve(ctx, ctx->tab_ew, tb); if (rc != ATOMO_OK) return rc; }
     { const int rc = table_commit(ctx, ctx->tab_ew, reinterpret_cast<const uint8_t*>(tmpl.data()), tb, st); if (rc != ATOMO_OK) return rc; }
-    // ... and the look-back status words and tickets of the sample / pack kernels start at zero
+  }
+  // ... and the look-back status words and tickets of the sample / pack kernels start at zero.  A call with one vector
+  // in the one-kernel form does all of this inside that kernel: one launch less.
+  auto begin = [&]() {
     launch_sp_begin(pay, gh, reinterpret_cast<const atomo_layer_header*>(ctx->tab_ew.d), n_vecs, nullptr,
                     reinterpret_cast<uint32_t*>(ew_zero_beg), (int64_t)((ew_zero_bytes + 3) / 4), st);
-  }
+  };
+  const bool begin_inside = n_vecs == 1 && fused[0];
+  EwBegin eb{};
+  eb.pay = pay; eb.tmpl = reinterpret_cast<const atomo_layer_header*>(ctx->tab_ew.d); eb.gh = gh; eb.on = begin_inside ? 1 : 0;
+  if (!begin_inside) begin();
 
   const PhiloxKey key{(uint32_t)seed, (uint32_t)(seed >> 32)};
   const uint32_t ks = kind_step_word(ATOMO_KIND_ENTRYWISE, step);
@@ -1006,10 +1013,11 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   stage_begin(ctx, ATOMO_STAGE_EW_PACK, st);
   for (int l = 0; l < n_vecs; ++l) {
     if (!fused[l]) { launch_ew_sample_pack(V[l], key, ks, st); continue; }
-    const int e = launch_ew_encode(V[l], s, key, ks, st);
+    const int e = launch_ew_encode(V[l], s, key, ks, eb, st);
     if (e == (int)cudaErrorCooperativeLaunchTooLarge) {
       // fewer CTAs fit the GPU at once than the occupancy query promised: the two-kernel form takes the same chunks
       cudaGetLastError();
+      if (begin_inside) begin();
       const int e2 = launch_ew_solve(V[l], s, st);
       if (e2 != 0) return fail_cuda(ctx, (cudaError_t)e2, "cudaLaunchCooperativeKernel(ew_solve)");
       launch_ew_sample_pack(V[l], key, ks, st);

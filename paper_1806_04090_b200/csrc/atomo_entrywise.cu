@@ -630,8 +630,18 @@ __global__ void __launch_bounds__(kEwThreads, kEwMinBlocks) ew_sample_pack_kerne
 // LIST: the form with the candidate list (64 registers, four CTAs per SM); without it the kernel is compiled for five.
 template <bool COMPACT, bool LIST>
 __global__ void __launch_bounds__(kEwThreads, LIST ? kEwEncodeBlocks : kEwMinBlocks)
-ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step) {
+ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step, EwBegin begin) {
   extern __shared__ uint32_t s_mask[];
+  if (begin.on) {
+    // a call with one vector: the payload header, the layer header and the chunks' status words are set here instead of
+    // by a kernel of their own; the grid barrier after the first pass orders them before their first use
+    if (blockIdx.x == 0) {
+      if (threadIdx.x == 0) *reinterpret_cast<atomo_payload_header*>(begin.pay) = begin.gh;
+      if (threadIdx.x < sizeof(atomo_layer_header) / 16)
+        reinterpret_cast<uint4*>(v.hdr)[threadIdx.x] = reinterpret_cast<const uint4*>(begin.tmpl + v.layer)[threadIdx.x];
+    }
+    if (threadIdx.x == 0) v.tile_status[blockIdx.x] = 0ull;
+  }
   const int64_t q = v.n_tiles / v.n_ctas, rem = v.n_tiles % v.n_ctas;
   const int64_t chunk = blockIdx.x;
   const int64_t tile0 = chunk * q + min(chunk, rem);
@@ -844,12 +854,12 @@ void launch_ew_sample_pack(const EwVec& v, PhiloxKey key, uint32_t kind_step, cu
     ew_sample_pack_kernel<false><<<(unsigned)v.n_ctas, kEwThreads, smem, st>>>(v, key, kind_step);
   }
 }
-int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st) {
+int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, const EwBegin& begin, cudaStream_t st) {
   const int64_t most = (v.n_tiles + v.n_ctas - 1) / v.n_ctas;
   // mask words; a second mask for the saturated atoms (compact format) or the sign bits (list)
   const size_t smem = (size_t)most * kEwWordsPerTile * sizeof(uint32_t) * ((v.compact || v.candidates) ? 2 : 1);
-  EwVec vv = v; double ss = s; PhiloxKey kk = key; uint32_t ks = kind_step;
-  void* args[] = {&vv, &ss, &kk, &ks};
+  EwVec vv = v; double ss = s; PhiloxKey kk = key; uint32_t ks = kind_step; EwBegin bb = begin;
+  void* args[] = {&vv, &ss, &kk, &ks, &bb};
   return (int)cudaLaunchCooperativeKernel(ew_encode_fn(v.compact != 0, v.candidates != 0), dim3((unsigned)v.n_ctas), dim3(kEwThreads), args, smem, st);
 }
 void launch_ew_decode(const EwDecode& d, cudaStream_t st) {

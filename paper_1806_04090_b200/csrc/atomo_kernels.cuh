@@ -56,7 +56,9 @@ void launch_ew_lq(const float* g, int64_t n, int pass, double q, double inv_amax
 int ew_sample_pack_ctas(int64_t n_tiles, bool compact);
 int ew_encode_ctas(int64_t n_tiles, bool compact, bool list);  // CTAs of the one-kernel form (with or without the candidate list); 0 = the vector needs the two-kernel form
 bool ew_list_pays(int64_t n, int64_t n_tiles, int ctas, double s);   // whether the candidate list is worth keeping at this budget
-int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, cudaStream_t st);   // cudaError_t
+// what the header kernel would do for a call with one vector, done by the one-kernel form itself (on = 0: not asked for)
+struct EwBegin { uint8_t* pay; const atomo_layer_header* tmpl; atomo_payload_header gh; int on; };
+int launch_ew_encode(const EwVec& v, double s, PhiloxKey key, uint32_t kind_step, const EwBegin& begin, cudaStream_t st);   // cudaError_t
 
 // ================================= spectral path =================================================
 constexpr int kMaxShort = 4096;       // largest short side (atoms per layer)
