@@ -125,6 +125,53 @@ __device__ __forceinline__ double tb_dot_part(const X* __restrict__ x, const T* 
   return acc;
 }
 
+// sum over the 8 lanes lx = lane % 8 of v[k]: lane lx ends with the total of k = lx
+__device__ __forceinline__ float rs8(float (&v)[8], int lane) {
+  const bool b4 = lane & 4, b2 = lane & 2, b1 = lane & 1;
+  float a[4];
+#pragma unroll
+  for (int m = 0; m < 4; ++m) {
+    const float send = b4 ? v[m] : v[m + 4], keep = b4 ? v[m + 4] : v[m];
+    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  float b[2];
+#pragma unroll
+  for (int m = 0; m < 2; ++m) {
+    const float send = b2 ? a[m] : a[m + 2], keep = b2 ? a[m + 2] : a[m];
+    b[m] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+  }
+  const float send = b1 ? b[0] : b[1], keep = b1 ? b[1] : b[0];
+  return keep + __shfl_xor_sync(0xffffffffu, send, 1);
+}
+// y[row] += v in fixed point: v 2^48 as a 64-bit integer, its upper 40 and lower 24 bits added to two 32-bit words.
+// Integer addition commutes, so the sums of y do not depend on the order in which the warps finish their tiles.  (At
+// most 64 additions per row and step: the lower word cannot overflow; |v| < 2^7, and the matrix has trace 1.)
+__device__ __forceinline__ void t1_add_fix(int32_t* yhi, uint32_t* ylo, int row, float v) {
+  const long long q = __float2ll_rn(v * 281474976710656.0f);
+  atomicAdd(yhi + row, (int32_t)(q >> 24));
+  atomicAdd(ylo + row, (uint32_t)(q & 0xffffffll));
+}
+// sum over the 4 lanes ly = lane / 8 of v[j]: lane ly ends with the total of j = ly
+__device__ __forceinline__ float rs4(float (&v)[4], int lane) {
+  const bool b2 = lane & 16, b1 = lane & 8;
+  float a[2];
+#pragma unroll
+  for (int m = 0; m < 2; ++m) {
+    const float send = b2 ? v[m] : v[m + 2], keep = b2 ? v[m + 2] : v[m];
+    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+  }
+  const float send = b1 ? a[0] : a[1], keep = b1 ? a[1] : a[0];
+  return keep + __shfl_xor_sync(0xffffffffu, send, 8);
+}
+
+// the same for one array of (upper, lower) word pairs
+__device__ __forceinline__ void tb_add_fix(int2* y, int row, float v) {
+  const long long q = __float2ll_rn(v * 281474976710656.0f);
+  atomicAdd(&y[row].x, (int32_t)(q >> 24));
+  atomicAdd(reinterpret_cast<uint32_t*>(&y[row].y), (uint32_t)(q & 0xffffffll));
+}
+__device__ __forceinline__ long long tb_fix_value(int2 v) { return (long long)v.x * 16777216ll + (long long)(uint32_t)v.y; }
+
 struct alignas(16) TbShared {
   double part_a[kTbMaxBlocks];     // per 32-row block: ||x||^2 partial of the current column
   double part_k[kTbMaxBlocks];     // per 32-row block: u^T p partial
@@ -165,6 +212,12 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   constexpr int TRg = sizeof(T) == 4 ? 4 : 2;
   T* const pan_u = s_gemm + 2 * kTbNB * 32 * TRg + 2 * kTbNB * 128;            // [kTbNB][kTbPanRows]
   T* const pan_w = pan_u + kTbNB * kTbPanRows;
+  // fp32 clusters: the product over the lower triangle adds its sums up in fixed point (tb_add_fix): the rows of this
+  // CTA in yloc (the storage of S.y), the columns -- rows of any CTA of the cluster -- in ycol, which the rows' owners
+  // read through distributed shared memory after the step's third barrier
+  constexpr bool kSym = sizeof(T) == 4 && C > 1;
+  int2* const ycol = reinterpret_cast<int2*>(pan_w + kTbNB * kTbPanRows);       // [32 nblk]: whole blocks, a ragged last one included
+  int2* const yloc = reinterpret_cast<int2*>(S.y);                             // [kTbThreads]
   // this thread's row: block (tid / 32) of this CTA = global block (tid / 32) * C + q
   const int gb = w * C + q;
   const int g = gb * 32 + lane;
@@ -180,6 +233,10 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   };
 
   for (int i = tid; i < r4; i += kTbThreads) s_u[i] = (T)0;
+  if (kSym) {
+    for (int i = tid; i < 32 * nblk; i += kTbThreads) ycol[i] = make_int2(0, 0);
+    yloc[tid] = make_int2(0, 0);
+  }
   if (C > 1) cluster.sync();                                                   // every CTA runs: remote stores may start
 
   TB_PROF_DECL
@@ -248,8 +305,102 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     }
     sync_all();
     TB_MARK(1)
-    // ---- y = A0 u over this CTA's live rows (warp w: lane position w of every block) and the panel dots ----
-    {
+    // ---- y = A0 u over this CTA's live rows and the panel dots ----
+    if constexpr (kSym) {
+      // The lower triangle only, in 32 x 32 sub-tiles (I, J), J <= I, I a row block of this CTA: a sub-tile gives its
+      // rows' sums to block I of y and, transposed, its columns' sums to block J (half the bytes of a product over
+      // full rows).  In a sub-tile a lane holds rows 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3; the sums
+      // over the 8 lanes of a row and the 4 lanes of a column are reduce-scatters.  Every sub-tile's sums are rounded
+      // to fixed point on their own and added as integers, so y does not depend on which warp or CTA took the
+      // sub-tile: the same bits for every cluster size.  The CTA's sub-tiles are dealt to its warps in equal runs.
+      const int sly = lane >> 3, slx = lane & 7;
+      const int jb0 = (c + 1) >> 5;                                            // first live block
+      const int lb0 = jb0 > q ? (jb0 - q + C - 1) / C : 0;                     // this CTA's first live row block
+      const int M = n_lblk - lb0;
+      const int c0n = lb0 * C + q - jb0 + 1;                                   // sub-tiles of that block's row (1 .. C)
+      const int N = M > 0 ? C * (M * (M - 1) / 2) + c0n * M : 0;
+      const int per = (N + kTbWarps - 1) / kTbWarps;
+      int k = w * per;
+      const int k_end = min(N, k + per);
+      if (k < k_end) {
+        auto before = [&](int m) { return C * (m * (m - 1) / 2) + c0n * m; }; // sub-tiles in the first m live row blocks
+        const float hb = (float)c0n - 0.5f * (float)C;
+        int m = (int)((sqrtf(hb * hb + 2.0f * (float)C * (float)k) - hb) / (float)C);
+        m = max(0, min(m, M - 1));
+        while (m + 1 < M && before(m + 1) <= k) ++m;
+        while (m > 0 && before(m) > k) --m;
+        int I = (lb0 + m) * C + q, J = jb0 + (k - before(m));
+        for (; k < k_end; ++k) {
+          const int row0 = 32 * I, col0 = 32 * J;
+          const bool diag = I == J;
+          const bool edge = row0 + 32 > r || col0 + 32 > r;                   // the matrix ends inside the sub-tile
+          float4 uj;
+          if (!edge) uj = *reinterpret_cast<const float4*>(s_u + col0 + 4 * slx);
+          else {
+            const int cc = col0 + 4 * slx;
+            uj = make_float4(cc < r ? s_u[cc] : 0.f, cc + 1 < r ? s_u[cc + 1] : 0.f, cc + 2 < r ? s_u[cc + 2] : 0.f, cc + 3 < r ? s_u[cc + 3] : 0.f);
+          }
+          const uint64_t uj01 = pack2(uj.x, uj.y), uj23 = pack2(uj.z, uj.w);
+          float rp[8];
+          uint64_t c01 = pack2(0.f, 0.f), c23 = pack2(0.f, 0.f);
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const int rbase = row0 + 8 * sly + 4 * half;                       // first of this lane's four rows
+            float4 v[4];
+            float ui[4];
+            if (!edge) {
+              const float* src = A + (int64_t)rbase * lda + col0 + 4 * slx;
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) v[kk] = ldcg4(src + (int64_t)kk * lda);
+              const float4 u4 = *reinterpret_cast<const float4*>(s_u + rbase);
+              ui[0] = u4.x; ui[1] = u4.y; ui[2] = u4.z; ui[3] = u4.w;
+            } else {
+              const int cc = col0 + 4 * slx;
+#pragma unroll
+              for (int kk = 0; kk < 4; ++kk) {
+                const int rr = rbase + kk;
+                v[kk] = (rr < r && cc < r) ? ldcg4(A + (int64_t)rr * lda + cc) : make_float4(0.f, 0.f, 0.f, 0.f);   // cc < r: the row's padded length holds the group
+                if (cc + 1 >= r) v[kk].y = 0.f;
+                if (cc + 2 >= r) v[kk].z = 0.f;
+                if (cc + 3 >= r) v[kk].w = 0.f;
+                ui[kk] = rr < r ? s_u[rr] : 0.f;
+              }
+            }
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+              float4 x = v[kk];
+              const int rr = 8 * sly + 4 * half + kk, cc = 4 * slx;           // position inside the sub-tile
+              if (diag) {                                                      // lower triangle only
+                if (cc + 0 > rr) x.x = 0.f;
+                if (cc + 1 > rr) x.y = 0.f;
+                if (cc + 2 > rr) x.z = 0.f;
+                if (cc + 3 > rr) x.w = 0.f;
+              }
+              float s0, s1;
+              unpack2(fma2(pack2(x.z, x.w), uj23, fma2(pack2(x.x, x.y), uj01, pack2(0.f, 0.f))), s0, s1);
+              rp[4 * half + kk] = s0 + s1;
+              if (diag) {                                                      // the diagonal entry counts once (with the rows)
+                if (cc + 0 == rr) x.x = 0.f;
+                if (cc + 1 == rr) x.y = 0.f;
+                if (cc + 2 == rr) x.z = 0.f;
+                if (cc + 3 == rr) x.w = 0.f;
+              }
+              const uint64_t ui2 = pack2(ui[kk], ui[kk]);
+              c01 = fma2(pack2(x.x, x.y), ui2, c01);
+              c23 = fma2(pack2(x.z, x.w), ui2, c23);
+            }
+          }
+          const float rsum = rs8(rp, lane);                                    // lane 8 ly + lx: row 8 ly + lx
+          float cv[4];
+          unpack2(c01, cv[0], cv[1]); unpack2(c23, cv[2], cv[3]);
+          const float csum = rs4(cv, lane);                                    // lane 8 ly + lx: column 4 lx + ly
+          tb_add_fix(yloc, ((I - q) / C) * 32 + lane, rsum);
+          tb_add_fix(ycol, col0 + 4 * slx + sly, csum);
+          if (++J > I) { I += C; J = jb0; }
+        }
+      }
+      TB_MARK(2)
+    } else {
       const int c0 = (c + 1) & ~3;
       using V4 = typename Vec4<T>::type;
       constexpr int RB = sizeof(T) == 4 ? 2 : 1;                               // rows per pass of a warp
@@ -315,6 +466,8 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
         }
       }
       TB_MARK(2)
+    }
+    {
       // Panel dots.  Dot number id belongs to CTA id mod C; eight warps share a dot (32-element blocks dealt in turn)
       // and their partial sums are added in warp order -- the same order whatever C is.  The owner sends the result to
       // every CTA of the cluster.
@@ -344,8 +497,18 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     TB_MARK(3)
     // ---- w = p - (u^T p) u with p = 2 (y - U a - W b) ----
     double p = 0.0;
+    double y_sym = 0.0;
+    if constexpr (kSym) {
+      if (valid) {                                                             // this row's sums: its own CTA's and every CTA's column sums
+        long long tot = tb_fix_value(yloc[tid]);
+        yloc[tid] = make_int2(0, 0);
+#pragma unroll
+        for (int rk = 0; rk < C; ++rk) tot += tb_fix_value(cluster.map_shared_rank(ycol, rk)[g]);
+        y_sym = (double)tot * 3.552713678800501e-15;                            // 2^-48
+      }
+    }
     if (live) {
-      double y = S.y[tid];
+      double y = kSym ? y_sym : S.y[tid];
       if (use_pan) {
         for (int t = 0; t < i; ++t)
           y -= (double)pan_u[t * kTbPanRows + tid] * S.dots[2 * t] + (double)pan_w[t * kTbPanRows + tid] * S.dots[2 * t + 1];
@@ -369,6 +532,9 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     }
     sync_all();
     const double K = tb_ordered_sum(S.part_k, nblk, lane);
+    if (kSym) {                                                                // every owner has read its rows: the column sums start the next step at zero
+      for (int i = tid; i < 32 * nblk; i += kTbThreads) ycol[i] = make_int2(0, 0);
+    }
     if (valid) {
       const T wv = (T)(live ? p - K * u_own : 0.0);
       W[(int64_t)(c - p0) * ldw + g] = wv;
@@ -529,48 +695,9 @@ struct alignas(16) T1Shared {
 // serves at little more than half its streaming rate).  Rows and columns from r on are zero.
 __device__ __forceinline__ float* t1_sub(float* At, int I, int J) { return At + ((size_t)(I * (I + 1) / 2 + J) << 10); }
 
-// sum over the 8 lanes lx = lane % 8 of v[k]: lane lx ends with the total of k = lx
-__device__ __forceinline__ float rs8(float (&v)[8], int lane) {
-  const bool b4 = lane & 4, b2 = lane & 2, b1 = lane & 1;
-  float a[4];
-#pragma unroll
-  for (int m = 0; m < 4; ++m) {
-    const float send = b4 ? v[m] : v[m + 4], keep = b4 ? v[m + 4] : v[m];
-    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-  }
-  float b[2];
-#pragma unroll
-  for (int m = 0; m < 2; ++m) {
-    const float send = b2 ? a[m] : a[m + 2], keep = b2 ? a[m + 2] : a[m];
-    b[m] = keep + __shfl_xor_sync(0xffffffffu, send, 2);
-  }
-  const float send = b1 ? b[0] : b[1], keep = b1 ? b[1] : b[0];
-  return keep + __shfl_xor_sync(0xffffffffu, send, 1);
-}
-// y[row] += v in fixed point: v 2^48 as a 64-bit integer, its upper 40 and lower 24 bits added to two 32-bit words.
-// Integer addition commutes, so the sums of y do not depend on the order in which the warps finish their tiles.  (At
-// most 64 additions per row and step: the lower word cannot overflow; |v| < 2^7, and the matrix has trace 1.)
-__device__ __forceinline__ void t1_add_fix(int32_t* yhi, uint32_t* ylo, int row, float v) {
-  const long long q = __float2ll_rn(v * 281474976710656.0f);
-  atomicAdd(yhi + row, (int32_t)(q >> 24));
-  atomicAdd(ylo + row, (uint32_t)(q & 0xffffffll));
-}
 // 16 bytes from global (L2) to shared memory without passing through registers; waited for with cp.async.wait_group
 __device__ __forceinline__ void t1_cp16(float* dst_smem, const float* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src) : "memory");
-}
-
-// sum over the 4 lanes ly = lane / 8 of v[j]: lane ly ends with the total of j = ly
-__device__ __forceinline__ float rs4(float (&v)[4], int lane) {
-  const bool b2 = lane & 16, b1 = lane & 8;
-  float a[2];
-#pragma unroll
-  for (int m = 0; m < 2; ++m) {
-    const float send = b2 ? v[m] : v[m + 2], keep = b2 ? v[m + 2] : v[m];
-    a[m] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-  }
-  const float send = b1 ? a[0] : a[1], keep = b1 ? a[1] : a[0];
-  return keep + __shfl_xor_sync(0xffffffffu, send, 8);
 }
 
 }  // namespace
@@ -1234,7 +1361,8 @@ namespace {
 template <typename T> size_t tb_smem_bytes(int r_max) {
   constexpr int TR = sizeof(T) == 4 ? 4 : 2;
   const size_t r4 = (size_t)((r_max + 3) & ~3);
-  return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128 + (sizeof(T) == 4 ? 2 * (size_t)kTbNB * kTbPanRows : 0)) * sizeof(T);
+  return sizeof(TbShared) + (r4 + 2 * (size_t)kTbNB * 32 * TR + 2 * (size_t)kTbNB * 128 + (sizeof(T) == 4 ? 2 * (size_t)kTbNB * kTbPanRows : 0)) * sizeof(T) +
+         (sizeof(T) == 4 ? (size_t)((r_max + 31) & ~31) * sizeof(int2) : 0);  // fp32: the column sums of the triangle-only product, whole 32-row blocks
 }
 size_t t1_smem_bytes() {
   return sizeof(T1Shared) + sizeof(float) * ((size_t)kT1MaxR + 2 * (size_t)kT1NB * kT1MaxR + 2 * (size_t)kT1MaxR + (size_t)kT1Warps * 1024);
