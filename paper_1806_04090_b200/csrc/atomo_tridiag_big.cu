@@ -557,10 +557,127 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       const int wr = w >> 3, wc = w & 7;                                       // warp: 8 TR rows x 16 columns
       const int ly = lane >> 2, lx = lane & 3;
       const int n_lrows = n_lblk * 32;
+      // One thread's TR x 4 outputs of the tile of local rows mr0 .. and columns hc0 ..: row operands of reflector t
+      // at ur / wrp + t * rstride (indexed by the row inside the tile), column operands at uc / wcp + t * 128.
+      // fp32: a warp's piece of a tile is one 32-row block by 16 columns.  A piece strictly above the diagonal is not
+      // computed: its mirror image, a piece strictly below the diagonal in another block's rows, writes both (the
+      // update is symmetric and so is A0).  Pieces that meet the diagonal are computed and written as they are.
+      auto update_piece = [&](const int mr0, const int hc0, const T* ur, const T* wrp, const int rstride, const T* uc, const T* wcp) {
+        const int lr0 = wr * (8 * TR) + ly * TR;                               // first local row (in the tile) of this thread
+        const int lc0 = wc * 16 + lx * 4;
+        bool mirror = false;
+        if (sizeof(T) == 4) {
+          const int blk_start = (((mr0 >> 5) + wr) * C + q) * 32;              // this warp's 32-row block
+          const int pc_start = hc0 + 16 * wc;
+          if (pc_start > blk_start + 31) return;                               // above the diagonal: written by its mirror image
+          mirror = pc_start + 15 < blk_start;
+        }
+        T acc[TR][4];
+#pragma unroll
+        for (int x = 0; x < TR; ++x)
+#pragma unroll
+          for (int y = 0; y < 4; ++y) acc[x][y] = 0;
+        for (int t = 0; t < nr; ++t) {
+          T ru[TR], rw[TR];
+          load_rows<T>(ur + t * rstride + lr0, ru);
+          load_rows<T>(wrp + t * rstride + lr0, rw);
+          const typename Vec4<T>::type cu = *reinterpret_cast<const typename Vec4<T>::type*>(uc + t * 128 + lc0);
+          const typename Vec4<T>::type cw = *reinterpret_cast<const typename Vec4<T>::type*>(wcp + t * 128 + lc0);
+#pragma unroll
+          for (int x = 0; x < TR; ++x) {
+            acc[x][0] = fma(ru[x], cw.x, acc[x][0]); acc[x][1] = fma(ru[x], cw.y, acc[x][1]);
+            acc[x][2] = fma(ru[x], cw.z, acc[x][2]); acc[x][3] = fma(ru[x], cw.w, acc[x][3]);
+            acc[x][0] = fma(rw[x], cu.x, acc[x][0]); acc[x][1] = fma(rw[x], cu.y, acc[x][1]);
+            acc[x][2] = fma(rw[x], cu.z, acc[x][2]); acc[x][3] = fma(rw[x], cu.w, acc[x][3]);
+          }
+        }
+        const int h = hc0 + lc0;
+        const int lrf = mr0 + lr0;
+        const int grf = ((lrf >> 5) * C + q) * 32 + (lrf & 31);                // first global row of this thread (its TR rows are consecutive)
+#pragma unroll
+        for (int x = 0; x < TR; ++x) {
+          const int gr = grf + x;
+          const bool on = (lrf >> 5) < n_lblk && gr < r && gr >= g0 && h < r;
+          if (on) {
+            T* dst = A + (int64_t)gr * lda + h;
+            if (h + 3 < r) {
+              typename Vec4<T>::type o = ldcg4(dst);
+              o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
+              st4(dst, o);
+              acc[x][0] = o.x; acc[x][1] = o.y; acc[x][2] = o.z; acc[x][3] = o.w;   // the new entries, for the mirror image
+            } else {
+              for (int y = 0; y < 4 && h + y < r; ++y) { const T o = __ldcg(dst + y) - acc[x][y]; dst[y] = o; acc[x][y] = o; }
+            }
+          }
+        }
+        if (mirror && (lrf >> 5) < n_lblk) {
+          // A0[h + y][grf .. grf + TR - 1] = the new A0[grf .. ][h + y]: rows h + y >= g0 only (the others are dead)
+#pragma unroll
+          for (int y = 0; y < 4; ++y) {
+            const int hr = h + y;
+            if (hr < g0 || hr >= r) continue;
+            T* dst = A + (int64_t)hr * lda + grf;
+            if (TR == 4 && grf >= g0 && grf + 3 < r) {
+              typename Vec4<T>::type o;
+              o.x = acc[0][y]; o.y = acc[1][y]; o.z = acc[TR > 2 ? 2 : 0][y]; o.w = acc[TR > 2 ? 3 : 0][y];
+              st4(dst, o);
+            } else {
+#pragma unroll
+              for (int x = 0; x < TR; ++x) if (grf + x >= g0 && grf + x < r) dst[x] = acc[x][y];
+            }
+          }
+        }
+      };
+      // last global row of the tile of local rows mr0 ..
+      auto tile_end = [&](int mr0) { return ((min(mr0 / 32 + MR / 32, n_lblk) - 1) * C + q) * 32 + 31; };
+      bool done = false;
+      if constexpr (sizeof(T) == 4) {
+        if (use_pan) {
+          // The panel entries of this CTA's rows are in shared memory already (pan_u, pan_w: at most two tiles of rows),
+          // so only the column operands are staged: chunks of 128 columns in two buffers, the next chunk on its way
+          // (cp.async) while this one is used by both row tiles -- one barrier per chunk and no wait for a load.
+          done = true;
+          const int row_end = tile_end(((n_lrows - 1) / MR) * MR);              // this CTA's last row
+          if (row_end >= g0) {
+            float* const s_c = reinterpret_cast<float*>(s_gemm);              // [2][u, w][kTbNB][128]
+            const int hc_first = g0 & ~127, hc_last = min(r - 1, row_end) & ~127;
+            auto fetch = [&](int hc0, int buf) {
+              float* du = s_c + buf * (2 * kTbNB * 128);
+              float* dw = du + kTbNB * 128;
+              for (int e = tid; e < nr * 128; e += kTbThreads) {
+                const int t = e >> 7, h = hc0 + (e & 127);
+                const int hs = h < r ? h : 0, nb = h < r ? 4 : 0;              // beyond the matrix: zero fill
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(du + e)),
+                             "l"(V + (int64_t)(p0 + t) * ldv + hs), "r"(nb) : "memory");
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dw + e)),
+                             "l"(reinterpret_cast<const float*>(W) + (int64_t)t * ldw + hs), "r"(nb) : "memory");
+              }
+              asm volatile("cp.async.commit_group;" ::: "memory");
+            };
+            __syncthreads();                                                   // nobody still reads the buffers' earlier contents
+            fetch(hc_first, 0);
+            int it = 0;
+            for (int hc0 = hc_first; hc0 <= hc_last; hc0 += 128, ++it) {
+              asm volatile("cp.async.wait_group 0;" ::: "memory");
+              __syncthreads();                                                 // this chunk has landed; the other buffer is free
+              if (hc0 + 128 <= hc_last) fetch(hc0 + 128, (it + 1) & 1);
+              const float* du = s_c + (it & 1) * (2 * kTbNB * 128);
+              const float* dw = du + kTbNB * 128;
+              for (int mr0 = 0; mr0 < n_lrows; mr0 += MR) {
+                const int te = tile_end(mr0);
+                if (te < g0 || hc0 > te) continue;                             // a dead tile, or every piece above the diagonal
+                update_piece(mr0, hc0, reinterpret_cast<const T*>(pan_u) + mr0, reinterpret_cast<const T*>(pan_w) + mr0, kTbPanRows,
+                             reinterpret_cast<const T*>(du), reinterpret_cast<const T*>(dw));
+              }
+            }
+          }
+        }
+      }
+      if (!done)
       for (int mr0 = 0; mr0 < n_lrows; mr0 += MR) {
-        // last global row of this tile; dead tiles are skipped
-        const int lb_last = min(mr0 / 32 + MR / 32, n_lblk) - 1;
-        if ((lb_last * C + q) * 32 + 31 < g0) continue;
+        // dead tiles are skipped
+        const int tile_row_end = tile_end(mr0);
+        if (tile_row_end < g0) continue;
         __syncthreads();
         for (int e = tid; e < nr * MR; e += kTbThreads) {
           const int t = e / MR, lr = mr0 + e % MR;
@@ -569,10 +686,6 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
           s_ur[t * MR + e % MR] = in ? (T)__ldcg(V + (int64_t)(p0 + t) * ldv + gr) : (T)0;
           s_wr[t * MR + e % MR] = in ? __ldcg(W + (int64_t)t * ldw + gr) : (T)0;
         }
-        // fp32: a warp's piece of a tile is one 32-row block by 16 columns.  A piece strictly above the diagonal is not
-        // computed: its mirror image, a piece strictly below the diagonal in another block's rows, writes both (the
-        // update is symmetric and so is A0).  Pieces that meet the diagonal are computed and written as they are.
-        const int tile_row_end = (lb_last * C + q) * 32 + 31;
         for (int hc0 = g0 & ~127; hc0 < r; hc0 += 128) {
           if (sizeof(T) == 4 && hc0 > tile_row_end) break;                      // every piece of this and the later chunks lies above the diagonal
           __syncthreads();
@@ -582,70 +695,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
             s_wc[e] = h < r ? __ldcg(W + (int64_t)t * ldw + h) : (T)0;
           }
           __syncthreads();
-          const int lr0 = wr * (8 * TR) + ly * TR;                             // first local row (in the tile) of this thread
-          const int lc0 = wc * 16 + lx * 4;
-          bool mirror = false;
-          if (sizeof(T) == 4) {
-            const int blk_start = (((mr0 >> 5) + wr) * C + q) * 32;            // this warp's 32-row block
-            const int pc_start = hc0 + 16 * wc;
-            if (pc_start > blk_start + 31) continue;                           // above the diagonal: written by its mirror image
-            mirror = pc_start + 15 < blk_start;
-          }
-          T acc[TR][4];
-#pragma unroll
-          for (int x = 0; x < TR; ++x)
-#pragma unroll
-            for (int y = 0; y < 4; ++y) acc[x][y] = 0;
-          for (int t = 0; t < nr; ++t) {
-            T ru[TR], rw[TR];
-            load_rows<T>(s_ur + t * MR + lr0, ru);
-            load_rows<T>(s_wr + t * MR + lr0, rw);
-            const typename Vec4<T>::type cu = *reinterpret_cast<const typename Vec4<T>::type*>(s_uc + t * 128 + lc0);
-            const typename Vec4<T>::type cw = *reinterpret_cast<const typename Vec4<T>::type*>(s_wc + t * 128 + lc0);
-#pragma unroll
-            for (int x = 0; x < TR; ++x) {
-              acc[x][0] = fma(ru[x], cw.x, acc[x][0]); acc[x][1] = fma(ru[x], cw.y, acc[x][1]);
-              acc[x][2] = fma(ru[x], cw.z, acc[x][2]); acc[x][3] = fma(ru[x], cw.w, acc[x][3]);
-              acc[x][0] = fma(rw[x], cu.x, acc[x][0]); acc[x][1] = fma(rw[x], cu.y, acc[x][1]);
-              acc[x][2] = fma(rw[x], cu.z, acc[x][2]); acc[x][3] = fma(rw[x], cu.w, acc[x][3]);
-            }
-          }
-          const int h = hc0 + lc0;
-          const int lrf = mr0 + lr0;
-          const int grf = ((lrf >> 5) * C + q) * 32 + (lrf & 31);              // first global row of this thread (its TR rows are consecutive)
-#pragma unroll
-          for (int x = 0; x < TR; ++x) {
-            const int gr = grf + x;
-            const bool on = (lrf >> 5) < n_lblk && gr < r && gr >= g0 && h < r;
-            if (on) {
-              T* dst = A + (int64_t)gr * lda + h;
-              if (h + 3 < r) {
-                typename Vec4<T>::type o = ldcg4(dst);
-                o.x -= acc[x][0]; o.y -= acc[x][1]; o.z -= acc[x][2]; o.w -= acc[x][3];
-                st4(dst, o);
-                acc[x][0] = o.x; acc[x][1] = o.y; acc[x][2] = o.z; acc[x][3] = o.w;   // the new entries, for the mirror image
-              } else {
-                for (int y = 0; y < 4 && h + y < r; ++y) { const T o = __ldcg(dst + y) - acc[x][y]; dst[y] = o; acc[x][y] = o; }
-              }
-            }
-          }
-          if (mirror && (lrf >> 5) < n_lblk) {
-            // A0[h + y][grf .. grf + TR - 1] = the new A0[grf .. ][h + y]: rows h + y >= g0 only (the others are dead)
-#pragma unroll
-            for (int y = 0; y < 4; ++y) {
-              const int hr = h + y;
-              if (hr < g0 || hr >= r) continue;
-              T* dst = A + (int64_t)hr * lda + grf;
-              if (TR == 4 && grf >= g0 && grf + 3 < r) {
-                typename Vec4<T>::type o;
-                o.x = acc[0][y]; o.y = acc[1][y]; o.z = acc[TR > 2 ? 2 : 0][y]; o.w = acc[TR > 2 ? 3 : 0][y];
-                st4(dst, o);
-              } else {
-#pragma unroll
-                for (int x = 0; x < TR; ++x) if (grf + x >= g0 && grf + x < r) dst[x] = acc[x][y];
-              }
-            }
-          }
+          update_piece(mr0, hc0, s_ur, s_wr, MR, s_uc, s_wc);
         }
       }
     }
