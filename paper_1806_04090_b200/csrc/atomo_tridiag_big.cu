@@ -212,12 +212,11 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   constexpr int TRg = sizeof(T) == 4 ? 4 : 2;
   T* const pan_u = s_gemm + 2 * kTbNB * 32 * TRg + 2 * kTbNB * 128;            // [kTbNB][kTbPanRows]
   T* const pan_w = pan_u + kTbNB * kTbPanRows;
-  // fp32 clusters: the product over the lower triangle adds its sums up in fixed point (tb_add_fix): the rows of this
-  // CTA in yloc (the storage of S.y), the columns -- rows of any CTA of the cluster -- in ycol, which the rows' owners
-  // read through distributed shared memory after the step's third barrier
+  // fp32 clusters: the product over the lower triangle adds its sums up in fixed point (tb_add_fix) in ycol, an array
+  // over all rows of the layer in every CTA, which the rows' owners read through distributed shared memory after the
+  // step's third barrier
   constexpr bool kSym = sizeof(T) == 4 && C > 1;
   int2* const ycol = reinterpret_cast<int2*>(pan_w + kTbNB * kTbPanRows);       // [32 nblk]: whole blocks, a ragged last one included
-  int2* const yloc = reinterpret_cast<int2*>(S.y);                             // [kTbThreads]
   // this thread's row: block (tid / 32) of this CTA = global block (tid / 32) * C + q
   const int gb = w * C + q;
   const int g = gb * 32 + lane;
@@ -235,7 +234,6 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
   for (int i = tid; i < r4; i += kTbThreads) s_u[i] = (T)0;
   if (kSym) {
     for (int i = tid; i < 32 * nblk; i += kTbThreads) ycol[i] = make_int2(0, 0);
-    yloc[tid] = make_int2(0, 0);
   }
   if (C > 1) cluster.sync();                                                   // every CTA runs: remote stores may start
 
@@ -307,29 +305,25 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     TB_MARK(1)
     // ---- y = A0 u over this CTA's live rows and the panel dots ----
     if constexpr (kSym) {
-      // The lower triangle only, in 32 x 32 sub-tiles (I, J), J <= I, I a row block of this CTA: a sub-tile gives its
-      // rows' sums to block I of y and, transposed, its columns' sums to block J (half the bytes of a product over
-      // full rows).  In a sub-tile a lane holds rows 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3; the sums
-      // over the 8 lanes of a row and the 4 lanes of a column are reduce-scatters.  Every sub-tile's sums are rounded
-      // to fixed point on their own and added as integers, so y does not depend on which warp or CTA took the
-      // sub-tile: the same bits for every cluster size.  The CTA's sub-tiles are dealt to its warps in equal runs.
+      // The lower triangle only, in 32 x 32 sub-tiles (I, J), J <= I: a sub-tile gives its rows' sums to block I of y
+      // and, transposed, its columns' sums to block J (half the bytes of a product over full rows).  The layer's live
+      // sub-tiles are dealt in equal runs to all warps of the cluster, whoever owns the rows: every CTA has the same
+      // work, and a row's owner finds the sums in the CTAs' ycol arrays after the barrier.  In a sub-tile a lane holds
+      // rows 8 ly + kk (kk = 0 .. 7) of columns 4 lx .. 4 lx + 3; the sums over the 8 lanes of a row and the 4 lanes
+      // of a column are reduce-scatters.  Every sub-tile's sums are rounded to fixed point on their own and added as
+      // integers, so y does not depend on which warp or CTA took the sub-tile: the same bits for every cluster size.
       const int sly = lane >> 3, slx = lane & 7;
       const int jb0 = (c + 1) >> 5;                                            // first live block
-      const int lb0 = jb0 > q ? (jb0 - q + C - 1) / C : 0;                     // this CTA's first live row block
-      const int M = n_lblk - lb0;
-      const int c0n = lb0 * C + q - jb0 + 1;                                   // sub-tiles of that block's row (1 .. C)
-      const int N = M > 0 ? C * (M * (M - 1) / 2) + c0n * M : 0;
-      const int per = (N + kTbWarps - 1) / kTbWarps;
-      int k = w * per;
+      const int nbl = nblk - jb0;                                              // live blocks
+      const int N = nbl * (nbl + 1) / 2;                                       // live sub-tiles of the layer
+      const int per = (N + C * kTbWarps - 1) / (C * kTbWarps);
+      int k = (q * kTbWarps + w) * per;
       const int k_end = min(N, k + per);
       if (k < k_end) {
-        auto before = [&](int m) { return C * (m * (m - 1) / 2) + c0n * m; }; // sub-tiles in the first m live row blocks
-        const float hb = (float)c0n - 0.5f * (float)C;
-        int m = (int)((sqrtf(hb * hb + 2.0f * (float)C * (float)k) - hb) / (float)C);
-        m = max(0, min(m, M - 1));
-        while (m + 1 < M && before(m + 1) <= k) ++m;
-        while (m > 0 && before(m) > k) --m;
-        int I = (lb0 + m) * C + q, J = jb0 + (k - before(m));
+        int ii = (int)((sqrtf(8.0f * (float)k + 1.0f) - 1.0f) * 0.5f);        // row of the triangle that holds sub-tile k
+        while ((ii + 1) * (ii + 2) / 2 <= k) ++ii;
+        while (ii * (ii + 1) / 2 > k) --ii;
+        int I = jb0 + ii, J = jb0 + (k - ii * (ii + 1) / 2);
         for (; k < k_end; ++k) {
           const int row0 = 32 * I, col0 = 32 * J;
           const bool diag = I == J;
@@ -394,9 +388,9 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
           float cv[4];
           unpack2(c01, cv[0], cv[1]); unpack2(c23, cv[2], cv[3]);
           const float csum = rs4(cv, lane);                                    // lane 8 ly + lx: column 4 lx + ly
-          tb_add_fix(yloc, ((I - q) / C) * 32 + lane, rsum);
+          tb_add_fix(ycol, row0 + lane, rsum);
           tb_add_fix(ycol, col0 + 4 * slx + sly, csum);
-          if (++J > I) { I += C; J = jb0; }
+          if (++J > I) { ++I; J = jb0; }
         }
       }
       TB_MARK(2)
@@ -499,9 +493,8 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     double p = 0.0;
     double y_sym = 0.0;
     if constexpr (kSym) {
-      if (valid) {                                                             // this row's sums: its own CTA's and every CTA's column sums
-        long long tot = tb_fix_value(yloc[tid]);
-        yloc[tid] = make_int2(0, 0);
+      if (valid) {                                                             // this row's sums, from every CTA of the cluster
+        long long tot = 0;
 #pragma unroll
         for (int rk = 0; rk < C; ++rk) tot += tb_fix_value(cluster.map_shared_rank(ycol, rk)[g]);
         y_sym = (double)tot * 3.552713678800501e-15;                            // 2^-48
