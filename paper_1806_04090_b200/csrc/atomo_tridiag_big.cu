@@ -493,7 +493,7 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     double p = 0.0;
     double y_sym = 0.0;
     if constexpr (kSym) {
-      if (valid) {                                                             // this row's sums, from every CTA of the cluster
+      if (live) {                                                              // this row's sums, from every CTA of the cluster (a dead row's are never used)
         long long tot = 0;
 #pragma unroll
         for (int rk = 0; rk < C; ++rk) tot += tb_fix_value(cluster.map_shared_rank(ycol, rk)[g]);
