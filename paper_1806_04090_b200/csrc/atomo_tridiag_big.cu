@@ -180,6 +180,7 @@ struct alignas(16) TbShared {
   double pc[2 * kTbNB];            // u_t[c], w_t[c]: the panel's entries in row c
   double y[kTbThreads];            // A0 u for this CTA's rows (local row order)
   double x0;                       // first entry of the pivot column
+  double p_next;                   // p of the next pivot row (row c + 1), from its owner
 };
 
 }  // namespace
@@ -239,13 +240,18 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
 
   TB_PROF_DECL
   const int n_ref = r - 2;                                                     // reflectors: columns 0 .. r-3
+  double w_carry = 0.0;                                                        // the newest panel column's entry in the next pivot row
   for (int c = 0; c < r; ++c) {
     const int p0 = c / kTbNB * kTbNB;
     const int i = c < n_ref ? c - p0 : 0;                                      // pending reflectors of this panel (the last panel is applied before the last two columns)
     // ---- the panel's entries in row c ----
+    // The newest reflector's two entries were stored by the owner of row c after the last barrier of the step before:
+    // they are not read from memory but formed here -- u from the copy every CTA has, w from the owner's p and K
+    // (w_carry) -- which is what lets a step end without a barrier.  The older ones are a full step old.
     if (tid < 2 * i) {
       const int t = tid >> 1;
-      S.pc[tid] = (tid & 1) ? (double)__ldcg(W + (int64_t)t * ldw + c) : (double)__ldcg(V + (int64_t)(p0 + t) * ldv + c);
+      if (t == i - 1) S.pc[tid] = (tid & 1) ? w_carry : (double)(float)s_u[c];
+      else S.pc[tid] = (tid & 1) ? (double)__ldcg(W + (int64_t)t * ldw + c) : (double)__ldcg(V + (int64_t)(p0 + t) * ldv + c);
     }
     __syncthreads();
     // ---- column c as the earlier reflectors of the panel left it ----
@@ -522,19 +528,21 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
     {
       const double kp = warp_sum(u_own * p);
       if (lane == 0 && gb < nblk) bcast(&S.part_k[gb], kp);
+      if (valid && g == c + 1) bcast(&S.p_next, p);                            // the next pivot row's p, for everybody's w_carry
     }
     sync_all();
     const double K = tb_ordered_sum(S.part_k, nblk, lane);
+    w_carry = (double)(T)fma(-K, (double)s_u[c + 1], S.p_next);               // w[c + 1] exactly as its owner stores it below
     if (kSym) {                                                                // every owner has read its rows: the column sums start the next step at zero
       for (int i = tid; i < 32 * nblk; i += kTbThreads) ycol[i] = make_int2(0, 0);
     }
     if (valid) {
-      const T wv = (T)(live ? p - K * u_own : 0.0);
+      const T wv = (T)(live ? fma(-K, u_own, p) : 0.0);
       W[(int64_t)(c - p0) * ldw + g] = wv;
       if (use_pan) pan_w[(c - p0) * kTbPanRows + tid] = wv;
     }
     const bool flush = (c - p0 == kTbNB - 1) || (c == n_ref - 1);
-    if (!flush) { sync_all(); TB_MARK(4) continue; }
+    if (!flush) { TB_MARK(4) continue; }                                        // no barrier: see the start of the step
     TB_MARK(4)
     // ---- end of the panel: A0 -= U W^T + W U^T on the rows and columns beyond c (this CTA's rows) ----
     if (C == 1) { __threadfence_block(); __syncthreads(); } else { __threadfence(); cluster.sync(); }
