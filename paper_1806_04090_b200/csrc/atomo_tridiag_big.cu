@@ -7,16 +7,17 @@
 //                           the CTAs in blocks of 32 (block b belongs to CTA b mod C).  Within a panel of 32 columns
 //                           the stored matrix A0 is not touched: step c forms column c as it would be after the
 //                           panel's earlier reflectors (A0[:, c] - U W[c]^T - W U[c]^T), the unit reflector u_c
-//                           (H_c = I - 2 u u^T), the product y = A0 u (the one pass over the trailing block: one
-//                           warp per row, the lanes along the row) with the same correction, and
-//                           w = 2 y - (2 u^T y) u.  After the panel the trailing block takes the rank-64 update
-//                           A0 -= U W^T + W U^T (register-tiled, 4 x 4 outputs per thread).  The reflectors go to
-//                           global memory as fp32 unit vectors for the back-transformation.
-//                           Storage type T = float: the matrix and the panel vectors are kept in fp32 and the long
-//                           sums (row products) run in fp32 over at most r / 128 terms per lane before they are
-//                           added in fp64; column updates, norms and all scalars are fp64.  T = double keeps
-//                           everything in fp64.  Every sum has a fixed order that does not depend on C: a row product
-//                           is one warp's, block-wide sums go over the 32-row blocks in ascending order.
+//                           (H_c = I - 2 u u^T), the product y = A0 u (the one pass over the trailing block) with the
+//                           same correction, and w = 2 y - (2 u^T y) u.  After the panel the trailing block takes the
+//                           rank-64 update A0 -= U W^T + W U^T (register-tiled, 4 x 4 outputs per thread).  The
+//                           reflectors go to global memory as fp32 unit vectors for the back-transformation.
+//                           Storage type T = float: the matrix and the panel vectors are kept in fp32; on clusters the
+//                           product goes over the lower triangle in 32 x 32 sub-tiles dealt evenly to all warps of the
+//                           cluster, each sub-tile's row and column sums (fp32 over 32 terms) rounded to fixed point
+//                           and added as integers; with C = 1 and for T = double (everything in fp64) a warp takes
+//                           a row, its lanes along the row.  Column updates, norms and all scalars are fp64.  Every sum has an order that does
+//                           not depend on C: a sub-tile's sums are one warp's and integers add in any order, block-wide
+//                           sums go over the 32-row blocks in ascending order.
 //   sp_eigvec_big_cta_kernel / sp_eigvec_big_kernel (short sides up to 1024 / above)
 //                         : vectors of the kept atoms: twisted factorisation of T - lambda I (the routine of the small
 //                           route, its work vectors in global memory), back-transformation u = Q z four reflectors at
@@ -25,8 +26,8 @@
 //                           atoms).
 //
 // The eigenvalues of T come from sp_bisect_kernel (atomo_tridiag.cu), as for the small layers.
-// Work per layer: the matrix-vector products read sum_c (r - c)^2 ~ r^3 / 3 matrix entries (the bound of this kernel:
-// bytes from L2 / HBM), the panel updates cost 2 r^3 / 3 multiply-adds.
+// Work per layer: the matrix-vector products read sum_c (r - c)^2 / 2 ~ r^3 / 6 matrix entries (one triangle; bytes
+// from L2 / HBM), the panel updates cost 2 r^3 / 3 multiply-adds.
 #include <cstdio>
 
 #include <cooperative_groups.h>
