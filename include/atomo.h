@@ -193,6 +193,11 @@ int atomo_set_entrywise_format(atomo_ctx* ctx, int32_t format, int64_t sat_cap);
  * twice).  Payloads, masks and decoded gradients are bit-identical in all forms.  Other values:
  * ATOMO_ERR_INVALID_ARG.     */
 int atomo_set_entrywise_launch(atomo_ctx* ctx, int32_t two_kernels);
+/* Test introspection, for vector `vec` of the context's last atomo_encode_entrywise call: the number of chunks (CTAs)
+ * of the one-kernel form (0 if the two-kernel form ran) and how many of them took their keep decisions on the
+ * candidate list rather than on a second read.  Synchronises the device.  Either pointer may be NULL.
+ * ATOMO_ERR_INVALID_ARG if there was no such vector.                                                     */
+int atomo_get_entrywise_list_chunks(atomo_ctx* ctx, int32_t vec, uint32_t* from_list /*HOST*/, uint32_t* chunks /*HOST*/);
 
 /* --- l_q budgets (Section 4) ------------------------------------------------------------------
  * s_out[l] (HOST) = ||g_l||_1 / ||g_l||_q for every vector: the budget at which entry-wise ATOMO is the

@@ -34,6 +34,7 @@ EXPORTS = [
     "atomo_payload_bytes_entrywise_compact", "atomo_set_entrywise_format", "atomo_get_stage_totals",
     "atomo_set_tridiag_ctas", "atomo_measure_fma_peak", "atomo_encode_spectral_from_svd", "atomo_get_table_uploads",
     "atomo_set_entrywise_launch",
+    "atomo_get_entrywise_list_chunks",
 ]
 
 
@@ -97,6 +98,7 @@ def load_library(path: str = LIB_PATH) -> ctypes.CDLL:
     lib.atomo_payload_bytes_entrywise_compact.restype = i64
     lib.atomo_set_entrywise_format.argtypes = [vp, i32, i64]
     lib.atomo_set_entrywise_launch.argtypes = [vp, i32]
+    lib.atomo_get_entrywise_list_chunks.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_uint32), ctypes.POINTER(ctypes.c_uint32)]
     lib.atomo_encode_spectral.argtypes = [vp, ctypes.POINTER(_Mat), i32, dbl, u64, u64, i32, vp, i64,
                                           ctypes.POINTER(_Debug), vp]
     lib.atomo_encode_entrywise.argtypes = [vp, ctypes.POINTER(_Vec), i32, dbl, u64, u64, i64, vp, i64,
@@ -549,6 +551,14 @@ class Atomo:
         taken on the candidate list of its first pass where that holds every kept atom; 1 / True: always the solve kernel
         followed by the sample / pack kernel; 2: the one-kernel form without the list.  Same payloads in every form."""
         self._check(self.lib.atomo_set_entrywise_launch(self._h, int(two_kernels)), "atomo_set_entrywise_launch")
+
+    def entrywise_list_chunks(self, vec: int = 0):
+        """(chunks of the last entry-wise encode of vector `vec` that decided on their candidate list, chunks of the
+        one-kernel form: 0 if the two-kernel form ran).  Synchronises."""
+        a, b = ctypes.c_uint32(0), ctypes.c_uint32(0)
+        self._check(self.lib.atomo_get_entrywise_list_chunks(self._h, int(vec), ctypes.byref(a), ctypes.byref(b)),
+                    "atomo_get_entrywise_list_chunks")
+        return int(a.value), int(b.value)
 
     def table_uploads(self):
         """(calls that uploaded their descriptor tables, calls that found them on the device) since the context was made."""

@@ -70,6 +70,8 @@ struct atomo_ctx {
   int eig_scheme_used = -1;          // what the last spectral encode actually ran
   int ew_format = ATOMO_EW_EXPLICIT; // payload format of entry-wise encodes
   int ew_launch = 0;                 // 0: one cooperative kernel per vector where it fits one wave; 1: always solve + sample/pack kernels
+  std::vector<EwState*> ew_last_state;   // per vector of the last entry-wise encode: its state record (device) ...
+  std::vector<int> ew_last_chunks;       // ... and its chunks in the one-kernel form (0: the two-kernel form ran)
   int64_t ew_sat_cap = 0;            // compact format: capacity of the saturated list
   int cluster_capacity[16] = {-1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1, -1};   // by log2(rp_max), -1 = not asked yet
   std::string err;
@@ -1017,6 +1019,7 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
     if (e == (int)cudaErrorCooperativeLaunchTooLarge) {
       // fewer CTAs fit the GPU at once than the occupancy query promised: the two-kernel form takes the same chunks
       cudaGetLastError();
+      fused[l] = 0;
       if (begin_inside) begin();
       const int e2 = launch_ew_solve(V[l], s, st);
       if (e2 != 0) return fail_cuda(ctx, (cudaError_t)e2, "cudaLaunchCooperativeKernel(ew_solve)");
@@ -1029,6 +1032,20 @@ int atomo_encode_entrywise(atomo_ctx* ctx, const atomo_vec* vecs, int32_t n_vecs
   }
   stage_end(ctx, ATOMO_STAGE_EW_PACK, st, (int64_t)(n_two + n_one));
   CK(cudaGetLastError());
+  ctx->ew_last_state.resize(n_vecs); ctx->ew_last_chunks.resize(n_vecs);
+  for (int l = 0; l < n_vecs; ++l) { ctx->ew_last_state[l] = V[l].state; ctx->ew_last_chunks[l] = fused[l] ? V[l].n_ctas : 0; }
+  return ATOMO_OK;
+}
+
+int atomo_get_entrywise_list_chunks(atomo_ctx* ctx, int32_t vec, uint32_t* from_list, uint32_t* chunks) {
+  if (!ctx || vec < 0 || vec >= (int32_t)ctx->ew_last_state.size()) return ATOMO_ERR_INVALID_ARG;
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaDeviceSynchronize());
+  uint32_t n = 0;
+  if (ctx->ew_last_chunks[vec] > 0)
+    CK(cudaMemcpy(&n, &ctx->ew_last_state[vec]->list_chunks, sizeof(n), cudaMemcpyDeviceToHost));
+  if (from_list) *from_list = n;
+  if (chunks) *chunks = (uint32_t)ctx->ew_last_chunks[vec];
   return ATOMO_OK;
 }
 

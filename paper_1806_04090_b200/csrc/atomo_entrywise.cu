@@ -458,6 +458,7 @@ __device__ __forceinline__ void ew_sample_pack_chunk(const EwVec& v, const Philo
                    cands->m32 >= scale * 4294967296.0f * (1.0f + 2.384185791015625e-07f);
   if (cands != nullptr) from_list = __syncthreads_or(ew_cand_count(*cands) > (uint32_t)kEwCandPerThread ? 1 : 0) == 0 && from_list;
   if (from_list) {
+    if (tid == 0) atomicAdd(&v.state->list_chunks, 1u);
     const float scale32 = scale * 4294967296.0f;
     const int n_w = n_my * kEwWordsPerTile;
     for (int wi = tid; wi < n_w; wi += kEwThreads) { s_mask[wi] = 0u; s_sat[wi] = 0u; }
@@ -632,6 +633,7 @@ template <bool COMPACT, bool LIST>
 __global__ void __launch_bounds__(kEwThreads, LIST ? kEwEncodeBlocks : kEwMinBlocks)
 ew_encode_kernel(EwVec v, double s, PhiloxKey key, uint32_t kind_step, EwBegin begin) {
   extern __shared__ uint32_t s_mask[];
+  if (blockIdx.x == 0 && threadIdx.x == 0) v.state->list_chunks = 0u;   // counted after the grid barrier
   if (begin.on) {
     // a call with one vector: the payload header, the layer header and the chunks' status words are set here instead of
     // by a kernel of their own; the grid barrier after the first pass orders them before their first use

@@ -19,6 +19,7 @@ struct EwState {
   float c;          // T / s_cur
   float theta_f, amax;
   uint32_t n_sat, rounds, done, nonfinite;
+  uint32_t list_chunks; // one-kernel form: chunks whose keep decisions were taken on the candidate list (test introspection)
 };
 
 struct EwVec {

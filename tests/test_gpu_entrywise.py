@@ -196,6 +196,44 @@ def test_lq_budget_front_end(atomo, oracle):
         atomo.atomo_lq_budget(ts[:1], 0.5)
 
 
+def test_which_chunks_decide_on_their_list(atomo):
+    """The one-kernel form counts the chunks that took their keep decisions on the candidate list of the first pass:
+    all of them on an s-balanced vector with a small budget; none when the probabilities are asked for, when the
+    vector is not s-balanced or the budget is large (the host then launches the form without the list) or in the
+    two-kernel form; some where a chunk's own estimate of sum |g| is off (half the vector zero: the chunks of the zero
+    half hold no candidate and confirm trivially, the others overestimate sum |g| twofold and read their part again)."""
+    import torch
+    rng = np.random.default_rng(78)
+    big = rng.laplace(0.0, 1e-3, 3_000_017).astype(np.float32)
+    spiky = big.copy(); spiky[rng.choice(spiky.size, 300, replace=False)] *= 1.0e4
+    half = big.copy(); half[: half.size // 2] = 0.0
+    t = lambda g: [torch.from_numpy(g).cuda()]
+    s = 0.01 * big.size
+    try:
+        atomo.atomo_encode_entrywise(t(big), s, seed=5, k_cap=int(1.2 * s) + 2000)
+        got, chunks = atomo.entrywise_list_chunks(0)
+        assert chunks > 100 and got == chunks
+        atomo.atomo_encode_entrywise(t(big), s, seed=5, k_cap=int(1.2 * s) + 2000, debug=True)
+        got_p, chunks_p = atomo.entrywise_list_chunks(0)                  # the form without the list: more, smaller CTAs
+        assert got_p == 0 and chunks_p > 100
+        atomo.atomo_encode_entrywise(t(spiky), 5000.0, seed=5, k_cap=8000)
+        assert atomo.entrywise_list_chunks(0) == (0, chunks)
+        # chunks of two tiles: a thread still expects few candidates at 4 % of the length, far too many at 12 %
+        atomo.atomo_encode_entrywise(t(big), 4.0 * s, seed=5, k_cap=int(4.8 * s) + 2000)
+        assert atomo.entrywise_list_chunks(0) == (chunks, chunks)
+        atomo.atomo_encode_entrywise(t(big), 12.0 * s, seed=5, k_cap=int(14.0 * s) + 2000)
+        got12, chunks12 = atomo.entrywise_list_chunks(0)
+        assert got12 == 0 and chunks12 > 100
+        atomo.atomo_encode_entrywise(t(half), s, seed=5, k_cap=int(1.2 * s) + 2000)
+        got_h, chunks_h = atomo.entrywise_list_chunks(0)
+        assert chunks_h == chunks and 0.3 * chunks < got_h < 0.7 * chunks
+        atomo.set_entrywise_launch(1)
+        atomo.atomo_encode_entrywise(t(big), s, seed=5, k_cap=int(1.2 * s) + 2000)
+        assert atomo.entrywise_list_chunks(0) == (0, 0)
+    finally:
+        atomo.set_entrywise_launch(0)
+
+
 @pytest.mark.parametrize("compact", [False, True])
 def test_launch_forms_agree(atomo, compact):
     """The one-kernel form (solve, grid barrier, sample and pack in one cooperative launch) and the two-kernel form
