@@ -310,11 +310,13 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       if (use_pan) pan_u[(c - p0) * kTbPanRows + tid] = (T)u_own;
       if (g == c + 1) td_e[c] = alpha;
       if (C == 1) s_u[g] = (T)u_own;
-      else if (!form_u) {
+      else if (!kSym) {
 #pragma unroll
         for (int rk = 0; rk < C; ++rk) cluster.map_shared_rank(s_u, rk)[g] = (T)u_own;
       }
     }
+    float* const u_pub = reinterpret_cast<float*>(S.y);                        // fp32 clusters above 2048 rows: the owners' entries of u, fetched after the barrier
+    if (kSym && !form_u) u_pub[tid] = (float)u_own;
     if (form_u) {
       const int h0 = 4 * tid;                                                  // this thread's four entries of the reflector
       if (h0 < r4) {
@@ -335,6 +337,16 @@ __global__ void __launch_bounds__(kTbThreads, 1) sp_tridiag_big_kernel(const SpL
       __syncthreads();
     } else {
       sync_all();
+      if (kSym) {                                                              // one 16-byte remote load per thread instead of a store to every CTA
+        const int h0 = 4 * tid;
+        if (h0 < r4) {
+          const int hb = h0 >> 5;
+          float4 uo = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (hb < nblk && h0 + 3 > c) uo = *reinterpret_cast<const float4*>(cluster.map_shared_rank(u_pub, hb % C) + (hb / C) * 32 + (h0 & 31));
+          *reinterpret_cast<float4*>(s_u + h0) = uo;
+        }
+        __syncthreads();
+      }
     }
     TB_MARK(1)
     // ---- y = A0 u over this CTA's live rows and the panel dots ----
